@@ -1,0 +1,135 @@
+"""TEST INFRASTRUCTURE -- CPU oracle of the region-selective denoising step.
+
+Only ``tests/``, the smoke check and the CPU-baseline leg of the benchmark may import this
+package; the CUDA library never does, and shares no code with it.  Parity status: every
+function here is pinned by the CPU test-suite against closed forms, brute force, invariants
+and independent library routines, except two conventions that nothing outside this build
+fixes ("parity unpinned"): the choice of the root-mean-square as the magnitude of the latent
+change, and the 16-bit width of the saliency quantisation.
+
+* ``partition``      -- Patch Partitioner (paper Sec. 4.1, Appendix A.3)
+* ``activity_gate``  -- Patch Gate (Sec. 4.2, Appendix A.1)
+* ``compact``        -- active set -> ragged token index list (Algorithm 1, PatchGate output)
+* ``regional_step``  -- all blocks on active tokens with stale K/V for skipped patches
+                        (Sec. 3, Sec. 5, Appendix A.6)
+* ``dense_step``     -- the ungated baseline trajectory, written separately
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import Dict, Optional
+
+import numpy as np
+
+from .build import build as _build
+from .gate import activity_gate, compact, initial_state  # noqa: F401
+from .partitioner import partition, partition_request, saliency, quantise, allocate, best_cut  # noqa: F401
+
+_lib = None
+_f = ctypes.POINTER(ctypes.c_float)
+_i = ctypes.POINTER(ctypes.c_int32)
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(_build())
+        _lib.fdo_adaln.restype = ctypes.c_int
+        _lib.fdo_regional_block.restype = ctypes.c_int
+        _lib.fdo_dense_block.restype = ctypes.c_int
+    return _lib
+
+
+def _fp(a: np.ndarray):
+    assert a.dtype == np.float32 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(_f)
+
+
+def _ip(a: Optional[np.ndarray]):
+    if a is None:
+        return None
+    assert a.dtype == np.int32 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(_i)
+
+
+def _c(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def adaln(cond: np.ndarray, w_ada: np.ndarray, b_ada: np.ndarray) -> np.ndarray:
+    """mod [B,6H] = W_ada SiLU(cond) + b_ada for one block."""
+    B, Hc = cond.shape
+    H = w_ada.shape[0] // 6
+    mod = np.empty((B, 6 * H), np.float32)
+    rc = _load().fdo_adaln(B, H, Hc, _fp(_c(cond)), _fp(_c(w_ada)), _fp(_c(b_ada)), _fp(mod))
+    assert rc == 0
+    return mod
+
+
+def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w: Dict[str, np.ndarray],
+                   l: int, kv_l: np.ndarray, heads: int, ln_eps: float = 1e-6,
+                   finish: Optional[np.ndarray] = None) -> np.ndarray:
+    """One block over the compact rows ``u_in`` [A,H]; ``kv_l`` [B,2,N,H] is updated in place."""
+    A, H = u_in.shape
+    B, _, N, _ = kv_l.shape
+    M = w["w_fc1"].shape[1]
+    assert kv_l.dtype == np.float32 and kv_l.flags["C_CONTIGUOUS"]
+    u_out = np.zeros((A, H), np.float32)
+    fin = None if finish is None else np.ascontiguousarray(finish, np.int32)
+    rc = _load().fdo_regional_block(
+        B, N, H, heads, H // heads, M, A, _ip(np.ascontiguousarray(active_idx, np.int32)), _fp(_c(mod)),
+        _fp(_c(w["w_qkv"][l])), _fp(_c(w["b_qkv"][l])), _fp(_c(w["w_o"][l])), _fp(_c(w["b_o"][l])),
+        _fp(_c(w["w_fc1"][l])), _fp(_c(w["b_fc1"][l])), _fp(_c(w["w_fc2"][l])), _fp(_c(w["b_fc2"][l])),
+        ctypes.c_float(ln_eps), _fp(_c(u_in)), _fp(u_out), _fp(kv_l),
+        0 if fin is None else int(fin.size), _ip(fin))
+    assert rc == 0
+    return u_out
+
+
+def regional_step(x: np.ndarray, cond: np.ndarray, labels: np.ndarray, mask: np.ndarray,
+                  w: Dict[str, np.ndarray], kv: np.ndarray, y: np.ndarray, heads: int, R: int,
+                  ln_eps: float = 1e-6, n_blocks: Optional[int] = None):
+    """The whole block stack on active tokens.
+
+    x [B,N,H]; kv [L,B,2,N,H] and y [B,N,H] are updated in place: rows of active tokens are
+    rewritten, every other row keeps what it held (the cached K/V and the cached output of the
+    step at which that token last ran).  Returns active_idx, cu_active.
+    """
+    B, N, H = x.shape
+    L = w["w_qkv"].shape[0] if n_blocks is None else n_blocks
+    active_idx, cu_active = compact(mask, labels, R)
+    u = np.ascontiguousarray(x.reshape(B * N, H)[active_idx], np.float32)
+    for l in range(L):
+        mod = adaln(cond, w["w_ada"][l], w["b_ada"][l])
+        u = regional_block(u, active_idx, mod, w, l, kv[l], heads, ln_eps)
+    y.reshape(B * N, H)[active_idx] = u
+    return active_idx, cu_active
+
+
+def dense_block(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], l: int, heads: int,
+                ln_eps: float = 1e-6):
+    """One ungated block on whole matrices. Returns x_out [B,N,H], kv [B,2,N,H]."""
+    B, N, H = x.shape
+    M = w["w_fc1"].shape[1]
+    Hc = cond.shape[1]
+    x_out = np.empty((B, N, H), np.float32)
+    kv = np.empty((B, 2, N, H), np.float32)
+    rc = _load().fdo_dense_block(
+        B, N, H, heads, H // heads, M, Hc, _fp(_c(cond)), _fp(_c(w["w_ada"][l])), _fp(_c(w["b_ada"][l])),
+        _fp(_c(w["w_qkv"][l])), _fp(_c(w["b_qkv"][l])), _fp(_c(w["w_o"][l])), _fp(_c(w["b_o"][l])),
+        _fp(_c(w["w_fc1"][l])), _fp(_c(w["b_fc1"][l])), _fp(_c(w["w_fc2"][l])), _fp(_c(w["b_fc2"][l])),
+        ctypes.c_float(ln_eps), _fp(_c(x)), _fp(x_out), _fp(kv))
+    assert rc == 0
+    return x_out, kv
+
+
+def dense_step(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], heads: int,
+               ln_eps: float = 1e-6, n_blocks: Optional[int] = None):
+    """The ungated block stack. Returns y [B,N,H] and kv [L,B,2,N,H]."""
+    L = w["w_qkv"].shape[0] if n_blocks is None else n_blocks
+    B, N, H = x.shape
+    kv = np.empty((L, B, 2, N, H), np.float32)
+    cur = np.ascontiguousarray(x, np.float32)
+    for l in range(L):
+        cur, kv[l] = dense_block(cur, cond, w, l, heads, ln_eps)
+    return cur, kv

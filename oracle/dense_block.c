@@ -1,0 +1,147 @@
+/*
+ * TEST INFRASTRUCTURE -- CPU oracle: one ordinary (ungated) adaLN-Zero transformer block.
+ *
+ * Only tests, the smoke check and the CPU-baseline leg of the benchmark may call this.
+ * It shares no code with the CUDA library, and none with the regional oracle either: it is
+ * a second, separately written statement of the block, working on whole matrices with no
+ * mask and no index list.  It exists so that "no region skipped gives the baseline
+ * trajectory" (paper Sec. 4.2, quality-bound theorem: the gap vanishes without gating) can
+ * be checked by comparing two independent programs.
+ *
+ * Same numeric convention as the regional oracle: fp32 storage, fp64 accumulation in
+ * ascending index order, one rounding per stored value.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* Y[r,o] = sum_k X[r,k] W[o,k] + bias[o] */
+static void matmul_nt_bias(const float* X, const float* W, const float* bias, size_t rows, int K,
+                           int O, float* Y) {
+#pragma omp parallel for schedule(static)
+    for (size_t r = 0; r < rows; ++r)
+        for (int o = 0; o < O; ++o) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k) acc += (double)X[r * K + k] * (double)W[(size_t)o * K + k];
+            Y[r * O + o] = (float)(acc + (double)bias[o]);
+        }
+}
+
+/* rows of one request: LayerNorm without affine, then * (1 + scale) + shift */
+static void layernorm_modulate(const float* X, size_t rows, int H, const float* shift,
+                               const float* scale, float eps, float* Y) {
+#pragma omp parallel for schedule(static)
+    for (size_t r = 0; r < rows; ++r) {
+        const float* x = X + r * H;
+        double m = 0.0;
+        for (int c = 0; c < H; ++c) m += (double)x[c];
+        m /= (double)H;
+        double v = 0.0;
+        for (int c = 0; c < H; ++c) { double d = (double)x[c] - m; v += d * d; }
+        v /= (double)H;
+        const double rs = 1.0 / sqrt(v + (double)eps);
+        for (int c = 0; c < H; ++c)
+            Y[r * H + c] = (float)((((double)x[c] - m) * rs) * (1.0 + (double)scale[c]) + (double)shift[c]);
+    }
+}
+
+/* O[i, h*dh + c] = sum_t softmax_t(Q_i . K_t / sqrt(dh)) V[t, h*dh + c], all N x N pairs */
+static void full_attention(const float* Q, const float* K, const float* V, int N, int heads, int dh,
+                           float* O) {
+    const int H = heads * dh;
+    const double scale = 1.0 / sqrt((double)dh);
+#pragma omp parallel
+    {
+        double* s = (double*)malloc(sizeof(double) * (size_t)N);
+        double* acc = (double*)malloc(sizeof(double) * (size_t)dh);
+#pragma omp for schedule(dynamic, 1) collapse(2)
+        for (int i = 0; i < N; ++i)
+            for (int h = 0; h < heads; ++h) {
+                double mx = -INFINITY;
+                for (int t = 0; t < N; ++t) {
+                    double d = 0.0;
+                    for (int c = 0; c < dh; ++c)
+                        d += (double)Q[(size_t)i * H + h * dh + c] * (double)K[(size_t)t * H + h * dh + c];
+                    s[t] = d * scale;
+                    if (s[t] > mx) mx = s[t];
+                }
+                double z = 0.0;
+                for (int c = 0; c < dh; ++c) acc[c] = 0.0;
+                for (int t = 0; t < N; ++t) {
+                    const double e = exp(s[t] - mx);
+                    z += e;
+                    for (int c = 0; c < dh; ++c) acc[c] += e * (double)V[(size_t)t * H + h * dh + c];
+                }
+                for (int c = 0; c < dh; ++c) O[(size_t)i * H + h * dh + c] = (float)(acc[c] / z);
+            }
+        free(s); free(acc);
+    }
+}
+
+/*
+ * x_in, x_out [B,N,H]; kv_out [B,2,N,H] receives K and V of every position.
+ * cond [B,Hc]; adaLN chunk order shift_msa, scale_msa, gate_msa, shift_mlp, scale_mlp, gate_mlp.
+ */
+int fdo_dense_block(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+                    const float* w_ada, const float* b_ada, const float* w_qkv, const float* b_qkv,
+                    const float* w_o, const float* b_o, const float* w_fc1, const float* b_fc1,
+                    const float* w_fc2, const float* b_fc2, float ln_eps, const float* x_in,
+                    float* x_out, float* kv_out) {
+    if (heads * dh != H) return 2;
+    const size_t NH = (size_t)N * H;
+    float* act = (float*)malloc(sizeof(float) * (size_t)Hc);
+    float* mod = (float*)malloc(sizeof(float) * (size_t)6 * H);
+    float* xh = (float*)malloc(sizeof(float) * NH);
+    float* qkv = (float*)malloc(sizeof(float) * NH * 3);
+    float* Q = (float*)malloc(sizeof(float) * NH);
+    float* att = (float*)malloc(sizeof(float) * NH);
+    float* proj = (float*)malloc(sizeof(float) * NH);
+    float* res = (float*)malloc(sizeof(float) * NH);
+    float* hid = (float*)malloc(sizeof(float) * (size_t)N * M);
+    int rc = 0;
+    if (!act || !mod || !xh || !qkv || !Q || !att || !proj || !res || !hid) { rc = 1; goto done; }
+
+    for (int b = 0; b < B; ++b) {
+        const float* X = x_in + (size_t)b * NH;
+        float* Kc = kv_out + ((size_t)b * 2 + 0) * NH;
+        float* Vc = kv_out + ((size_t)b * 2 + 1) * NH;
+
+        /* conditioning: six H-vectors from SiLU(cond) */
+        for (int c = 0; c < Hc; ++c) {
+            const double v = (double)cond[(size_t)b * Hc + c];
+            act[c] = (float)(v / (1.0 + exp(-v)));
+        }
+        matmul_nt_bias(act, w_ada, b_ada, 1, Hc, 6 * H, mod);
+        const float *shift_a = mod, *scale_a = mod + H, *gate_a = mod + 2 * H;
+        const float *shift_m = mod + 3 * H, *scale_m = mod + 4 * H, *gate_m = mod + 5 * H;
+
+        /* attention branch */
+        layernorm_modulate(X, (size_t)N, H, shift_a, scale_a, ln_eps, xh);
+        matmul_nt_bias(xh, w_qkv, b_qkv, (size_t)N, H, 3 * H, qkv);
+        for (int t = 0; t < N; ++t) {
+            memcpy(Q + (size_t)t * H, qkv + (size_t)t * 3 * H, sizeof(float) * (size_t)H);
+            memcpy(Kc + (size_t)t * H, qkv + (size_t)t * 3 * H + H, sizeof(float) * (size_t)H);
+            memcpy(Vc + (size_t)t * H, qkv + (size_t)t * 3 * H + 2 * H, sizeof(float) * (size_t)H);
+        }
+        full_attention(Q, Kc, Vc, N, heads, dh, att);
+        matmul_nt_bias(att, w_o, b_o, (size_t)N, H, H, proj);
+        for (size_t e = 0; e < NH; ++e)
+            res[e] = (float)((double)X[e] + (double)gate_a[e % H] * (double)proj[e]);
+
+        /* MLP branch */
+        layernorm_modulate(res, (size_t)N, H, shift_m, scale_m, ln_eps, xh);
+        matmul_nt_bias(xh, w_fc1, b_fc1, (size_t)N, H, M, hid);
+        for (size_t e = 0; e < (size_t)N * M; ++e) {
+            const double a = (double)hid[e];
+            hid[e] = (float)(0.5 * a * (1.0 + tanh(0.79788456080286535588 * (a + 0.044715 * a * a * a))));
+        }
+        matmul_nt_bias(hid, w_fc2, b_fc2, (size_t)N, M, H, proj);
+        float* Y = x_out + (size_t)b * NH;
+        for (size_t e = 0; e < NH; ++e)
+            Y[e] = (float)((double)res[e] + (double)gate_m[e % H] * (double)proj[e]);
+    }
+done:
+    free(act); free(mod); free(xh); free(qkv); free(Q); free(att); free(proj); free(res); free(hid);
+    return rc;
+}

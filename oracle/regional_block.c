@@ -1,0 +1,175 @@
+/*
+ * TEST INFRASTRUCTURE -- CPU oracle for one region-selective transformer block.
+ *
+ * Only tests, the smoke check and the CPU-baseline leg of the benchmark may call this.
+ * It shares no code with the CUDA library.
+ *
+ * What it computes (paper Sec. 3 "Adaptive execution", Sec. 5 worker backend, Appendix A.6):
+ * active patches are executed while skipped patches reuse cached state; active queries
+ * attend to the K/V of every position, where skipped positions keep the K/V of the step at
+ * which they last ran.  The block itself is the adaLN-Zero DiT block the paper builds on
+ * (Sec. 2.1): LayerNorm without affine, (1+scale)/shift modulation, gated residuals,
+ * tanh-GELU MLP.
+ *
+ * Numerics: every tensor is stored in fp32; every sum of more than a few terms is
+ * accumulated in fp64 in ascending index order and rounded to fp32 once.  Rows are handled
+ * one at a time with plain loops; OpenMP only spreads independent rows over cores.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static double silu_d(double x) { return x / (1.0 + exp(-x)); }
+
+static double gelu_tanh_d(double a) {
+    const double c = 0.79788456080286535588; /* sqrt(2/pi) */
+    return 0.5 * a * (1.0 + tanh(c * (a + 0.044715 * a * a * a)));
+}
+
+/* y[o] = sum_k x[k] * w[o*K + k] + bias[o], one output at a time */
+static void row_linear(const float* x, const float* w, const float* bias, int K, int O, float* y) {
+    for (int o = 0; o < O; ++o) {
+        const float* wr = w + (size_t)o * K;
+        double acc = 0.0;
+        for (int k = 0; k < K; ++k) acc += (double)x[k] * (double)wr[k];
+        y[o] = (float)(acc + (double)bias[o]);
+    }
+}
+
+/* LayerNorm (biased variance, no affine) followed by (1+scale), shift */
+static void row_ln_modulate(const float* u, const float* shift, const float* scale, int H,
+                            float ln_eps, float* out) {
+    double mean = 0.0;
+    for (int c = 0; c < H; ++c) mean += (double)u[c];
+    mean /= (double)H;
+    double var = 0.0;
+    for (int c = 0; c < H; ++c) { double d = (double)u[c] - mean; var += d * d; }
+    var /= (double)H;
+    const double rstd = 1.0 / sqrt(var + (double)ln_eps);
+    for (int c = 0; c < H; ++c)
+        out[c] = (float)((((double)u[c] - mean) * rstd) * (1.0 + (double)scale[c]) + (double)shift[c]);
+}
+
+/* mod[b, 6H] = W_ada * SiLU(cond[b]) + b_ada ; chunk order shift_msa, scale_msa, gate_msa,
+ * shift_mlp, scale_mlp, gate_mlp */
+int fdo_adaln(int B, int H, int Hc, const float* cond, const float* w_ada, const float* b_ada,
+              float* mod) {
+    float* s = (float*)malloc(sizeof(float) * (size_t)Hc);
+    if (!s) return 1;
+    for (int b = 0; b < B; ++b) {
+        for (int c = 0; c < Hc; ++c) s[c] = (float)silu_d((double)cond[(size_t)b * Hc + c]);
+        row_linear(s, w_ada, b_ada, Hc, 6 * H, mod + (size_t)b * 6 * H);
+    }
+    free(s);
+    return 0;
+}
+
+/*
+ * One block over the active rows only.
+ *   active_idx[A]   global token ids b*N + j, ascending
+ *   u_in/u_out[A,H] compact residual stream entering / leaving the block
+ *   kv[B,2,N,H]     this block's K (index 0) and V (index 1) cache, updated in place for
+ *                   active rows; every other row is left as it is
+ *   finish[n_finish] compact rows whose attention + MLP are evaluated (NULL = all A rows);
+ *                   K/V are always refreshed for all A rows because every query needs them.
+ * Rows outside `finish` get no u_out.
+ */
+int fdo_regional_block(int B, int N, int H, int heads, int dh, int M, int A,
+                       const int32_t* active_idx, const float* mod,
+                       const float* w_qkv, const float* b_qkv, const float* w_o, const float* b_o,
+                       const float* w_fc1, const float* b_fc1, const float* w_fc2, const float* b_fc2,
+                       float ln_eps, const float* u_in, float* u_out, float* kv,
+                       int n_finish, const int32_t* finish) {
+    if (heads * dh != H) return 2;
+    (void)B;
+    float* q_all = (float*)malloc(sizeof(float) * (size_t)(A > 0 ? A : 1) * H);
+    if (!q_all) return 1;
+    int err = 0;
+
+    /* pass 1: normalise, modulate, project; scatter K and V of every active row */
+#pragma omp parallel
+    {
+        float* uh = (float*)malloc(sizeof(float) * (size_t)H);
+        float* qkv = (float*)malloc(sizeof(float) * (size_t)3 * H);
+        if (!uh || !qkv) {
+#pragma omp atomic write
+            err = 1;
+        } else {
+#pragma omp for schedule(dynamic, 4)
+            for (int a = 0; a < A; ++a) {
+                const int b = active_idx[a] / N, j = active_idx[a] % N;
+                const float* md = mod + (size_t)b * 6 * H;
+                row_ln_modulate(u_in + (size_t)a * H, md + 0 * H, md + 1 * H, H, ln_eps, uh);
+                row_linear(uh, w_qkv, b_qkv, H, 3 * H, qkv);
+                memcpy(q_all + (size_t)a * H, qkv, sizeof(float) * (size_t)H);
+                memcpy(kv + (((size_t)b * 2 + 0) * N + j) * H, qkv + H, sizeof(float) * (size_t)H);
+                memcpy(kv + (((size_t)b * 2 + 1) * N + j) * H, qkv + 2 * H, sizeof(float) * (size_t)H);
+            }
+        }
+        free(uh); free(qkv);
+    }
+    if (err) { free(q_all); return err; }
+
+    /* pass 2: attention against all N cached keys of the row's request, then the MLP */
+    const int n_rows = finish ? n_finish : A;
+    const double sm_scale = 1.0 / sqrt((double)dh);
+#pragma omp parallel
+    {
+        double* s = (double*)malloc(sizeof(double) * (size_t)N);
+        double* oacc = (double*)malloc(sizeof(double) * (size_t)dh);
+        float* o = (float*)malloc(sizeof(float) * (size_t)H);
+        float* proj = (float*)malloc(sizeof(float) * (size_t)H);
+        float* r1 = (float*)malloc(sizeof(float) * (size_t)H);
+        float* mh = (float*)malloc(sizeof(float) * (size_t)H);
+        float* g = (float*)malloc(sizeof(float) * (size_t)M);
+        if (!s || !oacc || !o || !proj || !r1 || !mh || !g) {
+#pragma omp atomic write
+            err = 1;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int i = 0; i < n_rows; ++i) {
+                const int a = finish ? finish[i] : i;
+                const int b = active_idx[a] / N;
+                const float* md = mod + (size_t)b * 6 * H;
+                const float* Kb = kv + ((size_t)b * 2 + 0) * N * H;
+                const float* Vb = kv + ((size_t)b * 2 + 1) * N * H;
+                const float* q = q_all + (size_t)a * H;
+                for (int h = 0; h < heads; ++h) {
+                    const float* qh = q + h * dh;
+                    double smax = -INFINITY;
+                    for (int t = 0; t < N; ++t) {
+                        const float* kt = Kb + (size_t)t * H + h * dh;
+                        double acc = 0.0;
+                        for (int c = 0; c < dh; ++c) acc += (double)qh[c] * (double)kt[c];
+                        s[t] = acc * sm_scale;
+                        if (s[t] > smax) smax = s[t];
+                    }
+                    double denom = 0.0;
+                    for (int c = 0; c < dh; ++c) oacc[c] = 0.0;
+                    for (int t = 0; t < N; ++t) {
+                        const double p = exp(s[t] - smax);
+                        const float* vt = Vb + (size_t)t * H + h * dh;
+                        denom += p;
+                        for (int c = 0; c < dh; ++c) oacc[c] += p * (double)vt[c];
+                    }
+                    for (int c = 0; c < dh; ++c) o[h * dh + c] = (float)(oacc[c] / denom);
+                }
+                const float* u = u_in + (size_t)a * H;
+                row_linear(o, w_o, b_o, H, H, proj);
+                for (int c = 0; c < H; ++c)
+                    r1[c] = (float)((double)u[c] + (double)md[2 * H + c] * (double)proj[c]);
+                row_ln_modulate(r1, md + 3 * H, md + 4 * H, H, ln_eps, mh);
+                row_linear(mh, w_fc1, b_fc1, H, M, g);
+                for (int c = 0; c < M; ++c) g[c] = (float)gelu_tanh_d((double)g[c]);
+                row_linear(g, w_fc2, b_fc2, M, H, proj);
+                float* out = u_out + (size_t)a * H;
+                for (int c = 0; c < H; ++c)
+                    out[c] = (float)((double)r1[c] + (double)md[5 * H + c] * (double)proj[c]);
+            }
+        }
+        free(s); free(oacc); free(o); free(proj); free(r1); free(mh); free(g);
+    }
+    free(q_all);
+    return err;
+}
