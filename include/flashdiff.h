@@ -1,0 +1,176 @@
+/*
+ * libflashdiff -- region-selective denoising step of a diffusion transformer on one B200.
+ *
+ * C ABI.  Unless a parameter says "host", every pointer is a DEVICE pointer owned by the
+ * caller.  The library allocates no device memory: all scratch lives in the workspace the
+ * caller hands to fd_create.  Every call enqueues its work on `cuda_stream` (a cudaStream_t
+ * passed as void*; NULL = the default stream), performs no device-to-host synchronisation and
+ * returns as soon as the work is queued; stream order is the only ordering.
+ *
+ * Errors a host can see (null or misaligned pointers, shapes beyond the limits given at
+ * creation, unsupported head sizes) return a status with nothing launched.  Problems only the
+ * device can see (a label outside [0,R], a bounded wait that ran out) never trap: the kernel
+ * records a code in the workspace, skips the offending work, and fd_poll_status / fd_destroy
+ * report it.
+ */
+#ifndef FLASHDIFF_H_
+#define FLASHDIFF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fd_ctx fd_ctx; /* opaque; created by fd_create, released by fd_destroy */
+
+typedef enum {
+    FD_OK = 0,
+    FD_ERR_INVALID_ARG = 1, /* null / misaligned pointer, negative size                    */
+    FD_ERR_SHAPE = 2,       /* shape beyond the limits of fd_config or inconsistent         */
+    FD_ERR_STATE = 3,       /* device-side check failed (bad label, bad index)              */
+    FD_ERR_WORKSPACE = 4,   /* workspace too small or misaligned                            */
+    FD_ERR_UNSUPPORTED = 5, /* configuration this build has no kernel for                   */
+    FD_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed; see fd_last_error       */
+    FD_ERR_TIMEOUT = 7      /* a bounded device-side wait expired                           */
+} fd_status;
+
+typedef enum { FD_F32 = 0, FD_BF16 = 1 } fd_dtype;
+
+/* Which kernels run the dense contractions. */
+typedef enum {
+    FD_ENGINE_AUTO = 0,  /* tensor cores for FD_BF16, CUDA cores for FD_F32                 */
+    FD_ENGINE_SIMT = 1,  /* CUDA-core GEMM and attention (any dtype; validation path)       */
+    FD_ENGINE_TC = 2     /* tcgen05 / TMEM / TMA kernels (FD_BF16 only)                     */
+} fd_engine;
+
+/* Model shape and limits; copied at creation (host struct). */
+typedef struct {
+    int32_t n_blocks;    /* L                                                               */
+    int32_t hidden;      /* H = n_heads * head_dim                                          */
+    int32_t n_heads;
+    int32_t head_dim;
+    int32_t mlp_dim;     /* M                                                               */
+    int32_t cond_dim;    /* Hc, width of the conditioning vector                            */
+    int32_t max_batch;   /* largest B of any later call                                     */
+    int32_t max_tokens;  /* largest N (tokens per request) of any later call                */
+    int32_t max_regions; /* largest R of any later call                                     */
+    int32_t dtype;       /* fd_dtype of x, cond, y, kv_cache and all weights                */
+    int32_t engine;      /* fd_engine                                                       */
+    float ln_eps;        /* LayerNorm epsilon (1e-6 in DiT)                                 */
+    float gate_eta;      /* eta of the gate weight, Appendix A.1 Eq. (gate-weight)          */
+    int32_t max_skip_k;  /* K of the forced reactivation, Appendix A.1                      */
+} fd_config;
+
+/*
+ * Weights of all blocks (host struct of DEVICE pointers), borrowed until fd_destroy.
+ * Row-major with the input dimension contiguous, block index outermost, element type
+ * fd_config.dtype.  The six adaLN chunks of w_ada / b_ada are, in order: shift_msa,
+ * scale_msa, gate_msa, shift_mlp, scale_mlp, gate_mlp.  All pointers 16-byte aligned.
+ */
+typedef struct {
+    const void *w_qkv, *b_qkv; /* [L,3H,H], [L,3H]  rows: Q then K then V                   */
+    const void *w_o, *b_o;     /* [L,H,H],  [L,H]                                           */
+    const void *w_fc1, *b_fc1; /* [L,M,H],  [L,M]                                           */
+    const void *w_fc2, *b_fc2; /* [L,H,M],  [L,H]                                           */
+    const void *w_ada, *b_ada; /* [L,6H,Hc],[L,6H]                                          */
+} fd_weights;
+
+/* Bytes of device scratch fd_create needs for this configuration (0 if the config is bad). */
+size_t fd_workspace_bytes(const fd_config* cfg);
+
+/*
+ * Creates a context on the current CUDA device.  `workspace` (256-byte aligned, at least
+ * fd_workspace_bytes(cfg) bytes) is borrowed until fd_destroy and must not be touched by the
+ * caller in between.  Builds the TMA descriptors of the weights and of the workspace tensors.
+ * Synchronises the device once (set-up only).
+ */
+fd_status fd_create(const fd_config* cfg, const fd_weights* weights, void* workspace,
+                    size_t workspace_bytes, fd_ctx** out);
+
+/*
+ * Patch Partitioner (paper Sec. 4.1; Appendix A.3, Eq. otsu and the hierarchical-extension
+ * remark): groups the N tokens of each request into R regions from an early-step attention
+ * map.  Saliency S_j is the mean over `salient_cols` of attn_map[b,j,:]; the map is min-max
+ * normalised and quantised to 16 bits; a node is bisected at the threshold that maximises the
+ * between-class variance (focus: value >= threshold); its region budget is shared by
+ * r_f = argmin_r |r - R n_f/(n_f+n_c)|; both halves are split again until R regions exist.
+ * A cut is admissible only if each side can hold its regions with min_region_tokens ..
+ * max_region_tokens tokens per region (max_region_tokens <= 0: unbounded); a node without an
+ * admissible cut is chopped in token order into equal chunks.  Ties: lowest threshold,
+ * smallest r.  Regions are numbered by their smallest token index.
+ *
+ *   attn_map      [B,N,T] f32         salient_cols  [T_s] i32 or NULL (= all T columns)
+ *   labels_out    [B,N]   i32         region_sizes_out [B,R] i32 or NULL
+ * Needs 1 <= R <= N <= max_tokens, R <= max_regions, B <= max_batch, N < 65536.
+ */
+fd_status fd_partition_regions(fd_ctx* ctx, const float* attn_map, int B, int N, int T,
+                               const int32_t* salient_cols, int T_s, int R, int min_region_tokens,
+                               int max_region_tokens, int32_t* labels_out,
+                               int32_t* region_sizes_out, void* cuda_stream);
+
+/*
+ * Patch Gate (paper Sec. 4.2; Appendix A.1 Eq. delta-i, Eq. gate-weight, Eq.
+ * forced-reactivation; Algorithm 1, PatchGate) on the change of the latent between two
+ * neighbouring steps.  For every region i of request b:
+ *   - if the region ran at the previous step (prev_active = 1): delta_i = root mean square of
+ *     z_cur - z_prev over the region's tokens and D channels; otherwise delta_i stays frozen;
+ *   - w_i = (delta_i + eta) / sum_j (delta_j + eta);
+ *   - active iff w_i >= eps[b], or the region was skipped max_skip_k steps in a row;
+ *   - skip_count and prev_active are updated for the next evaluation.
+ * Tokens with label R are always active and take no part in the gate.
+ *
+ *   z_cur, z_prev [B,N,D] f32 (16-byte aligned)   labels [B,N] i32 in [0,R]   eps [B] f32
+ *   delta_state [B,R] f32, skip_count [B,R] i32, prev_active [B,R] u8   (in/out)
+ *   score_out [B,R] f32 (= delta), weight_out [B,R] f32, mask_out [B,R] u8
+ */
+fd_status fd_region_activity(fd_ctx* ctx, const float* z_cur, const float* z_prev,
+                             const int32_t* labels, int B, int N, int D, int R, const float* eps,
+                             float* delta_state, int32_t* skip_count, uint8_t* prev_active,
+                             float* score_out, float* weight_out, uint8_t* mask_out,
+                             void* cuda_stream);
+
+/*
+ * One denoising step of the block stack on the active regions only (paper Sec. 3 "Adaptive
+ * execution": active patches are refined, skipped patches reuse cached states; Sec. 5: active
+ * patches run against the previous step's K/V and refresh only their own K/V; Appendix A.6).
+ *   1. tokens whose region is active (mask[b,labels[b,j]] != 0, or label R) are compacted into
+ *      the ascending list active_idx_out (values b*N+j) with offsets cu_active_out [B+1];
+ *   2. per block: gather, LayerNorm + adaLN modulation, QKV projection; Q stays compact, the
+ *      K and V rows of active tokens overwrite kv_cache[l,b,0/1,j,:]; all other rows keep the
+ *      values of the step at which their token last ran;
+ *   3. each active query attends to all N keys of its request (fresh and cached);
+ *   4. out-projection, gated residual, LayerNorm + modulation, tanh-GELU MLP, gated residual;
+ *   5. after the last block the rows are scattered to y[b,j,:]; all other rows of y keep their
+ *      cached output.
+ * The first step on fresh kv_cache / y must use an all-ones mask (the warm-up steps).
+ *
+ *   x [B,N,H], cond [B,Hc], y [B,N,H], kv_cache [L,B,2,N,H]  of fd_config.dtype, 16-byte aligned
+ *   labels [B,N] i32, mask [B,R] u8
+ *   active_idx_out [B*N] i32 (capacity), cu_active_out [B+1] i32
+ */
+fd_status fd_regional_step(fd_ctx* ctx, const void* x, const void* cond, const int32_t* labels,
+                           const uint8_t* mask, int B, int N, int R, void* kv_cache, void* y,
+                           int32_t* active_idx_out, int32_t* cu_active_out, void* cuda_stream);
+
+/*
+ * Reads the device-side status word (synchronises `cuda_stream`).  Returns FD_OK, or the first
+ * device-side problem recorded since the last poll (FD_ERR_STATE / FD_ERR_TIMEOUT), and clears it.
+ */
+fd_status fd_poll_status(fd_ctx* ctx, void* cuda_stream);
+
+/* Number of kernels the library has launched through this context so far (host counter). */
+int64_t fd_launch_count(const fd_ctx* ctx);
+
+/* Releases the context (host memory only; the workspace goes back to the caller). */
+fd_status fd_destroy(fd_ctx* ctx);
+
+/* Text of the last error of this context (host string owned by the context; NULL ctx: text of
+ * the last failed fd_create on this thread). */
+const char* fd_last_error(const fd_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLASHDIFF_H_ */

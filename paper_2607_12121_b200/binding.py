@@ -1,0 +1,178 @@
+"""Thin ctypes binding of ``libflashdiff.so``: argument marshalling only.
+
+Every function mirrors one C entry point of ``include/flashdiff.h`` and takes torch CUDA
+tensors (device memory and streams are all PyTorch is used for).  No step of the method runs
+in Python.  Importing this module fails loudly if the shared library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libflashdiff.so")
+
+FD_OK = 0
+FD_ERR_INVALID_ARG, FD_ERR_SHAPE, FD_ERR_STATE, FD_ERR_WORKSPACE = 1, 2, 3, 4
+FD_ERR_UNSUPPORTED, FD_ERR_CUDA, FD_ERR_TIMEOUT = 5, 6, 7
+FD_F32, FD_BF16 = 0, 1
+FD_ENGINE_AUTO, FD_ENGINE_SIMT, FD_ENGINE_TC = 0, 1, 2
+
+EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region_activity",
+           "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error"]
+
+
+class FdConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("n_blocks", "hidden", "n_heads", "head_dim", "mlp_dim", "cond_dim", "max_batch",
+                 "max_tokens", "max_regions", "dtype", "engine")] + \
+               [("ln_eps", ctypes.c_float), ("gate_eta", ctypes.c_float), ("max_skip_k", ctypes.c_int32)]
+
+
+class FdWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2", "w_ada", "b_ada")]
+
+
+class FlashDiffError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__("libflashdiff status %d: %s" % (status, text))
+        self.status = status
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("libflashdiff.so is missing: run `python -m paper_2607_12121_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.fd_workspace_bytes.restype = sz
+    lib.fd_workspace_bytes.argtypes = [ctypes.POINTER(FdConfig)]
+    lib.fd_create.restype = i32
+    lib.fd_create.argtypes = [ctypes.POINTER(FdConfig), ctypes.POINTER(FdWeights), vp, sz, ctypes.POINTER(vp)]
+    lib.fd_partition_regions.restype = i32
+    lib.fd_partition_regions.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, i32, vp, vp, vp]
+    lib.fd_region_activity.restype = i32
+    lib.fd_region_activity.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.fd_regional_step.restype = i32
+    lib.fd_regional_step.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.fd_poll_status.restype = i32
+    lib.fd_poll_status.argtypes = [vp, vp]
+    lib.fd_launch_count.restype = ctypes.c_int64
+    lib.fd_launch_count.argtypes = [vp]
+    lib.fd_destroy.restype = i32
+    lib.fd_destroy.argtypes = [vp]
+    lib.fd_last_error.restype = ctypes.c_char_p
+    lib.fd_last_error.argtypes = [vp]
+    return lib
+
+
+lib = _load()
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+def _check(ctx_handle, status: int):
+    if status != FD_OK:
+        text = lib.fd_last_error(ctx_handle)
+        raise FlashDiffError(status, text.decode() if text else "")
+
+
+def fd_workspace_bytes(cfg: FdConfig) -> int:
+    return int(lib.fd_workspace_bytes(ctypes.byref(cfg)))
+
+
+class Context:
+    """Owns the fd_ctx handle plus the torch tensors the library borrows (weights, workspace)."""
+
+    def __init__(self, cfg: FdConfig, weights: Dict[str, "object"], device="cuda"):
+        import torch
+        self.cfg = cfg
+        self.dtype = torch.bfloat16 if cfg.dtype == FD_BF16 else torch.float32
+        self.weights = weights
+        for k, v in weights.items():
+            assert v.is_cuda and v.is_contiguous() and v.dtype == self.dtype, k
+        nbytes = fd_workspace_bytes(cfg)
+        if nbytes == 0:
+            raise FlashDiffError(FD_ERR_SHAPE, "fd_workspace_bytes rejected the configuration")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        w = FdWeights(**{k: weights[k].data_ptr() for k, _ in FdWeights._fields_})
+        handle = ctypes.c_void_p()
+        with torch.cuda.device(self.workspace.device):
+            st = lib.fd_create(ctypes.byref(cfg), ctypes.byref(w), self.workspace.data_ptr(), nbytes,
+                               ctypes.byref(handle))
+        _check(None, st)
+        self.handle = handle
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib.fd_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def launches(self) -> int:
+        return int(lib.fd_launch_count(self.handle))
+
+
+def fd_create(cfg: FdConfig, weights: Dict[str, "object"], device="cuda") -> Context:
+    return Context(cfg, weights, device)
+
+
+def fd_destroy(ctx: Context) -> None:
+    ctx.close()
+
+
+def fd_partition_regions(ctx: Context, attn_map, R: int, labels_out, region_sizes_out=None, salient_cols=None,
+                         min_region_tokens: int = 1, max_region_tokens: int = 0, stream=None) -> None:
+    B, N, T = attn_map.shape
+    T_s = 0 if salient_cols is None else int(salient_cols.numel())
+    _check(ctx.handle, lib.fd_partition_regions(
+        ctx.handle, _ptr(attn_map), B, N, T, _ptr(salient_cols), T_s, R, min_region_tokens, max_region_tokens,
+        _ptr(labels_out), _ptr(region_sizes_out), _stream(stream)))
+
+
+def fd_region_activity(ctx: Context, z_cur, z_prev, labels, R: int, eps, delta_state, skip_count, prev_active,
+                       score_out, weight_out, mask_out, stream=None) -> None:
+    B, N, D = z_cur.shape
+    _check(ctx.handle, lib.fd_region_activity(
+        ctx.handle, _ptr(z_cur), _ptr(z_prev), _ptr(labels), B, N, D, R, _ptr(eps), _ptr(delta_state),
+        _ptr(skip_count), _ptr(prev_active), _ptr(score_out), _ptr(weight_out), _ptr(mask_out), _stream(stream)))
+
+
+def fd_regional_step(ctx: Context, x, cond, labels, mask, R: int, kv_cache, y, active_idx_out, cu_active_out,
+                     stream=None) -> None:
+    B, N, _ = x.shape
+    _check(ctx.handle, lib.fd_regional_step(
+        ctx.handle, _ptr(x), _ptr(cond), _ptr(labels), _ptr(mask), B, N, R, _ptr(kv_cache), _ptr(y),
+        _ptr(active_idx_out), _ptr(cu_active_out), _stream(stream)))
+
+
+def fd_poll_status(ctx: Context, stream=None) -> None:
+    _check(ctx.handle, lib.fd_poll_status(ctx.handle, _stream(stream)))
+
+
+def make_config(wl, max_batch=None, max_tokens=None, max_regions=None, n_blocks=None, engine=FD_ENGINE_AUTO,
+                ln_eps=1e-6, gate_eta=1e-12, max_skip_k=5) -> FdConfig:
+    """fd_config from a workload description (anything with L, H, heads, head_dim, M, Hc, B, N, R, dtype)."""
+    return FdConfig(
+        n_blocks=wl.L if n_blocks is None else n_blocks, hidden=wl.H, n_heads=wl.heads, head_dim=wl.head_dim,
+        mlp_dim=wl.M, cond_dim=wl.Hc, max_batch=wl.B if max_batch is None else max_batch,
+        max_tokens=wl.N if max_tokens is None else max_tokens,
+        max_regions=wl.R if max_regions is None else max_regions,
+        dtype=FD_BF16 if wl.dtype == "bf16" else FD_F32, engine=engine, ln_eps=ln_eps, gate_eta=gate_eta,
+        max_skip_k=max_skip_k)

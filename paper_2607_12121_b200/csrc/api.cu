@@ -1,0 +1,368 @@
+// C-ABI of libflashdiff: argument checks, workspace layout, and the host-side planner that
+// queues one region-selective step (compaction, adaLN vectors, then per block: gather + LN +
+// modulation, QKV with K/V scatter, attention over all keys, out-projection, MLP, residual
+// scatter) on the caller's stream without ever reading the active count back to the host.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "common.cuh"
+#include "tc.cuh"
+
+namespace fd {
+int simt_attention_tile_rows();
+}
+
+using namespace fd;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    size_t control, acc_ss, acc_cnt, block_counts, tiles, mod, resid, act, q, o, g, part, total;
+    int Mcap, q_ld, tile_cap;
+};
+
+bool config_ok(const fd_config* c, std::string* why) {
+    auto bad = [&](const char* m) { if (why) *why = m; return false; };
+    if (!c) return bad("config is null");
+    if (c->n_blocks < 1 || c->hidden < 1 || c->n_heads < 1 || c->head_dim < 1 || c->mlp_dim < 1 || c->cond_dim < 1)
+        return bad("non-positive model dimension");
+    if (c->hidden != c->n_heads * c->head_dim) return bad("hidden != n_heads * head_dim");
+    if (c->max_batch < 1 || c->max_tokens < 1 || c->max_regions < 1) return bad("non-positive limit");
+    if ((long long)c->max_batch * c->max_tokens > (1LL << 30)) return bad("max_batch * max_tokens too large");
+    if (c->dtype != FD_F32 && c->dtype != FD_BF16) return bad("unknown dtype");
+    if (c->engine < FD_ENGINE_AUTO || c->engine > FD_ENGINE_TC) return bad("unknown engine");
+    if (c->hidden % 16 || c->mlp_dim % 16 || c->cond_dim % 8) return bad("hidden, mlp_dim must be multiples of 16 and cond_dim of 8");
+    if (c->head_dim % 4 || c->head_dim > 128) return bad("head_dim must be a multiple of 4, at most 128");
+    if (c->max_skip_k < 0 || !(c->ln_eps > 0.f) || c->gate_eta < 0.f) return bad("bad ln_eps / gate_eta / max_skip_k");
+    return true;
+}
+
+int esize(const fd_config& c) { return c.dtype == FD_BF16 ? 2 : 4; }
+
+Layout make_layout(const fd_config& c) {
+    Layout l{};
+    const size_t es = esize(c);
+    const size_t BR = (size_t)c.max_batch * c.max_regions;
+    l.Mcap = (int)align_up((size_t)c.max_batch * c.max_tokens, 128) + 128;
+    l.q_ld = c.hidden;
+    const int min_tile = 16;
+    l.tile_cap = c.max_batch * ((c.max_tokens + min_tile - 1) / min_tile + 1);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    l.control = take(sizeof(Control));
+    l.acc_ss = take(BR * sizeof(double));
+    l.acc_cnt = take(BR * sizeof(int32_t));
+    l.block_counts = take((size_t)c.max_batch * ((c.max_tokens + 2047) / 2048 + 1) * sizeof(int32_t));
+    l.tiles = take((size_t)l.tile_cap * sizeof(QTile));
+    l.mod = take((size_t)c.n_blocks * c.max_batch * 6 * c.hidden * sizeof(float));
+    l.resid = take((size_t)l.Mcap * c.hidden * sizeof(float));
+    l.act = take((size_t)l.Mcap * c.hidden * es);
+    l.q = take((size_t)l.Mcap * l.q_ld * es);
+    l.o = take((size_t)l.Mcap * c.hidden * es);
+    l.g = take((size_t)l.Mcap * c.mlp_dim * es);
+    l.part = take(partition_scratch_bytes(c.max_batch, c.max_tokens, c.max_regions));
+    l.total = off;
+    return l;
+}
+
+}  // namespace
+
+struct fd_ctx {
+    fd_config cfg;
+    fd_weights w;
+    Layout lay;
+    char* ws;
+    bool use_tc;
+    int tile_rows;
+    int64_t launches;
+    std::string err;
+    TcPlan* tc;
+
+    fd_status fail(fd_status s, const char* fmt, ...) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        err = buf;
+        return s;
+    }
+    template <typename P> P* at(size_t off) const { return reinterpret_cast<P*>(ws + off); }
+    Control* ctl() const { return at<Control>(lay.control); }
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+template <typename T>
+fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* labels, const uint8_t* mask, int B,
+                   int N, int R, void* kv_, void* y_, int32_t* active_idx, int32_t* cu_active, cudaStream_t st) {
+    const fd_config& cf = c->cfg;
+    const Layout& l = c->lay;
+    const int H = cf.hidden, M = cf.mlp_dim, L = cf.n_blocks, Hc = cf.cond_dim;
+    const T* x = static_cast<const T*>(x_);
+    const T* cond = static_cast<const T*>(cond_);
+    T* kv = static_cast<T*>(kv_);
+    Control* ctl = c->ctl();
+    float* mod = c->at<float>(l.mod);
+    float* resid = c->at<float>(l.resid);
+    T* act = c->at<T>(l.act);
+    T* q = c->at<T>(l.q);
+    T* o = c->at<T>(l.o);
+    T* g = c->at<T>(l.g);
+    QTile* tiles = c->at<QTile>(l.tiles);
+    const int rows_cap = B * N;
+    int nl = 0;
+    cudaError_t e;
+#define FD_TRY(call)                                                                                     \
+    do {                                                                                                 \
+        e = (call);                                                                                      \
+        if (e != cudaSuccess) {                                                                          \
+            c->launches += nl;                                                                           \
+            return c->fail(FD_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e));                  \
+        }                                                                                                \
+    } while (0)
+
+    FD_TRY(launch_compact(mask, labels, B, N, R, active_idx, cu_active, c->at<int32_t>(l.block_counts), tiles,
+                          c->tile_rows, ctl, st, &nl));
+    FD_TRY(launch_adaln<T>(cond, static_cast<const T*>(c->w.w_ada), static_cast<const T*>(c->w.b_ada), mod, L, B, H,
+                           Hc, st, &nl));
+    const int max_tiles = B * ((N + c->tile_rows - 1) / c->tile_rows);
+    for (int blk = 0; blk < L; ++blk) {
+        const float* mod_b = mod + (size_t)blk * B * 6 * H;
+        const T* w_qkv = static_cast<const T*>(c->w.w_qkv) + (size_t)blk * 3 * H * H;
+        const T* w_o = static_cast<const T*>(c->w.w_o) + (size_t)blk * H * H;
+        const T* w_fc1 = static_cast<const T*>(c->w.w_fc1) + (size_t)blk * M * H;
+        const T* w_fc2 = static_cast<const T*>(c->w.w_fc2) + (size_t)blk * H * M;
+        T* kv_b = kv + (size_t)blk * B * 2 * N * H;
+
+        EpiParams ep{};
+        ep.active_idx = active_idx;
+        ep.N = N;
+        ep.H = H;
+
+        // gather (first block) or read the residual stream; LayerNorm; attention-branch modulation
+        FD_TRY(launch_ln_modulate<T>(blk == 0 ? x : nullptr, resid, resid, act, active_idx, mod_b + 0 * H,
+                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl));
+        // QKV projection; K and V rows go straight into the cache
+        ep.bias = static_cast<const T*>(c->w.b_qkv) + (size_t)blk * 3 * H;
+        ep.q = q;
+        ep.q_ld = l.q_ld;
+        ep.kv = kv_b;
+        if (c->use_tc)
+            FD_TRY(tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));
+        else
+            FD_TRY(launch_simt_gemm<T>(EPI_QKV, act, H, w_qkv, 3 * H, H, rows_cap, ep, ctl, st, &nl));
+        // active queries against all N keys of their request
+        if (c->use_tc)
+            FD_TRY(tc_attention(c->tc, blk, kv_b, B, N, tiles, max_tiles, ctl, st, &nl));
+        else
+            FD_TRY(launch_simt_attention<T>(q, l.q_ld, kv_b, o, H, tiles, max_tiles, N, H, cf.n_heads, cf.head_dim,
+                                            ctl, st, &nl));
+        // out-projection, gated residual
+        ep.bias = static_cast<const T*>(c->w.b_o) + (size_t)blk * H;
+        ep.resid = resid;
+        ep.gate = mod_b + 2 * H;
+        ep.y = nullptr;
+        if (c->use_tc)
+            FD_TRY(tc_gemm(c->tc, TC_GEMM_OUT, blk, ep, ctl, st, &nl));
+        else
+            FD_TRY(launch_simt_gemm<T>(EPI_RESID, o, H, w_o, H, H, rows_cap, ep, ctl, st, &nl));
+        // MLP branch
+        FD_TRY(launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, mod_b + 3 * H, mod_b + 4 * H, 6 * H, N,
+                                     H, rows_cap, cf.ln_eps, ctl, st, &nl));
+        ep.bias = static_cast<const T*>(c->w.b_fc1) + (size_t)blk * M;
+        ep.out = g;
+        ep.out_ld = M;
+        if (c->use_tc)
+            FD_TRY(tc_gemm(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl));
+        else
+            FD_TRY(launch_simt_gemm<T>(EPI_GELU, act, H, w_fc1, M, H, rows_cap, ep, ctl, st, &nl));
+        ep.bias = static_cast<const T*>(c->w.b_fc2) + (size_t)blk * H;
+        ep.gate = mod_b + 5 * H;
+        ep.y = (blk == L - 1) ? y_ : nullptr;       // the last block scatters the rows back
+        if (c->use_tc)
+            FD_TRY(tc_gemm(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl));
+        else
+            FD_TRY(launch_simt_gemm<T>(EPI_RESID, g, M, w_fc2, H, M, rows_cap, ep, ctl, st, &nl));
+    }
+#undef FD_TRY
+    c->launches += nl;
+    return FD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t fd_workspace_bytes(const fd_config* cfg) {
+    if (!config_ok(cfg, nullptr)) return 0;
+    return make_layout(*cfg).total;
+}
+
+fd_status fd_create(const fd_config* cfg, const fd_weights* weights, void* workspace, size_t workspace_bytes,
+                    fd_ctx** out) {
+    if (!out) { g_create_error = "out is null"; return FD_ERR_INVALID_ARG; }
+    *out = nullptr;
+    std::string why;
+    if (!config_ok(cfg, &why)) { g_create_error = why; return FD_ERR_SHAPE; }
+    if (!weights) { g_create_error = "weights is null"; return FD_ERR_INVALID_ARG; }
+    const void* wp[10] = {weights->w_qkv, weights->b_qkv, weights->w_o, weights->b_o, weights->w_fc1,
+                          weights->b_fc1, weights->w_fc2, weights->b_fc2, weights->w_ada, weights->b_ada};
+    for (const void* p : wp)
+        if (!p || !aligned16(p)) { g_create_error = "weight pointer null or not 16-byte aligned"; return FD_ERR_INVALID_ARG; }
+    const Layout lay = make_layout(*cfg);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < lay.total) {
+        g_create_error = "workspace null, not 256-byte aligned, or smaller than fd_workspace_bytes";
+        return FD_ERR_WORKSPACE;
+    }
+    bool use_tc = false;
+    if (cfg->engine == FD_ENGINE_TC || (cfg->engine == FD_ENGINE_AUTO && cfg->dtype == FD_BF16)) {
+        std::string tc_why;
+        if (cfg->dtype == FD_BF16 && tc_supported(*cfg, &tc_why)) {
+            use_tc = true;
+        } else if (cfg->engine == FD_ENGINE_TC) {
+            g_create_error = "tensor-core engine unavailable for this configuration: " + tc_why;
+            return FD_ERR_UNSUPPORTED;
+        }
+    }
+    int dev_count = 0;
+    cudaError_t e = cudaGetDeviceCount(&dev_count);
+    if (e != cudaSuccess || dev_count == 0) {
+        g_create_error = std::string("no CUDA device: ") + cudaGetErrorString(e);
+        return FD_ERR_CUDA;
+    }
+    fd_ctx* c = new (std::nothrow) fd_ctx();
+    if (!c) { g_create_error = "out of host memory"; return FD_ERR_INVALID_ARG; }
+    c->cfg = *cfg;
+    c->w = *weights;
+    c->lay = lay;
+    c->ws = static_cast<char*>(workspace);
+    c->use_tc = use_tc;
+    c->tile_rows = use_tc ? tc_attention_tile_rows() : simt_attention_tile_rows();
+    c->launches = 0;
+    c->tc = nullptr;
+    // control block and gate accumulators start at zero; the compact buffers start finite
+    e = cudaMemset(workspace, 0, lay.mod);
+    if (e == cudaSuccess) e = cudaMemset(c->ws + lay.resid, 0, lay.part - lay.resid);
+    if (e == cudaSuccess && use_tc) {
+        TcBuffers tb{};
+        tb.act = c->ws + lay.act; tb.q = c->ws + lay.q; tb.o = c->ws + lay.o; tb.g = c->ws + lay.g;
+        tb.Mcap = lay.Mcap; tb.q_ld = lay.q_ld;
+        std::string tc_err;
+        c->tc = tc_plan_create(*cfg, *weights, tb, &tc_err);
+        if (!c->tc) {
+            g_create_error = "tensor-core plan: " + tc_err;
+            delete c;
+            return FD_ERR_CUDA;
+        }
+    }
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        g_create_error = std::string("workspace initialisation failed: ") + cudaGetErrorString(e);
+        tc_plan_destroy(c->tc);
+        delete c;
+        return FD_ERR_CUDA;
+    }
+    *out = c;
+    return FD_OK;
+}
+
+fd_status fd_partition_regions(fd_ctx* c, const float* attn_map, int B, int N, int T, const int32_t* salient_cols,
+                               int T_s, int R, int min_region_tokens, int max_region_tokens, int32_t* labels_out,
+                               int32_t* region_sizes_out, void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!attn_map || !labels_out) return c->fail(FD_ERR_INVALID_ARG, "attn_map / labels_out is null");
+    if (B < 1 || N < 1 || T < 1 || R < 1) return c->fail(FD_ERR_SHAPE, "B, N, T, R must be positive");
+    if (B > c->cfg.max_batch || N > c->cfg.max_tokens || R > c->cfg.max_regions)
+        return c->fail(FD_ERR_SHAPE, "B=%d N=%d R=%d exceed the limits %d/%d/%d", B, N, R, c->cfg.max_batch,
+                       c->cfg.max_tokens, c->cfg.max_regions);
+    if (R > N) return c->fail(FD_ERR_SHAPE, "R=%d exceeds N=%d", R, N);
+    if (N >= 65536) return c->fail(FD_ERR_UNSUPPORTED, "partitioner handles N < 65536");
+    if (salient_cols && T_s < 1) return c->fail(FD_ERR_SHAPE, "T_s must be positive when salient_cols is given");
+    if (min_region_tokens < 1) min_region_tokens = 1;
+    if (max_region_tokens <= 0 || max_region_tokens > N) max_region_tokens = N;
+    int nl = 0;
+    cudaError_t e = launch_partition(attn_map, B, N, T, salient_cols, salient_cols ? T_s : T, R, min_region_tokens,
+                                     max_region_tokens, labels_out, region_sizes_out, c->ws + c->lay.part, c->ctl(),
+                                     static_cast<cudaStream_t>(cuda_stream), &nl);
+    c->launches += nl;
+    if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "partition launch failed: %s", cudaGetErrorString(e));
+    return FD_OK;
+}
+
+fd_status fd_region_activity(fd_ctx* c, const float* z_cur, const float* z_prev, const int32_t* labels, int B, int N,
+                             int D, int R, const float* eps, float* delta_state, int32_t* skip_count,
+                             uint8_t* prev_active, float* score_out, float* weight_out, uint8_t* mask_out,
+                             void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!z_cur || !z_prev || !labels || !eps || !delta_state || !skip_count || !prev_active || !score_out ||
+        !weight_out || !mask_out)
+        return c->fail(FD_ERR_INVALID_ARG, "null pointer argument");
+    if (B < 1 || N < 1 || D < 1 || R < 1) return c->fail(FD_ERR_SHAPE, "B, N, D, R must be positive");
+    if (B > c->cfg.max_batch || N > c->cfg.max_tokens || R > c->cfg.max_regions)
+        return c->fail(FD_ERR_SHAPE, "B=%d N=%d R=%d exceed the limits %d/%d/%d", B, N, R, c->cfg.max_batch,
+                       c->cfg.max_tokens, c->cfg.max_regions);
+    int nl = 0;
+    cudaError_t e = launch_activity(z_cur, z_prev, labels, B, N, D, R, eps, delta_state, skip_count, prev_active,
+                                    score_out, weight_out, mask_out, c->cfg.gate_eta, c->cfg.max_skip_k,
+                                    c->at<double>(c->lay.acc_ss), c->at<int32_t>(c->lay.acc_cnt), c->ctl(),
+                                    static_cast<cudaStream_t>(cuda_stream), &nl);
+    c->launches += nl;
+    if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "activity launch failed: %s", cudaGetErrorString(e));
+    return FD_OK;
+}
+
+fd_status fd_regional_step(fd_ctx* c, const void* x, const void* cond, const int32_t* labels, const uint8_t* mask,
+                           int B, int N, int R, void* kv_cache, void* y, int32_t* active_idx_out,
+                           int32_t* cu_active_out, void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!x || !cond || !labels || !mask || !kv_cache || !y || !active_idx_out || !cu_active_out)
+        return c->fail(FD_ERR_INVALID_ARG, "null pointer argument");
+    if (!aligned16(x) || !aligned16(cond) || !aligned16(kv_cache) || !aligned16(y))
+        return c->fail(FD_ERR_INVALID_ARG, "x, cond, kv_cache, y must be 16-byte aligned");
+    if (B < 1 || N < 1 || R < 1) return c->fail(FD_ERR_SHAPE, "B, N, R must be positive");
+    if (B > c->cfg.max_batch || N > c->cfg.max_tokens || R > c->cfg.max_regions)
+        return c->fail(FD_ERR_SHAPE, "B=%d N=%d R=%d exceed the limits %d/%d/%d", B, N, R, c->cfg.max_batch,
+                       c->cfg.max_tokens, c->cfg.max_regions);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (c->cfg.dtype == FD_BF16)
+        return run_step<__nv_bfloat16>(c, x, cond, labels, mask, B, N, R, kv_cache, y, active_idx_out, cu_active_out, st);
+    return run_step<float>(c, x, cond, labels, mask, B, N, R, kv_cache, y, active_idx_out, cu_active_out, st);
+}
+
+fd_status fd_poll_status(fd_ctx* c, void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    Control h{};
+    cudaError_t e = cudaMemcpyAsync(&h, c->ctl(), sizeof(Control), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "status read failed: %s", cudaGetErrorString(e));
+    if (h.status != 0) {
+        cudaMemsetAsync(c->ctl(), 0, 2 * sizeof(int32_t), st);
+        return c->fail(static_cast<fd_status>(h.status), "device-side check failed: code %d, detail %d", h.status,
+                       h.detail);
+    }
+    return FD_OK;
+}
+
+int64_t fd_launch_count(const fd_ctx* c) { return c ? c->launches : 0; }
+
+fd_status fd_destroy(fd_ctx* c) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    tc_plan_destroy(c->tc);
+    delete c;
+    return FD_OK;
+}
+
+const char* fd_last_error(const fd_ctx* c) { return c ? c->err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

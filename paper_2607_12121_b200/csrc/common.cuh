@@ -1,0 +1,129 @@
+// Shared declarations of the libflashdiff kernels (device helpers, workspace layout, launch
+// prototypes).  Everything here is internal to the library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/flashdiff.h"
+
+namespace fd {
+
+// ---------------------------------------------------------------------------------------------
+// device-side status: word 0 = first error code (fd_status), word 1 = detail
+// ---------------------------------------------------------------------------------------------
+struct Control {
+    int32_t status;        // first device-side error, 0 = none
+    int32_t detail;
+    int32_t a_total;       // number of active rows of the current step
+    int32_t n_qtiles;      // number of attention query tiles of the current step
+    int32_t pad[12];
+};
+
+__device__ __forceinline__ void report(Control* c, int code, int detail) {
+    if (atomicCAS(&c->status, 0, code) == 0) c->detail = detail;
+}
+
+struct QTile {            // one attention work item: `rows` compact rows of one request
+    int32_t b, row0, rows, pad;
+};
+
+// ---------------------------------------------------------------------------------------------
+// storage-type helpers
+// ---------------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float gelu_tanh(float a) {
+    const float c = 0.7978845608028654f;
+    float u = c * (a + 0.044715f * a * a * a);
+    return 0.5f * a * (1.0f + tanhf(u));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// GEMM epilogues (shared by the CUDA-core and the tensor-core kernels)
+// ---------------------------------------------------------------------------------------------
+enum EpiKind { EPI_QKV = 0, EPI_RESID = 1, EPI_GELU = 2 };
+
+struct EpiParams {
+    const void* bias;          // [n_out] storage type
+    const int32_t* active_idx; // [A] global token id of each compact row
+    int32_t N;                 // tokens per request
+    int32_t H;                 // hidden width
+    // EPI_QKV
+    void* q;                   // [Mcap, q_ld] storage type
+    int32_t q_ld;
+    void* kv;                  // this block's cache [B,2,N,H] storage type
+    // EPI_RESID
+    float* resid;              // [Mcap,H] fp32, in/out
+    const float* gate;         // mod + chunk offset; row stride 6H per request
+    void* y;                   // [B*N,H] storage type or nullptr (only the last block scatters)
+    // EPI_GELU
+    void* out;                 // [Mcap,n_out] storage type
+    int32_t out_ld;
+};
+
+// ---------------------------------------------------------------------------------------------
+// host-side launchers (one per .cu file)
+// ---------------------------------------------------------------------------------------------
+struct Shape {
+    int L, H, heads, dh, M, Hc;
+    int B, N, R;
+    int Mcap;        // capacity (rows) of the compact buffers
+    float ln_eps;
+};
+
+// activity.cu
+cudaError_t launch_activity(const float* z_cur, const float* z_prev, const int32_t* labels, int B, int N,
+                            int D, int R, const float* eps, float* delta, int32_t* skip_count,
+                            uint8_t* prev_active, float* score, float* weight, uint8_t* mask, float eta,
+                            int K, double* acc_ss, int32_t* acc_cnt, Control* ctl, cudaStream_t st,
+                            int* n_launch);
+
+// compact.cu
+cudaError_t launch_compact(const uint8_t* mask, const int32_t* labels, int B, int N, int R,
+                           int32_t* active_idx, int32_t* cu_active, int32_t* block_counts, QTile* tiles,
+                           int tile_rows, Control* ctl, cudaStream_t st, int* n_launch);
+
+// rowops.cu
+template <typename T>
+cudaError_t launch_adaln(const T* cond, const T* w_ada, const T* b_ada, float* mod, int L, int B, int H,
+                         int Hc, cudaStream_t st, int* n_launch);
+template <typename T>
+cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
+                               const int32_t* active_idx, const float* shift, const float* scale,
+                               int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
+                               cudaStream_t st, int* n_launch);
+
+// simt_block.cu
+template <typename T>
+cudaError_t launch_simt_gemm(int kind, const T* a, int lda, const T* w, int n_out, int k, int rows_cap,
+                             const EpiParams& ep, const Control* ctl, cudaStream_t st, int* n_launch);
+template <typename T>
+cudaError_t launch_simt_attention(const T* q, int q_ld, const T* kv, T* o, int o_ld, const QTile* tiles,
+                                  int max_tiles, int N, int H, int heads, int dh, const Control* ctl,
+                                  cudaStream_t st, int* n_launch);
+
+// partition.cu
+size_t partition_scratch_bytes(int max_batch, int max_tokens, int max_regions);
+cudaError_t launch_partition(const float* attn_map, int B, int N, int T, const int32_t* salient_cols,
+                             int T_s, int R, int m_min, int m_max, int32_t* labels, int32_t* sizes,
+                             void* scratch, Control* ctl, cudaStream_t st, int* n_launch);
+
+}  // namespace fd

@@ -1,0 +1,253 @@
+// Row-wise, memory-bound pieces of the block: the adaLN conditioning vectors and the
+// gather + LayerNorm + modulation that feeds the QKV and MLP projections.  The block is the
+// adaLN-Zero DiT block the paper builds on (Sec. 2.1); only active rows are touched (Sec. 3).
+#include "common.cuh"
+
+namespace fd {
+
+namespace {
+
+// ---- 16-byte vector access to a row of storage type T, as floats -----------------------------
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+    static constexpr int N = 4;
+    __device__ static void load(const float* p, float* f) {
+        const float4 v = *reinterpret_cast<const float4*>(p);
+        f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+    }
+    __device__ static void store(float* p, const float* f) {
+        *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+    }
+};
+template <> struct Vec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    __device__ static void load(const __nv_bfloat16* p, float* f) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    __device__ static void store(__nv_bfloat16* p, const float* f) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// ---- adaLN: mod[l,b,o] = sum_c SiLU(cond[b,c]) W_ada[l,o,c] + b_ada[l,o] ----------------------
+constexpr int ADA_THREADS = 256;
+constexpr int ADA_BCH = 8;         // requests handled per pass over a weight row
+constexpr int ADA_ROWS = 32;       // weight rows per CTA
+
+template <typename T>
+__global__ void __launch_bounds__(ADA_THREADS)
+adaln_kernel(const T* __restrict__ cond, const T* __restrict__ w_ada, const T* __restrict__ b_ada,
+             float* __restrict__ mod, int L, int B, int H6, int Hc) {
+    extern __shared__ float s_act[];            // [min(B,ADA_BCH)][Hc]
+    constexpr int VN = Vec<T>::N;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long rows_total = (long long)L * H6;
+    for (int b0 = 0; b0 < B; b0 += ADA_BCH) {
+        const int nb = min(ADA_BCH, B - b0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < nb * Hc; i += ADA_THREADS) {
+            const float v = to_f<T>(cond[(size_t)(b0 + i / Hc) * Hc + (i % Hc)]);
+            s_act[i] = v / (1.0f + __expf(-v));
+        }
+        __syncthreads();
+        for (int r = warp; r < ADA_ROWS; r += ADA_THREADS / 32) {
+            const long long row = (long long)blockIdx.x * ADA_ROWS + r;
+            if (row >= rows_total) break;
+            const T* wr = w_ada + (size_t)row * Hc;
+            float acc[ADA_BCH];
+#pragma unroll
+            for (int b = 0; b < ADA_BCH; ++b) acc[b] = 0.f;
+            for (int c = lane * VN; c < Hc; c += 32 * VN) {
+                float w[VN];
+                Vec<T>::load(wr + c, w);
+#pragma unroll
+                for (int b = 0; b < ADA_BCH; ++b) {
+                    if (b < nb) {
+                        const float* a = s_act + b * Hc + c;
+#pragma unroll
+                        for (int k = 0; k < VN; ++k) acc[b] = fmaf(w[k], a[k], acc[b]);
+                    }
+                }
+            }
+            const int l = (int)(row / H6), o = (int)(row % H6);
+            const float bias = to_f<T>(b_ada[row]);
+#pragma unroll
+            for (int b = 0; b < ADA_BCH; ++b) {
+                if (b < nb) {
+                    const float v = warp_sum(acc[b]);
+                    if (lane == 0) mod[((size_t)l * B + (b0 + b)) * H6 + o] = v + bias;
+                }
+            }
+        }
+    }
+}
+
+// ---- gather + LayerNorm + modulation, one warp per active row --------------------------------
+constexpr int LN_THREADS = 256;
+constexpr int LN_MAXV = 16;        // float4 slots per lane: rows up to 32*4*16 = 2048 wide stay in registers
+
+template <typename T>
+__global__ void __launch_bounds__(LN_THREADS)
+ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
+                   float* __restrict__ resid_out, T* __restrict__ out, const int32_t* __restrict__ active_idx,
+                   const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
+                   int H, float ln_eps, const Control* __restrict__ ctl) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int a_total = ctl->a_total;
+    const int nv = H / 128;                       // float4 slots per lane (H % 128 == 0 on this path)
+    for (int row = blockIdx.x * (LN_THREADS / 32) + warp; row < a_total; row += gridDim.x * (LN_THREADS / 32)) {
+        const int tok = active_idx[row];
+        const int b = tok / N;
+        float v[LN_MAXV][4];
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < LN_MAXV; ++i) {
+            if (i < nv) {
+                const int c = (i * 32 + lane) * 4;
+                if (x_gather) {
+                    const T* src = x_gather + (size_t)tok * H + c;
+                    if constexpr (sizeof(T) == 2) {
+                        const uint2 u = *reinterpret_cast<const uint2*>(src);
+                        v[i][0] = __uint_as_float(u.x << 16); v[i][1] = __uint_as_float(u.x & 0xffff0000u);
+                        v[i][2] = __uint_as_float(u.y << 16); v[i][3] = __uint_as_float(u.y & 0xffff0000u);
+                    } else {
+                        const float4 u = *reinterpret_cast<const float4*>(src);
+                        v[i][0] = u.x; v[i][1] = u.y; v[i][2] = u.z; v[i][3] = u.w;
+                    }
+                    if (resid_out)
+                        *reinterpret_cast<float4*>(resid_out + (size_t)row * H + c) =
+                            make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
+                } else {
+                    const float4 u = *reinterpret_cast<const float4*>(resid_in + (size_t)row * H + c);
+                    v[i][0] = u.x; v[i][1] = u.y; v[i][2] = u.z; v[i][3] = u.w;
+                }
+                sum += (v[i][0] + v[i][1]) + (v[i][2] + v[i][3]);
+            }
+        }
+        const float mean = warp_sum(sum) / (float)H;
+        float sq = 0.f;
+#pragma unroll
+        for (int i = 0; i < LN_MAXV; ++i) {
+            if (i < nv) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { const float d = v[i][k] - mean; sq = fmaf(d, d, sq); }
+            }
+        }
+        const float rstd = rsqrtf(warp_sum(sq) / (float)H + ln_eps);
+        const float* sh = shift + (size_t)b * mod_stride;
+        const float* sc = scale + (size_t)b * mod_stride;
+#pragma unroll
+        for (int i = 0; i < LN_MAXV; ++i) {
+            if (i < nv) {
+                const int c = (i * 32 + lane) * 4;
+                const float4 s4 = *reinterpret_cast<const float4*>(sc + c);
+                const float4 h4 = *reinterpret_cast<const float4*>(sh + c);
+                const float o0 = (v[i][0] - mean) * rstd * (1.f + s4.x) + h4.x;
+                const float o1 = (v[i][1] - mean) * rstd * (1.f + s4.y) + h4.y;
+                const float o2 = (v[i][2] - mean) * rstd * (1.f + s4.z) + h4.z;
+                const float o3 = (v[i][3] - mean) * rstd * (1.f + s4.w) + h4.w;
+                T* dst = out + (size_t)row * H + c;
+                if constexpr (sizeof(T) == 2) {
+                    const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
+                    uint2 u;
+                    u.x = *reinterpret_cast<const uint32_t*>(&p0);
+                    u.y = *reinterpret_cast<const uint32_t*>(&p1);
+                    *reinterpret_cast<uint2*>(dst) = u;
+                } else {
+                    *reinterpret_cast<float4*>(dst) = make_float4(o0, o1, o2, o3);
+                }
+            }
+        }
+    }
+}
+
+// Any width: three passes over the row (the re-reads hit L1/L2).
+template <typename T>
+__global__ void __launch_bounds__(LN_THREADS)
+ln_modulate_generic_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
+                           float* __restrict__ resid_out, T* __restrict__ out,
+                           const int32_t* __restrict__ active_idx, const float* __restrict__ shift,
+                           const float* __restrict__ scale, int mod_stride, int N, int H, float ln_eps,
+                           const Control* __restrict__ ctl) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int a_total = ctl->a_total;
+    for (int row = blockIdx.x * (LN_THREADS / 32) + warp; row < a_total; row += gridDim.x * (LN_THREADS / 32)) {
+        const int tok = active_idx[row];
+        const int b = tok / N;
+        auto at = [&](int c) -> float {
+            return x_gather ? to_f<T>(x_gather[(size_t)tok * H + c]) : resid_in[(size_t)row * H + c];
+        };
+        float sum = 0.f;
+        for (int c = lane; c < H; c += 32) sum += at(c);
+        const float mean = warp_sum(sum) / (float)H;
+        float sq = 0.f;
+        for (int c = lane; c < H; c += 32) { const float d = at(c) - mean; sq = fmaf(d, d, sq); }
+        const float rstd = rsqrtf(warp_sum(sq) / (float)H + ln_eps);
+        const float* sh = shift + (size_t)b * mod_stride;
+        const float* sc = scale + (size_t)b * mod_stride;
+        for (int c = lane; c < H; c += 32) {
+            const float u = at(c);
+            if (x_gather && resid_out) resid_out[(size_t)row * H + c] = u;
+            out[(size_t)row * H + c] = from_f<T>((u - mean) * rstd * (1.f + sc[c]) + sh[c]);
+        }
+    }
+}
+
+}  // namespace
+
+template <typename T>
+cudaError_t launch_adaln(const T* cond, const T* w_ada, const T* b_ada, float* mod, int L, int B, int H,
+                         int Hc, cudaStream_t st, int* n_launch) {
+    const long long rows = (long long)L * 6 * H;
+    const int grid = (int)((rows + ADA_ROWS - 1) / ADA_ROWS);
+    const size_t smem = (size_t)min(B, ADA_BCH) * Hc * sizeof(float);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(adaln_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    adaln_kernel<T><<<grid, ADA_THREADS, smem, st>>>(cond, w_ada, b_ada, mod, L, B, 6 * H, Hc);
+    ++*n_launch;
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
+                               const int32_t* active_idx, const float* shift, const float* scale,
+                               int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
+                               cudaStream_t st, int* n_launch) {
+    const int rows_per_cta = LN_THREADS / 32;
+    const int grid = max(1, min((rows_cap + rows_per_cta - 1) / rows_per_cta, 148 * 8));
+    if (H % 128 == 0 && H <= 128 * LN_MAXV)
+        ln_modulate_kernel<T><<<grid, LN_THREADS, 0, st>>>(x_gather, resid_in, resid_out, out, active_idx, shift,
+                                                          scale, mod_stride, N, H, ln_eps, ctl);
+    else
+        ln_modulate_generic_kernel<T><<<grid, LN_THREADS, 0, st>>>(x_gather, resid_in, resid_out, out, active_idx,
+                                                                  shift, scale, mod_stride, N, H, ln_eps, ctl);
+    ++*n_launch;
+    return cudaGetLastError();
+}
+
+template cudaError_t launch_adaln<float>(const float*, const float*, const float*, float*, int, int, int, int,
+                                         cudaStream_t, int*);
+template cudaError_t launch_adaln<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*,
+                                                 float*, int, int, int, int, cudaStream_t, int*);
+template cudaError_t launch_ln_modulate<float>(const float*, const float*, float*, float*, const int32_t*,
+                                               const float*, const float*, int, int, int, int, float, const Control*,
+                                               cudaStream_t, int*);
+template cudaError_t launch_ln_modulate<__nv_bfloat16>(const __nv_bfloat16*, const float*, float*, __nv_bfloat16*,
+                                                       const int32_t*, const float*, const float*, int, int, int, int,
+                                                       float, const Control*, cudaStream_t, int*);
+
+}  // namespace fd

@@ -1,0 +1,125 @@
+"""GPU parity: gate (scores 1e-5 relative, mask bit-exact) and compaction (bit-exact)."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+import paper_2607_12121_b200 as fd
+from harness import dev, host, make_ctx, labels_for
+
+pytestmark = pytest.mark.gpu
+
+
+def _ctx(wl):
+    w = gen.block_weights(wl, 1, n_blocks=1)
+    return make_ctx(wl, w, n_blocks=1, engine=fd.FD_ENGINE_SIMT)
+
+
+class GateState:
+    def __init__(self, B, R):
+        self.delta = torch.zeros((B, R), dtype=torch.float32, device="cuda")
+        self.skip = torch.zeros((B, R), dtype=torch.int32, device="cuda")
+        self.prev = torch.ones((B, R), dtype=torch.uint8, device="cuda")
+        self.score = torch.empty((B, R), dtype=torch.float32, device="cuda")
+        self.weight = torch.empty((B, R), dtype=torch.float32, device="cuda")
+        self.mask = torch.empty((B, R), dtype=torch.uint8, device="cuda")
+
+
+def _gate(ctx, wl, z_cur, z_prev, labels, eps, st):
+    fd.fd_region_activity(ctx, z_cur, z_prev, labels, wl.R, eps, st.delta, st.skip, st.prev, st.score, st.weight,
+                          st.mask)
+    fd.fd_poll_status(ctx)
+    return host(st.score), host(st.weight), host(st.mask)
+
+
+@pytest.mark.parametrize("name,seed", [("tiny", 0), ("audio_small", 1), ("image_small", 2), ("mmdit_small", 3),
+                                       ("video_small", 4)])
+def test_gate_single_step(name, seed):
+    wl = gen.workload(name)
+    labels = labels_for(wl, seed)
+    if name == "tiny":
+        lat = gen.latent_pair(wl, seed, labels, eps_fixed=1e-2)
+    else:
+        lat = gen.latent_pair(wl, seed, labels, fractions=gen.request_fractions(wl, seed))
+    ost = oracle.initial_state(wl.B, wl.R)
+    o_score, o_weight, o_mask = oracle.activity_gate(lat["z_cur"], lat["z_prev"], labels, lat["eps"], ost, wl.R)
+    assert np.abs(o_weight / np.maximum(lat["eps"][:, None], 1e-30) - 1).min() >= 1e-3
+    ctx = _ctx(wl)
+    st = GateState(wl.B, wl.R)
+    score, weight, mask = _gate(ctx, wl, dev(lat["z_cur"]), dev(lat["z_prev"]), dev(labels), dev(lat["eps"]), st)
+    assert np.array_equal(mask, o_mask)
+    np.testing.assert_allclose(score, o_score, rtol=1e-5, atol=0)
+    np.testing.assert_allclose(weight, o_weight, rtol=1e-5, atol=0)
+    assert np.array_equal(host(st.prev), ost["prev_active"])
+    assert np.array_equal(host(st.skip), ost["skip_count"])
+
+
+def test_gate_multi_step_state_and_forced_reactivation():
+    wl = gen.workload("audio_small")
+    labels = gen.uniform_labels(wl)
+    lat = gen.latent_pair(wl, 7, labels, fractions=[0.25, 0.5, 0.75])
+    ctx = make_ctx(wl, gen.block_weights(wl, 1, n_blocks=1), n_blocks=1, engine=fd.FD_ENGINE_SIMT, max_skip_k=3)
+    st = GateState(wl.B, wl.R)
+    ost = oracle.initial_state(wl.B, wl.R)
+    rng = np.random.default_rng(0)
+    z_prev, z_cur = lat["z_prev"], lat["z_cur"]
+    step_delta = lat["z_cur"] - lat["z_prev"]
+    forced = False
+    for step in range(9):
+        o_score, o_weight, o_mask = oracle.activity_gate(z_cur, z_prev, labels, lat["eps"], ost, wl.R, K=3)
+        score, weight, mask = _gate(ctx, wl, dev(z_cur), dev(z_prev), dev(labels), dev(lat["eps"]), st)
+        assert np.array_equal(mask, o_mask), step
+        np.testing.assert_allclose(score, o_score, rtol=1e-5)
+        np.testing.assert_allclose(weight, o_weight, rtol=1e-5)
+        assert np.array_equal(host(st.skip), ost["skip_count"])
+        forced |= bool((o_mask.astype(bool) & (o_weight < lat["eps"][:, None])).any())
+        z_prev = z_cur
+        z_cur = (z_cur + step_delta * np.float32(rng.uniform(0.95, 1.05))).astype(np.float32)
+    assert forced
+
+
+def test_gate_odd_channel_count_uses_scalar_path():
+    wl = gen.workload("audio_small").replace(D=6)
+    labels = gen.uniform_labels(wl)
+    lat = gen.latent_pair(wl, 9, labels, fractions=[0.5, 0.5, 0.5])
+    ost = oracle.initial_state(wl.B, wl.R)
+    o_score, o_weight, o_mask = oracle.activity_gate(lat["z_cur"], lat["z_prev"], labels, lat["eps"], ost, wl.R)
+    ctx = _ctx(wl)
+    st = GateState(wl.B, wl.R)
+    score, weight, mask = _gate(ctx, wl, dev(lat["z_cur"]), dev(lat["z_prev"]), dev(labels), dev(lat["eps"]), st)
+    assert np.array_equal(mask, o_mask)
+    np.testing.assert_allclose(score, o_score, rtol=1e-5)
+
+
+@pytest.mark.parametrize("name", ["tiny", "audio_small", "mmdit_small", "video_small"])
+def test_compaction_bit_exact(name):
+    from harness import StepBuffers, gpu_step
+    wl = gen.workload(name)
+    labels = labels_for(wl, 5)
+    w = gen.block_weights(wl, 1, n_blocks=1)
+    ctx = make_ctx(wl, w, n_blocks=1, engine=fd.FD_ENGINE_SIMT)
+    inp = gen.step_inputs(wl, 5, labels)
+    buf = StepBuffers(wl, 1)
+    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    for fr in ([1.0] * wl.B, [0.5] * wl.B, [0.0] * wl.B, list(gen.request_fractions(wl, 3))):
+        mask = gen.region_mask(wl, 11, fr)
+        idx, cu = gpu_step(ctx, wl, dev(inp["x_cur"], dt), dev(inp["cond"], dt), dev(labels), dev(mask), buf)
+        o_idx, o_cu = oracle.compact(mask, labels, wl.R)
+        assert np.array_equal(cu, o_cu)
+        assert np.array_equal(idx, o_idx)
+
+
+def test_bad_label_is_reported_not_trapped():
+    wl = gen.workload("audio_small")
+    labels = gen.uniform_labels(wl).copy()
+    labels[1, 7] = wl.R + 3
+    lat = gen.latent_pair(wl, 1, gen.uniform_labels(wl), fractions=[0.5] * wl.B)
+    ctx = _ctx(wl)
+    st = GateState(wl.B, wl.R)
+    fd.fd_region_activity(ctx, dev(lat["z_cur"]), dev(lat["z_prev"]), dev(labels), wl.R, dev(lat["eps"]), st.delta,
+                          st.skip, st.prev, st.score, st.weight, st.mask)
+    with pytest.raises(fd.FlashDiffError) as ei:
+        fd.fd_poll_status(ctx)
+    assert ei.value.status == fd.FD_ERR_STATE
+    fd.fd_poll_status(ctx)          # cleared; the context stays usable

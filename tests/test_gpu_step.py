@@ -1,0 +1,126 @@
+"""GPU parity of the regional step against the oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+import paper_2607_12121_b200 as fd
+from harness import StepBuffers, dev, gpu_step, host, labels_for, make_ctx, max_abs, rel_l2, tdtype
+
+pytestmark = pytest.mark.gpu
+
+BF16_MAX_ABS, BF16_REL_L2 = 3e-2, 1e-2      # bf16 block outputs vs the fp32 oracle
+F32_MAX_ABS, F32_REL_L2 = 1e-4, 1e-5        # fp32 CUDA-core path vs the oracle
+
+
+def _tol(wl):
+    return (BF16_MAX_ABS, BF16_REL_L2) if wl.dtype == "bf16" else (F32_MAX_ABS, F32_REL_L2)
+
+
+def _check_step(wl, y, kv, y_ref, kv_ref, y_before, kv_before, idx):
+    """Active rows within tolerance; every other row of y and kv bit-identical to before."""
+    B, N, H = wl.B, wl.N, wl.H
+    ma, rl = _tol(wl)
+    act = np.zeros(B * N, bool)
+    act[idx] = True
+    yf, yr = y.reshape(B * N, H), y_ref.reshape(B * N, H)
+    assert max_abs(yf[act], yr[act]) <= ma
+    assert rel_l2(yf[act], yr[act]) <= rl
+    assert np.array_equal(yf[~act], y_before.reshape(B * N, H)[~act])
+    L = kv.shape[0]
+    a2 = act.reshape(B, N)
+    for l in range(L):
+        for s in range(2):
+            got, ref, old = kv[l][:, s], kv_ref[l][:, s], kv_before[l][:, s]
+            assert max_abs(got[a2], ref[a2]) <= ma
+            assert rel_l2(got[a2], ref[a2]) <= rl
+            assert np.array_equal(got[~a2], old[~a2])
+
+
+def _run_sequence(wl, seed, engine, masks, n_blocks=None):
+    """Warm-up (all active) on the previous step's tokens, then gated steps; both sides start
+    from the same zero caches and carry their own state forward."""
+    L = wl.L if n_blocks is None else n_blocks
+    labels = labels_for(wl, seed)
+    w = gen.block_weights(wl, seed, n_blocks=L)
+    inp = gen.step_inputs(wl, seed, labels)
+    ctx = make_ctx(wl, w, engine=engine, n_blocks=L)
+    buf = StepBuffers(wl, L)
+    dt = tdtype(wl)
+    B, N, H = wl.B, wl.N, wl.H
+    kv_ref = np.zeros((L, B, 2, N, H), np.float32)
+    y_ref = np.zeros((B, N, H), np.float32)
+    rng = np.random.default_rng(seed)
+    x_np = inp["x_prev"]
+    for step, mask in enumerate(masks):
+        if step == 1:
+            x_np = inp["x_cur"]
+        elif step > 1:
+            x_np = (x_np + np.float32(0.01) * rng.standard_normal(x_np.shape).astype(np.float32))
+            x_np = gen.round_bf16(x_np) if wl.dtype == "bf16" else x_np.astype(np.float32)
+        y_before, kv_before = host(buf.y), host(buf.kv)
+        idx, cu = gpu_step(ctx, wl, dev(x_np, dt), dev(inp["cond"], dt), dev(labels), dev(mask), buf)
+        o_idx, o_cu = oracle.regional_step(x_np, inp["cond"], labels, mask, w, kv_ref, y_ref, wl.heads, wl.R,
+                                           n_blocks=L)
+        assert np.array_equal(idx, o_idx) and np.array_equal(cu, o_cu)
+        _check_step(wl, host(buf.y), host(buf.kv), y_ref, kv_ref, y_before, kv_before, idx)
+    return ctx
+
+
+def test_tiny_fp32_eight_steps_fixed_schedule():
+    wl = gen.workload("tiny")
+    masks = gen.mask_schedule(wl, 0, 8)
+    _run_sequence(wl, 0, fd.FD_ENGINE_SIMT, masks)
+
+
+@pytest.mark.parametrize("name", ["audio_small", "image_small", "mmdit_small", "video_small"])
+def test_small_twins_simt_engine(name):
+    wl = gen.workload(name)
+    masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 3, gen.request_fractions(wl, 3)),
+             gen.region_mask(wl, 4, [0.34] * wl.B)]
+    _run_sequence(wl, 2, fd.FD_ENGINE_SIMT, masks)
+
+
+def test_all_active_step_equals_dense_oracle():
+    wl = gen.workload("audio_small")
+    labels = gen.uniform_labels(wl)
+    w = gen.block_weights(wl, 6)
+    inp = gen.step_inputs(wl, 6, labels)
+    ctx = make_ctx(wl, w, engine=fd.FD_ENGINE_SIMT)
+    buf = StepBuffers(wl, wl.L)
+    dt = tdtype(wl)
+    gpu_step(ctx, wl, dev(inp["x_cur"], dt), dev(inp["cond"], dt), dev(labels), dev(np.ones((wl.B, wl.R), np.uint8)), buf)
+    y_d, kv_d = oracle.dense_step(inp["x_cur"], inp["cond"], w, wl.heads)
+    assert max_abs(host(buf.y), y_d) <= BF16_MAX_ABS and rel_l2(host(buf.y), y_d) <= BF16_REL_L2
+    assert max_abs(host(buf.kv), kv_d) <= BF16_MAX_ABS and rel_l2(host(buf.kv), kv_d) <= BF16_REL_L2
+
+
+def test_empty_mask_touches_nothing():
+    wl = gen.workload("audio_small")
+    labels = gen.uniform_labels(wl)
+    w = gen.block_weights(wl, 8)
+    inp = gen.step_inputs(wl, 8, labels)
+    ctx = make_ctx(wl, w, engine=fd.FD_ENGINE_SIMT)
+    buf = StepBuffers(wl, wl.L)
+    buf.y.fill_(1.5)
+    buf.kv.fill_(-2.0)
+    dt = tdtype(wl)
+    idx, cu = gpu_step(ctx, wl, dev(inp["x_cur"], dt), dev(inp["cond"], dt), dev(labels),
+                       dev(np.zeros((wl.B, wl.R), np.uint8)), buf)
+    assert idx.size == 0 and not cu.any()
+    assert (host(buf.y) == 1.5).all() and (host(buf.kv) == -2.0).all()
+
+
+def test_host_side_argument_errors():
+    wl = gen.workload("audio_small")
+    w = gen.block_weights(wl, 1, n_blocks=1)
+    ctx = make_ctx(wl, w, n_blocks=1, engine=fd.FD_ENGINE_SIMT)
+    buf = StepBuffers(wl, 1)
+    dt = tdtype(wl)
+    x = torch.zeros((wl.B + 1, wl.N, wl.H), dtype=dt, device="cuda")
+    with pytest.raises(fd.FlashDiffError) as ei:
+        fd.fd_regional_step(ctx, x, x, x, x, wl.R, buf.kv, buf.y, buf.active_idx, buf.cu_active)
+    assert ei.value.status == fd.FD_ERR_SHAPE
+    bad = fd.make_config(wl.replace(H=250))
+    assert fd.fd_workspace_bytes(bad) == 0
