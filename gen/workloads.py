@@ -78,6 +78,21 @@ WORKLOADS["video_small"] = WORKLOADS["video"].replace(
     n_cells=12, m_min=8, m_max=128, D=16)
 
 
+# twins whose widths fit the tensor-core tiles (multiples of 128)
+WORKLOADS["audio_tc"] = WORKLOADS["audio"].replace(
+    name="audio_tc", L=2, H=256, heads=4, M=512, Hc=256, grid=(416,), B=3, R=26, D=16)
+WORKLOADS["mmdit_tc"] = WORKLOADS["mmdit"].replace(
+    name="mmdit_tc", L=2, H=384, heads=6, M=768, Hc=384, grid=(16, 20), n_text=27, B=2, R=16,
+    n_cells=16, m_min=8, m_max=64, D=16)
+WORKLOADS["video_tc"] = WORKLOADS["video"].replace(
+    name="video_tc", L=2, H=256, heads=2, M=640, Hc=256, grid=(6, 10, 14), B=1, R=24,
+    n_cells=12, m_min=8, m_max=128, D=16)
+WORKLOADS["image_tc"] = WORKLOADS["image"].replace(
+    name="image_tc", L=1, grid=(12, 16), B=2, R=12, n_cells=12, m_min=8, m_max=32)
+WORKLOADS["wide_tc"] = WORKLOADS["audio"].replace(
+    name="wide_tc", L=1, H=1024, heads=8, head_dim=128, M=3072, Hc=256, grid=(208,), B=2, R=13, D=16)
+
+
 def workload(name: str) -> Workload:
     return WORKLOADS[name]
 

@@ -79,7 +79,8 @@ struct fd_ctx {
     fd_weights w;
     Layout lay;
     char* ws;
-    bool use_tc;
+    bool use_tc;         // tensor-core GEMMs
+    bool use_tc_attn;    // tensor-core attention
     int tile_rows;
     int64_t launches;
     std::string err;
@@ -162,7 +163,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         else
             FD_TRY(launch_simt_gemm<T>(EPI_QKV, act, H, w_qkv, 3 * H, H, rows_cap, ep, ctl, st, &nl));
         // active queries against all N keys of their request
-        if (c->use_tc)
+        if (c->use_tc_attn)
             FD_TRY(tc_attention(c->tc, blk, kv_b, B, N, tiles, max_tiles, ctl, st, &nl));
         else
             FD_TRY(launch_simt_attention<T>(q, l.q_ld, kv_b, o, H, tiles, max_tiles, N, H, cf.n_heads, cf.head_dim,
@@ -247,7 +248,8 @@ fd_status fd_create(const fd_config* cfg, const fd_weights* weights, void* works
     c->lay = lay;
     c->ws = static_cast<char*>(workspace);
     c->use_tc = use_tc;
-    c->tile_rows = use_tc ? tc_attention_tile_rows() : simt_attention_tile_rows();
+    c->use_tc_attn = use_tc && tc_attention_supported(*cfg);
+    c->tile_rows = c->use_tc_attn ? tc_attention_tile_rows() : simt_attention_tile_rows();
     c->launches = 0;
     c->tc = nullptr;
     // control block and gate accumulators start at zero; the compact buffers start finite

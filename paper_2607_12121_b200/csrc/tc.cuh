@@ -1,5 +1,7 @@
 // Interface of the tensor-core engine (tcgen05 + TMEM + TMA kernels for the dense contractions).
 #pragma once
+#include <cuda.h>
+
 #include <string>
 
 #include "common.cuh"
@@ -16,6 +18,7 @@ struct TcBuffers {  // compact activation buffers inside the workspace (bf16)
 enum TcGemmKind { TC_GEMM_QKV = 0, TC_GEMM_OUT = 1, TC_GEMM_FC1 = 2, TC_GEMM_FC2 = 3 };
 
 bool tc_supported(const fd_config& cfg, std::string* why);
+bool tc_attention_supported(const fd_config& cfg);
 int tc_attention_tile_rows();
 TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffers& buf, std::string* err);
 void tc_plan_destroy(TcPlan* p);
@@ -23,5 +26,10 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
                     int* n_launch);
 cudaError_t tc_attention(TcPlan* p, int blk, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch);
+
+// host helper shared by the GEMM and attention plans: encodes a tiled bf16 tensor map
+// (rank <= 4; dims / strides innermost first; strides in bytes for dims 1..rank-1)
+bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                      const uint32_t* box, int swizzle_bytes, std::string* err);
 
 }  // namespace fd

@@ -1,0 +1,320 @@
+// Tensor-core GEMM for the dense contractions of the block on compacted tokens:
+//   C[row, n] = sum_k A[row, k] W[n, k]      A: compact activations [rows, K], W: weights [n_out, K]
+// both bf16 with K contiguous.  Persistent, warp-specialised kernel:
+//   warp 0      TMA producer: 128 x 64 activation tile and BN x 64 weight tile per stage, 128-byte swizzle
+//   warp 1      issues tcgen05.mma (M = 128, N = BN, K = 16) into a TMEM accumulator, two accumulator
+//               stages so the next tile's MMAs overlap this tile's epilogue
+//   warps 2..5  epilogue: tcgen05.ld of the fp32 accumulator (one row per thread), bias / GELU /
+//               gated residual / K-V scatter, 128-bit global stores
+// The number of active rows lives on the device; CTAs derive the tile count from it, so the host
+// never synchronises.  Rows of the last tile beyond the active count are computed and dropped.
+#include <cstdlib>
+
+#include "epilogue.cuh"
+#include "ptx.cuh"
+#include "tc.cuh"
+
+namespace fd {
+
+using namespace ptx;
+
+namespace {
+
+constexpr int BM = 128, BK = 64;
+constexpr int GEMM_THREADS = 192;
+constexpr int A_TILE_BYTES = BM * BK * 2;
+
+template <int BN> struct GemmCfg {
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int B_TILE_BYTES = BN * BK * 2;
+    static constexpr int SMEM = STAGES * (A_TILE_BYTES + B_TILE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int KIND, int BN>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int n_out,
+               int k_dim, EpiParams ep, Control* ctl) {
+    using Cfg = GemmCfg<BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    constexpr int B_TILE_BYTES = Cfg::B_TILE_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + STAGES * A_TILE_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * (A_TILE_BYTES + B_TILE_BYTES));
+    uint64_t* empty = full + STAGES;
+    uint64_t* tfull = empty + STAGES;
+    uint64_t* tempty = tfull + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int a_total = ctl->a_total;
+    const int m_tiles = (a_total + BM - 1) / BM;
+    const int n_tiles = n_out / BN;
+    const int total_tiles = m_tiles * n_tiles;
+    const int k_tiles = k_dim / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 4); }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tm_a);
+        prefetch_tmap(&tm_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, 2 * BN);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m = tile % m_tiles, n = tile / m_tiles;
+                for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+                    mbar_expect_tx(&full[s], A_TILE_BYTES + B_TILE_BYTES);
+                    tma_load_2d(sA + s * A_TILE_BYTES, &tm_a, kt * BK, m * BM, &full[s]);
+                    tma_load_2d(sB + s * B_TILE_BYTES, &tm_b, kt * BK, n * BN, &full[s]);
+                }
+            }
+            if (!ok) report(ctl, FD_ERR_TIMEOUT, 100 + (int)blockIdx.x);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(BM, BN, 0, 0);
+            uint32_t it = 0, t_it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t_it) {
+                const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
+                if (!mbar_wait(&tempty[acc], aph ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d = tmem_base + acc * BN;
+                for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t da = smem_desc(smem_u32(sA + s * A_TILE_BYTES), 16, 1024, SWZ_128B);
+                    const uint64_t db = smem_desc(smem_u32(sB + s * B_TILE_BYTES), 16, 1024, SWZ_128B);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)      // 32 bytes further along K inside the swizzle atom
+                        mma_bf16_ss(d, da + 2 * k, db + 2 * k, idesc, (kt | k) != 0);
+                    mma_commit(&empty[s]);                  // frees the stage when these MMAs are done
+                }
+                if (ok) mma_commit(&tfull[acc]);            // accumulator ready for the epilogue
+            }
+            if (!ok) report(ctl, FD_ERR_TIMEOUT, 200 + (int)blockIdx.x);
+        }
+    } else {
+        const int quad = warp & 3;                          // TMEM lane quadrant this warp may read
+        uint32_t t_it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t_it) {
+            const int m = tile % m_tiles, n = tile / m_tiles;
+            const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
+            if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const int row = m * BM + quad * 32 + lane;
+            const bool valid = row < a_total;
+            const int tok = valid ? ep.active_idx[row] : 0;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(t_row + c0, r);
+                tmem_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        const float v[4] = {__uint_as_float(r[4 * g]), __uint_as_float(r[4 * g + 1]),
+                                            __uint_as_float(r[4 * g + 2]), __uint_as_float(r[4 * g + 3])};
+                        epilogue4<__nv_bfloat16, KIND>(ep, row, n * BN + c0 + 4 * g, tok, v);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty[acc]);
+        }
+        if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 300 + (int)blockIdx.x);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 2 * BN);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn(std::string* err) {
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
+        if (err) *err = "cuTensorMapEncodeTiled is not available from the driver";
+        return nullptr;
+    }
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+    return fn;
+}
+
+int pick_bn(int n_out) { return (n_out % 256 == 0 && n_out >= 3072) ? 256 : 128; }
+
+}  // namespace
+
+bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                      const uint32_t* box, int swizzle_bytes, std::string* err) {
+    EncodeTiledFn fn = encode_fn(err);
+    if (!fn) return false;
+    cuuint64_t gd[5], gs[5];
+    cuuint32_t bx[5], es[5];
+    for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
+    CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                          : swizzle_bytes == 64  ? CU_TENSOR_MAP_SWIZZLE_64B
+                          : swizzle_bytes == 32  ? CU_TENSOR_MAP_SWIZZLE_32B
+                                                 : CU_TENSOR_MAP_SWIZZLE_NONE;
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, gd, gs, bx, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        if (err) *err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r);
+        return false;
+    }
+    return true;
+}
+
+struct GemmSpec {
+    CUtensorMap a;              // activation operand
+    int n_out, k, bn;
+};
+
+struct TcPlan {
+    fd_config cfg;
+    TcBuffers buf;
+    int sm_count;
+    GemmSpec spec[4];
+    CUtensorMap* w_maps;        // [L][4]
+    // attention (filled by the attention part)
+    void* attn;
+};
+
+bool tc_supported(const fd_config& c, std::string* why) {
+    auto bad = [&](const char* m) { if (why) *why = m; return false; };
+    if (c.dtype != FD_BF16) return bad("tensor-core engine needs bf16 storage");
+    if (c.hidden % 128 || c.mlp_dim % 128) return bad("hidden and mlp_dim must be multiples of 128");
+    return true;
+}
+
+void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::string* err);
+void tc_attention_plan_destroy(void* p);
+
+TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffers& buf, std::string* err) {
+    TcPlan* p = new TcPlan();
+    p->cfg = cfg;
+    p->buf = buf;
+    p->w_maps = new CUtensorMap[(size_t)cfg.n_blocks * 4];
+    p->attn = nullptr;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev);
+    // test knob: fewer persistent CTAs make every CTA walk many tiles (ring and accumulator wrap-around)
+    if (const char* lim = getenv("FD_TC_MAX_CTAS")) {
+        const int v = atoi(lim);
+        if (v > 0 && v < p->sm_count) p->sm_count = v;
+    }
+    const int H = cfg.hidden, M = cfg.mlp_dim;
+    const int n_out[4] = {3 * H, H, M, H};
+    const int kdim[4] = {H, H, H, M};
+    void* a_base[4] = {buf.act, buf.o, buf.act, buf.g};
+    const char* w_base[4] = {static_cast<const char*>(w.w_qkv), static_cast<const char*>(w.w_o),
+                             static_cast<const char*>(w.w_fc1), static_cast<const char*>(w.w_fc2)};
+    bool ok = true;
+    for (int g = 0; g < 4 && ok; ++g) {
+        GemmSpec& s = p->spec[g];
+        s.n_out = n_out[g];
+        s.k = kdim[g];
+        s.bn = pick_bn(n_out[g]);
+        const uint64_t dims[2] = {(uint64_t)kdim[g], (uint64_t)buf.Mcap};
+        const uint64_t strides[1] = {(uint64_t)kdim[g] * 2};
+        const uint32_t box[2] = {BK, BM};
+        ok = encode_tmap_bf16(&s.a, a_base[g], 2, dims, strides, box, 128, err);
+        for (int l = 0; l < cfg.n_blocks && ok; ++l) {
+            const uint64_t wd[2] = {(uint64_t)kdim[g], (uint64_t)n_out[g]};
+            const uint32_t wb[2] = {BK, (uint32_t)s.bn};
+            void* base = const_cast<char*>(w_base[g]) + (size_t)l * n_out[g] * kdim[g] * 2;
+            ok = encode_tmap_bf16(&p->w_maps[(size_t)l * 4 + g], base, 2, wd, strides, wb, 128, err);
+        }
+    }
+    if (ok) {
+        cudaError_t e = cudaSuccess;
+#define FD_SET_SMEM(K, N)                                                                                  \
+    if (e == cudaSuccess)                                                                                  \
+        e = cudaFuncSetAttribute(tc_gemm_kernel<K, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<N>::SMEM);
+        FD_SET_SMEM(EPI_QKV, 128) FD_SET_SMEM(EPI_QKV, 256) FD_SET_SMEM(EPI_RESID, 128) FD_SET_SMEM(EPI_RESID, 256)
+        FD_SET_SMEM(EPI_GELU, 128) FD_SET_SMEM(EPI_GELU, 256)
+#undef FD_SET_SMEM
+        if (e != cudaSuccess) {
+            ok = false;
+            if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
+        }
+    }
+    if (ok && tc_attention_supported(cfg)) {
+        p->attn = tc_attention_plan_create(cfg, buf, err);
+        ok = p->attn != nullptr;
+    }
+    if (!ok) {
+        tc_plan_destroy(p);
+        return nullptr;
+    }
+    return p;
+}
+
+void tc_plan_destroy(TcPlan* p) {
+    if (!p) return;
+    tc_attention_plan_destroy(p->attn);
+    delete[] p->w_maps;
+    delete p;
+}
+
+void* tc_plan_attn(TcPlan* p) { return p->attn; }
+int tc_plan_sm_count(TcPlan* p) { return p->sm_count; }
+
+cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
+                    int* n_launch) {
+    const GemmSpec& s = p->spec[kind];
+    const CUtensorMap& wm = p->w_maps[(size_t)blk * 4 + kind];
+    Control* c = const_cast<Control*>(ctl);
+    const int grid = p->sm_count;
+#define FD_LAUNCH(K, N) \
+    tc_gemm_kernel<K, N><<<grid, GEMM_THREADS, GemmCfg<N>::SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c)
+    if (kind == TC_GEMM_QKV) {
+        if (s.bn == 256) FD_LAUNCH(EPI_QKV, 256); else FD_LAUNCH(EPI_QKV, 128);
+    } else if (kind == TC_GEMM_FC1) {
+        if (s.bn == 256) FD_LAUNCH(EPI_GELU, 256); else FD_LAUNCH(EPI_GELU, 128);
+    } else {
+        if (s.bn == 256) FD_LAUNCH(EPI_RESID, 256); else FD_LAUNCH(EPI_RESID, 128);
+    }
+#undef FD_LAUNCH
+    ++*n_launch;
+    return cudaGetLastError();
+}
+
+}  // namespace fd

@@ -124,3 +124,20 @@ def test_host_side_argument_errors():
     assert ei.value.status == fd.FD_ERR_SHAPE
     bad = fd.make_config(wl.replace(H=250))
     assert fd.fd_workspace_bytes(bad) == 0
+
+
+@pytest.mark.parametrize("name", ["audio_tc", "mmdit_tc", "video_tc", "wide_tc", "image_tc"])
+def test_small_twins_tensor_core_engine(name):
+    wl = gen.workload(name)
+    masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 3, gen.request_fractions(wl, 3)),
+             gen.region_mask(wl, 4, [0.34] * wl.B)]
+    _run_sequence(wl, 2, fd.FD_ENGINE_TC, masks)
+
+
+def test_tensor_core_engine_few_ctas_walk_many_tiles(monkeypatch):
+    """Two persistent CTAs process every tile: the shared-memory ring and both TMEM accumulator
+    stages wrap around many times."""
+    monkeypatch.setenv("FD_TC_MAX_CTAS", "2")
+    wl = gen.workload("audio_tc")
+    masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 5, [0.6] * wl.B)]
+    _run_sequence(wl, 3, fd.FD_ENGINE_TC, masks)
