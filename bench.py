@@ -1,0 +1,449 @@
+#!/usr/bin/env python
+"""Benchmark of the region-selective denoising step (one JSON line on stdout).
+
+A "step" is one pass of the whole hot path over one ragged batch of synthetic requests:
+gate (activity score + mask) -> compaction -> all transformer blocks on the active tokens.
+Default workload: the audio-latent configuration (24 blocks, hidden 1536, 8 concurrent requests
+of 1024 tokens, per-request active fraction ~U[0.2,0.8]).
+
+  python bench.py --gpus 1 --steps 20 --warmup 5
+  python bench.py --impl reference        # the CPU oracle on the host cores (bounded sample)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "regional DiT step effective TFLOP/s (step ms, fraction of BF16 peak, vs dense step)"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def block_flops(A_b, N, H, M):
+    """Algorithmic FLOPs of one block: QKV 6AH^2, out 2AH^2, MLP 4AHM, attention 4 sum_b A_b N H."""
+    A = float(sum(A_b))
+    return {"gemm_qkv": 6 * A * H * H, "gemm_out": 2 * A * H * H, "gemm_fc1": 2 * A * H * M,
+            "gemm_fc2": 2 * A * H * M, "attention": 4.0 * sum(a * N * H for a in A_b)}
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd_, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd_)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, parts[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        os.unlink(self.path)
+        # samples under load: the upper half of the clock samples excludes idle ticks around the region
+        if sm:
+            hi = sorted(sm)[len(sm) // 2:]
+            return {"sm_mhz": statistics.median(hi), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                    "samples": len(sm)}
+        return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm / cpu_baseline: the oracle as it stands, on the host cores, on a bounded sample
+# ------------------------------------------------------------------------------------------------
+class OracleSample:
+    """Block 0 of the workload through the CPU oracle on a bounded sample: the first `n_req` requests;
+    gate + compaction + adaLN, K/V refresh of all their active rows, attention + MLP of `n_finish`
+    sampled active rows.  Inputs are prepared once; run() is what gets timed."""
+
+    def __init__(self, wl_name: str, seed: int):
+        import gen
+        import oracle
+        self.gen, self.oracle = gen, oracle
+        self.wl_full = gen.workload(wl_name)
+        self.seed = seed
+        oracle.adaln(np.zeros((1, 8), np.float32), np.zeros((6, 8), np.float32), np.zeros(6, np.float32))
+
+    def prepare(self, n_req: int, n_finish: int):
+        gen, oracle = self.gen, self.oracle
+        wl = self.wl_full.replace(B=max(1, min(n_req, self.wl_full.B)))
+        if wl.labels == "partition":
+            lab, _ = oracle.partition(gen.saliency_map(wl, self.seed), None, wl.R, wl.m_min, wl.m_max)
+            labels = np.ascontiguousarray(np.concatenate([lab, np.full((wl.B, wl.n_text), wl.R, np.int32)], axis=1))
+        else:
+            labels = gen.uniform_labels(wl)
+        self.wl, self.labels = wl, labels
+        self.w = gen.block_weights(wl, self.seed, n_blocks=1)
+        self.inp = gen.step_inputs(wl, self.seed, labels)
+        self.lat = gen.latent_pair(wl, self.seed, labels, fractions=gen.request_fractions(wl, self.seed))
+        self.n_finish = n_finish
+
+    def run(self):
+        oracle, wl = self.oracle, self.wl
+        kv = np.zeros((wl.B, 2, wl.N, wl.H), np.float32)
+        t0 = time.perf_counter()
+        state = oracle.initial_state(wl.B, wl.R)
+        _, _, mask = oracle.activity_gate(self.lat["z_cur"], self.lat["z_prev"], self.labels, self.lat["eps"],
+                                          state, wl.R)
+        idx, cu = oracle.compact(mask, self.labels, wl.R)
+        u = np.ascontiguousarray(self.inp["x_cur"].reshape(-1, wl.H)[idx])
+        mod = oracle.adaln(self.inp["cond"], self.w["w_ada"][0], self.w["b_ada"][0])
+        n = max(1, min(self.n_finish, idx.size))
+        fin = np.linspace(0, idx.size - 1, n).astype(np.int32)
+        oracle.regional_block(u, idx, mod, self.w, 0, kv, wl.heads, finish=fin)
+        dt = time.perf_counter() - t0
+        A, H, M, N = idx.size, wl.H, wl.M, wl.N
+        flops = 6.0 * A * H * H + n * (4.0 * N * H + 2.0 * H * H + 4.0 * H * M)
+        text = ("block 0 of %d of workload %s, first %d of %d requests: gate, compaction, adaLN, K/V refresh of "
+                "all %d active rows, attention+MLP of %d sampled rows"
+                % (self.wl_full.L, wl.name, wl.B, self.wl_full.B, A, n))
+        return dt, flops, text
+
+    def sized_for(self, seconds: float):
+        """Calibrates on a small sample, then sizes the sample for about `seconds` of CPU work."""
+        wl = self.wl_full
+        self.prepare(1, 16)
+        dt, fl, _ = self.run()
+        rate = fl / dt
+        budget = rate * seconds
+        per_req = 6.0 * (0.5 * wl.N) * wl.H * wl.H
+        per_row = 4.0 * wl.N * wl.H + 2.0 * wl.H * wl.H + 4.0 * wl.H * wl.M
+        n_req = int(max(1, min(wl.B, (0.6 * budget) // per_req)))
+        n_fin = int(max(16, min(4096, (budget - n_req * per_req) // per_row)))
+        self.prepare(n_req, n_fin)
+
+
+def omp_threads():
+    v = os.environ.get("OMP_NUM_THREADS")
+    return int(v) if v and v.isdigit() else (os.cpu_count() or 1)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleSample(args.workload, args.seed)
+    # the whole --steps/--warmup run should end within a few minutes: about 150 s of oracle time in total
+    smp.sized_for(min(30.0, 150.0 / max(1, args.steps + args.warmup)))
+    times, flops, text = [], 0.0, ""
+    for i in range(args.warmup + args.steps):
+        dt, flops, text = smp.run()
+        if i >= args.warmup:
+            times.append(dt)
+    t = sum(times) / len(times)
+    val = flops / t / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32 storage, f64 accumulate", "data": "synthetic",
+        "config": {"workload": args.workload, "sample": text},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": omp_threads(), "kind": "oracle", "sample": text},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def device_weights(wl, seed, device):
+    """Weights ~N(0, 0.02) drawn on the device (the full stacks are 1-2 GB): same recipe as the
+    numpy generator, different stream."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    H, M, Hc, L = wl.H, wl.M, wl.Hc, wl.L
+    shapes = {"w_qkv": (L, 3 * H, H), "b_qkv": (L, 3 * H), "w_o": (L, H, H), "b_o": (L, H),
+              "w_fc1": (L, M, H), "b_fc1": (L, M), "w_fc2": (L, H, M), "b_fc2": (L, H),
+              "w_ada": (L, 6 * H, Hc), "b_ada": (L, 6 * H)}
+    out = {}
+    for k, s in shapes.items():
+        t = torch.empty(s, dtype=torch.float32, device=device)
+        t.normal_(0.0, 0.02, generator=g)
+        out[k] = t.to(dt).contiguous()
+        del t
+    return out
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import gen
+    import paper_2607_12121_b200 as fd
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = gen.workload(args.workload)
+    if wl.labels == "partition":
+        raise SystemExit("bench workloads with partitioner labels are run through --workload audio for now")
+    seed = args.seed + 17 * rank                 # every rank owns its own batch of requests (weak scaling)
+    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    B, N, H, M, R, L, D = wl.B, wl.N, wl.H, wl.M, wl.R, wl.L, wl.D
+
+    labels_np = gen.uniform_labels(wl)
+    inp = gen.step_inputs(wl, seed, labels_np)
+    fr = gen.request_fractions(wl, seed) if args.fraction is None else np.full(B, args.fraction)
+    lat = gen.latent_pair(wl, seed, labels_np, fractions=fr)
+
+    weights = device_weights(wl, seed, dev)
+    cfg = fd.make_config(wl)
+    ctx = fd.fd_create(cfg, weights, device=dev)
+
+    def pin(a, tdt=None):
+        t = torch.from_numpy(np.ascontiguousarray(a))
+        if tdt is not None:
+            t = t.to(tdt)
+        return t.pin_memory()
+
+    h_x, h_xprev, h_cond = pin(inp["x_cur"], dt), pin(inp["x_prev"], dt), pin(inp["cond"], dt)
+    h_zc, h_zp, h_eps = pin(lat["z_cur"]), pin(lat["z_prev"]), pin(lat["eps"])
+    x, x_prev, cond = h_x.to(dev), h_xprev.to(dev), h_cond.to(dev)
+    z_cur, z_prev, eps = h_zc.to(dev), h_zp.to(dev), h_eps.to(dev)
+    labels = torch.from_numpy(labels_np).to(dev)
+    ones = torch.ones((B, R), dtype=torch.uint8, device=dev)
+    kv = torch.zeros((L, B, 2, N, H), dtype=dt, device=dev)
+    y = torch.zeros((B, N, H), dtype=dt, device=dev)
+    h_y = torch.empty((B, N, H), dtype=dt).pin_memory()
+    active_idx = torch.zeros(B * N, dtype=torch.int32, device=dev)
+    cu_active = torch.zeros(B + 1, dtype=torch.int32, device=dev)
+    delta = torch.zeros((B, R), dtype=torch.float32, device=dev)
+    skip = torch.zeros((B, R), dtype=torch.int32, device=dev)
+    prev = torch.ones((B, R), dtype=torch.uint8, device=dev)
+    score = torch.empty((B, R), dtype=torch.float32, device=dev)
+    weight = torch.empty((B, R), dtype=torch.float32, device=dev)
+    mask = torch.empty((B, R), dtype=torch.uint8, device=dev)
+
+    def dense_step(src):
+        fd.fd_regional_step(ctx, src, cond, labels, ones, R, kv, y, active_idx, cu_active)
+
+    def gated_step(xin=None, zc=None, zp=None, ep=None, cd=None):
+        # fresh gate state: every timed step sees the same "first gated step after the warm-up"
+        delta.zero_(); skip.zero_(); prev.fill_(1)
+        fd.fd_region_activity(ctx, z_cur if zc is None else zc, z_prev if zp is None else zp, labels, R,
+                              eps if ep is None else ep, delta, skip, prev, score, weight, mask)
+        fd.fd_regional_step(ctx, x if xin is None else xin, cond if cd is None else cd, labels, mask, R, kv, y,
+                            active_idx, cu_active)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / steps
+
+    # warm-up: one dense step on the previous step's tokens fills kv / y, then W gated steps
+    dense_step(x_prev)
+    for _ in range(max(args.warmup, 3)):
+        gated_step()
+    fd.fd_poll_status(ctx)
+    cu = cu_active.cpu().numpy()
+    A_b = np.diff(cu).astype(np.int64)
+    A = int(cu[-1])
+    f_tok = A / float(B * N)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = ctx.launches
+    ms_reg = timed(gated_step, args.steps)
+    launches = ctx.launches - launches0
+    clocks = sampler.stop()
+
+    # the same engine's dense step (mask of ones) and the per-kernel breakdown
+    for _ in range(2):
+        dense_step(x)
+    ms_dense = timed(lambda: dense_step(x), max(3, args.steps // 2))
+    dense_step(x_prev)                         # restore the cached state the gated step expects
+    fd.fd_profile_enable(ctx, True)
+    barrier()
+    for _ in range(args.steps):
+        gated_step()
+    prof = fd.fd_profile_read(ctx)
+    fd.fd_profile_enable(ctx, False)
+
+    # end to end through the C-ABI with host buffers: pinned H2D of the step's inputs, D2H of y
+    d_x, d_cond = torch.empty_like(x), torch.empty_like(cond)
+    d_zc, d_zp, d_eps = torch.empty_like(z_cur), torch.empty_like(z_prev), torch.empty_like(eps)
+
+    def e2e_step():
+        d_x.copy_(h_x, non_blocking=True); d_cond.copy_(h_cond, non_blocking=True)
+        d_zc.copy_(h_zc, non_blocking=True); d_zp.copy_(h_zp, non_blocking=True)
+        d_eps.copy_(h_eps, non_blocking=True)
+        gated_step(d_x, d_zc, d_zp, d_eps, d_cond)
+        h_y.copy_(y, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    ms_e2e = timed(e2e_step, args.steps)
+    h2d = sum(t.numel() * t.element_size() for t in (h_x, h_cond, h_zc, h_zp, h_eps))
+    d2h = h_y.numel() * h_y.element_size()
+    fd.fd_poll_status(ctx)
+
+    fl = block_flops(A_b, N, H, M)
+    step_flops = L * sum(fl.values())
+    dense_flops = L * sum(block_flops([N] * B, N, H, M).values())
+    peaks, peak_kind = load_peaks()
+    value = world * step_flops / (ms_reg * 1e-3) / 1e12
+    e2e_value = world * step_flops / (ms_e2e * 1e-3) / 1e12
+
+    # per-kernel breakdown of the profiled pass; the dominant group feeds the roofline object
+    es = 2 if wl.dtype == "bf16" else 4
+    bytes_per_launch = {
+        "ln_modulate": A * H * (4 + es), "adaln": L * 6 * H * wl.Hc * es,
+        "activity": 2.0 * 4 * D * float(N * B), "compact": 4.0 * B * N + 4.0 * A,
+    }
+    total_ms = sum(v[0] for v in prof.values()) or 1.0
+    breakdown = {}
+    for k, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        calls = args.steps * (L if k.startswith("gemm") or k == "attention" else (2 * L if k == "ln_modulate" else 1))
+        per_call_ms = ms / calls
+        ent = {"ms_per_step": ms / args.steps, "share": ms / total_ms, "calls_per_step": calls // args.steps,
+               "avg_call_us": per_call_ms * 1e3}
+        if k in fl:
+            ent["tflops"] = fl[k] / (per_call_ms * 1e-3) / 1e12
+        elif k in bytes_per_launch:
+            ent["gbs"] = bytes_per_launch[k] / (per_call_ms * 1e-3) / 1e9
+        breakdown[k] = ent
+    dom = max((k for k in breakdown if k in fl), key=lambda k: breakdown[k]["ms_per_step"])
+    tensor_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tp):
+        with open(tp) as f:
+            traffic = json.load(f).get(dom)
+    roofline = {"kernel": dom, "bound": "tensor", "achieved": breakdown[dom]["tflops"], "peak": tensor_peak,
+                "unit": "TFLOP/s", "frac": breakdown[dom]["tflops"] / tensor_peak, "traffic": traffic,
+                "peak_source": peak_kind + " (sustained bf16 matmul; the kernel is timed inside a long step)",
+                "flops_per_launch": fl[dom]}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_reg, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "blocks": L, "hidden": H, "heads": wl.heads, "head_dim": wl.head_dim,
+                   "mlp": M, "requests": B, "tokens_per_request": N, "regions": R,
+                   "active_tokens": A, "active_fraction": f_tok, "per_request_active": A_b.tolist(),
+                   "parallelism": "replicas x%d (no collectives)" % world,
+                   "l2": "inputs larger than L2: %.2f GB of weights stream through every step" %
+                         (sum(t.numel() * t.element_size() for t in weights.values()) / 1e9)},
+        "regional_step_ms": ms_reg, "dense_step_ms": ms_dense,
+        "dense_tflops": dense_flops / (ms_dense * 1e-3) / 1e12,
+        "frac_of_bf16_peak": value / world / float(peaks["bf16_tflops"]),
+        "speedup_vs_dense": ms_dense / ms_reg, "time_over_fraction_times_dense": ms_reg / (f_tok * ms_dense),
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "kernel_breakdown": breakdown,
+        "peaks": {"source": peak_kind, "bf16_tflops": peaks.get("bf16_tflops"),
+                  "bf16_tflops_sustained": peaks.get("bf16_tflops_sustained"), "hbm_gbs": peaks.get("hbm_gbs")},
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            smp = OracleSample(args.workload, args.seed)
+            smp.sized_for(15.0)
+            dt_cpu, fl_cpu, text = smp.run()
+            line["cpu_baseline"] = {"value": fl_cpu / dt_cpu / 1e12, "unit": "TFLOP/s", "cores": omp_threads(),
+                                    "kind": "oracle", "sample": text, "seconds": dt_cpu}
+        print(json.dumps(line))
+    fd.fd_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="audio")
+    ap.add_argument("--fraction", type=float, default=None, help="same active fraction for every request")
+    ap.add_argument("--seed", type=int, default=1000)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

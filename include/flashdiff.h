@@ -163,6 +163,28 @@ fd_status fd_poll_status(fd_ctx* ctx, void* cuda_stream);
 /* Number of kernels the library has launched through this context so far (host counter). */
 int64_t fd_launch_count(const fd_ctx* ctx);
 
+/*
+ * Optional per-kernel timing.  While enabled, every kernel group the library launches is bracketed
+ * by CUDA events on the caller's stream.  fd_profile_read synchronises `cuda_stream`, adds the
+ * elapsed milliseconds and the kernel counts per group into the two HOST arrays of
+ * FD_PROF_GROUPS entries, and forgets the recorded events.
+ */
+enum {
+    FD_PROF_ACTIVITY = 0, /* activity reduce + gate          */
+    FD_PROF_COMPACT = 1,  /* compaction (count + write)      */
+    FD_PROF_ADALN = 2,    /* adaLN conditioning vectors      */
+    FD_PROF_LN = 3,       /* gather + LayerNorm + modulation */
+    FD_PROF_GEMM_QKV = 4,
+    FD_PROF_ATTENTION = 5,
+    FD_PROF_GEMM_OUT = 6,
+    FD_PROF_GEMM_FC1 = 7,
+    FD_PROF_GEMM_FC2 = 8,
+    FD_PROF_PARTITION = 9,
+    FD_PROF_GROUPS = 10
+};
+fd_status fd_profile_enable(fd_ctx* ctx, int enable);
+fd_status fd_profile_read(fd_ctx* ctx, void* cuda_stream, float* ms_out, int32_t* kernels_out);
+
 /* Releases the context (host memory only; the workspace goes back to the caller). */
 fd_status fd_destroy(fd_ctx* ctx);
 

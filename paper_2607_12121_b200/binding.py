@@ -20,7 +20,10 @@ FD_F32, FD_BF16 = 0, 1
 FD_ENGINE_AUTO, FD_ENGINE_SIMT, FD_ENGINE_TC = 0, 1, 2
 
 EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region_activity",
-           "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error"]
+           "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
+           "fd_profile_enable", "fd_profile_read"]
+PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
+               "gemm_fc2", "partition"]
 
 
 class FdConfig(ctypes.Structure):
@@ -59,6 +62,10 @@ def _load() -> ctypes.CDLL:
     lib.fd_regional_step.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.fd_poll_status.restype = i32
     lib.fd_poll_status.argtypes = [vp, vp]
+    lib.fd_profile_enable.restype = i32
+    lib.fd_profile_enable.argtypes = [vp, i32]
+    lib.fd_profile_read.restype = i32
+    lib.fd_profile_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     lib.fd_launch_count.restype = ctypes.c_int64
     lib.fd_launch_count.argtypes = [vp]
     lib.fd_destroy.restype = i32
@@ -164,6 +171,19 @@ def fd_regional_step(ctx: Context, x, cond, labels, mask, R: int, kv_cache, y, a
 
 def fd_poll_status(ctx: Context, stream=None) -> None:
     _check(ctx.handle, lib.fd_poll_status(ctx.handle, _stream(stream)))
+
+
+def fd_profile_enable(ctx: Context, enable: bool) -> None:
+    _check(ctx.handle, lib.fd_profile_enable(ctx.handle, 1 if enable else 0))
+
+
+def fd_profile_read(ctx: Context, stream=None):
+    """Returns {group: (milliseconds, kernels)} accumulated since the last read."""
+    n = len(PROF_GROUPS)
+    ms = (ctypes.c_float * n)()
+    cnt = (ctypes.c_int32 * n)()
+    _check(ctx.handle, lib.fd_profile_read(ctx.handle, _stream(stream), ms, cnt))
+    return {PROF_GROUPS[i]: (float(ms[i]), int(cnt[i])) for i in range(n)}
 
 
 def make_config(wl, max_batch=None, max_tokens=None, max_regions=None, n_blocks=None, engine=FD_ENGINE_AUTO,

@@ -7,6 +7,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <vector>
 
 #include "common.cuh"
 #include "tc.cuh"
@@ -85,6 +86,29 @@ struct fd_ctx {
     int64_t launches;
     std::string err;
     TcPlan* tc;
+    // optional per-kernel timing
+    bool profiling = false;
+    struct Span { cudaEvent_t a, b; int group, kernels; };
+    std::vector<Span> spans;
+    std::vector<cudaEvent_t> pool;
+
+    cudaEvent_t get_event() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+    void span_begin(int group, cudaStream_t st) {
+        if (!profiling) return;
+        Span s{get_event(), get_event(), group, 0};
+        cudaEventRecord(s.a, st);
+        spans.push_back(s);
+    }
+    void span_end(int kernels, cudaStream_t st) {
+        if (!profiling) return;
+        spans.back().kernels = kernels;
+        cudaEventRecord(spans.back().b, st);
+    }
 
     fd_status fail(fd_status s, const char* fmt, ...) {
         char buf[512];
@@ -123,18 +147,21 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     const int rows_cap = B * N;
     int nl = 0;
     cudaError_t e;
-#define FD_TRY(call)                                                                                     \
+#define FD_TRY(group, call)                                                                              \
     do {                                                                                                 \
+        const int nl_before = nl;                                                                        \
+        c->span_begin(group, st);                                                                        \
         e = (call);                                                                                      \
+        c->span_end(nl - nl_before, st);                                                                 \
         if (e != cudaSuccess) {                                                                          \
             c->launches += nl;                                                                           \
             return c->fail(FD_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e));                  \
         }                                                                                                \
     } while (0)
 
-    FD_TRY(launch_compact(mask, labels, B, N, R, active_idx, cu_active, c->at<int32_t>(l.block_counts), tiles,
+    FD_TRY(FD_PROF_COMPACT, launch_compact(mask, labels, B, N, R, active_idx, cu_active, c->at<int32_t>(l.block_counts), tiles,
                           c->tile_rows, ctl, st, &nl));
-    FD_TRY(launch_adaln<T>(cond, static_cast<const T*>(c->w.w_ada), static_cast<const T*>(c->w.b_ada), mod, L, B, H,
+    FD_TRY(FD_PROF_ADALN, launch_adaln<T>(cond, static_cast<const T*>(c->w.w_ada), static_cast<const T*>(c->w.b_ada), mod, L, B, H,
                            Hc, st, &nl));
     const int max_tiles = B * ((N + c->tile_rows - 1) / c->tile_rows);
     for (int blk = 0; blk < L; ++blk) {
@@ -151,7 +178,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         ep.H = H;
 
         // gather (first block) or read the residual stream; LayerNorm; attention-branch modulation
-        FD_TRY(launch_ln_modulate<T>(blk == 0 ? x : nullptr, resid, resid, act, active_idx, mod_b + 0 * H,
+        FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(blk == 0 ? x : nullptr, resid, resid, act, active_idx, mod_b + 0 * H,
                                      mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl));
         // QKV projection; K and V rows go straight into the cache
         ep.bias = static_cast<const T*>(c->w.b_qkv) + (size_t)blk * 3 * H;
@@ -159,14 +186,14 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         ep.q_ld = l.q_ld;
         ep.kv = kv_b;
         if (c->use_tc)
-            FD_TRY(tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));
+            FD_TRY(FD_PROF_GEMM_QKV, tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));
         else
-            FD_TRY(launch_simt_gemm<T>(EPI_QKV, act, H, w_qkv, 3 * H, H, rows_cap, ep, ctl, st, &nl));
+            FD_TRY(FD_PROF_GEMM_QKV, launch_simt_gemm<T>(EPI_QKV, act, H, w_qkv, 3 * H, H, rows_cap, ep, ctl, st, &nl));
         // active queries against all N keys of their request
         if (c->use_tc_attn)
-            FD_TRY(tc_attention(c->tc, blk, kv_b, B, N, tiles, max_tiles, ctl, st, &nl));
+            FD_TRY(FD_PROF_ATTENTION, tc_attention(c->tc, blk, kv_b, B, N, tiles, max_tiles, ctl, st, &nl));
         else
-            FD_TRY(launch_simt_attention<T>(q, l.q_ld, kv_b, o, H, tiles, max_tiles, N, H, cf.n_heads, cf.head_dim,
+            FD_TRY(FD_PROF_ATTENTION, launch_simt_attention<T>(q, l.q_ld, kv_b, o, H, tiles, max_tiles, N, H, cf.n_heads, cf.head_dim,
                                             ctl, st, &nl));
         // out-projection, gated residual
         ep.bias = static_cast<const T*>(c->w.b_o) + (size_t)blk * H;
@@ -174,26 +201,26 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         ep.gate = mod_b + 2 * H;
         ep.y = nullptr;
         if (c->use_tc)
-            FD_TRY(tc_gemm(c->tc, TC_GEMM_OUT, blk, ep, ctl, st, &nl));
+            FD_TRY(FD_PROF_GEMM_OUT, tc_gemm(c->tc, TC_GEMM_OUT, blk, ep, ctl, st, &nl));
         else
-            FD_TRY(launch_simt_gemm<T>(EPI_RESID, o, H, w_o, H, H, rows_cap, ep, ctl, st, &nl));
+            FD_TRY(FD_PROF_GEMM_OUT, launch_simt_gemm<T>(EPI_RESID, o, H, w_o, H, H, rows_cap, ep, ctl, st, &nl));
         // MLP branch
-        FD_TRY(launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, mod_b + 3 * H, mod_b + 4 * H, 6 * H, N,
+        FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, mod_b + 3 * H, mod_b + 4 * H, 6 * H, N,
                                      H, rows_cap, cf.ln_eps, ctl, st, &nl));
         ep.bias = static_cast<const T*>(c->w.b_fc1) + (size_t)blk * M;
         ep.out = g;
         ep.out_ld = M;
         if (c->use_tc)
-            FD_TRY(tc_gemm(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl));
+            FD_TRY(FD_PROF_GEMM_FC1, tc_gemm(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl));
         else
-            FD_TRY(launch_simt_gemm<T>(EPI_GELU, act, H, w_fc1, M, H, rows_cap, ep, ctl, st, &nl));
+            FD_TRY(FD_PROF_GEMM_FC1, launch_simt_gemm<T>(EPI_GELU, act, H, w_fc1, M, H, rows_cap, ep, ctl, st, &nl));
         ep.bias = static_cast<const T*>(c->w.b_fc2) + (size_t)blk * H;
         ep.gate = mod_b + 5 * H;
         ep.y = (blk == L - 1) ? y_ : nullptr;       // the last block scatters the rows back
         if (c->use_tc)
-            FD_TRY(tc_gemm(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl));
+            FD_TRY(FD_PROF_GEMM_FC2, tc_gemm(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl));
         else
-            FD_TRY(launch_simt_gemm<T>(EPI_RESID, g, M, w_fc2, H, M, rows_cap, ep, ctl, st, &nl));
+            FD_TRY(FD_PROF_GEMM_FC2, launch_simt_gemm<T>(EPI_RESID, g, M, w_fc2, H, M, rows_cap, ep, ctl, st, &nl));
     }
 #undef FD_TRY
     c->launches += nl;
@@ -293,9 +320,11 @@ fd_status fd_partition_regions(fd_ctx* c, const float* attn_map, int B, int N, i
     if (min_region_tokens < 1) min_region_tokens = 1;
     if (max_region_tokens <= 0 || max_region_tokens > N) max_region_tokens = N;
     int nl = 0;
+    c->span_begin(FD_PROF_PARTITION, static_cast<cudaStream_t>(cuda_stream));
     cudaError_t e = launch_partition(attn_map, B, N, T, salient_cols, salient_cols ? T_s : T, R, min_region_tokens,
                                      max_region_tokens, labels_out, region_sizes_out, c->ws + c->lay.part, c->ctl(),
                                      static_cast<cudaStream_t>(cuda_stream), &nl);
+    c->span_end(nl, static_cast<cudaStream_t>(cuda_stream));
     c->launches += nl;
     if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "partition launch failed: %s", cudaGetErrorString(e));
     return FD_OK;
@@ -314,10 +343,12 @@ fd_status fd_region_activity(fd_ctx* c, const float* z_cur, const float* z_prev,
         return c->fail(FD_ERR_SHAPE, "B=%d N=%d R=%d exceed the limits %d/%d/%d", B, N, R, c->cfg.max_batch,
                        c->cfg.max_tokens, c->cfg.max_regions);
     int nl = 0;
+    c->span_begin(FD_PROF_ACTIVITY, static_cast<cudaStream_t>(cuda_stream));
     cudaError_t e = launch_activity(z_cur, z_prev, labels, B, N, D, R, eps, delta_state, skip_count, prev_active,
                                     score_out, weight_out, mask_out, c->cfg.gate_eta, c->cfg.max_skip_k,
                                     c->at<double>(c->lay.acc_ss), c->at<int32_t>(c->lay.acc_cnt), c->ctl(),
                                     static_cast<cudaStream_t>(cuda_stream), &nl);
+    c->span_end(nl, static_cast<cudaStream_t>(cuda_stream));
     c->launches += nl;
     if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "activity launch failed: %s", cudaGetErrorString(e));
     return FD_OK;
@@ -356,11 +387,37 @@ fd_status fd_poll_status(fd_ctx* c, void* cuda_stream) {
     return FD_OK;
 }
 
+fd_status fd_profile_enable(fd_ctx* c, int enable) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    c->profiling = enable != 0;
+    return FD_OK;
+}
+
+fd_status fd_profile_read(fd_ctx* c, void* cuda_stream, float* ms_out, int32_t* kernels_out) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!ms_out || !kernels_out) return c->fail(FD_ERR_INVALID_ARG, "null output array");
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "stream synchronise failed: %s", cudaGetErrorString(e));
+    for (auto& s : c->spans) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, s.a, s.b) == cudaSuccess && s.group >= 0 && s.group < FD_PROF_GROUPS) {
+            ms_out[s.group] += ms;
+            kernels_out[s.group] += s.kernels;
+        }
+        c->pool.push_back(s.a);
+        c->pool.push_back(s.b);
+    }
+    c->spans.clear();
+    return FD_OK;
+}
+
 int64_t fd_launch_count(const fd_ctx* c) { return c ? c->launches : 0; }
 
 fd_status fd_destroy(fd_ctx* c) {
     if (!c) return FD_ERR_INVALID_ARG;
     tc_plan_destroy(c->tc);
+    for (auto& s : c->spans) { c->pool.push_back(s.a); c->pool.push_back(s.b); }
+    for (cudaEvent_t ev : c->pool) cudaEventDestroy(ev);
     delete c;
     return FD_OK;
 }
