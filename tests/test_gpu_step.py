@@ -38,12 +38,15 @@ def _check_step(wl, y, kv, y_ref, kv_ref, y_before, kv_before, idx):
             assert np.array_equal(got[~a2], old[~a2])
 
 
-def _run_sequence(wl, seed, engine, masks, n_blocks=None):
+def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0):
     """Warm-up (all active) on the previous step's tokens, then gated steps; both sides start
     from the same zero caches and carry their own state forward."""
     L = wl.L if n_blocks is None else n_blocks
     labels = labels_for(wl, seed)
     w = gen.block_weights(wl, seed, n_blocks=L)
+    if qk_gain != 1.0:          # a power of two keeps the weights exact in bf16
+        w["w_qkv"][:, :wl.H] *= np.float32(qk_gain)       # query rows only: K/V keep their magnitude
+        w["b_qkv"][:, :wl.H] *= np.float32(qk_gain)
     inp = gen.step_inputs(wl, seed, labels)
     ctx = make_ctx(wl, w, engine=engine, n_blocks=L)
     buf = StepBuffers(wl, L)
@@ -141,3 +144,13 @@ def test_tensor_core_engine_few_ctas_walk_many_tiles(monkeypatch):
     wl = gen.workload("audio_tc")
     masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 5, [0.6] * wl.B)]
     _run_sequence(wl, 3, fd.FD_ENGINE_TC, masks)
+
+
+@pytest.mark.parametrize("name,engine", [("audio_tc", fd.FD_ENGINE_TC), ("video_tc", fd.FD_ENGINE_TC),
+                                         ("audio_tc", fd.FD_ENGINE_SIMT)])
+def test_peaked_attention_exercises_running_max(name, engine):
+    """Query weights scaled by 64: scores spread over many e-folds, so the running maximum moves
+    between key tiles and the accumulated output has to be rescaled."""
+    wl = gen.workload(name)
+    masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.5] * wl.B)]
+    _run_sequence(wl, 4, engine, masks, qk_gain=64.0)
