@@ -65,3 +65,82 @@ __device__ __forceinline__ void epilogue4(const EpiParams& ep, int row, int col,
 }
 
 }  // namespace fd
+
+// ---- 32-column variant for the tensor-core kernels (bf16 storage, H % 32 == 0) -----------------
+namespace fd {
+
+__device__ __forceinline__ float tanh_fast(float x) {
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float gelu_tanh_fast(float a) {
+    const float u = 0.7978845608028654f * fmaf(0.044715f * a * a, a, a);
+    return 0.5f * a * (1.0f + tanh_fast(u));
+}
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ void store8_bf16(__nv_bfloat16* p, const float* v) {
+    uint4 u;
+    u.x = pack2_bf16(v[0], v[1]); u.y = pack2_bf16(v[2], v[3]);
+    u.z = pack2_bf16(v[4], v[5]); u.w = pack2_bf16(v[6], v[7]);
+    *reinterpret_cast<uint4*>(p) = u;
+}
+
+// acc: 32 consecutive fp32 accumulator columns of one row, starting at column col (col % 32 == 0)
+template <int KIND>
+__device__ __forceinline__ void epilogue32(const EpiParams& ep, int row, int col, int tok, const uint32_t* acc) {
+    using T = __nv_bfloat16;
+    float v[32];
+    const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ep.bias) + col);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint4 b = __ldg(bp + q);
+        const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[8 * q + 2 * i] = __uint_as_float(acc[8 * q + 2 * i]) + __uint_as_float(w[i] << 16);
+            v[8 * q + 2 * i + 1] = __uint_as_float(acc[8 * q + 2 * i + 1]) + __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    if constexpr (KIND == EPI_QKV) {
+        const int sec = col / ep.H, c = col - sec * ep.H;
+        T* dst;
+        if (sec == 0) {
+            dst = reinterpret_cast<T*>(ep.q) + (size_t)row * ep.q_ld + c;
+        } else {
+            const int b = tok / ep.N, j = tok - b * ep.N;
+            dst = reinterpret_cast<T*>(ep.kv) + (((size_t)b * 2 + (sec - 1)) * ep.N + j) * ep.H + c;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) store8_bf16(dst + 8 * q, v + 8 * q);
+    } else if constexpr (KIND == EPI_RESID) {
+        const int b = tok / ep.N;
+        const float4* gp = reinterpret_cast<const float4*>(ep.gate + (size_t)b * 6 * ep.H + col);
+        float4* rp = reinterpret_cast<float4*>(ep.resid + (size_t)row * ep.H + col);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 g = __ldg(gp + q);
+            float4 r = rp[q];
+            r.x = fmaf(g.x, v[4 * q], r.x); r.y = fmaf(g.y, v[4 * q + 1], r.y);
+            r.z = fmaf(g.z, v[4 * q + 2], r.z); r.w = fmaf(g.w, v[4 * q + 3], r.w);
+            rp[q] = r;
+            v[4 * q] = r.x; v[4 * q + 1] = r.y; v[4 * q + 2] = r.z; v[4 * q + 3] = r.w;
+        }
+        if (ep.y) {
+            T* dst = reinterpret_cast<T*>(ep.y) + (size_t)tok * ep.H + col;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) store8_bf16(dst + 8 * q, v + 8 * q);
+        }
+    } else {
+        T* dst = reinterpret_cast<T*>(ep.out) + (size_t)row * ep.out_ld + col;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_fast(v[i]);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) store8_bf16(dst + 8 * q, v + 8 * q);
+    }
+}
+
+}  // namespace fd

@@ -42,9 +42,12 @@ template <> struct Vec<__nv_bfloat16> {
 };
 
 // ---- adaLN: mod[l,b,o] = sum_c SiLU(cond[b,c]) W_ada[l,o,c] + b_ada[l,o] ----------------------
+// HBM-bound on W_ada (read once).  SiLU(cond) of up to 8 requests sits in shared memory; every warp
+// streams 4 weight rows at a time with 128-bit loads so each shared-memory read feeds 4 rows.
 constexpr int ADA_THREADS = 256;
-constexpr int ADA_BCH = 8;         // requests handled per pass over a weight row
-constexpr int ADA_ROWS = 32;       // weight rows per CTA
+constexpr int ADA_BCH = 8;         // requests handled per pass over the weights
+constexpr int ADA_RPW = 4;         // weight rows a warp processes together
+constexpr int ADA_ROWS = 128;      // weight rows per CTA
 
 template <typename T>
 __global__ void __launch_bounds__(ADA_THREADS)
@@ -62,32 +65,49 @@ adaln_kernel(const T* __restrict__ cond, const T* __restrict__ w_ada, const T* _
             s_act[i] = v / (1.0f + __expf(-v));
         }
         __syncthreads();
-        for (int r = warp; r < ADA_ROWS; r += ADA_THREADS / 32) {
-            const long long row = (long long)blockIdx.x * ADA_ROWS + r;
-            if (row >= rows_total) break;
-            const T* wr = w_ada + (size_t)row * Hc;
-            float acc[ADA_BCH];
+        for (int r = warp * ADA_RPW; r < ADA_ROWS; r += (ADA_THREADS / 32) * ADA_RPW) {
+            const long long row0 = (long long)blockIdx.x * ADA_ROWS + r;
+            if (row0 >= rows_total) break;
+            float acc[ADA_RPW][ADA_BCH];
 #pragma unroll
-            for (int b = 0; b < ADA_BCH; ++b) acc[b] = 0.f;
+            for (int q = 0; q < ADA_RPW; ++q)
+#pragma unroll
+                for (int b = 0; b < ADA_BCH; ++b) acc[q][b] = 0.f;
             for (int c = lane * VN; c < Hc; c += 32 * VN) {
-                float w[VN];
-                Vec<T>::load(wr + c, w);
+                float w[ADA_RPW][VN];
+#pragma unroll
+                for (int q = 0; q < ADA_RPW; ++q) {
+                    const long long row = min(row0 + q, rows_total - 1);
+                    Vec<T>::load(w_ada + (size_t)row * Hc + c, w[q]);
+                }
 #pragma unroll
                 for (int b = 0; b < ADA_BCH; ++b) {
                     if (b < nb) {
-                        const float* a = s_act + b * Hc + c;
+                        float a[VN];
 #pragma unroll
-                        for (int k = 0; k < VN; ++k) acc[b] = fmaf(w[k], a[k], acc[b]);
+                        for (int k = 0; k < VN; k += 4) {
+                            const float4 t = *reinterpret_cast<const float4*>(s_act + b * Hc + c + k);
+                            a[k] = t.x; a[k + 1] = t.y; a[k + 2] = t.z; a[k + 3] = t.w;
+                        }
+#pragma unroll
+                        for (int q = 0; q < ADA_RPW; ++q)
+#pragma unroll
+                            for (int k = 0; k < VN; ++k) acc[q][b] = fmaf(w[q][k], a[k], acc[q][b]);
                     }
                 }
             }
-            const int l = (int)(row / H6), o = (int)(row % H6);
-            const float bias = to_f<T>(b_ada[row]);
 #pragma unroll
-            for (int b = 0; b < ADA_BCH; ++b) {
-                if (b < nb) {
-                    const float v = warp_sum(acc[b]);
-                    if (lane == 0) mod[((size_t)l * B + (b0 + b)) * H6 + o] = v + bias;
+            for (int q = 0; q < ADA_RPW; ++q) {
+                const long long row = row0 + q;
+#pragma unroll
+                for (int b = 0; b < ADA_BCH; ++b) {
+                    if (b < nb) {
+                        const float v = warp_sum(acc[q][b]);
+                        if (lane == 0 && row < rows_total) {
+                            const int l = (int)(row / H6), o = (int)(row % H6);
+                            mod[((size_t)l * B + (b0 + b)) * H6 + o] = v + to_f<T>(b_ada[row]);
+                        }
+                    }
                 }
             }
         }
@@ -95,11 +115,32 @@ adaln_kernel(const T* __restrict__ cond, const T* __restrict__ w_ada, const T* _
 }
 
 // ---- gather + LayerNorm + modulation, one warp per active row --------------------------------
-constexpr int LN_THREADS = 256;
-constexpr int LN_MAXV = 16;        // float4 slots per lane: rows up to 32*4*16 = 2048 wide stay in registers
+// Pass 1 streams the row once (128-bit loads) and accumulates sum and sum of squares of (x - x0),
+// x0 = the row's first element, which keeps the one-pass variance well conditioned.  Pass 2 reads
+// the row again (it is still in L1/L2), normalises, modulates and writes 128-bit vectors.  Nothing
+// of the row is kept in registers, so many warps per SM hide the memory latency.
+constexpr int LN_THREADS = 128;
 
 template <typename T>
-__global__ void __launch_bounds__(LN_THREADS)
+__device__ __forceinline__ void ln_load4(const T* x_gather, const float* resid_in, size_t g_off, size_t r_off,
+                                         float* f) {
+    if (x_gather) {
+        if constexpr (sizeof(T) == 2) {
+            const uint2 u = *reinterpret_cast<const uint2*>(x_gather + g_off);
+            f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+            f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+        } else {
+            const float4 u = *reinterpret_cast<const float4*>(x_gather + g_off);
+            f[0] = u.x; f[1] = u.y; f[2] = u.z; f[3] = u.w;
+        }
+    } else {
+        const float4 u = *reinterpret_cast<const float4*>(resid_in + r_off);
+        f[0] = u.x; f[1] = u.y; f[2] = u.z; f[3] = u.w;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(LN_THREADS, 8)
 ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
                    float* __restrict__ resid_out, T* __restrict__ out, const int32_t* __restrict__ active_idx,
                    const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
@@ -110,64 +151,47 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
     for (int row = blockIdx.x * (LN_THREADS / 32) + warp; row < a_total; row += gridDim.x * (LN_THREADS / 32)) {
         const int tok = active_idx[row];
         const int b = tok / N;
-        float v[LN_MAXV][4];
-        float sum = 0.f;
+        const size_t g0 = (size_t)tok * H, r0 = (size_t)row * H;
+        const float x0 = x_gather ? to_f<T>(x_gather[g0]) : resid_in[r0];
+        float sum = 0.f, sq = 0.f;
+#pragma unroll 4
+        for (int i = 0; i < nv; ++i) {
+            const int c = (i * 32 + lane) * 4;
+            float v[4];
+            ln_load4<T>(x_gather, resid_in, g0 + c, r0 + c, v);
+            if (x_gather && resid_out)
+                *reinterpret_cast<float4*>(resid_out + r0 + c) = make_float4(v[0], v[1], v[2], v[3]);
 #pragma unroll
-        for (int i = 0; i < LN_MAXV; ++i) {
-            if (i < nv) {
-                const int c = (i * 32 + lane) * 4;
-                if (x_gather) {
-                    const T* src = x_gather + (size_t)tok * H + c;
-                    if constexpr (sizeof(T) == 2) {
-                        const uint2 u = *reinterpret_cast<const uint2*>(src);
-                        v[i][0] = __uint_as_float(u.x << 16); v[i][1] = __uint_as_float(u.x & 0xffff0000u);
-                        v[i][2] = __uint_as_float(u.y << 16); v[i][3] = __uint_as_float(u.y & 0xffff0000u);
-                    } else {
-                        const float4 u = *reinterpret_cast<const float4*>(src);
-                        v[i][0] = u.x; v[i][1] = u.y; v[i][2] = u.z; v[i][3] = u.w;
-                    }
-                    if (resid_out)
-                        *reinterpret_cast<float4*>(resid_out + (size_t)row * H + c) =
-                            make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
-                } else {
-                    const float4 u = *reinterpret_cast<const float4*>(resid_in + (size_t)row * H + c);
-                    v[i][0] = u.x; v[i][1] = u.y; v[i][2] = u.z; v[i][3] = u.w;
-                }
-                sum += (v[i][0] + v[i][1]) + (v[i][2] + v[i][3]);
-            }
+            for (int k = 0; k < 4; ++k) { const float d = v[k] - x0; sum += d; sq = fmaf(d, d, sq); }
         }
-        const float mean = warp_sum(sum) / (float)H;
-        float sq = 0.f;
-#pragma unroll
-        for (int i = 0; i < LN_MAXV; ++i) {
-            if (i < nv) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) { const float d = v[i][k] - mean; sq = fmaf(d, d, sq); }
-            }
-        }
-        const float rstd = rsqrtf(warp_sum(sq) / (float)H + ln_eps);
+        sum = warp_sum(sum);
+        sq = warp_sum(sq);
+        const float dm = sum / (float)H;                       // mean - x0
+        const float var = fmaxf(sq / (float)H - dm * dm, 0.f);
+        const float rstd = rsqrtf(var + ln_eps);
+        const float mean = x0 + dm;
         const float* sh = shift + (size_t)b * mod_stride;
         const float* sc = scale + (size_t)b * mod_stride;
-#pragma unroll
-        for (int i = 0; i < LN_MAXV; ++i) {
-            if (i < nv) {
-                const int c = (i * 32 + lane) * 4;
-                const float4 s4 = *reinterpret_cast<const float4*>(sc + c);
-                const float4 h4 = *reinterpret_cast<const float4*>(sh + c);
-                const float o0 = (v[i][0] - mean) * rstd * (1.f + s4.x) + h4.x;
-                const float o1 = (v[i][1] - mean) * rstd * (1.f + s4.y) + h4.y;
-                const float o2 = (v[i][2] - mean) * rstd * (1.f + s4.z) + h4.z;
-                const float o3 = (v[i][3] - mean) * rstd * (1.f + s4.w) + h4.w;
-                T* dst = out + (size_t)row * H + c;
-                if constexpr (sizeof(T) == 2) {
-                    const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
-                    uint2 u;
-                    u.x = *reinterpret_cast<const uint32_t*>(&p0);
-                    u.y = *reinterpret_cast<const uint32_t*>(&p1);
-                    *reinterpret_cast<uint2*>(dst) = u;
-                } else {
-                    *reinterpret_cast<float4*>(dst) = make_float4(o0, o1, o2, o3);
-                }
+#pragma unroll 4
+        for (int i = 0; i < nv; ++i) {
+            const int c = (i * 32 + lane) * 4;
+            float v[4];
+            ln_load4<T>(x_gather, resid_in, g0 + c, r0 + c, v);
+            const float4 s4 = __ldg(reinterpret_cast<const float4*>(sc + c));
+            const float4 h4 = __ldg(reinterpret_cast<const float4*>(sh + c));
+            const float o0 = (v[0] - mean) * rstd * (1.f + s4.x) + h4.x;
+            const float o1 = (v[1] - mean) * rstd * (1.f + s4.y) + h4.y;
+            const float o2 = (v[2] - mean) * rstd * (1.f + s4.z) + h4.z;
+            const float o3 = (v[3] - mean) * rstd * (1.f + s4.w) + h4.w;
+            T* dst = out + r0 + c;
+            if constexpr (sizeof(T) == 2) {
+                const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
+                uint2 u;
+                u.x = *reinterpret_cast<const uint32_t*>(&p0);
+                u.y = *reinterpret_cast<const uint32_t*>(&p1);
+                *reinterpret_cast<uint2*>(dst) = u;
+            } else {
+                *reinterpret_cast<float4*>(dst) = make_float4(o0, o1, o2, o3);
             }
         }
     }
@@ -228,8 +252,8 @@ cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* 
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
                                cudaStream_t st, int* n_launch) {
     const int rows_per_cta = LN_THREADS / 32;
-    const int grid = max(1, min((rows_cap + rows_per_cta - 1) / rows_per_cta, 148 * 8));
-    if (H % 128 == 0 && H <= 128 * LN_MAXV)
+    const int grid = max(1, min((rows_cap + rows_per_cta - 1) / rows_per_cta, 148 * 16));
+    if (H % 128 == 0)
         ln_modulate_kernel<T><<<grid, LN_THREADS, 0, st>>>(x_gather, resid_in, resid_out, out, active_idx, shift,
                                                           scale, mod_stride, N, H, ln_eps, ctl);
     else

@@ -133,14 +133,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 uint32_t r[32];
                 tmem_ld32(t_row + c0, r);
                 tmem_wait_ld();
-                if (valid) {
-#pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        const float v[4] = {__uint_as_float(r[4 * g]), __uint_as_float(r[4 * g + 1]),
-                                            __uint_as_float(r[4 * g + 2]), __uint_as_float(r[4 * g + 3])};
-                        epilogue4<__nv_bfloat16, KIND>(ep, row, n * BN + c0 + 4 * g, tok, v);
-                    }
-                }
+                if (valid) epilogue32<KIND>(ep, row, n * BN + c0, tok, r);
             }
             tc_fence_before();
             __syncwarp();
@@ -175,7 +168,7 @@ EncodeTiledFn encode_fn(std::string* err) {
     return fn;
 }
 
-int pick_bn(int n_out) { return (n_out % 256 == 0 && n_out >= 3072) ? 256 : 128; }
+int pick_bn(int n_out) { return (n_out % 256 == 0) ? 256 : 128; }
 
 }  // namespace
 
@@ -220,6 +213,7 @@ bool tc_supported(const fd_config& c, std::string* why) {
     auto bad = [&](const char* m) { if (why) *why = m; return false; };
     if (c.dtype != FD_BF16) return bad("tensor-core engine needs bf16 storage");
     if (c.hidden % 128 || c.mlp_dim % 128) return bad("hidden and mlp_dim must be multiples of 128");
+    if (c.cond_dim % 8) return bad("cond_dim must be a multiple of 8");
     return true;
 }
 
