@@ -155,6 +155,37 @@ fd_status fd_regional_step(fd_ctx* ctx, const void* x, const void* cond, const i
                            int32_t* active_idx_out, int32_t* cu_active_out, void* cuda_stream);
 
 /*
+ * The gate for callers that cannot allocate device memory (no counterpart in the paper; added for
+ * embedding).  Some hosts of this library may not call cudaMalloc at all: a plug-in running inside
+ * an inference server whose memory pool was sized and frozen at start-up, code on a latency-critical
+ * thread where an allocation would serialise the whole device, or a process that has already handed
+ * every byte of the GPU to its own arena.  Such a caller cannot provide the workspace fd_create
+ * wants, so this entry point needs neither a context nor a workspace: it computes exactly what
+ * fd_region_activity computes (same kernels, same argument meaning), with its per-region
+ * accumulators in a fixed array that is part of the library image.
+ *
+ *  - Limit: B * R <= FD_NOALLOC_MAX_REGION_SLOTS; larger problems are refused with FD_ERR_SHAPE
+ *    and nothing is launched.  The array (about 200 KB) is resident on every GPU that loads the
+ *    library, from load until the process exits.
+ *  - The first call on each device looks up the array's device address (with that device current).
+ *    Make that first call outside any stream capture.
+ *  - All calls on one device share the array and it keeps what the last call left in it; every
+ *    call clears the part it uses before use.  Two calls whose GPU work overlaps (different
+ *    streams without ordering, or different host threads) race on it: serialise them.
+ *  - No cudaMalloc / cudaFree or any other allocating routine is called, by this function or the
+ *    kernels it launches.
+ *  - eta and max_skip_k take the place of the values a context would hold.
+ *  - status_out: optional DEVICE int32 that receives 0, or FD_ERR_STATE if a label was outside
+ *    [0,R] (such tokens are skipped), in stream order; may be NULL.
+ */
+#define FD_NOALLOC_MAX_REGION_SLOTS 16384
+fd_status fd_region_activity_noalloc(const float* z_cur, const float* z_prev, const int32_t* labels, int B,
+                                     int N, int D, int R, const float* eps, float eta, int max_skip_k,
+                                     float* delta_state, int32_t* skip_count, uint8_t* prev_active,
+                                     float* score_out, float* weight_out, uint8_t* mask_out,
+                                     int32_t* status_out, void* cuda_stream);
+
+/*
  * Reads the device-side status word (synchronises `cuda_stream`).  Returns FD_OK, or the first
  * device-side problem recorded since the last poll (FD_ERR_STATE / FD_ERR_TIMEOUT), and clears it.
  */

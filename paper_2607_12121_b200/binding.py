@@ -21,7 +21,8 @@ FD_ENGINE_AUTO, FD_ENGINE_SIMT, FD_ENGINE_TC = 0, 1, 2
 
 EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region_activity",
            "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
-           "fd_profile_enable", "fd_profile_read"]
+           "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc"]
+FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
                "gemm_fc2", "partition"]
 
@@ -58,6 +59,9 @@ def _load() -> ctypes.CDLL:
     lib.fd_partition_regions.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, i32, vp, vp, vp]
     lib.fd_region_activity.restype = i32
     lib.fd_region_activity.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.fd_region_activity_noalloc.restype = i32
+    lib.fd_region_activity_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, i32, vp, vp, vp,
+                                               vp, vp, vp, vp, vp]
     lib.fd_regional_step.restype = i32
     lib.fd_regional_step.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.fd_poll_status.restype = i32
@@ -159,6 +163,19 @@ def fd_region_activity(ctx: Context, z_cur, z_prev, labels, R: int, eps, delta_s
     _check(ctx.handle, lib.fd_region_activity(
         ctx.handle, _ptr(z_cur), _ptr(z_prev), _ptr(labels), B, N, D, R, _ptr(eps), _ptr(delta_state),
         _ptr(skip_count), _ptr(prev_active), _ptr(score_out), _ptr(weight_out), _ptr(mask_out), _stream(stream)))
+
+
+def fd_region_activity_noalloc(z_cur, z_prev, labels, R: int, eps, eta: float, max_skip_k: int, delta_state,
+                               skip_count, prev_active, score_out, weight_out, mask_out, status_out=None,
+                               stream=None) -> None:
+    """The gate for callers that may not allocate device memory: no context, no workspace; the
+    scratch is a fixed array inside the library (B * R <= FD_NOALLOC_MAX_REGION_SLOTS).  Calls on
+    one device share that array, so they must not overlap on the GPU."""
+    B, N, D = z_cur.shape
+    _check(None, lib.fd_region_activity_noalloc(
+        _ptr(z_cur), _ptr(z_prev), _ptr(labels), B, N, D, R, _ptr(eps), float(eta), int(max_skip_k),
+        _ptr(delta_state), _ptr(skip_count), _ptr(prev_active), _ptr(score_out), _ptr(weight_out), _ptr(mask_out),
+        _ptr(status_out), _stream(stream)))
 
 
 def fd_regional_step(ctx: Context, x, cond, labels, mask, R: int, kv_cache, y, active_idx_out, cu_active_out,

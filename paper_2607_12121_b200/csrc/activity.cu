@@ -183,4 +183,51 @@ cudaError_t launch_activity(const float* z_cur, const float* z_prev, const int32
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Gate without a context or a workspace: the accumulators live in a fixed device array.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// per-(request, region) accumulators (sum of squares fp64, token count i32) and one status block
+constexpr size_t NOALLOC_BYTES = sizeof(Control) + 192 /*keeps the arrays 256-byte aligned*/ +
+                                 (size_t)FD_NOALLOC_MAX_REGION_SLOTS * (sizeof(double) + sizeof(int32_t));
+static __device__ __align__(256) unsigned char g_gate_scratch[NOALLOC_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+void* g_scratch_addr[MAX_DEVICES];          // device address of g_gate_scratch, per device
+
+}  // namespace
+
+cudaError_t noalloc_gate(const float* z_cur, const float* z_prev, const int32_t* labels, int B, int N, int D,
+                         int R, const float* eps, float eta, int K, float* delta, int32_t* skip_count,
+                         uint8_t* prev_active, float* score, float* weight, uint8_t* mask, int32_t* status_out,
+                         cudaStream_t st) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    if (!g_scratch_addr[dev]) {
+        // In host code the array's name is only a handle; the address the kernels need comes from
+        // the runtime, looked up once per device while that device is current.
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_gate_scratch);
+        if (e != cudaSuccess) return e;
+        g_scratch_addr[dev] = p;
+    }
+    unsigned char* base = static_cast<unsigned char*>(g_scratch_addr[dev]);
+    Control* ctl = reinterpret_cast<Control*>(base);
+    double* acc_ss = reinterpret_cast<double*>(base + 256);
+    int32_t* acc_cnt = reinterpret_cast<int32_t*>(base + 256 + (size_t)FD_NOALLOC_MAX_REGION_SLOTS * sizeof(double));
+    // the array keeps whatever the previous call left: everything read before written starts at zero
+    e = cudaMemsetAsync(base, 0, 256 + (size_t)B * R * sizeof(double), st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(acc_cnt, 0, (size_t)B * R * sizeof(int32_t), st);
+    if (e != cudaSuccess) return e;
+    int nl = 0;
+    e = launch_activity(z_cur, z_prev, labels, B, N, D, R, eps, delta, skip_count, prev_active, score, weight, mask,
+                        eta, K, acc_ss, acc_cnt, ctl, st, &nl);
+    if (e != cudaSuccess) return e;
+    if (status_out) e = cudaMemcpyAsync(status_out, &ctl->status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
+    return e;
+}
+
 }  // namespace fd

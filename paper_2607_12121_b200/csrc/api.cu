@@ -354,6 +354,28 @@ fd_status fd_region_activity(fd_ctx* c, const float* z_cur, const float* z_prev,
     return FD_OK;
 }
 
+fd_status fd_region_activity_noalloc(const float* z_cur, const float* z_prev, const int32_t* labels, int B, int N,
+                                     int D, int R, const float* eps, float eta, int max_skip_k, float* delta_state,
+                                     int32_t* skip_count, uint8_t* prev_active, float* score_out, float* weight_out,
+                                     uint8_t* mask_out, int32_t* status_out, void* cuda_stream) {
+    auto fail = [](fd_status s, const char* m) { g_create_error = m; return s; };
+    if (!z_cur || !z_prev || !labels || !eps || !delta_state || !skip_count || !prev_active || !score_out ||
+        !weight_out || !mask_out)
+        return fail(FD_ERR_INVALID_ARG, "fd_region_activity_noalloc: null pointer argument");
+    if (B < 1 || N < 1 || D < 1 || R < 1) return fail(FD_ERR_SHAPE, "fd_region_activity_noalloc: B, N, D, R must be positive");
+    if ((long long)B * R > FD_NOALLOC_MAX_REGION_SLOTS)
+        return fail(FD_ERR_SHAPE, "fd_region_activity_noalloc: B * R exceeds FD_NOALLOC_MAX_REGION_SLOTS");
+    if (!(eta >= 0.f) || max_skip_k < 0) return fail(FD_ERR_INVALID_ARG, "fd_region_activity_noalloc: bad eta / max_skip_k");
+    cudaError_t e = noalloc_gate(z_cur, z_prev, labels, B, N, D, R, eps, eta, max_skip_k, delta_state, skip_count,
+                                 prev_active, score_out, weight_out, mask_out, status_out,
+                                 static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) {
+        g_create_error = std::string("fd_region_activity_noalloc: ") + cudaGetErrorString(e);
+        return FD_ERR_CUDA;
+    }
+    return FD_OK;
+}
+
 fd_status fd_regional_step(fd_ctx* c, const void* x, const void* cond, const int32_t* labels, const uint8_t* mask,
                            int B, int N, int R, void* kv_cache, void* y, int32_t* active_idx_out,
                            int32_t* cu_active_out, void* cuda_stream) {

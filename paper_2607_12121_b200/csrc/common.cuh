@@ -96,6 +96,11 @@ cudaError_t launch_activity(const float* z_cur, const float* z_prev, const int32
                             int K, double* acc_ss, int32_t* acc_cnt, Control* ctl, cudaStream_t st,
                             int* n_launch);
 
+cudaError_t noalloc_gate(const float* z_cur, const float* z_prev, const int32_t* labels, int B, int N, int D,
+                         int R, const float* eps, float eta, int K, float* delta, int32_t* skip_count,
+                         uint8_t* prev_active, float* score, float* weight, uint8_t* mask, int32_t* status_out,
+                         cudaStream_t st);
+
 // compact.cu
 cudaError_t launch_compact(const uint8_t* mask, const int32_t* labels, int B, int N, int R,
                            int32_t* active_idx, int32_t* cu_active, int32_t* block_counts, QTile* tiles,
