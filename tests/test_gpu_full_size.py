@@ -1,0 +1,95 @@
+"""Parity at the benchmark configurations' full shapes, in the launch configuration bench.py uses
+(engine AUTO).  The caches start from seeded random contents (any cached state is a valid input);
+the oracle refreshes K/V for every active row and finishes attention + MLP for a sample of rows."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+import paper_2607_12121_b200 as fd
+from harness import StepBuffers, dev, gpu_step, host, labels_for, make_ctx, max_abs, rel_l2, tdtype
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, REL_L2 = 3e-2, 1e-2
+
+
+def _full_shape_block(name, seed, fractions, n_sample=160):
+    wl = gen.workload(name).replace(L=1)
+    B, N, H = wl.B, wl.N, wl.H
+    labels = labels_for(wl, seed)
+    w = gen.block_weights(wl, seed, n_blocks=1)
+    inp = gen.step_inputs(wl, seed, labels)
+    mask = gen.region_mask(wl, seed, fractions)
+    rng = np.random.default_rng(seed)
+    kv0 = gen.round_bf16(0.5 * rng.standard_normal((1, B, 2, N, H), dtype=np.float32))
+    y0 = gen.round_bf16(rng.standard_normal((B, N, H), dtype=np.float32))
+
+    ctx = make_ctx(wl, w, n_blocks=1)
+    buf = StepBuffers(wl, 1)
+    dt = tdtype(wl)
+    buf.kv.copy_(dev(kv0, dt))
+    buf.y.copy_(dev(y0, dt))
+    idx, cu = gpu_step(ctx, wl, dev(inp["x_cur"], dt), dev(inp["cond"], dt), dev(labels), dev(mask), buf)
+
+    o_idx, o_cu = oracle.compact(mask, labels, wl.R)
+    assert np.array_equal(idx, o_idx) and np.array_equal(cu, o_cu)
+    u = np.ascontiguousarray(inp["x_cur"].reshape(B * N, H)[o_idx])
+    mod = oracle.adaln(inp["cond"], w["w_ada"][0], w["b_ada"][0])
+    kv_ref = kv0[0].copy()
+    pick = np.unique(np.concatenate([np.linspace(0, o_idx.size - 1, n_sample).astype(np.int32),
+                                     o_cu[1:] - 1, o_cu[:-1]]).clip(0, o_idx.size - 1)).astype(np.int32)
+    out = oracle.regional_block(u, o_idx, mod, w, 0, kv_ref, wl.heads, finish=pick)
+
+    act = np.zeros(B * N, bool)
+    act[o_idx] = True
+    a2 = act.reshape(B, N)
+    kv = host(buf.kv)[0]
+    for s in range(2):
+        assert max_abs(kv[:, s][a2], kv_ref[:, s][a2]) <= MAX_ABS
+        assert rel_l2(kv[:, s][a2], kv_ref[:, s][a2]) <= REL_L2
+        assert np.array_equal(kv[:, s][~a2], kv0[0][:, s][~a2])
+    y = host(buf.y).reshape(B * N, H)
+    rows = o_idx[pick]
+    assert max_abs(y[rows], out[pick]) <= MAX_ABS
+    assert rel_l2(y[rows], out[pick]) <= REL_L2
+    assert np.array_equal(y[~act], y0.reshape(B * N, H)[~act])
+    return ctx
+
+
+def test_audio_full_shape_ragged_batch():
+    wl = gen.workload("audio")
+    _full_shape_block("audio", 21, gen.request_fractions(wl, 21))
+
+
+def test_image_full_shape():
+    _full_shape_block("image", 22, [0.25, 0.5, 0.75, 1.0])
+
+
+def test_mmdit_full_shape_with_text_tokens():
+    _full_shape_block("mmdit", 23, [0.34, 0.76])
+
+
+def test_video_full_shape():
+    _full_shape_block("video", 24, [0.3], n_sample=96)
+
+
+def test_full_depth_drift_on_narrow_twin():
+    """All 24 blocks on a narrow twin: bf16 rounding must not accumulate past the tolerance."""
+    wl = gen.workload("audio_tc").replace(L=24)
+    labels = gen.uniform_labels(wl)
+    w = gen.block_weights(wl, 31)
+    inp = gen.step_inputs(wl, 31, labels)
+    ctx = make_ctx(wl, w)
+    buf = StepBuffers(wl, wl.L)
+    dt = tdtype(wl)
+    B, N, H = wl.B, wl.N, wl.H
+    kv_ref = np.zeros((wl.L, B, 2, N, H), np.float32)
+    y_ref = np.zeros((B, N, H), np.float32)
+    for x_np, mask in ((inp["x_prev"], np.ones((B, wl.R), np.uint8)), (inp["x_cur"], gen.region_mask(wl, 2, [0.5] * B))):
+        idx, _ = gpu_step(ctx, wl, dev(x_np, dt), dev(inp["cond"], dt), dev(labels), dev(mask), buf)
+        oracle.regional_step(x_np, inp["cond"], labels, mask, w, kv_ref, y_ref, wl.heads, wl.R)
+    y = host(buf.y)
+    print("24-block drift: max_abs %.4f rel_l2 %.5f max|y| %.2f" % (max_abs(y, y_ref), rel_l2(y, y_ref), np.abs(y_ref).max()))
+    assert max_abs(y, y_ref) <= MAX_ABS and rel_l2(y, y_ref) <= REL_L2
