@@ -234,6 +234,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     wl = gen.workload(args.workload)
+    if args.blocks:
+        wl = wl.replace(L=args.blocks)
     if wl.labels == "partition":
         raise SystemExit("bench workloads with partitioner labels are run through --workload audio for now")
     seed = args.seed + 17 * rank                 # every rank owns its own batch of requests (weak scaling)
@@ -438,6 +440,7 @@ def main():
     ap.add_argument("--fraction", type=float, default=None, help="same active fraction for every request")
     ap.add_argument("--seed", type=int, default=1000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--blocks", type=int, default=0, help="override the block count (profiling captures only)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -150,6 +150,141 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// CTA-pair variant: a cluster of two CTAs computes a 256 x 256 tile with tcgen05.mma.cta_group::2.
+// Each CTA stages its own 128 activation rows and one half (128 rows) of the weight tile, so the
+// shared-memory traffic per MMA drops by a third and the weight half is fetched once per pair.
+// The MMA is issued by one thread of the pair's first CTA; completion is broadcast to both CTAs'
+// barriers with a multicast commit.  No TMA load is multicast: every CTA fetches its own tiles.
+// ------------------------------------------------------------------------------------------------
+constexpr int PAIR_BN = 256;
+constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_B_BYTES = 128 * BK * 2;           // this CTA's half of the weight tile
+constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_BYTES;
+constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + 1024 + 256;
+
+template <int KIND>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int n_out,
+                    int k_dim, EpiParams ep, Control* ctl) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + PAIR_STAGES * A_TILE_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + PAIR_STAGES * PAIR_STAGE_BYTES);   // used in the first CTA
+    uint64_t* empty = full + PAIR_STAGES;                                                 // one set per CTA
+    uint64_t* tfull = empty + PAIR_STAGES;                                                // one set per CTA
+    uint64_t* tempty = tfull + 2;                                                         // used in the first CTA
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int a_total = ctl->a_total;
+    const int m_pairs = (a_total + 2 * BM - 1) / (2 * BM);
+    const int n_tiles = n_out / PAIR_BN;
+    const int total_tiles = m_pairs * n_tiles;
+    const int k_tiles = k_dim / BK;
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < PAIR_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tm_a);
+        prefetch_tmap(&tm_b);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, 2 * PAIR_BN);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                      // both CTAs' barriers exist before anything remote arrives
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
+                const int m = tile % m_pairs, n = tile / m_pairs;
+                for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+                    const int s = it % PAIR_STAGES;
+                    const uint32_t ph = (it / PAIR_STAGES) & 1;
+                    if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t bar = map_to_cta(smem_u32(&full[s]), 0);     // the first CTA's barrier counts both halves
+                    if (rank == 0) mbar_expect_tx(&full[s], 2 * PAIR_STAGE_BYTES);
+                    tma_load_2d_pair(sA + s * A_TILE_BYTES, &tm_a, kt * BK, m * 2 * BM + (int)rank * BM, bar);
+                    tma_load_2d_pair(sB + s * PAIR_B_BYTES, &tm_b, kt * BK, n * PAIR_BN + (int)rank * 128, bar);
+                }
+            }
+            if (!ok) report(ctl, FD_ERR_TIMEOUT, 700 + (int)blockIdx.x);
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = idesc_bf16(2 * BM, PAIR_BN, 0, 0);
+            uint32_t it = 0, t_it = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
+                const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
+                if (!mbar_wait(&tempty[acc], aph ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d = tmem_base + acc * PAIR_BN;
+                for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+                    const int s = it % PAIR_STAGES;
+                    const uint32_t ph = (it / PAIR_STAGES) & 1;
+                    if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t da = smem_desc(smem_u32(sA + s * A_TILE_BYTES), 16, 1024, SWZ_128B);
+                    const uint64_t db = smem_desc(smem_u32(sB + s * PAIR_B_BYTES), 16, 1024, SWZ_128B);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        mma_bf16_ss_pair(d, da + 2 * k, db + 2 * k, idesc, (kt | k) != 0);
+                    mma_commit_pair(&empty[s], 0x3);          // frees the stage in both CTAs
+                }
+                if (ok) mma_commit_pair(&tfull[acc], 0x3);    // both CTAs' epilogues may read their rows
+            }
+            if (!ok) report(ctl, FD_ERR_TIMEOUT, 800 + (int)blockIdx.x);
+        }
+    } else {
+        const int quad = warp & 3;
+        uint32_t t_it = 0;
+        bool ok = true;
+        for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
+            const int m = tile % m_pairs, n = tile / m_pairs;
+            const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
+            if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const int row = m * 2 * BM + (int)rank * BM + quad * 32 + lane;
+            const bool valid = row < a_total;
+            const int tok = valid ? ep.active_idx[row] : 0;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
+#pragma unroll 1
+            for (int c0 = 0; c0 < PAIR_BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(t_row + c0, r);
+                tmem_wait_ld();
+                if (valid) epilogue32<KIND>(ep, row, n * PAIR_BN + c0, tok, r);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty[acc]), 0));
+        }
+        if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 900 + (int)blockIdx.x);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                      // neither CTA leaves while its peer may still signal it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, 2 * PAIR_BN);
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -197,12 +332,14 @@ bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* di
 struct GemmSpec {
     CUtensorMap a;              // activation operand
     int n_out, k, bn;
+    bool pair;                  // CTA-pair kernel (256 x 256 tiles); weight boxes are then 128 rows
 };
 
 struct TcPlan {
     fd_config cfg;
     TcBuffers buf;
     int sm_count;
+    int pair_ctas;              // grid of the CTA-pair kernel: 2 x co-resident clusters
     GemmSpec spec[4];
     CUtensorMap* w_maps;        // [L][4]
     // attention (filled by the attention part)
@@ -234,6 +371,8 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         const int v = atoi(lim);
         if (v > 0 && v < p->sm_count) p->sm_count = v;
     }
+    bool use_pair = true;       // switch: FD_TC_PAIR=0 keeps every GEMM on the single-CTA kernel
+    if (const char* v = getenv("FD_TC_PAIR")) use_pair = atoi(v) != 0;
     const int H = cfg.hidden, M = cfg.mlp_dim;
     const int n_out[4] = {3 * H, H, M, H};
     const int kdim[4] = {H, H, H, M};
@@ -246,13 +385,14 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         s.n_out = n_out[g];
         s.k = kdim[g];
         s.bn = pick_bn(n_out[g]);
+        s.pair = use_pair && (n_out[g] % PAIR_BN == 0);
         const uint64_t dims[2] = {(uint64_t)kdim[g], (uint64_t)buf.Mcap};
         const uint64_t strides[1] = {(uint64_t)kdim[g] * 2};
         const uint32_t box[2] = {BK, BM};
         ok = encode_tmap_bf16(&s.a, a_base[g], 2, dims, strides, box, 128, err);
         for (int l = 0; l < cfg.n_blocks && ok; ++l) {
             const uint64_t wd[2] = {(uint64_t)kdim[g], (uint64_t)n_out[g]};
-            const uint32_t wb[2] = {BK, (uint32_t)s.bn};
+            const uint32_t wb[2] = {BK, s.pair ? 128u : (uint32_t)s.bn};
             void* base = const_cast<char*>(w_base[g]) + (size_t)l * n_out[g] * kdim[g] * 2;
             ok = encode_tmap_bf16(&p->w_maps[(size_t)l * 4 + g], base, 2, wd, strides, wb, 128, err);
         }
@@ -265,10 +405,34 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         FD_SET_SMEM(EPI_QKV, 128) FD_SET_SMEM(EPI_QKV, 256) FD_SET_SMEM(EPI_RESID, 128) FD_SET_SMEM(EPI_RESID, 256)
         FD_SET_SMEM(EPI_GELU, 128) FD_SET_SMEM(EPI_GELU, 256)
 #undef FD_SET_SMEM
+#define FD_SET_PAIR(K)                                                                                     \
+    if (e == cudaSuccess)                                                                                  \
+        e = cudaFuncSetAttribute(tc_gemm_pair_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM);
+        FD_SET_PAIR(EPI_QKV) FD_SET_PAIR(EPI_RESID) FD_SET_PAIR(EPI_GELU)
+#undef FD_SET_PAIR
         if (e != cudaSuccess) {
             ok = false;
             if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
         }
+    }
+    p->pair_ctas = p->sm_count & ~1;
+    if (ok) {
+        // as many CTA pairs as the device can keep resident at once (a pair needs both SMs of a TPC)
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3(p->sm_count & ~1);
+        lc.blockDim = dim3(GEMM_THREADS);
+        lc.dynamicSmemBytes = PAIR_SMEM;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        lc.attrs = at;
+        lc.numAttrs = 1;
+        int n_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, tc_gemm_pair_kernel<EPI_GELU>, &lc) == cudaSuccess && n_clusters > 0)
+            p->pair_ctas = min(p->sm_count & ~1, 2 * n_clusters);
+        else
+            cudaGetLastError();
+        if (p->pair_ctas < 2) p->pair_ctas = 2;
     }
     if (ok && tc_attention_supported(cfg)) {
         p->attn = tc_attention_plan_create(cfg, buf, err);
@@ -297,6 +461,17 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
     const CUtensorMap& wm = p->w_maps[(size_t)blk * 4 + kind];
     Control* c = const_cast<Control*>(ctl);
     const int grid = p->sm_count;
+    if (s.pair) {
+        const int pgrid = max(2, min(grid & ~1, p->pair_ctas));
+        if (kind == TC_GEMM_QKV)
+            tc_gemm_pair_kernel<EPI_QKV><<<pgrid, GEMM_THREADS, PAIR_SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c);
+        else if (kind == TC_GEMM_FC1)
+            tc_gemm_pair_kernel<EPI_GELU><<<pgrid, GEMM_THREADS, PAIR_SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c);
+        else
+            tc_gemm_pair_kernel<EPI_RESID><<<pgrid, GEMM_THREADS, PAIR_SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c);
+        ++*n_launch;
+        return cudaGetLastError();
+    }
 #define FD_LAUNCH(K, N) \
     tc_gemm_kernel<K, N><<<grid, GEMM_THREADS, GemmCfg<N>::SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c)
     if (kind == TC_GEMM_QKV) {
