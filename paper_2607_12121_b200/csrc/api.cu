@@ -25,7 +25,7 @@ thread_local std::string g_create_error;
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-    size_t control, acc_ss, acc_cnt, block_counts, tiles, mod, resid, act, q, o, g, part, total;
+    size_t control, acc_ss, acc_cnt, block_counts, tiles, ada_act, mod, resid, act, q, o, g, part, total;
     int Mcap, q_ld, tile_cap;
 };
 
@@ -62,6 +62,7 @@ Layout make_layout(const fd_config& c) {
     l.acc_cnt = take(BR * sizeof(int32_t));
     l.block_counts = take((size_t)c.max_batch * ((c.max_tokens + 2047) / 2048 + 1) * sizeof(int32_t));
     l.tiles = take((size_t)l.tile_cap * sizeof(QTile));
+    l.ada_act = take((size_t)2 * ((c.max_batch + 7) / 8 * 8) * c.cond_dim * 2);   // SiLU(cond): bf16 head + remainder
     l.mod = take((size_t)c.n_blocks * c.max_batch * 6 * c.hidden * sizeof(float));
     l.resid = take((size_t)l.Mcap * c.hidden * sizeof(float));
     l.act = take((size_t)l.Mcap * c.hidden * es);
@@ -162,7 +163,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     FD_TRY(FD_PROF_COMPACT, launch_compact(mask, labels, B, N, R, active_idx, cu_active, c->at<int32_t>(l.block_counts), tiles,
                           c->tile_rows, ctl, st, &nl));
     FD_TRY(FD_PROF_ADALN, launch_adaln<T>(cond, static_cast<const T*>(c->w.w_ada), static_cast<const T*>(c->w.b_ada), mod, L, B, H,
-                           Hc, st, &nl));
+                           Hc, c->ws + l.ada_act, st, &nl));
     const int max_tiles = B * ((N + c->tile_rows - 1) / c->tile_rows);
     for (int blk = 0; blk < L; ++blk) {
         const float* mod_b = mod + (size_t)blk * B * 6 * H;
@@ -280,7 +281,7 @@ fd_status fd_create(const fd_config* cfg, const fd_weights* weights, void* works
     c->launches = 0;
     c->tc = nullptr;
     // control block and gate accumulators start at zero; the compact buffers start finite
-    e = cudaMemset(workspace, 0, lay.mod);
+    e = cudaMemset(workspace, 0, lay.ada_act);
     if (e == cudaSuccess) e = cudaMemset(c->ws + lay.resid, 0, lay.part - lay.resid);
     if (e == cudaSuccess && use_tc) {
         TcBuffers tb{};

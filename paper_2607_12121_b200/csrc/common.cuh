@@ -109,7 +109,7 @@ cudaError_t launch_compact(const uint8_t* mask, const int32_t* labels, int B, in
 // rowops.cu
 template <typename T>
 cudaError_t launch_adaln(const T* cond, const T* w_ada, const T* b_ada, float* mod, int L, int B, int H,
-                         int Hc, cudaStream_t st, int* n_launch);
+                         int Hc, void* act_scratch, cudaStream_t st, int* n_launch);
 template <typename T>
 cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
                                const int32_t* active_idx, const float* shift, const float* scale,

@@ -114,6 +114,85 @@ adaln_kernel(const T* __restrict__ cond, const T* __restrict__ w_ada, const T* _
     }
 }
 
+// ---- adaLN on bf16 weights: a skinny contraction [L*6H, Hc] x [Hc, B] that must stream W_ada at HBM
+// speed.  CUDA cores would be arithmetic-bound here (8 FMAs per weight element), so the products go
+// through mma.sync m16n8k16 (16 weight rows x 8 requests per instruction).  SiLU(cond) is split into
+// a bf16 head and a bf16 remainder, so the activations keep fp32-level accuracy.
+__global__ void __launch_bounds__(256)
+adaln_act_kernel(const __nv_bfloat16* __restrict__ cond, __nv_bfloat16* __restrict__ act, int B, int B8, int Hc) {
+    // act[part][b][c], part 0 = head, part 1 = remainder; requests b >= B are zero
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= B8 * Hc) return;
+    const int b = i / Hc;
+    float v = 0.f;
+    if (b < B) { const float x = __bfloat162float(cond[i]); v = x / (1.0f + __expf(-x)); }
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    act[i] = hi;
+    act[(size_t)B8 * Hc + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+__device__ __forceinline__ void mma_16x8x16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                            uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+constexpr int ADM_WARPS = 8;
+constexpr int ADM_UNROLL = 4;       // 32-wide k blocks in flight per lane
+
+__global__ void __launch_bounds__(ADM_WARPS * 32)
+adaln_mma_kernel(const __nv_bfloat16* __restrict__ act, const __nv_bfloat16* __restrict__ w_ada,
+                 const __nv_bfloat16* __restrict__ b_ada, float* __restrict__ mod, long long rows_total, int B,
+                 int B8, int H6, int Hc) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const long long strip = (long long)blockIdx.x * ADM_WARPS + warp;       // 16 weight rows
+    const long long row0 = strip * 16;
+    if (row0 >= rows_total) return;
+    const long long ra = min(row0 + g, rows_total - 1), rb = min(row0 + g + 8, rows_total - 1);
+    const uint4* wa = reinterpret_cast<const uint4*>(w_ada + (size_t)ra * Hc) + t;   // 8 elements at k = 32 blk + 8 t
+    const uint4* wb = reinterpret_cast<const uint4*>(w_ada + (size_t)rb * Hc) + t;
+    for (int b0 = 0; b0 < B8; b0 += 8) {
+        // lane (g, t) supplies the activations of request b0 + g for the same 8 k positions
+        const uint4* ah = reinterpret_cast<const uint4*>(act + (size_t)(b0 + g) * Hc) + t;
+        const uint4* al = reinterpret_cast<const uint4*>(act + (size_t)B8 * Hc + (size_t)(b0 + g) * Hc) + t;
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        const int n_blk = Hc / 32;
+        for (int kb = 0; kb < n_blk; kb += ADM_UNROLL) {
+            uint4 va[ADM_UNROLL], vb[ADM_UNROLL], xh[ADM_UNROLL], xl[ADM_UNROLL];
+#pragma unroll
+            for (int u = 0; u < ADM_UNROLL; ++u) {
+                const int k4 = min(kb + u, n_blk - 1) * 4;
+                va[u] = __ldg(wa + k4);
+                vb[u] = __ldg(wb + k4);
+                xh[u] = __ldg(ah + k4);
+                xl[u] = __ldg(al + k4);
+            }
+#pragma unroll
+            for (int u = 0; u < ADM_UNROLL; ++u) {
+                if (kb + u < n_blk) {
+                    // the 8 k positions of this lane feed two k16 products: (x,y) then (z,w)
+                    mma_16x8x16(c, va[u].x, vb[u].x, va[u].y, vb[u].y, xh[u].x, xh[u].y);
+                    mma_16x8x16(c, va[u].z, vb[u].z, va[u].w, vb[u].w, xh[u].z, xh[u].w);
+                    mma_16x8x16(c, va[u].x, vb[u].x, va[u].y, vb[u].y, xl[u].x, xl[u].y);
+                    mma_16x8x16(c, va[u].z, vb[u].z, va[u].w, vb[u].w, xl[u].z, xl[u].w);
+                }
+            }
+        }
+        // c0,c1: row g, requests 2t, 2t+1;  c2,c3: row g + 8
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const long long row = row0 + g + (q >= 2 ? 8 : 0);
+            const int b = b0 + 2 * t + (q & 1);
+            if (row < rows_total && b < B) {
+                const int l = (int)(row / H6), o = (int)(row % H6);
+                mod[((size_t)l * B + b) * H6 + o] = c[q] + __bfloat162float(b_ada[row]);
+            }
+        }
+    }
+}
+
 // ---- gather + LayerNorm + modulation, one warp per active row --------------------------------
 // Pass 1 streams the row once (128-bit loads) and accumulates sum and sum of squares of (x - x0),
 // x0 = the row's first element, which keeps the one-pass variance well conditioned.  Pass 2 reads
@@ -233,8 +312,21 @@ ln_modulate_generic_kernel(const T* __restrict__ x_gather, const float* __restri
 
 template <typename T>
 cudaError_t launch_adaln(const T* cond, const T* w_ada, const T* b_ada, float* mod, int L, int B, int H,
-                         int Hc, cudaStream_t st, int* n_launch) {
+                         int Hc, void* act_scratch, cudaStream_t st, int* n_launch) {
     const long long rows = (long long)L * 6 * H;
+    if constexpr (sizeof(T) == 2) {
+        if (Hc % 32 == 0 && act_scratch) {
+            const int B8 = (B + 7) / 8 * 8;
+            __nv_bfloat16* act = static_cast<__nv_bfloat16*>(act_scratch);
+            adaln_act_kernel<<<(B8 * Hc + 255) / 256, 256, 0, st>>>(cond, act, B, B8, Hc);
+            ++*n_launch;
+            const long long strips = (rows + 15) / 16;
+            adaln_mma_kernel<<<(unsigned)((strips + ADM_WARPS - 1) / ADM_WARPS), ADM_WARPS * 32, 0, st>>>(
+                act, w_ada, b_ada, mod, rows, B, B8, 6 * H, Hc);
+            ++*n_launch;
+            return cudaGetLastError();
+        }
+    }
     const int grid = (int)((rows + ADA_ROWS - 1) / ADA_ROWS);
     const size_t smem = (size_t)min(B, ADA_BCH) * Hc * sizeof(float);
     if (smem > 48 * 1024) {
@@ -263,10 +355,10 @@ cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* 
     return cudaGetLastError();
 }
 
-template cudaError_t launch_adaln<float>(const float*, const float*, const float*, float*, int, int, int, int,
+template cudaError_t launch_adaln<float>(const float*, const float*, const float*, float*, int, int, int, int, void*,
                                          cudaStream_t, int*);
 template cudaError_t launch_adaln<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*,
-                                                 float*, int, int, int, int, cudaStream_t, int*);
+                                                 float*, int, int, int, int, void*, cudaStream_t, int*);
 template cudaError_t launch_ln_modulate<float>(const float*, const float*, float*, float*, const int32_t*,
                                                const float*, const float*, int, int, int, int, float, const Control*,
                                                cudaStream_t, int*);
