@@ -236,20 +236,33 @@ def run_ours(args):
     wl = gen.workload(args.workload)
     if args.blocks:
         wl = wl.replace(L=args.blocks)
-    if wl.labels == "partition":
-        raise SystemExit("bench workloads with partitioner labels are run through --workload audio for now")
     seed = args.seed + 17 * rank                 # every rank owns its own batch of requests (weak scaling)
     dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     B, N, H, M, R, L, D = wl.B, wl.N, wl.H, wl.M, wl.R, wl.L, wl.D
-
-    labels_np = gen.uniform_labels(wl)
-    inp = gen.step_inputs(wl, seed, labels_np)
-    fr = gen.request_fractions(wl, seed) if args.fraction is None else np.full(B, args.fraction)
-    lat = gen.latent_pair(wl, seed, labels_np, fractions=fr)
+    default_fraction = {"image": 0.5, "mmdit": 0.55, "video": 0.45}
 
     weights = device_weights(wl, seed, dev)
     cfg = fd.make_config(wl)
     ctx = fd.fd_create(cfg, weights, device=dev)
+
+    if wl.labels == "partition":
+        # labels come from the library's own partitioner on the synthetic early-step attention map
+        amap = torch.from_numpy(gen.saliency_map(wl, seed)).to(dev)
+        lab_grid = torch.empty((B, wl.n_grid), dtype=torch.int32, device=dev)
+        fd.fd_partition_regions(ctx, amap, R, lab_grid, None, None, wl.m_min, wl.m_max)
+        fd.fd_poll_status(ctx)
+        labels_np = np.concatenate([lab_grid.cpu().numpy(), np.full((B, wl.n_text), R, np.int32)], axis=1)
+        labels_np = np.ascontiguousarray(labels_np)
+    else:
+        labels_np = gen.uniform_labels(wl)
+    inp = gen.step_inputs(wl, seed, labels_np)
+    if args.fraction is not None:
+        fr = np.full(B, args.fraction)
+    elif wl.name in default_fraction:
+        fr = np.full(B, default_fraction[wl.name])
+    else:
+        fr = gen.request_fractions(wl, seed)
+    lat = gen.latent_pair(wl, seed, labels_np, fractions=fr)
 
     def pin(a, tdt=None):
         t = torch.from_numpy(np.ascontiguousarray(a))
