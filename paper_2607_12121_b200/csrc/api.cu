@@ -52,7 +52,8 @@ Layout make_layout(const fd_config& c) {
     const size_t es = esize(c);
     const size_t BR = (size_t)c.max_batch * c.max_regions;
     l.Mcap = (int)align_up((size_t)c.max_batch * c.max_tokens, 128) + 128;
-    l.q_ld = c.hidden;
+    // room for Q with padded heads (tensor-core attention stores head dim 72 as 80)
+    l.q_ld = c.dtype == FD_BF16 ? c.n_heads * tc_attention_head_pad(c.head_dim) : c.hidden;
     const int min_tile = 16;
     l.tile_cap = c.max_batch * ((c.max_tokens + min_tile - 1) / min_tile + 1);
     size_t off = 0;
@@ -185,6 +186,10 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         ep.bias = static_cast<const T*>(c->w.b_qkv) + (size_t)blk * 3 * H;
         ep.q = q;
         ep.q_ld = l.q_ld;
+        if (c->use_tc_attn && tc_attention_head_pad(cf.head_dim) != cf.head_dim) {
+            ep.q_head_dim = cf.head_dim;
+            ep.q_head_pad = tc_attention_head_pad(cf.head_dim);
+        }
         ep.kv = kv_b;
         if (c->use_tc)
             FD_TRY(FD_PROF_GEMM_QKV, tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));

@@ -69,6 +69,8 @@ struct EpiParams {
     // EPI_QKV
     void* q;                   // [Mcap, q_ld] storage type
     int32_t q_ld;
+    int32_t q_head_dim;        // 0, or the head dim when each head of Q is stored padded to q_head_pad columns
+    int32_t q_head_pad;
     void* kv;                  // this block's cache [B,2,N,H] storage type
     // EPI_RESID
     float* resid;              // [Mcap,H] fp32, in/out

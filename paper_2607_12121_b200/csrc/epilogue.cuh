@@ -109,6 +109,15 @@ __device__ __forceinline__ void epilogue32(const EpiParams& ep, int row, int col
         const int sec = col / ep.H, c = col - sec * ep.H;
         T* dst;
         if (sec == 0) {
+            if (ep.q_head_dim) {             // heads padded (72 -> 80): place every 8-column group inside its head
+                T* qrow = reinterpret_cast<T*>(ep.q) + (size_t)row * ep.q_ld;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int c8 = c + 8 * q, hd = c8 / ep.q_head_dim;
+                    store8_bf16(qrow + hd * ep.q_head_pad + (c8 - hd * ep.q_head_dim), v + 8 * q);
+                }
+                return;
+            }
             dst = reinterpret_cast<T*>(ep.q) + (size_t)row * ep.q_ld + c;
         } else {
             const int b = tok / ep.N, j = tok - b * ep.N;

@@ -31,11 +31,18 @@ constexpr int ATT_THREADS = 352;
 constexpr int QROWS = 128, KEYS = 128;
 constexpr int SUB_BYTES = 128 * 64 * 2;          // one [128 x 64] bf16 sub-tile, 128-byte rows
 
+constexpr int TAIL_BYTES = 128 * 16 * 2;         // one [128 x 16] bf16 sub-tile, 32-byte rows (head dim 72 only)
+
+// Head dim 72 runs as 80: a 64-wide sub-tile (128-byte swizzle) plus a 16-wide one (32-byte swizzle).
+// Q is stored with every head padded to 80 columns of which the last 8 are zero, so the 8 columns
+// the 16-wide K sub-tile reads past its head contribute nothing; the matching 8 columns of O are
+// never stored.
 template <int D> struct AttCfg {
-    static constexpr int SUBS = D / 64;
-    static constexpr int TILE_BYTES = SUBS * SUB_BYTES;
+    static constexpr int DP = D == 72 ? 80 : D;                       // head dim as the MMAs see it
+    static constexpr int SUBS = D / 64;                               // 64-wide sub-tiles
+    static constexpr int TILE_BYTES = SUBS * SUB_BYTES + (D == 72 ? TAIL_BYTES : 0);
     // K/V rings deep enough that a tile is requested several tile periods before it is needed
-    static constexpr int STAGES = D == 64 ? 5 : 2;
+    static constexpr int STAGES = D == 128 ? 2 : (D == 72 ? 4 : 5);
     static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 3584;
 };
 
@@ -55,9 +62,11 @@ constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384, TMEM_COLS = 512;
 template <int D>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
+                    const __grid_constant__ CUtensorMap tm_q_tail, const __grid_constant__ CUtensorMap tm_kv_tail,
                     __nv_bfloat16* __restrict__ o, int o_ld, const QTile* __restrict__ tiles, int heads, int N,
                     float scale_log2, Control* ctl) {
     using Cfg = AttCfg<D>;
+    constexpr int DP = Cfg::DP;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int TILE_BYTES = Cfg::TILE_BYTES;
     extern __shared__ __align__(1024) uint8_t smem[];    // 128-byte swizzled tiles need 1024-byte alignment
@@ -133,7 +142,9 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 mbar_expect_tx(&q_full[qs], TILE_BYTES);
 #pragma unroll
                 for (int sb = 0; sb < Cfg::SUBS; ++sb)
-                    tma_load_2d(sQ + qs * TILE_BYTES + sb * SUB_BYTES, &tm_q, head * D + sb * 64, t.row0, &q_full[qs]);
+                    tma_load_2d(sQ + qs * TILE_BYTES + sb * SUB_BYTES, &tm_q, head * DP + sb * 64, t.row0, &q_full[qs]);
+                if constexpr (D == 72)
+                    tma_load_2d(sQ + qs * TILE_BYTES + SUB_BYTES, &tm_q_tail, head * DP + 64, t.row0, &q_full[qs]);
                 for (int j = 0; j < n_kv; ++j, ++gk) {
                     const int s = gk % STAGES;
                     const uint32_t ph = ((gk / STAGES) & 1) ^ 1;
@@ -143,12 +154,18 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int sb = 0; sb < Cfg::SUBS; ++sb)
                         tma_load_3d(sK + s * TILE_BYTES + sb * SUB_BYTES, &tm_kv, head * D + sb * 64, j * KEYS,
                                     t.b * 2 + 0, &k_full[s]);
+                    if constexpr (D == 72)
+                        tma_load_3d(sK + s * TILE_BYTES + SUB_BYTES, &tm_kv_tail, head * D + 64, j * KEYS, t.b * 2 + 0,
+                                    &k_full[s]);
                     if (!mbar_wait(&v_empty[s], ph, abort_flag)) { ok = false; break; }
                     mbar_expect_tx(&v_full[s], TILE_BYTES);
 #pragma unroll
                     for (int sb = 0; sb < Cfg::SUBS; ++sb)
                         tma_load_3d(sV + s * TILE_BYTES + sb * SUB_BYTES, &tm_kv, head * D + sb * 64, j * KEYS,
                                     t.b * 2 + 1, &v_full[s]);
+                    if constexpr (D == 72)
+                        tma_load_3d(sV + s * TILE_BYTES + SUB_BYTES, &tm_kv_tail, head * D + 64, j * KEYS, t.b * 2 + 1,
+                                    &v_full[s]);
                 }
             }
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 400 + (int)blockIdx.x);
@@ -173,11 +190,14 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const uint32_t d = tmem_base + COL_S + (g & 1) * 128;
                     const uint32_t k_addr = smem_u32(sK + s * TILE_BYTES);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
+                    for (int ks = 0; ks < Cfg::SUBS * 4; ++ks) {
                         const uint32_t off = (ks / 4) * SUB_BYTES + (ks % 4) * 32;
                         mma_bf16_ss(d, smem_desc(q_addr + off, 16, 1024, SWZ_128B),
                                     smem_desc(k_addr + off, 16, 1024, SWZ_128B), idesc_qk, ks != 0);
                     }
+                    if constexpr (D == 72)      // columns 64..79: 32-byte rows, 8-row groups 256 bytes apart
+                        mma_bf16_ss(d, smem_desc(q_addr + SUB_BYTES, 16, 256, SWZ_32B),
+                                    smem_desc(k_addr + SUB_BYTES, 16, 256, SWZ_32B), idesc_qk, 1);
                     mma_commit(&k_empty[s]);
                     mma_commit(&s_full[g & 1]);
                     if (j == n_kv - 1) mma_commit(&q_empty[qs]);
@@ -188,7 +208,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     } else if (warp == 2) {
         // ---------------------------------------------------------------- O += P V issuer
         if (lane == 0) {
-            constexpr uint32_t idesc_pv = idesc_bf16(QROWS, D, 0, 1);      // V: head dim contiguous (N-major)
+            constexpr uint32_t idesc_pv = idesc_bf16(QROWS, D == 72 ? 64 : D, 0, 1);   // V: head dim contiguous (N-major)
+            constexpr uint32_t idesc_pv_tail = idesc_bf16(QROWS, 16, 0, 1);
             uint32_t g = 0;
             bool ok = true;
             int item_i = 0;
@@ -207,6 +228,9 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         // 16 keys further: 16 rows of 128 bytes; the second 64-wide half of V sits SUB_BYTES away
                         mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
                                     (j | ks) != 0);
+                        if constexpr (D == 72)  // output columns 64..79 from the 16-wide sub-tile (16 keys = 512 bytes)
+                            mma_bf16_ts(d + 64, a + ks * 8, smem_desc(v_addr + SUB_BYTES + ks * 512, 16, 256, SWZ_32B),
+                                        idesc_pv_tail, (j | ks) != 0);
                     }
                     mma_commit(&v_empty[s]);
                     mma_commit(&pv_done[g & 1]);
@@ -220,7 +244,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int half = (warp - 3) >> 2;                     // which 64 keys of a tile / which half of O
         const int r = quad * 32 + lane;                       // query row inside the tile
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-        constexpr int DH = D / 2;                             // output columns this thread owns
+        // output columns this thread owns: [half * DH, half * DH + DH), and for head dim 72 thread 0 also 64..79
+        constexpr int DH = D == 72 ? 32 : D / 2;
         uint32_t g0 = 0;
         bool ok = true;
         int item_i = 0;
@@ -274,6 +299,16 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
                             tmem_st32(lane_addr + COL_O + half * DH + c * 32, orr);
                         }
+                        if constexpr (D == 72) {
+                            if (half == 0) {
+                                uint32_t ot[16];
+                                tmem_ld16(lane_addr + COL_O + 64, ot);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) ot[i] = __float_as_uint(__uint_as_float(ot[i]) * f);
+                                tmem_st16(lane_addr + COL_O + 64, ot);
+                            }
+                        }
                         tmem_wait_st();
                     }
                 }
@@ -326,6 +361,21 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                 }
             }
+            if constexpr (D == 72) {
+                if (half == 0) {                          // columns 64..71 of the head
+                    uint32_t ot[8];
+                    tmem_ld8(lane_addr + COL_O + 64, ot);
+                    tmem_wait_ld();
+                    if (r < t.rows) {
+                        uint4 u;
+                        u.x = pack_bf16(__uint_as_float(ot[0]) * inv, __uint_as_float(ot[1]) * inv);
+                        u.y = pack_bf16(__uint_as_float(ot[2]) * inv, __uint_as_float(ot[3]) * inv);
+                        u.z = pack_bf16(__uint_as_float(ot[4]) * inv, __uint_as_float(ot[5]) * inv);
+                        u.w = pack_bf16(__uint_as_float(ot[6]) * inv, __uint_as_float(ot[7]) * inv);
+                        *reinterpret_cast<uint4*>(o + (size_t)(t.row0 + r) * o_ld + head * D + 64) = u;
+                    }
+                }
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(o_free);
@@ -343,22 +393,24 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 }
 
 struct AttnPlan {
-    CUtensorMap q_map;
-    int heads, dh, H, q_ld;
+    CUtensorMap q_map, q_tail_map;
+    int heads, dh, dp, H, q_ld;
     void* o;
 };
 
 }  // namespace
 
 bool tc_attention_supported(const fd_config& c) {
-    return c.dtype == FD_BF16 && (c.head_dim == 64 || c.head_dim == 128);
+    return c.dtype == FD_BF16 && (c.head_dim == 64 || c.head_dim == 128 || c.head_dim == 72);
 }
 int tc_attention_tile_rows() { return QROWS; }
+int tc_attention_head_pad(int head_dim) { return head_dim == 72 ? 80 : head_dim; }
 
 void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::string* err) {
     AttnPlan* a = new AttnPlan();
     a->heads = cfg.n_heads;
     a->dh = cfg.head_dim;
+    a->dp = tc_attention_head_pad(cfg.head_dim);
     a->H = cfg.hidden;
     a->q_ld = buf.q_ld;
     a->o = buf.o;
@@ -366,10 +418,14 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
     const uint64_t strides[1] = {(uint64_t)buf.q_ld * 2};
     const uint32_t box[2] = {64, QROWS};
     bool ok = encode_tmap_bf16(&a->q_map, buf.q, 2, dims, strides, box, 128, err);
+    const uint32_t box_tail[2] = {16, QROWS};
+    if (ok) ok = encode_tmap_bf16(&a->q_tail_map, buf.q, 2, dims, strides, box_tail, 32, err);
     cudaError_t e = cudaSuccess;
     if (ok) e = cudaFuncSetAttribute(tc_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<64>::SMEM);
     if (ok && e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<128>::SMEM);
+    if (ok && e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_attention_kernel<72>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<72>::SMEM);
     if (e != cudaSuccess) {
         ok = false;
         if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
@@ -384,22 +440,25 @@ cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, c
                          const Control* ctl, cudaStream_t st, int* n_launch) {
     AttnPlan* a = static_cast<AttnPlan*>(tc_plan_attn(p));
     if (!a) return cudaErrorNotSupported;
-    CUtensorMap kv_map;
+    CUtensorMap kv_map, kv_tail_map;
     const uint64_t dims[3] = {(uint64_t)a->H, (uint64_t)N, (uint64_t)B * 2};
     const uint64_t strides[2] = {(uint64_t)a->H * 2, (uint64_t)N * a->H * 2};
     const uint32_t box[3] = {64, KEYS, 1};
+    const uint32_t box_tail[3] = {16, KEYS, 1};
     std::string err;
     if (!encode_tmap_bf16(&kv_map, kv_block, 3, dims, strides, box, 128, &err)) return cudaErrorInvalidValue;
+    if (!encode_tmap_bf16(&kv_tail_map, kv_block, 3, dims, strides, box_tail, 32, &err)) return cudaErrorInvalidValue;
     const int grid = max(1, min(tc_plan_sm_count(p), max_tiles * a->heads));
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)a->dh);
     Control* c = const_cast<Control*>(ctl);
     __nv_bfloat16* o = static_cast<__nv_bfloat16*>(a->o);
-    if (a->dh == 64)
-        tc_attention_kernel<64><<<grid, ATT_THREADS, AttCfg<64>::SMEM, st>>>(a->q_map, kv_map, o, a->H, tiles, a->heads, N,
-                                                                           scale_log2, c);
-    else
-        tc_attention_kernel<128><<<grid, ATT_THREADS, AttCfg<128>::SMEM, st>>>(a->q_map, kv_map, o, a->H, tiles, a->heads,
-                                                                             N, scale_log2, c);
+#define FD_ATT(DD)                                                                                                  \
+    tc_attention_kernel<DD><<<grid, ATT_THREADS, AttCfg<DD>::SMEM, st>>>(a->q_map, kv_map, a->q_tail_map, kv_tail_map, o, \
+                                                                          a->H, tiles, a->heads, N, scale_log2, c)
+    if (a->dh == 64) FD_ATT(64);
+    else if (a->dh == 128) FD_ATT(128);
+    else FD_ATT(72);
+#undef FD_ATT
     ++*n_launch;
     return cudaGetLastError();
 }
