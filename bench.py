@@ -221,22 +221,20 @@ def device_weights(wl, seed, device):
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     import gen
     import paper_2607_12121_b200 as fd
+    from paper_2607_12121_b200 import replicas
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rep = replicas.from_env()
+    rank, world, local = rep.rank, rep.world, rep.local_rank
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init(rep, "nccl", dev)
 
     wl = gen.workload(args.workload)
     if args.blocks:
         wl = wl.replace(L=args.blocks)
-    seed = args.seed + 17 * rank                 # every rank owns its own batch of requests (weak scaling)
+    seed = replicas.replica_seed(rep, args.seed)     # every rank owns its own batch of requests (weak scaling)
     dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     B, N, H, M, R, L, D = wl.B, wl.N, wl.H, wl.M, wl.R, wl.L, wl.D
     default_fraction = {"image": 0.5, "mmdit": 0.55, "video": 0.45}
@@ -301,8 +299,7 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier(rep)
         torch.cuda.synchronize()
 
     def timed(fn, steps):
@@ -313,11 +310,7 @@ def run_ours(args):
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = replicas.max_over_ranks(rep, e0.elapsed_time(e1), dev)
         return ms / steps
 
     # warm-up: one dense step on the previous step's tokens fills kv / y, then W gated steps
@@ -372,8 +365,9 @@ def run_ours(args):
     step_flops = L * sum(fl.values())
     dense_flops = L * sum(block_flops([N] * B, N, H, M).values())
     peaks, peak_kind = load_peaks()
-    value = world * step_flops / (ms_reg * 1e-3) / 1e12
-    e2e_value = world * step_flops / (ms_e2e * 1e-3) / 1e12
+    flops_all = replicas.sum_over_ranks(rep, step_flops, dev)          # every replica has its own active set
+    value = replicas.job_throughput(flops_all, ms_reg) / 1e12
+    e2e_value = replicas.job_throughput(flops_all, ms_e2e) / 1e12
 
     # per-kernel breakdown of the profiled pass; the dominant group feeds the roofline object
     es = 2 if wl.dtype == "bf16" else 4
@@ -439,8 +433,7 @@ def run_ours(args):
                                     "kind": "oracle", "sample": text, "seconds": dt_cpu}
         print(json.dumps(line))
     fd.fd_destroy(ctx)
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown(rep)
 
 
 def main():
