@@ -392,10 +392,13 @@ def run_ours(args):
     dom = max((k for k in breakdown if k in fl), key=lambda k: breakdown[k]["ms_per_step"])
     tensor_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
     traffic = None
-    tp = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tp):
+    tp = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.txt")
+    if os.path.exists(tp) and wl.name == "audio" and not args.blocks:
         with open(tp) as f:
-            traffic = json.load(f).get(dom)
+            for ln in f:
+                parts = ln.split()
+                if len(parts) == 2 and parts[0] == dom:
+                    traffic = int(parts[1])
     roofline = {"kernel": dom, "bound": "tensor", "achieved": breakdown[dom]["tflops"], "peak": tensor_peak,
                 "unit": "TFLOP/s", "frac": breakdown[dom]["tflops"] / tensor_peak, "traffic": traffic,
                 "peak_source": peak_kind + " (sustained bf16 matmul; the kernel is timed inside a long step)",
