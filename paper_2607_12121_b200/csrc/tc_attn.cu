@@ -11,6 +11,11 @@
 //                tcgen05.ld of the scores, row maximum swapped through shared memory, running maximum
 //                with lazy rescaling of O (only when it grew by more than 2^8), exp2, P written to
 //                TMEM as packed bf16; at the end O / l is stored as bf16
+// At head dim 64 there is room in TMEM for two output accumulators, and the two threads of a row do
+// not talk to each other inside the key loop at all: thread h keeps its own running maximum and row
+// sum over "its" 64 keys of every tile, its P half feeds a product into its own accumulator O_h, and
+// the halves drift out of phase so that one warp's exp2 phase overlaps the other's TMEM traffic.  The
+// partial results are merged at the end, O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1), a_h = 2^(m_h - m).
 // The two MMA issuers run independently, so waiting for the softmax of tile g never delays the
 // score product of tile g+1.  Keys past N in the last tile are zero-filled by TMA and masked.
 #include <cuda_bf16.h>
@@ -67,6 +72,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     float scale_log2, Control* ctl) {
     using Cfg = AttCfg<D>;
     constexpr int DP = Cfg::DP;
+    constexpr bool SPLIT = D == 64;                      // per-half accumulators, no exchange in the key loop
     constexpr int STAGES = Cfg::STAGES;
     constexpr int TILE_BYTES = Cfg::TILE_BYTES;
     extern __shared__ __align__(1024) uint8_t smem[];    // 128-byte swizzled tiles need 1024-byte alignment
@@ -79,9 +85,9 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint64_t* v_full = k_empty + STAGES;
     uint64_t* v_empty = v_full + STAGES;
     uint64_t* s_full = v_empty + STAGES;      // [2]  score tile ready
-    uint64_t* p_full = s_full + 2;            // [2]  P written (and the score buffer consumed)
-    uint64_t* pv_done = p_full + 2;           // [2]  the product that read this P buffer has completed
-    uint64_t* q_full = pv_done + 2;           // [2]
+    uint64_t* p_full = s_full + 2;            // [2][2]  P written (and the score buffer consumed); [buffer][half], half 1 only if SPLIT
+    uint64_t* pv_done = p_full + 4;           // [2][2]  the product that read this P buffer (half) has completed
+    uint64_t* q_full = pv_done + 4;           // [2]
     uint64_t* q_empty = q_full + 2;           // [2]
     uint64_t* o_free = q_empty + 2;
     uint64_t* x_bar = o_free + 1;             // [4 quadrants][2]: the two threads of a row swap their partial maxima
@@ -108,9 +114,10 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 8); mbar_init(&pv_done[i], 1);
+            mbar_init(&s_full[i], 1);
             mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1);
         }
+        for (int i = 0; i < 4; ++i) { mbar_init(&p_full[i], SPLIT ? 4 : 8); mbar_init(&pv_done[i], 1); }
         for (int i = 0; i < 8; ++i) mbar_init(&x_bar[i], 64);
         for (int i = 0; i < 4; ++i) mbar_init(&l_bar[i], 64);
         mbar_init(o_free, 8);
@@ -185,7 +192,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const int s = g % STAGES;
                     if (!mbar_wait(&k_full[s], (g / STAGES) & 1, abort_flag)) { ok = false; break; }
                     // the score buffer is free once the softmax has finished the tile that used it last
-                    if (g >= 2 && !mbar_wait(&p_full[g & 1], ((g - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if (g >= 2 && !mbar_wait(&p_full[(g & 1) * 2], ((g - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if (SPLIT && g >= 2 && !mbar_wait(&p_full[(g & 1) * 2 + 1], ((g - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d = tmem_base + COL_S + (g & 1) * 128;
                     const uint32_t k_addr = smem_u32(sK + s * TILE_BYTES);
@@ -218,11 +226,28 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const int s = g % STAGES;
                     if (!mbar_wait(&v_full[s], (g / STAGES) & 1, abort_flag)) { ok = false; break; }
                     if (j == 0 && item_i > 0 && !mbar_wait(o_free, (item_i - 1) & 1, abort_flag)) { ok = false; break; }
-                    if (!mbar_wait(&p_full[g & 1], (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                    const uint32_t v_addr = smem_u32(sV + s * TILE_BYTES);
+                    if constexpr (SPLIT) {
+                        // keys 0..63 of the tile feed O_0, keys 64..127 feed O_1, each as soon as its P half is there
+                        for (int hh = 0; hh < 2 && ok; ++hh) {
+                            if (!mbar_wait(&p_full[(g & 1) * 2 + hh], (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                            const uint32_t d = tmem_base + COL_O + hh * 64;
+                            const uint32_t a = tmem_base + COL_P + (g & 1) * 64 + hh * 32;
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + (hh * 4 + ks) * 2048, SUB_BYTES, 1024, SWZ_128B),
+                                            idesc_pv, (j | ks) != 0);
+                            mma_commit(&pv_done[(g & 1) * 2 + hh]);
+                        }
+                        if (!ok) break;
+                        mma_commit(&v_empty[s]);
+                        continue;
+                    }
+                    if (!mbar_wait(&p_full[(g & 1) * 2], (g >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d = tmem_base + COL_O;
                     const uint32_t a = tmem_base + COL_P + (g & 1) * 64;
-                    const uint32_t v_addr = smem_u32(sV + s * TILE_BYTES);
 #pragma unroll
                     for (int ks = 0; ks < KEYS / 16; ++ks) {
                         // 16 keys further: 16 rows of 128 bytes; the second 64-wide half of V sits SUB_BYTES away
@@ -233,155 +258,288 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                         idesc_pv_tail, (j | ks) != 0);
                     }
                     mma_commit(&v_empty[s]);
-                    mma_commit(&pv_done[g & 1]);
+                    mma_commit(&pv_done[(g & 1) * 2]);
                 }
             }
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 550 + (int)blockIdx.x);
         }
     } else {
         // ---------------------------------------------------------------- softmax
-        const int quad = warp & 3;
-        const int half = (warp - 3) >> 2;                     // which 64 keys of a tile / which half of O
-        const int r = quad * 32 + lane;                       // query row inside the tile
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-        // output columns this thread owns: [half * DH, half * DH + DH), and for head dim 72 thread 0 also 64..79
-        constexpr int DH = D == 72 ? 32 : D / 2;
-        uint32_t g0 = 0;
-        bool ok = true;
-        int item_i = 0;
-        const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
-        for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
-            const QTile t = tiles[w % n_tiles];
-            const int head = w / n_tiles;
-            float m = -INFINITY, l = 0.f;
-            for (int j = 0; j < n_kv && ok; ++j) {
-                const uint32_t g = g0 + j, bs = g & 1;
-                if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                uint32_t sr[64];
-                tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64, sr);
-                tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + 32, sr + 32);
-                tmem_wait_ld();
-                if (j == n_kv - 1 && rem < KEYS) {
+        if constexpr (SPLIT) {
+            const int quad = warp & 3;
+            const int half = (warp - 3) >> 2;                     // which 64 keys of every tile, and which accumulator
+            const int r = quad * 32 + lane;                       // query row inside the tile
+            const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+            const uint32_t o_addr = lane_addr + COL_O + half * 64;
+            uint32_t g0 = 0;
+            bool ok = true;
+            int item_i = 0;
+            const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
+            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
+                const QTile t = tiles[w % n_tiles];
+                const int head = w / n_tiles;
+                float m = -INFINITY, l = 0.f;
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    const uint32_t g = g0 + j, bs = g & 1;
+                    if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    uint32_t sr[64];
+                    tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64, sr);
+                    tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + 32, sr + 32);
+                    tmem_wait_ld();
+                    const bool tail = j == n_kv - 1 && rem < KEYS;
+                    if (tail) {
 #pragma unroll
-                    for (int i = 0; i < 64; ++i) if (half * 64 + i >= rem) sr[i] = 0xff800000u;          // -inf
-                }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                        for (int i = 0; i < 64; ++i) if (half * 64 + i >= rem) sr[i] = 0xff800000u;      // -inf
+                    }
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < 64; i += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(sr[i]));
-                    mx1 = fmaxf(mx1, __uint_as_float(sr[i + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(sr[i + 2]));
-                    mx3 = fmaxf(mx3, __uint_as_float(sr[i + 3]));
-                }
-                float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                // row maximum over all 128 keys: swap partial maxima with the row's other thread
-                s_xmax[bs * 256 + half * 128 + r] = mx;
-                mbar_arrive(&x_bar[quad * 2 + bs]);
-                if (!mbar_wait(&x_bar[quad * 2 + bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
-                mx = fmaxf(mx, s_xmax[bs * 256 + (half ^ 1) * 128 + r]);
-                if (j == 0) {
-                    m = mx;
-                } else {
-                    const bool need = (mx - m) * scale_log2 > 8.0f;
-                    if (__any_sync(0xffffffffu, need)) {
-                        // all earlier P V products must have landed before O is rescaled
-                        if (!mbar_wait(&pv_done[(g - 1) & 1], ((g - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
-                        const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
-                        if (need) { l *= f; m = mx; }
+                    for (int i = 0; i < 64; i += 4) {
+                        mx0 = fmaxf(mx0, __uint_as_float(sr[i]));
+                        mx1 = fmaxf(mx1, __uint_as_float(sr[i + 1]));
+                        mx2 = fmaxf(mx2, __uint_as_float(sr[i + 2]));
+                        mx3 = fmaxf(mx3, __uint_as_float(sr[i + 3]));
+                    }
+                    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                    // a half with no valid key in the last tile keeps its state (mx = -inf, every p = 0);
+                    // both conditions below are the same for all rows of the warp
+                    const bool no_keys = tail && half * 64 >= rem;
+                    if (j == 0) {
+                        m = mx;
+                    } else if (!no_keys) {
+                        const bool need = (mx - m) * scale_log2 > 8.0f;
+                        if (__any_sync(0xffffffffu, need)) {
+                            // this half's earlier P V products must have landed before O_h is rescaled
+                            if (!mbar_wait(&pv_done[((g - 1) & 1) * 2 + half], ((g - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                            const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
+                            if (need) { l *= f; m = mx; }
 #pragma unroll
-                        for (int c = 0; c < DH / 32; ++c) {
-                            uint32_t orr[32];
-                            tmem_ld32(lane_addr + COL_O + half * DH + c * 32, orr);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
-                            tmem_st32(lane_addr + COL_O + half * DH + c * 32, orr);
-                        }
-                        if constexpr (D == 72) {
-                            if (half == 0) {
-                                uint32_t ot[16];
-                                tmem_ld16(lane_addr + COL_O + 64, ot);
+                            for (int c = 0; c < 2; ++c) {
+                                uint32_t orr[32];
+                                tmem_ld32(o_addr + c * 32, orr);
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int i = 0; i < 16; ++i) ot[i] = __float_as_uint(__uint_as_float(ot[i]) * f);
-                                tmem_st16(lane_addr + COL_O + 64, ot);
+                                for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
+                                tmem_st32(o_addr + c * 32, orr);
                             }
+                            tmem_wait_st();
                         }
-                        tmem_wait_st();
                     }
-                }
-                const float mb = m * scale_log2;
-                uint32_t pk[32];
-                float su0 = 0.f, su1 = 0.f, su2 = 0.f, su3 = 0.f;
+                    const float mb = (m == -INFINITY ? 0.f : m) * scale_log2;
+                    uint32_t pk[32];
+                    float su0 = 0.f, su1 = 0.f, su2 = 0.f, su3 = 0.f;
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -mb));
-                    const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -mb));
-                    const float p2 = ex2(fmaf(__uint_as_float(sr[2 * i + 2]), scale_log2, -mb));
-                    const float p3 = ex2(fmaf(__uint_as_float(sr[2 * i + 3]), scale_log2, -mb));
-                    su0 += p0; su1 += p1; su2 += p2; su3 += p3;
-                    pk[i] = pack_bf16(p0, p1);
-                    pk[i + 1] = pack_bf16(p2, p3);
+                    for (int i = 0; i < 32; i += 2) {
+                        const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -mb));
+                        const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -mb));
+                        const float p2 = ex2(fmaf(__uint_as_float(sr[2 * i + 2]), scale_log2, -mb));
+                        const float p3 = ex2(fmaf(__uint_as_float(sr[2 * i + 3]), scale_log2, -mb));
+                        su0 += p0; su1 += p1; su2 += p2; su3 += p3;
+                        pk[i] = pack_bf16(p0, p1);
+                        pk[i + 1] = pack_bf16(p2, p3);
+                    }
+                    l += (su0 + su1) + (su2 + su3);
+                    // this half of the P buffer is free once the product that read it two tiles ago has completed
+                    if (g >= 2 && !mbar_wait(&pv_done[bs * 2 + half], ((g >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                    tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pk);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&p_full[bs * 2 + half]);
                 }
-                l += (su0 + su1) + (su2 + su3);
-                // the P buffer is free once the product that read it two tiles ago has completed
-                if (g >= 2 && !mbar_wait(&pv_done[bs], ((g >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
-                tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pk);
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&p_full[bs]);
-            }
-            if (!ok) break;
-            // epilogue: O / l for the rows of this tile (l = the two halves' partial sums)
-            const uint32_t gl = g0 + n_kv - 1;
-            s_xsum[half * 128 + r] = l;
-            mbar_arrive(&l_bar[quad]);
-            if (!mbar_wait(&l_bar[quad], item_i & 1, abort_flag)) { ok = false; break; }
-            const float inv = 1.0f / (l + s_xsum[(half ^ 1) * 128 + r]);
-            if (!mbar_wait(&pv_done[gl & 1], (gl >> 1) & 1, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            __nv_bfloat16* dst = o + (size_t)(t.row0 + r) * o_ld + head * D + half * DH;
-#pragma unroll
-            for (int c = 0; c < DH / 32; ++c) {
-                uint32_t orr[32];
-                tmem_ld32(lane_addr + COL_O + half * DH + c * 32, orr);
+                if (!ok) break;
+                // merge the two halves' partial results and store the row
+                s_xmax[half * 128 + r] = m;
+                s_xsum[half * 128 + r] = l;
+                mbar_arrive(&l_bar[quad]);
+                if (!mbar_wait(&l_bar[quad], item_i & 1, abort_flag)) { ok = false; break; }
+                const float m_o = s_xmax[(half ^ 1) * 128 + r], l_o = s_xsum[(half ^ 1) * 128 + r];
+                const float m_all = fmaxf(m, m_o);                // half 0 always has a valid key, so this is finite
+                const float a_me = m == -INFINITY ? 0.f : ex2((m - m_all) * scale_log2);
+                const float a_ot = m_o == -INFINITY ? 0.f : ex2((m_o - m_all) * scale_log2);
+                const float inv = 1.0f / (a_me * l + a_ot * l_o);
+                const float w_0 = (half == 0 ? a_me : a_ot) * inv, w_1 = (half == 0 ? a_ot : a_me) * inv;   // weights of O_0, O_1
+                // every product of this item must have landed: the last tile, both halves
+                const uint32_t ge = g0 + n_kv - 1;
+                if (!mbar_wait(&pv_done[(ge & 1) * 2], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&pv_done[(ge & 1) * 2 + 1], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                // this thread stores columns [32 half, 32 half + 32) of the head
+                __nv_bfloat16* dst = o + (size_t)(t.row0 + r) * o_ld + head * D + half * 32;
+                uint32_t o0[32], o1[32];
+                tmem_ld32(lane_addr + COL_O + half * 32, o0);
+                tmem_ld32(lane_addr + COL_O + 64 + half * 32, o1);
                 tmem_wait_ld();
                 if (r < t.rows) {
+                    float v[32];
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
+                    for (int i = 0; i < 32; ++i) {
+                        // a zero weight must also silence whatever an untouched accumulator holds
+                        const float x0 = w_0 != 0.f ? __uint_as_float(o0[i]) * w_0 : 0.f;
+                        const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
+                        v[i] = x0 + x1;
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
                         uint4 u;
-                        u.x = pack_bf16(__uint_as_float(orr[8 * v + 0]) * inv, __uint_as_float(orr[8 * v + 1]) * inv);
-                        u.y = pack_bf16(__uint_as_float(orr[8 * v + 2]) * inv, __uint_as_float(orr[8 * v + 3]) * inv);
-                        u.z = pack_bf16(__uint_as_float(orr[8 * v + 4]) * inv, __uint_as_float(orr[8 * v + 5]) * inv);
-                        u.w = pack_bf16(__uint_as_float(orr[8 * v + 6]) * inv, __uint_as_float(orr[8 * v + 7]) * inv);
-                        *reinterpret_cast<uint4*>(dst + c * 32 + v * 8) = u;
+                        u.x = pack_bf16(v[8 * q + 0], v[8 * q + 1]);
+                        u.y = pack_bf16(v[8 * q + 2], v[8 * q + 3]);
+                        u.z = pack_bf16(v[8 * q + 4], v[8 * q + 5]);
+                        u.w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
+                        *reinterpret_cast<uint4*>(dst + q * 8) = u;
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(o_free);
+                g0 += n_kv;
             }
-            if constexpr (D == 72) {
-                if (half == 0) {                          // columns 64..71 of the head
-                    uint32_t ot[8];
-                    tmem_ld8(lane_addr + COL_O + 64, ot);
+            if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 650 + (int)blockIdx.x);
+        } else {
+            const int quad = warp & 3;
+            const int half = (warp - 3) >> 2;                     // which 64 keys of a tile / which half of O
+            const int r = quad * 32 + lane;                       // query row inside the tile
+            const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+            // output columns this thread owns: [half * DH, half * DH + DH), and for head dim 72 thread 0 also 64..79
+            constexpr int DH = D == 72 ? 32 : D / 2;
+            uint32_t g0 = 0;
+            bool ok = true;
+            int item_i = 0;
+            const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
+            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
+                const QTile t = tiles[w % n_tiles];
+                const int head = w / n_tiles;
+                float m = -INFINITY, l = 0.f;
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    const uint32_t g = g0 + j, bs = g & 1;
+                    if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    uint32_t sr[64];
+                    tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64, sr);
+                    tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + 32, sr + 32);
+                    tmem_wait_ld();
+                    if (j == n_kv - 1 && rem < KEYS) {
+    #pragma unroll
+                        for (int i = 0; i < 64; ++i) if (half * 64 + i >= rem) sr[i] = 0xff800000u;          // -inf
+                    }
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+    #pragma unroll
+                    for (int i = 0; i < 64; i += 4) {
+                        mx0 = fmaxf(mx0, __uint_as_float(sr[i]));
+                        mx1 = fmaxf(mx1, __uint_as_float(sr[i + 1]));
+                        mx2 = fmaxf(mx2, __uint_as_float(sr[i + 2]));
+                        mx3 = fmaxf(mx3, __uint_as_float(sr[i + 3]));
+                    }
+                    float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                    // row maximum over all 128 keys: swap partial maxima with the row's other thread
+                    s_xmax[bs * 256 + half * 128 + r] = mx;
+                    mbar_arrive(&x_bar[quad * 2 + bs]);
+                    if (!mbar_wait(&x_bar[quad * 2 + bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                    mx = fmaxf(mx, s_xmax[bs * 256 + (half ^ 1) * 128 + r]);
+                    if (j == 0) {
+                        m = mx;
+                    } else {
+                        const bool need = (mx - m) * scale_log2 > 8.0f;
+                        if (__any_sync(0xffffffffu, need)) {
+                            // all earlier P V products must have landed before O is rescaled
+                            if (!mbar_wait(&pv_done[((g - 1) & 1) * 2], ((g - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                            const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
+                            if (need) { l *= f; m = mx; }
+    #pragma unroll
+                            for (int c = 0; c < DH / 32; ++c) {
+                                uint32_t orr[32];
+                                tmem_ld32(lane_addr + COL_O + half * DH + c * 32, orr);
+                                tmem_wait_ld();
+    #pragma unroll
+                                for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
+                                tmem_st32(lane_addr + COL_O + half * DH + c * 32, orr);
+                            }
+                            if constexpr (D == 72) {
+                                if (half == 0) {
+                                    uint32_t ot[16];
+                                    tmem_ld16(lane_addr + COL_O + 64, ot);
+                                    tmem_wait_ld();
+    #pragma unroll
+                                    for (int i = 0; i < 16; ++i) ot[i] = __float_as_uint(__uint_as_float(ot[i]) * f);
+                                    tmem_st16(lane_addr + COL_O + 64, ot);
+                                }
+                            }
+                            tmem_wait_st();
+                        }
+                    }
+                    const float mb = m * scale_log2;
+                    uint32_t pk[32];
+                    float su0 = 0.f, su1 = 0.f, su2 = 0.f, su3 = 0.f;
+    #pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -mb));
+                        const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -mb));
+                        const float p2 = ex2(fmaf(__uint_as_float(sr[2 * i + 2]), scale_log2, -mb));
+                        const float p3 = ex2(fmaf(__uint_as_float(sr[2 * i + 3]), scale_log2, -mb));
+                        su0 += p0; su1 += p1; su2 += p2; su3 += p3;
+                        pk[i] = pack_bf16(p0, p1);
+                        pk[i + 1] = pack_bf16(p2, p3);
+                    }
+                    l += (su0 + su1) + (su2 + su3);
+                    // the P buffer is free once the product that read it two tiles ago has completed
+                    if (g >= 2 && !mbar_wait(&pv_done[bs * 2], ((g >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                    tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pk);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&p_full[bs * 2]);
+                }
+                if (!ok) break;
+                // epilogue: O / l for the rows of this tile (l = the two halves' partial sums)
+                const uint32_t gl = g0 + n_kv - 1;
+                s_xsum[half * 128 + r] = l;
+                mbar_arrive(&l_bar[quad]);
+                if (!mbar_wait(&l_bar[quad], item_i & 1, abort_flag)) { ok = false; break; }
+                const float inv = 1.0f / (l + s_xsum[(half ^ 1) * 128 + r]);
+                if (!mbar_wait(&pv_done[(gl & 1) * 2], (gl >> 1) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                __nv_bfloat16* dst = o + (size_t)(t.row0 + r) * o_ld + head * D + half * DH;
+    #pragma unroll
+                for (int c = 0; c < DH / 32; ++c) {
+                    uint32_t orr[32];
+                    tmem_ld32(lane_addr + COL_O + half * DH + c * 32, orr);
                     tmem_wait_ld();
                     if (r < t.rows) {
-                        uint4 u;
-                        u.x = pack_bf16(__uint_as_float(ot[0]) * inv, __uint_as_float(ot[1]) * inv);
-                        u.y = pack_bf16(__uint_as_float(ot[2]) * inv, __uint_as_float(ot[3]) * inv);
-                        u.z = pack_bf16(__uint_as_float(ot[4]) * inv, __uint_as_float(ot[5]) * inv);
-                        u.w = pack_bf16(__uint_as_float(ot[6]) * inv, __uint_as_float(ot[7]) * inv);
-                        *reinterpret_cast<uint4*>(o + (size_t)(t.row0 + r) * o_ld + head * D + 64) = u;
+    #pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 u;
+                            u.x = pack_bf16(__uint_as_float(orr[8 * v + 0]) * inv, __uint_as_float(orr[8 * v + 1]) * inv);
+                            u.y = pack_bf16(__uint_as_float(orr[8 * v + 2]) * inv, __uint_as_float(orr[8 * v + 3]) * inv);
+                            u.z = pack_bf16(__uint_as_float(orr[8 * v + 4]) * inv, __uint_as_float(orr[8 * v + 5]) * inv);
+                            u.w = pack_bf16(__uint_as_float(orr[8 * v + 6]) * inv, __uint_as_float(orr[8 * v + 7]) * inv);
+                            *reinterpret_cast<uint4*>(dst + c * 32 + v * 8) = u;
+                        }
                     }
                 }
+                if constexpr (D == 72) {
+                    if (half == 0) {                          // columns 64..71 of the head
+                        uint32_t ot[8];
+                        tmem_ld8(lane_addr + COL_O + 64, ot);
+                        tmem_wait_ld();
+                        if (r < t.rows) {
+                            uint4 u;
+                            u.x = pack_bf16(__uint_as_float(ot[0]) * inv, __uint_as_float(ot[1]) * inv);
+                            u.y = pack_bf16(__uint_as_float(ot[2]) * inv, __uint_as_float(ot[3]) * inv);
+                            u.z = pack_bf16(__uint_as_float(ot[4]) * inv, __uint_as_float(ot[5]) * inv);
+                            u.w = pack_bf16(__uint_as_float(ot[6]) * inv, __uint_as_float(ot[7]) * inv);
+                            *reinterpret_cast<uint4*>(o + (size_t)(t.row0 + r) * o_ld + head * D + 64) = u;
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(o_free);
+                g0 += n_kv;
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(o_free);
-            g0 += n_kv;
+            if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 600 + (int)blockIdx.x);
         }
-        if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 600 + (int)blockIdx.x);
     }
 
     tc_fence_before();

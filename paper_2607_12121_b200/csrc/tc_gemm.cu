@@ -21,7 +21,7 @@ using namespace ptx;
 namespace {
 
 constexpr int BM = 128, BK = 64;
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;        // TMA warp, MMA warp, 8 epilogue warps (two per TMEM lane quadrant)
 constexpr int A_TILE_BYTES = BM * BK * 2;
 
 template <int BN> struct GemmCfg {
@@ -57,7 +57,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tm_a);
@@ -117,6 +117,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         }
     } else {
         const int quad = warp & 3;                          // TMEM lane quadrant this warp may read
+        const int chalf = (warp - 2) >> 2;                  // which half of the tile's columns
         uint32_t t_it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t_it) {
@@ -129,7 +130,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const int tok = valid ? ep.active_idx[row] : 0;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(t_row + c0, r);
                 tmem_wait_ld();
@@ -189,7 +190,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < PAIR_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 16); }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tm_a);
@@ -251,6 +252,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         }
     } else {
         const int quad = warp & 3;
+        const int chalf = (warp - 2) >> 2;                  // which half of the tile's columns
         uint32_t t_it = 0;
         bool ok = true;
         for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
@@ -263,7 +265,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             const int tok = valid ? ep.active_idx[row] : 0;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
 #pragma unroll 1
-            for (int c0 = 0; c0 < PAIR_BN; c0 += 32) {
+            for (int c0 = chalf * (PAIR_BN / 2); c0 < (chalf + 1) * (PAIR_BN / 2); c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(t_row + c0, r);
                 tmem_wait_ld();
