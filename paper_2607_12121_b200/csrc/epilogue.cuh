@@ -7,6 +7,7 @@
 //   EPI_GELU  bias and tanh-GELU.
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace fd {
 
@@ -66,8 +67,17 @@ __device__ __forceinline__ void epilogue4(const EpiParams& ep, int row, int col,
 
 }  // namespace fd
 
-// ---- 32-column variant for the tensor-core kernels (bf16 storage, H % 32 == 0) -----------------
+// ---- tensor-core epilogues: 16-byte units transposed through shared memory ----------------------
+// After tcgen05.ld every thread holds consecutive columns of ONE row, so storing straight from those
+// registers makes each warp instruction touch 32 different rows (16 bytes out of 32 different
+// 128-byte lines).  That pattern saturates the L1/LSU pipe and slows the MMAs running next to it.
+// Instead the warp's chunk (32 rows x 128 bytes of output) goes through a 4 KB shared-memory tile in
+// 16-byte units: row t writes its 8 units, then lane t reads unit (t % 8) of rows 4 i + t / 8.  Each
+// global instruction then covers 4 complete 128-byte row segments.  The unit index is XORed with the
+// row's low bits so that both the writes and the reads are bank-conflict free.
 namespace fd {
+
+constexpr int EPI_STAGE_BYTES_PER_WARP = 32 * 128;
 
 __device__ __forceinline__ float tanh_fast(float x) {
     float y;
@@ -82,73 +92,164 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
     const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&h);
 }
-__device__ __forceinline__ void store8_bf16(__nv_bfloat16* p, const float* v) {
-    uint4 u;
-    u.x = pack2_bf16(v[0], v[1]); u.y = pack2_bf16(v[2], v[3]);
-    u.z = pack2_bf16(v[4], v[5]); u.w = pack2_bf16(v[6], v[7]);
-    *reinterpret_cast<uint4*>(p) = u;
+__device__ __forceinline__ uint4* unit_ptr(uint8_t* stage, int row, int u) {
+    return reinterpret_cast<uint4*>(stage + row * 128 + ((u ^ (row & 7)) << 4));
 }
 
-// acc: 32 consecutive fp32 accumulator columns of one row, starting at column col (col % 32 == 0)
-template <int KIND>
-__device__ __forceinline__ void epilogue32(const EpiParams& ep, int row, int col, int tok, const uint32_t* acc) {
+// What lane t knows about "its" row (row_base + t) of the warp's 32 rows, computed once per tile so that the
+// chunk loops contain no divisions and no 64-bit multiplies; other lanes fetch it with shuffles.
+struct RowInfo {
+    int gate_off;      // b * 6H: offset of the request's adaLN vectors
+    uint32_t y_lo, y_hi;   // tok * H: element offset of the row in y (EPI_RESID) or of the token in the K plane (EPI_QKV)
+};
+
+// EPI_RESID: 32 fp32 accumulator columns per row; resid += gate * (acc + bias); the last block also
+// scatters the row into y.
+__device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
+                                                     int n_rows, int col0, const uint32_t* acc, const RowInfo& ri) {
     using T = __nv_bfloat16;
-    float v[32];
-    const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ep.bias) + col);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const uint4 b = __ldg(bp + q);
-        const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+    for (int u = 0; u < 8; ++u) *unit_ptr(stage, lane, u) = make_uint4(acc[4 * u], acc[4 * u + 1], acc[4 * u + 2], acc[4 * u + 3]);
+    __syncwarp();
+    const int u = lane & 7, rsub = lane >> 3;
+    const int col = col0 + u * 4;
+    float bias[4];
+    load4<T>(reinterpret_cast<const T*>(ep.bias) + col, bias);
+    float* rp = ep.resid + (size_t)(row_base + rsub) * ep.H + col;      // rows rsub, rsub + 4, ...
+    const size_t rstride = (size_t)4 * ep.H;
+    const float* gp = ep.gate + col;
+    float4 rv[8], gv[8];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            v[8 * q + 2 * i] = __uint_as_float(acc[8 * q + 2 * i]) + __uint_as_float(w[i] << 16);
-            v[8 * q + 2 * i + 1] = __uint_as_float(acc[8 * q + 2 * i + 1]) + __uint_as_float(w[i] & 0xffff0000u);
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + rsub;
+        const int go = __shfl_sync(0xffffffffu, ri.gate_off, r);
+        if (r < n_rows) {
+            rv[i] = *reinterpret_cast<const float4*>(rp + i * rstride);
+            gv[i] = __ldg(reinterpret_cast<const float4*>(gp + go));
         }
     }
-    if constexpr (KIND == EPI_QKV) {
-        const int sec = col / ep.H, c = col - sec * ep.H;
-        T* dst;
-        if (sec == 0) {
-            if (ep.q_head_dim) {             // heads padded (72 -> 80): place every 8-column group inside its head
-                T* qrow = reinterpret_cast<T*>(ep.q) + (size_t)row * ep.q_ld;
+    T* yb = reinterpret_cast<T*>(ep.y);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int c8 = c + 8 * q, hd = c8 / ep.q_head_dim;
-                    store8_bf16(qrow + hd * ep.q_head_pad + (c8 - hd * ep.q_head_dim), v + 8 * q);
-                }
-                return;
-            }
-            dst = reinterpret_cast<T*>(ep.q) + (size_t)row * ep.q_ld + c;
-        } else {
-            const int b = tok / ep.N, j = tok - b * ep.N;
-            dst = reinterpret_cast<T*>(ep.kv) + (((size_t)b * 2 + (sec - 1)) * ep.N + j) * ep.H + c;
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + rsub;
+        const uint32_t ylo = __shfl_sync(0xffffffffu, ri.y_lo, r), yhi = __shfl_sync(0xffffffffu, ri.y_hi, r);
+        if (r < n_rows) {
+            const uint4 a = *unit_ptr(stage, r, u);
+            float4 v = rv[i];
+            v.x = fmaf(gv[i].x, __uint_as_float(a.x) + bias[0], v.x); v.y = fmaf(gv[i].y, __uint_as_float(a.y) + bias[1], v.y);
+            v.z = fmaf(gv[i].z, __uint_as_float(a.z) + bias[2], v.z); v.w = fmaf(gv[i].w, __uint_as_float(a.w) + bias[3], v.w);
+            *reinterpret_cast<float4*>(rp + i * rstride) = v;
+            if (yb) store4<T>(yb + (((size_t)yhi << 32) | ylo) + col, v.x, v.y, v.z, v.w);
         }
+    }
+    __syncwarp();
+}
+
+// EPI_QKV / EPI_GELU: 64 fp32 accumulator columns per row, bf16 outputs (8 columns per 16-byte unit).
+template <int KIND>
+__device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
+                                                    int n_rows, int col0, const uint32_t* acc, const RowInfo& ri) {
+    using T = __nv_bfloat16;
+    const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ep.bias) + col0);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) store8_bf16(dst + 8 * q, v + 8 * q);
-    } else if constexpr (KIND == EPI_RESID) {
-        const int b = tok / ep.N;
-        const float4* gp = reinterpret_cast<const float4*>(ep.gate + (size_t)b * 6 * ep.H + col);
-        float4* rp = reinterpret_cast<float4*>(ep.resid + (size_t)row * ep.H + col);
+    for (int u = 0; u < 8; ++u) {
+        const uint4 b = __ldg(bp + u);
+        const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+        float v[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const float4 g = __ldg(gp + q);
-            float4 r = rp[q];
-            r.x = fmaf(g.x, v[4 * q], r.x); r.y = fmaf(g.y, v[4 * q + 1], r.y);
-            r.z = fmaf(g.z, v[4 * q + 2], r.z); r.w = fmaf(g.w, v[4 * q + 3], r.w);
-            rp[q] = r;
-            v[4 * q] = r.x; v[4 * q + 1] = r.y; v[4 * q + 2] = r.z; v[4 * q + 3] = r.w;
+        for (int k = 0; k < 4; ++k) {
+            v[2 * k] = __uint_as_float(acc[8 * u + 2 * k]) + __uint_as_float(w[k] << 16);
+            v[2 * k + 1] = __uint_as_float(acc[8 * u + 2 * k + 1]) + __uint_as_float(w[k] & 0xffff0000u);
         }
-        if (ep.y) {
-            T* dst = reinterpret_cast<T*>(ep.y) + (size_t)tok * ep.H + col;
+        if constexpr (KIND == EPI_GELU) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) store8_bf16(dst + 8 * q, v + 8 * q);
+            for (int k = 0; k < 8; ++k) v[k] = gelu_tanh_fast(v[k]);
+        }
+        *unit_ptr(stage, lane, u) = make_uint4(pack2_bf16(v[0], v[1]), pack2_bf16(v[2], v[3]), pack2_bf16(v[4], v[5]),
+                                               pack2_bf16(v[6], v[7]));
+    }
+    __syncwarp();
+    const int u = lane & 7, rsub = lane >> 3;
+    const int col = col0 + u * 8;
+    if constexpr (KIND == EPI_GELU) {
+        T* ob = reinterpret_cast<T*>(ep.out) + (size_t)(row_base + rsub) * ep.out_ld + col;
+        const size_t ostride = (size_t)4 * ep.out_ld;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = 4 * i + rsub;
+            if (r < n_rows) *reinterpret_cast<uint4*>(ob + i * ostride) = *unit_ptr(stage, r, u);
         }
     } else {
-        T* dst = reinterpret_cast<T*>(ep.out) + (size_t)row * ep.out_ld + col;
+        const int sec = col0 / ep.H;                              // the 64 columns of a chunk share their section
+        const int c = col - sec * ep.H;
+        if (sec == 0) {
+            int qc = c;
+            if (ep.q_head_dim) { const int hd = c / ep.q_head_dim; qc = hd * ep.q_head_pad + (c - hd * ep.q_head_dim); }
+            T* qb = reinterpret_cast<T*>(ep.q) + (size_t)(row_base + rsub) * ep.q_ld + qc;
+            const size_t qstride = (size_t)4 * ep.q_ld;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_fast(v[i]);
+            for (int i = 0; i < 8; ++i) {
+                const int r = 4 * i + rsub;
+                if (r < n_rows) *reinterpret_cast<uint4*>(qb + i * qstride) = *unit_ptr(stage, r, u);
+            }
+        } else {
+            T* kvb = reinterpret_cast<T*>(ep.kv) + (size_t)(sec - 1) * ep.N * ep.H + c;     // K plane, or V plane N*H further
 #pragma unroll
-        for (int q = 0; q < 4; ++q) store8_bf16(dst + 8 * q, v + 8 * q);
+            for (int i = 0; i < 8; ++i) {
+                const int r = 4 * i + rsub;
+                const uint32_t lo = __shfl_sync(0xffffffffu, ri.y_lo, r), hi = __shfl_sync(0xffffffffu, ri.y_hi, r);
+                if (r < n_rows) *reinterpret_cast<uint4*>(kvb + (((size_t)hi << 32) | lo)) = *unit_ptr(stage, r, u);
+            }
+        }
+    }
+    __syncwarp();
+}
+
+// The residual rows an EPI_RESID tile will read usually sit in DRAM by the time the GEMM runs (32 MB of
+// fp32 rows, several kernels since they were written).  The epilogue warps are idle while the tile's MMAs
+// run, so they pull their rows' segments into L2 first; the loads in the epilogue then cost an L2 hit.
+__device__ __forceinline__ void epilogue_prefetch_resid(const EpiParams& ep, int lane, int row_base, int a_total,
+                                                        int col_begin, int n_cols) {
+    const int row = row_base + lane;
+    if (row < a_total) {
+        const char* p = reinterpret_cast<const char*>(ep.resid + (size_t)row * ep.H + col_begin);
+        for (int off = 0; off < n_cols * 4; off += 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p + off));
+    }
+}
+
+// one warp's share of a tile: rows [row_base, row_base + 32), columns [c_begin, c_end) of the accumulator at t_row
+template <int KIND>
+__device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stage, int lane, int row_base, int a_total,
+                                              uint32_t t_row, int tile_col0, int c_begin, int c_end) {
+    const bool live = row_base < a_total;                        // warp-uniform
+    const int n_rows = a_total - row_base;
+    RowInfo ri{0, 0u, 0u};
+    if (KIND != EPI_GELU && live && lane < n_rows) {
+        const int tok = ep.active_idx[row_base + lane];
+        const int b = tok / ep.N;
+        ri.gate_off = b * 6 * ep.H;
+        const size_t off = KIND == EPI_RESID ? (size_t)tok * ep.H : ((size_t)b * 2 * ep.N + (tok - b * ep.N)) * ep.H;
+        ri.y_lo = (uint32_t)off;
+        ri.y_hi = (uint32_t)(off >> 32);
+    }
+    if constexpr (KIND == EPI_RESID) {
+#pragma unroll 1
+        for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+            uint32_t r[32];
+            ptx::tmem_ld32(t_row + c0, r);
+            ptx::tmem_wait_ld();
+            if (live) epilogue_resid_chunk(ep, stage, lane, row_base, n_rows, tile_col0 + c0, r, ri);
+        }
+    } else {
+#pragma unroll 1
+        for (int c0 = c_begin; c0 < c_end; c0 += 64) {
+            uint32_t r[64];
+            ptx::tmem_ld32(t_row + c0, r);
+            ptx::tmem_ld32(t_row + c0 + 32, r + 32);
+            ptx::tmem_wait_ld();
+            if (live) epilogue_bf16_chunk<KIND>(ep, stage, lane, row_base, n_rows, tile_col0 + c0, r, ri);
+        }
     }
 }
 

@@ -24,10 +24,14 @@ constexpr int BM = 128, BK = 64;
 constexpr int GEMM_THREADS = 320;        // TMA warp, MMA warp, 8 epilogue warps (two per TMEM lane quadrant)
 constexpr int A_TILE_BYTES = BM * BK * 2;
 
+constexpr int EPI_WARPS = 8;
+constexpr int EPI_STAGE_BYTES = EPI_WARPS * EPI_STAGE_BYTES_PER_WARP;     // transposition tiles of the epilogue warps
+
 template <int BN> struct GemmCfg {
-    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int STAGES = BN == 256 ? 3 : 5;
     static constexpr int B_TILE_BYTES = BN * BK * 2;
-    static constexpr int SMEM = STAGES * (A_TILE_BYTES + B_TILE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int SMEM = STAGES * (A_TILE_BYTES + B_TILE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                                EPI_STAGE_BYTES;
 };
 
 template <int KIND, int BN>
@@ -47,6 +51,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     uint64_t* tempty = tfull + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint8_t* epi_stage = smem + STAGES * (A_TILE_BYTES + B_TILE_BYTES) + 256;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int a_total = ctl->a_total;
@@ -123,19 +128,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t_it) {
             const int m = tile % m_tiles, n = tile / m_tiles;
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
+            if constexpr (KIND == EPI_RESID)
+                epilogue_prefetch_resid(ep, lane, m * BM + quad * 32, a_total, n * BN + chalf * (BN / 2), BN / 2);
             if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const int row = m * BM + quad * 32 + lane;
-            const bool valid = row < a_total;
-            const int tok = valid ? ep.active_idx[row] : 0;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
-#pragma unroll 1
-            for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(t_row + c0, r);
-                tmem_wait_ld();
-                if (valid) epilogue32<KIND>(ep, row, n * BN + c0, tok, r);
-            }
+            epilogue_warp<KIND>(ep, epi_stage + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane, m * BM + quad * 32, a_total,
+                                t_row, n * BN, chalf * (BN / 2), (chalf + 1) * (BN / 2));
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty[acc]);
@@ -159,10 +158,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 // barriers with a multicast commit.  No TMA load is multicast: every CTA fetches its own tiles.
 // ------------------------------------------------------------------------------------------------
 constexpr int PAIR_BN = 256;
-constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_STAGES = 5;
 constexpr int PAIR_B_BYTES = 128 * BK * 2;           // this CTA's half of the weight tile
 constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_BYTES;
-constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + 1024 + 256;
+constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + 1024 + 256 + EPI_STAGE_BYTES;
 
 template <int KIND>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
@@ -178,6 +177,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     uint64_t* tempty = tfull + 2;                                                         // used in the first CTA
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint8_t* epi_stage = smem + PAIR_STAGES * PAIR_STAGE_BYTES + 256;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -258,19 +258,15 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
             const int m = tile % m_pairs, n = tile / m_pairs;
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
+            if constexpr (KIND == EPI_RESID)
+                epilogue_prefetch_resid(ep, lane, m * 2 * BM + (int)rank * BM + quad * 32, a_total,
+                                        n * PAIR_BN + chalf * (PAIR_BN / 2), PAIR_BN / 2);
             if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const int row = m * 2 * BM + (int)rank * BM + quad * 32 + lane;
-            const bool valid = row < a_total;
-            const int tok = valid ? ep.active_idx[row] : 0;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
-#pragma unroll 1
-            for (int c0 = chalf * (PAIR_BN / 2); c0 < (chalf + 1) * (PAIR_BN / 2); c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(t_row + c0, r);
-                tmem_wait_ld();
-                if (valid) epilogue32<KIND>(ep, row, n * PAIR_BN + c0, tok, r);
-            }
+            epilogue_warp<KIND>(ep, epi_stage + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane,
+                                m * 2 * BM + (int)rank * BM + quad * 32, a_total, t_row, n * PAIR_BN,
+                                chalf * (PAIR_BN / 2), (chalf + 1) * (PAIR_BN / 2));
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty[acc]), 0));
