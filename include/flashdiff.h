@@ -191,6 +191,13 @@ fd_status fd_region_activity_noalloc(const float* z_cur, const float* z_prev, co
  */
 fd_status fd_poll_status(fd_ctx* ctx, void* cuda_stream);
 
+/*
+ * Self-test of the bounded device-side waits: launches one thread that waits on a barrier nothing ever
+ * signals.  The wait gives up after its poll limit (about a second), the kernel records FD_ERR_TIMEOUT and
+ * returns normally; the next fd_poll_status reports FD_ERR_TIMEOUT and the context stays usable.
+ */
+fd_status fd_selftest_bounded_wait(fd_ctx* ctx, void* cuda_stream);
+
 /* Number of kernels the library has launched through this context so far (host counter). */
 int64_t fd_launch_count(const fd_ctx* ctx);
 

@@ -21,7 +21,7 @@ FD_ENGINE_AUTO, FD_ENGINE_SIMT, FD_ENGINE_TC = 0, 1, 2
 
 EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region_activity",
            "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
-           "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc"]
+           "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
                "gemm_fc2", "partition"]
@@ -70,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.fd_profile_enable.argtypes = [vp, i32]
     lib.fd_profile_read.restype = i32
     lib.fd_profile_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
+    lib.fd_selftest_bounded_wait.restype = i32
+    lib.fd_selftest_bounded_wait.argtypes = [vp, vp]
     lib.fd_launch_count.restype = ctypes.c_int64
     lib.fd_launch_count.argtypes = [vp]
     lib.fd_destroy.restype = i32
@@ -188,6 +190,10 @@ def fd_regional_step(ctx: Context, x, cond, labels, mask, R: int, kv_cache, y, a
 
 def fd_poll_status(ctx: Context, stream=None) -> None:
     _check(ctx.handle, lib.fd_poll_status(ctx.handle, _stream(stream)))
+
+
+def fd_selftest_bounded_wait(ctx: Context, stream=None) -> None:
+    _check(ctx.handle, lib.fd_selftest_bounded_wait(ctx.handle, _stream(stream)))
 
 
 def fd_profile_enable(ctx: Context, enable: bool) -> None:

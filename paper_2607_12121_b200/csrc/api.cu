@@ -439,6 +439,15 @@ fd_status fd_profile_read(fd_ctx* c, void* cuda_stream, float* ms_out, int32_t* 
     return FD_OK;
 }
 
+fd_status fd_selftest_bounded_wait(fd_ctx* c, void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    int nl = 0;
+    cudaError_t e = launch_bounded_wait_selftest(c->ctl(), static_cast<cudaStream_t>(cuda_stream), &nl);
+    c->launches += nl;
+    if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "self-test launch failed: %s", cudaGetErrorString(e));
+    return FD_OK;
+}
+
 int64_t fd_launch_count(const fd_ctx* c) { return c ? c->launches : 0; }
 
 fd_status fd_destroy(fd_ctx* c) {

@@ -28,6 +28,8 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
 cudaError_t tc_attention(TcPlan* p, int blk, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch);
 
+cudaError_t launch_bounded_wait_selftest(Control* ctl, cudaStream_t st, int* n_launch);
+
 // host helper shared by the GEMM and attention plans: encodes a tiled bf16 tensor map
 // (rank <= 4; dims / strides innermost first; strides in bytes for dims 1..rank-1)
 bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,

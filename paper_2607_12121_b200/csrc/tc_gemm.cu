@@ -283,6 +283,20 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     }
 }
 
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever arrives on.  The wait
+// gives up after its poll limit (about a second), records FD_ERR_TIMEOUT in the control block and the
+// kernel returns normally, so the context stays usable.
+__global__ void bounded_wait_selftest_kernel(Control* ctl) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+        if (!mbar_wait(&bar, 0, &abort_flag)) report(ctl, FD_ERR_TIMEOUT, 999);
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -448,6 +462,12 @@ void tc_plan_destroy(TcPlan* p) {
     tc_attention_plan_destroy(p->attn);
     delete[] p->w_maps;
     delete p;
+}
+
+cudaError_t launch_bounded_wait_selftest(Control* ctl, cudaStream_t st, int* n_launch) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(ctl);
+    ++*n_launch;
+    return cudaGetLastError();
 }
 
 void* tc_plan_attn(TcPlan* p) { return p->attn; }

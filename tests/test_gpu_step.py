@@ -154,3 +154,37 @@ def test_peaked_attention_exercises_running_max(name, engine):
     wl = gen.workload(name)
     masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.5] * wl.B)]
     _run_sequence(wl, 4, engine, masks, qk_gain=64.0)
+
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    """A device-side wait that nothing satisfies gives up after its limit: the kernel returns, the status
+    word says FD_ERR_TIMEOUT, and the same context then runs a normal step."""
+    wl = gen.workload("audio_tc")
+    labels = gen.uniform_labels(wl)
+    w = gen.block_weights(wl, 9)
+    inp = gen.step_inputs(wl, 9, labels)
+    ctx = make_ctx(wl, w)
+    fd.fd_selftest_bounded_wait(ctx)
+    with pytest.raises(fd.FlashDiffError) as ei:
+        fd.fd_poll_status(ctx)
+    assert ei.value.status == fd.FD_ERR_TIMEOUT
+    buf = StepBuffers(wl, wl.L)
+    dt = tdtype(wl)
+    idx, cu = gpu_step(ctx, wl, dev(inp["x_cur"], dt), dev(inp["cond"], dt), dev(labels),
+                       dev(np.ones((wl.B, wl.R), np.uint8)), buf)
+    assert idx.size == wl.B * wl.N
+    y_d, _ = oracle.dense_step(inp["x_cur"], inp["cond"], w, wl.heads)
+    assert max_abs(host(buf.y), y_d) <= BF16_MAX_ABS and rel_l2(host(buf.y), y_d) <= BF16_REL_L2
+
+
+@pytest.mark.parametrize("n_tok,regions,heads,head_dim", [(40, 5, 4, 64), (64, 4, 4, 64), (130, 13, 4, 64),
+                                                        (200, 8, 4, 64), (40, 5, 2, 128), (130, 13, 2, 128),
+                                                        (1, 1, 4, 64)])
+def test_tensor_core_engine_ragged_key_counts(n_tok, regions, heads, head_dim):
+    """Key counts around the 128-key tile and its 64-key halves: a single partial tile, a tile whose second
+    half has no valid key, a last tile with two keys, and a single token."""
+    wl = gen.workload("audio_tc").replace(grid=(n_tok,), R=regions, B=2, heads=heads, head_dim=head_dim, L=1)
+    masks = [np.ones((wl.B, wl.R), np.uint8)]
+    if regions > 1:
+        masks.append(gen.region_mask(wl, 7, [0.6, 0.4]))
+    _run_sequence(wl, 5, fd.FD_ENGINE_TC, masks, qk_gain=16.0)
