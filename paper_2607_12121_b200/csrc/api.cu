@@ -166,6 +166,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     FD_TRY(FD_PROF_ADALN, launch_adaln<T>(cond, static_cast<const T*>(c->w.w_ada), static_cast<const T*>(c->w.b_ada), mod, L, B, H,
                            Hc, c->ws + l.ada_act, st, &nl));
     const int max_tiles = B * ((N + c->tile_rows - 1) / c->tile_rows);
+    const bool pdl = c->use_tc && c->tc && tc_plan_pdl(c->tc);
     for (int blk = 0; blk < L; ++blk) {
         const float* mod_b = mod + (size_t)blk * B * 6 * H;
         const T* w_qkv = static_cast<const T*>(c->w.w_qkv) + (size_t)blk * 3 * H * H;
@@ -181,7 +182,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
 
         // gather (first block) or read the residual stream; LayerNorm; attention-branch modulation
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(blk == 0 ? x : nullptr, resid, resid, act, active_idx, mod_b + 0 * H,
-                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl));
+                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl));
         // QKV projection; K and V rows go straight into the cache
         ep.bias = static_cast<const T*>(c->w.b_qkv) + (size_t)blk * 3 * H;
         ep.q = q;
@@ -212,7 +213,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             FD_TRY(FD_PROF_GEMM_OUT, launch_simt_gemm<T>(EPI_RESID, o, H, w_o, H, H, rows_cap, ep, ctl, st, &nl));
         // MLP branch
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, mod_b + 3 * H, mod_b + 4 * H, 6 * H, N,
-                                     H, rows_cap, cf.ln_eps, ctl, st, &nl));
+                                     H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl));
         ep.bias = static_cast<const T*>(c->w.b_fc1) + (size_t)blk * M;
         ep.out = g;
         ep.out_ld = M;

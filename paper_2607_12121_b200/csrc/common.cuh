@@ -116,7 +116,7 @@ template <typename T>
 cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
                                const int32_t* active_idx, const float* shift, const float* scale,
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
-                               cudaStream_t st, int* n_launch);
+                               cudaStream_t st, int* n_launch, bool pdl);
 
 // simt_block.cu
 template <typename T>

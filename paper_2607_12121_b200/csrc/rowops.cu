@@ -2,6 +2,7 @@
 // gather + LayerNorm + modulation that feeds the QKV and MLP projections.  The block is the
 // adaLN-Zero DiT block the paper builds on (Sec. 2.1); only active rows are touched (Sec. 3).
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace fd {
 
@@ -225,6 +226,7 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
                    const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
                    int H, float ln_eps, const Control* __restrict__ ctl) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    ptx::pdl_wait();                              // the rows come from the kernel launched just before
     const int a_total = ctl->a_total;
     const int nv = H / 128;                       // float4 slots per lane (H % 128 == 0 on this path)
     for (int row = blockIdx.x * (LN_THREADS / 32) + warp; row < a_total; row += gridDim.x * (LN_THREADS / 32)) {
@@ -274,6 +276,9 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
             }
         }
     }
+    // a multi-wave kernel: let the successor start only when this CTA is done, so that its waiting CTAs
+    // do not take registers away from the waves still to run
+    ptx::pdl_trigger();
 }
 
 // Any width: three passes over the row (the re-reads hit L1/L2).
@@ -342,13 +347,15 @@ template <typename T>
 cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
                                const int32_t* active_idx, const float* shift, const float* scale,
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
-                               cudaStream_t st, int* n_launch) {
+                               cudaStream_t st, int* n_launch, bool pdl) {
     const int rows_per_cta = LN_THREADS / 32;
     const int grid = max(1, min((rows_cap + rows_per_cta - 1) / rows_per_cta, 148 * 16));
-    if (H % 128 == 0)
-        ln_modulate_kernel<T><<<grid, LN_THREADS, 0, st>>>(x_gather, resid_in, resid_out, out, active_idx, shift,
-                                                          scale, mod_stride, N, H, ln_eps, ctl);
-    else
+    if (H % 128 == 0) {
+        cudaError_t e = ptx::launch_kernel(ln_modulate_kernel<T>, grid, LN_THREADS, 0, st, pdl, x_gather, resid_in, resid_out,
+                                           out, active_idx, shift, scale, mod_stride, N, H, ln_eps, ctl);
+        ++*n_launch;
+        return e;
+    } else
         ln_modulate_generic_kernel<T><<<grid, LN_THREADS, 0, st>>>(x_gather, resid_in, resid_out, out, active_idx,
                                                                   shift, scale, mod_stride, N, H, ln_eps, ctl);
     ++*n_launch;
@@ -361,9 +368,9 @@ template cudaError_t launch_adaln<__nv_bfloat16>(const __nv_bfloat16*, const __n
                                                  float*, int, int, int, int, void*, cudaStream_t, int*);
 template cudaError_t launch_ln_modulate<float>(const float*, const float*, float*, float*, const int32_t*,
                                                const float*, const float*, int, int, int, int, float, const Control*,
-                                               cudaStream_t, int*);
+                                               cudaStream_t, int*, bool);
 template cudaError_t launch_ln_modulate<__nv_bfloat16>(const __nv_bfloat16*, const float*, float*, __nv_bfloat16*,
                                                        const int32_t*, const float*, const float*, int, int, int, int,
-                                                       float, const Control*, cudaStream_t, int*);
+                                                       float, const Control*, cudaStream_t, int*, bool);
 
 }  // namespace fd

@@ -20,6 +20,7 @@ enum TcGemmKind { TC_GEMM_QKV = 0, TC_GEMM_OUT = 1, TC_GEMM_FC1 = 2, TC_GEMM_FC2
 bool tc_supported(const fd_config& cfg, std::string* why);
 bool tc_attention_supported(const fd_config& cfg);
 int tc_attention_tile_rows();
+bool tc_plan_pdl(TcPlan* p);                // kernels of the step are launched with programmatic stream serialization
 int tc_attention_head_pad(int head_dim);   // head dim as stored in the padded Q buffer
 TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffers& buf, std::string* err);
 void tc_plan_destroy(TcPlan* p);

@@ -29,6 +29,7 @@ using namespace ptx;
 
 void* tc_plan_attn(TcPlan* p);
 int tc_plan_sm_count(TcPlan* p);
+bool tc_plan_pdl(TcPlan* p);
 
 namespace {
 
@@ -102,10 +103,6 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (threadIdx.x == 0) report(ctl, FD_ERR_STATE, -1024);
         return;
     }
-    // items are ordered head-major: the CTAs running at the same time work on the same one or two heads,
-    // so that head's K/V stays in L2 however long the key sequence is
-    const int n_tiles = ctl->n_qtiles;
-    const int n_items = n_tiles * heads;
     const int n_kv = (N + KEYS - 1) / KEYS;
 
     if (threadIdx.x == 0) {
@@ -134,6 +131,13 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above is local set-up; from here on the kernel reads what earlier kernels wrote
+    pdl_trigger();
+    pdl_wait();
+    // items are ordered head-major: the CTAs running at the same time work on the same one or two heads,
+    // so that head's K/V stays in L2 however long the key sequence is
+    const int n_tiles = ctl->n_qtiles;
+    const int n_items = n_tiles * heads;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -610,15 +614,16 @@ cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, c
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)a->dh);
     Control* c = const_cast<Control*>(ctl);
     __nv_bfloat16* o = static_cast<__nv_bfloat16*>(a->o);
+    cudaError_t e = cudaSuccess;
 #define FD_ATT(DD)                                                                                                  \
-    tc_attention_kernel<DD><<<grid, ATT_THREADS, AttCfg<DD>::SMEM, st>>>(a->q_map, kv_map, a->q_tail_map, kv_tail_map, o, \
-                                                                          a->H, tiles, a->heads, N, scale_log2, c)
+    e = launch_kernel(tc_attention_kernel<DD>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, tc_plan_pdl(p), a->q_map, kv_map, \
+                      a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c)
     if (a->dh == 64) FD_ATT(64);
     else if (a->dh == 128) FD_ATT(128);
     else FD_ATT(72);
 #undef FD_ATT
     ++*n_launch;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace fd

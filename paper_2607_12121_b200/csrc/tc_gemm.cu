@@ -54,11 +54,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     uint8_t* epi_stage = smem + STAGES * (A_TILE_BYTES + B_TILE_BYTES) + 256;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int a_total = ctl->a_total;
-    const int m_tiles = (a_total + BM - 1) / BM;
-    const int n_tiles = n_out / BN;
-    const int total_tiles = m_tiles * n_tiles;
-    const int k_tiles = k_dim / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -76,6 +71,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above is local set-up; from here on the kernel reads what earlier kernels wrote
+    pdl_trigger();
+    pdl_wait();
+    const int a_total = ctl->a_total;
+    const int m_tiles = (a_total + BM - 1) / BM;
+    const int n_tiles = n_out / BN;
+    const int total_tiles = m_tiles * n_tiles;
+    const int k_tiles = k_dim / BK;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -181,11 +184,6 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
-    const int a_total = ctl->a_total;
-    const int m_pairs = (a_total + 2 * BM - 1) / (2 * BM);
-    const int n_tiles = n_out / PAIR_BN;
-    const int total_tiles = m_pairs * n_tiles;
-    const int k_tiles = k_dim / BK;
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
@@ -205,6 +203,14 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     cluster_sync_all();                      // both CTAs' barriers exist before anything remote arrives
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above is local set-up; from here on the kernel reads what earlier kernels wrote
+    pdl_trigger();
+    pdl_wait();
+    const int a_total = ctl->a_total;
+    const int m_pairs = (a_total + 2 * BM - 1) / (2 * BM);
+    const int n_tiles = n_out / PAIR_BN;
+    const int total_tiles = m_pairs * n_tiles;
+    const int k_tiles = k_dim / BK;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -351,6 +357,7 @@ struct TcPlan {
     fd_config cfg;
     TcBuffers buf;
     int sm_count;
+    bool pdl;                   // launch the tensor-core kernels with programmatic stream serialization
     int pair_ctas;              // grid of the CTA-pair kernel: 2 x co-resident clusters
     GemmSpec spec[4];
     CUtensorMap* w_maps;        // [L][4]
@@ -383,6 +390,8 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         const int v = atoi(lim);
         if (v > 0 && v < p->sm_count) p->sm_count = v;
     }
+    p->pdl = true;              // switch: FD_PDL=0 launches every kernel fully serialized
+    if (const char* v = getenv("FD_PDL")) p->pdl = atoi(v) != 0;
     bool use_pair = true;       // switch: FD_TC_PAIR=0 keeps every GEMM on the single-CTA kernel
     if (const char* v = getenv("FD_TC_PAIR")) use_pair = atoi(v) != 0;
     const int H = cfg.hidden, M = cfg.mlp_dim;
@@ -471,6 +480,7 @@ cudaError_t launch_bounded_wait_selftest(Control* ctl, cudaStream_t st, int* n_l
 }
 
 void* tc_plan_attn(TcPlan* p) { return p->attn; }
+bool tc_plan_pdl(TcPlan* p) { return p->pdl; }
 int tc_plan_sm_count(TcPlan* p) { return p->sm_count; }
 
 cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
@@ -481,17 +491,19 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
     const int grid = p->sm_count;
     if (s.pair) {
         const int pgrid = max(2, min(grid & ~1, p->pair_ctas));
+        cudaError_t e;
         if (kind == TC_GEMM_QKV)
-            tc_gemm_pair_kernel<EPI_QKV><<<pgrid, GEMM_THREADS, PAIR_SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c);
+            e = launch_kernel(tc_gemm_pair_kernel<EPI_QKV>, pgrid, GEMM_THREADS, PAIR_SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c);
         else if (kind == TC_GEMM_FC1)
-            tc_gemm_pair_kernel<EPI_GELU><<<pgrid, GEMM_THREADS, PAIR_SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c);
+            e = launch_kernel(tc_gemm_pair_kernel<EPI_GELU>, pgrid, GEMM_THREADS, PAIR_SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c);
         else
-            tc_gemm_pair_kernel<EPI_RESID><<<pgrid, GEMM_THREADS, PAIR_SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c);
+            e = launch_kernel(tc_gemm_pair_kernel<EPI_RESID>, pgrid, GEMM_THREADS, PAIR_SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c);
         ++*n_launch;
-        return cudaGetLastError();
+        return e;
     }
+    cudaError_t e = cudaSuccess;
 #define FD_LAUNCH(K, N) \
-    tc_gemm_kernel<K, N><<<grid, GEMM_THREADS, GemmCfg<N>::SMEM, st>>>(s.a, wm, s.n_out, s.k, ep, c)
+    e = launch_kernel(tc_gemm_kernel<K, N>, grid, GEMM_THREADS, GemmCfg<N>::SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c)
     if (kind == TC_GEMM_QKV) {
         if (s.bn == 256) FD_LAUNCH(EPI_QKV, 256); else FD_LAUNCH(EPI_QKV, 128);
     } else if (kind == TC_GEMM_FC1) {
@@ -501,7 +513,7 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
     }
 #undef FD_LAUNCH
     ++*n_launch;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace fd
