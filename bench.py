@@ -361,6 +361,39 @@ def run_ours(args):
     d2h = h_y.numel() * h_y.element_size()
     fd.fd_poll_status(ctx)
 
+    # streaming rate of the activity reduction on a batch large enough to be bandwidth bound (at the
+    # benchmark shapes the gate moves a few MB and is launch-latency bound): 256 requests x 8192 tokens x 64
+    # channels, all regions fresh, through the allocation-free entry point
+    probe = None
+    if not args.no_probe:
+        pB, pN, pD, pR = 256, 8192, 64, 64
+        pz0 = torch.randn((pB, pN, pD), dtype=torch.float32, device=dev)
+        pz1 = pz0 + 0.01 * torch.randn_like(pz0)
+        plab = (torch.arange(pN, device=dev, dtype=torch.int32) // (pN // pR)).repeat(pB, 1).contiguous()
+        peps = torch.full((pB,), 1e-3, dtype=torch.float32, device=dev)
+        pst = [torch.zeros((pB, pR), dtype=torch.float32, device=dev), torch.zeros((pB, pR), dtype=torch.int32, device=dev),
+               torch.ones((pB, pR), dtype=torch.uint8, device=dev)]
+        pout = [torch.empty((pB, pR), dtype=torch.float32, device=dev), torch.empty((pB, pR), dtype=torch.float32, device=dev),
+                torch.empty((pB, pR), dtype=torch.uint8, device=dev)]
+
+        def probe_step():
+            pst[2].fill_(1)
+            fd.fd_region_activity_noalloc(pz1, pz0, plab, pR, peps, 1e-12, 5, pst[0], pst[1], pst[2], pout[0], pout[1], pout[2])
+
+        for _ in range(3):
+            probe_step()
+        torch.cuda.synchronize()
+        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pe0.record()
+        for _ in range(10):
+            probe_step()
+        pe1.record()
+        torch.cuda.synchronize()
+        p_ms = pe0.elapsed_time(pe1) / 10
+        p_bytes = 2.0 * pz0.numel() * 4 + plab.numel() * 4
+        del pz0, pz1, plab
+        probe = {"bytes": p_bytes, "ms": p_ms, "gbs": p_bytes / (p_ms * 1e-3) / 1e9}
+
     fl = block_flops(A_b, N, H, M)
     step_flops = L * sum(fl.values())
     dense_flops = L * sum(block_flops([N] * B, N, H, M).values())
@@ -424,6 +457,8 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": roofline,
         "kernel_breakdown": breakdown,
+        "activity_probe": None if probe is None else dict(probe, frac_of_hbm=probe["gbs"] / float(peaks["hbm_gbs"]),
+                                                         workload="256 requests x 8192 tokens x 64 channels, 64 regions"),
         "peaks": {"source": peak_kind, "bf16_tflops": peaks.get("bf16_tflops"),
                   "bf16_tflops_sustained": peaks.get("bf16_tflops_sustained"), "hbm_gbs": peaks.get("hbm_gbs")},
     }
@@ -449,6 +484,7 @@ def main():
     ap.add_argument("--fraction", type=float, default=None, help="same active fraction for every request")
     ap.add_argument("--seed", type=int, default=1000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-probe", action="store_true", help="skip the bandwidth probe of the activity kernel")
     ap.add_argument("--blocks", type=int, default=0, help="override the block count (profiling captures only)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -16,7 +16,7 @@ constexpr int ACT_THREADS = 256;
 
 // V = float4 vectors per token (D / 4).  GROUP = lanes that share one token.
 template <int UNROLL>
-__global__ void __launch_bounds__(ACT_THREADS)
+__global__ void __launch_bounds__(ACT_THREADS, 8)
 activity_reduce_kernel(const float4* __restrict__ z_cur, const float4* __restrict__ z_prev,
                        const int32_t* __restrict__ labels, const uint8_t* __restrict__ prev_active,
                        int N, int V, int R, int tokens_per_cta, double* __restrict__ acc_ss,
@@ -37,6 +37,12 @@ activity_reduce_kernel(const float4* __restrict__ z_cur, const float4* __restric
         int group = 1;
         while (group < 32 && (V % (group * 2)) == 0) group *= 2;
         const long long span = (long long)ACT_THREADS * UNROLL;
+        // Each group leader keeps a running sum for the region it is currently in and only touches the
+        // shared accumulators when the region changes: consecutive tokens mostly share their region, and
+        // fp64 shared-memory atomics on one hot address would otherwise serialise the whole CTA.
+        const bool leader = (threadIdx.x & (group - 1)) == 0;
+        int cur_lab = -1, cur_cnt = 0;
+        float cur_sum = 0.f;
         for (long long i0 = 0; i0 < n_vec; i0 += span) {
             float part[UNROLL];
             int lab[UNROLL];
@@ -49,10 +55,10 @@ activity_reduce_kernel(const float4* __restrict__ z_cur, const float4* __restric
                 lead[u] = false;
                 if (i < n_vec) {
                     const int tok = t0 + (int)(i / V);
-                    const int l = lab_b[tok];
+                    const int l = __ldg(lab_b + tok);
                     if (l < 0 || l > R) {
                         report(ctl, FD_ERR_STATE, tok);
-                    } else if (l < R && pa_b[l]) {
+                    } else if (l < R && __ldg(pa_b + l)) {
                         const size_t e = base + (size_t)t0 * V + (size_t)i;
                         const float4 a = __ldg(z_cur + e);
                         const float4 p = __ldg(z_prev + e);
@@ -68,11 +74,24 @@ activity_reduce_kernel(const float4* __restrict__ z_cur, const float4* __restric
                 float v = part[u];
                 // lanes [g*group, (g+1)*group) hold vectors of the same token
                 for (int o = group >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (lab[u] >= 0) {
-                    if ((threadIdx.x & (group - 1)) == 0) atomicAdd(&s_ss[lab[u]], (double)v);
-                    if (lead[u]) atomicAdd(&s_cnt[lab[u]], 1);
+                if (lab[u] >= 0 && leader) {
+                    if (lab[u] != cur_lab) {
+                        if (cur_lab >= 0) {
+                            atomicAdd(&s_ss[cur_lab], (double)cur_sum);
+                            if (cur_cnt) atomicAdd(&s_cnt[cur_lab], cur_cnt);
+                        }
+                        cur_lab = lab[u];
+                        cur_sum = 0.f;
+                        cur_cnt = 0;
+                    }
+                    cur_sum += v;
+                    cur_cnt += lead[u] ? 1 : 0;      // the first vector of a token sits on a group leader
                 }
             }
+        }
+        if (cur_lab >= 0) {
+            atomicAdd(&s_ss[cur_lab], (double)cur_sum);
+            if (cur_cnt) atomicAdd(&s_cnt[cur_lab], cur_cnt);
         }
     }
     __syncthreads();
@@ -160,9 +179,12 @@ cudaError_t launch_activity(const float* z_cur, const float* z_prev, const int32
     const bool vec = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(z_cur) | reinterpret_cast<uintptr_t>(z_prev)) % 16 == 0);
     if (vec) {
         const int V = D / 4;
-        // 32 KB of each operand per CTA: enough CTAs to cover the SMs at the benchmark shapes,
-        // enough work per CTA to amortise the shared-memory flush
-        int tokens_per_cta = max(1, 2048 / V);
+        // At least 32 KB of each operand per CTA (enough work to amortise set-up and the flush); for large
+        // batches fewer, longer chunks: about 16 CTAs per SM in total keep every SM streaming without a long tail.
+        const int by_size = (int)(((long long)N * V + 2047) / 2048);
+        const int by_sms = (148 * 16 + B - 1) / B;
+        const int want = max(1, min(by_size, by_sms));
+        const int tokens_per_cta = (N + want - 1) / want;
         const int chunks = (N + tokens_per_cta - 1) / tokens_per_cta;
         dim3 grid(chunks, B);
         const size_t smem = (size_t)R * (sizeof(double) + sizeof(int32_t));
