@@ -118,6 +118,33 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
     float* rp = ep.resid + (size_t)(row_base + rsub) * ep.H + col;      // rows rsub, rsub + 4, ...
     const size_t rstride = (size_t)4 * ep.H;
     const float* gp = ep.gate + col;
+    T* yb = reinterpret_cast<T*>(ep.y);
+    if (!yb) {
+        // Every element of the residual stream receives exactly one contribution from this kernel, so the
+        // update is a plain "add to memory": a vector reduction instruction does it without reading the row
+        // back into the SM (no load latency in the epilogue, half the memory instructions); the result is the
+        // same single fp32 addition as load / add / store.
+        float4 gv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int go = __shfl_sync(0xffffffffu, ri.gate_off, 4 * i + rsub);
+            if (4 * i + rsub < n_rows) gv[i] = __ldg(reinterpret_cast<const float4*>(gp + go));
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = 4 * i + rsub;
+            if (r < n_rows) {
+                const uint4 a = *unit_ptr(stage, r, u);
+                const float x = gv[i].x * (__uint_as_float(a.x) + bias[0]), y = gv[i].y * (__uint_as_float(a.y) + bias[1]);
+                const float z = gv[i].z * (__uint_as_float(a.z) + bias[2]), w = gv[i].w * (__uint_as_float(a.w) + bias[3]);
+                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(rp + i * rstride), "f"(x), "f"(y), "f"(z), "f"(w)
+                             : "memory");
+            }
+        }
+        __syncwarp();
+        return;
+    }
+    // last block: the final value is needed for the scatter into y, so read, add, write
     float4 rv[8], gv[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -128,7 +155,6 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
             gv[i] = __ldg(reinterpret_cast<const float4*>(gp + go));
         }
     }
-    T* yb = reinterpret_cast<T*>(ep.y);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int r = 4 * i + rsub;
@@ -139,7 +165,7 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
             v.x = fmaf(gv[i].x, __uint_as_float(a.x) + bias[0], v.x); v.y = fmaf(gv[i].y, __uint_as_float(a.y) + bias[1], v.y);
             v.z = fmaf(gv[i].z, __uint_as_float(a.z) + bias[2], v.z); v.w = fmaf(gv[i].w, __uint_as_float(a.w) + bias[3], v.w);
             *reinterpret_cast<float4*>(rp + i * rstride) = v;
-            if (yb) store4<T>(yb + (((size_t)yhi << 32) | ylo) + col, v.x, v.y, v.z, v.w);
+            store4<T>(yb + (((size_t)yhi << 32) | ylo) + col, v.x, v.y, v.z, v.w);
         }
     }
     __syncwarp();

@@ -131,7 +131,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t_it) {
             const int m = tile % m_tiles, n = tile / m_tiles;
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
-            if constexpr (KIND == EPI_RESID)
+            if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * BM + quad * 32, a_total, n * BN + chalf * (BN / 2), BN / 2);
             if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
@@ -264,7 +264,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
             const int m = tile % m_pairs, n = tile / m_pairs;
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
-            if constexpr (KIND == EPI_RESID)
+            if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * 2 * BM + (int)rank * BM + quad * 32, a_total,
                                         n * PAIR_BN + chalf * (PAIR_BN / 2), PAIR_BN / 2);
             if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
