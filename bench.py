@@ -62,7 +62,7 @@ class ClockSampler:
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -76,7 +76,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.out.close()
-        sm, mx, reasons = [], [], set()
+        sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         with open(self.path) as f:
             for line in f:
@@ -84,19 +84,20 @@ class ClockSampler:
                 if len(parts) < 9:
                     continue
                 try:
-                    sm.append(float(parts[1]))
-                    mx.append(float(parts[2]))
+                    c, m, pw = float(parts[1]), float(parts[2]), float(parts[3])
                 except ValueError:
                     continue
+                sm.append(c); mx.append(m); power.append(pw)
                 for n, v in zip(names, parts[5:9]):
                     if v.lower().startswith("active"):
                         reasons.add(n)
         os.unlink(self.path)
-        # samples under load: the upper half of the clock samples excludes idle ticks around the region
+        # the sampler runs only around the timed region; drop samples taken while the GPU drew little power
+        # (the ticks just before the first and after the last step)
         if sm:
-            hi = sorted(sm)[len(sm) // 2:]
-            return {"sm_mhz": statistics.median(hi), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                    "samples": len(sm)}
+            busy = [c for c, p in zip(sm, power) if p >= 0.5 * max(power)] or sm
+            return {"sm_mhz": statistics.median(busy), "sm_min_mhz": min(busy), "sm_max_mhz": max(mx),
+                    "power_w_max": max(power), "reasons": sorted(reasons), "samples": len(busy)}
         return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
 
 

@@ -74,9 +74,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait.  `abort_flag` (shared memory) lets one role's time-out release the others.
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    // the non-blocking test first: it returns sooner than try_wait when the phase has already completed
+    if (mbar_test_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it > 64) {

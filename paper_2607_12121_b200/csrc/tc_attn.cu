@@ -49,7 +49,7 @@ template <int D> struct AttCfg {
     static constexpr int TILE_BYTES = SUBS * SUB_BYTES + (D == 72 ? TAIL_BYTES : 0);
     // K/V rings deep enough that a tile is requested several tile periods before it is needed
     static constexpr int STAGES = D == 128 ? 2 : (D == 72 ? 4 : 5);
-    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 3584;
+    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 3584 + (D == 64 ? 256 * 80 : 0);
 };
 
 __device__ __forceinline__ float ex2(float x) {
@@ -97,6 +97,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* s_xmax = reinterpret_cast<float*>(tmem_slot + 2);      // [2 buffers][2 halves][128 rows]
     float* s_xsum = s_xmax + 512;                                 // [2 halves][128 rows]
+    uint8_t* s_stage = reinterpret_cast<uint8_t*>(bars) + 3584;   // [256 softmax threads][80 bytes], head dim 64 only
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (smem_u32(smem) & 1023u) {                        // never expected; refuse rather than compute garbage
@@ -275,17 +276,87 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int r = quad * 32 + lane;                       // query row inside the tile
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
             const uint32_t o_addr = lane_addr + COL_O + half * 64;
+            // staging slot of this thread's 64 output bytes; the slots are 80 bytes apart so that the 16-byte
+            // stores of a quarter warp fall into different banks
+            uint8_t* stage = s_stage + (threadIdx.x - 96) * 80;
             uint32_t g0 = 0;
             bool ok = true;
             int item_i = 0;
             const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
+            // The end of an item (merge the halves, normalise, store) is deferred until the first key tile of
+            // the next item has been through the softmax: the tensor core finishes the last product of the
+            // old item while these warps already work on the new one.
+            float pend_m = 0.f, pend_l = 0.f;
+            int pend_row0 = 0, pend_rows = 0, pend_head = 0, pend_item = -1;
+            uint32_t pend_ge = 0;
+            auto finish = [&]() -> bool {
+                // merge the two halves' partial results and store the row
+                s_xmax[half * 128 + r] = pend_m;
+                s_xsum[half * 128 + r] = pend_l;
+                mbar_arrive(&l_bar[quad]);
+                if (!mbar_wait(&l_bar[quad], pend_item & 1, abort_flag)) return false;
+                const float m_o = s_xmax[(half ^ 1) * 128 + r], l_o = s_xsum[(half ^ 1) * 128 + r];
+                const float m_all = fmaxf(pend_m, m_o);           // half 0 always has a valid key, so this is finite
+                const float a_me = pend_m == -INFINITY ? 0.f : ex2((pend_m - m_all) * scale_log2);
+                const float a_ot = m_o == -INFINITY ? 0.f : ex2((m_o - m_all) * scale_log2);
+                const float inv = 1.0f / (a_me * pend_l + a_ot * l_o);
+                const float w_0 = (half == 0 ? a_me : a_ot) * inv, w_1 = (half == 0 ? a_ot : a_me) * inv;   // weights of O_0, O_1
+                // every product of the item must have landed: the last tile, both halves
+                if (!mbar_wait(&pv_done[(pend_ge & 1) * 2], (pend_ge >> 1) & 1, abort_flag)) return false;
+                if (!mbar_wait(&pv_done[(pend_ge & 1) * 2 + 1], (pend_ge >> 1) & 1, abort_flag)) return false;
+                tc_fence_after();
+                // this thread stores columns [32 half, 32 half + 32) of the head
+                uint32_t o0[32], o1[32];
+                tmem_ld32(lane_addr + COL_O + half * 32, o0);
+                tmem_ld32(lane_addr + COL_O + 64 + half * 32, o1);
+                tmem_wait_ld();
+                // the accumulators are free for the next item as soon as they are in registers
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(o_free);
+                // Each thread holds 64 contiguous output bytes of its own row; stored as they are, one store
+                // instruction would touch 32 different lines.  The warp transposes through its staging slots so
+                // that four neighbouring lanes write one row's 64 bytes: 8 lines per instruction.
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    // a zero weight must also silence whatever an untouched accumulator holds
+                    const float x0 = w_0 != 0.f ? __uint_as_float(o0[i]) * w_0 : 0.f;
+                    const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
+                    v[i] = x0 + x1;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint4 u;
+                    u.x = pack_bf16(v[8 * q + 0], v[8 * q + 1]);
+                    u.y = pack_bf16(v[8 * q + 2], v[8 * q + 3]);
+                    u.z = pack_bf16(v[8 * q + 4], v[8 * q + 5]);
+                    u.w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
+                    *reinterpret_cast<uint4*>(stage + q * 16) = u;
+                }
+                __syncwarp();
+                {
+                    const uint8_t* wstage = stage - lane * 80;    // this warp's 32 slots
+                    __nv_bfloat16* obase = o + (size_t)(pend_row0 + quad * 32) * o_ld + pend_head * D + half * 32 + (lane & 3) * 8;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int rr = k * 8 + (lane >> 2);       // row inside the warp's 32
+                        const uint4 u = *reinterpret_cast<const uint4*>(wstage + rr * 80 + (lane & 3) * 16);
+                        if (quad * 32 + rr < pend_rows) *reinterpret_cast<uint4*>(obase + (size_t)rr * o_ld) = u;
+                    }
+                }
+                __syncwarp();                                     // the slots are rewritten at the end of the next item
+                return true;
+            };
+            QTile t_next = blockIdx.x < n_items ? tiles[blockIdx.x % n_tiles] : QTile{0, 0, 0, 0};
             for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
-                const QTile t = tiles[w % n_tiles];
+                const QTile t = t_next;
+                if (w + (int)gridDim.x < n_items) t_next = tiles[(w + gridDim.x) % n_tiles];
                 const int head = w / n_tiles;
                 float m = -INFINITY, l = 0.f;
-                for (int j = 0; j < n_kv && ok; ++j) {
+                auto tile = [&](const int j) -> bool {
                     const uint32_t g = g0 + j, bs = g & 1;
-                    if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) return false;
                     tc_fence_after();
                     uint32_t sr[64];
                     tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64, sr);
@@ -314,7 +385,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         const bool need = (mx - m) * scale_log2 > 8.0f;
                         if (__any_sync(0xffffffffu, need)) {
                             // this half's earlier P V products must have landed before O_h is rescaled
-                            if (!mbar_wait(&pv_done[((g - 1) & 1) * 2 + half], ((g - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                            if (!mbar_wait(&pv_done[((g - 1) & 1) * 2 + half], ((g - 1) >> 1) & 1, abort_flag)) return false;
                             tc_fence_after();
                             const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
                             if (need) { l *= f; m = mx; }
@@ -345,60 +416,26 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                     l += (su0 + su1) + (su2 + su3);
                     // this half of the P buffer is free once the product that read it two tiles ago has completed
-                    if (g >= 2 && !mbar_wait(&pv_done[bs * 2 + half], ((g >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                    if (g >= 2 && !mbar_wait(&pv_done[bs * 2 + half], ((g >> 1) - 1) & 1, abort_flag)) return false;
                     tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pk);
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&p_full[bs * 2 + half]);
-                }
+                    return true;
+                };
+                // the previous item ends after this item's first tile: its last product has had a whole tile's time
+                // to complete, and the first product of this item waits for the accumulators to be handed over
+                if (!tile(0)) { ok = false; break; }
+                if (pend_item >= 0 && !finish()) { ok = false; break; }
+                for (int j = 1; j < n_kv; ++j)
+                    if (!tile(j)) { ok = false; break; }
                 if (!ok) break;
-                // merge the two halves' partial results and store the row
-                s_xmax[half * 128 + r] = m;
-                s_xsum[half * 128 + r] = l;
-                mbar_arrive(&l_bar[quad]);
-                if (!mbar_wait(&l_bar[quad], item_i & 1, abort_flag)) { ok = false; break; }
-                const float m_o = s_xmax[(half ^ 1) * 128 + r], l_o = s_xsum[(half ^ 1) * 128 + r];
-                const float m_all = fmaxf(m, m_o);                // half 0 always has a valid key, so this is finite
-                const float a_me = m == -INFINITY ? 0.f : ex2((m - m_all) * scale_log2);
-                const float a_ot = m_o == -INFINITY ? 0.f : ex2((m_o - m_all) * scale_log2);
-                const float inv = 1.0f / (a_me * l + a_ot * l_o);
-                const float w_0 = (half == 0 ? a_me : a_ot) * inv, w_1 = (half == 0 ? a_ot : a_me) * inv;   // weights of O_0, O_1
-                // every product of this item must have landed: the last tile, both halves
-                const uint32_t ge = g0 + n_kv - 1;
-                if (!mbar_wait(&pv_done[(ge & 1) * 2], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
-                if (!mbar_wait(&pv_done[(ge & 1) * 2 + 1], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                // this thread stores columns [32 half, 32 half + 32) of the head
-                __nv_bfloat16* dst = o + (size_t)(t.row0 + r) * o_ld + head * D + half * 32;
-                uint32_t o0[32], o1[32];
-                tmem_ld32(lane_addr + COL_O + half * 32, o0);
-                tmem_ld32(lane_addr + COL_O + 64 + half * 32, o1);
-                tmem_wait_ld();
-                if (r < t.rows) {
-                    float v[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        // a zero weight must also silence whatever an untouched accumulator holds
-                        const float x0 = w_0 != 0.f ? __uint_as_float(o0[i]) * w_0 : 0.f;
-                        const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
-                        v[i] = x0 + x1;
-                    }
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint4 u;
-                        u.x = pack_bf16(v[8 * q + 0], v[8 * q + 1]);
-                        u.y = pack_bf16(v[8 * q + 2], v[8 * q + 3]);
-                        u.z = pack_bf16(v[8 * q + 4], v[8 * q + 5]);
-                        u.w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
-                        *reinterpret_cast<uint4*>(dst + q * 8) = u;
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(o_free);
+                pend_m = m; pend_l = l; pend_row0 = t.row0; pend_rows = t.rows; pend_head = head; pend_item = item_i;
+                pend_ge = g0 + n_kv - 1;
                 g0 += n_kv;
             }
+            if (ok && pend_item >= 0 && !finish()) ok = false;
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 650 + (int)blockIdx.x);
         } else {
             const int quad = warp & 3;
