@@ -57,6 +57,49 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// ---- two fp32 values per instruction (add/sub/fma .f32x2) --------------------------------------------
+__device__ __forceinline__ uint64_t pair(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpair(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// 2^x for two arguments on the FMA pipe: x = n + f with n the nearest integer, 2^f as a cubic on [-1/2, 1/2]
+// (relative error 7.5e-5, far below the bf16 rounding P gets), n added into the exponent field.  Arguments
+// below -125 are clamped, so a masked score gives 2^-125 instead of 0: nothing a row sum can see.
+__device__ __forceinline__ uint64_t ex2_poly2(uint64_t x) {
+    float xa, xb;
+    unpair(x, xa, xb);
+    x = pair(fmaxf(xa, -125.0f), fmaxf(xb, -125.0f));
+    const uint64_t magic = pair(12582912.0f, 12582912.0f);          // 1.5 * 2^23: the sum's low mantissa bits hold n
+    const uint64_t xn = add2(x, magic);
+    const uint64_t f = sub2(x, sub2(xn, magic));
+    uint64_t pl = fma2(pair(0.0551716648042202f, 0.0551716648042202f), f, pair(0.2426111251115799f, 0.2426111251115799f));
+    pl = fma2(pl, f, pair(0.6932609677314758f, 0.6932609677314758f));
+    pl = fma2(pl, f, pair(0.9999280571937561f, 0.9999280571937561f));
+    float pa, pb, na, nb;
+    unpair(pl, pa, pb);
+    unpair(xn, na, nb);
+    pa = __int_as_float(__float_as_int(pa) + (__float_as_int(na) << 23));
+    pb = __int_as_float(__float_as_int(pb) + (__float_as_int(nb) << 23));
+    return pair(pa, pb);
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&h);
@@ -403,18 +446,35 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                     const float mb = (m == -INFINITY ? 0.f : m) * scale_log2;
                     uint32_t pk[32];
-                    float su0 = 0.f, su1 = 0.f, su2 = 0.f, su3 = 0.f;
+                    // of every 8 exponentials 6 go to the special-function unit and 2 to the FMA pipe: the special-
+                    // function unit alone (16 results per clock and SM) would take longer than the tile's products
+                    const uint64_t sc2 = pair(scale_log2, scale_log2), nmb2 = pair(-mb, -mb);
+                    uint64_t sua = pair(0.f, 0.f), sub_ = pair(0.f, 0.f);
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -mb));
-                        const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -mb));
-                        const float p2 = ex2(fmaf(__uint_as_float(sr[2 * i + 2]), scale_log2, -mb));
-                        const float p3 = ex2(fmaf(__uint_as_float(sr[2 * i + 3]), scale_log2, -mb));
-                        su0 += p0; su1 += p1; su2 += p2; su3 += p3;
-                        pk[i] = pack_bf16(p0, p1);
-                        pk[i + 1] = pack_bf16(p2, p3);
+                    for (int i = 0; i < 32; i += 4) {
+                        float p[8];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const uint64_t x = fma2(pair(__uint_as_float(sr[2 * i + 2 * e]), __uint_as_float(sr[2 * i + 2 * e + 1])), sc2, nmb2);
+                            if (e < 3) {
+                                float xa, xb;
+                                unpair(x, xa, xb);
+                                p[2 * e] = ex2(xa);
+                                p[2 * e + 1] = ex2(xb);
+                            } else {
+                                unpair(ex2_poly2(x), p[2 * e], p[2 * e + 1]);
+                            }
+                        }
+                        sua = add2(sua, add2(pair(p[0], p[1]), pair(p[2], p[3])));
+                        sub_ = add2(sub_, add2(pair(p[4], p[5]), pair(p[6], p[7])));
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) pk[i + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
                     }
-                    l += (su0 + su1) + (su2 + su3);
+                    {
+                        float s0, s1;
+                        unpair(add2(sua, sub_), s0, s1);
+                        l += s0 + s1;
+                    }
                     // this half of the P buffer is free once the product that read it two tiles ago has completed
                     if (g >= 2 && !mbar_wait(&pv_done[bs * 2 + half], ((g >> 1) - 1) & 1, abort_flag)) return false;
                     tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pk);
