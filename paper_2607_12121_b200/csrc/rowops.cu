@@ -281,6 +281,63 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
     ptx::pdl_trigger();
 }
 
+// The same with the row held in registers (NV float4 slots per lane, H = 128 NV): every load of a row is in
+// flight at once and the row is read a single time.
+template <typename T, int NV>
+__global__ void __launch_bounds__(LN_THREADS, 4)
+ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
+                       float* __restrict__ resid_out, T* __restrict__ out, const int32_t* __restrict__ active_idx,
+                       const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
+                       float ln_eps, const Control* __restrict__ ctl) {
+    constexpr int H = NV * 128;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    ptx::pdl_wait();                              // the rows come from the kernel launched just before
+    const int a_total = ctl->a_total;
+    for (int row = blockIdx.x * (LN_THREADS / 32) + warp; row < a_total; row += gridDim.x * (LN_THREADS / 32)) {
+        const int tok = active_idx[row];
+        const int b = tok / N;
+        const size_t g0 = (size_t)tok * H, r0 = (size_t)row * H;
+        float v[NV][4];
+#pragma unroll
+        for (int i = 0; i < NV; ++i) ln_load4<T>(x_gather, resid_in, g0 + (i * 32 + lane) * 4, r0 + (i * 32 + lane) * 4, v[i]);
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) sum += (v[i][0] + v[i][1]) + (v[i][2] + v[i][3]);
+        const float mean = warp_sum(sum) / (float)H;
+        float sq = 0.f;
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { const float d = v[i][k] - mean; sq = fmaf(d, d, sq); }
+        const float rstd = rsqrtf(warp_sum(sq) / (float)H + ln_eps);
+        const float* sh = shift + (size_t)b * mod_stride;
+        const float* sc = scale + (size_t)b * mod_stride;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int c = (i * 32 + lane) * 4;
+            if (x_gather && resid_out)
+                *reinterpret_cast<float4*>(resid_out + r0 + c) = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
+            const float4 s4 = __ldg(reinterpret_cast<const float4*>(sc + c));
+            const float4 h4 = __ldg(reinterpret_cast<const float4*>(sh + c));
+            const float o0 = (v[i][0] - mean) * rstd * (1.f + s4.x) + h4.x;
+            const float o1 = (v[i][1] - mean) * rstd * (1.f + s4.y) + h4.y;
+            const float o2 = (v[i][2] - mean) * rstd * (1.f + s4.z) + h4.z;
+            const float o3 = (v[i][3] - mean) * rstd * (1.f + s4.w) + h4.w;
+            T* dst = out + r0 + c;
+            if constexpr (sizeof(T) == 2) {
+                const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
+                uint2 u;
+                u.x = *reinterpret_cast<const uint32_t*>(&p0);
+                u.y = *reinterpret_cast<const uint32_t*>(&p1);
+                *reinterpret_cast<uint2*>(dst) = u;
+            } else {
+                *reinterpret_cast<float4*>(dst) = make_float4(o0, o1, o2, o3);
+            }
+        }
+    }
+    ptx::pdl_trigger();
+}
+
 // Any width: three passes over the row (the re-reads hit L1/L2).
 template <typename T>
 __global__ void __launch_bounds__(LN_THREADS)
@@ -350,6 +407,18 @@ cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* 
                                cudaStream_t st, int* n_launch, bool pdl) {
     const int rows_per_cta = LN_THREADS / 32;
     const int grid = max(1, min((rows_cap + rows_per_cta - 1) / rows_per_cta, 148 * 16));
+#define FD_LN_REG(NV)                                                                                              \
+    if (H == NV * 128) {                                                                                           \
+        cudaError_t e = ptx::launch_kernel(ln_modulate_reg_kernel<T, NV>, grid, LN_THREADS, 0, st, pdl, x_gather,  \
+                                           resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N,      \
+                                           ln_eps, ctl);                                                           \
+        ++*n_launch;                                                                                               \
+        return e;                                                                                                  \
+    }
+    FD_LN_REG(8)
+    FD_LN_REG(9)
+    FD_LN_REG(12)
+#undef FD_LN_REG
     if (H % 128 == 0) {
         cudaError_t e = ptx::launch_kernel(ln_modulate_kernel<T>, grid, LN_THREADS, 0, st, pdl, x_gather, resid_in, resid_out,
                                            out, active_idx, shift, scale, mod_stride, N, H, ln_eps, ctl);
