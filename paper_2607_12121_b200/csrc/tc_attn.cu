@@ -33,7 +33,7 @@ bool tc_plan_pdl(TcPlan* p);
 
 namespace {
 
-constexpr int ATT_THREADS = 352;
+constexpr int ATT_THREADS = 512;          // 4 warpgroups: TMA/issuers, softmax x 2, item epilogue (head dim 64)
 constexpr int QROWS = 128, KEYS = 128;
 constexpr int SUB_BYTES = 128 * 64 * 2;          // one [128 x 64] bf16 sub-tile, 128-byte rows
 
@@ -49,8 +49,13 @@ template <int D> struct AttCfg {
     static constexpr int TILE_BYTES = SUBS * SUB_BYTES + (D == 72 ? TAIL_BYTES : 0);
     // K/V rings deep enough that a tile is requested several tile periods before it is needed
     static constexpr int STAGES = D == 128 ? 2 : (D == 72 ? 4 : 5);
-    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 3584 + (D == 64 ? 256 * 80 : 0);
+    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + (D == 64 ? 128 * 144 : 0);
 };
+
+// Register re-balancing between warpgroups: the kernel starts with 128 registers per thread (512 threads);
+// the issuing and the epilogue warpgroups give most of theirs back and the two softmax warpgroups take them.
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -105,6 +110,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+// The running maximum of a row is only replaced (and the accumulators rescaled, which stalls the pipeline on the
+// previous product) when the new maximum exceeds it by this many powers of two.  P and the accumulators are
+// floating point with an 8-bit exponent, so a stale maximum costs no precision; 2^24 times the key count times
+// |V| stays far inside the fp32 range.
+constexpr float RESCALE_LOG2 = 24.0f;
+
 // TMEM columns: two score buffers, the output accumulator, two P buffers (bf16 pairs)
 constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384, TMEM_COLS = 512;
 
@@ -136,11 +147,13 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint64_t* o_free = q_empty + 2;
     uint64_t* x_bar = o_free + 1;             // [4 quadrants][2]: the two threads of a row swap their partial maxima
     uint64_t* l_bar = x_bar + 8;              // [4 quadrants]: ... and, once per item, their partial sums
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(l_bar + 4);
+    uint64_t* stat_full = l_bar + 4;          // [2]  head dim 64: an item's row statistics are in shared memory
+    uint64_t* stat_free = stat_full + 2;      // [2]  ... and have been read
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(stat_free + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* s_xmax = reinterpret_cast<float*>(tmem_slot + 2);      // [2 buffers][2 halves][128 rows]
-    float* s_xsum = s_xmax + 512;                                 // [2 halves][128 rows]
-    uint8_t* s_stage = reinterpret_cast<uint8_t*>(bars) + 3584;   // [256 softmax threads][80 bytes], head dim 64 only
+    float* s_xsum = s_xmax + 512;                                 // [2 halves][128 rows]; head dim 64: [2 items][2 halves][128 rows]
+    uint8_t* s_stage = reinterpret_cast<uint8_t*>(bars) + 4608;   // [128 rows][144 bytes], head dim 64 only
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (smem_u32(smem) & 1023u) {                        // never expected; refuse rather than compute garbage
@@ -161,7 +174,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         for (int i = 0; i < 4; ++i) { mbar_init(&p_full[i], SPLIT ? 4 : 8); mbar_init(&pv_done[i], 1); }
         for (int i = 0; i < 8; ++i) mbar_init(&x_bar[i], 64);
         for (int i = 0; i < 4; ++i) mbar_init(&l_bar[i], 64);
-        mbar_init(o_free, 8);
+        mbar_init(o_free, SPLIT ? 4 : 8);
+        for (int i = 0; i < 2; ++i) { mbar_init(&stat_full[i], 8); mbar_init(&stat_free[i], 4); }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tm_q);
@@ -175,6 +189,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const int wg = warp >> 2;                            // 0: TMA + MMA issuers, 1 and 2: softmax, 3: item epilogue
     // everything above is local set-up; from here on the kernel reads what earlier kernels wrote
     pdl_trigger();
     pdl_wait();
@@ -183,6 +198,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int n_tiles = ctl->n_qtiles;
     const int n_items = n_tiles * heads;
 
+    if (wg == 0) {
+    reg_dec<48>();
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
@@ -311,91 +328,21 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 550 + (int)blockIdx.x);
         }
-    } else {
+    }
+    } else if (wg == 1 || wg == 2) {
         // ---------------------------------------------------------------- softmax
+        if constexpr (SPLIT) reg_inc<184>(); else reg_inc<200>();
         if constexpr (SPLIT) {
             const int quad = warp & 3;
-            const int half = (warp - 3) >> 2;                     // which 64 keys of every tile, and which accumulator
+            const int half = wg - 1;                              // which 64 keys of every tile, and which accumulator
             const int r = quad * 32 + lane;                       // query row inside the tile
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
             const uint32_t o_addr = lane_addr + COL_O + half * 64;
-            // staging slot of this thread's 64 output bytes; the slots are 80 bytes apart so that the 16-byte
-            // stores of a quarter warp fall into different banks
-            uint8_t* stage = s_stage + (threadIdx.x - 96) * 80;
             uint32_t g0 = 0;
             bool ok = true;
             int item_i = 0;
             const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
-            // The end of an item (merge the halves, normalise, store) is deferred until the first key tile of
-            // the next item has been through the softmax: the tensor core finishes the last product of the
-            // old item while these warps already work on the new one.
-            float pend_m = 0.f, pend_l = 0.f;
-            int pend_row0 = 0, pend_rows = 0, pend_head = 0, pend_item = -1;
-            uint32_t pend_ge = 0;
-            auto finish = [&]() -> bool {
-                // merge the two halves' partial results and store the row
-                s_xmax[half * 128 + r] = pend_m;
-                s_xsum[half * 128 + r] = pend_l;
-                mbar_arrive(&l_bar[quad]);
-                if (!mbar_wait(&l_bar[quad], pend_item & 1, abort_flag)) return false;
-                const float m_o = s_xmax[(half ^ 1) * 128 + r], l_o = s_xsum[(half ^ 1) * 128 + r];
-                const float m_all = fmaxf(pend_m, m_o);           // half 0 always has a valid key, so this is finite
-                const float a_me = pend_m == -INFINITY ? 0.f : ex2((pend_m - m_all) * scale_log2);
-                const float a_ot = m_o == -INFINITY ? 0.f : ex2((m_o - m_all) * scale_log2);
-                const float inv = 1.0f / (a_me * pend_l + a_ot * l_o);
-                const float w_0 = (half == 0 ? a_me : a_ot) * inv, w_1 = (half == 0 ? a_ot : a_me) * inv;   // weights of O_0, O_1
-                // every product of the item must have landed: the last tile, both halves
-                if (!mbar_wait(&pv_done[(pend_ge & 1) * 2], (pend_ge >> 1) & 1, abort_flag)) return false;
-                if (!mbar_wait(&pv_done[(pend_ge & 1) * 2 + 1], (pend_ge >> 1) & 1, abort_flag)) return false;
-                tc_fence_after();
-                // this thread stores columns [32 half, 32 half + 32) of the head
-                uint32_t o0[32], o1[32];
-                tmem_ld32(lane_addr + COL_O + half * 32, o0);
-                tmem_ld32(lane_addr + COL_O + 64 + half * 32, o1);
-                tmem_wait_ld();
-                // the accumulators are free for the next item as soon as they are in registers
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(o_free);
-                // Each thread holds 64 contiguous output bytes of its own row; stored as they are, one store
-                // instruction would touch 32 different lines.  The warp transposes through its staging slots so
-                // that four neighbouring lanes write one row's 64 bytes: 8 lines per instruction.
-                float v[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    // a zero weight must also silence whatever an untouched accumulator holds
-                    const float x0 = w_0 != 0.f ? __uint_as_float(o0[i]) * w_0 : 0.f;
-                    const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
-                    v[i] = x0 + x1;
-                }
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint4 u;
-                    u.x = pack_bf16(v[8 * q + 0], v[8 * q + 1]);
-                    u.y = pack_bf16(v[8 * q + 2], v[8 * q + 3]);
-                    u.z = pack_bf16(v[8 * q + 4], v[8 * q + 5]);
-                    u.w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
-                    *reinterpret_cast<uint4*>(stage + q * 16) = u;
-                }
-                __syncwarp();
-                {
-                    const uint8_t* wstage = stage - lane * 80;    // this warp's 32 slots
-                    __nv_bfloat16* obase = o + (size_t)(pend_row0 + quad * 32) * o_ld + pend_head * D + half * 32 + (lane & 3) * 8;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int rr = k * 8 + (lane >> 2);       // row inside the warp's 32
-                        const uint4 u = *reinterpret_cast<const uint4*>(wstage + rr * 80 + (lane & 3) * 16);
-                        if (quad * 32 + rr < pend_rows) *reinterpret_cast<uint4*>(obase + (size_t)rr * o_ld) = u;
-                    }
-                }
-                __syncwarp();                                     // the slots are rewritten at the end of the next item
-                return true;
-            };
-            QTile t_next = blockIdx.x < n_items ? tiles[blockIdx.x % n_tiles] : QTile{0, 0, 0, 0};
             for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
-                const QTile t = t_next;
-                if (w + (int)gridDim.x < n_items) t_next = tiles[(w + gridDim.x) % n_tiles];
-                const int head = w / n_tiles;
                 float m = -INFINITY, l = 0.f;
                 auto tile = [&](const int j) -> bool {
                     const uint32_t g = g0 + j, bs = g & 1;
@@ -425,7 +372,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (j == 0) {
                         m = mx;
                     } else if (!no_keys) {
-                        const bool need = (mx - m) * scale_log2 > 8.0f;
+                        const bool need = (mx - m) * scale_log2 > RESCALE_LOG2;
                         if (__any_sync(0xffffffffu, need)) {
                             // this half's earlier P V products must have landed before O_h is rescaled
                             if (!mbar_wait(&pv_done[((g - 1) & 1) * 2 + half], ((g - 1) >> 1) & 1, abort_flag)) return false;
@@ -484,22 +431,23 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (lane == 0) mbar_arrive(&p_full[bs * 2 + half]);
                     return true;
                 };
-                // the previous item ends after this item's first tile: its last product has had a whole tile's time
-                // to complete, and the first product of this item waits for the accumulators to be handed over
-                if (!tile(0)) { ok = false; break; }
-                if (pend_item >= 0 && !finish()) { ok = false; break; }
-                for (int j = 1; j < n_kv; ++j)
+                for (int j = 0; j < n_kv; ++j)
                     if (!tile(j)) { ok = false; break; }
                 if (!ok) break;
-                pend_m = m; pend_l = l; pend_row0 = t.row0; pend_rows = t.rows; pend_head = head; pend_item = item_i;
-                pend_ge = g0 + n_kv - 1;
+                // hand the row's statistics of this half to the epilogue warps and go on with the next item;
+                // the slot was last used two items ago
+                const int slot = item_i & 1;
+                if (item_i >= 2 && !mbar_wait(&stat_free[slot], ((item_i >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                s_xmax[(slot * 2 + half) * 128 + r] = m;
+                s_xsum[(slot * 2 + half) * 128 + r] = l;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&stat_full[slot]);
                 g0 += n_kv;
             }
-            if (ok && pend_item >= 0 && !finish()) ok = false;
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 650 + (int)blockIdx.x);
         } else {
             const int quad = warp & 3;
-            const int half = (warp - 3) >> 2;                     // which 64 keys of a tile / which half of O
+            const int half = wg - 1;                              // which 64 keys of a tile / which half of O
             const int r = quad * 32 + lane;                       // query row inside the tile
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
             // output columns this thread owns: [half * DH, half * DH + DH), and for head dim 72 thread 0 also 64..79
@@ -541,7 +489,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (j == 0) {
                         m = mx;
                     } else {
-                        const bool need = (mx - m) * scale_log2 > 8.0f;
+                        const bool need = (mx - m) * scale_log2 > RESCALE_LOG2;
                         if (__any_sync(0xffffffffu, need)) {
                             // all earlier P V products must have landed before O is rescaled
                             if (!mbar_wait(&pv_done[((g - 1) & 1) * 2], ((g - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -640,6 +588,84 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 g0 += n_kv;
             }
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 600 + (int)blockIdx.x);
+        }
+    } else {
+        // ---------------------------------------------------------------- item epilogue (head dim 64)
+        if constexpr (SPLIT) reg_dec<96>(); else reg_dec<48>();
+        // One thread per query row: merge the two halves' accumulators with the statistics the softmax warps
+        // left, normalise and store, while those warps are already in the next item's key loop.
+        if constexpr (SPLIT) {
+            const int quad = warp & 3;
+            const int r = quad * 32 + lane;
+            const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+            // staging rows are 144 bytes apart so that the 16-byte stores of a quarter warp fall into different banks
+            uint8_t* wstage = s_stage + quad * 32 * 144;
+            uint32_t g0 = 0;
+            bool ok = true;
+            int item_i = 0;
+            QTile t_next = blockIdx.x < n_items ? tiles[blockIdx.x % n_tiles] : QTile{0, 0, 0, 0};
+            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
+                const QTile t = t_next;
+                if (w + (int)gridDim.x < n_items) t_next = tiles[(w + gridDim.x) % n_tiles];
+                const int head = w / n_tiles;
+                const int slot = item_i & 1;
+                if (!mbar_wait(&stat_full[slot], (item_i >> 1) & 1, abort_flag)) { ok = false; break; }
+                const float m0 = s_xmax[(slot * 2 + 0) * 128 + r], l0 = s_xsum[(slot * 2 + 0) * 128 + r];
+                const float m1 = s_xmax[(slot * 2 + 1) * 128 + r], l1 = s_xsum[(slot * 2 + 1) * 128 + r];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&stat_free[slot]);
+                // every product of the item must have landed: the last tile, both halves
+                const uint32_t ge = g0 + n_kv - 1;
+                if (!mbar_wait(&pv_done[(ge & 1) * 2], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&pv_done[(ge & 1) * 2 + 1], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const float m_all = fmaxf(m0, m1);                // half 0 always has a valid key, so this is finite
+                const float a0 = m0 == -INFINITY ? 0.f : ex2((m0 - m_all) * scale_log2);
+                const float a1 = m1 == -INFINITY ? 0.f : ex2((m1 - m_all) * scale_log2);
+                const float inv = 1.0f / (a0 * l0 + a1 * l1);
+                const float w_0 = a0 * inv, w_1 = a1 * inv;       // weights of O_0, O_1
+                // a rolled loop on purpose: this code runs once per item, and the fewer instructions it fetches the
+                // less it disturbs the softmax warps that share the instruction caches
+#pragma unroll 1
+                for (int q = 0; q < 8; ++q) {
+                    uint32_t o0[8], o1[8];
+                    tmem_ld8(lane_addr + COL_O + q * 8, o0);
+                    tmem_ld8(lane_addr + COL_O + 64 + q * 8, o1);
+                    tmem_wait_ld();
+                    if (q == 7) {
+                        // the accumulators are free for the next item as soon as they are in registers
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(o_free);
+                    }
+                    float v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        // a zero weight must also silence whatever an untouched accumulator holds
+                        const float x0 = w_0 != 0.f ? __uint_as_float(o0[i]) * w_0 : 0.f;
+                        const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
+                        v[i] = x0 + x1;
+                    }
+                    uint4 u;
+                    u.x = pack_bf16(v[0], v[1]);
+                    u.y = pack_bf16(v[2], v[3]);
+                    u.z = pack_bf16(v[4], v[5]);
+                    u.w = pack_bf16(v[6], v[7]);
+                    *reinterpret_cast<uint4*>(wstage + lane * 144 + q * 16) = u;
+                }
+                __syncwarp();
+                // eight neighbouring lanes write one row's 128 bytes: 4 lines per store instruction instead of 32
+                __nv_bfloat16* obase = o + (size_t)(t.row0 + quad * 32) * o_ld + head * D + (lane & 7) * 8;
+#pragma unroll 1
+                for (int k = 0; k < 8; ++k) {
+                    const int rr = k * 4 + (lane >> 3);           // row inside the warp's 32
+                    const uint4 u = *reinterpret_cast<const uint4*>(wstage + rr * 144 + (lane & 7) * 16);
+                    if (quad * 32 + rr < t.rows) *reinterpret_cast<uint4*>(obase + (size_t)rr * o_ld) = u;
+                }
+                __syncwarp();                                     // the staging rows are rewritten by the next item
+                g0 += n_kv;
+            }
+            if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 700 + (int)blockIdx.x);
         }
     }
 
