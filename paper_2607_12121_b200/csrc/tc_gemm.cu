@@ -160,16 +160,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 // The MMA is issued by one thread of the pair's first CTA; completion is broadcast to both CTAs'
 // barriers with a multicast commit.  No TMA load is multicast: every CTA fetches its own tiles.
 // ------------------------------------------------------------------------------------------------
-constexpr int PAIR_BN = 256;
+// The tile is 256 rows x PAIR_BN columns with PAIR_BN = 256, or 192 for output widths that are a multiple of
+// 192 but not of 256 (1152, 3456): those would otherwise fall back to 128 x 128 single-CTA tiles, which the
+// operand fetch limits to a quarter of the tensor pipe.
 constexpr int PAIR_STAGES = 5;
-constexpr int PAIR_B_BYTES = 128 * BK * 2;           // this CTA's half of the weight tile
-constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_BYTES;
-constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + 1024 + 256 + EPI_STAGE_BYTES;
+template <int PAIR_BN> struct PairCfg {
+    static constexpr int B_BYTES = (PAIR_BN / 2) * BK * 2;          // this CTA's half of the weight tile
+    static constexpr int STAGE_BYTES = A_TILE_BYTES + B_BYTES;
+    static constexpr int SMEM = PAIR_STAGES * STAGE_BYTES + 1024 + 256 + EPI_STAGE_BYTES;
+    static constexpr int TMEM_COLS = 512;                            // two accumulators of PAIR_BN columns
+};
 
-template <int KIND>
+template <int KIND, int PAIR_BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int n_out,
                     int k_dim, EpiParams ep, Control* ctl) {
+    constexpr int PAIR_B_BYTES = PairCfg<PAIR_BN>::B_BYTES, PAIR_STAGE_BYTES = PairCfg<PAIR_BN>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sA = smem;
@@ -195,7 +201,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         prefetch_tmap(&tm_b);
     }
     if (warp == 1) {
-        tmem_alloc_pair(tmem_slot, 2 * PAIR_BN);
+        tmem_alloc_pair(tmem_slot, PairCfg<PAIR_BN>::TMEM_COLS);
         tmem_relinquish_pair();
     }
     tc_fence_before();
@@ -225,7 +231,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                     const uint32_t bar = map_to_cta(smem_u32(&full[s]), 0);     // the first CTA's barrier counts both halves
                     if (rank == 0) mbar_expect_tx(&full[s], 2 * PAIR_STAGE_BYTES);
                     tma_load_2d_pair(sA + s * A_TILE_BYTES, &tm_a, kt * BK, m * 2 * BM + (int)rank * BM, bar);
-                    tma_load_2d_pair(sB + s * PAIR_B_BYTES, &tm_b, kt * BK, n * PAIR_BN + (int)rank * 128, bar);
+                    tma_load_2d_pair(sB + s * PAIR_B_BYTES, &tm_b, kt * BK, n * PAIR_BN + (int)rank * (PAIR_BN / 2), bar);
                 }
             }
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 700 + (int)blockIdx.x);
@@ -258,7 +264,12 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         }
     } else {
         const int quad = warp & 3;
-        const int chalf = (warp - 2) >> 2;                  // which half of the tile's columns
+        const int chalf = (warp - 2) >> 2;                  // which part of the tile's columns
+        // column ranges of the two warps of a lane quadrant: halves, in whole chunks of the epilogue (32 columns
+        // for the fp32 residual update, 64 for the bf16 outputs)
+        constexpr int CH = KIND == EPI_RESID ? 32 : 64;
+        constexpr int C_SPLIT = ((PAIR_BN / 2 + CH - 1) / CH) * CH;
+        const int c_lo = chalf == 0 ? 0 : C_SPLIT, c_hi = chalf == 0 ? C_SPLIT : PAIR_BN;
         uint32_t t_it = 0;
         bool ok = true;
         for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
@@ -266,13 +277,12 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
             if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * 2 * BM + (int)rank * BM + quad * 32, a_total,
-                                        n * PAIR_BN + chalf * (PAIR_BN / 2), PAIR_BN / 2);
+                                        n * PAIR_BN + c_lo, c_hi - c_lo);
             if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
             epilogue_warp<KIND>(ep, epi_stage + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane,
-                                m * 2 * BM + (int)rank * BM + quad * 32, a_total, t_row, n * PAIR_BN,
-                                chalf * (PAIR_BN / 2), (chalf + 1) * (PAIR_BN / 2));
+                                m * 2 * BM + (int)rank * BM + quad * 32, a_total, t_row, n * PAIR_BN, c_lo, c_hi);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty[acc]), 0));
@@ -285,7 +295,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     cluster_sync_all();                      // neither CTA leaves while its peer may still signal it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc_pair(tmem_base, 2 * PAIR_BN);
+        tmem_dealloc_pair(tmem_base, PairCfg<PAIR_BN>::TMEM_COLS);
     }
 }
 
@@ -322,6 +332,7 @@ EncodeTiledFn encode_fn(std::string* err) {
 }
 
 int pick_bn(int n_out) { return (n_out % 256 == 0) ? 256 : 128; }
+int pick_pair_bn(int n_out) { return n_out % 256 == 0 ? 256 : (n_out % 192 == 0 ? 192 : 0); }
 
 }  // namespace
 
@@ -350,7 +361,7 @@ bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* di
 struct GemmSpec {
     CUtensorMap a;              // activation operand
     int n_out, k, bn;
-    bool pair;                  // CTA-pair kernel (256 x 256 tiles); weight boxes are then 128 rows
+    int pair_bn;                // CTA-pair kernel with 256 x pair_bn tiles (0: single-CTA kernel); weight boxes are then pair_bn / 2 rows
 };
 
 struct TcPlan {
@@ -406,14 +417,14 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         s.n_out = n_out[g];
         s.k = kdim[g];
         s.bn = pick_bn(n_out[g]);
-        s.pair = use_pair && (n_out[g] % PAIR_BN == 0);
+        s.pair_bn = use_pair ? pick_pair_bn(n_out[g]) : 0;
         const uint64_t dims[2] = {(uint64_t)kdim[g], (uint64_t)buf.Mcap};
         const uint64_t strides[1] = {(uint64_t)kdim[g] * 2};
         const uint32_t box[2] = {BK, BM};
         ok = encode_tmap_bf16(&s.a, a_base[g], 2, dims, strides, box, 128, err);
         for (int l = 0; l < cfg.n_blocks && ok; ++l) {
             const uint64_t wd[2] = {(uint64_t)kdim[g], (uint64_t)n_out[g]};
-            const uint32_t wb[2] = {BK, s.pair ? 128u : (uint32_t)s.bn};
+            const uint32_t wb[2] = {BK, s.pair_bn ? (uint32_t)s.pair_bn / 2 : (uint32_t)s.bn};
             void* base = const_cast<char*>(w_base[g]) + (size_t)l * n_out[g] * kdim[g] * 2;
             ok = encode_tmap_bf16(&p->w_maps[(size_t)l * 4 + g], base, 2, wd, strides, wb, 128, err);
         }
@@ -426,10 +437,11 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         FD_SET_SMEM(EPI_QKV, 128) FD_SET_SMEM(EPI_QKV, 256) FD_SET_SMEM(EPI_RESID, 128) FD_SET_SMEM(EPI_RESID, 256)
         FD_SET_SMEM(EPI_GELU, 128) FD_SET_SMEM(EPI_GELU, 256)
 #undef FD_SET_SMEM
-#define FD_SET_PAIR(K)                                                                                     \
+#define FD_SET_PAIR(K, N)                                                                                  \
     if (e == cudaSuccess)                                                                                  \
-        e = cudaFuncSetAttribute(tc_gemm_pair_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM);
-        FD_SET_PAIR(EPI_QKV) FD_SET_PAIR(EPI_RESID) FD_SET_PAIR(EPI_GELU)
+        e = cudaFuncSetAttribute(tc_gemm_pair_kernel<K, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<N>::SMEM);
+        FD_SET_PAIR(EPI_QKV, 256) FD_SET_PAIR(EPI_RESID, 256) FD_SET_PAIR(EPI_GELU, 256)
+        FD_SET_PAIR(EPI_QKV, 192) FD_SET_PAIR(EPI_RESID, 192) FD_SET_PAIR(EPI_GELU, 192)
 #undef FD_SET_PAIR
         if (e != cudaSuccess) {
             ok = false;
@@ -442,14 +454,14 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         cudaLaunchConfig_t lc = {};
         lc.gridDim = dim3(p->sm_count & ~1);
         lc.blockDim = dim3(GEMM_THREADS);
-        lc.dynamicSmemBytes = PAIR_SMEM;
+        lc.dynamicSmemBytes = PairCfg<256>::SMEM;
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         lc.attrs = at;
         lc.numAttrs = 1;
         int n_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&n_clusters, tc_gemm_pair_kernel<EPI_GELU>, &lc) == cudaSuccess && n_clusters > 0)
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, tc_gemm_pair_kernel<EPI_GELU, 256>, &lc) == cudaSuccess && n_clusters > 0)
             p->pair_ctas = min(p->sm_count & ~1, 2 * n_clusters);
         else
             cudaGetLastError();
@@ -489,15 +501,19 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
     const CUtensorMap& wm = p->w_maps[(size_t)blk * 4 + kind];
     Control* c = const_cast<Control*>(ctl);
     const int grid = p->sm_count;
-    if (s.pair) {
+    if (s.pair_bn) {
         const int pgrid = max(2, min(grid & ~1, p->pair_ctas));
-        cudaError_t e;
-        if (kind == TC_GEMM_QKV)
-            e = launch_kernel(tc_gemm_pair_kernel<EPI_QKV>, pgrid, GEMM_THREADS, PAIR_SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c);
-        else if (kind == TC_GEMM_FC1)
-            e = launch_kernel(tc_gemm_pair_kernel<EPI_GELU>, pgrid, GEMM_THREADS, PAIR_SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c);
-        else
-            e = launch_kernel(tc_gemm_pair_kernel<EPI_RESID>, pgrid, GEMM_THREADS, PAIR_SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c);
+        cudaError_t e = cudaSuccess;
+#define FD_LAUNCH_PAIR(K, N) \
+    e = launch_kernel(tc_gemm_pair_kernel<K, N>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c)
+        if (kind == TC_GEMM_QKV) {
+            if (s.pair_bn == 256) FD_LAUNCH_PAIR(EPI_QKV, 256); else FD_LAUNCH_PAIR(EPI_QKV, 192);
+        } else if (kind == TC_GEMM_FC1) {
+            if (s.pair_bn == 256) FD_LAUNCH_PAIR(EPI_GELU, 256); else FD_LAUNCH_PAIR(EPI_GELU, 192);
+        } else {
+            if (s.pair_bn == 256) FD_LAUNCH_PAIR(EPI_RESID, 256); else FD_LAUNCH_PAIR(EPI_RESID, 192);
+        }
+#undef FD_LAUNCH_PAIR
         ++*n_launch;
         return e;
     }
