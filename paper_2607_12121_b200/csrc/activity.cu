@@ -1,12 +1,15 @@
 // Patch Gate on the latent change (paper Sec. 4.2; Appendix A.1 Eq. delta-i, Eq. gate-weight,
 // Eq. forced-reactivation).
 //
-// Kernel 1 streams z_cur / z_prev once with 128-bit loads and accumulates, per region, the sum of
-// squared differences (fp32 inside a token, fp64 across tokens) and the token count.  Tokens of
-// regions whose change magnitude is frozen (skipped at the previous step) are not read at all.
+// Kernel 1 streams z_cur / z_prev once and accumulates, per region, the sum of squared differences
+// (fp32 within a run of tokens of one region, fp64 across runs and CTAs) and the token count.  Tokens of
+// regions whose change magnitude is frozen (skipped at the previous step) are not read at all.  Its main
+// form stages both operands through shared memory with bulk copies (below); rows wider than a ring
+// stage, unaligned rows and very large region counts take the plain-load forms.
 // Kernel 2 (one CTA per request) turns the sums into delta, weights, mask and the next state, and
 // clears the accumulators for the next call.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace fd {
 
@@ -103,6 +106,168 @@ activity_reduce_kernel(const float4* __restrict__ z_cur, const float4* __restric
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The streaming form of kernel 1.  z is [B, N, D] contiguous, so a CTA's share of the B*N tokens is
+// one byte range of z_cur and one of z_prev.  A producer warp brings both in with bulk copies,
+// 8 KB per operand and ring stage, several stages ahead; eight consumer warps reduce a stage from
+// shared memory.  The bytes in flight no longer depend on registers or occupancy, which is what a
+// read-only stream needs to approach the HBM rate.  A chunk whose tokens all belong to frozen
+// regions is not copied at all.
+// ---------------------------------------------------------------------------------------------
+constexpr int BULK_STAGES = 4;
+constexpr int BULK_CHUNK_BYTES = 8192;                   // per operand and stage
+constexpr int BULK_MAX_TOK = BULK_CHUNK_BYTES / 16;      // tokens of a chunk at the narrowest row (D = 4)
+constexpr int BULK_CONSUMERS = 256;
+constexpr int BULK_THREADS = BULK_CONSUMERS + 32;
+constexpr int BULK_FIXED_SMEM = BULK_STAGES * 2 * BULK_CHUNK_BYTES + BULK_STAGES * BULK_MAX_TOK * 4 + 128;
+
+__global__ void __launch_bounds__(BULK_THREADS)
+activity_reduce_bulk_kernel(const char* __restrict__ z_cur, const char* __restrict__ z_prev,
+                            const int32_t* __restrict__ labels, const uint8_t* __restrict__ prev_active,
+                            int B, int N, int V, int R, int c_tok, long long tokens_per_cta,
+                            double* __restrict__ acc_ss, int32_t* __restrict__ acc_cnt, Control* ctl) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* ring = smem;                                          // [stage][operand][BULK_CHUNK_BYTES]
+    int* s_lab = reinterpret_cast<int*>(smem + BULK_STAGES * 2 * BULK_CHUNK_BYTES);   // [stage][token]: region, or -1 = not read
+    uint64_t* full = reinterpret_cast<uint64_t*>(s_lab + BULK_STAGES * BULK_MAX_TOK);
+    uint64_t* empty = full + BULK_STAGES;
+    int* s_skip = reinterpret_cast<int*>(empty + BULK_STAGES);           // [stage]: nothing was copied
+    volatile int* abort_flag = s_skip + BULK_STAGES;
+    double* s_ss = reinterpret_cast<double*>(smem + BULK_FIXED_SMEM);
+    int32_t* s_cnt = reinterpret_cast<int32_t*>(s_ss + R);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row_bytes = V * 16;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < BULK_STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], BULK_CONSUMERS / 32); }
+        *abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    for (int i = threadIdx.x; i < R; i += BULK_THREADS) { s_ss[i] = 0.0; s_cnt[i] = 0; }
+    __syncthreads();
+    const long long total = (long long)B * N;
+    const long long lo = (long long)blockIdx.x * tokens_per_cta;
+    const long long hi = lo + tokens_per_cta < total ? lo + tokens_per_cta : total;
+    uint32_t it = 0;                                     // ring position, continues across requests
+    bool ok = true;
+    // lanes sharing one token: the largest power of two dividing gcd(V, 32)
+    int group = 1;
+    while (group < 32 && (V % (group * 2)) == 0) group *= 2;
+    const bool leader = (lane & (group - 1)) == 0;
+    const int q_step = 32 / V, r_step = 32 % V;          // how token index and vector index move when i grows by 32
+    if (lo < hi) {
+        for (int b = (int)(lo / N); b <= (int)((hi - 1) / N); ++b) {
+            const long long s0 = lo > (long long)b * N ? lo : (long long)b * N;
+            const long long s1 = hi < (long long)(b + 1) * N ? hi : (long long)(b + 1) * N;
+            const int n_chunks = (int)((s1 - s0 + c_tok - 1) / c_tok);
+            if (warp == BULK_CONSUMERS / 32) {
+                // ------------------------------------------------------------ producer warp
+                const uint8_t* pa_b = prev_active + (size_t)b * R;
+                for (int k = 0; k < n_chunks && ok; ++k, ++it) {
+                    const int st = it % BULK_STAGES;
+                    const long long g0 = s0 + (long long)k * c_tok;
+                    const int n_tok = (int)(s1 - g0 < c_tok ? s1 - g0 : c_tok);
+                    if (!ptx::mbar_wait(&empty[st], ((it / BULK_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    // what the consumers need to know about the chunk's tokens: the region whose sum a token
+                    // feeds, or -1 (background token, or a region whose change magnitude is frozen)
+                    bool live = false;
+                    for (int t = lane; t < n_tok; t += 32) {
+                        int l = __ldg(labels + g0 + t);
+                        if (l < 0 || l > R) {
+                            report(ctl, FD_ERR_STATE, (int)((g0 + t) % N));
+                            l = -1;
+                        } else if (l == R || !__ldg(pa_b + l)) {
+                            l = -1;
+                        }
+                        s_lab[st * BULK_MAX_TOK + t] = l;
+                        live |= l >= 0;
+                    }
+                    live = __any_sync(0xffffffffu, live);
+                    __syncwarp();                                        // every lane's labels are written before lane 0 signals
+                    if (lane == 0) {
+                        s_skip[st] = live ? 0 : 1;
+                        if (live) {
+                            const uint32_t bytes = (uint32_t)n_tok * row_bytes;
+                            ptx::mbar_expect_tx(&full[st], 2 * bytes);
+                            ptx::bulk_load(ring + (st * 2 + 0) * BULK_CHUNK_BYTES, z_cur + (size_t)g0 * row_bytes, bytes, &full[st]);
+                            ptx::bulk_load(ring + (st * 2 + 1) * BULK_CHUNK_BYTES, z_prev + (size_t)g0 * row_bytes, bytes, &full[st]);
+                        } else {
+                            ptx::mbar_arrive(&full[st]);
+                        }
+                    }
+                    __syncwarp();
+                }
+                if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 1000 + (int)blockIdx.x);
+            } else {
+                // ------------------------------------------------------------ consumer warps
+                // Every lane sums "its" vector column over consecutive tokens of one region; the lanes of a
+                // token are only added up (and the shared accumulators touched) when the region changes.
+                int cur_lab = -1, cur_cnt = 0;
+                float cur_sum = 0.f;
+                auto flush = [&](bool chg, int next_lab) {
+                    float v = chg ? cur_sum : 0.f;
+                    for (int o = group >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (chg) {
+                        if (leader && cur_lab >= 0) {
+                            atomicAdd(&s_ss[cur_lab], (double)v);
+                            if (cur_cnt) atomicAdd(&s_cnt[cur_lab], cur_cnt);
+                        }
+                        cur_lab = next_lab;
+                        cur_sum = 0.f;
+                        cur_cnt = 0;
+                    }
+                };
+                for (int k = 0; k < n_chunks && ok; ++k, ++it) {
+                    const int st = it % BULK_STAGES;
+                    if (!ptx::mbar_wait(&full[st], (it / BULK_STAGES) & 1, abort_flag)) { ok = false; break; }
+                    if (!s_skip[st]) {
+                        const long long g0 = s0 + (long long)k * c_tok;
+                        const int n_tok = (int)(s1 - g0 < c_tok ? s1 - g0 : c_tok);
+                        // every warp takes a contiguous run of the chunk's tokens
+                        const int tok_per_warp = (n_tok + BULK_CONSUMERS / 32 - 1) / (BULK_CONSUMERS / 32);
+                        const int w0 = min(warp * tok_per_warp, n_tok);
+                        const int w1 = min(w0 + tok_per_warp, n_tok);
+                        const int n_vec = (w1 - w0) * V;
+                        const float4* cur = reinterpret_cast<const float4*>(ring + (st * 2 + 0) * BULK_CHUNK_BYTES) + w0 * V;
+                        const float4* prv = reinterpret_cast<const float4*>(ring + (st * 2 + 1) * BULK_CHUNK_BYTES) + w0 * V;
+                        const int* lab = s_lab + st * BULK_MAX_TOK + w0;
+                        int tok = lane / V, vi = lane - tok * V;         // token and vector index of element i = i0 + lane
+                        for (int i0 = 0; i0 < n_vec; i0 += 32) {
+                            const int i = i0 + lane;
+                            const bool in = i < n_vec;
+                            const int l = in ? lab[tok] : cur_lab;       // lanes past the end keep their state
+                            if (__any_sync(0xffffffffu, l != cur_lab)) flush(l != cur_lab, l);
+                            if (in && l >= 0) {
+                                const float4 a = cur[i], p = prv[i];
+                                const float dx = a.x - p.x, dy = a.y - p.y, dz = a.z - p.z, dw = a.w - p.w;
+                                cur_sum += dx * dx + dy * dy + dz * dz + dw * dw;
+                                cur_cnt += vi == 0 ? 1 : 0;              // first vector of the token: counts the token once
+                            }
+                            tok += q_step;
+                            vi += r_step;
+                            if (vi >= V) { vi -= V; ++tok; }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&empty[st]);
+                }
+                flush(true, -1);                                         // the request ends: nothing stays in registers
+                if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 1100 + (int)blockIdx.x);
+            }
+            // the request's sums leave the CTA before the next request's tokens are added
+            __syncthreads();
+            for (int i = threadIdx.x; i < R; i += BULK_THREADS) {
+                if (s_cnt[i] != 0 || s_ss[i] != 0.0) {
+                    atomicAdd(&acc_ss[(size_t)b * R + i], s_ss[i]);
+                    atomicAdd(&acc_cnt[(size_t)b * R + i], s_cnt[i]);
+                    s_ss[i] = 0.0;
+                    s_cnt[i] = 0;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
 // Scalar fallback when D is not a multiple of 4 or the rows are not 16-byte aligned.
 __global__ void __launch_bounds__(ACT_THREADS)
 activity_reduce_scalar_kernel(const float* __restrict__ z_cur, const float* __restrict__ z_prev,
@@ -177,7 +342,26 @@ cudaError_t launch_activity(const float* z_cur, const float* z_prev, const int32
                             int K, double* acc_ss, int32_t* acc_cnt, Control* ctl, cudaStream_t st,
                             int* n_launch) {
     const bool vec = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(z_cur) | reinterpret_cast<uintptr_t>(z_prev)) % 16 == 0);
-    if (vec) {
+    const size_t bulk_smem = (size_t)BULK_FIXED_SMEM + (size_t)R * (sizeof(double) + sizeof(int32_t));
+    if (vec && D * 4 <= BULK_CHUNK_BYTES && bulk_smem <= 200 * 1024) {
+        const int V = D / 4;
+        const int c_tok = BULK_CHUNK_BYTES / (D * 4);
+        // three CTAs per SM fit (64 KB of ring each); every CTA gets one contiguous share of the B*N tokens, at
+        // least four chunks so that the ring fills, in whole chunks
+        const long long total = (long long)B * N;
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const long long max_ctas = (long long)sms * 3;
+        long long per = (total + max_ctas - 1) / max_ctas;
+        if (per < 4LL * c_tok) per = 4LL * c_tok;
+        per = (per + c_tok - 1) / c_tok * c_tok;
+        const int grid = (int)((total + per - 1) / per);
+        cudaError_t ea = cudaFuncSetAttribute(activity_reduce_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk_smem);
+        if (ea != cudaSuccess) return ea;
+        activity_reduce_bulk_kernel<<<grid, BULK_THREADS, bulk_smem, st>>>(
+            reinterpret_cast<const char*>(z_cur), reinterpret_cast<const char*>(z_prev), labels, prev_active, B, N, V,
+            R, c_tok, per, acc_ss, acc_cnt, ctl);
+    } else if (vec) {
         const int V = D / 4;
         // At least 32 KB of each operand per CTA (enough work to amortise set-up and the flush); for large
         // batches fewer, longer chunks: about 16 CTAs per SM in total keep every SM streaming without a long tail.
