@@ -151,7 +151,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint64_t* stat_free = stat_full + 2;      // [2]  ... and have been read
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(stat_free + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    float* s_xmax = reinterpret_cast<float*>(tmem_slot + 2);      // [2 buffers][2 halves][128 rows]
+    float* s_xmax = reinterpret_cast<float*>(tmem_slot + 2);      // head dim 64: row maxima, [2 items][2 halves][128 rows]
     float* s_xsum = s_xmax + 512;                                 // [2 halves][128 rows]; head dim 64: [2 items][2 halves][128 rows]
     uint8_t* s_stage = reinterpret_cast<uint8_t*>(bars) + 4608;   // [128 rows][144 bytes], head dim 64 only
 
@@ -231,13 +231,19 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                     &k_full[s]);
                     if (!mbar_wait(&v_empty[s], ph, abort_flag)) { ok = false; break; }
                     mbar_expect_tx(&v_full[s], TILE_BYTES);
+                    if constexpr (D == 72) {
+                        // V of a 72-wide head as five 16-column blocks (32-byte swizzle): one product of width 80 then
+                        // reads all of them, where a 64-wide plus a 16-wide block would need two products per 16 keys
 #pragma unroll
-                    for (int sb = 0; sb < Cfg::SUBS; ++sb)
-                        tma_load_3d(sV + s * TILE_BYTES + sb * SUB_BYTES, &tm_kv, head * D + sb * 64, j * KEYS,
-                                    t.b * 2 + 1, &v_full[s]);
-                    if constexpr (D == 72)
-                        tma_load_3d(sV + s * TILE_BYTES + SUB_BYTES, &tm_kv_tail, head * D + 64, j * KEYS, t.b * 2 + 1,
-                                    &v_full[s]);
+                        for (int a = 0; a < 5; ++a)
+                            tma_load_3d(sV + s * TILE_BYTES + a * TAIL_BYTES, &tm_kv_tail, head * D + a * 16, j * KEYS,
+                                        t.b * 2 + 1, &v_full[s]);
+                    } else {
+#pragma unroll
+                        for (int sb = 0; sb < Cfg::SUBS; ++sb)
+                            tma_load_3d(sV + s * TILE_BYTES + sb * SUB_BYTES, &tm_kv, head * D + sb * 64, j * KEYS,
+                                        t.b * 2 + 1, &v_full[s]);
+                    }
                 }
             }
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 400 + (int)blockIdx.x);
@@ -281,8 +287,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     } else if (warp == 2) {
         // ---------------------------------------------------------------- O += P V issuer
         if (lane == 0) {
-            constexpr uint32_t idesc_pv = idesc_bf16(QROWS, D == 72 ? 64 : D, 0, 1);   // V: head dim contiguous (N-major)
-            constexpr uint32_t idesc_pv_tail = idesc_bf16(QROWS, 16, 0, 1);
+            constexpr uint32_t idesc_pv = idesc_bf16(QROWS, DP, 0, 1);   // V: head dim contiguous (N-major)
             uint32_t g = 0;
             bool ok = true;
             int item_i = 0;
@@ -315,12 +320,14 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const uint32_t a = tmem_base + COL_P + (g & 1) * 64;
 #pragma unroll
                     for (int ks = 0; ks < KEYS / 16; ++ks) {
-                        // 16 keys further: 16 rows of 128 bytes; the second 64-wide half of V sits SUB_BYTES away
-                        mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
-                                    (j | ks) != 0);
-                        if constexpr (D == 72)  // output columns 64..79 from the 16-wide sub-tile (16 keys = 512 bytes)
-                            mma_bf16_ts(d + 64, a + ks * 8, smem_desc(v_addr + SUB_BYTES + ks * 512, 16, 256, SWZ_32B),
-                                        idesc_pv_tail, (j | ks) != 0);
+                        if constexpr (D == 72)
+                            // 16 keys further: two 8-key groups of 256 bytes; the 16-column blocks sit TAIL_BYTES apart
+                            mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 512, TAIL_BYTES, 256, SWZ_32B), idesc_pv,
+                                        (j | ks) != 0);
+                        else
+                            // 16 keys further: 16 rows of 128 bytes; the second 64-wide half of V sits SUB_BYTES away
+                            mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
+                                        (j | ks) != 0);
                     }
                     mma_commit(&v_empty[s]);
                     mma_commit(&pv_done[(g & 1) * 2]);
@@ -520,18 +527,34 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                     const float mb = m * scale_log2;
                     uint32_t pk[32];
-                    float su0 = 0.f, su1 = 0.f, su2 = 0.f, su3 = 0.f;
-    #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -mb));
-                        const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -mb));
-                        const float p2 = ex2(fmaf(__uint_as_float(sr[2 * i + 2]), scale_log2, -mb));
-                        const float p3 = ex2(fmaf(__uint_as_float(sr[2 * i + 3]), scale_log2, -mb));
-                        su0 += p0; su1 += p1; su2 += p2; su3 += p3;
-                        pk[i] = pack_bf16(p0, p1);
-                        pk[i + 1] = pack_bf16(p2, p3);
+                    // of every 8 exponentials 6 go to the special-function unit and 2 to the FMA pipe
+                    const uint64_t sc2 = pair(scale_log2, scale_log2), nmb2 = pair(-mb, -mb);
+                    uint64_t sua = pair(0.f, 0.f), sub_ = pair(0.f, 0.f);
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        float p[8];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const uint64_t x = fma2(pair(__uint_as_float(sr[2 * i + 2 * e]), __uint_as_float(sr[2 * i + 2 * e + 1])), sc2, nmb2);
+                            if (e < 3) {
+                                float xa, xb;
+                                unpair(x, xa, xb);
+                                p[2 * e] = ex2(xa);
+                                p[2 * e + 1] = ex2(xb);
+                            } else {
+                                unpair(ex2_poly2(x), p[2 * e], p[2 * e + 1]);
+                            }
+                        }
+                        sua = add2(sua, add2(pair(p[0], p[1]), pair(p[2], p[3])));
+                        sub_ = add2(sub_, add2(pair(p[4], p[5]), pair(p[6], p[7])));
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) pk[i + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
                     }
-                    l += (su0 + su1) + (su2 + su3);
+                    {
+                        float s0, s1;
+                        unpair(add2(sua, sub_), s0, s1);
+                        l += s0 + s1;
+                    }
                     // the P buffer is free once the product that read it two tiles ago has completed
                     if (g >= 2 && !mbar_wait(&pv_done[bs * 2], ((g >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
                     tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pk);
