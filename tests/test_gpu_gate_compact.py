@@ -92,6 +92,49 @@ def test_gate_odd_channel_count_uses_scalar_path():
     np.testing.assert_allclose(score, o_score, rtol=1e-5)
 
 
+def test_gate_streaming_kernel_edges():
+    """Shapes that cross every boundary of the streaming reduction: a token count that is no multiple of the ring
+    stage, a channel count whose vector count is no power of two, requests that share a CTA, runs of frozen
+    regions longer than a stage (copied by nobody), always-active tokens (label R) and a frozen/fresh mix."""
+    B, N, D, R, K, eta = 3, 1000, 48, 7, 5, 1e-12
+    rng = np.random.default_rng(123)
+    labels = np.empty((B, N), np.int32)
+    for b in range(B):
+        t, runs = 0, []
+        while t < N:
+            n = int(rng.integers(1, 260))
+            runs.append((min(n, N - t), int(rng.integers(0, R + 1))))
+            t += n
+        labels[b] = np.concatenate([np.full(n, l, np.int32) for n, l in runs])[:N]
+    labels[0, 100:420] = 2                                  # a long run of a region that is frozen below
+    z_prev = rng.standard_normal((B, N, D)).astype(np.float32)
+    scale = np.float32(10.0) ** rng.uniform(-3, -1, size=(B, N, 1)).astype(np.float32)
+    z_cur = (z_prev + scale * rng.standard_normal((B, N, D)).astype(np.float32)).astype(np.float32)
+    ost = oracle.initial_state(B, R)
+    ost["prev_active"][:, 2] = 0
+    ost["prev_active"][1, 5] = 0
+    ost["delta"][:, 2] = np.float32(0.02)
+    ost["delta"][1, 5] = np.float32(0.004)
+    ost["skip_count"][:, 2] = 1
+    ost["skip_count"][1, 5] = 2
+    eps = np.array([0.11, 0.14, 0.17], np.float32)
+    st = GateState(B, R)
+    st.delta.copy_(dev(ost["delta"])); st.skip.copy_(dev(ost["skip_count"])); st.prev.copy_(dev(ost["prev_active"]))
+    o_score, o_weight, o_mask = oracle.activity_gate(z_cur, z_prev, labels, eps, ost, R, K=K, eta=eta)
+    assert np.abs(o_weight / eps[:, None] - 1).min() >= 1e-3       # no decision sits on the threshold
+    assert 0 < o_mask.sum() < B * R
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    fd.fd_region_activity_noalloc(dev(z_cur), dev(z_prev), dev(labels), R, dev(eps), eta, K, st.delta, st.skip,
+                                  st.prev, st.score, st.weight, st.mask, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(host(st.mask), o_mask)
+    np.testing.assert_allclose(host(st.score), o_score, rtol=1e-5, atol=0)
+    np.testing.assert_allclose(host(st.weight), o_weight, rtol=1e-5, atol=0)
+    assert np.array_equal(host(st.prev), ost["prev_active"])
+    assert np.array_equal(host(st.skip), ost["skip_count"])
+
+
 @pytest.mark.parametrize("name", ["tiny", "audio_small", "mmdit_small", "video_small"])
 def test_compaction_bit_exact(name):
     from harness import StepBuffers, gpu_step
