@@ -137,11 +137,17 @@ def test_small_twins_tensor_core_engine(name):
     _run_sequence(wl, 2, fd.FD_ENGINE_TC, masks)
 
 
-def test_tensor_core_engine_few_ctas_walk_many_tiles(monkeypatch):
-    """Two persistent CTAs process every tile: the shared-memory ring and both TMEM accumulator
-    stages wrap around many times."""
+@pytest.mark.parametrize("name,n_tok", [("audio_tc", None), ("audio_tc", 130), ("audio_tc", 100), ("image_tc", None),
+                                        ("wide_tc", None)])
+def test_tensor_core_engine_few_ctas_walk_many_tiles(monkeypatch, name, n_tok):
+    """Two persistent CTAs process every tile: the shared-memory rings and both TMEM accumulator
+    stages wrap around many times, and every attention CTA runs many items back to back (with four, two
+    and one key tiles per item: the hand-over of an item's statistics and accumulators to the epilogue
+    warps, and of the score / P buffers between items, at every key-loop length)."""
     monkeypatch.setenv("FD_TC_MAX_CTAS", "2")
-    wl = gen.workload("audio_tc")
+    wl = gen.workload(name)
+    if n_tok is not None:
+        wl = wl.replace(grid=(n_tok,), R=10, L=1)
     masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 5, [0.6] * wl.B)]
     _run_sequence(wl, 3, fd.FD_ENGINE_TC, masks)
 
