@@ -85,7 +85,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m = tile % m_tiles, n = tile / m_tiles;
+                const int m = tile / n_tiles, n = tile % n_tiles;
                 for (int kt = 0; kt < k_tiles; ++kt, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
@@ -129,7 +129,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         uint32_t t_it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t_it) {
-            const int m = tile % m_tiles, n = tile / m_tiles;
+            const int m = tile / n_tiles, n = tile % n_tiles;
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
             if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * BM + quad * 32, a_total, n * BN + chalf * (BN / 2), BN / 2);
@@ -223,7 +223,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             uint32_t it = 0;
             bool ok = true;
             for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
-                const int m = tile % m_pairs, n = tile / m_pairs;
+                const int m = tile / n_tiles, n = tile % n_tiles;
                 for (int kt = 0; kt < k_tiles; ++kt, ++it) {
                     const int s = it % PAIR_STAGES;
                     const uint32_t ph = (it / PAIR_STAGES) & 1;
@@ -273,7 +273,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         uint32_t t_it = 0;
         bool ok = true;
         for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
-            const int m = tile % m_pairs, n = tile / m_pairs;
+            const int m = tile / n_tiles, n = tile % n_tiles;
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
             if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * 2 * BM + (int)rank * BM + quad * 32, a_total,
