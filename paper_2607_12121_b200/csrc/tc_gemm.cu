@@ -174,7 +174,7 @@ template <int PAIR_BN> struct PairCfg {
 template <int KIND, int PAIR_BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int n_out,
-                    int k_dim, EpiParams ep, Control* ctl) {
+                    int k_dim, int stream_a, EpiParams ep, Control* ctl) {
     constexpr int PAIR_B_BYTES = PairCfg<PAIR_BN>::B_BYTES, PAIR_STAGE_BYTES = PairCfg<PAIR_BN>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -222,6 +222,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            const uint64_t evict_first = l2_evict_first();
             for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
                 const int m = tile / n_tiles, n = tile % n_tiles;
                 for (int kt = 0; kt < k_tiles; ++kt, ++it) {
@@ -230,7 +231,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                     if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
                     const uint32_t bar = map_to_cta(smem_u32(&full[s]), 0);     // the first CTA's barrier counts both halves
                     if (rank == 0) mbar_expect_tx(&full[s], 2 * PAIR_STAGE_BYTES);
-                    tma_load_2d_pair(sA + s * A_TILE_BYTES, &tm_a, kt * BK, m * 2 * BM + (int)rank * BM, bar);
+                    if (stream_a)
+                        tma_load_2d_pair_hint(sA + s * A_TILE_BYTES, &tm_a, kt * BK, m * 2 * BM + (int)rank * BM, bar, evict_first);
+                    else
+                        tma_load_2d_pair(sA + s * A_TILE_BYTES, &tm_a, kt * BK, m * 2 * BM + (int)rank * BM, bar);
                     tma_load_2d_pair(sB + s * PAIR_B_BYTES, &tm_b, kt * BK, n * PAIR_BN + (int)rank * (PAIR_BN / 2), bar);
                 }
             }
@@ -503,9 +507,12 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
     const int grid = p->sm_count;
     if (s.pair_bn) {
         const int pgrid = max(2, min(grid & ~1, p->pair_ctas));
+        // fc2's input (rows x mlp_dim) is the one operand of the step larger than what L2 keeps beside the residual
+        // stream; each of its row blocks is read by the block's column tiles together and then not again
+        const int stream_a = kind == TC_GEMM_FC2 ? 1 : 0;
         cudaError_t e = cudaSuccess;
 #define FD_LAUNCH_PAIR(K, N) \
-    e = launch_kernel(tc_gemm_pair_kernel<K, N>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c)
+    e = launch_kernel(tc_gemm_pair_kernel<K, N>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, stream_a, ep, c)
         if (kind == TC_GEMM_QKV) {
             if (s.pair_bn == 256) FD_LAUNCH_PAIR(EPI_QKV, 256); else FD_LAUNCH_PAIR(EPI_QKV, 192);
         } else if (kind == TC_GEMM_FC1) {
