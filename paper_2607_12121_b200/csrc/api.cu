@@ -293,6 +293,7 @@ fd_status fd_create(const fd_config* cfg, const fd_weights* weights, void* works
         TcBuffers tb{};
         tb.act = c->ws + lay.act; tb.q = c->ws + lay.q; tb.o = c->ws + lay.o; tb.g = c->ws + lay.g;
         tb.Mcap = lay.Mcap; tb.q_ld = lay.q_ld;
+        tb.resid = c->ws + lay.resid;
         std::string tc_err;
         c->tc = tc_plan_create(*cfg, *weights, tb, &tc_err);
         if (!c->tc) {

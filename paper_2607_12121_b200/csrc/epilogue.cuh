@@ -6,6 +6,7 @@
 //             the row into y,
 //   EPI_GELU  bias and tanh-GELU.
 #pragma once
+#include <cuda.h>
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -171,6 +172,47 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
     __syncwarp();
 }
 
+// EPI_RESID through the TMA: the warp's 32 x 32 products gate * (acc + bias) go back into its staging tile as
+// plain fp32 rows and one bulk tensor reduction adds the tile onto the residual stream.  The SM's load/store path
+// issues per-thread reductions at about 9 bytes per clock, which made this epilogue as long as the main loop of a
+// K = 1536 tile; the bulk form hands whole 128-byte rows to the L2.
+__device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
+                                                         int n_rows, int col0, const uint32_t* acc, const RowInfo& ri,
+                                                         const CUtensorMap* tm_r) {
+    using T = __nv_bfloat16;
+    if (lane == 0) ptx::bulk_wait_read_all();                      // the previous chunk's reduction has read the tile
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) *unit_ptr(stage, lane, k) = make_uint4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
+    __syncwarp();
+    const int u = lane & 7, rsub = lane >> 3;
+    const int col = col0 + u * 4;
+    float bias[4];
+    load4<T>(reinterpret_cast<const T*>(ep.bias) + col, bias);
+    const float* gp = ep.gate + col;
+    float4 gv[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int go = __shfl_sync(0xffffffffu, ri.gate_off, 4 * i + rsub);
+        gv[i] = 4 * i + rsub < n_rows ? __ldg(reinterpret_cast<const float4*>(gp + go)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    // The tile is rewritten in place, row by row: the eight lanes of a row read their (swizzled) units, then write the
+    // row's 128 bytes in plain order; rows past the last active row add zeros.
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + rsub;
+        const uint4 a = *unit_ptr(stage, r, u);
+        __syncwarp();
+        float4 v;
+        v.x = gv[i].x * (__uint_as_float(a.x) + bias[0]); v.y = gv[i].y * (__uint_as_float(a.y) + bias[1]);
+        v.z = gv[i].z * (__uint_as_float(a.z) + bias[2]); v.w = gv[i].w * (__uint_as_float(a.w) + bias[3]);
+        *reinterpret_cast<float4*>(stage + r * 128 + u * 16) = v;
+    }
+    ptx::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) ptx::tma_reduce_add_2d(tm_r, col0, row_base, stage);
+}
+
 // EPI_QKV / EPI_GELU: 64 fp32 accumulator columns per row, bf16 outputs (8 columns per 16-byte unit).
 template <int KIND>
 __device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
@@ -247,7 +289,8 @@ __device__ __forceinline__ void epilogue_prefetch_resid(const EpiParams& ep, int
 // one warp's share of a tile: rows [row_base, row_base + 32), columns [c_begin, c_end) of the accumulator at t_row
 template <int KIND>
 __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stage, int lane, int row_base, int a_total,
-                                              uint32_t t_row, int tile_col0, int c_begin, int c_end) {
+                                              uint32_t t_row, int tile_col0, int c_begin, int c_end,
+                                              const CUtensorMap* tm_r = nullptr) {
     const bool live = row_base < a_total;                        // warp-uniform
     const int n_rows = a_total - row_base;
     RowInfo ri{0, 0u, 0u};
@@ -265,7 +308,10 @@ __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stag
             uint32_t r[32];
             ptx::tmem_ld32(t_row + c0, r);
             ptx::tmem_wait_ld();
-            if (live) epilogue_resid_chunk(ep, stage, lane, row_base, n_rows, tile_col0 + c0, r, ri);
+            if (live) {
+                if (tm_r && !ep.y) epilogue_resid_chunk_tma(ep, stage, lane, row_base, n_rows, tile_col0 + c0, r, ri, tm_r);
+                else epilogue_resid_chunk(ep, stage, lane, row_base, n_rows, tile_col0 + c0, r, ri);
+            }
         }
     } else {
 #pragma unroll 1

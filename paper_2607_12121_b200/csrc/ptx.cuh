@@ -118,6 +118,18 @@ __device__ __forceinline__ void bulk_load(void* sdst, const void* gsrc, uint32_t
                  ::"r"(smem_u32(sdst)), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
+// Bulk tensor reduction shared -> global: adds a [box] tile of fp32 values in shared memory (written by this CTA,
+// made visible with fence_proxy_async_smem) onto the tensor at (x, y); rows or columns outside the tensor are
+// dropped.  The issuing thread closes one bulk group per call.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* m, int x, int y, const void* ssrc) {
+    asm volatile(
+        "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];\n\t"
+        "cp.async.bulk.commit_group;"
+        ::"l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(smem_u32(ssrc))
+        : "memory");
+}
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* m, int x, int y, int z, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"

@@ -12,6 +12,7 @@ struct TcPlan;      // TMA descriptors of weights and workspace tensors, built o
 
 struct TcBuffers {  // compact activation buffers inside the workspace (bf16)
     void *act, *q, *o, *g;
+    void* resid;    // fp32 residual stream [Mcap, hidden]
     int Mcap, q_ld;
 };
 

@@ -173,8 +173,9 @@ template <int PAIR_BN> struct PairCfg {
 
 template <int KIND, int PAIR_BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
-tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int n_out,
-                    int k_dim, int stream_a, EpiParams ep, Control* ctl) {
+tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                    const __grid_constant__ CUtensorMap tm_r, int n_out, int k_dim, int stream_a, int tma_resid, EpiParams ep,
+                    Control* ctl) {
     constexpr int PAIR_B_BYTES = PairCfg<PAIR_BN>::B_BYTES, PAIR_STAGE_BYTES = PairCfg<PAIR_BN>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -286,11 +287,13 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
             epilogue_warp<KIND>(ep, epi_stage + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane,
-                                m * 2 * BM + (int)rank * BM + quad * 32, a_total, t_row, n * PAIR_BN, c_lo, c_hi);
+                                m * 2 * BM + (int)rank * BM + quad * 32, a_total, t_row, n * PAIR_BN, c_lo, c_hi,
+                                (KIND == EPI_RESID && tma_resid) ? &tm_r : nullptr);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty[acc]), 0));
         }
+        if (KIND == EPI_RESID && lane == 0) bulk_wait_all();      // this thread's bulk reductions have landed
         if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 900 + (int)blockIdx.x);
     }
 
@@ -340,8 +343,8 @@ int pick_pair_bn(int n_out) { return n_out % 256 == 0 ? 256 : (n_out % 192 == 0 
 
 }  // namespace
 
-bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                      const uint32_t* box, int swizzle_bytes, std::string* err) {
+static bool encode_tmap(CUtensorMap* out, CUtensorMapDataType dtype, void* base, int rank, const uint64_t* dims,
+                        const uint64_t* strides_bytes, const uint32_t* box, int swizzle_bytes, std::string* err) {
     EncodeTiledFn fn = encode_fn(err);
     if (!fn) return false;
     cuuint64_t gd[5], gs[5];
@@ -352,7 +355,7 @@ bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* di
                           : swizzle_bytes == 64  ? CU_TENSOR_MAP_SWIZZLE_64B
                           : swizzle_bytes == 32  ? CU_TENSOR_MAP_SWIZZLE_32B
                                                  : CU_TENSOR_MAP_SWIZZLE_NONE;
-    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, gd, gs, bx, es,
+    CUresult r = fn(out, dtype, (cuuint32_t)rank, base, gd, gs, bx, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -360,6 +363,11 @@ bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* di
         return false;
     }
     return true;
+}
+
+bool encode_tmap_bf16(CUtensorMap* out, void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                      const uint32_t* box, int swizzle_bytes, std::string* err) {
+    return encode_tmap(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, base, rank, dims, strides_bytes, box, swizzle_bytes, err);
 }
 
 struct GemmSpec {
@@ -375,6 +383,8 @@ struct TcPlan {
     bool pdl;                   // launch the tensor-core kernels with programmatic stream serialization
     int pair_ctas;              // grid of the CTA-pair kernel: 2 x co-resident clusters
     GemmSpec spec[4];
+    CUtensorMap resid_map;      // fp32 residual stream [Mcap, H], 32 x 32 boxes for the bulk reductions of EPI_RESID
+    bool tma_resid;
     CUtensorMap* w_maps;        // [L][4]
     // attention (filled by the attention part)
     void* attn;
@@ -432,6 +442,14 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
             void* base = const_cast<char*>(w_base[g]) + (size_t)l * n_out[g] * kdim[g] * 2;
             ok = encode_tmap_bf16(&p->w_maps[(size_t)l * 4 + g], base, 2, wd, strides, wb, 128, err);
         }
+    }
+    p->tma_resid = true;        // switch: FD_TMA_RESID=0 keeps the per-thread vector reductions
+    if (const char* v = getenv("FD_TMA_RESID")) p->tma_resid = atoi(v) != 0;
+    if (ok) {
+        const uint64_t rd[2] = {(uint64_t)H, (uint64_t)buf.Mcap};
+        const uint64_t rs[1] = {(uint64_t)H * 4};
+        const uint32_t rb[2] = {32, 32};
+        ok = encode_tmap(&p->resid_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, buf.resid, 2, rd, rs, rb, 0, err);
     }
     if (ok) {
         cudaError_t e = cudaSuccess;
@@ -512,7 +530,8 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
         const int stream_a = kind == TC_GEMM_FC2 ? 1 : 0;
         cudaError_t e = cudaSuccess;
 #define FD_LAUNCH_PAIR(K, N) \
-    e = launch_kernel(tc_gemm_pair_kernel<K, N>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, stream_a, ep, c)
+    e = launch_kernel(tc_gemm_pair_kernel<K, N>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, s.a, wm, p->resid_map, s.n_out, s.k, \
+                      stream_a, p->tma_resid ? 1 : 0, ep, c)
         if (kind == TC_GEMM_QKV) {
             if (s.pair_bn == 256) FD_LAUNCH_PAIR(EPI_QKV, 256); else FD_LAUNCH_PAIR(EPI_QKV, 192);
         } else if (kind == TC_GEMM_FC1) {
