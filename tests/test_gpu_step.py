@@ -152,6 +152,16 @@ def test_tensor_core_engine_few_ctas_walk_many_tiles(monkeypatch, name, n_tok):
     _run_sequence(wl, 3, fd.FD_ENGINE_TC, masks)
 
 
+@pytest.mark.parametrize("switch", ["FD_TMA_RESID", "FD_TC_PAIR", "FD_PDL"])
+def test_tensor_core_engine_switched_off_variants(monkeypatch, switch):
+    """The library's switches select older forms of a kernel (per-thread residual reductions instead of the bulk
+    tensor reduction, single-CTA instead of CTA-pair GEMM tiles, fully serialized launches); they stay correct."""
+    monkeypatch.setenv(switch, "0")
+    wl = gen.workload("mmdit_tc")
+    masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 8, [0.5] * wl.B)]
+    _run_sequence(wl, 6, fd.FD_ENGINE_TC, masks)
+
+
 @pytest.mark.parametrize("name,engine", [("audio_tc", fd.FD_ENGINE_TC), ("video_tc", fd.FD_ENGINE_TC),
                                          ("audio_tc", fd.FD_ENGINE_SIMT)])
 def test_peaked_attention_exercises_running_max(name, engine):
