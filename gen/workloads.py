@@ -138,6 +138,20 @@ def block_weights(wl: Workload, seed: int, n_blocks: Optional[int] = None,
     return out
 
 
+def sampler_weights(wl: Workload, seed: int) -> Dict[str, np.ndarray]:
+    """Patch embedding (D -> H, bias, positional table) and final layer (H -> D, bias), rounded to the
+    storage type: w_in [H,D], b_in [H], pos [N,H], w_out [D,H], b_out [D]."""
+    g = _rng(seed, 909)
+    H, D, N = wl.H, wl.D, wl.N
+    return {
+        "w_in": _store(wl, g.standard_normal((H, D), dtype=np.float32) / np.float32(np.sqrt(D))),
+        "b_in": _store(wl, g.standard_normal((H,), dtype=np.float32) * np.float32(0.1)),
+        "pos": _store(wl, g.standard_normal((N, H), dtype=np.float32) * np.float32(0.5)),
+        "w_out": _store(wl, g.standard_normal((D, H), dtype=np.float32) / np.float32(np.sqrt(H))),
+        "b_out": _store(wl, g.standard_normal((D,), dtype=np.float32) * np.float32(0.1)),
+    }
+
+
 def uniform_labels(wl: Workload) -> np.ndarray:
     """Caller-written partitions: 2-D square blocks or contiguous 1-D segments. int32 [B,N]."""
     if wl.labels == "blocks2d":

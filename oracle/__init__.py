@@ -13,6 +13,8 @@ change, and the 16-bit width of the saliency quantisation.
 * ``regional_step``  -- all blocks on active tokens with stale K/V for skipped patches
                         (Sec. 3, Sec. 5, Appendix A.6)
 * ``dense_step``     -- the ungated baseline trajectory, written separately
+* ``sampler_embed``, ``sampler_update`` -- patch embedding and the latent update with cached drift
+                        (Appendix A.1, Eq. sf-update)
 """
 from __future__ import annotations
 
@@ -23,6 +25,7 @@ import numpy as np
 
 from .build import build as _build
 from .gate import activity_gate, compact, initial_state  # noqa: F401
+from .sampler import embed as sampler_embed, update as sampler_update, token_drift  # noqa: F401
 from .partitioner import partition, partition_request, saliency, quantise, allocate, best_cut  # noqa: F401
 
 _lib = None
