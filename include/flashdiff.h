@@ -155,6 +155,42 @@ fd_status fd_regional_step(fd_ctx* ctx, const void* x, const void* cond, const i
                            int32_t* active_idx_out, int32_t* cu_active_out, void* cuda_stream);
 
 /*
+ * Sampler closure around the step: patch embedding before it, final layer and latent update after it
+ * (Appendix A.1, Eq. sf-update: an active patch moves along its fresh drift, a skipped patch along
+ * the drift cached at its most recent active step).  With these two calls a gated multi-step loop
+ *     x = embed(z);  mask = gate(z, z_prev);  y = step(x, mask);  z_next = update(z, y)
+ * runs entirely on the device.  Both maps are per token, so a "patch" is the set of tokens with its label.
+ *
+ * Weights (host struct of DEVICE pointers, element type fd_config.dtype, 16-byte aligned, borrowed for
+ * the duration of the call):
+ *   w_in [H,D], b_in [H], pos [N,H]   patch embedding  x[b,j,:] = z[b,j,:] w_in^T + b_in + pos[j,:]
+ *   w_out [D,H], b_out [D]            final layer      drift = LayerNorm(y row, no affine, fd_config.ln_eps) w_out^T + b_out
+ * D = latent_dim: a multiple of 4, at most 256.
+ */
+typedef struct {
+    const void *w_in, *b_in, *pos;
+    const void *w_out, *b_out;
+    int32_t latent_dim;
+} fd_sampler_weights;
+
+/*   z [B,N,D] f32  ->  x_out [B,N,H] of fd_config.dtype (all tokens; the step reads the active ones).  */
+fd_status fd_embed_latent(fd_ctx* ctx, const fd_sampler_weights* sw, const float* z, int B, int N, void* x_out,
+                          void* cuda_stream);
+
+/*
+ * One application of Eq. sf-update after fd_regional_step:
+ *   for every active token (active_idx / cu_active as the step wrote them): drift[b,j,:] = final layer of y[b,j,:];
+ *   for every token: z_next[b,j,:] = z[b,j,:] + h[b] * drift[b,j,:]   (the cached drift where the token was skipped).
+ *   z, z_next, drift_cache [B,N,D] f32 (z_next may be z); y [B,N,H] of fd_config.dtype; h [B] f32;
+ *   active_idx [>= A] i32, cu_active [B+1] i32 (DEVICE; A = cu_active[B] is read on the device).
+ * drift_cache is in/out state: rows of active tokens are overwritten, the others are only read, so the first
+ * call must follow an all-active step.
+ */
+fd_status fd_update_latent(fd_ctx* ctx, const fd_sampler_weights* sw, const float* z, const void* y,
+                           const int32_t* active_idx, const int32_t* cu_active, const float* h, int B, int N,
+                           float* drift_cache, float* z_next, void* cuda_stream);
+
+/*
  * The gate for callers that cannot allocate device memory (no counterpart in the paper; added for
  * embedding).  Some hosts of this library may not call cudaMalloc at all: a plug-in running inside
  * an inference server whose memory pool was sized and frozen at start-up, code on a latency-critical
@@ -218,7 +254,8 @@ enum {
     FD_PROF_GEMM_FC1 = 7,
     FD_PROF_GEMM_FC2 = 8,
     FD_PROF_PARTITION = 9,
-    FD_PROF_GROUPS = 10
+    FD_PROF_SAMPLER = 10, /* patch embedding, final layer, latent update */
+    FD_PROF_GROUPS = 11
 };
 fd_status fd_profile_enable(fd_ctx* ctx, int enable);
 fd_status fd_profile_read(fd_ctx* ctx, void* cuda_stream, float* ms_out, int32_t* kernels_out);

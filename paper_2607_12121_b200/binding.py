@@ -21,10 +21,11 @@ FD_ENGINE_AUTO, FD_ENGINE_SIMT, FD_ENGINE_TC = 0, 1, 2
 
 EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region_activity",
            "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
-           "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait"]
+           "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait",
+           "fd_embed_latent", "fd_update_latent"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
-               "gemm_fc2", "partition"]
+               "gemm_fc2", "partition", "sampler"]
 
 
 class FdConfig(ctypes.Structure):
@@ -37,6 +38,10 @@ class FdConfig(ctypes.Structure):
 class FdWeights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
                 ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2", "w_ada", "b_ada")]
+
+
+class FdSamplerWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("w_in", "b_in", "pos", "w_out", "b_out")] + [("latent_dim", ctypes.c_int32)]
 
 
 class FlashDiffError(RuntimeError):
@@ -72,6 +77,10 @@ def _load() -> ctypes.CDLL:
     lib.fd_profile_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     lib.fd_selftest_bounded_wait.restype = i32
     lib.fd_selftest_bounded_wait.argtypes = [vp, vp]
+    lib.fd_embed_latent.restype = i32
+    lib.fd_embed_latent.argtypes = [vp, ctypes.POINTER(FdSamplerWeights), vp, i32, i32, vp, vp]
+    lib.fd_update_latent.restype = i32
+    lib.fd_update_latent.argtypes = [vp, ctypes.POINTER(FdSamplerWeights), vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     lib.fd_launch_count.restype = ctypes.c_int64
     lib.fd_launch_count.argtypes = [vp]
     lib.fd_destroy.restype = i32
@@ -186,6 +195,28 @@ def fd_regional_step(ctx: Context, x, cond, labels, mask, R: int, kv_cache, y, a
     _check(ctx.handle, lib.fd_regional_step(
         ctx.handle, _ptr(x), _ptr(cond), _ptr(labels), _ptr(mask), B, N, R, _ptr(kv_cache), _ptr(y),
         _ptr(active_idx_out), _ptr(cu_active_out), _stream(stream)))
+
+
+def make_sampler_weights(tensors: dict, latent_dim: int) -> FdSamplerWeights:
+    """fd_sampler_weights from device tensors w_in [H,D], b_in [H], pos [N,H], w_out [D,H], b_out [D]
+    (keep the tensors alive while the struct is in use)."""
+    return FdSamplerWeights(*[_ptr(tensors[k]) for k in ("w_in", "b_in", "pos", "w_out", "b_out")], int(latent_dim))
+
+
+def fd_embed_latent(ctx: Context, sw: FdSamplerWeights, z, x_out, stream=None) -> None:
+    """x_out[b,j,:] = z[b,j,:] w_in^T + b_in + pos[j,:]  (z [B,N,D] f32)."""
+    B, N, _ = z.shape
+    _check(ctx.handle, lib.fd_embed_latent(ctx.handle, ctypes.byref(sw), _ptr(z), B, N, _ptr(x_out), _stream(stream)))
+
+
+def fd_update_latent(ctx: Context, sw: FdSamplerWeights, z, y, active_idx, cu_active, h, drift_cache, z_next,
+                     stream=None) -> None:
+    """Final layer on the active tokens' rows of y (refreshing drift_cache there), then
+    z_next = z + h[b] * drift_cache for every token."""
+    B, N, _ = z.shape
+    _check(ctx.handle, lib.fd_update_latent(ctx.handle, ctypes.byref(sw), _ptr(z), _ptr(y), _ptr(active_idx),
+                                            _ptr(cu_active), _ptr(h), B, N, _ptr(drift_cache), _ptr(z_next),
+                                            _stream(stream)))
 
 
 def fd_poll_status(ctx: Context, stream=None) -> None:

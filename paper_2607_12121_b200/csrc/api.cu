@@ -362,6 +362,74 @@ fd_status fd_region_activity(fd_ctx* c, const float* z_cur, const float* z_prev,
     return FD_OK;
 }
 
+namespace {
+fd_status sampler_args_ok(fd_ctx* c, const fd_sampler_weights* sw, int B, int N) {
+    if (!sw) return c->fail(FD_ERR_INVALID_ARG, "null sampler weights");
+    if (!sw->w_in || !sw->b_in || !sw->pos || !sw->w_out || !sw->b_out) return c->fail(FD_ERR_INVALID_ARG, "null sampler weight pointer");
+    if (!aligned16(sw->w_in) || !aligned16(sw->b_in) || !aligned16(sw->pos) || !aligned16(sw->w_out) || !aligned16(sw->b_out))
+        return c->fail(FD_ERR_INVALID_ARG, "sampler weights must be 16-byte aligned");
+    if (sw->latent_dim < 4 || sw->latent_dim % 4 || sw->latent_dim > 256)
+        return c->fail(FD_ERR_SHAPE, "latent_dim must be a multiple of 4 in [4, 256]");
+    if (B < 1 || N < 1) return c->fail(FD_ERR_SHAPE, "B and N must be positive");
+    if (B > c->cfg.max_batch || N > c->cfg.max_tokens)
+        return c->fail(FD_ERR_SHAPE, "B=%d N=%d exceed the limits %d/%d", B, N, c->cfg.max_batch, c->cfg.max_tokens);
+    return FD_OK;
+}
+}  // namespace
+
+fd_status fd_embed_latent(fd_ctx* c, const fd_sampler_weights* sw, const float* z, int B, int N, void* x_out,
+                          void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!z || !x_out) return c->fail(FD_ERR_INVALID_ARG, "null pointer argument");
+    if (!aligned16(z) || !aligned16(x_out)) return c->fail(FD_ERR_INVALID_ARG, "z and x_out must be 16-byte aligned");
+    fd_status s = sampler_args_ok(c, sw, B, N);
+    if (s != FD_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int nl = 0;
+    c->span_begin(FD_PROF_SAMPLER, st);
+    cudaError_t e;
+    if (c->cfg.dtype == FD_BF16)
+        e = launch_embed<__nv_bfloat16>(z, static_cast<const __nv_bfloat16*>(sw->w_in), static_cast<const __nv_bfloat16*>(sw->b_in),
+                                        static_cast<const __nv_bfloat16*>(sw->pos), static_cast<__nv_bfloat16*>(x_out), B, N,
+                                        sw->latent_dim, c->cfg.hidden, st, &nl);
+    else
+        e = launch_embed<float>(z, static_cast<const float*>(sw->w_in), static_cast<const float*>(sw->b_in),
+                                static_cast<const float*>(sw->pos), static_cast<float*>(x_out), B, N, sw->latent_dim,
+                                c->cfg.hidden, st, &nl);
+    c->span_end(nl, st);
+    c->launches += nl;
+    if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "embed launch failed: %s", cudaGetErrorString(e));
+    return FD_OK;
+}
+
+fd_status fd_update_latent(fd_ctx* c, const fd_sampler_weights* sw, const float* z, const void* y,
+                           const int32_t* active_idx, const int32_t* cu_active, const float* h, int B, int N,
+                           float* drift_cache, float* z_next, void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!z || !y || !active_idx || !cu_active || !h || !drift_cache || !z_next)
+        return c->fail(FD_ERR_INVALID_ARG, "null pointer argument");
+    if (!aligned16(z) || !aligned16(y) || !aligned16(drift_cache) || !aligned16(z_next))
+        return c->fail(FD_ERR_INVALID_ARG, "z, y, drift_cache and z_next must be 16-byte aligned");
+    fd_status s = sampler_args_ok(c, sw, B, N);
+    if (s != FD_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int nl = 0;
+    c->span_begin(FD_PROF_SAMPLER, st);
+    cudaError_t e;
+    if (c->cfg.dtype == FD_BF16)
+        e = launch_update<__nv_bfloat16>(z, static_cast<const __nv_bfloat16*>(y), active_idx, cu_active, h,
+                                         static_cast<const __nv_bfloat16*>(sw->w_out), static_cast<const __nv_bfloat16*>(sw->b_out),
+                                         drift_cache, z_next, B, N, sw->latent_dim, c->cfg.hidden, c->cfg.ln_eps, st, &nl);
+    else
+        e = launch_update<float>(z, static_cast<const float*>(y), active_idx, cu_active, h, static_cast<const float*>(sw->w_out),
+                                 static_cast<const float*>(sw->b_out), drift_cache, z_next, B, N, sw->latent_dim, c->cfg.hidden,
+                                 c->cfg.ln_eps, st, &nl);
+    c->span_end(nl, st);
+    c->launches += nl;
+    if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "latent update launch failed: %s", cudaGetErrorString(e));
+    return FD_OK;
+}
+
 fd_status fd_region_activity_noalloc(const float* z_cur, const float* z_prev, const int32_t* labels, int B, int N,
                                      int D, int R, const float* eps, float eta, int max_skip_k, float* delta_state,
                                      int32_t* skip_count, uint8_t* prev_active, float* score_out, float* weight_out,

@@ -127,6 +127,15 @@ cudaError_t launch_simt_attention(const T* q, int q_ld, const T* kv, T* o, int o
                                   int max_tiles, int N, int H, int heads, int dh, const Control* ctl,
                                   cudaStream_t st, int* n_launch);
 
+// sampler.cu
+template <typename T>
+cudaError_t launch_embed(const float* z, const T* w_in, const T* b_in, const T* pos, T* x, int B, int N, int D, int H,
+                         cudaStream_t st, int* n_launch);
+template <typename T>
+cudaError_t launch_update(const float* z, const T* y, const int32_t* active_idx, const int32_t* cu_active, const float* h,
+                          const T* w_out, const T* b_out, float* drift, float* z_next, int B, int N, int D, int H,
+                          float ln_eps, cudaStream_t st, int* n_launch);
+
 // partition.cu
 size_t partition_scratch_bytes(int max_batch, int max_tokens, int max_regions);
 cudaError_t launch_partition(const float* attn_map, int B, int N, int T, const int32_t* salient_cols,
