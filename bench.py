@@ -403,6 +403,37 @@ def run_ours(args):
     d2h = h_y.numel() * h_y.element_size()
     fd.fd_poll_status(ctx)
 
+    # sampler closure around the step (outside the timed step, which is the hot path alone): patch embedding of all
+    # tokens, final layer on the active rows, latent update; timed with CUDA events on the same shapes
+    sw_np = gen.sampler_weights(wl, seed)
+    sw_dev = {k: torch.from_numpy(v).to(dev).to(dt) for k, v in sw_np.items()}
+    sw = fd.make_sampler_weights(sw_dev, D)
+    s_drift = torch.zeros((B, N, D), dtype=torch.float32, device=dev)
+    s_zn = torch.empty((B, N, D), dtype=torch.float32, device=dev)
+    s_x = torch.empty((B, N, H), dtype=dt, device=dev)
+    s_h = torch.full((B,), 0.02, dtype=torch.float32, device=dev)
+
+    def time_us(fn, reps=10):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e3
+
+    emb_us = time_us(lambda: fd.fd_embed_latent(ctx, sw, z_cur, s_x))
+    upd_us = time_us(lambda: fd.fd_update_latent(ctx, sw, z_cur, y, active_idx, cu_active, s_h, s_drift, s_zn))
+    es = 2 if dt == torch.bfloat16 else 4
+    emb_bytes = B * N * (D * 4 + H * es) + N * H * es
+    upd_bytes = A * (H * es + D * 4) + 3 * B * N * D * 4
+    sampler = {"embed_us": emb_us, "embed_gbs": emb_bytes / emb_us / 1e3, "update_us": upd_us,
+               "update_gbs": upd_bytes / upd_us / 1e3, "note": "outside the timed step; algorithmic bytes / CUDA-event time"}
+    fd.fd_poll_status(ctx)
+
     # streaming rate of the activity reduction on a batch large enough to be bandwidth bound (at the
     # benchmark shapes the gate moves a few MB and is launch-latency bound): 256 requests x 8192 tokens x 64
     # channels, all regions fresh, through the allocation-free entry point
@@ -502,6 +533,7 @@ def run_ours(args):
         "kernel_breakdown": breakdown,
         "activity_probe": None if probe is None else dict(probe, frac_of_hbm=probe["gbs"] / float(peaks["hbm_gbs"]),
                                                          workload="256 requests x 8192 tokens x 64 channels, 64 regions"),
+        "sampler": sampler,
         "peaks": {"source": peak_kind, "bf16_tflops": peaks.get("bf16_tflops"),
                   "bf16_tflops_sustained": peaks.get("bf16_tflops_sustained"), "hbm_gbs": peaks.get("hbm_gbs")},
     }
