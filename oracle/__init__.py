@@ -24,7 +24,7 @@ from typing import Dict, Optional
 import numpy as np
 
 from .build import build as _build
-from .gate import activity_gate, compact, initial_state  # noqa: F401
+from .gate import activity_gate, attention_gate, attention_mass, compact, initial_state  # noqa: F401
 from .sampler import embed as sampler_embed, update as sampler_update, token_drift  # noqa: F401
 from .partitioner import partition, partition_request, saliency, quantise, allocate, best_cut  # noqa: F401
 
@@ -107,6 +107,27 @@ def regional_step(x: np.ndarray, cond: np.ndarray, labels: np.ndarray, mask: np.
         u = regional_block(u, active_idx, mod, w, l, kv[l], heads, ln_eps)
     y.reshape(B * N, H)[active_idx] = u
     return active_idx, cu_active
+
+
+def block0_projection(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], active_idx: np.ndarray,
+                      part: int = 0, ln_eps: float = 1e-6) -> np.ndarray:
+    """Rows of the first block's Q (part 0), K (1) or V (2) for the active tokens, [A,H] fp32: LayerNorm +
+    adaLN modulation of the gathered rows, then that third of the QKV projection.  The queries, together with the
+    block's key cache after the step, are what ``attention_mass`` needs."""
+    B, N, H = x.shape
+    mod = adaln(cond, w["w_ada"][0], w["b_ada"][0]).astype(np.float64)
+    u = x.reshape(B * N, H)[active_idx].astype(np.float64)
+    mean = u.mean(-1, keepdims=True)
+    var = ((u - mean) ** 2).mean(-1, keepdims=True)
+    b = np.asarray(active_idx, np.int64) // N
+    un = (u - mean) / np.sqrt(var + ln_eps) * (1.0 + mod[b, H:2 * H]) + mod[b, 0:H]        # scale_msa, shift_msa
+    rows = slice(part * H, (part + 1) * H)
+    out = un @ w["w_qkv"][0][rows].astype(np.float64).T + w["b_qkv"][0][rows].astype(np.float64)
+    return out.astype(np.float32)
+
+
+def block0_queries(x, cond, w, active_idx, ln_eps: float = 1e-6) -> np.ndarray:
+    return block0_projection(x, cond, w, active_idx, 0, ln_eps)
 
 
 def dense_block(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], l: int, heads: int,
