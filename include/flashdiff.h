@@ -155,6 +155,34 @@ fd_status fd_regional_step(fd_ctx* ctx, const void* x, const void* cond, const i
                            int32_t* active_idx_out, int32_t* cu_active_out, void* cuda_stream);
 
 /*
+ * The Patch Gate on the paper's own signal (Sec. 4.2): the refinement importance of a patch is the block mean of
+ * the self-attention matrix over the patch,  R_i = (1/|A_i|^2) sum_{u,v in A_i} SA[u,v],  and the gate weights are
+ * the normalised changes  Delta_i = |R_i - Rbar_i|  (Rbar_i = the importance at the patch's last executed step;
+ * a skipped patch keeps its Delta_i).  SA is taken from the FIRST block of the step, softmax probabilities averaged
+ * over heads.
+ *
+ * fd_regional_step_mass is fd_regional_step that additionally writes
+ *   region_mass_out [B,R] f64 (DEVICE):  sum over the ACTIVE queries u of region i and over the keys v of region i
+ *   of SA[u,v] (zero for regions that did not run; tokens with label R belong to no region).
+ * The tensor-core engine computes the mass in a second, CUDA-core pass over the first block's scores.
+ *
+ * fd_region_activity_attn turns it into the next step's mask: for every region executed at the step that produced
+ * region_mass (prev_active = 1),  R_i = region_mass / region_sizes^2,  Delta_i = |R_i - Rbar_i|,  Rbar_i <- R_i;
+ * weights, threshold, forced reactivation and the skip_count / prev_active updates are those of fd_region_activity.
+ *   region_sizes [B,R] i32 (tokens per region, as fd_partition_regions returns them)
+ *   state in/out: rbar_state, delta_state [B,R] f32 (start at zero), skip_count [B,R] i32, prev_active [B,R] u8
+ *   outputs [B,R]: importance_out f32 (Rbar after the update), weight_out f32, mask_out u8
+ */
+fd_status fd_regional_step_mass(fd_ctx* ctx, const void* x, const void* cond, const int32_t* labels,
+                                const uint8_t* mask, int B, int N, int R, void* kv_cache, void* y,
+                                int32_t* active_idx_out, int32_t* cu_active_out, double* region_mass_out,
+                                void* cuda_stream);
+fd_status fd_region_activity_attn(fd_ctx* ctx, const double* region_mass, const int32_t* region_sizes, int B, int R,
+                                  const float* eps, float* rbar_state, float* delta_state, int32_t* skip_count,
+                                  uint8_t* prev_active, float* importance_out, float* weight_out, uint8_t* mask_out,
+                                  void* cuda_stream);
+
+/*
  * Sampler closure around the step: patch embedding before it, final layer and latent update after it
  * (Appendix A.1, Eq. sf-update: an active patch moves along its fresh drift, a skipped patch along
  * the drift cached at its most recent active step).  With these two calls a gated multi-step loop

@@ -22,7 +22,7 @@ FD_ENGINE_AUTO, FD_ENGINE_SIMT, FD_ENGINE_TC = 0, 1, 2
 EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region_activity",
            "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
            "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait",
-           "fd_embed_latent", "fd_update_latent"]
+           "fd_embed_latent", "fd_update_latent", "fd_regional_step_mass", "fd_region_activity_attn"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
                "gemm_fc2", "partition", "sampler"]
@@ -77,6 +77,10 @@ def _load() -> ctypes.CDLL:
     lib.fd_profile_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     lib.fd_selftest_bounded_wait.restype = i32
     lib.fd_selftest_bounded_wait.argtypes = [vp, vp]
+    lib.fd_regional_step_mass.restype = i32
+    lib.fd_regional_step_mass.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.fd_region_activity_attn.restype = i32
+    lib.fd_region_activity_attn.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.fd_embed_latent.restype = i32
     lib.fd_embed_latent.argtypes = [vp, ctypes.POINTER(FdSamplerWeights), vp, i32, i32, vp, vp]
     lib.fd_update_latent.restype = i32
@@ -217,6 +221,24 @@ def fd_update_latent(ctx: Context, sw: FdSamplerWeights, z, y, active_idx, cu_ac
     _check(ctx.handle, lib.fd_update_latent(ctx.handle, ctypes.byref(sw), _ptr(z), _ptr(y), _ptr(active_idx),
                                             _ptr(cu_active), _ptr(h), B, N, _ptr(drift_cache), _ptr(z_next),
                                             _stream(stream)))
+
+
+def fd_regional_step_mass(ctx: Context, x, cond, labels, mask, R: int, kv_cache, y, active_idx_out, cu_active_out,
+                          region_mass_out, stream=None) -> None:
+    """fd_regional_step that also writes region_mass_out [B,R] f64: the first block's own-region attention mass."""
+    B, N, _ = x.shape
+    _check(ctx.handle, lib.fd_regional_step_mass(
+        ctx.handle, _ptr(x), _ptr(cond), _ptr(labels), _ptr(mask), B, N, R, _ptr(kv_cache), _ptr(y),
+        _ptr(active_idx_out), _ptr(cu_active_out), _ptr(region_mass_out), _stream(stream)))
+
+
+def fd_region_activity_attn(ctx: Context, region_mass, region_sizes, eps, rbar_state, delta_state, skip_count,
+                            prev_active, importance_out, weight_out, mask_out, stream=None) -> None:
+    """The gate on the attention-mass signal: Delta_i = |R_i - Rbar_i| with R_i = mass_i / size_i^2."""
+    B, R = region_mass.shape
+    _check(ctx.handle, lib.fd_region_activity_attn(
+        ctx.handle, _ptr(region_mass), _ptr(region_sizes), B, R, _ptr(eps), _ptr(rbar_state), _ptr(delta_state),
+        _ptr(skip_count), _ptr(prev_active), _ptr(importance_out), _ptr(weight_out), _ptr(mask_out), _stream(stream)))
 
 
 def fd_poll_status(ctx: Context, stream=None) -> None:

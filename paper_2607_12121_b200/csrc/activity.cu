@@ -334,7 +334,61 @@ gate_kernel(int R, int D, const float* __restrict__ eps, float eta, int K, doubl
     }
 }
 
+// The same gate on the paper's own signal (Sec. 4.2): R_i = mass_i / |A_i|^2 for the patches executed at the step that
+// produced `mass`; Delta_i = |R_i - Rbar_i| and Rbar_i <- R_i for those, frozen Delta_i for the skipped ones.
+__global__ void __launch_bounds__(256)
+attn_gate_kernel(int R, const double* __restrict__ mass, const int32_t* __restrict__ region_sizes, const float* __restrict__ eps,
+                 float eta, int K, float* __restrict__ rbar, float* __restrict__ delta_state, int32_t* __restrict__ skip_count,
+                 uint8_t* __restrict__ prev_active, float* __restrict__ importance, float* __restrict__ weight,
+                 uint8_t* __restrict__ mask) {
+    __shared__ double s_red[256];
+    const int b = blockIdx.x;
+    const size_t o = (size_t)b * R;
+    double local = 0.0;
+    for (int i = threadIdx.x; i < R; i += blockDim.x) {
+        float d;
+        if (prev_active[o + i]) {
+            const double n = (double)region_sizes[o + i];
+            const float r = n > 0.0 ? (float)(mass[o + i] / (n * n)) : 0.f;
+            d = (float)fabs((double)r - (double)rbar[o + i]);
+            delta_state[o + i] = d;
+            rbar[o + i] = r;
+        } else {
+            d = delta_state[o + i];
+        }
+        importance[o + i] = rbar[o + i];
+        local += (double)d + (double)eta;
+    }
+    s_red[threadIdx.x] = local;
+    __syncthreads();
+    for (int s = blockDim.x >> 1; s > 0; s >>= 1) {
+        if (threadIdx.x < s) s_red[threadIdx.x] += s_red[threadIdx.x + s];
+        __syncthreads();
+    }
+    const double dn = s_red[0];
+    const double e = (double)eps[b];
+    for (int i = threadIdx.x; i < R; i += blockDim.x) {
+        const double num = (double)delta_state[o + i] + (double)eta;
+        const bool gate_on = dn > 0.0 ? (num >= e * dn) : true;      // w_i >= eps
+        weight[o + i] = dn > 0.0 ? (float)(num / dn) : 1.0f / (float)R;
+        const int sk = skip_count[o + i];
+        const bool on = gate_on || (sk >= K);                        // forced reactivation
+        mask[o + i] = on ? 1 : 0;
+        prev_active[o + i] = on ? 1 : 0;
+        skip_count[o + i] = on ? 0 : sk + 1;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_attn_gate(const double* region_mass, const int32_t* region_sizes, int B, int R, const float* eps,
+                             float eta, int K, float* rbar, float* delta, int32_t* skip_count, uint8_t* prev_active,
+                             float* importance, float* weight, uint8_t* mask, cudaStream_t st, int* n_launch) {
+    attn_gate_kernel<<<B, 256, 0, st>>>(R, region_mass, region_sizes, eps, eta, K, rbar, delta, skip_count, prev_active,
+                                        importance, weight, mask);
+    ++*n_launch;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_activity(const float* z_cur, const float* z_prev, const int32_t* labels, int B, int N,
                             int D, int R, const float* eps, float* delta, int32_t* skip_count,

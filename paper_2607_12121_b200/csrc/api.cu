@@ -131,7 +131,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 
 
 template <typename T>
 fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* labels, const uint8_t* mask, int B,
-                   int N, int R, void* kv_, void* y_, int32_t* active_idx, int32_t* cu_active, cudaStream_t st) {
+                   int N, int R, void* kv_, void* y_, int32_t* active_idx, int32_t* cu_active, cudaStream_t st,
+                   double* region_mass = nullptr) {
     const fd_config& cf = c->cfg;
     const Layout& l = c->lay;
     const int H = cf.hidden, M = cf.mlp_dim, L = cf.n_blocks, Hc = cf.cond_dim;
@@ -196,12 +197,24 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             FD_TRY(FD_PROF_GEMM_QKV, tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));
         else
             FD_TRY(FD_PROF_GEMM_QKV, launch_simt_gemm<T>(EPI_QKV, act, H, w_qkv, 3 * H, H, rows_cap, ep, ctl, st, &nl));
-        // active queries against all N keys of their request
-        if (c->use_tc_attn)
+        // active queries against all N keys of their request; the first block can also report, per region, the
+        // softmax mass its queries put on keys of their own region (paper Sec. 4.2)
+        double* mass = blk == 0 ? region_mass : nullptr;
+        if (mass) {
+            e = cudaMemsetAsync(mass, 0, (size_t)B * R * sizeof(double), st);
+            if (e != cudaSuccess) { c->launches += nl; return c->fail(FD_ERR_CUDA, "memset failed: %s", cudaGetErrorString(e)); }
+        }
+        if (c->use_tc_attn) {
             FD_TRY(FD_PROF_ATTENTION, tc_attention(c->tc, blk, kv_b, B, N, tiles, max_tiles, ctl, st, &nl));
-        else
+            if (mass)       // the tensor-core kernel has no mass output yet: a second pass on the CUDA cores, mass only
+                FD_TRY(FD_PROF_ATTENTION, launch_simt_attention<T>(q, l.q_ld, kv_b, static_cast<T*>(nullptr), H, tiles,
+                                                max_tiles, N, H, cf.n_heads, cf.head_dim, ctl, st, &nl,
+                                                tc_attention_head_pad(cf.head_dim), labels, active_idx, mass, R,
+                                                c->tile_rows / simt_attention_tile_rows()));
+        } else {
             FD_TRY(FD_PROF_ATTENTION, launch_simt_attention<T>(q, l.q_ld, kv_b, o, H, tiles, max_tiles, N, H, cf.n_heads, cf.head_dim,
-                                            ctl, st, &nl));
+                                            ctl, st, &nl, 0, labels, active_idx, mass, R));
+        }
         // out-projection, gated residual
         ep.bias = static_cast<const T*>(c->w.b_o) + (size_t)blk * H;
         ep.resid = resid;
@@ -452,10 +465,9 @@ fd_status fd_region_activity_noalloc(const float* z_cur, const float* z_prev, co
     return FD_OK;
 }
 
-fd_status fd_regional_step(fd_ctx* c, const void* x, const void* cond, const int32_t* labels, const uint8_t* mask,
-                           int B, int N, int R, void* kv_cache, void* y, int32_t* active_idx_out,
-                           int32_t* cu_active_out, void* cuda_stream) {
-    if (!c) return FD_ERR_INVALID_ARG;
+static fd_status fd_regional_step_check(fd_ctx* c, const void* x, const void* cond, const int32_t* labels, const uint8_t* mask,
+                                        int B, int N, int R, void* kv_cache, void* y, int32_t* active_idx_out,
+                                        int32_t* cu_active_out) {
     if (!x || !cond || !labels || !mask || !kv_cache || !y || !active_idx_out || !cu_active_out)
         return c->fail(FD_ERR_INVALID_ARG, "null pointer argument");
     if (!aligned16(x) || !aligned16(cond) || !aligned16(kv_cache) || !aligned16(y))
@@ -464,10 +476,55 @@ fd_status fd_regional_step(fd_ctx* c, const void* x, const void* cond, const int
     if (B > c->cfg.max_batch || N > c->cfg.max_tokens || R > c->cfg.max_regions)
         return c->fail(FD_ERR_SHAPE, "B=%d N=%d R=%d exceed the limits %d/%d/%d", B, N, R, c->cfg.max_batch,
                        c->cfg.max_tokens, c->cfg.max_regions);
+    return FD_OK;
+}
+
+fd_status fd_regional_step(fd_ctx* c, const void* x, const void* cond, const int32_t* labels, const uint8_t* mask,
+                           int B, int N, int R, void* kv_cache, void* y, int32_t* active_idx_out,
+                           int32_t* cu_active_out, void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    fd_status s = fd_regional_step_check(c, x, cond, labels, mask, B, N, R, kv_cache, y, active_idx_out, cu_active_out);
+    if (s != FD_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (c->cfg.dtype == FD_BF16)
         return run_step<__nv_bfloat16>(c, x, cond, labels, mask, B, N, R, kv_cache, y, active_idx_out, cu_active_out, st);
     return run_step<float>(c, x, cond, labels, mask, B, N, R, kv_cache, y, active_idx_out, cu_active_out, st);
+}
+
+fd_status fd_regional_step_mass(fd_ctx* c, const void* x, const void* cond, const int32_t* labels, const uint8_t* mask, int B,
+                                int N, int R, void* kv_cache, void* y, int32_t* active_idx_out, int32_t* cu_active_out,
+                                double* region_mass_out, void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!region_mass_out) return c->fail(FD_ERR_INVALID_ARG, "region_mass_out is null");
+    fd_status s = fd_regional_step_check(c, x, cond, labels, mask, B, N, R, kv_cache, y, active_idx_out, cu_active_out);
+    if (s != FD_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (c->cfg.dtype == FD_BF16)
+        return run_step<__nv_bfloat16>(c, x, cond, labels, mask, B, N, R, kv_cache, y, active_idx_out, cu_active_out, st,
+                                       region_mass_out);
+    return run_step<float>(c, x, cond, labels, mask, B, N, R, kv_cache, y, active_idx_out, cu_active_out, st, region_mass_out);
+}
+
+fd_status fd_region_activity_attn(fd_ctx* c, const double* region_mass, const int32_t* region_sizes, int B, int R,
+                                  const float* eps, float* rbar_state, float* delta_state, int32_t* skip_count,
+                                  uint8_t* prev_active, float* importance_out, float* weight_out, uint8_t* mask_out,
+                                  void* cuda_stream) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!region_mass || !region_sizes || !eps || !rbar_state || !delta_state || !skip_count || !prev_active ||
+        !importance_out || !weight_out || !mask_out)
+        return c->fail(FD_ERR_INVALID_ARG, "null pointer argument");
+    if (B < 1 || R < 1) return c->fail(FD_ERR_SHAPE, "B and R must be positive");
+    if (B > c->cfg.max_batch || R > c->cfg.max_regions)
+        return c->fail(FD_ERR_SHAPE, "B=%d R=%d exceed the limits %d/%d", B, R, c->cfg.max_batch, c->cfg.max_regions);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int nl = 0;
+    c->span_begin(FD_PROF_ACTIVITY, st);
+    cudaError_t e = launch_attn_gate(region_mass, region_sizes, B, R, eps, c->cfg.gate_eta, c->cfg.max_skip_k, rbar_state,
+                                     delta_state, skip_count, prev_active, importance_out, weight_out, mask_out, st, &nl);
+    c->span_end(nl, st);
+    c->launches += nl;
+    if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "attention gate launch failed: %s", cudaGetErrorString(e));
+    return FD_OK;
 }
 
 fd_status fd_poll_status(fd_ctx* c, void* cuda_stream) {

@@ -68,25 +68,44 @@ constexpr int AT_MAXD = 128;
 
 template <typename T>
 __global__ void __launch_bounds__(128)
-simt_attention_kernel(const T* __restrict__ q, int q_ld, const T* __restrict__ kv, T* __restrict__ o, int o_ld,
-                      const QTile* __restrict__ tiles, int N, int H, int dh, float sm_scale,
-                      const Control* __restrict__ ctl) {
+simt_attention_kernel(const T* __restrict__ q, int q_ld, int q_head_stride, const T* __restrict__ kv, T* __restrict__ o,
+                      int o_ld, const QTile* __restrict__ tiles, int N, int H, int dh, float sm_scale,
+                      const Control* __restrict__ ctl, const int32_t* __restrict__ labels,
+                      const int32_t* __restrict__ active_idx, double* __restrict__ region_mass, int R, float inv_heads,
+                      int sub_tiles) {
     __shared__ float Qs[AT_ROWS][AT_MAXD];
     __shared__ float Ks[AT_KEYS][AT_MAXD + 1];
     __shared__ float Vs[AT_KEYS][AT_MAXD];
-    if ((int)blockIdx.x >= ctl->n_qtiles) return;
-    const QTile tile = tiles[blockIdx.x];
+    // sub_tiles > 1: the work list was built for larger query tiles; this CTA takes one AT_ROWS slice of one
+    if ((int)blockIdx.x / sub_tiles >= ctl->n_qtiles) return;
+    QTile tile = tiles[blockIdx.x / sub_tiles];
+    {
+        const int sub = (int)blockIdx.x % sub_tiles;
+        tile.row0 += sub * AT_ROWS;
+        tile.rows = min(AT_ROWS, tile.rows - sub * AT_ROWS);
+        if (tile.rows <= 0) return;
+    }
     const int head = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T* Kb = kv + ((size_t)tile.b * 2 + 0) * N * H + (size_t)head * dh;
     const T* Vb = kv + ((size_t)tile.b * 2 + 1) * N * H + (size_t)head * dh;
     for (int i = threadIdx.x; i < AT_ROWS * dh; i += 128) {
         const int r = i / dh, c = i - r * dh;
-        Qs[r][c] = r < tile.rows ? to_f<T>(q[(size_t)(tile.row0 + r) * q_ld + head * dh + c]) * sm_scale : 0.f;
+        Qs[r][c] = r < tile.rows ? to_f<T>(q[(size_t)(tile.row0 + r) * q_ld + head * q_head_stride + c]) * sm_scale : 0.f;
     }
     constexpr int RPW = AT_ROWS / 4;           // rows per warp
     constexpr int CPL = AT_MAXD / 32;          // output channels per lane
     float m[RPW], l[RPW], acc[RPW][CPL];
+    // paper Sec. 4.2: the part of a query's softmax mass that falls on keys of the query's own region
+    // (accumulated like l, against the same running maximum); only when region_mass is given
+    float own[RPW];
+    int row_lab[RPW];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) {
+        own[r] = 0.f;
+        const int lr = warp * RPW + r;
+        row_lab[r] = (region_mass && lr < tile.rows) ? labels[active_idx[tile.row0 + lr]] : -1;
+    }
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
         m[r] = -INFINITY; l[r] = 0.f;
@@ -103,6 +122,7 @@ simt_attention_kernel(const T* __restrict__ q, int q_ld, const T* __restrict__ k
         }
         __syncthreads();
         const bool key_ok = (t0 + lane) < N;
+        const int key_lab = (region_mass && key_ok) ? labels[(size_t)tile.b * N + t0 + lane] : -2;
 #pragma unroll
         for (int r = 0; r < RPW; ++r) {
             const float* qr = Qs[warp * RPW + r];
@@ -113,6 +133,7 @@ simt_attention_kernel(const T* __restrict__ q, int q_ld, const T* __restrict__ k
             const float p = key_ok ? __expf(s - m_new) : 0.f;
             const float corr = __expf(m[r] - m_new);     // m = -inf on the first tile gives 0
             l[r] = l[r] * corr + warp_sum(p);
+            if (region_mass) own[r] = own[r] * corr + warp_sum(key_lab == row_lab[r] ? p : 0.f);
             m[r] = m_new;
 #pragma unroll
             for (int c = 0; c < CPL; ++c) acc[r][c] *= corr;
@@ -131,11 +152,15 @@ simt_attention_kernel(const T* __restrict__ q, int q_ld, const T* __restrict__ k
         const int lr = warp * RPW + r;
         if (lr < tile.rows) {
             const float inv = 1.0f / l[r];
+            if (o) {
 #pragma unroll
-            for (int c = 0; c < CPL; ++c) {
-                const int ch = lane + 32 * c;
-                if (ch < dh) o[(size_t)(tile.row0 + lr) * o_ld + head * dh + ch] = from_f<T>(acc[r][c] * inv);
+                for (int c = 0; c < CPL; ++c) {
+                    const int ch = lane + 32 * c;
+                    if (ch < dh) o[(size_t)(tile.row0 + lr) * o_ld + head * dh + ch] = from_f<T>(acc[r][c] * inv);
+                }
             }
+            if (region_mass && lane == 0 && row_lab[r] >= 0 && row_lab[r] < R)
+                atomicAdd(&region_mass[(size_t)tile.b * R + row_lab[r]], (double)(own[r] * inv * inv_heads));
         }
     }
 }
@@ -158,10 +183,12 @@ cudaError_t launch_simt_gemm(int kind, const T* a, int lda, const T* w, int n_ou
 template <typename T>
 cudaError_t launch_simt_attention(const T* q, int q_ld, const T* kv, T* o, int o_ld, const QTile* tiles,
                                   int max_tiles, int N, int H, int heads, int dh, const Control* ctl,
-                                  cudaStream_t st, int* n_launch) {
-    dim3 grid(max_tiles, heads);
-    simt_attention_kernel<T><<<grid, 128, 0, st>>>(q, q_ld, kv, o, o_ld, tiles, N, H, dh,
-                                                  1.0f / sqrtf((float)dh), ctl);
+                                  cudaStream_t st, int* n_launch, int q_head_stride, const int32_t* labels,
+                                  const int32_t* active_idx, double* region_mass, int R, int sub_tiles) {
+    dim3 grid(max_tiles * sub_tiles, heads);
+    simt_attention_kernel<T><<<grid, 128, 0, st>>>(q, q_ld, q_head_stride > 0 ? q_head_stride : dh, kv, o, o_ld, tiles, N, H, dh,
+                                                  1.0f / sqrtf((float)dh), ctl, labels, active_idx, region_mass, R,
+                                                  1.0f / (float)heads, sub_tiles);
     ++*n_launch;
     return cudaGetLastError();
 }
@@ -173,9 +200,11 @@ template cudaError_t launch_simt_gemm<float>(int, const float*, int, const float
 template cudaError_t launch_simt_gemm<__nv_bfloat16>(int, const __nv_bfloat16*, int, const __nv_bfloat16*, int, int,
                                                      int, const EpiParams&, const Control*, cudaStream_t, int*);
 template cudaError_t launch_simt_attention<float>(const float*, int, const float*, float*, int, const QTile*, int, int,
-                                                  int, int, int, const Control*, cudaStream_t, int*);
+                                                  int, int, int, const Control*, cudaStream_t, int*, int, const int32_t*,
+                                                  const int32_t*, double*, int, int);
 template cudaError_t launch_simt_attention<__nv_bfloat16>(const __nv_bfloat16*, int, const __nv_bfloat16*,
                                                           __nv_bfloat16*, int, const QTile*, int, int, int, int, int,
-                                                          const Control*, cudaStream_t, int*);
+                                                          const Control*, cudaStream_t, int*, int, const int32_t*,
+                                                          const int32_t*, double*, int, int);
 
 }  // namespace fd
