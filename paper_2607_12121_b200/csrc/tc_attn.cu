@@ -49,7 +49,7 @@ template <int D> struct AttCfg {
     static constexpr int TILE_BYTES = SUBS * SUB_BYTES + (D == 72 ? TAIL_BYTES : 0);
     // K/V rings deep enough that a tile is requested several tile periods before it is needed
     static constexpr int STAGES = D == 128 ? 2 : (D == 72 ? 4 : 5);
-    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + (D == 64 ? 128 * 144 : 0);
+    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + (D == 64 ? 128 * 144 + 2048 : 0);
 };
 
 // Register re-balancing between warpgroups: the kernel starts with 128 registers per thread (512 threads);
@@ -119,12 +119,23 @@ constexpr float RESCALE_LOG2 = 24.0f;
 // TMEM columns: two score buffers, the output accumulator, two P buffers (bf16 pairs)
 constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384, TMEM_COLS = 512;
 
-template <int D>
+// What the MASS variant (head dim 64, launched for a step's first block when asked) needs on top: per region, the
+// softmax mass its active queries put on keys of their own region (paper Sec. 4.2).
+struct MassArgs {
+    const int32_t* labels;       // [B, N]
+    const int32_t* active_idx;   // compact row -> global token id
+    double* region_mass;         // [B, R], accumulated with atomics
+    int R;
+    float inv_heads;
+};
+
+template <int D, bool MASS = false>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
                     const __grid_constant__ CUtensorMap tm_q_tail, const __grid_constant__ CUtensorMap tm_kv_tail,
                     __nv_bfloat16* __restrict__ o, int o_ld, const QTile* __restrict__ tiles, int heads, int N,
-                    float scale_log2, Control* ctl) {
+                    float scale_log2, Control* ctl, MassArgs ma) {
+    static_assert(!MASS || D == 64, "the mass output exists for head dim 64 only");
     using Cfg = AttCfg<D>;
     constexpr int DP = Cfg::DP;
     constexpr bool SPLIT = D == 64;                      // per-half accumulators, no exchange in the key loop
@@ -154,6 +165,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     float* s_xmax = reinterpret_cast<float*>(tmem_slot + 2);      // head dim 64: row maxima, [2 items][2 halves][128 rows]
     float* s_xsum = s_xmax + 512;                                 // [2 halves][128 rows]; head dim 64: [2 items][2 halves][128 rows]
     uint8_t* s_stage = reinterpret_cast<uint8_t*>(bars) + 4608;   // [128 rows][144 bytes], head dim 64 only
+    float* s_xown = reinterpret_cast<float*>(s_stage + 128 * 144);   // MASS: own-region mass, [2 items][2 halves][128 rows]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (smem_u32(smem) & 1023u) {                        // never expected; refuse rather than compute garbage
@@ -351,6 +363,15 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
             for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
                 float m = -INFINITY, l = 0.f;
+                // MASS: the part of l that comes from keys carrying the query's own region label
+                float own = 0.f;
+                int my_lab = -1;
+                const int32_t* key_lab = nullptr;
+                if constexpr (MASS) {
+                    const QTile t = tiles[w % n_tiles];
+                    if (r < t.rows) my_lab = ma.labels[ma.active_idx[t.row0 + r]];
+                    key_lab = ma.labels + (size_t)t.b * N;
+                }
                 auto tile = [&](const int j) -> bool {
                     const uint32_t g = g0 + j, bs = g & 1;
                     if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) return false;
@@ -359,6 +380,12 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64, sr);
                     tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + 32, sr + 32);
                     tmem_wait_ld();
+                    int kl0 = -2, kl1 = -2;                      // MASS: labels of this half's keys lane, lane + 32
+                    if constexpr (MASS) {
+                        const int k0 = j * KEYS + half * 64 + lane;
+                        if (k0 < N) kl0 = __ldg(key_lab + k0);
+                        if (k0 + 32 < N) kl1 = __ldg(key_lab + k0 + 32);
+                    }
                     const bool tail = j == n_kv - 1 && rem < KEYS;
                     if (tail) {
 #pragma unroll
@@ -385,7 +412,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             if (!mbar_wait(&pv_done[((g - 1) & 1) * 2 + half], ((g - 1) >> 1) & 1, abort_flag)) return false;
                             tc_fence_after();
                             const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
-                            if (need) { l *= f; m = mx; }
+                            if (need) { l *= f; m = mx; own *= f; }
 #pragma unroll
                             for (int c = 0; c < 2; ++c) {
                                 uint32_t orr[32];
@@ -410,7 +437,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const uint64_t x = fma2(pair(__uint_as_float(sr[2 * i + 2 * e]), __uint_as_float(sr[2 * i + 2 * e + 1])), sc2, nmb2);
-                            if (e < 3) {
+                            if (MASS || e < 3) {                 // MASS: no polynomial share, the body must stay small
                                 float xa, xb;
                                 unpair(x, xa, xb);
                                 p[2 * e] = ex2(xa);
@@ -421,6 +448,16 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         }
                         sua = add2(sua, add2(pair(p[0], p[1]), pair(p[2], p[3])));
                         sub_ = add2(sub_, add2(pair(p[4], p[5]), pair(p[6], p[7])));
+                        if constexpr (MASS) {
+                            // the 8 keys of this group: positions 2 i .. 2 i + 7 of this half; their labels sit in lanes
+                            // (2 i + e) % 32 of kl0 / kl1 (a key past N has p = 0 and the label -2)
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                const int kk = 2 * i + e;
+                                const int kl = __shfl_sync(0xffffffffu, kk < 32 ? kl0 : kl1, kk & 31);
+                                own += kl == my_lab ? p[e] : 0.f;
+                            }
+                        }
 #pragma unroll
                         for (int e = 0; e < 4; ++e) pk[i + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
                     }
@@ -447,6 +484,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (item_i >= 2 && !mbar_wait(&stat_free[slot], ((item_i >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
                 s_xmax[(slot * 2 + half) * 128 + r] = m;
                 s_xsum[(slot * 2 + half) * 128 + r] = l;
+                if constexpr (MASS) s_xown[(slot * 2 + half) * 128 + r] = own;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&stat_full[slot]);
                 g0 += n_kv;
@@ -635,6 +673,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (!mbar_wait(&stat_full[slot], (item_i >> 1) & 1, abort_flag)) { ok = false; break; }
                 const float m0 = s_xmax[(slot * 2 + 0) * 128 + r], l0 = s_xsum[(slot * 2 + 0) * 128 + r];
                 const float m1 = s_xmax[(slot * 2 + 1) * 128 + r], l1 = s_xsum[(slot * 2 + 1) * 128 + r];
+                float own0 = 0.f, own1 = 0.f;
+                if constexpr (MASS) { own0 = s_xown[(slot * 2 + 0) * 128 + r]; own1 = s_xown[(slot * 2 + 1) * 128 + r]; }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&stat_free[slot]);
                 // every product of the item must have landed: the last tile, both halves
@@ -647,6 +687,19 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const float a1 = m1 == -INFINITY ? 0.f : ex2((m1 - m_all) * scale_log2);
                 const float inv = 1.0f / (a0 * l0 + a1 * l1);
                 const float w_0 = a0 * inv, w_1 = a1 * inv;       // weights of O_0, O_1
+                if constexpr (MASS) {
+                    // consecutive compact rows mostly share their region: the lanes of one label add up first, so that a
+                    // region receives one atomic per warp instead of one per row
+                    int lab = -1;
+                    if (r < t.rows) lab = ma.labels[ma.active_idx[t.row0 + r]];
+                    if (lab >= ma.R) lab = -1;
+                    const float mine = lab >= 0 ? (w_0 * own0 + w_1 * own1) * ma.inv_heads : 0.f;
+                    const uint32_t peers = __match_any_sync(0xffffffffu, lab);
+                    float sum = 0.f;
+                    for (uint32_t rest = peers; rest; rest &= rest - 1)
+                        sum += __shfl_sync(peers, mine, __ffs(rest) - 1);
+                    if (lab >= 0 && lane == __ffs(peers) - 1) atomicAdd(&ma.region_mass[(size_t)t.b * ma.R + lab], (double)sum);
+                }
                 // a rolled loop on purpose: this code runs once per item, and the fewer instructions it fetches the
                 // less it disturbs the softmax warps that share the instruction caches
 #pragma unroll 1
@@ -731,6 +784,8 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
     cudaError_t e = cudaSuccess;
     if (ok) e = cudaFuncSetAttribute(tc_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<64>::SMEM);
     if (ok && e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_attention_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<64>::SMEM);
+    if (ok && e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<128>::SMEM);
     if (ok && e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_attention_kernel<72>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<72>::SMEM);
@@ -744,8 +799,11 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
 
 void tc_attention_plan_destroy(void* p) { delete static_cast<AttnPlan*>(p); }
 
+bool tc_attention_has_mass(const fd_config& c) { return tc_attention_supported(c) && c.head_dim == 64; }
+
 cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
-                         const Control* ctl, cudaStream_t st, int* n_launch) {
+                         const Control* ctl, cudaStream_t st, int* n_launch, const int32_t* labels,
+                         const int32_t* active_idx, double* region_mass, int R) {
     AttnPlan* a = static_cast<AttnPlan*>(tc_plan_attn(p));
     if (!a) return cudaErrorNotSupported;
     CUtensorMap kv_map, kv_tail_map;
@@ -760,11 +818,15 @@ cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, c
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)a->dh);
     Control* c = const_cast<Control*>(ctl);
     __nv_bfloat16* o = static_cast<__nv_bfloat16*>(a->o);
+    MassArgs ma{labels, active_idx, region_mass, R, 1.0f / (float)a->heads};
     cudaError_t e = cudaSuccess;
 #define FD_ATT(DD)                                                                                                  \
     e = launch_kernel(tc_attention_kernel<DD>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, tc_plan_pdl(p), a->q_map, kv_map, \
-                      a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c)
-    if (a->dh == 64) FD_ATT(64);
+                      a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c, ma)
+    if (a->dh == 64 && region_mass) {
+        e = launch_kernel(tc_attention_kernel<64, true>, grid, ATT_THREADS, AttCfg<64>::SMEM, st, tc_plan_pdl(p), a->q_map, kv_map,
+                          a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c, ma);
+    } else if (a->dh == 64) FD_ATT(64);
     else if (a->dh == 128) FD_ATT(128);
     else FD_ATT(72);
 #undef FD_ATT
