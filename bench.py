@@ -434,6 +434,30 @@ def run_ours(args):
                "update_gbs": upd_bytes / upd_us / 1e3, "note": "outside the timed step; algorithmic bytes / CUDA-event time"}
     fd.fd_poll_status(ctx)
 
+    # the paper's own gate signal (Sec. 4.2): extra cost of collecting the first block's own-region attention mass
+    # inside the step, and the gate evaluated on it (outside the timed step, whose gate is the latent-change one)
+    mass = torch.zeros((B, R), dtype=torch.float64, device=dev)
+    sizes = torch.from_numpy(np.stack([np.bincount(l[l < R], minlength=R) for l in labels_np]).astype(np.int32)).to(dev)
+    g_rbar = torch.zeros((B, R), dtype=torch.float32, device=dev)
+    g_imp = torch.empty((B, R), dtype=torch.float32, device=dev)
+
+    def mass_step():
+        fd.fd_regional_step_mass(ctx, x, cond, labels, mask, R, kv, y, active_idx, cu_active, mass)
+
+    def plain_step():
+        fd.fd_regional_step(ctx, x, cond, labels, mask, R, kv, y, active_idx, cu_active)
+
+    ms_plain = time_us(plain_step, 5) / 1e3
+    ms_mass = time_us(mass_step, 5) / 1e3
+    gate_attn_us = time_us(lambda: fd.fd_region_activity_attn(ctx, mass, sizes, eps, g_rbar, delta, skip, prev, g_imp,
+                                                              weight, mask))
+    attn_signal = {"step_ms": ms_plain, "step_with_mass_ms": ms_mass, "mass_extra_ms": ms_mass - ms_plain,
+                   "gate_us": gate_attn_us,
+                   "note": "first block's own-region softmax mass (fused in the tensor-core kernel at head dim 64, "
+                           "a CUDA-core pass otherwise) + the gate on it; outside the timed step"}
+    delta.zero_(); skip.zero_(); prev.fill_(1)
+    fd.fd_poll_status(ctx)
+
     # streaming rate of the activity reduction on a batch large enough to be bandwidth bound (at the
     # benchmark shapes the gate moves a few MB and is launch-latency bound): 256 requests x 8192 tokens x 64
     # channels, all regions fresh, through the allocation-free entry point
@@ -534,6 +558,7 @@ def run_ours(args):
         "activity_probe": None if probe is None else dict(probe, frac_of_hbm=probe["gbs"] / float(peaks["hbm_gbs"]),
                                                          workload="256 requests x 8192 tokens x 64 channels, 64 regions"),
         "sampler": sampler,
+        "attention_gate_signal": attn_signal,
         "peaks": {"source": peak_kind, "bf16_tflops": peaks.get("bf16_tflops"),
                   "bf16_tflops_sustained": peaks.get("bf16_tflops_sustained"), "hbm_gbs": peaks.get("hbm_gbs")},
     }
