@@ -447,8 +447,12 @@ def run_ours(args):
     def plain_step():
         fd.fd_regional_step(ctx, x, cond, labels, mask, R, kv, y, active_idx, cu_active)
 
-    ms_plain = time_us(plain_step, 5) / 1e3
-    ms_mass = time_us(mass_step, 5) / 1e3
+    # alternate the two forms: under the power cap the clock drifts over seconds, which would bias whichever ran second
+    tp, tm = [], []
+    for _ in range(4):
+        tp.append(time_us(plain_step, 3) / 1e3)
+        tm.append(time_us(mass_step, 3) / 1e3)
+    ms_plain, ms_mass = float(np.median(tp)), float(np.median(tm))
     gate_attn_us = time_us(lambda: fd.fd_region_activity_attn(ctx, mass, sizes, eps, g_rbar, delta, skip, prev, g_imp,
                                                               weight, mask))
     attn_signal = {"step_ms": ms_plain, "step_with_mass_ms": ms_mass, "mass_extra_ms": ms_mass - ms_plain,
