@@ -457,8 +457,8 @@ def run_ours(args):
                                                               weight, mask))
     attn_signal = {"step_ms": ms_plain, "step_with_mass_ms": ms_mass, "mass_extra_ms": ms_mass - ms_plain,
                    "gate_us": gate_attn_us,
-                   "note": "first block's own-region softmax mass (fused in the tensor-core kernel at head dim 64, "
-                           "a CUDA-core pass otherwise) + the gate on it; outside the timed step"}
+                   "note": "first block's own-region softmax mass (fused in a variant of the tensor-core attention "
+                           "kernel) + the gate on it; outside the timed step"}
     delta.zero_(); skip.zero_(); prev.fill_(1)
     fd.fd_poll_status(ctx)
 

@@ -49,7 +49,7 @@ template <int D> struct AttCfg {
     static constexpr int TILE_BYTES = SUBS * SUB_BYTES + (D == 72 ? TAIL_BYTES : 0);
     // K/V rings deep enough that a tile is requested several tile periods before it is needed
     static constexpr int STAGES = D == 128 ? 2 : (D == 72 ? 4 : 5);
-    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + (D == 64 ? 128 * 144 + 2048 : 0);
+    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + (D == 64 ? 128 * 144 : 0) + 2048;
 };
 
 // Register re-balancing between warpgroups: the kernel starts with 128 registers per thread (512 threads);
@@ -135,7 +135,6 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const __grid_constant__ CUtensorMap tm_q_tail, const __grid_constant__ CUtensorMap tm_kv_tail,
                     __nv_bfloat16* __restrict__ o, int o_ld, const QTile* __restrict__ tiles, int heads, int N,
                     float scale_log2, Control* ctl, MassArgs ma) {
-    static_assert(!MASS || D == 64, "the mass output exists for head dim 64 only");
     using Cfg = AttCfg<D>;
     constexpr int DP = Cfg::DP;
     constexpr bool SPLIT = D == 64;                      // per-half accumulators, no exchange in the key loop
@@ -165,7 +164,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     float* s_xmax = reinterpret_cast<float*>(tmem_slot + 2);      // head dim 64: row maxima, [2 items][2 halves][128 rows]
     float* s_xsum = s_xmax + 512;                                 // [2 halves][128 rows]; head dim 64: [2 items][2 halves][128 rows]
     uint8_t* s_stage = reinterpret_cast<uint8_t*>(bars) + 4608;   // [128 rows][144 bytes], head dim 64 only
-    float* s_xown = reinterpret_cast<float*>(s_stage + 128 * 144);   // MASS: own-region mass, [2 items][2 halves][128 rows]
+    // MASS: own-region mass, head dim 64 [2 items][2 halves][128 rows], otherwise [2 halves][128 rows]
+    float* s_xown = reinterpret_cast<float*>(s_stage + (D == 64 ? 128 * 144 : 0));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (smem_u32(smem) & 1023u) {                        // never expected; refuse rather than compute garbage
@@ -505,10 +505,25 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const QTile t = tiles[w % n_tiles];
                 const int head = w / n_tiles;
                 float m = -INFINITY, l = 0.f;
+                // MASS: the part of l that comes from keys carrying the query's own region label
+                float own = 0.f;
+                int my_lab = -1;
+                const int32_t* key_lab = nullptr;
+                if constexpr (MASS) {
+                    if (r < t.rows) my_lab = ma.labels[ma.active_idx[t.row0 + r]];
+                    if (my_lab >= ma.R) my_lab = -1;
+                    key_lab = ma.labels + (size_t)t.b * N;
+                }
                 for (int j = 0; j < n_kv && ok; ++j) {
                     const uint32_t g = g0 + j, bs = g & 1;
                     if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
+                    int kl0 = -2, kl1 = -2;                      // MASS: labels of this half's keys lane, lane + 32
+                    if constexpr (MASS) {
+                        const int k0 = j * KEYS + half * 64 + lane;
+                        if (k0 < N) kl0 = __ldg(key_lab + k0);
+                        if (k0 + 32 < N) kl1 = __ldg(key_lab + k0 + 32);
+                    }
                     uint32_t sr[64];
                     tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64, sr);
                     tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + 32, sr + 32);
@@ -540,7 +555,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             if (!mbar_wait(&pv_done[((g - 1) & 1) * 2], ((g - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
                             tc_fence_after();
                             const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
-                            if (need) { l *= f; m = mx; }
+                            if (need) { l *= f; m = mx; own *= f; }
     #pragma unroll
                             for (int c = 0; c < DH / 32; ++c) {
                                 uint32_t orr[32];
@@ -574,7 +589,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const uint64_t x = fma2(pair(__uint_as_float(sr[2 * i + 2 * e]), __uint_as_float(sr[2 * i + 2 * e + 1])), sc2, nmb2);
-                            if (e < 3) {
+                            if (MASS || e < 3) {                 // MASS: no polynomial share, the body must stay small
                                 float xa, xb;
                                 unpair(x, xa, xb);
                                 p[2 * e] = ex2(xa);
@@ -585,6 +600,14 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         }
                         sua = add2(sua, add2(pair(p[0], p[1]), pair(p[2], p[3])));
                         sub_ = add2(sub_, add2(pair(p[4], p[5]), pair(p[6], p[7])));
+                        if constexpr (MASS) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                const int kk = 2 * i + e;
+                                const int kl = __shfl_sync(0xffffffffu, kk < 32 ? kl0 : kl1, kk & 31);
+                                own += kl == my_lab ? p[e] : 0.f;
+                            }
+                        }
 #pragma unroll
                         for (int e = 0; e < 4; ++e) pk[i + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
                     }
@@ -605,9 +628,20 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // epilogue: O / l for the rows of this tile (l = the two halves' partial sums)
                 const uint32_t gl = g0 + n_kv - 1;
                 s_xsum[half * 128 + r] = l;
+                if constexpr (MASS) s_xown[half * 128 + r] = own;
                 mbar_arrive(&l_bar[quad]);
                 if (!mbar_wait(&l_bar[quad], item_i & 1, abort_flag)) { ok = false; break; }
                 const float inv = 1.0f / (l + s_xsum[(half ^ 1) * 128 + r]);
+                if constexpr (MASS) {
+                    if (half == 0) {      // one of the row's two threads reports; the lanes of one label add up first
+                        const float mine = my_lab >= 0 ? (own + s_xown[128 + r]) * inv * ma.inv_heads : 0.f;
+                        const uint32_t peers = __match_any_sync(0xffffffffu, my_lab);
+                        float sum = 0.f;
+                        for (uint32_t rest = peers; rest; rest &= rest - 1) sum += __shfl_sync(peers, mine, __ffs(rest) - 1);
+                        if (my_lab >= 0 && lane == __ffs(peers) - 1)
+                            atomicAdd(&ma.region_mass[(size_t)t.b * ma.R + my_lab], (double)sum);
+                    }
+                }
                 if (!mbar_wait(&pv_done[(gl & 1) * 2], (gl >> 1) & 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 __nv_bfloat16* dst = o + (size_t)(t.row0 + r) * o_ld + head * D + half * DH;
@@ -786,6 +820,10 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
     if (ok && e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_attention_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<64>::SMEM);
     if (ok && e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_attention_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<128>::SMEM);
+    if (ok && e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_attention_kernel<72, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<72>::SMEM);
+    if (ok && e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<128>::SMEM);
     if (ok && e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_attention_kernel<72>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<72>::SMEM);
@@ -799,7 +837,7 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
 
 void tc_attention_plan_destroy(void* p) { delete static_cast<AttnPlan*>(p); }
 
-bool tc_attention_has_mass(const fd_config& c) { return tc_attention_supported(c) && c.head_dim == 64; }
+bool tc_attention_has_mass(const fd_config& c) { return tc_attention_supported(c); }
 
 cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch, const int32_t* labels,
@@ -823,10 +861,15 @@ cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, c
 #define FD_ATT(DD)                                                                                                  \
     e = launch_kernel(tc_attention_kernel<DD>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, tc_plan_pdl(p), a->q_map, kv_map, \
                       a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c, ma)
-    if (a->dh == 64 && region_mass) {
-        e = launch_kernel(tc_attention_kernel<64, true>, grid, ATT_THREADS, AttCfg<64>::SMEM, st, tc_plan_pdl(p), a->q_map, kv_map,
-                          a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c, ma);
+#define FD_ATT_MASS(DD)                                                                                             \
+    e = launch_kernel(tc_attention_kernel<DD, true>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, tc_plan_pdl(p), a->q_map, kv_map, \
+                      a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c, ma)
+    if (region_mass) {
+        if (a->dh == 64) FD_ATT_MASS(64);
+        else if (a->dh == 128) FD_ATT_MASS(128);
+        else FD_ATT_MASS(72);
     } else if (a->dh == 64) FD_ATT(64);
+#undef FD_ATT_MASS
     else if (a->dh == 128) FD_ATT(128);
     else FD_ATT(72);
 #undef FD_ATT
