@@ -205,14 +205,8 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             if (e != cudaSuccess) { c->launches += nl; return c->fail(FD_ERR_CUDA, "memset failed: %s", cudaGetErrorString(e)); }
         }
         if (c->use_tc_attn) {
-            const bool fused = mass && tc_attention_has_mass(cf);
             FD_TRY(FD_PROF_ATTENTION, tc_attention(c->tc, blk, kv_b, B, N, tiles, max_tiles, ctl, st, &nl, labels, active_idx,
-                                                   fused ? mass : nullptr, R));
-            if (mass && !fused)     // other head dims: a second pass on the CUDA cores, mass only
-                FD_TRY(FD_PROF_ATTENTION, launch_simt_attention<T>(q, l.q_ld, kv_b, static_cast<T*>(nullptr), H, tiles,
-                                                max_tiles, N, H, cf.n_heads, cf.head_dim, ctl, st, &nl,
-                                                tc_attention_head_pad(cf.head_dim), labels, active_idx, mass, R,
-                                                c->tile_rows / simt_attention_tile_rows()));
+                                                   mass, R));
         } else {
             FD_TRY(FD_PROF_ATTENTION, launch_simt_attention<T>(q, l.q_ld, kv_b, o, H, tiles, max_tiles, N, H, cf.n_heads, cf.head_dim,
                                             ctl, st, &nl, 0, labels, active_idx, mass, R));

@@ -126,8 +126,7 @@ template <typename T>
 cudaError_t launch_simt_attention(const T* q, int q_ld, const T* kv, T* o, int o_ld, const QTile* tiles,
                                   int max_tiles, int N, int H, int heads, int dh, const Control* ctl,
                                   cudaStream_t st, int* n_launch, int q_head_stride = 0, const int32_t* labels = nullptr,
-                                  const int32_t* active_idx = nullptr, double* region_mass = nullptr, int R = 0,
-                                  int sub_tiles = 1);
+                                  const int32_t* active_idx = nullptr, double* region_mass = nullptr, int R = 0);
 // activity.cu: the gate on the attention-mass signal
 cudaError_t launch_attn_gate(const double* region_mass, const int32_t* region_sizes, int B, int R, const float* eps,
                              float eta, int K, float* rbar, float* delta, int32_t* skip_count, uint8_t* prev_active,

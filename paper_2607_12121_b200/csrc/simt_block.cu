@@ -71,20 +71,12 @@ __global__ void __launch_bounds__(128)
 simt_attention_kernel(const T* __restrict__ q, int q_ld, int q_head_stride, const T* __restrict__ kv, T* __restrict__ o,
                       int o_ld, const QTile* __restrict__ tiles, int N, int H, int dh, float sm_scale,
                       const Control* __restrict__ ctl, const int32_t* __restrict__ labels,
-                      const int32_t* __restrict__ active_idx, double* __restrict__ region_mass, int R, float inv_heads,
-                      int sub_tiles) {
+                      const int32_t* __restrict__ active_idx, double* __restrict__ region_mass, int R, float inv_heads) {
     __shared__ float Qs[AT_ROWS][AT_MAXD];
     __shared__ float Ks[AT_KEYS][AT_MAXD + 1];
     __shared__ float Vs[AT_KEYS][AT_MAXD];
-    // sub_tiles > 1: the work list was built for larger query tiles; this CTA takes one AT_ROWS slice of one
-    if ((int)blockIdx.x / sub_tiles >= ctl->n_qtiles) return;
-    QTile tile = tiles[blockIdx.x / sub_tiles];
-    {
-        const int sub = (int)blockIdx.x % sub_tiles;
-        tile.row0 += sub * AT_ROWS;
-        tile.rows = min(AT_ROWS, tile.rows - sub * AT_ROWS);
-        if (tile.rows <= 0) return;
-    }
+    if ((int)blockIdx.x >= ctl->n_qtiles) return;
+    const QTile tile = tiles[blockIdx.x];
     const int head = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T* Kb = kv + ((size_t)tile.b * 2 + 0) * N * H + (size_t)head * dh;
@@ -152,12 +144,10 @@ simt_attention_kernel(const T* __restrict__ q, int q_ld, int q_head_stride, cons
         const int lr = warp * RPW + r;
         if (lr < tile.rows) {
             const float inv = 1.0f / l[r];
-            if (o) {
 #pragma unroll
-                for (int c = 0; c < CPL; ++c) {
-                    const int ch = lane + 32 * c;
-                    if (ch < dh) o[(size_t)(tile.row0 + lr) * o_ld + head * dh + ch] = from_f<T>(acc[r][c] * inv);
-                }
+            for (int c = 0; c < CPL; ++c) {
+                const int ch = lane + 32 * c;
+                if (ch < dh) o[(size_t)(tile.row0 + lr) * o_ld + head * dh + ch] = from_f<T>(acc[r][c] * inv);
             }
             if (region_mass && lane == 0 && row_lab[r] >= 0 && row_lab[r] < R)
                 atomicAdd(&region_mass[(size_t)tile.b * R + row_lab[r]], (double)(own[r] * inv * inv_heads));
@@ -184,11 +174,11 @@ template <typename T>
 cudaError_t launch_simt_attention(const T* q, int q_ld, const T* kv, T* o, int o_ld, const QTile* tiles,
                                   int max_tiles, int N, int H, int heads, int dh, const Control* ctl,
                                   cudaStream_t st, int* n_launch, int q_head_stride, const int32_t* labels,
-                                  const int32_t* active_idx, double* region_mass, int R, int sub_tiles) {
-    dim3 grid(max_tiles * sub_tiles, heads);
+                                  const int32_t* active_idx, double* region_mass, int R) {
+    dim3 grid(max_tiles, heads);
     simt_attention_kernel<T><<<grid, 128, 0, st>>>(q, q_ld, q_head_stride > 0 ? q_head_stride : dh, kv, o, o_ld, tiles, N, H, dh,
                                                   1.0f / sqrtf((float)dh), ctl, labels, active_idx, region_mass, R,
-                                                  1.0f / (float)heads, sub_tiles);
+                                                  1.0f / (float)heads);
     ++*n_launch;
     return cudaGetLastError();
 }
@@ -201,10 +191,10 @@ template cudaError_t launch_simt_gemm<__nv_bfloat16>(int, const __nv_bfloat16*, 
                                                      int, const EpiParams&, const Control*, cudaStream_t, int*);
 template cudaError_t launch_simt_attention<float>(const float*, int, const float*, float*, int, const QTile*, int, int,
                                                   int, int, int, const Control*, cudaStream_t, int*, int, const int32_t*,
-                                                  const int32_t*, double*, int, int);
+                                                  const int32_t*, double*, int);
 template cudaError_t launch_simt_attention<__nv_bfloat16>(const __nv_bfloat16*, int, const __nv_bfloat16*,
                                                           __nv_bfloat16*, int, const QTile*, int, int, int, int, int,
                                                           const Control*, cudaStream_t, int*, int, const int32_t*,
-                                                          const int32_t*, double*, int, int);
+                                                          const int32_t*, double*, int);
 
 }  // namespace fd

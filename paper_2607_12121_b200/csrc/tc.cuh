@@ -27,11 +27,10 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
 void tc_plan_destroy(TcPlan* p);
 cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
                     int* n_launch);
-// region_mass (optional; tc_attention_has_mass says whether this configuration has the fused variant): [B, R] f64, receives the own-region softmax mass
+// region_mass (optional): [B, R] f64, receives the own-region softmax mass
 cudaError_t tc_attention(TcPlan* p, int blk, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch, const int32_t* labels = nullptr,
                          const int32_t* active_idx = nullptr, double* region_mass = nullptr, int R = 0);
-bool tc_attention_has_mass(const fd_config& cfg);
 
 cudaError_t launch_bounded_wait_selftest(Control* ctl, cudaStream_t st, int* n_launch);
 

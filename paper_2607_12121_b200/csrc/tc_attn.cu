@@ -837,7 +837,6 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
 
 void tc_attention_plan_destroy(void* p) { delete static_cast<AttnPlan*>(p); }
 
-bool tc_attention_has_mass(const fd_config& c) { return tc_attention_supported(c); }
 
 cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch, const int32_t* labels,
