@@ -164,7 +164,7 @@ fd_status fd_regional_step(fd_ctx* ctx, const void* x, const void* cond, const i
  * fd_regional_step_mass is fd_regional_step that additionally writes
  *   region_mass_out [B,R] f64 (DEVICE):  sum over the ACTIVE queries u of region i and over the keys v of region i
  *   of SA[u,v] (zero for regions that did not run; tokens with label R belong to no region).
- * The tensor-core engine computes the mass in a second, CUDA-core pass over the first block's scores.
+ * Both engines accumulate the mass inside the first block's attention kernel.
  *
  * fd_region_activity_attn turns it into the next step's mask: for every region executed at the step that produced
  * region_mass (prev_active = 1),  R_i = region_mass / region_sizes^2,  Delta_i = |R_i - Rbar_i|,  Rbar_i <- R_i;
@@ -287,6 +287,33 @@ enum {
 };
 fd_status fd_profile_enable(fd_ctx* ctx, int enable);
 fd_status fd_profile_read(fd_ctx* ctx, void* cuda_stream, float* ms_out, int32_t* kernels_out);
+
+/*
+ * Host-side batch former (Sec. 4.3, patch monotasks).  Pure host code: every pointer below is HOST memory, no
+ * context, no CUDA call, no allocation; safe to call from any thread.
+ *
+ * fd_sched_pack -- the least-maximum-load rule (the equation of Sec. 4.3, "Monotask Packing").  Monotasks are
+ * assigned one after another in the given order; monotask j of cost[j] goes to
+ *     g* = argmin_g  max_g' ( load[g'] + cost[j] if g' == g else load[g'] ).
+ * Among devices that tie on that maximum, home[j] (the device that already holds patches of the same request;
+ * -1 for a warm-up monotask, which has none) wins if it is one of them, else the one with the smallest own load,
+ * else the smallest index.  load [n_devices] f64 is read and updated in place; assign_out [n_tasks] receives g*.
+ * O(n_devices) per monotask.  Errors: FD_ERR_INVALID_ARG for null pointers, n_devices < 1, n_tasks < 0, a
+ * negative or non-finite cost or load, or home[j] >= n_devices (nothing is written in that case).
+ *
+ * fd_sched_form_batch -- which requests run the next device step.  A request's step is one unit (its active
+ * patches run together; switching happens only at step boundaries, i.e. when this is called).  Requests are
+ * visited by (priority descending, arrival ascending, index ascending); a request is taken if its active_tokens
+ * still fit into what is left of token_budget and its state is resident or a residency slot (max_resident minus the
+ * number of resident requests) is free, in which case it takes the slot; a request that does not fit is passed over
+ * and lower-priority ones may use the leftover.  A request without active tokens is taken only if it is resident.
+ *   priority, arrival [n] i32/i64; active_tokens [n] i32 (>= 0); resident [n] u8 in/out; chosen_out [n] u8.
+ * Errors: FD_ERR_INVALID_ARG for null pointers, n < 0, negative tokens or budget, max_resident < 0.
+ */
+fd_status fd_sched_pack(int n_devices, double* load, int n_tasks, const double* cost, const int32_t* home,
+                        int32_t* assign_out);
+fd_status fd_sched_form_batch(int n, const int32_t* priority, const int64_t* arrival, const int32_t* active_tokens,
+                              uint8_t* resident, int64_t token_budget, int max_resident, uint8_t* chosen_out);
 
 /* Releases the context (host memory only; the workspace goes back to the caller). */
 fd_status fd_destroy(fd_ctx* ctx);

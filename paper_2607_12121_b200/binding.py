@@ -22,7 +22,8 @@ FD_ENGINE_AUTO, FD_ENGINE_SIMT, FD_ENGINE_TC = 0, 1, 2
 EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region_activity",
            "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
            "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait",
-           "fd_embed_latent", "fd_update_latent", "fd_regional_step_mass", "fd_region_activity_attn"]
+           "fd_embed_latent", "fd_update_latent", "fd_regional_step_mass", "fd_region_activity_attn",
+           "fd_sched_pack", "fd_sched_form_batch"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
                "gemm_fc2", "partition", "sampler"]
@@ -81,6 +82,10 @@ def _load() -> ctypes.CDLL:
     lib.fd_regional_step_mass.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.fd_region_activity_attn.restype = i32
     lib.fd_region_activity_attn.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.fd_sched_pack.restype = i32
+    lib.fd_sched_pack.argtypes = [i32, vp, i32, vp, vp, vp]
+    lib.fd_sched_form_batch.restype = i32
+    lib.fd_sched_form_batch.argtypes = [i32, vp, vp, vp, vp, ctypes.c_int64, i32, vp]
     lib.fd_embed_latent.restype = i32
     lib.fd_embed_latent.argtypes = [vp, ctypes.POINTER(FdSamplerWeights), vp, i32, i32, vp, vp]
     lib.fd_update_latent.restype = i32
@@ -239,6 +244,40 @@ def fd_region_activity_attn(ctx: Context, region_mass, region_sizes, eps, rbar_s
     _check(ctx.handle, lib.fd_region_activity_attn(
         ctx.handle, _ptr(region_mass), _ptr(region_sizes), B, R, _ptr(eps), _ptr(rbar_state), _ptr(delta_state),
         _ptr(skip_count), _ptr(prev_active), _ptr(importance_out), _ptr(weight_out), _ptr(mask_out), _stream(stream)))
+
+
+def fd_sched_pack(load, cost, home):
+    """Least-maximum-load packing (Sec. 4.3) of monotasks in the given order.  ``load`` [G] float64 numpy array is
+    updated in place; returns the device of every monotask as an int32 array."""
+    import numpy as np
+    assert load.dtype == np.float64 and load.flags["C_CONTIGUOUS"]
+    cost = np.ascontiguousarray(cost, np.float64)
+    home = np.ascontiguousarray(home, np.int32)
+    assign = np.empty(cost.size, np.int32)
+    st = lib.fd_sched_pack(int(load.size), load.ctypes.data_as(ctypes.c_void_p), int(cost.size),
+                           cost.ctypes.data_as(ctypes.c_void_p), home.ctypes.data_as(ctypes.c_void_p),
+                           assign.ctypes.data_as(ctypes.c_void_p))
+    if st != FD_OK:
+        raise FlashDiffError(st, "fd_sched_pack: invalid argument")
+    return assign
+
+
+def fd_sched_form_batch(priority, arrival, active_tokens, resident, token_budget: int, max_resident: int):
+    """Which requests run the next step (Sec. 4.3).  ``resident`` [n] uint8 numpy array is updated in place;
+    returns the uint8 array of chosen requests."""
+    import numpy as np
+    assert resident.dtype == np.uint8 and resident.flags["C_CONTIGUOUS"]
+    priority = np.ascontiguousarray(priority, np.int32)
+    arrival = np.ascontiguousarray(arrival, np.int64)
+    active_tokens = np.ascontiguousarray(active_tokens, np.int32)
+    chosen = np.zeros(resident.size, np.uint8)
+    st = lib.fd_sched_form_batch(int(resident.size), priority.ctypes.data_as(ctypes.c_void_p),
+                                 arrival.ctypes.data_as(ctypes.c_void_p), active_tokens.ctypes.data_as(ctypes.c_void_p),
+                                 resident.ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(int(token_budget)),
+                                 int(max_resident), chosen.ctypes.data_as(ctypes.c_void_p))
+    if st != FD_OK:
+        raise FlashDiffError(st, "fd_sched_form_batch: invalid argument")
+    return chosen
 
 
 def fd_poll_status(ctx: Context, stream=None) -> None:

@@ -72,6 +72,19 @@ def replica_seed(rep: Replica, seed: int) -> int:
     return seed + 17 * rep.rank
 
 
+def place_requests(rep: Replica, costs, load=None):
+    """Which replica serves which incoming request: each request is one monotask without a home and goes, in
+    arrival order, to the replica the least-maximum-load rule picks (Sec. 4.3; for such a task that is the least
+    loaded replica).  Every rank evaluates the same rule on the same numbers, so no exchange is needed.
+    Returns (replica of every request [n] int32, loads after placement [world] float64)."""
+    import numpy as np
+    from .binding import fd_sched_pack
+    load = np.zeros(rep.world, np.float64) if load is None else np.array(load, np.float64)
+    costs = np.asarray(costs, np.float64)
+    where = fd_sched_pack(load, costs, np.full(costs.size, -1, np.int32))
+    return where, load
+
+
 def job_throughput(units_all_ranks: float, slowest_ms: float) -> float:
     """Whole-job rate: units processed by all replicas divided by the slowest replica's time."""
     return units_all_ranks / (slowest_ms * 1e-3)

@@ -58,7 +58,12 @@ def _replica_worker(rank, world, port, out):
     replicas.barrier(rep)
     slow = replicas.max_over_ranks(rep, 10.0 + 5.0 * rank)
     units = replicas.sum_over_ranks(rep, 100.0 * (rank + 1))
-    out[rank] = (slow, units, replicas.replica_seed(rep, 1000), rep.is_lead)
+    # request placement: both ranks derive the same assignment without talking to each other
+    costs = [900, 300, 300, 500, 100, 700]
+    where, load = replicas.place_requests(rep, costs)
+    mine = float(sum(c for c, g in zip(costs, where) if g == rank))
+    placed = replicas.sum_over_ranks(rep, mine)
+    out[rank] = (slow, units, replicas.replica_seed(rep, 1000), rep.is_lead, where.tolist(), load.tolist(), placed)
     replicas.barrier(rep)
     replicas.shutdown(rep)
 
@@ -73,6 +78,9 @@ def test_replicas_over_gloo_world_size_two():
     assert res[0][1] == res[1][1] == 300.0                # units of all replicas
     assert res[0][2] != res[1][2]                         # each replica draws its own requests
     assert res[0][3] and not res[1][3]
+    assert res[0][4] == res[1][4] == [0, 1, 1, 1, 0, 0]    # 900 | 300 300 500 | then 100, 700 to the lighter side
+    assert res[0][5] == res[1][5] == [1700.0, 1100.0]
+    assert res[0][6] == 2800.0                            # every request is served exactly once
     assert replicas.job_throughput(300.0, 15.0) == pytest.approx(20000.0)
 
 
