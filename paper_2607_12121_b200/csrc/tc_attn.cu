@@ -275,8 +275,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const int s = g % STAGES;
                     if (!mbar_wait(&k_full[s], (g / STAGES) & 1, abort_flag)) { ok = false; break; }
                     // the score buffer is free once the softmax has finished the tile that used it last
-                    if (g >= 2 && !mbar_wait(&p_full[(g & 1) * 2], ((g - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
-                    if (SPLIT && g >= 2 && !mbar_wait(&p_full[(g & 1) * 2 + 1], ((g - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if (g >= 2 && !mbar_wait(&p_full[(g & 1) * 2 + (SPLIT ? 1 : 0)], ((g - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d = tmem_base + COL_S + (g & 1) * 128;
                     const uint32_t k_addr = smem_u32(sK + s * TILE_BYTES);
@@ -310,20 +309,17 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (j == 0 && item_i > 0 && !mbar_wait(o_free, (item_i - 1) & 1, abort_flag)) { ok = false; break; }
                     const uint32_t v_addr = smem_u32(sV + s * TILE_BYTES);
                     if constexpr (SPLIT) {
-                        // keys 0..63 of the tile feed O_0, keys 64..127 feed O_1, each as soon as its P half is there
-                        for (int hh = 0; hh < 2 && ok; ++hh) {
-                            if (!mbar_wait(&p_full[(g & 1) * 2 + hh], (g >> 1) & 1, abort_flag)) { ok = false; break; }
-                            tc_fence_after();
-                            const uint32_t d = tmem_base + COL_O + hh * 64;
-                            const uint32_t a = tmem_base + COL_P + (g & 1) * 64 + hh * 32;
+                        // the tiles of one parity accumulate into their own O: even tiles O_0, odd tiles O_1
+                        if (!mbar_wait(&p_full[(g & 1) * 2], (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t d = tmem_base + COL_O + (g & 1) * 64;
+                        const uint32_t a = tmem_base + COL_P + (g & 1) * 64;
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks)
-                                mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + (hh * 4 + ks) * 2048, SUB_BYTES, 1024, SWZ_128B),
-                                            idesc_pv, (j | ks) != 0);
-                            mma_commit(&pv_done[(g & 1) * 2 + hh]);
-                        }
-                        if (!ok) break;
+                        for (int ks = 0; ks < KEYS / 16; ++ks)
+                            mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
+                                        j >= 2 || ks != 0);
                         mma_commit(&v_empty[s]);
+                        mma_commit(&pv_done[(g & 1) * 2]);
                         continue;
                     }
                     if (!mbar_wait(&p_full[(g & 1) * 2], (g >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -352,15 +348,22 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // ---------------------------------------------------------------- softmax
         if constexpr (SPLIT) reg_inc<184>(); else reg_inc<200>();
         if constexpr (SPLIT) {
+            // Warpgroup `par` owns the key tiles of its parity (by the CTA-wide tile counter) with their score buffer,
+            // P buffer and accumulator O_par: one thread per query row, all 128 keys of the tile.  The two warpgroups
+            // never wait for each other, so on every scheduler one warp's exponentials overlap the other's loads,
+            // maxima, conversions and barrier hand-offs.
             const int quad = warp & 3;
-            const int half = wg - 1;                              // which 64 keys of every tile, and which accumulator
+            const int par = wg - 1;
             const int r = quad * 32 + lane;                       // query row inside the tile
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-            const uint32_t o_addr = lane_addr + COL_O + half * 64;
+            const uint32_t o_addr = lane_addr + COL_O + par * 64;
+            const uint32_t s_addr = lane_addr + COL_S + par * 128;
+            const uint32_t p_addr = lane_addr + COL_P + par * 64;
             uint32_t g0 = 0;
             bool ok = true;
             int item_i = 0;
             const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
+            const uint64_t sc2 = pair(scale_log2, scale_log2);
             for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
                 float m = -INFINITY, l = 0.f;
                 // MASS: the part of l that comes from keys carrying the query's own region label
@@ -372,119 +375,114 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (r < t.rows) my_lab = ma.labels[ma.active_idx[t.row0 + r]];
                     key_lab = ma.labels + (size_t)t.b * N;
                 }
-                auto tile = [&](const int j) -> bool {
-                    const uint32_t g = g0 + j, bs = g & 1;
-                    if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) return false;
+                for (int j = ((g0 & 1) == (uint32_t)par ? 0 : 1); j < n_kv && ok; j += 2) {
+                    const uint32_t g = g0 + j;
+                    if (!mbar_wait(&s_full[par], (g >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    uint32_t sr[64];
-                    tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64, sr);
-                    tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + 32, sr + 32);
-                    tmem_wait_ld();
-                    int kl0 = -2, kl1 = -2;                      // MASS: labels of this half's keys lane, lane + 32
-                    if constexpr (MASS) {
-                        const int k0 = j * KEYS + half * 64 + lane;
-                        if (k0 < N) kl0 = __ldg(key_lab + k0);
-                        if (k0 + 32 < N) kl1 = __ldg(key_lab + k0 + 32);
-                    }
                     const bool tail = j == n_kv - 1 && rem < KEYS;
+                    const bool first = j < 2;                    // this warpgroup's first tile of the item
+                    uint32_t sr[128];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sr + c * 32);
+                    tmem_wait_ld();
+                    // the scores are in registers: the buffer can take this warpgroup's next tile already
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&p_full[par * 2 + 1]);
                     if (tail) {
 #pragma unroll
-                        for (int i = 0; i < 64; ++i) if (half * 64 + i >= rem) sr[i] = 0xff800000u;      // -inf
+                        for (int i = 0; i < 128; ++i) if (i >= rem) sr[i] = 0xff800000u;          // -inf
                     }
                     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                    for (int i = 0; i < 64; i += 4) {
+                    for (int i = 0; i < 128; i += 4) {
                         mx0 = fmaxf(mx0, __uint_as_float(sr[i]));
                         mx1 = fmaxf(mx1, __uint_as_float(sr[i + 1]));
                         mx2 = fmaxf(mx2, __uint_as_float(sr[i + 2]));
                         mx3 = fmaxf(mx3, __uint_as_float(sr[i + 3]));
                     }
                     const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                    // a half with no valid key in the last tile keeps its state (mx = -inf, every p = 0);
-                    // both conditions below are the same for all rows of the warp
-                    const bool no_keys = tail && half * 64 >= rem;
-                    if (j == 0) {
+                    // the P buffer is free, and O_par complete, once the product of this warpgroup's previous tile is done
+                    if (g >= 2 && !mbar_wait(&pv_done[par * 2], ((g >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                    if (first) {
                         m = mx;
-                    } else if (!no_keys) {
+                    } else {
                         const bool need = (mx - m) * scale_log2 > RESCALE_LOG2;
                         if (__any_sync(0xffffffffu, need)) {
-                            // this half's earlier P V products must have landed before O_h is rescaled
-                            if (!mbar_wait(&pv_done[((g - 1) & 1) * 2 + half], ((g - 1) >> 1) & 1, abort_flag)) return false;
                             tc_fence_after();
                             const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
-                            if (need) { l *= f; m = mx; own *= f; }
-#pragma unroll
-                            for (int c = 0; c < 2; ++c) {
-                                uint32_t orr[32];
-                                tmem_ld32(o_addr + c * 32, orr);
+                            if (need) { l *= f; own *= f; m = mx; }
+#pragma unroll 1
+                            for (int c = 0; c < 8; ++c) {        // rare, and 128 scores are live: small pieces
+                                uint32_t orr[8];
+                                tmem_ld8(o_addr + c * 8, orr);
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
-                                tmem_st32(o_addr + c * 32, orr);
+                                for (int i = 0; i < 8; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
+                                tmem_st8(o_addr + c * 8, orr);
                             }
                             tmem_wait_st();
                         }
                     }
-                    const float mb = (m == -INFINITY ? 0.f : m) * scale_log2;
-                    uint32_t pk[32];
-                    // of every 8 exponentials 6 go to the special-function unit and 2 to the FMA pipe: the special-
-                    // function unit alone (16 results per clock and SM) would take longer than the tile's products
-                    const uint64_t sc2 = pair(scale_log2, scale_log2), nmb2 = pair(-mb, -mb);
+                    const float mb = m * scale_log2;
+                    const uint64_t nmb2 = pair(-mb, -mb);
                     uint64_t sua = pair(0.f, 0.f), sub_ = pair(0.f, 0.f);
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        float p[8];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const uint64_t x = fma2(pair(__uint_as_float(sr[2 * i + 2 * e]), __uint_as_float(sr[2 * i + 2 * e + 1])), sc2, nmb2);
-                            if (MASS || e < 3) {                 // MASS: no polynomial share, the body must stay small
-                                float xa, xb;
-                                unpair(x, xa, xb);
-                                p[2 * e] = ex2(xa);
-                                p[2 * e + 1] = ex2(xb);
-                            } else {
-                                unpair(ex2_poly2(x), p[2 * e], p[2 * e + 1]);
-                            }
-                        }
-                        sua = add2(sua, add2(pair(p[0], p[1]), pair(p[2], p[3])));
-                        sub_ = add2(sub_, add2(pair(p[4], p[5]), pair(p[6], p[7])));
+                    for (int c = 0; c < 4; ++c) {
+                        int kl = -2;                             // MASS: label of key `lane` of this chunk
                         if constexpr (MASS) {
-                            // the 8 keys of this group: positions 2 i .. 2 i + 7 of this half; their labels sit in lanes
-                            // (2 i + e) % 32 of kl0 / kl1 (a key past N has p = 0 and the label -2)
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                const int kk = 2 * i + e;
-                                const int kl = __shfl_sync(0xffffffffu, kk < 32 ? kl0 : kl1, kk & 31);
-                                own += kl == my_lab ? p[e] : 0.f;
-                            }
+                            const int k0 = j * KEYS + c * 32 + lane;
+                            if (k0 < N) kl = __ldg(key_lab + k0);
                         }
+                        uint32_t pk[16];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) pk[i + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
+                        for (int i = 0; i < 16; i += 4) {
+                            float p[8];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const uint64_t x = fma2(pair(__uint_as_float(sr[c * 32 + 2 * i + 2 * e]),
+                                                             __uint_as_float(sr[c * 32 + 2 * i + 2 * e + 1])), sc2, nmb2);
+                                if (MASS || e < 3) {             // MASS: no polynomial share, the body must stay small
+                                    float xa, xb;
+                                    unpair(x, xa, xb);
+                                    p[2 * e] = ex2(xa);
+                                    p[2 * e + 1] = ex2(xb);
+                                } else {
+                                    unpair(ex2_poly2(x), p[2 * e], p[2 * e + 1]);
+                                }
+                            }
+                            sua = add2(sua, add2(pair(p[0], p[1]), pair(p[2], p[3])));
+                            sub_ = add2(sub_, add2(pair(p[4], p[5]), pair(p[6], p[7])));
+                            if constexpr (MASS) {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    const int klk = __shfl_sync(0xffffffffu, kl, 2 * i + e);
+                                    own += klk == my_lab ? p[e] : 0.f;
+                                }
+                            }
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) pk[i + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
+                        }
+                        tmem_st16(p_addr + c * 16, pk);
                     }
                     {
                         float s0, s1;
                         unpair(add2(sua, sub_), s0, s1);
                         l += s0 + s1;
                     }
-                    // this half of the P buffer is free once the product that read it two tiles ago has completed
-                    if (g >= 2 && !mbar_wait(&pv_done[bs * 2 + half], ((g >> 1) - 1) & 1, abort_flag)) return false;
-                    tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pk);
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&p_full[bs * 2 + half]);
-                    return true;
-                };
-                for (int j = 0; j < n_kv; ++j)
-                    if (!tile(j)) { ok = false; break; }
+                    if (lane == 0) mbar_arrive(&p_full[par * 2]);
+                }
                 if (!ok) break;
-                // hand the row's statistics of this half to the epilogue warps and go on with the next item;
-                // the slot was last used two items ago
+                // hand the row's statistics of this warpgroup's tiles to the epilogue warps and go on with the next
+                // item; the slot was last used two items ago.  No tile at all (one-tile items): m = -inf, l = 0.
                 const int slot = item_i & 1;
                 if (item_i >= 2 && !mbar_wait(&stat_free[slot], ((item_i >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
-                s_xmax[(slot * 2 + half) * 128 + r] = m;
-                s_xsum[(slot * 2 + half) * 128 + r] = l;
-                if constexpr (MASS) s_xown[(slot * 2 + half) * 128 + r] = own;
+                s_xmax[(slot * 2 + par) * 128 + r] = m;
+                s_xsum[(slot * 2 + par) * 128 + r] = l;
+                if constexpr (MASS) s_xown[(slot * 2 + par) * 128 + r] = own;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&stat_full[slot]);
                 g0 += n_kv;
@@ -711,12 +709,11 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if constexpr (MASS) { own0 = s_xown[(slot * 2 + 0) * 128 + r]; own1 = s_xown[(slot * 2 + 1) * 128 + r]; }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&stat_free[slot]);
-                // every product of the item must have landed: the last tile, both halves
+                // every product of the item must have landed: they complete in issue order, so the last tile's does it
                 const uint32_t ge = g0 + n_kv - 1;
                 if (!mbar_wait(&pv_done[(ge & 1) * 2], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
-                if (!mbar_wait(&pv_done[(ge & 1) * 2 + 1], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const float m_all = fmaxf(m0, m1);                // half 0 always has a valid key, so this is finite
+                const float m_all = fmaxf(m0, m1);                // finite: at least one of the two had a tile
                 const float a0 = m0 == -INFINITY ? 0.f : ex2((m0 - m_all) * scale_log2);
                 const float a1 = m1 == -INFINITY ? 0.f : ex2((m1 - m_all) * scale_log2);
                 const float inv = 1.0f / (a0 * l0 + a1 * l1);
