@@ -2,22 +2,23 @@
 // of active tokens, previous-step rows of skipped tokens; paper Sec. 5 and Appendix A.6).
 //
 // One work item = one query tile (up to 128 compact rows of one request) x one head.  Persistent,
-// warp-specialised CTAs walk the device-built work list:
+// warp-specialised CTAs of four warpgroups walk the device-built work list:
 //   warp 0       TMA producer: Q tile (double buffered across items), K and V tiles (128 keys) in rings
 //   warp 1       issues S = Q K^T (tcgen05.mma, both operands in shared memory) into one of two TMEM
-//                score buffers as soon as the softmax has consumed that buffer's previous tile
+//                score buffers as soon as the softmax has handed that buffer back
 //   warp 2       issues O += P V with P read from TMEM and V as an N-major shared-memory operand
-//   warps 3..10  softmax, two threads per query row (each takes 64 of the 128 keys of a tile):
-//                tcgen05.ld of the scores, row maximum swapped through shared memory, running maximum
-//                with lazy rescaling of O (only when it grew by more than 2^8), exp2, P written to
-//                TMEM as packed bf16; at the end O / l is stored as bf16
-// At head dim 64 there is room in TMEM for two output accumulators, and the two threads of a row do
-// not talk to each other inside the key loop at all: thread h keeps its own running maximum and row
-// sum over "its" 64 keys of every tile, its P half feeds a product into its own accumulator O_h, and
-// the halves drift out of phase so that one warp's exp2 phase overlaps the other's TMEM traffic.  The
-// partial results are merged at the end, O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1), a_h = 2^(m_h - m).
-// The two MMA issuers run independently, so waiting for the softmax of tile g never delays the
-// score product of tile g+1.  Keys past N in the last tile are zero-filled by TMA and masked.
+//   warps 4..11  softmax: tcgen05.ld of the scores, running maximum with lazy rescaling of O (only
+//                when it grew by more than 2^24), exp2, P written to TMEM as packed bf16
+//   warps 12..15 head dim 64: item epilogue (merge, normalise, store) while the softmax warps go on
+// Head dims 128 and 72 (run as 80): one accumulator; two threads per query row, each with 64 of a
+// tile's 128 keys, swap their partial maxima through shared memory and end the item themselves.
+// Head dim 64: TMEM has room for two accumulators, so warpgroup p takes the key tiles of parity p
+// with its own score buffer, P buffer, accumulator O_p and running maximum / row sum: one thread per
+// row copies the tile's 128 scores to registers and hands the score buffer back at once, so that the
+// next S = Q K^T of its parity runs under this tile's exponentials; the two warpgroups never wait
+// for each other.  The partial results are merged at the end of the item by the epilogue warpgroup,
+// O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1), a_p = 2^(m_p - m).
+// Keys past N in the last tile are zero-filled by TMA and masked.
 #include <cuda_bf16.h>
 
 #include "ptx.cuh"
@@ -155,8 +156,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint64_t* v_full = k_empty + STAGES;
     uint64_t* v_empty = v_full + STAGES;
     uint64_t* s_full = v_empty + STAGES;      // [2]  score tile ready
-    uint64_t* p_full = s_full + 2;            // [2][2]  P written (and the score buffer consumed); [buffer][half], half 1 only if SPLIT
-    uint64_t* pv_done = p_full + 4;           // [2][2]  the product that read this P buffer (half) has completed
+    uint64_t* p_full = s_full + 2;            // [2][2]  [buffer][0]: P written; [buffer][1] (head dim 64): the buffer's scores are in registers
+    uint64_t* pv_done = p_full + 4;           // [2][2]  [buffer][0]: the product that read this P buffer has completed
     uint64_t* q_full = pv_done + 4;           // [2]
     uint64_t* q_empty = q_full + 2;           // [2]
     uint64_t* o_free = q_empty + 2;
