@@ -81,3 +81,60 @@ def form_batch(priority: Sequence[int], arrival: Sequence[int], active_tokens: S
         chosen[i] = 1
         left -= t
     return chosen, np.asarray(res, np.uint8)
+
+
+# ---------------------------------------------------------------------------------------------
+# Adaptive patch granularity (Sec. 4.1, "Adaptive Patch Granularity")
+# ---------------------------------------------------------------------------------------------
+# The paper: performance as a function of the number of patches R is unimodal, and R is tuned online by a
+# bounded binary search on observed performance -- while a larger R improves performance the search keeps
+# refining, when performance degrades it comes back.  Reading (the paper gives no more than that): a search
+# state (accepted R with its observed performance, a direction, a step).  The first observation belongs to
+# the starting R.  Every later observation belongs to the candidate proposed last: better than the accepted
+# one -> the candidate becomes the accepted R and the search continues in the same direction with the same
+# step; not better -> the direction flips and the step halves (never below 1).  A candidate is the accepted
+# R plus direction * step, clamped to [r_min, r_max]; a candidate equal to the accepted R counts as "not
+# better" without being run.  Two failures in a row at step 1 (both neighbours are no better) end the
+# search: the accepted R is returned from then on.  The initial step is half the range, rounded up.
+class RSearch:
+    def __init__(self, r_min: int, r_max: int, r_start: int):
+        assert r_min <= r_start <= r_max
+        self.r_min, self.r_max = int(r_min), int(r_max)
+        self.accepted = int(r_start)
+        self.candidate = int(r_start)
+        self.step = max(1, (self.r_max - self.r_min + 1) // 2)
+        self.dir = 1
+        self.ref = None
+        self.fails_at_one = 0
+        self.converged = self.r_min == self.r_max
+
+    def _propose(self) -> int:
+        while not self.converged:
+            c = min(self.r_max, max(self.r_min, self.accepted + self.dir * self.step))
+            if c != self.accepted:
+                self.candidate = c
+                return c
+            self._fail()                                  # clamped onto the accepted R: nothing to run
+        self.candidate = self.accepted
+        return self.accepted
+
+    def _fail(self):
+        if self.step == 1:
+            self.fails_at_one += 1
+            if self.fails_at_one >= 2:
+                self.converged = True
+        self.dir = -self.dir
+        self.step = max(1, self.step // 2)
+
+    def update(self, perf: float) -> int:
+        """Reports the performance (higher is better) observed with the R returned last; returns the next R."""
+        if self.converged:
+            return self.accepted
+        if self.ref is None:
+            self.ref = float(perf)
+        elif float(perf) > self.ref:
+            self.accepted, self.ref = self.candidate, float(perf)
+            self.fails_at_one = 0
+        else:
+            self._fail()
+        return self._propose()

@@ -135,3 +135,50 @@ def test_form_batch_is_the_lexicographic_maximum_over_feasible_sets():
         assert int(tok[chosen.astype(bool)].sum()) <= budget
         assert int(res_after.sum()) <= max(max_res, int(res.sum()))
         assert np.array_equal(res_after, res | (chosen & (1 - res)).astype(res.dtype))
+
+
+def _run_search(f, lo, hi, start, limit=200):
+    s = sch.RSearch(lo, hi, start)
+    r, evals = start, 0
+    while not s.converged and evals < limit:
+        r = s.update(f(r))
+        evals += 1
+    return s.accepted, evals
+
+
+def test_rsearch_finds_the_peak_of_every_small_unimodal_profile():
+    """Brute force: every strictly unimodal profile on ranges up to 9 values (all peak positions, random slopes),
+    every starting point: the search ends on the arg max within a bounded number of observations."""
+    g = np.random.default_rng(7)
+    for n in range(1, 10):
+        for peak in range(n):
+            for trial in range(6):
+                up = np.sort(g.random(peak))
+                down = np.sort(g.random(n - peak - 1))[::-1]
+                prof = np.concatenate([up, [2.0], down]) + np.arange(n) * 0          # strictly unimodal, peak value 2
+                for start in range(n):
+                    got, evals = _run_search(lambda r: prof[r - 4], 4, 4 + n - 1, 4 + start)
+                    assert got == 4 + peak, (prof, start)
+                    assert evals <= 4 * int(np.ceil(np.log2(n + 1))) + 6
+
+
+def test_rsearch_is_logarithmic_on_large_ranges_and_hand_example():
+    for lo, hi in ((1, 64), (2, 257), (8, 1024)):
+        for peak in (lo, hi, (lo + hi) // 2, lo + 5, hi - 3):
+            f = lambda r: -abs(r - peak)
+            for start in (lo, hi, (lo + 3 * hi) // 4):
+                got, evals = _run_search(f, lo, hi, start, limit=500)
+                assert got == peak
+                assert evals <= 4 * int(np.ceil(np.log2(hi - lo + 1))) + 6
+    # hand-worked: range 1..16, start 4, peak at 11, f = -|r - 11|; initial step 8
+    s = sch.RSearch(1, 16, 4)
+    seq = [4]
+    while not s.converged:
+        seq.append(s.update(-abs(seq[-1] - 11)))
+    # 4 (ref -7) -> 12 (-1, accepted) -> 16 (clamped 20; -5 worse: flip, step 4) -> 8 (-3 worse: flip, step 2)
+    # -> 14 (-3 worse: flip, step 1) -> 11 (0, accepted) -> 10 (worse: flip, 1st failure at step 1) -> 12 (worse: 2nd) -> stop
+    assert seq == [4, 12, 16, 8, 14, 11, 10, 12, 11]
+    assert s.accepted == 11
+    # a single admissible value needs no search
+    s = sch.RSearch(5, 5, 5)
+    assert s.converged and s.update(1.0) == 5
