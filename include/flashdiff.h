@@ -315,6 +315,29 @@ fd_status fd_sched_pack(int n_devices, double* load, int n_tasks, const double* 
 fd_status fd_sched_form_batch(int n, const int32_t* priority, const int64_t* arrival, const int32_t* active_tokens,
                               uint8_t* resident, int64_t token_budget, int max_resident, uint8_t* chosen_out);
 
+/*
+ * Adaptive patch granularity (Sec. 4.1): performance as a function of the number of patches R is unimodal, and R is
+ * tuned online by a bounded binary search on the performance observed for past requests.  Pure host code; the state
+ * is a plain struct owned by the caller (HOST memory).
+ *   fd_rsearch_init    R in [r_min, r_max], first R to run = r_start; initial step = half the range, rounded up.
+ *   fd_rsearch_update  observed_perf (higher is better) belongs to the R returned last (the first call: to r_start).
+ *                      Better than the accepted R's -> the candidate becomes the accepted R, same direction and step;
+ *                      not better -> the direction flips and the step halves (never below 1).  The next candidate is
+ *                      accepted + direction * step clamped to the range; one that equals the accepted R counts as not
+ *                      better without being run.  Two failures in a row at step 1 end the search (converged = 1): the
+ *                      accepted R is returned from then on.  *next_r receives the R to run next.
+ * Errors: FD_ERR_INVALID_ARG for null pointers, r_min < 1, r_min > r_max, r_start outside the range, a NaN performance.
+ */
+typedef struct {
+    int32_t r_min, r_max;
+    int32_t accepted, candidate; /* accepted R and the one being evaluated */
+    int32_t step, dir;           /* dir = +1 / -1 */
+    int32_t have_ref, fails_at_one, converged;
+    double ref_perf;             /* performance observed with the accepted R */
+} fd_rsearch;
+fd_status fd_rsearch_init(fd_rsearch* st, int r_min, int r_max, int r_start);
+fd_status fd_rsearch_update(fd_rsearch* st, double observed_perf, int32_t* next_r);
+
 /* Releases the context (host memory only; the workspace goes back to the caller). */
 fd_status fd_destroy(fd_ctx* ctx);
 

@@ -4,5 +4,5 @@ The product is the C-ABI shared library built from ``csrc/``; this package is it
 Python binding.  There is no CPU or PyTorch fallback: importing fails if the library is absent.
 """
 from .binding import *  # noqa: F401,F403
-from .binding import (lib, Context, FdConfig, FdWeights, FdSamplerWeights, FlashDiffError, make_config,  # noqa: F401
+from .binding import (lib, Context, FdConfig, FdWeights, FdSamplerWeights, FdRSearch, FlashDiffError, make_config,  # noqa: F401
                       make_sampler_weights, EXPORTS, LIB_PATH)

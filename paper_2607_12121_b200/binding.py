@@ -23,7 +23,7 @@ EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region
            "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
            "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait",
            "fd_embed_latent", "fd_update_latent", "fd_regional_step_mass", "fd_region_activity_attn",
-           "fd_sched_pack", "fd_sched_form_batch"]
+           "fd_sched_pack", "fd_sched_form_batch", "fd_rsearch_init", "fd_rsearch_update"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
                "gemm_fc2", "partition", "sampler"]
@@ -43,6 +43,11 @@ class FdWeights(ctypes.Structure):
 
 class FdSamplerWeights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("w_in", "b_in", "pos", "w_out", "b_out")] + [("latent_dim", ctypes.c_int32)]
+
+
+class FdRSearch(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("r_min", "r_max", "accepted", "candidate", "step", "dir", "have_ref",
+                                              "fails_at_one", "converged")] + [("ref_perf", ctypes.c_double)]
 
 
 class FlashDiffError(RuntimeError):
@@ -86,6 +91,10 @@ def _load() -> ctypes.CDLL:
     lib.fd_sched_pack.argtypes = [i32, vp, i32, vp, vp, vp]
     lib.fd_sched_form_batch.restype = i32
     lib.fd_sched_form_batch.argtypes = [i32, vp, vp, vp, vp, ctypes.c_int64, i32, vp]
+    lib.fd_rsearch_init.restype = i32
+    lib.fd_rsearch_init.argtypes = [ctypes.POINTER(FdRSearch), i32, i32, i32]
+    lib.fd_rsearch_update.restype = i32
+    lib.fd_rsearch_update.argtypes = [ctypes.POINTER(FdRSearch), ctypes.c_double, ctypes.POINTER(ctypes.c_int32)]
     lib.fd_embed_latent.restype = i32
     lib.fd_embed_latent.argtypes = [vp, ctypes.POINTER(FdSamplerWeights), vp, i32, i32, vp, vp]
     lib.fd_update_latent.restype = i32
@@ -278,6 +287,24 @@ def fd_sched_form_batch(priority, arrival, active_tokens, resident, token_budget
     if st != FD_OK:
         raise FlashDiffError(st, "fd_sched_form_batch: invalid argument")
     return chosen
+
+
+def fd_rsearch_init(r_min: int, r_max: int, r_start: int) -> FdRSearch:
+    """State of the adaptive patch-granularity search (Sec. 4.1); the first R to run is ``r_start``."""
+    st = FdRSearch()
+    rc = lib.fd_rsearch_init(ctypes.byref(st), int(r_min), int(r_max), int(r_start))
+    if rc != FD_OK:
+        raise FlashDiffError(rc, "fd_rsearch_init: invalid argument")
+    return st
+
+
+def fd_rsearch_update(st: FdRSearch, observed_perf: float) -> int:
+    """Reports the performance observed with the R returned last; returns the R to run next."""
+    nxt = ctypes.c_int32()
+    rc = lib.fd_rsearch_update(ctypes.byref(st), float(observed_perf), ctypes.byref(nxt))
+    if rc != FD_OK:
+        raise FlashDiffError(rc, "fd_rsearch_update: invalid argument")
+    return int(nxt.value)
 
 
 def fd_poll_status(ctx: Context, stream=None) -> None:

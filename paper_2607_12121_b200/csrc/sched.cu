@@ -1,4 +1,5 @@
-// Host-side batch former (Sec. 4.3: patch monotasks, least-maximum-load packing).  No device code.
+// Host-side policies of the paper's scheduler: the batch former (Sec. 4.3: patch monotasks, least-maximum-load
+// packing) and the adaptive patch-granularity search (Sec. 4.1).  No device code.
 #include <cmath>
 #include <cstdint>
 
@@ -74,6 +75,56 @@ fd_status fd_sched_form_batch(int n, const int32_t* priority, const int64_t* arr
         chosen_out[i] = take ? 1 : 0;
         if (take) left -= t;
     }
+    return FD_OK;
+}
+
+// ---- adaptive patch granularity (Sec. 4.1) ----------------------------------------------------
+
+static void rsearch_fail(fd_rsearch* st) {
+    if (st->step == 1 && ++st->fails_at_one >= 2) st->converged = 1;
+    st->dir = -st->dir;
+    st->step = st->step / 2 > 1 ? st->step / 2 : 1;
+}
+
+fd_status fd_rsearch_init(fd_rsearch* st, int r_min, int r_max, int r_start) {
+    if (!st || r_min < 1 || r_min > r_max || r_start < r_min || r_start > r_max) return FD_ERR_INVALID_ARG;
+    st->r_min = r_min;
+    st->r_max = r_max;
+    st->accepted = st->candidate = r_start;
+    const int half = (r_max - r_min + 1) / 2;
+    st->step = half > 1 ? half : 1;
+    st->dir = 1;
+    st->have_ref = 0;
+    st->fails_at_one = 0;
+    st->converged = r_min == r_max;
+    st->ref_perf = 0.0;
+    return FD_OK;
+}
+
+fd_status fd_rsearch_update(fd_rsearch* st, double observed_perf, int32_t* next_r) {
+    if (!st || !next_r || observed_perf != observed_perf) return FD_ERR_INVALID_ARG;
+    if (!st->converged) {
+        if (!st->have_ref) {
+            st->have_ref = 1;
+            st->ref_perf = observed_perf;
+        } else if (observed_perf > st->ref_perf) {
+            st->accepted = st->candidate;
+            st->ref_perf = observed_perf;
+            st->fails_at_one = 0;
+        } else {
+            rsearch_fail(st);
+        }
+        // next candidate; one that is clamped onto the accepted R is a failure that costs no run
+        while (!st->converged) {
+            int64_t c = (int64_t)st->accepted + (int64_t)st->dir * st->step;
+            if (c < st->r_min) c = st->r_min;
+            if (c > st->r_max) c = st->r_max;
+            if ((int32_t)c != st->accepted) { st->candidate = (int32_t)c; break; }
+            rsearch_fail(st);
+        }
+    }
+    if (st->converged) st->candidate = st->accepted;
+    *next_r = st->candidate;
     return FD_OK;
 }
 

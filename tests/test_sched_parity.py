@@ -97,3 +97,43 @@ def test_batch_former_drives_a_step_mask():
     step_mask = gate * chosen[:, None]
     assert (sizes * step_mask).sum() <= tok.sum() // 2
     assert chosen.any() and not chosen.all()
+
+
+def test_rsearch_matches_oracle_step_by_step():
+    g = np.random.default_rng(21)
+    for _ in range(300):
+        lo = int(g.integers(1, 20))
+        hi = lo + int(g.integers(0, 200))
+        start = int(g.integers(lo, hi + 1))
+        kind = int(g.integers(0, 3))
+        peak = int(g.integers(lo, hi + 1))
+        noise = g.random(hi - lo + 1) * (0.0 if kind == 0 else 3.0)           # kind 0: unimodal; else: noisy profiles
+        flat = kind == 2                                                      # plateaus: ties count as "not better"
+        f = lambda r: (-(abs(r - peak) // 4) if flat else -abs(r - peak)) + noise[r - lo]
+        ref = sch.RSearch(lo, hi, start)
+        st = fd.fd_rsearch_init(lo, hi, start)
+        r = start
+        for it in range(400):
+            want = ref.update(f(r))
+            got = fd.fd_rsearch_update(st, f(r))
+            assert got == want, (lo, hi, start, it)
+            assert (st.accepted, st.step, st.dir, bool(st.converged)) == (ref.accepted, ref.step, ref.dir, ref.converged)
+            r = got
+            if ref.converged:
+                break
+        assert ref.converged
+        if kind == 0:
+            assert st.accepted == peak
+
+
+def test_rsearch_invalid_arguments():
+    with pytest.raises(fd.FlashDiffError):
+        fd.fd_rsearch_init(0, 8, 4)
+    with pytest.raises(fd.FlashDiffError):
+        fd.fd_rsearch_init(4, 3, 4)
+    with pytest.raises(fd.FlashDiffError):
+        fd.fd_rsearch_init(2, 8, 9)
+    st = fd.fd_rsearch_init(2, 8, 4)
+    with pytest.raises(fd.FlashDiffError):
+        fd.fd_rsearch_update(st, float("nan"))
+    assert st.accepted == 4 and not st.have_ref
