@@ -283,8 +283,8 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
 
 // The same with the row held in registers (NV float4 slots per lane, H = 128 NV): every load of a row is in
 // flight at once and the row is read a single time.
-template <typename T, int NV>
-__global__ void __launch_bounds__(LN_THREADS, 4)
+template <typename T, int NV, bool GATHER>
+__global__ void __launch_bounds__(LN_THREADS, 6)
 ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
                        float* __restrict__ resid_out, T* __restrict__ out, const int32_t* __restrict__ active_idx,
                        const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
@@ -295,43 +295,67 @@ ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__
     const int a_total = ctl->a_total;
     for (int row = blockIdx.x * (LN_THREADS / 32) + warp; row < a_total; row += gridDim.x * (LN_THREADS / 32)) {
         const int tok = active_idx[row];
-        const int b = tok / N;
-        const size_t g0 = (size_t)tok * H, r0 = (size_t)row * H;
+        // one base pointer per stream and constant offsets: every lane's i-th vector is 32 vectors further
         float v[NV][4];
+        if constexpr (GATHER) {
+            const T* src = x_gather + (size_t)tok * H + lane * 4;
 #pragma unroll
-        for (int i = 0; i < NV; ++i) ln_load4<T>(x_gather, resid_in, g0 + (i * 32 + lane) * 4, r0 + (i * 32 + lane) * 4, v[i]);
-        float sum = 0.f;
+            for (int i = 0; i < NV; ++i) ln_load4<T>(src, nullptr, i * 128, 0, v[i]);
+            if (resid_out) {
+                float4* keep = reinterpret_cast<float4*>(resid_out + (size_t)row * H) + lane;
 #pragma unroll
-        for (int i = 0; i < NV; ++i) sum += (v[i][0] + v[i][1]) + (v[i][2] + v[i][3]);
-        const float mean = warp_sum(sum) / (float)H;
-        float sq = 0.f;
+                for (int i = 0; i < NV; ++i) keep[i * 32] = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
+            }
+        } else {
+            const float4* src = reinterpret_cast<const float4*>(resid_in + (size_t)row * H) + lane;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const float4 u = src[i * 32];
+                v[i][0] = u.x; v[i][1] = u.y; v[i][2] = u.z; v[i][3] = u.w;
+            }
+        }
+        // one pass, shifted by the row's first element (keeps the cancellation in sq - sum^2 harmless); four
+        // independent accumulator pairs and the two reductions side by side keep the dependent chains short
+        const float x0 = __shfl_sync(0xffffffffu, v[0][0], 0);
+        float su[4] = {0.f, 0.f, 0.f, 0.f}, sq4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int i = 0; i < NV; ++i)
 #pragma unroll
-            for (int k = 0; k < 4; ++k) { const float d = v[i][k] - mean; sq = fmaf(d, d, sq); }
-        const float rstd = rsqrtf(warp_sum(sq) / (float)H + ln_eps);
-        const float* sh = shift + (size_t)b * mod_stride;
-        const float* sc = scale + (size_t)b * mod_stride;
+            for (int k = 0; k < 4; ++k) {
+                const float d = v[i][k] - x0;
+                su[k] += d;
+                sq4[k] = fmaf(d, d, sq4[k]);
+            }
+        float sum = (su[0] + su[1]) + (su[2] + su[3]);
+        float sq = (sq4[0] + sq4[1]) + (sq4[2] + sq4[3]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        }
+        const float dm = sum / (float)H;                       // mean - x0
+        const float rstd = rsqrtf(fmaxf(sq / (float)H - dm * dm, 0.f) + ln_eps);
+        const float mean = x0 + dm;
+        const int b = tok / N;
+        const float4* sc4 = reinterpret_cast<const float4*>(scale + (size_t)b * mod_stride) + lane;
+        const float4* sh4 = reinterpret_cast<const float4*>(shift + (size_t)b * mod_stride) + lane;
+        T* dst = out + (size_t)row * H + lane * 4;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
-            const int c = (i * 32 + lane) * 4;
-            if (x_gather && resid_out)
-                *reinterpret_cast<float4*>(resid_out + r0 + c) = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
-            const float4 s4 = __ldg(reinterpret_cast<const float4*>(sc + c));
-            const float4 h4 = __ldg(reinterpret_cast<const float4*>(sh + c));
+            const float4 s4 = __ldg(sc4 + i * 32);
+            const float4 h4 = __ldg(sh4 + i * 32);
             const float o0 = (v[i][0] - mean) * rstd * (1.f + s4.x) + h4.x;
             const float o1 = (v[i][1] - mean) * rstd * (1.f + s4.y) + h4.y;
             const float o2 = (v[i][2] - mean) * rstd * (1.f + s4.z) + h4.z;
             const float o3 = (v[i][3] - mean) * rstd * (1.f + s4.w) + h4.w;
-            T* dst = out + r0 + c;
             if constexpr (sizeof(T) == 2) {
                 const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
                 uint2 u;
                 u.x = *reinterpret_cast<const uint32_t*>(&p0);
                 u.y = *reinterpret_cast<const uint32_t*>(&p1);
-                *reinterpret_cast<uint2*>(dst) = u;
+                *reinterpret_cast<uint2*>(dst + i * 128) = u;
             } else {
-                *reinterpret_cast<float4*>(dst) = make_float4(o0, o1, o2, o3);
+                *reinterpret_cast<float4*>(dst + i * 128) = make_float4(o0, o1, o2, o3);
             }
         }
     }
@@ -409,9 +433,11 @@ cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* 
     const int grid = max(1, min((rows_cap + rows_per_cta - 1) / rows_per_cta, 148 * 16));
 #define FD_LN_REG(NV)                                                                                              \
     if (H == NV * 128) {                                                                                           \
-        cudaError_t e = ptx::launch_kernel(ln_modulate_reg_kernel<T, NV>, grid, LN_THREADS, 0, st, pdl, x_gather,  \
-                                           resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N,      \
-                                           ln_eps, ctl);                                                           \
+        cudaError_t e = x_gather                                                                                    \
+            ? ptx::launch_kernel(ln_modulate_reg_kernel<T, NV, true>, grid, LN_THREADS, 0, st, pdl, x_gather,      \
+                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl)   \
+            : ptx::launch_kernel(ln_modulate_reg_kernel<T, NV, false>, grid, LN_THREADS, 0, st, pdl, x_gather,     \
+                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl);  \
         ++*n_launch;                                                                                               \
         return e;                                                                                                  \
     }
