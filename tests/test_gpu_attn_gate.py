@@ -25,9 +25,14 @@ def _step_mass(ctx, wl, x, cond, labels, mask, buf, mass):
 
 @pytest.mark.parametrize("name,engine", [("tiny", fd.FD_ENGINE_SIMT), ("audio_small", fd.FD_ENGINE_SIMT),
                                          ("mmdit_small", fd.FD_ENGINE_SIMT), ("audio_tc", fd.FD_ENGINE_TC),
-                                         ("image_tc", fd.FD_ENGINE_TC), ("wide_tc", fd.FD_ENGINE_TC)])
-def test_region_mass_matches_oracle(name, engine):
-    wl = gen.workload(name)
+                                         ("image_tc", fd.FD_ENGINE_TC), ("wide_tc", fd.FD_ENGINE_TC),
+                                         ("mmdit_tc", fd.FD_ENGINE_TC), ("audio_tc_few_ctas", fd.FD_ENGINE_TC)])
+def test_region_mass_matches_oracle(monkeypatch, name, engine):
+    if name.endswith("_few_ctas"):        # several items per CTA, odd key-tile count: the tile parity an item starts on alternates
+        monkeypatch.setenv("FD_TC_MAX_CTAS", "2")
+        wl = gen.workload(name[:-len("_few_ctas")]).replace(grid=(330,), R=10)
+    else:
+        wl = gen.workload(name)
     labels = labels_for(wl, 4)
     w = gen.block_weights(wl, 4)
     w["w_qkv"][:, :wl.H] *= np.float32(4.0)                      # sharper attention: the mass differs from region to region
@@ -50,7 +55,7 @@ def test_region_mass_matches_oracle(name, engine):
         assert np.all(got[~ran] == 0.0)                          # regions that did not run report nothing
         tol = 2e-2 if wl.dtype == "bf16" else 1e-4               # bf16 Q / K rounding moves softmax probabilities by ~1 %
         np.testing.assert_allclose(got[ran], ref[ran], rtol=tol, atol=1e-6)
-    assert ref[ran].std() / ref[ran].mean() > 0.01               # the signal is not trivially uniform
+    assert ref[ran].std() / ref[ran].mean() > 0.005              # the signal is not trivially uniform
 
 
 def test_attention_gate_matches_oracle_over_steps():

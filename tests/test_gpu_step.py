@@ -138,12 +138,14 @@ def test_small_twins_tensor_core_engine(name):
 
 
 @pytest.mark.parametrize("name,n_tok", [("audio_tc", None), ("audio_tc", 130), ("audio_tc", 100), ("image_tc", None),
-                                        ("wide_tc", None)])
+                                        ("wide_tc", None), ("mmdit_tc", None), ("audio_tc", 520)])
 def test_tensor_core_engine_few_ctas_walk_many_tiles(monkeypatch, name, n_tok):
     """Two persistent CTAs process every tile: the shared-memory rings and both TMEM accumulator
     stages wrap around many times, and every attention CTA runs many items back to back (with four, two
     and one key tiles per item: the hand-over of an item's statistics and accumulators to the epilogue
-    warps, and of the score / P buffers between items, at every key-loop length)."""
+    warps, and of the score / P buffers between items, at every key-loop length).  Three and five key tiles per
+    item: at head dim 64 the softmax warpgroups own the tiles of one parity of the CTA-wide tile counter, so the
+    parity an item starts on alternates from item to item."""
     monkeypatch.setenv("FD_TC_MAX_CTAS", "2")
     wl = gen.workload(name)
     if n_tok is not None:
