@@ -12,12 +12,13 @@
 //   warps 12..15 head dim 64: item epilogue (merge, normalise, store) while the softmax warps go on
 // Head dims 128 and 72 (run as 80): one accumulator; two threads per query row, each with 64 of a
 // tile's 128 keys, swap their partial maxima through shared memory and end the item themselves.
-// Head dim 64: TMEM has room for two accumulators, so warpgroup p takes the key tiles of parity p
-// with its own score buffer, P buffer, accumulator O_p and running maximum / row sum: one thread per
-// row copies the tile's 128 scores to registers and hands the score buffer back at once, so that the
-// next S = Q K^T of its parity runs under this tile's exponentials; the two warpgroups never wait
-// for each other.  The partial results are merged at the end of the item by the epilogue warpgroup,
-// O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1), a_p = 2^(m_p - m).
+// Head dim 64: warpgroup p takes the key tiles of parity p with its own P buffer, accumulator O_p
+// and running maximum / row sum: one thread per row copies the tile's 128 scores to registers and
+// hands the (single) score buffer back at once, so that the next S = Q K^T runs under this tile's
+// exponentials; the two warpgroups never wait for each other.  TMEM then has room for four
+// accumulators (item parity x tile parity): the next item's products start while the epilogue
+// warpgroup still merges this item's partial results, O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1),
+// a_p = 2^(m_p - m).
 // Keys past N in the last tile are zero-filled by TMA and masked.
 #include <cuda_bf16.h>
 
@@ -124,6 +125,8 @@ constexpr float RESCALE_LOG2 = 24.0f;
 
 // TMEM columns: two score buffers, the output accumulator, two P buffers (bf16 pairs)
 constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384, TMEM_COLS = 512;
+// head dim 64: one score buffer, two P buffers (tile parity), four accumulators (item parity x tile parity)
+constexpr uint32_t COL64_S = 0, COL64_P = 128, COL64_O = 256;
 
 // What the MASS variant (head dim 64, launched for a step's first block when asked) needs on top: per region, the
 // softmax mass its active queries put on keys of their own region (paper Sec. 4.2).
@@ -161,11 +164,12 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint64_t* q_full = pv_done + 4;           // [2]
     uint64_t* q_empty = q_full + 2;           // [2]
     uint64_t* o_free = q_empty + 2;
-    uint64_t* x_bar = o_free + 1;             // [4 quadrants][2]: the two threads of a row swap their partial maxima
+    uint64_t* x_bar = o_free + 2;             // [4 quadrants][2]: the two threads of a row swap their partial maxima
     uint64_t* l_bar = x_bar + 8;              // [4 quadrants]: ... and, once per item, their partial sums
     uint64_t* stat_full = l_bar + 4;          // [2]  head dim 64: an item's row statistics are in shared memory
     uint64_t* stat_free = stat_full + 2;      // [2]  ... and have been read
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(stat_free + 2);
+    uint64_t* item_done = stat_free + 2;      // [2]  head dim 64: every product of an item (by item parity) has completed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(item_done + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* s_xmax = reinterpret_cast<float*>(tmem_slot + 2);      // head dim 64: row maxima, [2 items][2 halves][128 rows]
     float* s_xsum = s_xmax + 512;                                 // [2 halves][128 rows]; head dim 64: [2 items][2 halves][128 rows]
@@ -192,8 +196,9 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         for (int i = 0; i < 4; ++i) { mbar_init(&p_full[i], SPLIT ? 4 : 8); mbar_init(&pv_done[i], 1); }
         for (int i = 0; i < 8; ++i) mbar_init(&x_bar[i], 64);
         for (int i = 0; i < 4; ++i) mbar_init(&l_bar[i], 64);
-        mbar_init(o_free, SPLIT ? 4 : 8);
-        for (int i = 0; i < 2; ++i) { mbar_init(&stat_full[i], 8); mbar_init(&stat_free[i], 4); }
+        mbar_init(&o_free[0], SPLIT ? 4 : 8);
+        mbar_init(&o_free[1], SPLIT ? 4 : 8);
+        for (int i = 0; i < 2; ++i) { mbar_init(&stat_full[i], 8); mbar_init(&stat_free[i], 4); mbar_init(&item_done[i], 1); }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tm_q);
@@ -281,9 +286,14 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const int s = g % STAGES;
                     if (!mbar_wait(&k_full[s], (g / STAGES) & 1, abort_flag)) { ok = false; break; }
                     // the score buffer is free once the softmax has finished the tile that used it last
-                    if (g >= 2 && !mbar_wait(&p_full[(g & 1) * 2 + (SPLIT ? 1 : 0)], ((g - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if constexpr (SPLIT) {
+                        // one score buffer: free once the previous tile's scores are in its warpgroup's registers
+                        if (g >= 1 && !mbar_wait(&p_full[((g - 1) & 1) * 2 + 1], ((g - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                    } else {
+                        if (g >= 2 && !mbar_wait(&p_full[(g & 1) * 2], ((g - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+                    }
                     tc_fence_after();
-                    const uint32_t d = tmem_base + COL_S + (g & 1) * 128;
+                    const uint32_t d = tmem_base + (SPLIT ? COL64_S : COL_S + (g & 1) * 128);
                     const uint32_t k_addr = smem_u32(sK + s * TILE_BYTES);
 #pragma unroll
                     for (int ks = 0; ks < Cfg::SUBS * 4; ++ks) {
@@ -312,20 +322,28 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int j = 0; j < n_kv; ++j, ++g) {
                     const int s = g % STAGES;
                     if (!mbar_wait(&v_full[s], (g / STAGES) & 1, abort_flag)) { ok = false; break; }
-                    if (j == 0 && item_i > 0 && !mbar_wait(o_free, (item_i - 1) & 1, abort_flag)) { ok = false; break; }
+                    if constexpr (SPLIT) {
+                        // the accumulators alternate from item to item: these were last used two items ago
+                        if (j == 0 && item_i >= 2 && !mbar_wait(&o_free[item_i & 1], ((item_i >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                    } else {
+                        if (j == 0 && item_i > 0 && !mbar_wait(&o_free[0], (item_i - 1) & 1, abort_flag)) { ok = false; break; }
+                    }
                     const uint32_t v_addr = smem_u32(sV + s * TILE_BYTES);
                     if constexpr (SPLIT) {
                         // the tiles of one parity accumulate into their own O: even tiles O_0, odd tiles O_1
                         if (!mbar_wait(&p_full[(g & 1) * 2], (g >> 1) & 1, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t d = tmem_base + COL_O + (g & 1) * 64;
-                        const uint32_t a = tmem_base + COL_P + (g & 1) * 64;
+                        const uint32_t d = tmem_base + COL64_O + ((item_i & 1) * 2 + (g & 1)) * 64;
+                        const uint32_t a = tmem_base + COL64_P + (g & 1) * 64;
 #pragma unroll
                         for (int ks = 0; ks < KEYS / 16; ++ks)
                             mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
                                         j >= 2 || ks != 0);
                         mma_commit(&v_empty[s]);
                         mma_commit(&pv_done[(g & 1) * 2]);
+                        // the item's products complete in issue order: this one covers them all.  (Its own barrier: the
+                        // per-tile ones run on into the next item and their parity would alias for a late epilogue.)
+                        if (j == n_kv - 1) mma_commit(&item_done[item_i & 1]);
                         continue;
                     }
                     if (!mbar_wait(&p_full[(g & 1) * 2], (g >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -362,9 +380,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int par = wg - 1;
             const int r = quad * 32 + lane;                       // query row inside the tile
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-            const uint32_t o_addr = lane_addr + COL_O + par * 64;
-            const uint32_t s_addr = lane_addr + COL_S + par * 128;
-            const uint32_t p_addr = lane_addr + COL_P + par * 64;
+            const uint32_t s_addr = lane_addr + COL64_S;
+            const uint32_t p_addr = lane_addr + COL64_P + par * 64;
             uint32_t g0 = 0;
             bool ok = true;
             int item_i = 0;
@@ -372,6 +389,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const uint64_t sc2 = pair(scale_log2, scale_log2);
             for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
                 float m = -INFINITY, l = 0.f;
+                const uint32_t o_addr = lane_addr + COL64_O + ((item_i & 1) * 2 + par) * 64;
                 // MASS: the part of l that comes from keys carrying the query's own region label
                 float own = 0.f;
                 int my_lab = -1;
@@ -682,7 +700,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(o_free);
+                if (lane == 0) mbar_arrive(&o_free[0]);
                 g0 += n_kv;
             }
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 600 + (int)blockIdx.x);
@@ -698,7 +716,6 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
             // staging rows are 144 bytes apart so that the 16-byte stores of a quarter warp fall into different banks
             uint8_t* wstage = s_stage + quad * 32 * 144;
-            uint32_t g0 = 0;
             bool ok = true;
             int item_i = 0;
             QTile t_next = blockIdx.x < n_items ? tiles[blockIdx.x % n_tiles] : QTile{0, 0, 0, 0};
@@ -714,9 +731,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if constexpr (MASS) { own0 = s_xown[(slot * 2 + 0) * 128 + r]; own1 = s_xown[(slot * 2 + 1) * 128 + r]; }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&stat_free[slot]);
-                // every product of the item must have landed: they complete in issue order, so the last tile's does it
-                const uint32_t ge = g0 + n_kv - 1;
-                if (!mbar_wait(&pv_done[(ge & 1) * 2], (ge >> 1) & 1, abort_flag)) { ok = false; break; }
+                // every product of the item must have landed
+                if (!mbar_wait(&item_done[slot], (item_i >> 1) & 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const float m_all = fmaxf(m0, m1);                // finite: at least one of the two had a tile
                 const float a0 = m0 == -INFINITY ? 0.f : ex2((m0 - m_all) * scale_log2);
@@ -741,14 +757,14 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll 1
                 for (int q = 0; q < 8; ++q) {
                     uint32_t o0[8], o1[8];
-                    tmem_ld8(lane_addr + COL_O + q * 8, o0);
-                    tmem_ld8(lane_addr + COL_O + 64 + q * 8, o1);
+                    tmem_ld8(lane_addr + COL64_O + slot * 128 + q * 8, o0);
+                    tmem_ld8(lane_addr + COL64_O + slot * 128 + 64 + q * 8, o1);
                     tmem_wait_ld();
                     if (q == 7) {
                         // the accumulators are free for the next item as soon as they are in registers
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(o_free);
+                        if (lane == 0) mbar_arrive(&o_free[slot]);
                     }
                     float v[8];
 #pragma unroll
@@ -775,7 +791,6 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (quad * 32 + rr < t.rows) *reinterpret_cast<uint4*>(obase + (size_t)rr * o_ld) = u;
                 }
                 __syncwarp();                                     // the staging rows are rewritten by the next item
-                g0 += n_kv;
             }
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 700 + (int)blockIdx.x);
         }
