@@ -25,7 +25,7 @@ thread_local std::string g_create_error;
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-    size_t control, acc_ss, acc_cnt, block_counts, tiles, ada_act, mod, resid, act, q, o, g, part, total;
+    size_t control, acc_ss, acc_cnt, block_counts, tiles, ada_act, mod, resid, act, q, o, g, part, attn_ws, total;
     int Mcap, q_ld, tile_cap;
 };
 
@@ -71,6 +71,7 @@ Layout make_layout(const fd_config& c) {
     l.o = take((size_t)l.Mcap * c.hidden * es);
     l.g = take((size_t)l.Mcap * c.mlp_dim * es);
     l.part = take(partition_scratch_bytes(c.max_batch, c.max_tokens, c.max_regions));
+    l.attn_ws = take(c.dtype == FD_BF16 && tc_attention_supported(c) ? tc_attention_scratch_bytes(c.head_dim) : 0);
     l.total = off;
     return l;
 }
@@ -303,6 +304,8 @@ fd_status fd_create(const fd_config* cfg, const fd_weights* weights, void* works
         tb.act = c->ws + lay.act; tb.q = c->ws + lay.q; tb.o = c->ws + lay.o; tb.g = c->ws + lay.g;
         tb.Mcap = lay.Mcap; tb.q_ld = lay.q_ld;
         tb.resid = c->ws + lay.resid;
+        tb.attn_ws = c->ws + lay.attn_ws;
+        tb.attn_slots = TC_ATTENTION_SLOTS;
         std::string tc_err;
         c->tc = tc_plan_create(*cfg, *weights, tb, &tc_err);
         if (!c->tc) {

@@ -14,6 +14,8 @@ struct TcBuffers {  // compact activation buffers inside the workspace (bf16)
     void *act, *q, *o, *g;
     void* resid;    // fp32 residual stream [Mcap, hidden]
     int Mcap, q_ld;
+    void* attn_ws;  // scratch of the attention kernel: one slot per CTA for the pieces of cut items (may be null)
+    int attn_slots;
 };
 
 enum TcGemmKind { TC_GEMM_QKV = 0, TC_GEMM_OUT = 1, TC_GEMM_FC1 = 2, TC_GEMM_FC2 = 3 };
@@ -23,6 +25,8 @@ bool tc_attention_supported(const fd_config& cfg);
 int tc_attention_tile_rows();
 bool tc_plan_pdl(TcPlan* p);                // kernels of the step are launched with programmatic stream serialization
 int tc_attention_head_pad(int head_dim);   // head dim as stored in the padded Q buffer
+constexpr int TC_ATTENTION_SLOTS = 256;    // CTAs the attention scratch has room for
+size_t tc_attention_scratch_bytes(int head_dim);
 TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffers& buf, std::string* err);
 void tc_plan_destroy(TcPlan* p);
 cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,

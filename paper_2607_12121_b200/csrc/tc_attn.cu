@@ -20,6 +20,8 @@
 // warpgroup still merges this item's partial results, O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1),
 // a_p = 2^(m_p - m).
 // Keys past N in the last tile are zero-filled by TMA and masked.
+// For long key sequences the items of the last, partly filled round are cut along the keys (CutPlan below) and
+// attn_combine_kernel puts their pieces together.
 #include <cuda_bf16.h>
 
 #include "ptx.cuh"
@@ -138,12 +140,45 @@ struct MassArgs {
     float inv_heads;
 };
 
+// Work of one CTA.  Item blockIdx.x + k * gridDim.x in round k, as long as whole rounds last.  The items left over
+// for a last, partly filled round are cut along the key sequence into `parts` pieces of `steps` key tiles so that
+// (nearly) all CTAs take part in that round too; a piece leaves its un-normalised accumulator and row statistics
+// in the CTA's scratch slot and a small kernel launched behind this one puts the pieces of an item together.
+struct CutPlan { int n_rounds, n_tail, parts, steps; };
+__host__ __device__ inline CutPlan cut_plan(int n_items, int n_kv, int grid, bool may_cut) {
+    CutPlan c;
+    c.n_rounds = n_items / grid;
+    c.n_tail = n_items - c.n_rounds * grid;
+    c.parts = 1;
+    c.steps = n_kv;
+    if (may_cut && c.n_tail > 0) {
+        const int s_max = (grid / c.n_tail) < n_kv ? (grid / c.n_tail) : n_kv;
+        if (s_max >= 2) {
+            c.steps = (n_kv + s_max - 1) / s_max;
+            c.parts = (n_kv + c.steps - 1) / c.steps;
+        }
+    }
+    return c;
+}
+struct Task { int w, j0, j1, piece; };      // piece: 1 = a cut item's piece (result goes to the scratch slot)
+__device__ __forceinline__ bool next_task(const CutPlan& c, int n_kv, int k, Task& t) {
+    if (k < c.n_rounds) { t = Task{(int)blockIdx.x + k * (int)gridDim.x, 0, n_kv, 0}; return true; }
+    if (k > c.n_rounds || (int)blockIdx.x >= c.n_tail * c.parts) return false;
+    const int ti = (int)blockIdx.x / c.parts, pt = (int)blockIdx.x - ti * c.parts;
+    const int j0 = pt * c.steps, j1 = j0 + c.steps < n_kv ? j0 + c.steps : n_kv;
+    t = Task{c.n_rounds * (int)gridDim.x + ti, j0, j1, c.parts > 1 ? 1 : 0};
+    return true;
+}
+// scratch slot of a CTA: [128 rows][DP + 4] floats: the un-normalised output row, then running maximum, row sum,
+// own-region mass
+__host__ __device__ inline size_t split_slot_floats(int dp) { return (size_t)128 * (dp + 4); }
+
 template <int D, bool MASS = false>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
                     const __grid_constant__ CUtensorMap tm_q_tail, const __grid_constant__ CUtensorMap tm_kv_tail,
                     __nv_bfloat16* __restrict__ o, int o_ld, const QTile* __restrict__ tiles, int heads, int N,
-                    float scale_log2, Control* ctl, MassArgs ma) {
+                    float scale_log2, float* __restrict__ split_ws, Control* ctl, MassArgs ma) {
     using Cfg = AttCfg<D>;
     constexpr int DP = Cfg::DP;
     constexpr bool SPLIT = D == 64;                      // per-half accumulators, no exchange in the key loop
@@ -220,6 +255,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // so that head's K/V stays in L2 however long the key sequence is
     const int n_tiles = ctl->n_qtiles;
     const int n_items = n_tiles * heads;
+    const CutPlan cut = cut_plan(n_items, n_kv, (int)gridDim.x, split_ws != nullptr);
 
     if (wg == 0) {
     reg_dec<48>();
@@ -229,7 +265,9 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             uint32_t gk = 0;
             bool ok = true;
             int item_i = 0;
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
+            Task tk;
+            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+                const int w = tk.w;
                 const QTile t = tiles[w % n_tiles];
                 const int head = w / n_tiles;
                 const int qs = item_i & 1;
@@ -240,7 +278,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tma_load_2d(sQ + qs * TILE_BYTES + sb * SUB_BYTES, &tm_q, head * DP + sb * 64, t.row0, &q_full[qs]);
                 if constexpr (D == 72)
                     tma_load_2d(sQ + qs * TILE_BYTES + SUB_BYTES, &tm_q_tail, head * DP + 64, t.row0, &q_full[qs]);
-                for (int j = 0; j < n_kv; ++j, ++gk) {
+                for (int j = tk.j0; j < tk.j1; ++j, ++gk) {
                     const int s = gk % STAGES;
                     const uint32_t ph = ((gk / STAGES) & 1) ^ 1;
                     if (!mbar_wait(&k_empty[s], ph, abort_flag)) { ok = false; break; }
@@ -278,11 +316,13 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             uint32_t g = 0;
             bool ok = true;
             int item_i = 0;
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
+            Task tk;
+            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+                const int w = tk.w;
                 const int qs = item_i & 1;
                 if (!mbar_wait(&q_full[qs], (item_i >> 1) & 1, abort_flag)) { ok = false; break; }
                 const uint32_t q_addr = smem_u32(sQ + qs * TILE_BYTES);
-                for (int j = 0; j < n_kv; ++j, ++g) {
+                for (int j = tk.j0; j < tk.j1; ++j, ++g) {
                     const int s = g % STAGES;
                     if (!mbar_wait(&k_full[s], (g / STAGES) & 1, abort_flag)) { ok = false; break; }
                     // the score buffer is free once the softmax has finished the tile that used it last
@@ -306,7 +346,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                     smem_desc(k_addr + SUB_BYTES, 16, 256, SWZ_32B), idesc_qk, 1);
                     mma_commit(&k_empty[s]);
                     mma_commit(&s_full[g & 1]);
-                    if (j == n_kv - 1) mma_commit(&q_empty[qs]);
+                    if (j == tk.j1 - 1) mma_commit(&q_empty[qs]);
                 }
             }
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 500 + (int)blockIdx.x);
@@ -318,15 +358,17 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             uint32_t g = 0;
             bool ok = true;
             int item_i = 0;
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
-                for (int j = 0; j < n_kv; ++j, ++g) {
+            Task tk;
+            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+                const int w = tk.w;
+                for (int j = tk.j0; j < tk.j1; ++j, ++g) {
                     const int s = g % STAGES;
                     if (!mbar_wait(&v_full[s], (g / STAGES) & 1, abort_flag)) { ok = false; break; }
                     if constexpr (SPLIT) {
                         // the accumulators alternate from item to item: these were last used two items ago
-                        if (j == 0 && item_i >= 2 && !mbar_wait(&o_free[item_i & 1], ((item_i >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                        if (j == tk.j0 && item_i >= 2 && !mbar_wait(&o_free[item_i & 1], ((item_i >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
                     } else {
-                        if (j == 0 && item_i > 0 && !mbar_wait(&o_free[0], (item_i - 1) & 1, abort_flag)) { ok = false; break; }
+                        if (j == tk.j0 && item_i > 0 && !mbar_wait(&o_free[0], (item_i - 1) & 1, abort_flag)) { ok = false; break; }
                     }
                     const uint32_t v_addr = smem_u32(sV + s * TILE_BYTES);
                     if constexpr (SPLIT) {
@@ -338,12 +380,12 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int ks = 0; ks < KEYS / 16; ++ks)
                             mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
-                                        j >= 2 || ks != 0);
+                                        j - tk.j0 >= 2 || ks != 0);
                         mma_commit(&v_empty[s]);
                         mma_commit(&pv_done[(g & 1) * 2]);
                         // the item's products complete in issue order: this one covers them all.  (Its own barrier: the
                         // per-tile ones run on into the next item and their parity would alias for a late epilogue.)
-                        if (j == n_kv - 1) mma_commit(&item_done[item_i & 1]);
+                        if (j == tk.j1 - 1) mma_commit(&item_done[item_i & 1]);
                         continue;
                     }
                     if (!mbar_wait(&p_full[(g & 1) * 2], (g >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -355,11 +397,11 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         if constexpr (D == 72)
                             // 16 keys further: two 8-key groups of 256 bytes; the 16-column blocks sit TAIL_BYTES apart
                             mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 512, TAIL_BYTES, 256, SWZ_32B), idesc_pv,
-                                        (j | ks) != 0);
+                                        (j != tk.j0 || ks != 0));
                         else
                             // 16 keys further: 16 rows of 128 bytes; the second 64-wide half of V sits SUB_BYTES away
                             mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
-                                        (j | ks) != 0);
+                                        (j != tk.j0 || ks != 0));
                     }
                     mma_commit(&v_empty[s]);
                     mma_commit(&pv_done[(g & 1) * 2]);
@@ -387,7 +429,9 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             int item_i = 0;
             const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
             const uint64_t sc2 = pair(scale_log2, scale_log2);
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
+            Task tk;
+            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+                const int w = tk.w;
                 float m = -INFINITY, l = 0.f;
                 const uint32_t o_addr = lane_addr + COL64_O + ((item_i & 1) * 2 + par) * 64;
                 // MASS: the part of l that comes from keys carrying the query's own region label
@@ -399,12 +443,12 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (r < t.rows) my_lab = ma.labels[ma.active_idx[t.row0 + r]];
                     key_lab = ma.labels + (size_t)t.b * N;
                 }
-                for (int j = ((g0 & 1) == (uint32_t)par ? 0 : 1); j < n_kv && ok; j += 2) {
-                    const uint32_t g = g0 + j;
+                for (int j = tk.j0 + ((g0 & 1) == (uint32_t)par ? 0 : 1); j < tk.j1 && ok; j += 2) {
+                    const uint32_t g = g0 + (j - tk.j0);
                     if (!mbar_wait(&s_full[par], (g >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const bool tail = j == n_kv - 1 && rem < KEYS;
-                    const bool first = j < 2;                    // this warpgroup's first tile of the item
+                    const bool first = j - tk.j0 < 2;            // this warpgroup's first tile of the item (or piece)
                     uint32_t sr[128];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sr + c * 32);
@@ -508,7 +552,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if constexpr (MASS) s_xown[(slot * 2 + par) * 128 + r] = own;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&stat_full[slot]);
-                g0 += n_kv;
+                g0 += tk.j1 - tk.j0;
             }
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 650 + (int)blockIdx.x);
         } else {
@@ -522,7 +566,9 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             bool ok = true;
             int item_i = 0;
             const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
+            Task tk;
+            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+                const int w = tk.w;
                 const QTile t = tiles[w % n_tiles];
                 const int head = w / n_tiles;
                 float m = -INFINITY, l = 0.f;
@@ -535,8 +581,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (my_lab >= ma.R) my_lab = -1;
                     key_lab = ma.labels + (size_t)t.b * N;
                 }
-                for (int j = 0; j < n_kv && ok; ++j) {
-                    const uint32_t g = g0 + j, bs = g & 1;
+                for (int j = tk.j0; j < tk.j1 && ok; ++j) {
+                    const uint32_t g = g0 + (j - tk.j0), bs = g & 1;
                     if (!mbar_wait(&s_full[bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     int kl0 = -2, kl1 = -2;                      // MASS: labels of this half's keys lane, lane + 32
@@ -567,7 +613,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     mbar_arrive(&x_bar[quad * 2 + bs]);
                     if (!mbar_wait(&x_bar[quad * 2 + bs], (g >> 1) & 1, abort_flag)) { ok = false; break; }
                     mx = fmaxf(mx, s_xmax[bs * 256 + (half ^ 1) * 128 + r]);
-                    if (j == 0) {
+                    if (j == tk.j0) {
                         m = mx;
                     } else {
                         const bool need = (mx - m) * scale_log2 > RESCALE_LOG2;
@@ -647,13 +693,21 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 if (!ok) break;
                 // epilogue: O / l for the rows of this tile (l = the two halves' partial sums)
-                const uint32_t gl = g0 + n_kv - 1;
+                const uint32_t gl = g0 + (tk.j1 - tk.j0) - 1;
                 s_xsum[half * 128 + r] = l;
                 if constexpr (MASS) s_xown[half * 128 + r] = own;
                 mbar_arrive(&l_bar[quad]);
                 if (!mbar_wait(&l_bar[quad], item_i & 1, abort_flag)) { ok = false; break; }
-                const float inv = 1.0f / (l + s_xsum[(half ^ 1) * 128 + r]);
-                if constexpr (MASS) {
+                // a cut item's piece stays un-normalised: its rows, maximum, sum (and mass) go to the CTA's scratch slot
+                const bool piece = tk.piece != 0;
+                const float inv = piece ? 1.0f : 1.0f / (l + s_xsum[(half ^ 1) * 128 + r]);
+                float* prow = split_ws + (size_t)blockIdx.x * split_slot_floats(DP) + (size_t)r * (DP + 4);
+                if (piece && half == 0) {
+                    prow[DP] = m;
+                    prow[DP + 1] = l + s_xsum[128 + r];
+                    if constexpr (MASS) prow[DP + 2] = own + s_xown[128 + r];
+                }
+                if (MASS && !piece) {
                     if (half == 0) {      // one of the row's two threads reports; the lanes of one label add up first
                         const float mine = my_lab >= 0 ? (own + s_xown[128 + r]) * inv * ma.inv_heads : 0.f;
                         const uint32_t peers = __match_any_sync(0xffffffffu, my_lab);
@@ -671,7 +725,13 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     uint32_t orr[32];
                     tmem_ld32(lane_addr + COL_O + half * DH + c * 32, orr);
                     tmem_wait_ld();
-                    if (r < t.rows) {
+                    if (piece) {
+    #pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            *reinterpret_cast<float4*>(prow + half * DH + c * 32 + v * 4) =
+                                make_float4(__uint_as_float(orr[4 * v]), __uint_as_float(orr[4 * v + 1]),
+                                            __uint_as_float(orr[4 * v + 2]), __uint_as_float(orr[4 * v + 3]));
+                    } else if (r < t.rows) {
     #pragma unroll
                         for (int v = 0; v < 4; ++v) {
                             uint4 u;
@@ -688,7 +748,12 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         uint32_t ot[8];
                         tmem_ld8(lane_addr + COL_O + 64, ot);
                         tmem_wait_ld();
-                        if (r < t.rows) {
+                        if (piece) {
+                            *reinterpret_cast<float4*>(prow + 64) = make_float4(__uint_as_float(ot[0]), __uint_as_float(ot[1]),
+                                                                                __uint_as_float(ot[2]), __uint_as_float(ot[3]));
+                            *reinterpret_cast<float4*>(prow + 68) = make_float4(__uint_as_float(ot[4]), __uint_as_float(ot[5]),
+                                                                                __uint_as_float(ot[6]), __uint_as_float(ot[7]));
+                        } else if (r < t.rows) {
                             uint4 u;
                             u.x = pack_bf16(__uint_as_float(ot[0]) * inv, __uint_as_float(ot[1]) * inv);
                             u.y = pack_bf16(__uint_as_float(ot[2]) * inv, __uint_as_float(ot[3]) * inv);
@@ -701,7 +766,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&o_free[0]);
-                g0 += n_kv;
+                g0 += tk.j1 - tk.j0;
             }
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 600 + (int)blockIdx.x);
         }
@@ -718,10 +783,10 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             uint8_t* wstage = s_stage + quad * 32 * 144;
             bool ok = true;
             int item_i = 0;
-            QTile t_next = blockIdx.x < n_items ? tiles[blockIdx.x % n_tiles] : QTile{0, 0, 0, 0};
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x, ++item_i) {
-                const QTile t = t_next;
-                if (w + (int)gridDim.x < n_items) t_next = tiles[(w + gridDim.x) % n_tiles];
+            Task tk;
+            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+                const int w = tk.w;
+                const QTile t = tiles[w % n_tiles];
                 const int head = w / n_tiles;
                 const int slot = item_i & 1;
                 if (!mbar_wait(&stat_full[slot], (item_i >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -737,9 +802,17 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const float m_all = fmaxf(m0, m1);                // finite: at least one of the two had a tile
                 const float a0 = m0 == -INFINITY ? 0.f : ex2((m0 - m_all) * scale_log2);
                 const float a1 = m1 == -INFINITY ? 0.f : ex2((m1 - m_all) * scale_log2);
-                const float inv = 1.0f / (a0 * l0 + a1 * l1);
+                // a cut item's piece stays un-normalised: its rows, maximum, sum (and mass) go to the CTA's scratch slot
+                const bool piece = tk.piece != 0;
+                const float inv = piece ? 1.0f : 1.0f / (a0 * l0 + a1 * l1);
                 const float w_0 = a0 * inv, w_1 = a1 * inv;       // weights of O_0, O_1
-                if constexpr (MASS) {
+                float* prow = split_ws + (size_t)blockIdx.x * split_slot_floats(DP) + (size_t)r * (DP + 4);
+                if (piece) {
+                    prow[DP] = m_all;
+                    prow[DP + 1] = a0 * l0 + a1 * l1;
+                    if constexpr (MASS) prow[DP + 2] = a0 * own0 + a1 * own1;
+                }
+                if (MASS && !piece) {
                     // consecutive compact rows mostly share their region: the lanes of one label add up first, so that a
                     // region receives one atomic per warp instead of one per row
                     int lab = -1;
@@ -774,6 +847,11 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
                         v[i] = x0 + x1;
                     }
+                    if (piece) {
+                        *reinterpret_cast<float4*>(prow + q * 8) = make_float4(v[0], v[1], v[2], v[3]);
+                        *reinterpret_cast<float4*>(prow + q * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                        continue;
+                    }
                     uint4 u;
                     u.x = pack_bf16(v[0], v[1]);
                     u.y = pack_bf16(v[2], v[3]);
@@ -781,6 +859,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     u.w = pack_bf16(v[6], v[7]);
                     *reinterpret_cast<uint4*>(wstage + lane * 144 + q * 16) = u;
                 }
+                if (piece) continue;
                 __syncwarp();
                 // eight neighbouring lanes write one row's 128 bytes: 4 lines per store instruction instead of 32
                 __nv_bfloat16* obase = o + (size_t)(t.row0 + quad * 32) * o_ld + head * D + (lane & 7) * 8;
@@ -804,10 +883,69 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 }
 
+// Puts the pieces of the cut items together: O = sum_p c_p O_p / sum_p c_p l_p with c_p = 2^((m_p - m) scale).
+// One CTA per cut item (att_grid = the grid the attention kernel ran with); a thread takes four neighbouring
+// columns of a row at a time, so that a row's threads read and write whole lines and every thread has several
+// independent loads in flight (the statistics of a row are re-read by its threads: L1 hits).
+constexpr int COMBINE_THREADS = 256;
+template <int D, bool MASS>
+__global__ void __launch_bounds__(COMBINE_THREADS)
+attn_combine_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o, int o_ld, const QTile* __restrict__ tiles,
+                    int heads, int N, int att_grid, float scale_log2, const Control* __restrict__ ctl, MassArgs ma) {
+    constexpr int DP = AttCfg<D>::DP;
+    constexpr int CG = D / 4;                          // column groups of a row
+    pdl_trigger();
+    pdl_wait();
+    const int n_tiles = ctl->n_qtiles;
+    const int n_items = n_tiles * heads;
+    const int n_kv = (N + KEYS - 1) / KEYS;
+    const CutPlan cut = cut_plan(n_items, n_kv, att_grid, true);
+    if (cut.parts < 2) return;
+    const size_t slot = split_slot_floats(DP);
+    for (int ti = blockIdx.x; ti < cut.n_tail; ti += gridDim.x) {
+        const int w = cut.n_rounds * att_grid + ti;
+        const QTile t = tiles[w % n_tiles];
+        const int head = w / n_tiles;
+        // blockIdx.y picks the work items: one per thread, so that a thread's two rounds of loads are all there is
+        for (int idx = blockIdx.y * COMBINE_THREADS + threadIdx.x; idx < t.rows * CG; idx += gridDim.y * COMBINE_THREADS) {
+            const int r = idx / CG, cg = idx - r * CG;
+            const float* base = ws + (size_t)ti * cut.parts * slot + (size_t)r * (DP + 4);
+            float m = -INFINITY;
+            for (int p = 0; p < cut.parts; ++p) m = fmaxf(m, base[p * slot + DP]);
+            float l = 0.f, own = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int p = 0; p < cut.parts; ++p) {
+                const float* row = base + p * slot;
+                const float c = ex2((row[DP] - m) * scale_log2);
+                const float4 x = *reinterpret_cast<const float4*>(row + cg * 4);
+                l = fmaf(c, row[DP + 1], l);
+                if constexpr (MASS) own = fmaf(c, row[DP + 2], own);
+                acc.x = fmaf(c, x.x, acc.x); acc.y = fmaf(c, x.y, acc.y);
+                acc.z = fmaf(c, x.z, acc.z); acc.w = fmaf(c, x.w, acc.w);
+            }
+            const float inv = 1.0f / l;
+            uint2 u;
+            u.x = pack_bf16(acc.x * inv, acc.y * inv);
+            u.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2*>(o + (size_t)(t.row0 + r) * o_ld + head * D + cg * 4) = u;
+            if constexpr (MASS) {
+                if (cg == 0) {
+                    const int lab = ma.labels[ma.active_idx[t.row0 + r]];
+                    if (lab >= 0 && lab < ma.R)
+                        atomicAdd(&ma.region_mass[(size_t)t.b * ma.R + lab], (double)(own * inv * ma.inv_heads));
+                }
+            }
+        }
+    }
+}
+
 struct AttnPlan {
     CUtensorMap q_map, q_tail_map;
     int heads, dh, dp, H, q_ld;
     void* o;
+    float* split_ws;        // one slot per CTA for the pieces of cut items (nullptr: items are never cut)
+    int split_slots;
+    int split_mode;
 };
 
 }  // namespace
@@ -817,6 +955,9 @@ bool tc_attention_supported(const fd_config& c) {
 }
 int tc_attention_tile_rows() { return QROWS; }
 int tc_attention_head_pad(int head_dim) { return head_dim == 72 ? 80 : head_dim; }
+size_t tc_attention_scratch_bytes(int head_dim) {
+    return (size_t)TC_ATTENTION_SLOTS * split_slot_floats(tc_attention_head_pad(head_dim)) * sizeof(float);
+}
 
 void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::string* err) {
     AttnPlan* a = new AttnPlan();
@@ -826,6 +967,10 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
     a->H = cfg.hidden;
     a->q_ld = buf.q_ld;
     a->o = buf.o;
+    a->split_ws = static_cast<float*>(buf.attn_ws);
+    a->split_slots = buf.attn_slots;
+    a->split_mode = 1;
+    if (const char* v = getenv("FD_ATT_SPLIT")) a->split_mode = atoi(v);
     const uint64_t dims[2] = {(uint64_t)buf.q_ld, (uint64_t)buf.Mcap};
     const uint64_t strides[1] = {(uint64_t)buf.q_ld * 2};
     const uint32_t box[2] = {64, QROWS};
@@ -874,22 +1019,36 @@ cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, c
     __nv_bfloat16* o = static_cast<__nv_bfloat16*>(a->o);
     MassArgs ma{labels, active_idx, region_mass, R, 1.0f / (float)a->heads};
     cudaError_t e = cudaSuccess;
-#define FD_ATT(DD)                                                                                                  \
-    e = launch_kernel(tc_attention_kernel<DD>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, tc_plan_pdl(p), a->q_map, kv_map, \
-                      a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c, ma)
-#define FD_ATT_MASS(DD)                                                                                             \
-    e = launch_kernel(tc_attention_kernel<DD, true>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, tc_plan_pdl(p), a->q_map, kv_map, \
-                      a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, c, ma)
+    // the items of the last, partly filled round are cut into pieces
+    // (switch FD_ATT_SPLIT, read when the context is created: 0 = never, 2 = at every length, for tests)
+    const int split_mode = a->split_mode;
+    const bool split_on = split_mode != 0;
+    // ... for long key sequences only: a piece pays an item's fixed costs (Q load, pipeline fill, hand-over) and the pieces
+    // need a second, small kernel; measured, that is a loss at 1024 and 2048 keys and a gain of 3-8 % from 4096 on
+    const bool long_keys = N >= 24 * KEYS || split_mode == 2;
+    float* split_ws = (split_on && long_keys && a->split_ws && grid <= a->split_slots) ? a->split_ws : nullptr;
+    const bool pdl = tc_plan_pdl(p);
+    const int cgrid = max(1, grid / 2);             // at most grid / 2 items can be cut
+#define FD_ATT(DD, MM)                                                                                              \
+    do {                                                                                                            \
+        e = launch_kernel(tc_attention_kernel<DD, MM>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, pdl, a->q_map, kv_map,   \
+                          a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, split_ws, c, ma);    \
+        ++*n_launch;                                                                                                \
+        if (e == cudaSuccess && split_ws) {                                                                         \
+            e = launch_kernel(attn_combine_kernel<DD, MM>, dim3(cgrid, (QROWS * (DD / 4) + COMBINE_THREADS - 1) / COMBINE_THREADS),  \
+                              COMBINE_THREADS, 0, st, pdl, (const float*)split_ws, o, a->H, tiles,                  \
+                              a->heads, N, grid, scale_log2, ctl, ma);                                              \
+            ++*n_launch;                                                                                            \
+        }                                                                                                           \
+    } while (0)
     if (region_mass) {
-        if (a->dh == 64) FD_ATT_MASS(64);
-        else if (a->dh == 128) FD_ATT_MASS(128);
-        else FD_ATT_MASS(72);
-    } else if (a->dh == 64) FD_ATT(64);
-#undef FD_ATT_MASS
-    else if (a->dh == 128) FD_ATT(128);
-    else FD_ATT(72);
+        if (a->dh == 64) FD_ATT(64, true);
+        else if (a->dh == 128) FD_ATT(128, true);
+        else FD_ATT(72, true);
+    } else if (a->dh == 64) FD_ATT(64, false);
+    else if (a->dh == 128) FD_ATT(128, false);
+    else FD_ATT(72, false);
 #undef FD_ATT
-    ++*n_launch;
     return e;
 }
 

@@ -26,9 +26,14 @@ def _step_mass(ctx, wl, x, cond, labels, mask, buf, mass):
 @pytest.mark.parametrize("name,engine", [("tiny", fd.FD_ENGINE_SIMT), ("audio_small", fd.FD_ENGINE_SIMT),
                                          ("mmdit_small", fd.FD_ENGINE_SIMT), ("audio_tc", fd.FD_ENGINE_TC),
                                          ("image_tc", fd.FD_ENGINE_TC), ("wide_tc", fd.FD_ENGINE_TC),
-                                         ("mmdit_tc", fd.FD_ENGINE_TC), ("audio_tc_few_ctas", fd.FD_ENGINE_TC)])
+                                         ("mmdit_tc", fd.FD_ENGINE_TC), ("audio_tc_few_ctas", fd.FD_ENGINE_TC),
+                                         ("audio_tc_cut", fd.FD_ENGINE_TC), ("image_tc_cut", fd.FD_ENGINE_TC),
+                                         ("wide_tc_cut", fd.FD_ENGINE_TC)])
 def test_region_mass_matches_oracle(monkeypatch, name, engine):
-    if name.endswith("_few_ctas"):        # several items per CTA, odd key-tile count: the tile parity an item starts on alternates
+    if name.endswith("_cut"):             # the attention items are cut along the keys and put together by a second kernel
+        monkeypatch.setenv("FD_ATT_SPLIT", "2")
+        wl = gen.workload(name[:-len("_cut")])
+    elif name.endswith("_few_ctas"):        # several items per CTA, odd key-tile count: the tile parity an item starts on alternates
         monkeypatch.setenv("FD_TC_MAX_CTAS", "2")
         wl = gen.workload(name[:-len("_few_ctas")]).replace(grid=(330,), R=10)
     else:

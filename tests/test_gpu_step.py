@@ -154,6 +154,27 @@ def test_tensor_core_engine_few_ctas_walk_many_tiles(monkeypatch, name, n_tok):
     _run_sequence(wl, 3, fd.FD_ENGINE_TC, masks)
 
 
+@pytest.mark.parametrize("name,n_tok,max_ctas", [("audio_tc", None, None), ("audio_tc", 700, "8"), ("mmdit_tc", None, "8"),
+                                                 ("image_tc", None, None), ("image_tc", 520, "8"), ("wide_tc", None, "8"),
+                                                 ("audio_tc", 100, None)])
+def test_attention_items_cut_along_the_keys(monkeypatch, name, n_tok, max_ctas):
+    """The items of the last, partly filled round of attention CTAs are cut into pieces along the key sequence (forced
+    here at every length; by default only long sequences are cut) and a second kernel puts the pieces together: with
+    all SMs (every item is cut: fewer items than CTAs) and with 8 CTAs (whole rounds first, then 2 to 8 pieces per
+    left-over item), pieces of one key tile (one softmax warpgroup idle at head dim 64) and of several."""
+    monkeypatch.setenv("FD_ATT_SPLIT", "2")
+    if max_ctas:
+        monkeypatch.setenv("FD_TC_MAX_CTAS", max_ctas)
+    wl = gen.workload(name)
+    if n_tok is not None:
+        wl = wl.replace(grid=(n_tok,), R=10, L=1)
+    masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.6] * wl.B)]
+    cut = _run_sequence(wl, 4, fd.FD_ENGINE_TC, masks).launches
+    monkeypatch.setenv("FD_ATT_SPLIT", "0")
+    whole = _run_sequence(wl, 4, fd.FD_ENGINE_TC, masks).launches
+    assert cut == whole + len(masks) * wl.L                     # the second kernel ran behind every attention launch
+
+
 @pytest.mark.parametrize("switch", ["FD_TMA_RESID", "FD_TC_PAIR", "FD_PDL"])
 def test_tensor_core_engine_switched_off_variants(monkeypatch, switch):
     """The library's switches select older forms of a kernel (per-thread residual reductions instead of the bulk
