@@ -161,7 +161,14 @@ __host__ __device__ inline CutPlan cut_plan(int n_items, int n_kv, int grid, boo
     return c;
 }
 struct Task { int w, j0, j1, piece; };      // piece: 1 = a cut item's piece (result goes to the scratch slot)
-__device__ __forceinline__ bool next_task(const CutPlan& c, int n_kv, int k, Task& t) {
+// CUT = false: whole items only, round after round (the plan is not looked at: the compiler sees constant bounds)
+template <bool CUT>
+__device__ __forceinline__ bool next_task(const CutPlan& c, int n_items, int n_kv, int k, Task& t) {
+    if constexpr (!CUT) {
+        const int w = (int)blockIdx.x + k * (int)gridDim.x;
+        t = Task{w, 0, n_kv, 0};
+        return w < n_items;
+    }
     if (k < c.n_rounds) { t = Task{(int)blockIdx.x + k * (int)gridDim.x, 0, n_kv, 0}; return true; }
     if (k > c.n_rounds || (int)blockIdx.x >= c.n_tail * c.parts) return false;
     const int ti = (int)blockIdx.x / c.parts, pt = (int)blockIdx.x - ti * c.parts;
@@ -173,7 +180,7 @@ __device__ __forceinline__ bool next_task(const CutPlan& c, int n_kv, int k, Tas
 // own-region mass
 __host__ __device__ inline size_t split_slot_floats(int dp) { return (size_t)128 * (dp + 4); }
 
-template <int D, bool MASS = false>
+template <int D, bool MASS = false, bool CUT = false>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
                     const __grid_constant__ CUtensorMap tm_q_tail, const __grid_constant__ CUtensorMap tm_kv_tail,
@@ -255,7 +262,8 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // so that head's K/V stays in L2 however long the key sequence is
     const int n_tiles = ctl->n_qtiles;
     const int n_items = n_tiles * heads;
-    const CutPlan cut = cut_plan(n_items, n_kv, (int)gridDim.x, split_ws != nullptr);
+    static_assert(!(MASS && CUT), "the first block's mass variant never cuts items");
+    const CutPlan cut = CUT ? cut_plan(n_items, n_kv, (int)gridDim.x, split_ws != nullptr) : CutPlan{0, 0, 1, 0};
 
     if (wg == 0) {
     reg_dec<48>();
@@ -266,7 +274,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             bool ok = true;
             int item_i = 0;
             Task tk;
-            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+            for (int k = 0; ok && next_task<CUT>(cut, n_items, n_kv, k, tk); ++k, ++item_i) {
                 const int w = tk.w;
                 const QTile t = tiles[w % n_tiles];
                 const int head = w / n_tiles;
@@ -317,7 +325,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             bool ok = true;
             int item_i = 0;
             Task tk;
-            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+            for (int k = 0; ok && next_task<CUT>(cut, n_items, n_kv, k, tk); ++k, ++item_i) {
                 const int w = tk.w;
                 const int qs = item_i & 1;
                 if (!mbar_wait(&q_full[qs], (item_i >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -359,7 +367,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             bool ok = true;
             int item_i = 0;
             Task tk;
-            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+            for (int k = 0; ok && next_task<CUT>(cut, n_items, n_kv, k, tk); ++k, ++item_i) {
                 const int w = tk.w;
                 for (int j = tk.j0; j < tk.j1; ++j, ++g) {
                     const int s = g % STAGES;
@@ -430,7 +438,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
             const uint64_t sc2 = pair(scale_log2, scale_log2);
             Task tk;
-            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+            for (int k = 0; ok && next_task<CUT>(cut, n_items, n_kv, k, tk); ++k, ++item_i) {
                 const int w = tk.w;
                 float m = -INFINITY, l = 0.f;
                 const uint32_t o_addr = lane_addr + COL64_O + ((item_i & 1) * 2 + par) * 64;
@@ -567,7 +575,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             int item_i = 0;
             const int rem = N - (n_kv - 1) * KEYS;                // valid keys of the last tile
             Task tk;
-            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+            for (int k = 0; ok && next_task<CUT>(cut, n_items, n_kv, k, tk); ++k, ++item_i) {
                 const int w = tk.w;
                 const QTile t = tiles[w % n_tiles];
                 const int head = w / n_tiles;
@@ -699,7 +707,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 mbar_arrive(&l_bar[quad]);
                 if (!mbar_wait(&l_bar[quad], item_i & 1, abort_flag)) { ok = false; break; }
                 // a cut item's piece stays un-normalised: its rows, maximum, sum (and mass) go to the CTA's scratch slot
-                const bool piece = tk.piece != 0;
+                const bool piece = CUT && tk.piece != 0;
                 const float inv = piece ? 1.0f : 1.0f / (l + s_xsum[(half ^ 1) * 128 + r]);
                 float* prow = split_ws + (size_t)blockIdx.x * split_slot_floats(DP) + (size_t)r * (DP + 4);
                 if (piece && half == 0) {
@@ -783,10 +791,13 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             uint8_t* wstage = s_stage + quad * 32 * 144;
             bool ok = true;
             int item_i = 0;
-            Task tk;
-            for (int k = 0; ok && next_task(cut, n_kv, k, tk); ++k, ++item_i) {
+            Task tk, tk_next;
+            // the work item's descriptor is fetched one item ahead
+            QTile t_next = next_task<CUT>(cut, n_items, n_kv, 0, tk_next) ? tiles[tk_next.w % n_tiles] : QTile{0, 0, 0, 0};
+            for (int k = 0; ok && next_task<CUT>(cut, n_items, n_kv, k, tk); ++k, ++item_i) {
                 const int w = tk.w;
-                const QTile t = tiles[w % n_tiles];
+                const QTile t = t_next;
+                if (next_task<CUT>(cut, n_items, n_kv, k + 1, tk_next)) t_next = tiles[tk_next.w % n_tiles];
                 const int head = w / n_tiles;
                 const int slot = item_i & 1;
                 if (!mbar_wait(&stat_full[slot], (item_i >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -803,7 +814,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const float a0 = m0 == -INFINITY ? 0.f : ex2((m0 - m_all) * scale_log2);
                 const float a1 = m1 == -INFINITY ? 0.f : ex2((m1 - m_all) * scale_log2);
                 // a cut item's piece stays un-normalised: its rows, maximum, sum (and mass) go to the CTA's scratch slot
-                const bool piece = tk.piece != 0;
+                const bool piece = CUT && tk.piece != 0;
                 const float inv = piece ? 1.0f : 1.0f / (a0 * l0 + a1 * l1);
                 const float w_0 = a0 * inv, w_1 = a1 * inv;       // weights of O_0, O_1
                 float* prow = split_ws + (size_t)blockIdx.x * split_slot_floats(DP) + (size_t)r * (DP + 4);
@@ -888,10 +899,10 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 // columns of a row at a time, so that a row's threads read and write whole lines and every thread has several
 // independent loads in flight (the statistics of a row are re-read by its threads: L1 hits).
 constexpr int COMBINE_THREADS = 256;
-template <int D, bool MASS>
+template <int D>
 __global__ void __launch_bounds__(COMBINE_THREADS)
 attn_combine_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o, int o_ld, const QTile* __restrict__ tiles,
-                    int heads, int N, int att_grid, float scale_log2, const Control* __restrict__ ctl, MassArgs ma) {
+                    int heads, int N, int att_grid, float scale_log2, const Control* __restrict__ ctl) {
     constexpr int DP = AttCfg<D>::DP;
     constexpr int CG = D / 4;                          // column groups of a row
     pdl_trigger();
@@ -912,14 +923,13 @@ attn_combine_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o,
             const float* base = ws + (size_t)ti * cut.parts * slot + (size_t)r * (DP + 4);
             float m = -INFINITY;
             for (int p = 0; p < cut.parts; ++p) m = fmaxf(m, base[p * slot + DP]);
-            float l = 0.f, own = 0.f;
+            float l = 0.f;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int p = 0; p < cut.parts; ++p) {
                 const float* row = base + p * slot;
                 const float c = ex2((row[DP] - m) * scale_log2);
                 const float4 x = *reinterpret_cast<const float4*>(row + cg * 4);
                 l = fmaf(c, row[DP + 1], l);
-                if constexpr (MASS) own = fmaf(c, row[DP + 2], own);
                 acc.x = fmaf(c, x.x, acc.x); acc.y = fmaf(c, x.y, acc.y);
                 acc.z = fmaf(c, x.z, acc.z); acc.w = fmaf(c, x.w, acc.w);
             }
@@ -928,13 +938,6 @@ attn_combine_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o,
             u.x = pack_bf16(acc.x * inv, acc.y * inv);
             u.y = pack_bf16(acc.z * inv, acc.w * inv);
             *reinterpret_cast<uint2*>(o + (size_t)(t.row0 + r) * o_ld + head * D + cg * 4) = u;
-            if constexpr (MASS) {
-                if (cg == 0) {
-                    const int lab = ma.labels[ma.active_idx[t.row0 + r]];
-                    if (lab >= 0 && lab < ma.R)
-                        atomicAdd(&ma.region_mass[(size_t)t.b * ma.R + lab], (double)(own * inv * ma.inv_heads));
-                }
-            }
         }
     }
 }
@@ -979,6 +982,12 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
     if (ok) ok = encode_tmap_bf16(&a->q_tail_map, buf.q, 2, dims, strides, box_tail, 32, err);
     cudaError_t e = cudaSuccess;
     if (ok) e = cudaFuncSetAttribute(tc_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<64>::SMEM);
+    if (ok && e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_attention_kernel<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<64>::SMEM);
+    if (ok && e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_attention_kernel<72, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<72>::SMEM);
+    if (ok && e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_attention_kernel<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<128>::SMEM);
     if (ok && e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_attention_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<64>::SMEM);
     if (ok && e == cudaSuccess)
@@ -1026,28 +1035,33 @@ cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, c
     // ... for long key sequences only: a piece pays an item's fixed costs (Q load, pipeline fill, hand-over) and the pieces
     // need a second, small kernel; measured, that is a loss at 1024 and 2048 keys and a gain of 3-8 % from 4096 on
     const bool long_keys = N >= 24 * KEYS || split_mode == 2;
-    float* split_ws = (split_on && long_keys && a->split_ws && grid <= a->split_slots) ? a->split_ws : nullptr;
+    // (not in the launch that also collects the first block's attention mass)
+    float* split_ws = (split_on && long_keys && !region_mass && a->split_ws && grid <= a->split_slots) ? a->split_ws : nullptr;
     const bool pdl = tc_plan_pdl(p);
     const int cgrid = max(1, grid / 2);             // at most grid / 2 items can be cut
-#define FD_ATT(DD, MM)                                                                                              \
+#define FD_ATT(DD, MM, CC)                                                                                          \
     do {                                                                                                            \
-        e = launch_kernel(tc_attention_kernel<DD, MM>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, pdl, a->q_map, kv_map,   \
+        e = launch_kernel(tc_attention_kernel<DD, MM, CC>, grid, ATT_THREADS, AttCfg<DD>::SMEM, st, pdl, a->q_map, kv_map, \
                           a->q_tail_map, kv_tail_map, o, a->H, tiles, a->heads, N, scale_log2, split_ws, c, ma);    \
         ++*n_launch;                                                                                                \
-        if (e == cudaSuccess && split_ws) {                                                                         \
-            e = launch_kernel(attn_combine_kernel<DD, MM>, dim3(cgrid, (QROWS * (DD / 4) + COMBINE_THREADS - 1) / COMBINE_THREADS),  \
-                              COMBINE_THREADS, 0, st, pdl, (const float*)split_ws, o, a->H, tiles,                  \
-                              a->heads, N, grid, scale_log2, ctl, ma);                                              \
+        if (e == cudaSuccess && (CC)) {                                                                             \
+            e = launch_kernel(attn_combine_kernel<DD>, dim3(cgrid, (QROWS * (DD / 4) + COMBINE_THREADS - 1) / COMBINE_THREADS), \
+                              COMBINE_THREADS, 0, st, pdl, (const float*)split_ws, o, a->H, tiles, a->heads, N, grid, \
+                              scale_log2, ctl);                                                                     \
             ++*n_launch;                                                                                            \
         }                                                                                                           \
     } while (0)
     if (region_mass) {
-        if (a->dh == 64) FD_ATT(64, true);
-        else if (a->dh == 128) FD_ATT(128, true);
-        else FD_ATT(72, true);
-    } else if (a->dh == 64) FD_ATT(64, false);
-    else if (a->dh == 128) FD_ATT(128, false);
-    else FD_ATT(72, false);
+        if (a->dh == 64) FD_ATT(64, true, false);
+        else if (a->dh == 128) FD_ATT(128, true, false);
+        else FD_ATT(72, true, false);
+    } else if (split_ws) {
+        if (a->dh == 64) FD_ATT(64, false, true);
+        else if (a->dh == 128) FD_ATT(128, false, true);
+        else FD_ATT(72, false, true);
+    } else if (a->dh == 64) FD_ATT(64, false, false);
+    else if (a->dh == 128) FD_ATT(128, false, false);
+    else FD_ATT(72, false, false);
 #undef FD_ATT
     return e;
 }
