@@ -286,15 +286,12 @@ __device__ __forceinline__ void epilogue_prefetch_resid(const EpiParams& ep, int
     }
 }
 
-// one warp's share of a tile: rows [row_base, row_base + 32), columns [c_begin, c_end) of the accumulator at t_row
+// Per-lane row data of a warp's 32 rows (request, cache / output row): depends only on the tile, so the caller can
+// fetch it while the tile's products are still running.
 template <int KIND>
-__device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stage, int lane, int row_base, int a_total,
-                                              uint32_t t_row, int tile_col0, int c_begin, int c_end,
-                                              const CUtensorMap* tm_r = nullptr) {
-    const bool live = row_base < a_total;                        // warp-uniform
-    const int n_rows = a_total - row_base;
+__device__ __forceinline__ RowInfo epilogue_row_info(const EpiParams& ep, int lane, int row_base, int a_total) {
     RowInfo ri{0, 0u, 0u};
-    if (KIND != EPI_GELU && live && lane < n_rows) {
+    if (KIND != EPI_GELU && row_base + lane < a_total) {
         const int tok = ep.active_idx[row_base + lane];
         const int b = tok / ep.N;
         ri.gate_off = b * 6 * ep.H;
@@ -302,6 +299,16 @@ __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stag
         ri.y_lo = (uint32_t)off;
         ri.y_hi = (uint32_t)(off >> 32);
     }
+    return ri;
+}
+
+// one warp's share of a tile: rows [row_base, row_base + 32), columns [c_begin, c_end) of the accumulator at t_row
+template <int KIND>
+__device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stage, int lane, int row_base, int a_total,
+                                              uint32_t t_row, int tile_col0, int c_begin, int c_end, const RowInfo& ri,
+                                              const CUtensorMap* tm_r = nullptr) {
+    const bool live = row_base < a_total;                        // warp-uniform
+    const int n_rows = a_total - row_base;
     if constexpr (KIND == EPI_RESID) {
 #pragma unroll 1
         for (int c0 = c_begin; c0 < c_end; c0 += 32) {

@@ -133,11 +133,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
             if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * BM + quad * 32, a_total, n * BN + chalf * (BN / 2), BN / 2);
+            // the rows' request / cache-row data while the tile's products are still running
+            const RowInfo ri = epilogue_row_info<KIND>(ep, lane, m * BM + quad * 32, a_total);
             if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BN;
             epilogue_warp<KIND>(ep, epi_stage + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane, m * BM + quad * 32, a_total,
-                                t_row, n * BN, chalf * (BN / 2), (chalf + 1) * (BN / 2));
+                                t_row, n * BN, chalf * (BN / 2), (chalf + 1) * (BN / 2), ri);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty[acc]);
@@ -283,11 +285,13 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * 2 * BM + (int)rank * BM + quad * 32, a_total,
                                         n * PAIR_BN + c_lo, c_hi - c_lo);
+            // the rows' request / cache-row data while the tile's products are still running
+            const RowInfo ri = epilogue_row_info<KIND>(ep, lane, m * 2 * BM + (int)rank * BM + quad * 32, a_total);
             if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
             epilogue_warp<KIND>(ep, epi_stage + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane,
-                                m * 2 * BM + (int)rank * BM + quad * 32, a_total, t_row, n * PAIR_BN, c_lo, c_hi,
+                                m * 2 * BM + (int)rank * BM + quad * 32, a_total, t_row, n * PAIR_BN, c_lo, c_hi, ri,
                                 (KIND == EPI_RESID && tma_resid) ? &tm_r : nullptr);
             tc_fence_before();
             __syncwarp();
