@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 MAX_ABS, REL_L2 = 3e-2, 1e-2
 
 
-def _full_shape_block(name, seed, fractions, n_sample=160):
+def _full_shape_block(name, seed, fractions, n_sample=160, with_mass=False):
     wl = gen.workload(name).replace(L=1)
     B, N, H = wl.B, wl.N, wl.H
     labels = labels_for(wl, seed)
@@ -31,7 +31,15 @@ def _full_shape_block(name, seed, fractions, n_sample=160):
     dt = tdtype(wl)
     buf.kv.copy_(dev(kv0, dt))
     buf.y.copy_(dev(y0, dt))
-    idx, cu = gpu_step(ctx, wl, dev(inp["x_cur"], dt), dev(inp["cond"], dt), dev(labels), dev(mask), buf)
+    if with_mass:       # the step that also collects the first block's own-region attention mass (Sec. 4.2)
+        mass = torch.full((B, wl.R), -1.0, dtype=torch.float64, device="cuda")
+        fd.fd_regional_step_mass(ctx, dev(inp["x_cur"], dt), dev(inp["cond"], dt), dev(labels), dev(mask), wl.R, buf.kv,
+                                 buf.y, buf.active_idx, buf.cu_active, mass)
+        fd.fd_poll_status(ctx)
+        cu = host(buf.cu_active)
+        idx = host(buf.active_idx)[: cu[-1]]
+    else:
+        idx, cu = gpu_step(ctx, wl, dev(inp["x_cur"], dt), dev(inp["cond"], dt), dev(labels), dev(mask), buf)
 
     o_idx, o_cu = oracle.compact(mask, labels, wl.R)
     assert np.array_equal(idx, o_idx) and np.array_equal(cu, o_cu)
@@ -55,6 +63,14 @@ def _full_shape_block(name, seed, fractions, n_sample=160):
     assert max_abs(y[rows], out[pick]) <= MAX_ABS
     assert rel_l2(y[rows], out[pick]) <= REL_L2
     assert np.array_equal(y[~act], y0.reshape(B * N, H)[~act])
+    if with_mass:
+        # keys as the block's attention saw them: refreshed rows of active tokens, cached rows of the others
+        q = oracle.block0_queries(inp["x_cur"], inp["cond"], w, o_idx)
+        ref = oracle.attention_mass(q, kv_ref[:, 0], labels, o_idx, wl.heads, wl.R)
+        got = host(mass)
+        ran = mask.astype(bool)
+        assert np.all(got[~ran] == 0.0)
+        np.testing.assert_allclose(got[ran], ref[ran], rtol=2e-2, atol=1e-6)      # bf16 Q / K move the probabilities by ~1 %
     return ctx
 
 
@@ -69,6 +85,21 @@ def test_image_full_shape():
 
 def test_mmdit_full_shape_with_text_tokens():
     _full_shape_block("mmdit", 23, [0.34, 0.76])
+
+
+def test_audio_full_shape_attention_mass():
+    """Head dim 64, 1056 attention work items: the mass variant of the kernel at the benchmark's shape."""
+    wl = gen.workload("audio")
+    _full_shape_block("audio", 25, gen.request_fractions(wl, 25), with_mass=True)
+
+
+def test_image_full_shape_attention_mass():
+    _full_shape_block("image", 26, [0.25, 0.5, 0.75, 1.0], with_mass=True)
+
+
+def test_mmdit_full_shape_attention_mass_with_text_tokens():
+    """Text tokens carry the label R: always active, part of no region."""
+    _full_shape_block("mmdit", 27, [0.34, 0.76], with_mass=True)
 
 
 def test_video_full_shape():
