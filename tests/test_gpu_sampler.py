@@ -19,7 +19,8 @@ def _sampler(wl, seed):
 
 
 @pytest.mark.parametrize("name,engine", [("tiny", fd.FD_ENGINE_SIMT), ("audio_small", fd.FD_ENGINE_SIMT),
-                                         ("image_tc", fd.FD_ENGINE_TC), ("mmdit_tc", fd.FD_ENGINE_TC)])
+                                         ("image_tc", fd.FD_ENGINE_TC), ("mmdit_tc", fd.FD_ENGINE_TC),
+                                         ("audio", fd.FD_ENGINE_AUTO), ("video", fd.FD_ENGINE_AUTO)])     # full shapes
 def test_embed_latent(name, engine):
     wl = gen.workload(name)
     ctx = make_ctx(wl, gen.block_weights(wl, 1, n_blocks=1), n_blocks=1, engine=engine)
@@ -37,7 +38,8 @@ def test_embed_latent(name, engine):
 
 @pytest.mark.parametrize("name,engine,frac", [("tiny", fd.FD_ENGINE_SIMT, 0.5), ("audio_small", fd.FD_ENGINE_SIMT, 0.3),
                                               ("image_tc", fd.FD_ENGINE_TC, 0.7), ("mmdit_tc", fd.FD_ENGINE_TC, 1.0),
-                                              ("audio_small", fd.FD_ENGINE_SIMT, 0.0)])
+                                              ("audio_small", fd.FD_ENGINE_SIMT, 0.0),
+                                              ("audio", fd.FD_ENGINE_AUTO, 0.64), ("video", fd.FD_ENGINE_AUTO, 0.45)])
 def test_update_latent(name, engine, frac):
     """Active tokens get a fresh drift from their row of y; every other token keeps its cached drift bit for bit
     and moves along it; rows of y that belong to skipped tokens are not read (NaN there is harmless)."""
