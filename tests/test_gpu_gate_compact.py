@@ -34,7 +34,7 @@ def _gate(ctx, wl, z_cur, z_prev, labels, eps, st):
 
 
 @pytest.mark.parametrize("name,seed", [("tiny", 0), ("audio_small", 1), ("image_small", 2), ("mmdit_small", 3),
-                                       ("video_small", 4)])
+                                       ("video_small", 4), ("audio", 5), ("mmdit", 6), ("video", 7)])        # ... and full shapes
 def test_gate_single_step(name, seed):
     wl = gen.workload(name)
     labels = labels_for(wl, seed)
