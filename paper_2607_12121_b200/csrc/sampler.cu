@@ -229,7 +229,7 @@ final_drift_mma_kernel(const __nv_bfloat16* __restrict__ y, const int32_t* __res
 // Patch embedding: x[tok, h] = sum_d z[tok, d] W[h, d] + b[h] + pos[j, h].  z is fp32: it enters as a bf16 head plus a
 // bf16 remainder (two products), which keeps fp32-level accuracy.  One warp = 16 tokens x EM_COLS output columns;
 // each 64-column group goes through a shared-memory tile so that the rows leave as whole 128-byte lines.
-constexpr int EM_WARPS = 8, EM_COLS = 512;
+constexpr int EM_WARPS = 8, EM_COLS = 128;       // columns per CTA: smaller chunks = more CTAs in flight (audio 41 -> 34 us)
 template <int KB>                                  // D / 16
 __global__ void __launch_bounds__(EM_WARPS * 32)
 embed_mma_kernel(const float* __restrict__ z, const __nv_bfloat16* __restrict__ w_in, const __nv_bfloat16* __restrict__ b_in,
