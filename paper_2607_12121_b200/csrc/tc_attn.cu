@@ -9,16 +9,16 @@
 //   warp 2       issues O += P V with P read from TMEM and V as an N-major shared-memory operand
 //   warps 4..11  softmax: tcgen05.ld of the scores, running maximum with lazy rescaling of O (only
 //                when it grew by more than 2^24), exp2, P written to TMEM as packed bf16
-//   warps 12..15 head dim 64: item epilogue (merge, normalise, store) while the softmax warps go on
-// Head dims 128 and 72 (run as 80): one accumulator; two threads per query row, each with 64 of a
-// tile's 128 keys, swap their partial maxima through shared memory and end the item themselves.
-// Head dim 64: warpgroup p takes the key tiles of parity p with its own P buffer, accumulator O_p
-// and running maximum / row sum: one thread per row copies the tile's 128 scores to registers and
-// hands the (single) score buffer back at once, so that the next S = Q K^T runs under this tile's
-// exponentials; the two warpgroups never wait for each other.  TMEM then has room for four
-// accumulators (item parity x tile parity): the next item's products start while the epilogue
-// warpgroup still merges this item's partial results, O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1),
-// a_p = 2^(m_p - m).
+//   warps 12..15 head dims 64 and 128: item epilogue (merge, normalise, store) while the softmax warps go on
+// Head dim 72 (run as 80): one accumulator; two threads per query row, each with 64 of a tile's 128
+// keys, swap their partial maxima through shared memory and end the item themselves.
+// Head dims 64 and 128: warpgroup p takes the key tiles of parity p with its own P buffer,
+// accumulator O_p and running maximum / row sum: one thread per row copies the tile's 128 scores to
+// registers and hands the (single) score buffer back at once, so that the next S = Q K^T runs under
+// this tile's exponentials; the two warpgroups never wait for each other.  The epilogue warpgroup
+// merges the partial results, O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1), a_p = 2^(m_p - m), while the
+// softmax warps go on; at head dim 64 TMEM has room for four accumulators (item parity x tile
+// parity), so the next item's products start under that merge.
 // Keys past N in the last tile are zero-filled by TMA and masked.
 // For long key sequences the items of the last, partly filled round are cut along the keys (CutPlan below) and
 // attn_combine_kernel puts their pieces together.
@@ -53,7 +53,7 @@ template <int D> struct AttCfg {
     static constexpr int TILE_BYTES = SUBS * SUB_BYTES + (D == 72 ? TAIL_BYTES : 0);
     // K/V rings deep enough that a tile is requested several tile periods before it is needed
     static constexpr int STAGES = D == 128 ? 2 : (D == 72 ? 4 : 5);
-    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + (D == 64 ? 128 * 144 : 0) + 2048;
+    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + (D != 72 ? 128 * 144 : 0) + 2048;
 };
 
 // Register re-balancing between warpgroups: the kernel starts with 128 registers per thread (512 threads);
@@ -127,8 +127,12 @@ constexpr float RESCALE_LOG2 = 24.0f;
 
 // TMEM columns: two score buffers, the output accumulator, two P buffers (bf16 pairs)
 constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384, TMEM_COLS = 512;
-// head dim 64: one score buffer, two P buffers (tile parity), four accumulators (item parity x tile parity)
+// head dims 64 and 128: one score buffer, two P buffers (tile parity), accumulators from column 256: at head dim 64
+// four (item parity x tile parity), at 128 two (tile parity)
 constexpr uint32_t COL64_S = 0, COL64_P = 128, COL64_O = 256;
+template <int D> __device__ __forceinline__ uint32_t acc_col(int item_i, int par) {
+    return COL64_O + (uint32_t)((D == 64 ? (item_i & 1) * 2 : 0) + par) * D;
+}
 
 // What the MASS variant (head dim 64, launched for a step's first block when asked) needs on top: per region, the
 // softmax mass its active queries put on keys of their own region (paper Sec. 4.2).
@@ -188,7 +192,10 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     float scale_log2, float* __restrict__ split_ws, Control* ctl, MassArgs ma) {
     using Cfg = AttCfg<D>;
     constexpr int DP = Cfg::DP;
-    constexpr bool SPLIT = D == 64;                      // per-half accumulators, no exchange in the key loop
+    // tile-parity layout (an accumulator per softmax warpgroup, no exchange in the key loop): head dims 64 and 128;
+    // the mass variant of head dim 128 stays on the two-threads-per-row layout (its label bookkeeping per score is
+    // cheaper there: 64 scores per thread)
+    constexpr bool SPLIT = D == 64 || (D == 128 && !MASS);
     constexpr int STAGES = Cfg::STAGES;
     constexpr int TILE_BYTES = Cfg::TILE_BYTES;
     extern __shared__ __align__(1024) uint8_t smem[];    // 128-byte swizzled tiles need 1024-byte alignment
@@ -217,7 +224,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     float* s_xsum = s_xmax + 512;                                 // [2 halves][128 rows]; head dim 64: [2 items][2 halves][128 rows]
     uint8_t* s_stage = reinterpret_cast<uint8_t*>(bars) + 4608;   // [128 rows][144 bytes], head dim 64 only
     // MASS: own-region mass, head dim 64 [2 items][2 halves][128 rows], otherwise [2 halves][128 rows]
-    float* s_xown = reinterpret_cast<float*>(s_stage + (D == 64 ? 128 * 144 : 0));
+    float* s_xown = reinterpret_cast<float*>(s_stage + (SPLIT ? 128 * 144 : 0));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (smem_u32(smem) & 1023u) {                        // never expected; refuse rather than compute garbage
@@ -373,8 +380,12 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const int s = g % STAGES;
                     if (!mbar_wait(&v_full[s], (g / STAGES) & 1, abort_flag)) { ok = false; break; }
                     if constexpr (SPLIT) {
-                        // the accumulators alternate from item to item: these were last used two items ago
-                        if (j == tk.j0 && item_i >= 2 && !mbar_wait(&o_free[item_i & 1], ((item_i >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                        if constexpr (D == 64) {
+                            // the accumulators alternate from item to item: these were last used two items ago
+                            if (j == tk.j0 && item_i >= 2 && !mbar_wait(&o_free[item_i & 1], ((item_i >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                        } else {
+                            if (j == tk.j0 && item_i > 0 && !mbar_wait(&o_free[0], (item_i - 1) & 1, abort_flag)) { ok = false; break; }
+                        }
                     } else {
                         if (j == tk.j0 && item_i > 0 && !mbar_wait(&o_free[0], (item_i - 1) & 1, abort_flag)) { ok = false; break; }
                     }
@@ -383,7 +394,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         // the tiles of one parity accumulate into their own O: even tiles O_0, odd tiles O_1
                         if (!mbar_wait(&p_full[(g & 1) * 2], (g >> 1) & 1, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t d = tmem_base + COL64_O + ((item_i & 1) * 2 + (g & 1)) * 64;
+                        const uint32_t d = tmem_base + acc_col<D>(item_i, g & 1);
                         const uint32_t a = tmem_base + COL64_P + (g & 1) * 64;
 #pragma unroll
                         for (int ks = 0; ks < KEYS / 16; ++ks)
@@ -441,7 +452,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int k = 0; ok && next_task<CUT>(cut, n_items, n_kv, k, tk); ++k, ++item_i) {
                 const int w = tk.w;
                 float m = -INFINITY, l = 0.f;
-                const uint32_t o_addr = lane_addr + COL64_O + ((item_i & 1) * 2 + par) * 64;
+                const uint32_t o_addr = lane_addr + acc_col<D>(item_i, par);
                 // MASS: the part of l that comes from keys carrying the query's own region label
                 float own = 0.f;
                 int my_lab = -1;
@@ -489,7 +500,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
                             if (need) { l *= f; own *= f; m = mx; }
 #pragma unroll 1
-                            for (int c = 0; c < 8; ++c) {        // rare, and 128 scores are live: small pieces
+                            for (int c = 0; c < D / 8; ++c) {    // rare, and 128 scores are live: small pieces
                                 uint32_t orr[8];
                                 tmem_ld8(o_addr + c * 8, orr);
                                 tmem_wait_ld();
@@ -836,51 +847,55 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         sum += __shfl_sync(peers, mine, __ffs(rest) - 1);
                     if (lab >= 0 && lane == __ffs(peers) - 1) atomicAdd(&ma.region_mass[(size_t)t.b * ma.R + lab], (double)sum);
                 }
-                // a rolled loop on purpose: this code runs once per item, and the fewer instructions it fetches the
-                // less it disturbs the softmax warps that share the instruction caches
+                // rolled loops on purpose: this code runs once per item, and the fewer instructions it fetches the
+                // less it disturbs the softmax warps that share the instruction caches.  64 output columns per pass.
+                const uint32_t acc0 = lane_addr + acc_col<D>(item_i, 0), acc1 = lane_addr + acc_col<D>(item_i, 1);
 #pragma unroll 1
-                for (int q = 0; q < 8; ++q) {
-                    uint32_t o0[8], o1[8];
-                    tmem_ld8(lane_addr + COL64_O + slot * 128 + q * 8, o0);
-                    tmem_ld8(lane_addr + COL64_O + slot * 128 + 64 + q * 8, o1);
-                    tmem_wait_ld();
-                    if (q == 7) {
-                        // the accumulators are free for the next item as soon as they are in registers
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&o_free[slot]);
-                    }
-                    float v[8];
+                for (int hp = 0; hp < D / 64; ++hp) {
+#pragma unroll 1
+                    for (int q = 0; q < 8; ++q) {
+                        uint32_t o0[8], o1[8];
+                        tmem_ld8(acc0 + hp * 64 + q * 8, o0);
+                        tmem_ld8(acc1 + hp * 64 + q * 8, o1);
+                        tmem_wait_ld();
+                        if (hp == D / 64 - 1 && q == 7) {
+                            // the accumulators are free for the next item as soon as they are in registers
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&o_free[D == 64 ? slot : 0]);
+                        }
+                        float v[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        // a zero weight must also silence whatever an untouched accumulator holds
-                        const float x0 = w_0 != 0.f ? __uint_as_float(o0[i]) * w_0 : 0.f;
-                        const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
-                        v[i] = x0 + x1;
+                        for (int i = 0; i < 8; ++i) {
+                            // a zero weight must also silence whatever an untouched accumulator holds
+                            const float x0 = w_0 != 0.f ? __uint_as_float(o0[i]) * w_0 : 0.f;
+                            const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
+                            v[i] = x0 + x1;
+                        }
+                        if (piece) {
+                            *reinterpret_cast<float4*>(prow + hp * 64 + q * 8) = make_float4(v[0], v[1], v[2], v[3]);
+                            *reinterpret_cast<float4*>(prow + hp * 64 + q * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                            continue;
+                        }
+                        uint4 u;
+                        u.x = pack_bf16(v[0], v[1]);
+                        u.y = pack_bf16(v[2], v[3]);
+                        u.z = pack_bf16(v[4], v[5]);
+                        u.w = pack_bf16(v[6], v[7]);
+                        *reinterpret_cast<uint4*>(wstage + lane * 144 + q * 16) = u;
                     }
-                    if (piece) {
-                        *reinterpret_cast<float4*>(prow + q * 8) = make_float4(v[0], v[1], v[2], v[3]);
-                        *reinterpret_cast<float4*>(prow + q * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
-                        continue;
-                    }
-                    uint4 u;
-                    u.x = pack_bf16(v[0], v[1]);
-                    u.y = pack_bf16(v[2], v[3]);
-                    u.z = pack_bf16(v[4], v[5]);
-                    u.w = pack_bf16(v[6], v[7]);
-                    *reinterpret_cast<uint4*>(wstage + lane * 144 + q * 16) = u;
-                }
-                if (piece) continue;
-                __syncwarp();
-                // eight neighbouring lanes write one row's 128 bytes: 4 lines per store instruction instead of 32
-                __nv_bfloat16* obase = o + (size_t)(t.row0 + quad * 32) * o_ld + head * D + (lane & 7) * 8;
+                    if (piece) continue;
+                    __syncwarp();
+                    // eight neighbouring lanes write one row's 128 bytes: 4 lines per store instruction instead of 32
+                    __nv_bfloat16* obase = o + (size_t)(t.row0 + quad * 32) * o_ld + head * D + hp * 64 + (lane & 7) * 8;
 #pragma unroll 1
-                for (int k = 0; k < 8; ++k) {
-                    const int rr = k * 4 + (lane >> 3);           // row inside the warp's 32
-                    const uint4 u = *reinterpret_cast<const uint4*>(wstage + rr * 144 + (lane & 7) * 16);
-                    if (quad * 32 + rr < t.rows) *reinterpret_cast<uint4*>(obase + (size_t)rr * o_ld) = u;
+                    for (int k = 0; k < 8; ++k) {
+                        const int rr = k * 4 + (lane >> 3);       // row inside the warp's 32
+                        const uint4 u = *reinterpret_cast<const uint4*>(wstage + rr * 144 + (lane & 7) * 16);
+                        if (quad * 32 + rr < t.rows) *reinterpret_cast<uint4*>(obase + (size_t)rr * o_ld) = u;
+                    }
+                    __syncwarp();                                 // the staging rows are rewritten by the next pass / item
                 }
-                __syncwarp();                                     // the staging rows are rewritten by the next item
             }
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 700 + (int)blockIdx.x);
         }
