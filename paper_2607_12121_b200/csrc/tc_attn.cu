@@ -9,16 +9,17 @@
 //   warp 2       issues O += P V with P read from TMEM and V as an N-major shared-memory operand
 //   warps 4..11  softmax: tcgen05.ld of the scores, running maximum with lazy rescaling of O (only
 //                when it grew by more than 2^24), exp2, P written to TMEM as packed bf16
-//   warps 12..15 head dims 64 and 128: item epilogue (merge, normalise, store) while the softmax warps go on
-// Head dim 72 (run as 80): one accumulator; two threads per query row, each with 64 of a tile's 128
-// keys, swap their partial maxima through shared memory and end the item themselves.
-// Head dims 64 and 128: warpgroup p takes the key tiles of parity p with its own P buffer,
+//   warps 12..15 item epilogue (merge, normalise, store) while the softmax warps go on
+// Warpgroup p takes the key tiles of parity p with its own P buffer,
 // accumulator O_p and running maximum / row sum: one thread per row copies the tile's 128 scores to
 // registers and hands the (single) score buffer back at once, so that the next S = Q K^T runs under
 // this tile's exponentials; the two warpgroups never wait for each other.  The epilogue warpgroup
 // merges the partial results, O = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1), a_p = 2^(m_p - m), while the
 // softmax warps go on; at head dim 64 TMEM has room for four accumulators (item parity x tile
-// parity), so the next item's products start under that merge.
+// parity), so the next item's products start under that merge.  Head dim 72 runs as 80.
+// The mass variants of head dims 72 and 128 keep an older layout: one accumulator; two threads per query
+// row, each with 64 of a tile's 128 keys, swap their partial maxima through shared memory and end the item
+// themselves.
 // Keys past N in the last tile are zero-filled by TMA and masked.
 // For long key sequences the items of the last, partly filled round are cut along the keys (CutPlan below) and
 // attn_combine_kernel puts their pieces together.
@@ -53,7 +54,7 @@ template <int D> struct AttCfg {
     static constexpr int TILE_BYTES = SUBS * SUB_BYTES + (D == 72 ? TAIL_BYTES : 0);
     // K/V rings deep enough that a tile is requested several tile periods before it is needed
     static constexpr int STAGES = D == 128 ? 2 : (D == 72 ? 4 : 5);
-    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + (D != 72 ? 128 * 144 : 0) + 2048;
+    static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + 128 * 144 + 2048;
 };
 
 // Register re-balancing between warpgroups: the kernel starts with 128 registers per thread (512 threads);
@@ -131,7 +132,7 @@ constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384, TMEM_COLS = 512;
 // four (item parity x tile parity), at 128 two (tile parity)
 constexpr uint32_t COL64_S = 0, COL64_P = 128, COL64_O = 256;
 template <int D> __device__ __forceinline__ uint32_t acc_col(int item_i, int par) {
-    return COL64_O + (uint32_t)((D == 64 ? (item_i & 1) * 2 : 0) + par) * D;
+    return COL64_O + (uint32_t)((D == 64 ? (item_i & 1) * 2 : 0) + par) * (D == 72 ? 80 : D);
 }
 
 // What the MASS variant (head dim 64, launched for a step's first block when asked) needs on top: per region, the
@@ -192,10 +193,10 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     float scale_log2, float* __restrict__ split_ws, Control* ctl, MassArgs ma) {
     using Cfg = AttCfg<D>;
     constexpr int DP = Cfg::DP;
-    // tile-parity layout (an accumulator per softmax warpgroup, no exchange in the key loop): head dims 64 and 128;
-    // the mass variant of head dim 128 stays on the two-threads-per-row layout (its label bookkeeping per score is
-    // cheaper there: 64 scores per thread)
-    constexpr bool SPLIT = D == 64 || (D == 128 && !MASS);
+    // tile-parity layout (an accumulator per softmax warpgroup, no exchange in the key loop); the mass variants of head
+    // dims 72 and 128 stay on the two-threads-per-row layout (their label bookkeeping per score is cheaper there: 64
+    // scores per thread)
+    constexpr bool SPLIT = D == 64 || !MASS;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int TILE_BYTES = Cfg::TILE_BYTES;
     extern __shared__ __align__(1024) uint8_t smem[];    // 128-byte swizzled tiles need 1024-byte alignment
@@ -397,9 +398,15 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         const uint32_t d = tmem_base + acc_col<D>(item_i, g & 1);
                         const uint32_t a = tmem_base + COL64_P + (g & 1) * 64;
 #pragma unroll
-                        for (int ks = 0; ks < KEYS / 16; ++ks)
-                            mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
-                                        j - tk.j0 >= 2 || ks != 0);
+                        for (int ks = 0; ks < KEYS / 16; ++ks) {
+                            if constexpr (D == 72)
+                                // 16 keys further: two 8-key groups of 256 bytes; the 16-column blocks sit TAIL_BYTES apart
+                                mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 512, TAIL_BYTES, 256, SWZ_32B), idesc_pv,
+                                            j - tk.j0 >= 2 || ks != 0);
+                            else
+                                mma_bf16_ts(d, a + ks * 8, smem_desc(v_addr + ks * 2048, SUB_BYTES, 1024, SWZ_128B), idesc_pv,
+                                            j - tk.j0 >= 2 || ks != 0);
+                        }
                         mma_commit(&v_empty[s]);
                         mma_commit(&pv_done[(g & 1) * 2]);
                         // the item's products complete in issue order: this one covers them all.  (Its own barrier: the
@@ -858,7 +865,7 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         tmem_ld8(acc0 + hp * 64 + q * 8, o0);
                         tmem_ld8(acc1 + hp * 64 + q * 8, o1);
                         tmem_wait_ld();
-                        if (hp == D / 64 - 1 && q == 7) {
+                        if (D != 72 && hp == D / 64 - 1 && q == 7) {
                             // the accumulators are free for the next item as soon as they are in registers
                             tc_fence_before();
                             __syncwarp();
@@ -895,6 +902,34 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         if (quad * 32 + rr < t.rows) *reinterpret_cast<uint4*>(obase + (size_t)rr * o_ld) = u;
                     }
                     __syncwarp();                                 // the staging rows are rewritten by the next pass / item
+                }
+                if constexpr (D == 72) {
+                    // columns 64..71 of the head: 16 bytes per row, stored by the row's thread
+                    uint32_t o0[8], o1[8];
+                    tmem_ld8(acc0 + 64, o0);
+                    tmem_ld8(acc1 + 64, o1);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&o_free[0]);
+                    float v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float x0 = w_0 != 0.f ? __uint_as_float(o0[i]) * w_0 : 0.f;
+                        const float x1 = w_1 != 0.f ? __uint_as_float(o1[i]) * w_1 : 0.f;
+                        v[i] = x0 + x1;
+                    }
+                    if (piece) {
+                        *reinterpret_cast<float4*>(prow + 64) = make_float4(v[0], v[1], v[2], v[3]);
+                        *reinterpret_cast<float4*>(prow + 68) = make_float4(v[4], v[5], v[6], v[7]);
+                    } else if (r < t.rows) {
+                        uint4 u;
+                        u.x = pack_bf16(v[0], v[1]);
+                        u.y = pack_bf16(v[2], v[3]);
+                        u.z = pack_bf16(v[4], v[5]);
+                        u.w = pack_bf16(v[6], v[7]);
+                        *reinterpret_cast<uint4*>(o + (size_t)(t.row0 + r) * o_ld + head * D + 64) = u;
+                    }
                 }
             }
             if (!ok && lane == 0) report(ctl, FD_ERR_TIMEOUT, 700 + (int)blockIdx.x);
