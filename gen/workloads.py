@@ -87,6 +87,11 @@ WORKLOADS["mmdit_tc"] = WORKLOADS["mmdit"].replace(
 WORKLOADS["video_tc"] = WORKLOADS["video"].replace(
     name="video_tc", L=2, H=256, heads=2, M=640, Hc=256, grid=(6, 10, 14), B=1, R=24,
     n_cells=12, m_min=8, m_max=128, D=16)
+# config 4's scaled-down twin for full-depth, multi-step parity: all 30 blocks, 3136 keys (long enough for the
+# attention's default cut-and-combine path), 32 spatio-temporal regions
+WORKLOADS["video_twin"] = WORKLOADS["video"].replace(
+    name="video_twin", H=256, heads=2, M=640, Hc=256, grid=(7, 16, 28), B=1, R=32,
+    n_cells=6, m_min=16, m_max=256, D=16)
 WORKLOADS["image_tc"] = WORKLOADS["image"].replace(
     name="image_tc", L=1, grid=(12, 16), B=2, R=12, n_cells=12, m_min=8, m_max=32)
 WORKLOADS["wide_tc"] = WORKLOADS["audio"].replace(
@@ -314,3 +319,35 @@ def mask_schedule(wl: Workload, seed: int, steps: int, fraction: float = 0.5) ->
 def request_fractions(wl: Workload, seed: int, lo: float = 0.2, hi: float = 0.8) -> np.ndarray:
     """Per-request active fraction ~U[lo,hi] (requests at different denoising steps)."""
     return _rng(seed, 808).uniform(lo, hi, size=wl.B)
+
+
+def latent_sequence(wl: Workload, seed: int, labels: np.ndarray,
+                    fractions_per_step: Sequence[Sequence[float]]):
+    """Latents of a run of neighbouring steps with a target active fraction per step and request.
+
+    z_0 ~ N(0,1); step t moves every region by its own noise scale, z_t = z_{t-1} + sigma_t[region] * N(0,1), where
+    sigma_t and the threshold eps_t are drawn exactly as in ``latent_pair`` for the fractions of step t (a fresh
+    log-uniform draw per step, the k loudest pushed up and the others down by sqrt(2), eps in the gap).  Regions
+    a gate keeps frozen carry older magnitudes, so the measured fraction of a step need not equal its target.
+    Returns a list of dicts with z_cur, z_prev, eps (one per step).
+    """
+    B, N, D, R = wl.B, wl.N, wl.D, wl.R
+    g = _rng(seed, 1212)
+    z = g.standard_normal((B, N, D), dtype=np.float32)
+    out = []
+    for t, fractions in enumerate(fractions_per_step):
+        assert len(fractions) == B
+        sigma = np.exp(g.uniform(np.log(1e-4), np.log(1e-1), size=(B, R)))
+        eps = np.empty(B, dtype=np.float32)
+        for b in range(B):
+            k = min(max(int(round(float(fractions[b]) * R)), 1), R)
+            order = np.argsort(-sigma[b], kind="stable")
+            sigma[b, order[:k]] *= np.sqrt(2.0)
+            sigma[b, order[k:]] /= np.sqrt(2.0)
+            eps[b] = 0.0 if k == R else np.float32(np.sqrt(sigma[b, order[k - 1]] * sigma[b, order[k]]) / sigma[b].sum())
+        sig_tok = np.take_along_axis(np.concatenate([sigma, np.zeros((B, 1))], axis=1),
+                                     labels.astype(np.int64), axis=1).astype(np.float32)
+        z_next = (z + sig_tok[..., None] * g.standard_normal((B, N, D), dtype=np.float32)).astype(np.float32)
+        out.append({"z_cur": z_next, "z_prev": z, "eps": eps})
+        z = z_next
+    return out

@@ -10,8 +10,15 @@
  * Errors a host can see (null or misaligned pointers, shapes beyond the limits given at
  * creation, unsupported head sizes) return a status with nothing launched.  Problems only the
  * device can see (a label outside [0,R], a bounded wait that ran out) never trap: the kernel
- * records a code in the workspace, skips the offending work, and fd_poll_status / fd_destroy
- * report it.
+ * records a code in the workspace and skips the offending work.  No call reads that word back by
+ * itself (that would be a synchronisation): fd_poll_status synchronises the stream and returns
+ * it, and fd_destroy returns whatever is still unpolled.
+ *
+ * Test-only switches, read from the environment when a context is created; they select older or
+ * restricted forms of a kernel and are not part of the interface: FD_PDL=0 (fully serialised
+ * launches), FD_TC_PAIR=0 (single-CTA GEMM tiles), FD_TMA_RESID=0 (per-thread residual
+ * reductions), FD_ATT_SPLIT=0|2 (never / always cut attention items along the keys),
+ * FD_TC_MAX_CTAS=n (cap on persistent CTAs).
  */
 #ifndef FLASHDIFF_H_
 #define FLASHDIFF_H_
@@ -149,6 +156,7 @@ fd_status fd_region_activity(fd_ctx* ctx, const float* z_cur, const float* z_pre
  *   x [B,N,H], cond [B,Hc], y [B,N,H], kv_cache [L,B,2,N,H]  of fd_config.dtype, 16-byte aligned
  *   labels [B,N] i32, mask [B,R] u8
  *   active_idx_out [B*N] i32 (capacity), cu_active_out [B+1] i32
+ * Needs 1 <= R <= N <= max_tokens, R <= max_regions, B <= max_batch; the i32 arrays 4-byte aligned.
  */
 fd_status fd_regional_step(fd_ctx* ctx, const void* x, const void* cond, const int32_t* labels,
                            const uint8_t* mask, int B, int N, int R, void* kv_cache, void* y,
@@ -239,8 +247,9 @@ fd_status fd_update_latent(fd_ctx* ctx, const fd_sampler_weights* sw, const floa
  *  - No cudaMalloc / cudaFree or any other allocating routine is called, by this function or the
  *    kernels it launches.
  *  - eta and max_skip_k take the place of the values a context would hold.
- *  - status_out: optional DEVICE int32 that receives 0, or FD_ERR_STATE if a label was outside
- *    [0,R] (such tokens are skipped), in stream order; may be NULL.
+ *  - status_out: optional DEVICE int32 that receives, in stream order, 0, FD_ERR_STATE if a label was
+ *    outside [0,R] (such tokens are skipped), or FD_ERR_TIMEOUT if a bounded wait of the streaming
+ *    reduction ran out (the result is then incomplete); may be NULL.
  */
 #define FD_NOALLOC_MAX_REGION_SLOTS 16384
 fd_status fd_region_activity_noalloc(const float* z_cur, const float* z_prev, const int32_t* labels, int B,
@@ -338,7 +347,9 @@ typedef struct {
 fd_status fd_rsearch_init(fd_rsearch* st, int r_min, int r_max, int r_start);
 fd_status fd_rsearch_update(fd_rsearch* st, double observed_perf, int32_t* next_r);
 
-/* Releases the context (host memory only; the workspace goes back to the caller). */
+/* Releases the context (host memory only; the workspace goes back to the caller).  Synchronises the
+ * device first and returns FD_OK, or a device-side status (FD_ERR_STATE / FD_ERR_TIMEOUT) that was
+ * recorded and never polled; the context is released either way. */
 fd_status fd_destroy(fd_ctx* ctx);
 
 /* Text of the last error of this context (host string owned by the context; NULL ctx: text of

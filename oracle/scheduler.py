@@ -12,8 +12,8 @@ Two policies of the paper's Patch Scheduler, restated for requests that share on
                 written out literally: for every candidate g the maximum over all g' is formed and
                 the candidate with the smallest maximum wins.  Readings where the paper is silent:
                 among candidates that tie on that maximum the monotask's *home* (the device that
-                already holds patches of the same request: "locality-aware", "co-locates dependent
-                regions") wins if it is one of them, otherwise the candidate with the smallest own
+                already holds patches of the same request; Sec. 4.3 "Monotask Packing" asks for
+                placement that respects locality) wins if it is one of them, otherwise the candidate with the smallest own
                 load, otherwise the smallest index.  A warm-up monotask has no home, so it goes to
                 the least loaded device, which is what the paper states for the warm-up phase.
 
@@ -25,8 +25,9 @@ Two policies of the paper's Patch Scheduler, restated for requests that share on
                 descending, arrival number ascending, index ascending); a request is taken if its
                 active tokens still fit into the token budget and its state is resident or a
                 residency slot is free (then it takes the slot); a request that does not fit is
-                passed over and lower-priority ones may use the leftover ("when a worker has
-                leftover resources it dispatches the highest-priority monotask").  The paper's
+                passed over and lower-priority ones may use the leftover (Sec. 4.3 "Efficient Patch
+                Switching with Monotasks": spare capacity goes to the best-ranked waiting
+                monotask).  The paper's
                 worker keeps at most two requests' state; here the bound is a parameter.  A
                 request without active tokens costs nothing and is taken if it is resident (its
                 step is a pure cached-drift update).

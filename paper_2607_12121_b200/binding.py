@@ -153,10 +153,12 @@ class Context:
         _check(None, st)
         self.handle = handle
 
-    def close(self):
+    def close(self) -> int:
+        st = FD_OK
         if getattr(self, "handle", None):
-            lib.fd_destroy(self.handle)
+            st = int(lib.fd_destroy(self.handle))
             self.handle = None
+        return st
 
     def __del__(self):
         try:
@@ -173,8 +175,9 @@ def fd_create(cfg: FdConfig, weights: Dict[str, "object"], device="cuda") -> Con
     return Context(cfg, weights, device)
 
 
-def fd_destroy(ctx: Context) -> None:
-    ctx.close()
+def fd_destroy(ctx: Context) -> int:
+    """Releases the context; returns FD_OK or a device-side status that was never polled."""
+    return ctx.close()
 
 
 def fd_partition_regions(ctx: Context, attn_map, R: int, labels_out, region_sizes_out=None, salient_cols=None,

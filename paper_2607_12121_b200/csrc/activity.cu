@@ -5,17 +5,22 @@
 // (fp32 within a run of tokens of one region, fp64 across runs and CTAs) and the token count.  Tokens of
 // regions whose change magnitude is frozen (skipped at the previous step) are not read at all.  Its main
 // form stages both operands through shared memory with bulk copies (below); rows wider than a ring
-// stage, unaligned rows and very large region counts take the plain-load forms.
+// stage take the plain vector-load form (per-CTA shared accumulators, up to ACT_SMEM_LIMIT / 12 regions);
+// unaligned rows, channel counts that are no multiple of 4 and larger region counts take the scalar form,
+// which adds straight into the global accumulators.
 // Kernel 2 (one CTA per request) turns the sums into delta, weights, mask and the next state, and
 // clears the accumulators for the next call.
 #include "common.cuh"
 #include "ptx.cuh"
+
+#include <mutex>
 
 namespace fd {
 
 namespace {
 
 constexpr int ACT_THREADS = 256;
+constexpr int ACT_SMEM_LIMIT = 200 * 1024;   // dynamic shared memory the reduction kernels may ask for
 
 // V = float4 vectors per token (D / 4).  GROUP = lanes that share one token.
 template <int UNROLL>
@@ -390,46 +395,78 @@ cudaError_t launch_attn_gate(const double* region_mass, const int32_t* region_si
     return cudaGetLastError();
 }
 
+namespace {
+
+// Per-device set-up of the reduction kernels, done once: the dynamic shared-memory ceiling is a property
+// of the function (not of a launch), so it is raised to the fixed upper bound here instead of to a
+// call-dependent value on every call, and the SM count is looked up once.
+constexpr int MAX_DEVICES = 64;
+std::mutex g_setup_mu;
+int g_sm_count[MAX_DEVICES];                // 0 = not set up yet
+
+cudaError_t activity_setup(int* sms) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_setup_mu);
+    if (!g_sm_count[dev]) {
+        int n = 0;
+        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(activity_reduce_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ACT_SMEM_LIMIT);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(activity_reduce_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, ACT_SMEM_LIMIT);
+        if (e != cudaSuccess) return e;
+        g_sm_count[dev] = n > 0 ? n : 148;
+    }
+    *sms = g_sm_count[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
 cudaError_t launch_activity(const float* z_cur, const float* z_prev, const int32_t* labels, int B, int N,
                             int D, int R, const float* eps, float* delta, int32_t* skip_count,
                             uint8_t* prev_active, float* score, float* weight, uint8_t* mask, float eta,
                             int K, double* acc_ss, int32_t* acc_cnt, Control* ctl, cudaStream_t st,
                             int* n_launch) {
+    int sms = 148;
+    cudaError_t es = activity_setup(&sms);
+    if (es != cudaSuccess) return es;
     const bool vec = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(z_cur) | reinterpret_cast<uintptr_t>(z_prev)) % 16 == 0);
-    const size_t bulk_smem = (size_t)BULK_FIXED_SMEM + (size_t)R * (sizeof(double) + sizeof(int32_t));
-    if (vec && D * 4 <= BULK_CHUNK_BYTES && bulk_smem <= 200 * 1024) {
+    const size_t acc_smem = (size_t)R * (sizeof(double) + sizeof(int32_t));
+    const size_t bulk_smem = (size_t)BULK_FIXED_SMEM + acc_smem;
+    if (vec && D * 4 <= BULK_CHUNK_BYTES && bulk_smem <= (size_t)ACT_SMEM_LIMIT) {
         const int V = D / 4;
         const int c_tok = BULK_CHUNK_BYTES / (D * 4);
         // three CTAs per SM fit (64 KB of ring each); every CTA gets one contiguous share of the B*N tokens, at
         // least four chunks so that the ring fills, in whole chunks
         const long long total = (long long)B * N;
-        int dev = 0, sms = 148;
-        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         const long long max_ctas = (long long)sms * 3;
         long long per = (total + max_ctas - 1) / max_ctas;
         if (per < 4LL * c_tok) per = 4LL * c_tok;
         per = (per + c_tok - 1) / c_tok * c_tok;
         const int grid = (int)((total + per - 1) / per);
-        cudaError_t ea = cudaFuncSetAttribute(activity_reduce_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk_smem);
-        if (ea != cudaSuccess) return ea;
         activity_reduce_bulk_kernel<<<grid, BULK_THREADS, bulk_smem, st>>>(
             reinterpret_cast<const char*>(z_cur), reinterpret_cast<const char*>(z_prev), labels, prev_active, B, N, V,
             R, c_tok, per, acc_ss, acc_cnt, ctl);
-    } else if (vec) {
+    } else if (vec && acc_smem <= (size_t)ACT_SMEM_LIMIT) {
         const int V = D / 4;
         // At least 32 KB of each operand per CTA (enough work to amortise set-up and the flush); for large
         // batches fewer, longer chunks: about 16 CTAs per SM in total keep every SM streaming without a long tail.
         const int by_size = (int)(((long long)N * V + 2047) / 2048);
-        const int by_sms = (148 * 16 + B - 1) / B;
+        const int by_sms = (sms * 16 + B - 1) / B;
         const int want = max(1, min(by_size, by_sms));
         const int tokens_per_cta = (N + want - 1) / want;
         const int chunks = (N + tokens_per_cta - 1) / tokens_per_cta;
         dim3 grid(chunks, B);
-        const size_t smem = (size_t)R * (sizeof(double) + sizeof(int32_t));
-        activity_reduce_kernel<4><<<grid, ACT_THREADS, smem, st>>>(
+        activity_reduce_kernel<4><<<grid, ACT_THREADS, acc_smem, st>>>(
             reinterpret_cast<const float4*>(z_cur), reinterpret_cast<const float4*>(z_prev), labels,
             prev_active, N, V, R, tokens_per_cta, acc_ss, acc_cnt, ctl);
     } else {
+        // any alignment, any channel count, any region count: one warp per token, sums added straight into the
+        // global accumulators
         dim3 grid(min(1024, (N + 7) / 8), B);
         activity_reduce_scalar_kernel<<<grid, ACT_THREADS, 0, st>>>(z_cur, z_prev, labels, prev_active, N,
                                                                     D, R, acc_ss, acc_cnt, ctl);
@@ -453,8 +490,8 @@ constexpr size_t NOALLOC_BYTES = sizeof(Control) + 192 /*keeps the arrays 256-by
                                  (size_t)FD_NOALLOC_MAX_REGION_SLOTS * (sizeof(double) + sizeof(int32_t));
 static __device__ __align__(256) unsigned char g_gate_scratch[NOALLOC_BYTES];
 
-constexpr int MAX_DEVICES = 64;
 void* g_scratch_addr[MAX_DEVICES];          // device address of g_gate_scratch, per device
+std::mutex g_scratch_mu;
 
 }  // namespace
 
@@ -466,15 +503,19 @@ cudaError_t noalloc_gate(const float* z_cur, const float* z_prev, const int32_t*
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
-    if (!g_scratch_addr[dev]) {
-        // In host code the array's name is only a handle; the address the kernels need comes from
-        // the runtime, looked up once per device while that device is current.
-        void* p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_gate_scratch);
-        if (e != cudaSuccess) return e;
-        g_scratch_addr[dev] = p;
+    unsigned char* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mu);
+        if (!g_scratch_addr[dev]) {
+            // In host code the array's name is only a handle; the address the kernels need comes from
+            // the runtime, looked up once per device while that device is current.
+            void* p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_gate_scratch);
+            if (e != cudaSuccess) return e;
+            g_scratch_addr[dev] = p;
+        }
+        base = static_cast<unsigned char*>(g_scratch_addr[dev]);
     }
-    unsigned char* base = static_cast<unsigned char*>(g_scratch_addr[dev]);
     Control* ctl = reinterpret_cast<Control*>(base);
     double* acc_ss = reinterpret_cast<double*>(base + 256);
     int32_t* acc_cnt = reinterpret_cast<int32_t*>(base + 256 + (size_t)FD_NOALLOC_MAX_REGION_SLOTS * sizeof(double));

@@ -129,6 +129,7 @@ struct fd_ctx {
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3) == 0; }
 
 template <typename T>
 fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* labels, const uint8_t* mask, int B,
@@ -475,6 +476,9 @@ static fd_status fd_regional_step_check(fd_ctx* c, const void* x, const void* co
     if (B > c->cfg.max_batch || N > c->cfg.max_tokens || R > c->cfg.max_regions)
         return c->fail(FD_ERR_SHAPE, "B=%d N=%d R=%d exceed the limits %d/%d/%d", B, N, R, c->cfg.max_batch,
                        c->cfg.max_tokens, c->cfg.max_regions);
+    if (R > N) return c->fail(FD_ERR_SHAPE, "R=%d exceeds N=%d", R, N);
+    if (!aligned4(labels) || !aligned4(active_idx_out) || !aligned4(cu_active_out))
+        return c->fail(FD_ERR_INVALID_ARG, "labels, active_idx_out, cu_active_out must be 4-byte aligned");
     return FD_OK;
 }
 
@@ -578,11 +582,26 @@ int64_t fd_launch_count(const fd_ctx* c) { return c ? c->launches : 0; }
 
 fd_status fd_destroy(fd_ctx* c) {
     if (!c) return FD_ERR_INVALID_ARG;
+    // Wait for whatever the context still has in flight (the workspace goes back to the caller), then report a
+    // device-side problem nobody has polled for yet.
+    fd_status pending = FD_OK;
+    Control h{};
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&h, c->ctl(), sizeof(Control), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) {
+        pending = FD_ERR_CUDA;
+        g_create_error = std::string("fd_destroy: ") + cudaGetErrorString(e);
+    } else if (h.status != 0) {
+        pending = static_cast<fd_status>(h.status);
+        char buf[128];
+        snprintf(buf, sizeof buf, "fd_destroy: unpolled device-side status %d, detail %d", h.status, h.detail);
+        g_create_error = buf;
+    }
     tc_plan_destroy(c->tc);
     for (auto& s : c->spans) { c->pool.push_back(s.a); c->pool.push_back(s.b); }
     for (cudaEvent_t ev : c->pool) cudaEventDestroy(ev);
     delete c;
-    return FD_OK;
+    return pending;
 }
 
 const char* fd_last_error(const fd_ctx* c) { return c ? c->err.c_str() : g_create_error.c_str(); }

@@ -10,6 +10,7 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    config.addinivalue_line("markers", "slow: many minutes of CPU oracle work; runs only with FD_SLOW=1")
 
 
 def pytest_collection_modifyitems(config, items):
@@ -18,6 +19,11 @@ def pytest_collection_modifyitems(config, items):
         has_gpu = torch.cuda.is_available()
     except Exception:  # pragma: no cover
         has_gpu = False
+    if os.environ.get("FD_SLOW", "0") != "1":
+        slow = pytest.mark.skip(reason="slow: set FD_SLOW=1")
+        for item in items:
+            if "slow" in item.keywords:
+                item.add_marker(slow)
     if has_gpu:
         return
     skip = pytest.mark.skip(reason="no CUDA device")

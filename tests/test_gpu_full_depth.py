@@ -1,0 +1,131 @@
+"""Parity over the whole block stack and over several gated steps: rounding must not build up across 24-30
+blocks at full width, and the K/V cache, the cached outputs and the gate state must stay in step with the oracle
+while regions are skipped, kept frozen and forced back on."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+import paper_2607_12121_b200 as fd
+from harness import StepBuffers, dev, gpu_step, host, labels_for, make_ctx, max_abs, rel_l2, tdtype
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, REL_L2 = 3e-2, 1e-2
+
+
+def _audio_full_depth(n_requests, n_gated):
+    """The audio configuration at its real width and depth (24 blocks, hidden 1536, 1024 tokens per request):
+    dense warm-up on the previous step's tokens, then gated steps; every element of y and of the K/V cache is compared."""
+    wl = gen.workload("audio").replace(B=n_requests)
+    B, N, H, L = wl.B, wl.N, wl.H, wl.L
+    labels = gen.uniform_labels(wl)
+    w = gen.block_weights(wl, 51)
+    inp = gen.step_inputs(wl, 51, labels)
+    ctx = make_ctx(wl, w)
+    buf = StepBuffers(wl, L)
+    dt = tdtype(wl)
+    kv_ref = np.zeros((L, B, 2, N, H), np.float32)
+    y_ref = np.zeros((B, N, H), np.float32)
+    rng = np.random.default_rng(51)
+    x_np = inp["x_prev"]
+    masks = [np.ones((B, wl.R), np.uint8)] + [gen.region_mask(wl, 60 + s, gen.request_fractions(wl, 60 + s))
+                                              for s in range(n_gated)]
+    for step, mask in enumerate(masks):
+        if step == 1:
+            x_np = inp["x_cur"]
+        elif step > 1:
+            x_np = gen.round_bf16(x_np + np.float32(0.01) * rng.standard_normal(x_np.shape).astype(np.float32))
+        y_before = host(buf.y)
+        idx, cu = gpu_step(ctx, wl, dev(x_np, dt), dev(inp["cond"], dt), dev(labels), dev(mask), buf)
+        o_idx, o_cu = oracle.regional_step(x_np, inp["cond"], labels, mask, w, kv_ref, y_ref, wl.heads, wl.R)
+        assert np.array_equal(idx, o_idx) and np.array_equal(cu, o_cu)
+        act = np.zeros(B * N, bool)
+        act[idx] = True
+        y = host(buf.y).reshape(B * N, H)
+        ma, rl = max_abs(y[act], y_ref.reshape(B * N, H)[act]), rel_l2(y[act], y_ref.reshape(B * N, H)[act])
+        print("audio x%d, %d blocks, step %d (%d active rows): y max_abs %.4f rel_l2 %.5f" % (B, L, step, idx.size, ma, rl))
+        assert ma <= MAX_ABS and rl <= REL_L2
+        assert np.array_equal(y[~act], y_before.reshape(B * N, H)[~act])
+        for l in (0, L // 2, L - 1):
+            got = host(buf.kv[l])
+            assert max_abs(got, kv_ref[l]) <= MAX_ABS and rel_l2(got, kv_ref[l]) <= REL_L2
+    assert fd.fd_destroy(ctx) == fd.FD_OK
+
+
+def test_audio_full_depth_full_width_two_requests():
+    _audio_full_depth(2, 1)
+
+
+@pytest.mark.slow
+def test_audio_full_depth_full_width_whole_batch():
+    """All 8 requests, warm-up + 2 gated steps: about 25 TFLOP of oracle work (ten minutes on 16 cores); runs
+    only when FD_SLOW=1."""
+    _audio_full_depth(8, 2)
+
+
+def test_video_twin_all_blocks_gated_steps_with_kv_kept():
+    """The video configuration's scaled-down twin, all 30 blocks: warm-up, then 6 steps whose masks come from the
+    gate (state carried from step to step, target fraction falling from 0.6 to 0.3, forced reactivation after 2
+    skipped steps), the K/V cache and the cached outputs kept across steps on both sides."""
+    wl = gen.workload("video_twin")
+    B, N, H, L, R, K = wl.B, wl.N, wl.H, wl.L, wl.R, 2
+    labels = labels_for(wl, 52)
+    w = gen.block_weights(wl, 52)
+    inp = gen.step_inputs(wl, 52, labels)
+    n_steps = 6
+    fr = np.linspace(0.6, 0.3, n_steps)
+    lat = gen.latent_sequence(wl, 52, labels, [[f] * B for f in fr])
+    ctx = make_ctx(wl, w, max_skip_k=K)
+    buf = StepBuffers(wl, L)
+    dt = tdtype(wl)
+    kv_ref = np.zeros((L, B, 2, N, H), np.float32)
+    y_ref = np.zeros((B, N, H), np.float32)
+    ost = oracle.initial_state(B, R)
+    delta = torch.zeros((B, R), dtype=torch.float32, device="cuda")
+    skip = torch.zeros((B, R), dtype=torch.int32, device="cuda")
+    prev = torch.ones((B, R), dtype=torch.uint8, device="cuda")
+    score = torch.empty((B, R), dtype=torch.float32, device="cuda")
+    weight = torch.empty((B, R), dtype=torch.float32, device="cuda")
+    mask_d = torch.empty((B, R), dtype=torch.uint8, device="cuda")
+    rng = np.random.default_rng(52)
+    x_np = inp["x_prev"]
+    gpu_step(ctx, wl, dev(x_np, dt), dev(inp["cond"], dt), dev(labels), dev(np.ones((B, R), np.uint8)), buf)
+    oracle.regional_step(x_np, inp["cond"], labels, np.ones((B, R), np.uint8), w, kv_ref, y_ref, wl.heads, R)
+    x_np = inp["x_cur"]
+    forced, fractions = False, []
+    for step in range(n_steps):
+        z = lat[step]
+        _, o_w, o_mask = oracle.activity_gate(z["z_cur"], z["z_prev"], labels, z["eps"], ost, R, K=K)
+        live = o_w > 0                                   # eps = 0 (target fraction 1) cannot sit on a weight
+        assert np.abs(o_w[live] / np.maximum(z["eps"][:, None], 1e-30).repeat(R, 1)[live] - 1).min() >= 1e-3
+        fd.fd_region_activity(ctx, dev(z["z_cur"]), dev(z["z_prev"]), dev(labels), R, dev(z["eps"]), delta, skip, prev,
+                              score, weight, mask_d)
+        assert np.array_equal(host(mask_d), o_mask), step
+        forced |= bool((o_mask.astype(bool) & (o_w < z["eps"][:, None])).any())
+        y_before, kv_before = host(buf.y), host(buf.kv[L - 1])
+        idx, cu = gpu_step(ctx, wl, dev(x_np, dt), dev(inp["cond"], dt), dev(labels), mask_d, buf)
+        o_idx, o_cu = oracle.regional_step(x_np, inp["cond"], labels, o_mask, w, kv_ref, y_ref, wl.heads, R)
+        assert np.array_equal(idx, o_idx) and np.array_equal(cu, o_cu)
+        fractions.append(idx.size / float(B * N))
+        act = np.zeros(B * N, bool)
+        act[idx] = True
+        y = host(buf.y).reshape(B * N, H)
+        yr = y_ref.reshape(B * N, H)
+        ma, rl = max_abs(y[act], yr[act]), rel_l2(y[act], yr[act])
+        print("video twin step %d: active fraction %.3f, y max_abs %.4f rel_l2 %.5f" % (step, fractions[-1], ma, rl))
+        assert ma <= MAX_ABS and rl <= REL_L2
+        assert np.array_equal(y[~act], y_before.reshape(B * N, H)[~act])
+        a2 = act.reshape(B, N)
+        for l in (0, L - 1):
+            got = host(buf.kv[l])
+            assert max_abs(got, kv_ref[l]) <= MAX_ABS and rel_l2(got, kv_ref[l]) <= REL_L2
+        got = host(buf.kv[L - 1])
+        for s in range(2):
+            assert np.array_equal(got[:, s][~a2], kv_before[:, s][~a2])
+        x_np = gen.round_bf16(x_np + np.float32(0.02) * rng.standard_normal(x_np.shape).astype(np.float32))
+    assert forced and min(fractions) < 0.6 and all(0 < f < 1 for f in fractions)
+    assert fd.fd_destroy(ctx) == fd.FD_OK

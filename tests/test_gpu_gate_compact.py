@@ -34,7 +34,8 @@ def _gate(ctx, wl, z_cur, z_prev, labels, eps, st):
 
 
 @pytest.mark.parametrize("name,seed", [("tiny", 0), ("audio_small", 1), ("image_small", 2), ("mmdit_small", 3),
-                                       ("video_small", 4), ("audio", 5), ("mmdit", 6), ("video", 7)])        # ... and full shapes
+                                       ("video_small", 4), ("audio", 5), ("mmdit", 6), ("video", 7),
+                                       ("image", 8)])                                        # ... and full shapes
 def test_gate_single_step(name, seed):
     wl = gen.workload(name)
     labels = labels_for(wl, seed)
@@ -135,6 +136,74 @@ def test_gate_streaming_kernel_edges():
     assert np.array_equal(host(st.skip), ost["skip_count"])
 
 
+def _eps_in_a_gap(weight):
+    """A threshold per request that sits in the widest relative gap between neighbouring weights of the
+    middle half of the sorted weights, so that no decision lands within 1e-3 of it."""
+    eps = np.empty(weight.shape[0], np.float32)
+    for b, w in enumerate(weight):
+        s = np.sort(w.astype(np.float64))
+        lo, hi = len(s) // 4, max(len(s) // 4 + 1, 3 * len(s) // 4)
+        k = lo + int(np.argmax(s[lo + 1:hi + 1] / np.maximum(s[lo:hi], 1e-300)))
+        eps[b] = np.float32(np.sqrt(s[k] * s[k + 1]))
+    return eps
+
+
+@pytest.mark.parametrize("B,N,D,R,via", [(2, 300, 2052, 9, "ctx"),            # rows wider than a ring stage
+                                         (2, 300, 2052, 9, "noalloc"),
+                                         (1, 24000, 8, 12000, "noalloc"),     # accumulators beyond the default shared-memory size
+                                         (1, 16400, 4, 16384, "noalloc"),     # the entry point's largest region count
+                                         (1, 20000, 4, 18000, "ctx")])        # accumulators beyond any shared-memory size
+def test_gate_reductions_beyond_the_streaming_form(B, N, D, R, via):
+    """Shapes the bulk-copy reduction does not take: the plain vector-load kernel with its per-CTA accumulators in
+    (opt-in sized) shared memory, and the one-warp-per-token kernel that adds straight into global memory."""
+    K, eta = 5, 1e-12
+    rng = np.random.default_rng(1000 + R + D)
+    labels = rng.integers(0, R + 1, size=(B, N)).astype(np.int32)
+    labels[:, : min(N, R)] = np.arange(min(N, R), dtype=np.int32)            # every region has at least one token
+    z_prev = rng.standard_normal((B, N, D)).astype(np.float32)
+    scale = (np.float32(10.0) ** rng.uniform(-3, -1, size=(B, R + 1)).astype(np.float32))
+    sc_tok = np.take_along_axis(scale, labels.astype(np.int64), axis=1)[..., None]
+    z_cur = (z_prev + sc_tok * rng.standard_normal((B, N, D)).astype(np.float32)).astype(np.float32)
+    frozen = rng.random((B, R)) < 0.1
+
+    def start_state():
+        st = oracle.initial_state(B, R)
+        st["prev_active"][frozen] = 0
+        st["delta"][frozen] = np.float32(0.01)
+        st["skip_count"][frozen] = 2
+        return st
+
+    probe = start_state()
+    _, w0, _ = oracle.activity_gate(z_cur, z_prev, labels, np.zeros(B, np.float32), probe, R, K=K, eta=eta)
+    eps = _eps_in_a_gap(w0)
+    ost = start_state()
+    o_score, o_weight, o_mask = oracle.activity_gate(z_cur, z_prev, labels, eps, ost, R, K=K, eta=eta)
+    assert np.abs(o_weight / eps[:, None] - 1).min() >= 1e-3
+    assert 0 < o_mask.sum() < B * R
+    st = GateState(B, R)
+    first = start_state()
+    st.delta.copy_(dev(first["delta"])); st.skip.copy_(dev(first["skip_count"])); st.prev.copy_(dev(first["prev_active"]))
+    if via == "noalloc":
+        status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        fd.fd_region_activity_noalloc(dev(z_cur), dev(z_prev), dev(labels), R, dev(eps), eta, K, st.delta, st.skip,
+                                      st.prev, st.score, st.weight, st.mask, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+    else:
+        wl = gen.workload("audio_small").replace(grid=(N,), B=B, R=R, D=D, L=1)
+        ctx = make_ctx(wl, gen.block_weights(wl, 1, n_blocks=1), n_blocks=1, engine=fd.FD_ENGINE_SIMT, max_skip_k=K,
+                       gate_eta=eta)
+        fd.fd_region_activity(ctx, dev(z_cur), dev(z_prev), dev(labels), R, dev(eps), st.delta, st.skip, st.prev,
+                              st.score, st.weight, st.mask)
+        fd.fd_poll_status(ctx)
+        assert fd.fd_destroy(ctx) == fd.FD_OK
+    assert np.array_equal(host(st.mask), o_mask)
+    np.testing.assert_allclose(host(st.score), o_score, rtol=1e-5, atol=0)
+    np.testing.assert_allclose(host(st.weight), o_weight, rtol=1e-5, atol=0)
+    assert np.array_equal(host(st.prev), ost["prev_active"])
+    assert np.array_equal(host(st.skip), ost["skip_count"])
+
+
 @pytest.mark.parametrize("name", ["tiny", "audio_small", "mmdit_small", "video_small"])
 def test_compaction_bit_exact(name):
     from harness import StepBuffers, gpu_step
@@ -166,3 +235,7 @@ def test_bad_label_is_reported_not_trapped():
         fd.fd_poll_status(ctx)
     assert ei.value.status == fd.FD_ERR_STATE
     fd.fd_poll_status(ctx)          # cleared; the context stays usable
+    # a status nobody polled for comes back from fd_destroy
+    fd.fd_region_activity(ctx, dev(lat["z_cur"]), dev(lat["z_prev"]), dev(labels), wl.R, dev(lat["eps"]), st.delta,
+                          st.skip, st.prev, st.score, st.weight, st.mask)
+    assert fd.fd_destroy(ctx) == fd.FD_ERR_STATE

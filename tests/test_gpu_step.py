@@ -125,6 +125,21 @@ def test_host_side_argument_errors():
     with pytest.raises(fd.FlashDiffError) as ei:
         fd.fd_regional_step(ctx, x, x, x, x, wl.R, buf.kv, buf.y, buf.active_idx, buf.cu_active)
     assert ei.value.status == fd.FD_ERR_SHAPE
+    # more regions than tokens; misaligned index arrays: refused on the host, nothing launched
+    small = torch.zeros((1, 8, wl.H), dtype=dt, device="cuda")
+    lab = torch.zeros((wl.B * wl.N + 1,), dtype=torch.int32, device="cuda")
+    n0 = ctx.launches
+    with pytest.raises(fd.FlashDiffError) as ei:
+        fd.fd_regional_step(ctx, small, small, lab, lab, 9, buf.kv, buf.y, buf.active_idx, buf.cu_active)
+    assert ei.value.status == fd.FD_ERR_SHAPE
+    xs = torch.zeros((wl.B, wl.N, wl.H), dtype=dt, device="cuda")
+    odd = lab.view(torch.uint8)[1:1 + 4 * wl.B * wl.N]          # an int32 array that starts on an odd byte
+    for args in ((odd, buf.active_idx, buf.cu_active), (lab, odd, buf.cu_active), (lab, buf.active_idx, odd)):
+        with pytest.raises(fd.FlashDiffError) as ei:
+            fd.fd_regional_step(ctx, xs, xs, args[0], lab, wl.R, buf.kv, buf.y, args[1], args[2])
+        assert ei.value.status == fd.FD_ERR_INVALID_ARG
+    assert ctx.launches == n0
+    assert fd.fd_destroy(ctx) == fd.FD_OK
     bad = fd.make_config(wl.replace(H=250))
     assert fd.fd_workspace_bytes(bad) == 0
 
@@ -186,13 +201,28 @@ def test_tensor_core_engine_switched_off_variants(monkeypatch, switch):
 
 
 @pytest.mark.parametrize("name,engine", [("audio_tc", fd.FD_ENGINE_TC), ("video_tc", fd.FD_ENGINE_TC),
-                                         ("audio_tc", fd.FD_ENGINE_SIMT)])
+                                         ("image_tc", fd.FD_ENGINE_TC), ("audio_tc", fd.FD_ENGINE_SIMT)])
 def test_peaked_attention_exercises_running_max(name, engine):
     """Query weights scaled by 64: scores spread over many e-folds, so the running maximum moves
     between key tiles and the accumulated output has to be rescaled."""
     wl = gen.workload(name)
     masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.5] * wl.B)]
     _run_sequence(wl, 4, engine, masks, qk_gain=64.0)
+
+
+@pytest.mark.parametrize("name,n_tok,max_ctas", [("image_tc", 520, "8"), ("image_tc", None, None), ("audio_tc", 700, "8"),
+                                                 ("wide_tc", None, "8")])
+def test_peaked_attention_with_items_cut_along_the_keys(monkeypatch, name, n_tok, max_ctas):
+    """Peaked softmax and forced key cuts together: the pieces of an item hold very different running maxima, so the
+    second kernel's rescaling of every piece decides the result (head dims 72, 64 and 128)."""
+    monkeypatch.setenv("FD_ATT_SPLIT", "2")
+    if max_ctas:
+        monkeypatch.setenv("FD_TC_MAX_CTAS", max_ctas)
+    wl = gen.workload(name)
+    if n_tok is not None:
+        wl = wl.replace(grid=(n_tok,), R=10, L=1)
+    masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.6] * wl.B)]
+    _run_sequence(wl, 4, fd.FD_ENGINE_TC, masks, qk_gain=64.0)
 
 
 def test_bounded_wait_reports_timeout_and_context_stays_usable():

@@ -156,3 +156,29 @@ def test_affine_change_of_the_map_keeps_the_partition():
     a = P.partition_request(S, 5)
     b = P.partition_request((S * np.float32(4.0) + np.float32(8.0)).astype(np.float32), 5)
     assert np.array_equal(a, b)
+
+
+def test_hand_worked_three_region_cases_pin_which_side_gets_r_f():
+    """Sec. 4.1 allocation rule worked by hand: the FOCUS side (saliency >= threshold) hosts
+    r_f = argmin_r |r - R n_f / (n_f + n_c)| regions, the context side the rest.
+
+    Case 1: saliency 0,0,0,0,1,1 and R = 3.  The only threshold separates {4,5} (focus, n_f = 2) from {0..3}
+    (context, n_c = 4); R n_f / n = 1, so r_f = 1 and r_c = 2: the focus stays whole, the context (all values equal,
+    no further threshold) is chopped in index order into {0,1} and {2,3}.  Giving r_f to the wrong side would keep
+    the context whole and split the focus instead.
+    Case 2: five tokens at 0, then 0.9, 1.0, 0.9, 1.0 and R = 3.  Otsu separates the zeros (n_c = 5) from the rest
+    (n_f = 4); R n_f / n = 4/3, so r_f = 1 (distance 1/3 against 2/3 for r = 2) and r_c = 2: focus {5,6,7,8} is one
+    region, the zeros are chopped into {0,1,2} and {3,4}.  The wrong side would give {0..4}, {5,7}, {6,8}.
+    Case 3: the mirror image of case 1 with the large side in focus: saliency 1,1,1,1,0,0 gives n_f = 4, n_c = 2,
+    R n_f / n = 2, r_f = 2: the focus is chopped into {0,1}, {2,3} and the context {4,5} stays whole."""
+    def run(values, R):
+        S = np.asarray(values, np.float32)
+        lab, sizes = oracle.partition(S.reshape(1, -1, 1), None, R)
+        return lab[0].tolist(), sizes[0].tolist()
+
+    assert run([0, 0, 0, 0, 1, 1], 3) == ([0, 0, 1, 1, 2, 2], [2, 2, 2])
+    assert run([0, 0, 0, 0, 0, 0.9, 1.0, 0.9, 1.0], 3) == ([0, 0, 0, 1, 1, 2, 2, 2, 2], [3, 2, 4])
+    assert run([1, 1, 1, 1, 0, 0], 3) == ([0, 0, 1, 1, 2, 2], [2, 2, 2])
+    # the same rule one level down: 12 tokens, two loud ones, R = 4 -> r_f = argmin |r - 4*2/12| = 1
+    lab, sizes = run([0] * 10 + [1, 1], 4)
+    assert lab == [0, 0, 0, 0, 1, 1, 1, 2, 2, 2, 3, 3] and sizes == [4, 3, 3, 2]

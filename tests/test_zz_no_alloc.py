@@ -1,4 +1,4 @@
-"""The allocation-free gate entry point against the regular one.
+"""The allocation-free gate entry point against the regular one and against the CPU oracle.
 
 fd_region_activity_noalloc serves callers that may not allocate device memory (a plug-in inside a
 server with a frozen memory pool, a latency-critical thread, a process whose arena already owns
@@ -11,6 +11,7 @@ import pytest
 import torch
 
 import gen
+import oracle
 import paper_2607_12121_b200 as fd
 from harness import dev, host, make_ctx
 
@@ -35,6 +36,7 @@ def test_noalloc_gate_matches_regular_gate_on_two_calls_in_a_row():
                    gate_eta=eta)
     labels = dev(labels_np)
     ref, got = _State(wl.B, wl.R), _State(wl.B, wl.R)
+    ost = oracle.initial_state(wl.B, wl.R)          # the oracle carries its own state through the same two calls
     status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
     # two different problems back to back: the second call must not see the first call's sums
     for call, (seed, fr) in enumerate([(11, [0.25, 0.5, 0.75]), (12, [0.6, 0.3, 0.45])]):
@@ -53,6 +55,12 @@ def test_noalloc_gate_matches_regular_gate_on_two_calls_in_a_row():
         assert np.array_equal(host(got.skip), host(ref.skip))
         assert np.array_equal(host(got.prev), host(ref.prev))
         assert np.array_equal(host(got.delta), host(got.score))
+        o_score, o_weight, o_mask = oracle.activity_gate(lat["z_cur"], lat["z_prev"], labels_np, lat["eps"], ost, wl.R,
+                                                         K=K, eta=eta)
+        assert np.array_equal(host(got.mask), o_mask), call
+        np.testing.assert_allclose(host(got.score), o_score, rtol=1e-5, atol=0)
+        np.testing.assert_allclose(host(got.weight), o_weight, rtol=1e-5, atol=0)
+        assert np.array_equal(host(got.skip), ost["skip_count"])
         assert 0 < host(got.mask).sum() < wl.B * wl.R
 
 
