@@ -3,10 +3,14 @@
 
 A "step" is one pass of the whole hot path over one ragged batch of synthetic requests:
 gate (activity score + mask) -> compaction -> all transformer blocks on the active tokens.
-Default workload: the audio-latent configuration (24 blocks, hidden 1536, 8 concurrent requests
-of 1024 tokens, per-request active fraction ~U[0.2,0.8]).
+Headline workload: the 480p video configuration (30 blocks, hidden 1536, 12 heads x 128, 32760 tokens,
+256 regions), the largest one that fits a single GPU.  With one GPU the audio, image and joint text-image
+configurations are measured as well (step, dense step, per-kernel rates) and the active fraction is swept;
+all of it lands inside the line's `roofline` object.
 
   python bench.py --gpus 1 --steps 20 --warmup 5
+  python bench.py --gpus 4                 # starts 4 replicas (one process per GPU) by itself
+  python bench.py --workload audio --also ""   # one workload only
   python bench.py --impl reference        # the CPU oracle on the host cores (bounded sample)
 """
 from __future__ import annotations
@@ -200,6 +204,17 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
+DEFAULT_FRACTION = {"image": 0.5, "mmdit": 0.55, "video": 0.45}
+# active-fraction sweeps: the image and joint text-image configurations at their stated fractions, the video
+# configuration at steps 0/12/25/37/49 of its 50-step schedule (fraction falling linearly from 0.6 to 0.3)
+SWEEPS = {
+    "image": [("f0.25", 0.25), ("f0.50", 0.5), ("f0.75", 0.75), ("f1.00", 1.0)],
+    "mmdit": [("f0.34", 0.34), ("f0.55", 0.55), ("f0.76", 0.76), ("f1.00", 1.0)],
+    "video": [("step%d" % s, 0.6 - 0.3 * s / 49.0) for s in (0, 12, 25, 37, 49)],
+}
+CONTRACTIONS = ("gemm_qkv", "attention", "gemm_out", "gemm_fc1", "gemm_fc2")
+
+
 def device_weights(wl, seed, device):
     """Weights ~N(0, 0.02) drawn on the device (the full stacks are 1-2 GB): same recipe as the
     numpy generator, different stream."""
@@ -220,6 +235,207 @@ def device_weights(wl, seed, device):
     return out
 
 
+def dram_traffic(workload, kernel):
+    """DRAM bytes per launch of `kernel` on `workload` from the ncu capture summarised under profiles/ (a text
+    table; a profiler cannot run inside the benchmark).  None when no capture of that pair exists."""
+    tp = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.txt")
+    if not os.path.exists(tp):
+        return None
+    with open(tp) as f:
+        for ln in f:
+            parts = ln.split()
+            if len(parts) == 3 and parts[0] == workload and parts[1] == kernel:
+                return int(parts[2])
+    return None
+
+
+class Engine:
+    """One workload resident on the device: weights, context, labels, inputs, caches, gate state."""
+
+    def __init__(self, name, seed, dev, rep, blocks=0):
+        import torch
+        import gen
+        import paper_2607_12121_b200 as fd
+        from paper_2607_12121_b200 import replicas
+        self.torch, self.gen, self.fd, self.replicas = torch, gen, fd, replicas
+        self.rep, self.dev, self.seed = rep, dev, seed
+        wl = gen.workload(name)
+        if blocks:
+            wl = wl.replace(L=blocks)
+        self.wl = wl
+        self.dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+        B, N, H, R, L = wl.B, wl.N, wl.H, wl.R, wl.L
+        self.weights = device_weights(wl, seed, dev)
+        self.ctx = fd.fd_create(fd.make_config(wl), self.weights, device=dev)
+        if wl.labels == "partition":
+            # labels come from the library's own partitioner on the synthetic early-step attention map
+            amap = torch.from_numpy(gen.saliency_map(wl, seed)).to(dev)
+            lab_grid = torch.empty((B, wl.n_grid), dtype=torch.int32, device=dev)
+            fd.fd_partition_regions(self.ctx, amap, R, lab_grid, None, None, wl.m_min, wl.m_max)
+            fd.fd_poll_status(self.ctx)
+            labels_np = np.concatenate([lab_grid.cpu().numpy(), np.full((B, wl.n_text), R, np.int32)], axis=1)
+            self.labels_np = np.ascontiguousarray(labels_np)
+        else:
+            self.labels_np = gen.uniform_labels(wl)
+        inp = gen.step_inputs(wl, seed, self.labels_np)
+        self.h_x, self.h_xprev, self.h_cond = (self.pin(inp[k], self.dt) for k in ("x_cur", "x_prev", "cond"))
+        self.x, self.x_prev, self.cond = self.h_x.to(dev), self.h_xprev.to(dev), self.h_cond.to(dev)
+        self.labels = torch.from_numpy(self.labels_np).to(dev)
+        self.ones = torch.ones((B, R), dtype=torch.uint8, device=dev)
+        self.kv = torch.zeros((L, B, 2, N, H), dtype=self.dt, device=dev)
+        self.y = torch.zeros((B, N, H), dtype=self.dt, device=dev)
+        self.active_idx = torch.zeros(B * N, dtype=torch.int32, device=dev)
+        self.cu_active = torch.zeros(B + 1, dtype=torch.int32, device=dev)
+        self.delta = torch.zeros((B, R), dtype=torch.float32, device=dev)
+        self.skip = torch.zeros((B, R), dtype=torch.int32, device=dev)
+        self.prev = torch.ones((B, R), dtype=torch.uint8, device=dev)
+        self.score = torch.empty((B, R), dtype=torch.float32, device=dev)
+        self.weight = torch.empty((B, R), dtype=torch.float32, device=dev)
+        self.mask = torch.empty((B, R), dtype=torch.uint8, device=dev)
+        self.dense_step(self.x_prev)          # dense warm-up on the previous step's tokens fills kv / y
+
+    def pin(self, a, tdt=None):
+        t = self.torch.from_numpy(np.ascontiguousarray(a))
+        if tdt is not None:
+            t = t.to(tdt)
+        return t.pin_memory()
+
+    def set_fraction(self, fraction=None):
+        """Latents of two neighbouring steps whose gate lets `fraction` of every request's regions through
+        (None: the workload's default; audio: one draw ~U[0.2,0.8] per request)."""
+        wl = self.wl
+        if fraction is not None:
+            fr = np.full(wl.B, fraction)
+        elif wl.name in DEFAULT_FRACTION:
+            fr = np.full(wl.B, DEFAULT_FRACTION[wl.name])
+        else:
+            fr = self.gen.request_fractions(wl, self.seed)
+        lat = self.gen.latent_pair(wl, self.seed, self.labels_np, fractions=fr)
+        self.h_zc, self.h_zp, self.h_eps = self.pin(lat["z_cur"]), self.pin(lat["z_prev"]), self.pin(lat["eps"])
+        self.z_cur, self.z_prev, self.eps = self.h_zc.to(self.dev), self.h_zp.to(self.dev), self.h_eps.to(self.dev)
+
+    def dense_step(self, src=None):
+        self.fd.fd_regional_step(self.ctx, self.x if src is None else src, self.cond, self.labels, self.ones, self.wl.R,
+                                 self.kv, self.y, self.active_idx, self.cu_active)
+
+    def gated_step(self, xin=None, zc=None, zp=None, ep=None, cd=None):
+        # fresh gate state: every timed step sees the same "first gated step after the warm-up"
+        self.delta.zero_(); self.skip.zero_(); self.prev.fill_(1)
+        fd = self.fd
+        fd.fd_region_activity(self.ctx, self.z_cur if zc is None else zc, self.z_prev if zp is None else zp, self.labels,
+                              self.wl.R, self.eps if ep is None else ep, self.delta, self.skip, self.prev, self.score,
+                              self.weight, self.mask)
+        fd.fd_regional_step(self.ctx, self.x if xin is None else xin, self.cond if cd is None else cd, self.labels,
+                            self.mask, self.wl.R, self.kv, self.y, self.active_idx, self.cu_active)
+
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        self.replicas.barrier(self.rep)
+        self.torch.cuda.synchronize()
+
+    def timed(self, fn, steps):
+        """Milliseconds per call: CUDA events on the launching stream, barrier + synchronize on both sides, the
+        slowest replica's time."""
+        torch = self.torch
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        self.barrier()
+        return self.replicas.max_over_ranks(self.rep, e0.elapsed_time(e1), self.dev) / steps
+
+    def active(self):
+        self.fd.fd_poll_status(self.ctx)
+        cu = self.cu_active.cpu().numpy()
+        return np.diff(cu).astype(np.int64), int(cu[-1])
+
+    def kernel_table(self, steps, A_b, peaks):
+        """Per-kernel rates from a profiled pass of `steps` gated steps (CUDA events the library records around every
+        kernel group on the caller's stream)."""
+        fd, wl = self.fd, self.wl
+        B, N, H, M, L, D = wl.B, wl.N, wl.H, wl.M, wl.L, wl.D
+        A = int(sum(A_b))
+        fd.fd_profile_enable(self.ctx, True)
+        self.barrier()
+        for _ in range(steps):
+            self.gated_step()
+        prof = fd.fd_profile_read(self.ctx)
+        fd.fd_profile_enable(self.ctx, False)
+        fl = block_flops(A_b, N, H, M)
+        es = 2 if wl.dtype == "bf16" else 4
+        bytes_per_launch = {"ln_modulate": A * H * (4 + es), "adaln": L * 6 * H * wl.Hc * es,
+                            "activity": 2.0 * 4 * D * float(N * B), "compact": 4.0 * B * N + 4.0 * A}
+        total_ms = sum(v[0] for v in prof.values()) or 1.0
+        burst, sust, hbm = float(peaks["bf16_tflops"]), float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])), float(peaks["hbm_gbs"])
+        table = {}
+        for k, (ms, cnt) in prof.items():
+            if cnt == 0:
+                continue
+            per_step = L if k.startswith("gemm") or k == "attention" else (2 * L if k == "ln_modulate" else 1)
+            us = ms / (steps * per_step) * 1e3
+            ent = {"ms_per_step": round(ms / steps, 4), "share": round(ms / total_ms, 4), "calls_per_step": per_step,
+                   "avg_call_us": round(us, 2)}
+            if k in fl:
+                tf = fl[k] / (us * 1e-6) / 1e12
+                ent.update(tflops=round(tf, 1), frac_burst=round(tf / burst, 3), frac_sustained=round(tf / sust, 3),
+                           flops_per_launch=fl[k])
+            elif k in bytes_per_launch:
+                gbs = bytes_per_launch[k] / (us * 1e-6) / 1e9
+                ent.update(gbs=round(gbs, 1), frac_hbm=round(gbs / hbm, 3), bytes_per_launch=bytes_per_launch[k])
+            table[k] = ent
+        return table
+
+    def measure(self, steps, warmup, peaks, fraction=None, kernels=True, dense_ms=None):
+        """Gated step, the same engine's dense step, and (optionally) the per-kernel table at one active fraction."""
+        wl = self.wl
+        self.set_fraction(fraction)
+        for _ in range(max(warmup, 3)):
+            self.gated_step()
+        A_b, A = self.active()
+        f_tok = A / float(wl.B * wl.N)
+        ms_reg = self.timed(self.gated_step, steps)
+        if dense_ms is None:
+            for _ in range(2):
+                self.dense_step()
+            dense_ms = self.timed(self.dense_step, max(3, steps // 2))
+            self.dense_step(self.x_prev)                    # restore the cached state the gated step expects
+        fl = block_flops(A_b, wl.N, wl.H, wl.M)
+        step_flops = wl.L * sum(fl.values())
+        dense_flops = wl.L * sum(block_flops([wl.N] * wl.B, wl.N, wl.H, wl.M).values())
+        out = {"active_tokens": A, "active_fraction": round(f_tok, 4), "step_ms": round(ms_reg, 4),
+               "dense_step_ms": round(dense_ms, 4), "tflops": round(step_flops / (ms_reg * 1e-3) / 1e12, 1),
+               "dense_tflops": round(dense_flops / (dense_ms * 1e-3) / 1e12, 1),
+               "speedup_vs_dense": round(dense_ms / ms_reg, 3),
+               "t_over_f_dense": round(ms_reg / (f_tok * dense_ms), 3)}
+        if kernels:
+            out["kernels"] = self.kernel_table(steps, A_b, peaks)
+        return out, A_b, step_flops
+
+    def close(self):
+        st = self.fd.fd_destroy(self.ctx)
+        self.__dict__.clear()                 # drops the weights, caches and inputs
+        return st
+
+
+def side_workload(name, seed, dev, rep, steps, warmup, peaks):
+    """Step, dense step, per-kernel table and the fraction sweep of a workload that is not the headline."""
+    import torch
+    eng = Engine(name, seed, dev, rep)
+    res, _, _ = eng.measure(steps, warmup, peaks)
+    sweep = {}
+    for tag, f in SWEEPS.get(name, []):
+        r, _, _ = eng.measure(max(5, steps // 2), 3, peaks, fraction=f, kernels=False, dense_ms=res["dense_step_ms"])
+        sweep[tag] = {k: r[k] for k in ("active_fraction", "step_ms", "tflops", "speedup_vs_dense", "t_over_f_dense")}
+    if sweep:
+        res["sweep"] = sweep
+    eng.close()
+    del eng
+    torch.cuda.empty_cache()
+    return res
+
+
 def run_ours(args):
     import torch
     import gen
@@ -231,127 +447,43 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     replicas.init(rep, "nccl", dev)
+    peaks, peak_kind = load_peaks()
 
-    wl = gen.workload(args.workload)
-    if args.blocks:
-        wl = wl.replace(L=args.blocks)
     seed = replicas.replica_seed(rep, args.seed)     # every rank owns its own batch of requests (weak scaling)
-    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    eng = Engine(args.workload, seed, dev, rep, blocks=args.blocks)
+    wl, ctx, dt = eng.wl, eng.ctx, eng.dt
     B, N, H, M, R, L, D = wl.B, wl.N, wl.H, wl.M, wl.R, wl.L, wl.D
-    default_fraction = {"image": 0.5, "mmdit": 0.55, "video": 0.45}
-
-    weights = device_weights(wl, seed, dev)
-    cfg = fd.make_config(wl)
-    ctx = fd.fd_create(cfg, weights, device=dev)
-
-    if wl.labels == "partition":
-        # labels come from the library's own partitioner on the synthetic early-step attention map
-        amap = torch.from_numpy(gen.saliency_map(wl, seed)).to(dev)
-        lab_grid = torch.empty((B, wl.n_grid), dtype=torch.int32, device=dev)
-        fd.fd_partition_regions(ctx, amap, R, lab_grid, None, None, wl.m_min, wl.m_max)
-        fd.fd_poll_status(ctx)
-        labels_np = np.concatenate([lab_grid.cpu().numpy(), np.full((B, wl.n_text), R, np.int32)], axis=1)
-        labels_np = np.ascontiguousarray(labels_np)
-    else:
-        labels_np = gen.uniform_labels(wl)
-    inp = gen.step_inputs(wl, seed, labels_np)
-    if args.fraction is not None:
-        fr = np.full(B, args.fraction)
-    elif wl.name in default_fraction:
-        fr = np.full(B, default_fraction[wl.name])
-    else:
-        fr = gen.request_fractions(wl, seed)
-    lat = gen.latent_pair(wl, seed, labels_np, fractions=fr)
-
-    def pin(a, tdt=None):
-        t = torch.from_numpy(np.ascontiguousarray(a))
-        if tdt is not None:
-            t = t.to(tdt)
-        return t.pin_memory()
-
-    h_x, h_xprev, h_cond = pin(inp["x_cur"], dt), pin(inp["x_prev"], dt), pin(inp["cond"], dt)
-    h_zc, h_zp, h_eps = pin(lat["z_cur"]), pin(lat["z_prev"]), pin(lat["eps"])
-    x, x_prev, cond = h_x.to(dev), h_xprev.to(dev), h_cond.to(dev)
-    z_cur, z_prev, eps = h_zc.to(dev), h_zp.to(dev), h_eps.to(dev)
-    labels = torch.from_numpy(labels_np).to(dev)
-    ones = torch.ones((B, R), dtype=torch.uint8, device=dev)
-    kv = torch.zeros((L, B, 2, N, H), dtype=dt, device=dev)
-    y = torch.zeros((B, N, H), dtype=dt, device=dev)
-    h_y = torch.empty((B, N, H), dtype=dt).pin_memory()
-    active_idx = torch.zeros(B * N, dtype=torch.int32, device=dev)
-    cu_active = torch.zeros(B + 1, dtype=torch.int32, device=dev)
-    delta = torch.zeros((B, R), dtype=torch.float32, device=dev)
-    skip = torch.zeros((B, R), dtype=torch.int32, device=dev)
-    prev = torch.ones((B, R), dtype=torch.uint8, device=dev)
-    score = torch.empty((B, R), dtype=torch.float32, device=dev)
-    weight = torch.empty((B, R), dtype=torch.float32, device=dev)
-    mask = torch.empty((B, R), dtype=torch.uint8, device=dev)
-
-    def dense_step(src):
-        fd.fd_regional_step(ctx, src, cond, labels, ones, R, kv, y, active_idx, cu_active)
-
-    def gated_step(xin=None, zc=None, zp=None, ep=None, cd=None):
-        # fresh gate state: every timed step sees the same "first gated step after the warm-up"
-        delta.zero_(); skip.zero_(); prev.fill_(1)
-        fd.fd_region_activity(ctx, z_cur if zc is None else zc, z_prev if zp is None else zp, labels, R,
-                              eps if ep is None else ep, delta, skip, prev, score, weight, mask)
-        fd.fd_regional_step(ctx, x if xin is None else xin, cond if cd is None else cd, labels, mask, R, kv, y,
-                            active_idx, cu_active)
-
-    def barrier():
-        torch.cuda.synchronize()
-        replicas.barrier(rep)
-        torch.cuda.synchronize()
-
-    def timed(fn, steps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
-            fn()
-        e1.record()
-        barrier()
-        ms = replicas.max_over_ranks(rep, e0.elapsed_time(e1), dev)
-        return ms / steps
-
-    # warm-up: one dense step on the previous step's tokens fills kv / y, then W gated steps
-    dense_step(x_prev)
+    eng.set_fraction(args.fraction)
     for _ in range(max(args.warmup, 3)):
-        gated_step()
-    fd.fd_poll_status(ctx)
-    cu = cu_active.cpu().numpy()
-    A_b = np.diff(cu).astype(np.int64)
-    A = int(cu[-1])
+        eng.gated_step()
+    A_b, A = eng.active()
     f_tok = A / float(B * N)
 
     sampler = ClockSampler(local)
     sampler.start()
     launches0 = ctx.launches
-    ms_reg = timed(gated_step, args.steps)
+    ms_reg = eng.timed(eng.gated_step, args.steps)
     launches = ctx.launches - launches0
     clocks = sampler.stop()
 
     # the same engine's dense step (mask of ones) and the per-kernel breakdown
     for _ in range(2):
-        dense_step(x)
-    ms_dense = timed(lambda: dense_step(x), max(3, args.steps // 2))
-    dense_step(x_prev)                         # restore the cached state the gated step expects
-    fd.fd_profile_enable(ctx, True)
-    barrier()
-    for _ in range(args.steps):
-        gated_step()
-    prof = fd.fd_profile_read(ctx)
-    fd.fd_profile_enable(ctx, False)
+        eng.dense_step()
+    ms_dense = eng.timed(eng.dense_step, max(3, args.steps // 2))
+    eng.dense_step(eng.x_prev)                         # restore the cached state the gated step expects
+    breakdown = eng.kernel_table(args.steps, A_b, peaks)
 
     # End to end through the C-ABI with host buffers: every step's inputs come from pinned host memory and its
     # result y goes back to pinned host memory, all inside the timed region.  The copies run on their own
     # streams, double-buffered, the way a serving loop would run them: the upload of step i+1 and the download
     # of step i-1 overlap the kernels of step i (y itself is state the next step updates in place, so a step
     # first snapshots it into a staging buffer with a device copy).
+    x, cond, y, z_cur, z_prev, eps = eng.x, eng.cond, eng.y, eng.z_cur, eng.z_prev, eng.eps
     cur = torch.cuda.current_stream()
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
     d_in = [[torch.empty_like(t) for t in (x, cond, z_cur, z_prev, eps)] for _ in range(2)]
-    h_in = (h_x, h_cond, h_zc, h_zp, h_eps)
+    h_in = (eng.h_x, eng.h_cond, eng.h_zc, eng.h_zp, eng.h_eps)
+    h_y = torch.empty((B, N, H), dtype=dt).pin_memory()
     y_stage = [torch.empty_like(y) for _ in range(2)]
     h_ys = [h_y, torch.empty_like(h_y).pin_memory()]
     in_ready = [torch.cuda.Event() for _ in range(2)]
@@ -372,7 +504,7 @@ def run_ours(args):
             in_ready[sl].record(s_in)
         cur.wait_event(in_ready[sl])
         dx, dc, dzc, dzp, dep = d_in[sl]
-        gated_step(dx, dzc, dzp, dep, dc)
+        eng.gated_step(dx, dzc, dzp, dep, dc)
         in_free[sl].record(cur)
         if i >= 2:
             cur.wait_event(out_done[sl])                     # the staging buffer's previous download has finished
@@ -386,7 +518,7 @@ def run_ours(args):
             out_done[sl ^ 1].synchronize()                   # the host has the previous step's result
 
     def e2e_run(steps):
-        barrier()
+        eng.barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
@@ -394,24 +526,15 @@ def run_ours(args):
         last = (e2e_i[0] - 1) & 1
         cur.wait_event(out_done[last])                       # the last result is on the host when the clock stops
         e1.record()
-        barrier()
+        eng.barrier()
         return replicas.max_over_ranks(rep, e0.elapsed_time(e1), dev) / steps
 
     e2e_run(2)
     ms_e2e = e2e_run(args.steps)
-    h2d = sum(t.numel() * t.element_size() for t in (h_x, h_cond, h_zc, h_zp, h_eps))
+    h2d = sum(t.numel() * t.element_size() for t in h_in)
     d2h = h_y.numel() * h_y.element_size()
     fd.fd_poll_status(ctx)
-
-    # sampler closure around the step (outside the timed step, which is the hot path alone): patch embedding of all
-    # tokens, final layer on the active rows, latent update; timed with CUDA events on the same shapes
-    sw_np = gen.sampler_weights(wl, seed)
-    sw_dev = {k: torch.from_numpy(v).to(dev).to(dt) for k, v in sw_np.items()}
-    sw = fd.make_sampler_weights(sw_dev, D)
-    s_drift = torch.zeros((B, N, D), dtype=torch.float32, device=dev)
-    s_zn = torch.empty((B, N, D), dtype=torch.float32, device=dev)
-    s_x = torch.empty((B, N, H), dtype=dt, device=dev)
-    s_h = torch.full((B,), 0.02, dtype=torch.float32, device=dev)
+    del d_in, y_stage
 
     def time_us(fn, reps=10):
         for _ in range(2):
@@ -425,42 +548,53 @@ def run_ours(args):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / reps * 1e3
 
-    emb_us = time_us(lambda: fd.fd_embed_latent(ctx, sw, z_cur, s_x))
-    upd_us = time_us(lambda: fd.fd_update_latent(ctx, sw, z_cur, y, active_idx, cu_active, s_h, s_drift, s_zn))
-    es = 2 if dt == torch.bfloat16 else 4
-    emb_bytes = B * N * (D * 4 + H * es) + N * H * es
-    upd_bytes = A * (H * es + D * 4) + 3 * B * N * D * 4
-    sampler = {"embed_us": emb_us, "embed_gbs": emb_bytes / emb_us / 1e3, "update_us": upd_us,
-               "update_gbs": upd_bytes / upd_us / 1e3, "note": "outside the timed step; algorithmic bytes / CUDA-event time"}
-    fd.fd_poll_status(ctx)
+    extras = {}
+    if not args.no_extras:
+        # sampler closure around the step (outside the timed step, which is the hot path alone): patch embedding of all
+        # tokens, final layer on the active rows, latent update; timed with CUDA events on the same shapes
+        sw_np = gen.sampler_weights(wl, seed)
+        sw_dev = {k: torch.from_numpy(v).to(dev).to(dt) for k, v in sw_np.items()}
+        sw = fd.make_sampler_weights(sw_dev, D)
+        s_drift = torch.zeros((B, N, D), dtype=torch.float32, device=dev)
+        s_zn = torch.empty((B, N, D), dtype=torch.float32, device=dev)
+        s_x = torch.empty((B, N, H), dtype=dt, device=dev)
+        s_h = torch.full((B,), 0.02, dtype=torch.float32, device=dev)
+        emb_us = time_us(lambda: fd.fd_embed_latent(ctx, sw, z_cur, s_x))
+        upd_us = time_us(lambda: fd.fd_update_latent(ctx, sw, z_cur, y, eng.active_idx, eng.cu_active, s_h, s_drift, s_zn))
+        es = 2 if dt == torch.bfloat16 else 4
+        emb_bytes = B * N * (D * 4 + H * es) + N * H * es
+        upd_bytes = A * (H * es + D * 4) + 3 * B * N * D * 4
+        extras["sampler"] = {"embed_us": emb_us, "embed_gbs": emb_bytes / emb_us / 1e3, "update_us": upd_us,
+                             "update_gbs": upd_bytes / upd_us / 1e3,
+                             "note": "outside the timed step; algorithmic bytes / CUDA-event time"}
+        fd.fd_poll_status(ctx)
 
-    # the paper's own gate signal (Sec. 4.2): extra cost of collecting the first block's own-region attention mass
-    # inside the step, and the gate evaluated on it (outside the timed step, whose gate is the latent-change one)
-    mass = torch.zeros((B, R), dtype=torch.float64, device=dev)
-    sizes = torch.from_numpy(np.stack([np.bincount(l[l < R], minlength=R) for l in labels_np]).astype(np.int32)).to(dev)
-    g_rbar = torch.zeros((B, R), dtype=torch.float32, device=dev)
-    g_imp = torch.empty((B, R), dtype=torch.float32, device=dev)
+        # the paper's own gate signal (Sec. 4.2): extra cost of collecting the first block's own-region attention mass
+        # inside the step, and the gate evaluated on it (outside the timed step, whose gate is the latent-change one)
+        mass = torch.zeros((B, R), dtype=torch.float64, device=dev)
+        sizes = torch.from_numpy(np.stack([np.bincount(l[l < R], minlength=R) for l in eng.labels_np]).astype(np.int32)).to(dev)
+        g_rbar = torch.zeros((B, R), dtype=torch.float32, device=dev)
+        g_imp = torch.empty((B, R), dtype=torch.float32, device=dev)
 
-    def mass_step():
-        fd.fd_regional_step_mass(ctx, x, cond, labels, mask, R, kv, y, active_idx, cu_active, mass)
+        def mass_step():
+            fd.fd_regional_step_mass(ctx, x, cond, eng.labels, eng.mask, R, eng.kv, y, eng.active_idx, eng.cu_active, mass)
 
-    def plain_step():
-        fd.fd_regional_step(ctx, x, cond, labels, mask, R, kv, y, active_idx, cu_active)
+        def plain_step():
+            fd.fd_regional_step(ctx, x, cond, eng.labels, eng.mask, R, eng.kv, y, eng.active_idx, eng.cu_active)
 
-    # alternate the two forms: under the power cap the clock drifts over seconds, which would bias whichever ran second
-    tp, tm = [], []
-    for _ in range(4):
-        tp.append(time_us(plain_step, 3) / 1e3)
-        tm.append(time_us(mass_step, 3) / 1e3)
-    ms_plain, ms_mass = float(np.median(tp)), float(np.median(tm))
-    gate_attn_us = time_us(lambda: fd.fd_region_activity_attn(ctx, mass, sizes, eps, g_rbar, delta, skip, prev, g_imp,
-                                                              weight, mask))
-    attn_signal = {"step_ms": ms_plain, "step_with_mass_ms": ms_mass, "mass_extra_ms": ms_mass - ms_plain,
-                   "gate_us": gate_attn_us,
-                   "note": "first block's own-region softmax mass (fused in a variant of the tensor-core attention "
-                           "kernel) + the gate on it; outside the timed step"}
-    delta.zero_(); skip.zero_(); prev.fill_(1)
-    fd.fd_poll_status(ctx)
+        # alternate the two forms: under the power cap the clock drifts over seconds, which would bias whichever ran second
+        tp, tm = [], []
+        for _ in range(3):
+            tp.append(time_us(plain_step, 2) / 1e3)
+            tm.append(time_us(mass_step, 2) / 1e3)
+        ms_plain, ms_mass = float(np.median(tp)), float(np.median(tm))
+        gate_attn_us = time_us(lambda: fd.fd_region_activity_attn(ctx, mass, sizes, eps, g_rbar, eng.delta, eng.skip, eng.prev,
+                                                                  g_imp, eng.weight, eng.mask))
+        extras["attention_gate_signal"] = {
+            "step_ms": ms_plain, "step_with_mass_ms": ms_mass, "mass_extra_ms": ms_mass - ms_plain, "gate_us": gate_attn_us,
+            "note": "first block's own-region softmax mass (fused in a variant of the tensor-core attention kernel) + "
+                    "the gate on it; outside the timed step"}
+        fd.fd_poll_status(ctx)
 
     # streaming rate of the activity reduction on a batch large enough to be bandwidth bound (at the
     # benchmark shapes the gate moves a few MB and is launch-latency bound): 256 requests x 8192 tokens x 64
@@ -481,62 +615,57 @@ def run_ours(args):
             pst[2].fill_(1)
             fd.fd_region_activity_noalloc(pz1, pz0, plab, pR, peps, 1e-12, 5, pst[0], pst[1], pst[2], pout[0], pout[1], pout[2])
 
-        for _ in range(3):
-            probe_step()
-        torch.cuda.synchronize()
-        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        pe0.record()
-        for _ in range(10):
-            probe_step()
-        pe1.record()
-        torch.cuda.synchronize()
-        p_ms = pe0.elapsed_time(pe1) / 10
+        p_ms = time_us(probe_step, 10) / 1e3
         p_bytes = 2.0 * pz0.numel() * 4 + plab.numel() * 4
         del pz0, pz1, plab
-        probe = {"bytes": p_bytes, "ms": p_ms, "gbs": p_bytes / (p_ms * 1e-3) / 1e9}
+        probe = {"bytes": p_bytes, "ms": p_ms, "gbs": p_bytes / (p_ms * 1e-3) / 1e9,
+                 "frac_of_hbm": p_bytes / (p_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
+                 "workload": "256 requests x 8192 tokens x 64 channels, 64 regions"}
 
     fl = block_flops(A_b, N, H, M)
     step_flops = L * sum(fl.values())
     dense_flops = L * sum(block_flops([N] * B, N, H, M).values())
-    peaks, peak_kind = load_peaks()
     flops_all = replicas.sum_over_ranks(rep, step_flops, dev)          # every replica has its own active set
     value = replicas.job_throughput(flops_all, ms_reg) / 1e12
     e2e_value = replicas.job_throughput(flops_all, ms_e2e) / 1e12
 
-    # per-kernel breakdown of the profiled pass; the dominant group feeds the roofline object
-    es = 2 if wl.dtype == "bf16" else 4
-    bytes_per_launch = {
-        "ln_modulate": A * H * (4 + es), "adaln": L * 6 * H * wl.Hc * es,
-        "activity": 2.0 * 4 * D * float(N * B), "compact": 4.0 * B * N + 4.0 * A,
-    }
-    total_ms = sum(v[0] for v in prof.values()) or 1.0
-    breakdown = {}
-    for k, (ms, cnt) in prof.items():
-        if cnt == 0:
-            continue
-        calls = args.steps * (L if k.startswith("gemm") or k == "attention" else (2 * L if k == "ln_modulate" else 1))
-        per_call_ms = ms / calls
-        ent = {"ms_per_step": ms / args.steps, "share": ms / total_ms, "calls_per_step": calls // args.steps,
-               "avg_call_us": per_call_ms * 1e3}
-        if k in fl:
-            ent["tflops"] = fl[k] / (per_call_ms * 1e-3) / 1e12
-        elif k in bytes_per_launch:
-            ent["gbs"] = bytes_per_launch[k] / (per_call_ms * 1e-3) / 1e9
-        breakdown[k] = ent
+    # the headline workload's own fraction sweep, then the other workloads (one GPU only: replicas repeat the headline)
+    sweep, others = {}, {}
+    if world == 1 and not args.no_sweep:
+        for tag, f in SWEEPS.get(wl.name, []):
+            r, _, _ = eng.measure(max(5, args.steps // 4), 3, peaks, fraction=f, kernels=False, dense_ms=ms_dense)
+            sweep[tag] = {k: r[k] for k in ("active_fraction", "step_ms", "tflops", "speedup_vs_dense", "t_over_f_dense")}
+    weight_gb = sum(t.numel() * t.element_size() for t in eng.weights.values()) / 1e9
+    st_destroy = eng.close()
+    del eng, x, cond, y, z_cur, z_prev, eps
+    torch.cuda.empty_cache()
+    if world == 1:
+        for name in [n for n in args.also.split(",") if n and n != wl.name]:
+            others[name] = side_workload(name, seed, dev, rep, args.steps, args.warmup, peaks)
+
+    # roofline object: the kernel group with the largest share of the step
     dom = max((k for k in breakdown if k in fl), key=lambda k: breakdown[k]["ms_per_step"])
-    tensor_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-    traffic = None
-    tp = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.txt")
-    if os.path.exists(tp) and wl.name == "audio" and not args.blocks:
-        with open(tp) as f:
-            for ln in f:
-                parts = ln.split()
-                if len(parts) == 2 and parts[0] == dom:
-                    traffic = int(parts[1])
-    roofline = {"kernel": dom, "bound": "tensor", "achieved": breakdown[dom]["tflops"], "peak": tensor_peak,
-                "unit": "TFLOP/s", "frac": breakdown[dom]["tflops"] / tensor_peak, "traffic": traffic,
-                "peak_source": peak_kind + " (sustained bf16 matmul; the kernel is timed inside a long step)",
-                "flops_per_launch": fl[dom]}
+    burst = float(peaks["bf16_tflops"])
+    sust = float(peaks.get("bf16_tflops_sustained", burst))
+    timed_s = ms_reg * args.steps * 1e-3
+    # a kernel timed alone (or in a pass shorter than a second) is held against the burst figure; inside a timed
+    # region of seconds under the power cap, against the sustained one
+    long_region = timed_s >= 1.0
+    peak = sust if long_region else burst
+    ach = breakdown[dom]["tflops"]
+    roofline = {
+        "kernel": dom, "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": round(ach / peak, 4),
+        "traffic": dram_traffic(wl.name, dom) if not args.blocks else None,
+        "peak_source": "%s %s bf16 matmul (timed region %.2f s)" % (peak_kind, "sustained" if long_region else "burst", timed_s),
+        "frac_burst": round(ach / burst, 4), "frac_sustained": round(ach / sust, 4), "timed_region_s": round(timed_s, 3),
+        "flops_per_launch": fl[dom], "avg_launch_us": breakdown[dom]["avg_call_us"],
+        "step_ms": round(ms_reg, 4), "dense_step_ms": round(ms_dense, 4), "active_fraction": round(f_tok, 4),
+        "speedup_vs_dense": round(ms_dense / ms_reg, 3), "t_over_f_dense": round(ms_reg / (f_tok * ms_dense), 3),
+        "step_tflops": round(value / world, 1), "step_frac_burst": round(value / world / burst, 4),
+        "step_frac_sustained": round(value / world / sust, 4),
+        "kernels": breakdown, "sweep": sweep, "workloads": others,
+        "activity_probe": probe,
+    }
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
@@ -546,11 +675,10 @@ def run_ours(args):
                    "mlp": M, "requests": B, "tokens_per_request": N, "regions": R,
                    "active_tokens": A, "active_fraction": f_tok, "per_request_active": A_b.tolist(),
                    "parallelism": "replicas x%d (no collectives)" % world,
-                   "l2": "inputs larger than L2: %.2f GB of weights stream through every step" %
-                         (sum(t.numel() * t.element_size() for t in weights.values()) / 1e9)},
+                   "l2": "inputs larger than L2: %.2f GB of weights stream through every step" % weight_gb},
         "regional_step_ms": ms_reg, "dense_step_ms": ms_dense,
         "dense_tflops": dense_flops / (ms_dense * 1e-3) / 1e12,
-        "frac_of_bf16_peak": value / world / float(peaks["bf16_tflops"]),
+        "frac_of_bf16_peak": value / world / burst,
         "speedup_vs_dense": ms_dense / ms_reg, "time_over_fraction_times_dense": ms_reg / (f_tok * ms_dense),
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h,
@@ -558,14 +686,11 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": roofline,
-        "kernel_breakdown": breakdown,
-        "activity_probe": None if probe is None else dict(probe, frac_of_hbm=probe["gbs"] / float(peaks["hbm_gbs"]),
-                                                         workload="256 requests x 8192 tokens x 64 channels, 64 regions"),
-        "sampler": sampler,
-        "attention_gate_signal": attn_signal,
         "peaks": {"source": peak_kind, "bf16_tflops": peaks.get("bf16_tflops"),
                   "bf16_tflops_sustained": peaks.get("bf16_tflops_sustained"), "hbm_gbs": peaks.get("hbm_gbs")},
+        "destroy_status": int(st_destroy),
     }
+    line.update(extras)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             smp = OracleSample(args.workload, args.seed)
@@ -574,8 +699,47 @@ def run_ours(args):
             line["cpu_baseline"] = {"value": fl_cpu / dt_cpu / 1e12, "unit": "TFLOP/s", "cores": omp_threads(),
                                     "kind": "oracle", "sample": text, "seconds": dt_cpu}
         print(json.dumps(line))
-    fd.fd_destroy(ctx)
     replicas.shutdown(rep)
+
+
+def run_stub(args):
+    """The replica plumbing of the benchmark without a GPU (for tests of the multi-process launch path): every
+    rank joins a gloo group, "steps" by sleeping, and rank 0 prints the line with the whole job's rate."""
+    from paper_2607_12121_b200 import replicas
+    rep = replicas.from_env()
+    replicas.init(rep, "gloo")
+
+    def run(n):
+        replicas.barrier(rep)
+        t0 = time.perf_counter()
+        for _ in range(n):
+            time.sleep(args.stub_step_ms * 1e-3)
+        replicas.barrier(rep)
+        return replicas.max_over_ranks(rep, (time.perf_counter() - t0) * 1e3) / n
+
+    run(max(1, args.warmup))
+    ms = run(args.steps)
+    units = replicas.sum_over_ranks(rep, 1.0)
+    if rep.is_lead:
+        print(json.dumps({"metric": "stub steps/s", "value": replicas.job_throughput(units, ms), "unit": "steps/s",
+                          "n_gpus": rep.world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                          "higher_is_better": True, "scaling": "weak", "stub": True, "gpu_launches": 0}))
+    replicas.shutdown(rep)
+
+
+def spawn_replicas(args):
+    """`--gpus N` without a launcher around it: start N ranks of this script under torch.distributed.run on this
+    node (one process per GPU) and pass their output through."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")            # the communicator / transport lines go to stderr
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.run(cmd, env=env).returncode
 
 
 def main():
@@ -584,14 +748,24 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="audio")
+    ap.add_argument("--workload", default="video")
+    ap.add_argument("--also", default="audio,image,mmdit",
+                    help="other workloads measured after the headline one (one GPU only); '' for none")
     ap.add_argument("--fraction", type=float, default=None, help="same active fraction for every request")
     ap.add_argument("--seed", type=int, default=1000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-probe", action="store_true", help="skip the bandwidth probe of the activity kernel")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the active-fraction sweeps")
+    ap.add_argument("--no-extras", action="store_true", help="skip the sampler and attention-gate timings")
     ap.add_argument("--blocks", type=int, default=0, help="override the block count (profiling captures only)")
+    ap.add_argument("--stub-step-ms", type=float, default=None,
+                    help="no GPU: ranks join a gloo group and sleep this long per step (launch-path tests)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_replicas(args))
+    if args.stub_step_ms is not None:
+        run_stub(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

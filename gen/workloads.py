@@ -351,3 +351,24 @@ def latent_sequence(wl: Workload, seed: int, labels: np.ndarray,
         out.append({"z_cur": z_next, "z_prev": z, "eps": eps})
         z = z_next
     return out
+
+
+def block_variants(wl: Workload, seed: int, n_blocks: Optional[int] = None, qk_norm: bool = True, rope: bool = True,
+                   rope_base: float = 10000.0) -> Dict[str, np.ndarray]:
+    """Inputs of the block variants: QK-RMSNorm weights ~ 1 + N(0, 0.1) per block and head channel
+    (q_norm_w, k_norm_w [L, head_dim], rounded to the storage type) and rotary tables for positions 0..N-1 with the
+    usual frequencies base^(-2i/d) (rope_cos, rope_sin [N, head_dim/2] fp32).  Only draws and tabulates inputs."""
+    L = wl.L if n_blocks is None else n_blocks
+    dh = wl.head_dim
+    out: Dict[str, np.ndarray] = {}
+    if qk_norm:
+        g = _rng(seed, 1313)
+        out["q_norm_w"] = _store(wl, 1.0 + 0.1 * g.standard_normal((L, dh), dtype=np.float32))
+        out["k_norm_w"] = _store(wl, 1.0 + 0.1 * g.standard_normal((L, dh), dtype=np.float32))
+        out["qk_norm_eps"] = 1e-6
+    if rope:
+        freq = rope_base ** (-2.0 * np.arange(dh // 2, dtype=np.float64) / dh)
+        ang = np.arange(wl.N, dtype=np.float64)[:, None] * freq[None, :]
+        out["rope_cos"] = np.cos(ang).astype(np.float32)
+        out["rope_sin"] = np.sin(ang).astype(np.float32)
+    return out

@@ -163,6 +163,33 @@ fd_status fd_regional_step(fd_ctx* ctx, const void* x, const void* cond, const i
                            int32_t* active_idx_out, int32_t* cu_active_out, void* cuda_stream);
 
 /*
+ * Block variants of the models the paper evaluates (Sec. 6.1; FLUX.1-dev, SD3-Medium and Wan2.1 normalise queries
+ * and keys and / or rotate them by position).  The paper does not define them; the conventions here are those of the
+ * published architectures:
+ *   QK-RMSNorm  every head slice x [head_dim] of a query / key row becomes
+ *               x / sqrt(mean(x^2) + qk_norm_eps) * w,  w = q_norm_w[l] for queries, k_norm_w[l] for keys of block l
+ *               (one weight vector per block, shared by all heads);
+ *   RoPE        then the channel pairs (2i, 2i+1) of every head are rotated by the angle of the token's position:
+ *               (a, b) -> (a cos - b sin, a sin + b cos) with cos = rope_cos[j, i], sin = rope_sin[j, i], j the token's
+ *               index inside its request (the caller tabulates the angles, so 1-D, axial or constant-for-text positions
+ *               are all expressible).
+ * Applied to the fresh Q and K rows of every block right after the QKV projection; the cache keeps keys in this final
+ * form, so rows of skipped tokens never need re-rotation.  V is unchanged.
+ *   q_norm_w, k_norm_w [L, head_dim] of fd_config.dtype, both or neither (NULL = no normalisation)
+ *   rope_cos, rope_sin [max_tokens, head_dim/2] f32, both or neither (NULL = no rotation; needs an even head_dim)
+ * DEVICE pointers, 4-byte aligned (8-byte for f32 weights), borrowed until the next call or fd_destroy.  v = NULL switches
+ * every variant off.  Takes effect for the steps queued after the call returns.
+ */
+typedef struct {
+    const void* q_norm_w;
+    const void* k_norm_w;
+    float qk_norm_eps;
+    const float* rope_cos;
+    const float* rope_sin;
+} fd_block_variants;
+fd_status fd_set_block_variants(fd_ctx* ctx, const fd_block_variants* v);
+
+/*
  * The Patch Gate on the paper's own signal (Sec. 4.2): the refinement importance of a patch is the block mean of
  * the self-attention matrix over the patch,  R_i = (1/|A_i|^2) sum_{u,v in A_i} SA[u,v],  and the gate weights are
  * the normalised changes  Delta_i = |R_i - Rbar_i|  (Rbar_i = the importance at the patch's last executed step;
@@ -292,7 +319,8 @@ enum {
     FD_PROF_GEMM_FC2 = 8,
     FD_PROF_PARTITION = 9,
     FD_PROF_SAMPLER = 10, /* patch embedding, final layer, latent update */
-    FD_PROF_GROUPS = 11
+    FD_PROF_QK_VARIANTS = 11, /* QK-RMSNorm + rotary embedding (block variants) */
+    FD_PROF_GROUPS = 12
 };
 fd_status fd_profile_enable(fd_ctx* ctx, int enable);
 fd_status fd_profile_read(fd_ctx* ctx, void* cuda_stream, float* ms_out, int32_t* kernels_out);

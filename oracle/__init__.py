@@ -40,6 +40,8 @@ def _load():
         _lib.fdo_adaln.restype = ctypes.c_int
         _lib.fdo_regional_block.restype = ctypes.c_int
         _lib.fdo_dense_block.restype = ctypes.c_int
+        _lib.fdo_regional_block_v.restype = ctypes.c_int
+        _lib.fdo_dense_block_v.restype = ctypes.c_int
     return _lib
 
 
@@ -69,9 +71,30 @@ def adaln(cond: np.ndarray, w_ada: np.ndarray, b_ada: np.ndarray) -> np.ndarray:
     return mod
 
 
+def _variant_args(variants, l: int, dh: int, N: int):
+    """ctypes arguments of the block variants of block ``l`` (QK-RMSNorm weights [L,dh], RoPE tables [N,dh/2]);
+    ``variants`` is None or a dict with any of q_norm_w, k_norm_w, qk_norm_eps, rope_cos, rope_sin."""
+    v = variants or {}
+    keep = []
+
+    def arr(a, shape):
+        if a is None:
+            return None
+        a = _c(a)
+        assert a.shape == shape, (a.shape, shape)
+        keep.append(a)
+        return _fp(a)
+
+    qn = arr(None if v.get("q_norm_w") is None else v["q_norm_w"][l], (dh,))
+    kn = arr(None if v.get("k_norm_w") is None else v["k_norm_w"][l], (dh,))
+    rc = arr(v.get("rope_cos"), (N, dh // 2))
+    rs = arr(v.get("rope_sin"), (N, dh // 2))
+    return (qn, kn, ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))), rc, rs), keep
+
+
 def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w: Dict[str, np.ndarray],
                    l: int, kv_l: np.ndarray, heads: int, ln_eps: float = 1e-6,
-                   finish: Optional[np.ndarray] = None) -> np.ndarray:
+                   finish: Optional[np.ndarray] = None, variants=None) -> np.ndarray:
     """One block over the compact rows ``u_in`` [A,H]; ``kv_l`` [B,2,N,H] is updated in place."""
     A, H = u_in.shape
     B, _, N, _ = kv_l.shape
@@ -79,19 +102,20 @@ def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w:
     assert kv_l.dtype == np.float32 and kv_l.flags["C_CONTIGUOUS"]
     u_out = np.zeros((A, H), np.float32)
     fin = None if finish is None else np.ascontiguousarray(finish, np.int32)
-    rc = _load().fdo_regional_block(
+    vargs, _keep = _variant_args(variants, l, H // heads, N)
+    rc = _load().fdo_regional_block_v(
         B, N, H, heads, H // heads, M, A, _ip(np.ascontiguousarray(active_idx, np.int32)), _fp(_c(mod)),
         _fp(_c(w["w_qkv"][l])), _fp(_c(w["b_qkv"][l])), _fp(_c(w["w_o"][l])), _fp(_c(w["b_o"][l])),
         _fp(_c(w["w_fc1"][l])), _fp(_c(w["b_fc1"][l])), _fp(_c(w["w_fc2"][l])), _fp(_c(w["b_fc2"][l])),
         ctypes.c_float(ln_eps), _fp(_c(u_in)), _fp(u_out), _fp(kv_l),
-        0 if fin is None else int(fin.size), _ip(fin))
+        0 if fin is None else int(fin.size), _ip(fin), *vargs)
     assert rc == 0
     return u_out
 
 
 def regional_step(x: np.ndarray, cond: np.ndarray, labels: np.ndarray, mask: np.ndarray,
                   w: Dict[str, np.ndarray], kv: np.ndarray, y: np.ndarray, heads: int, R: int,
-                  ln_eps: float = 1e-6, n_blocks: Optional[int] = None):
+                  ln_eps: float = 1e-6, n_blocks: Optional[int] = None, variants=None):
     """The whole block stack on active tokens.
 
     x [B,N,H]; kv [L,B,2,N,H] and y [B,N,H] are updated in place: rows of active tokens are
@@ -104,7 +128,7 @@ def regional_step(x: np.ndarray, cond: np.ndarray, labels: np.ndarray, mask: np.
     u = np.ascontiguousarray(x.reshape(B * N, H)[active_idx], np.float32)
     for l in range(L):
         mod = adaln(cond, w["w_ada"][l], w["b_ada"][l])
-        u = regional_block(u, active_idx, mod, w, l, kv[l], heads, ln_eps)
+        u = regional_block(u, active_idx, mod, w, l, kv[l], heads, ln_eps, variants=variants)
     y.reshape(B * N, H)[active_idx] = u
     return active_idx, cu_active
 
@@ -131,29 +155,52 @@ def block0_queries(x, cond, w, active_idx, ln_eps: float = 1e-6) -> np.ndarray:
 
 
 def dense_block(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], l: int, heads: int,
-                ln_eps: float = 1e-6):
+                ln_eps: float = 1e-6, variants=None):
     """One ungated block on whole matrices. Returns x_out [B,N,H], kv [B,2,N,H]."""
     B, N, H = x.shape
     M = w["w_fc1"].shape[1]
     Hc = cond.shape[1]
     x_out = np.empty((B, N, H), np.float32)
     kv = np.empty((B, 2, N, H), np.float32)
-    rc = _load().fdo_dense_block(
+    vargs, _keep = _variant_args(variants, l, H // heads, N)
+    rc = _load().fdo_dense_block_v(
         B, N, H, heads, H // heads, M, Hc, _fp(_c(cond)), _fp(_c(w["w_ada"][l])), _fp(_c(w["b_ada"][l])),
         _fp(_c(w["w_qkv"][l])), _fp(_c(w["b_qkv"][l])), _fp(_c(w["w_o"][l])), _fp(_c(w["b_o"][l])),
         _fp(_c(w["w_fc1"][l])), _fp(_c(w["b_fc1"][l])), _fp(_c(w["w_fc2"][l])), _fp(_c(w["b_fc2"][l])),
-        ctypes.c_float(ln_eps), _fp(_c(x)), _fp(x_out), _fp(kv))
+        ctypes.c_float(ln_eps), _fp(_c(x)), _fp(x_out), _fp(kv), *vargs)
     assert rc == 0
     return x_out, kv
 
 
 def dense_step(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], heads: int,
-               ln_eps: float = 1e-6, n_blocks: Optional[int] = None):
+               ln_eps: float = 1e-6, n_blocks: Optional[int] = None, variants=None):
     """The ungated block stack. Returns y [B,N,H] and kv [L,B,2,N,H]."""
     L = w["w_qkv"].shape[0] if n_blocks is None else n_blocks
     B, N, H = x.shape
     kv = np.empty((L, B, 2, N, H), np.float32)
     cur = np.ascontiguousarray(x, np.float32)
     for l in range(L):
-        cur, kv[l] = dense_block(cur, cond, w, l, heads, ln_eps)
+        cur, kv[l] = dense_block(cur, cond, w, l, heads, ln_eps, variants=variants)
     return cur, kv
+
+
+def qk_variants(q: np.ndarray, k: np.ndarray, heads: int, pos: Optional[np.ndarray] = None, q_norm_w=None, k_norm_w=None,
+                qk_norm_eps: float = 1e-6, rope_cos=None, rope_sin=None, program: str = "regional"):
+    """QK-RMSNorm and RoPE as one of the two C programs applies them to query / key rows [n,H] (copies are returned).
+    ``program`` = "regional" takes the positions ``pos`` [n]; "dense" takes row t at position t."""
+    q, k = _c(q).copy(), _c(k).copy()
+    n, H = q.shape
+    dh = H // heads
+    opt = lambda a: None if a is None else _fp(_c(a))
+    keep = [None if a is None else _c(a) for a in (q_norm_w, k_norm_w, rope_cos, rope_sin)]
+    ptr = [None if a is None else _fp(a) for a in keep]
+    if program == "regional":
+        pos = np.arange(n, dtype=np.int32) if pos is None else np.ascontiguousarray(pos, np.int32)
+        rc = _load().fdo_regional_qk_variants(n, heads, dh, _ip(pos), _fp(q), _fp(k), ptr[0], ptr[1],
+                                              ctypes.c_float(qk_norm_eps), ptr[2], ptr[3])
+    else:
+        assert pos is None
+        rc = _load().fdo_dense_qk_variants(n, heads, dh, _fp(q), _fp(k), ptr[0], ptr[1], ctypes.c_float(qk_norm_eps),
+                                           ptr[2], ptr[3])
+    assert rc == 0
+    return q, k

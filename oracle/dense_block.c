@@ -80,15 +80,77 @@ static void full_attention(const float* Q, const float* K, const float* V, int N
 }
 
 /*
+ * Block variants (this build's readings of the architectures of the paper's evaluated models, Sec. 6.1), on whole
+ * [N,H] matrices of one request.  rms_norm_heads: every head slice of every row is divided by its root mean square
+ * (plus eps under the root) and multiplied channel-wise by gamma[dh].  rotate_pairs: the even/odd channel pairs of
+ * every head are turned by the angle tabulated for the row's position t, i.e. multiplied as complex numbers
+ * (even + i odd) by (cos + i sin).
+ */
+static void rms_norm_heads(float* X, int N, int heads, int dh, const float* gamma, float eps) {
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < N; ++t)
+        for (int h = 0; h < heads; ++h) {
+            float* v = X + ((size_t)t * heads + h) * dh;
+            double sq = 0.0;
+            for (int c = 0; c < dh; ++c) sq += (double)v[c] * (double)v[c];
+            const double inv = 1.0 / sqrt(sq / (double)dh + (double)eps);
+            for (int c = 0; c < dh; ++c) v[c] = (float)((double)v[c] * inv * (double)gamma[c]);
+        }
+}
+
+static void rotate_pairs(float* X, int N, int heads, int dh, const float* cos_t, const float* sin_t) {
+    const int half = dh / 2;
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < N; ++t)
+        for (int h = 0; h < heads; ++h) {
+            float* v = X + ((size_t)t * heads + h) * dh;
+            for (int i = 0; i < half; ++i) {
+                const double re = (double)v[2 * i], im = (double)v[2 * i + 1];
+                const double cr = (double)cos_t[(size_t)t * half + i], ci = (double)sin_t[(size_t)t * half + i];
+                v[2 * i] = (float)(re * cr - im * ci);          /* real part of (re + i im)(cr + i ci) */
+                v[2 * i + 1] = (float)(re * ci + im * cr);      /* imaginary part */
+            }
+        }
+}
+
+/* test hook: the variants on given Q and K matrices [N,H] of one request (row t sits at position t) */
+int fdo_dense_qk_variants(int N, int heads, int dh, float* Q, float* K, const float* qn_w, const float* kn_w,
+                          float qk_eps, const float* rope_cos, const float* rope_sin) {
+    if (qn_w) rms_norm_heads(Q, N, heads, dh, qn_w, qk_eps);
+    if (kn_w) rms_norm_heads(K, N, heads, dh, kn_w, qk_eps);
+    if (rope_cos) { rotate_pairs(Q, N, heads, dh, rope_cos, rope_sin); rotate_pairs(K, N, heads, dh, rope_cos, rope_sin); }
+    return 0;
+}
+
+/*
  * x_in, x_out [B,N,H]; kv_out [B,2,N,H] receives K and V of every position.
  * cond [B,Hc]; adaLN chunk order shift_msa, scale_msa, gate_msa, shift_mlp, scale_mlp, gate_mlp.
+ * fdo_dense_block_v adds the block variants (NULL = off): qn_w, kn_w [dh]; rope_cos, rope_sin [N, dh/2].
  */
+int fdo_dense_block_v(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+                      const float* w_ada, const float* b_ada, const float* w_qkv, const float* b_qkv,
+                      const float* w_o, const float* b_o, const float* w_fc1, const float* b_fc1,
+                      const float* w_fc2, const float* b_fc2, float ln_eps, const float* x_in,
+                      float* x_out, float* kv_out, const float* qn_w, const float* kn_w, float qk_eps,
+                      const float* rope_cos, const float* rope_sin);
+
 int fdo_dense_block(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                     const float* w_ada, const float* b_ada, const float* w_qkv, const float* b_qkv,
                     const float* w_o, const float* b_o, const float* w_fc1, const float* b_fc1,
                     const float* w_fc2, const float* b_fc2, float ln_eps, const float* x_in,
                     float* x_out, float* kv_out) {
+    return fdo_dense_block_v(B, N, H, heads, dh, M, Hc, cond, w_ada, b_ada, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2,
+                             b_fc2, ln_eps, x_in, x_out, kv_out, NULL, NULL, 0.f, NULL, NULL);
+}
+
+int fdo_dense_block_v(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+                      const float* w_ada, const float* b_ada, const float* w_qkv, const float* b_qkv,
+                      const float* w_o, const float* b_o, const float* w_fc1, const float* b_fc1,
+                      const float* w_fc2, const float* b_fc2, float ln_eps, const float* x_in,
+                      float* x_out, float* kv_out, const float* qn_w, const float* kn_w, float qk_eps,
+                      const float* rope_cos, const float* rope_sin) {
     if (heads * dh != H) return 2;
+    if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
     const size_t NH = (size_t)N * H;
     float* act = (float*)malloc(sizeof(float) * (size_t)Hc);
     float* mod = (float*)malloc(sizeof(float) * (size_t)6 * H);
@@ -123,6 +185,12 @@ int fdo_dense_block(int B, int N, int H, int heads, int dh, int M, int Hc, const
             memcpy(Q + (size_t)t * H, qkv + (size_t)t * 3 * H, sizeof(float) * (size_t)H);
             memcpy(Kc + (size_t)t * H, qkv + (size_t)t * 3 * H + H, sizeof(float) * (size_t)H);
             memcpy(Vc + (size_t)t * H, qkv + (size_t)t * 3 * H + 2 * H, sizeof(float) * (size_t)H);
+        }
+        if (qn_w) rms_norm_heads(Q, N, heads, dh, qn_w, qk_eps);
+        if (kn_w) rms_norm_heads(Kc, N, heads, dh, kn_w, qk_eps);
+        if (rope_cos) {
+            rotate_pairs(Q, N, heads, dh, rope_cos, rope_sin);
+            rotate_pairs(Kc, N, heads, dh, rope_cos, rope_sin);
         }
         full_attention(Q, Kc, Vc, N, heads, dh, att);
         matmul_nt_bias(att, w_o, b_o, (size_t)N, H, H, proj);

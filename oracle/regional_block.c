@@ -51,6 +51,53 @@ static void row_ln_modulate(const float* u, const float* shift, const float* sca
         out[c] = (float)((((double)u[c] - mean) * rstd) * (1.0 + (double)scale[c]) + (double)shift[c]);
 }
 
+/*
+ * Block variants of the models the paper evaluates (Sec. 6.1: FLUX.1-dev, SD3-Medium, Wan2.1 use them; the
+ * paper itself does not define them, so these are this build's readings of the published architectures):
+ *   QK-RMSNorm: per head, x_c <- x_c / sqrt(mean_c x_c^2 + eps) * gamma_c, applied to queries (gamma_q) and keys
+ *               (gamma_k) right after the projection; gamma has one entry per head channel, shared by all heads;
+ *   RoPE:       after the norm, the channel pairs (2i, 2i+1) of every head are rotated by the angle whose cosine
+ *               and sine the caller tabulated for the token's position: (a, b) <- (a cos - b sin, a sin + b cos).
+ * The key is cached in this final form.  Either table may be NULL (variant off).
+ */
+static void head_rms_norm(float* x, int dh, const float* gamma, float eps) {
+    double ss = 0.0;
+    for (int c = 0; c < dh; ++c) ss += (double)x[c] * (double)x[c];
+    const double r = 1.0 / sqrt(ss / (double)dh + (double)eps);
+    for (int c = 0; c < dh; ++c) x[c] = (float)((double)x[c] * r * (double)gamma[c]);
+}
+
+static void head_rope(float* x, int dh, const float* cs, const float* sn) {
+    for (int i = 0; i < dh / 2; ++i) {
+        const double a = (double)x[2 * i], b = (double)x[2 * i + 1];
+        const double c = (double)cs[i], s = (double)sn[i];
+        x[2 * i] = (float)(a * c - b * s);
+        x[2 * i + 1] = (float)(a * s + b * c);
+    }
+}
+
+/* q and k rows [H] of the token at position j of its request, all heads, in place */
+static void row_qk_variants(float* q, float* k, int heads, int dh, int j, const float* qn_w, const float* kn_w,
+                            float qk_eps, const float* rope_cos, const float* rope_sin) {
+    for (int h = 0; h < heads; ++h) {
+        if (qn_w) head_rms_norm(q + h * dh, dh, qn_w, qk_eps);
+        if (kn_w) head_rms_norm(k + h * dh, dh, kn_w, qk_eps);
+        if (rope_cos) {
+            head_rope(q + h * dh, dh, rope_cos + (size_t)j * (dh / 2), rope_sin + (size_t)j * (dh / 2));
+            head_rope(k + h * dh, dh, rope_cos + (size_t)j * (dh / 2), rope_sin + (size_t)j * (dh / 2));
+        }
+    }
+}
+
+/* test hook: the variants applied to given q / k rows [n, H] of tokens at positions pos[n] */
+int fdo_regional_qk_variants(int n, int heads, int dh, const int32_t* pos, float* q, float* k, const float* qn_w,
+                             const float* kn_w, float qk_eps, const float* rope_cos, const float* rope_sin) {
+    for (int r = 0; r < n; ++r)
+        row_qk_variants(q + (size_t)r * heads * dh, k + (size_t)r * heads * dh, heads, dh, pos[r], qn_w, kn_w, qk_eps,
+                        rope_cos, rope_sin);
+    return 0;
+}
+
 /* mod[b, 6H] = W_ada * SiLU(cond[b]) + b_ada ; chunk order shift_msa, scale_msa, gate_msa,
  * shift_mlp, scale_mlp, gate_mlp */
 int fdo_adaln(int B, int H, int Hc, const float* cond, const float* w_ada, const float* b_ada,
@@ -74,14 +121,36 @@ int fdo_adaln(int B, int H, int Hc, const float* cond, const float* w_ada, const
  *   finish[n_finish] compact rows whose attention + MLP are evaluated (NULL = all A rows);
  *                   K/V are always refreshed for all A rows because every query needs them.
  * Rows outside `finish` get no u_out.
+ * fdo_regional_block_v adds the block variants: qn_w, kn_w [dh] (QK-RMSNorm, NULL = off), rope_cos, rope_sin
+ * [N, dh/2] (NULL = off).
  */
+int fdo_regional_block_v(int B, int N, int H, int heads, int dh, int M, int A,
+                         const int32_t* active_idx, const float* mod,
+                         const float* w_qkv, const float* b_qkv, const float* w_o, const float* b_o,
+                         const float* w_fc1, const float* b_fc1, const float* w_fc2, const float* b_fc2,
+                         float ln_eps, const float* u_in, float* u_out, float* kv,
+                         int n_finish, const int32_t* finish,
+                         const float* qn_w, const float* kn_w, float qk_eps, const float* rope_cos, const float* rope_sin);
+
 int fdo_regional_block(int B, int N, int H, int heads, int dh, int M, int A,
                        const int32_t* active_idx, const float* mod,
                        const float* w_qkv, const float* b_qkv, const float* w_o, const float* b_o,
                        const float* w_fc1, const float* b_fc1, const float* w_fc2, const float* b_fc2,
                        float ln_eps, const float* u_in, float* u_out, float* kv,
                        int n_finish, const int32_t* finish) {
+    return fdo_regional_block_v(B, N, H, heads, dh, M, A, active_idx, mod, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2,
+                                b_fc2, ln_eps, u_in, u_out, kv, n_finish, finish, NULL, NULL, 0.f, NULL, NULL);
+}
+
+int fdo_regional_block_v(int B, int N, int H, int heads, int dh, int M, int A,
+                       const int32_t* active_idx, const float* mod,
+                       const float* w_qkv, const float* b_qkv, const float* w_o, const float* b_o,
+                       const float* w_fc1, const float* b_fc1, const float* w_fc2, const float* b_fc2,
+                         float ln_eps, const float* u_in, float* u_out, float* kv,
+                         int n_finish, const int32_t* finish,
+                         const float* qn_w, const float* kn_w, float qk_eps, const float* rope_cos, const float* rope_sin) {
     if (heads * dh != H) return 2;
+    if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
     (void)B;
     float* q_all = (float*)malloc(sizeof(float) * (size_t)(A > 0 ? A : 1) * H);
     if (!q_all) return 1;
@@ -102,6 +171,7 @@ int fdo_regional_block(int B, int N, int H, int heads, int dh, int M, int A,
                 const float* md = mod + (size_t)b * 6 * H;
                 row_ln_modulate(u_in + (size_t)a * H, md + 0 * H, md + 1 * H, H, ln_eps, uh);
                 row_linear(uh, w_qkv, b_qkv, H, 3 * H, qkv);
+                row_qk_variants(qkv, qkv + H, heads, dh, j, qn_w, kn_w, qk_eps, rope_cos, rope_sin);
                 memcpy(q_all + (size_t)a * H, qkv, sizeof(float) * (size_t)H);
                 memcpy(kv + (((size_t)b * 2 + 0) * N + j) * H, qkv + H, sizeof(float) * (size_t)H);
                 memcpy(kv + (((size_t)b * 2 + 1) * N + j) * H, qkv + 2 * H, sizeof(float) * (size_t)H);

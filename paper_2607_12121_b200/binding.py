@@ -23,10 +23,10 @@ EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region
            "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
            "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait",
            "fd_embed_latent", "fd_update_latent", "fd_regional_step_mass", "fd_region_activity_attn",
-           "fd_sched_pack", "fd_sched_form_batch", "fd_rsearch_init", "fd_rsearch_update"]
+           "fd_sched_pack", "fd_sched_form_batch", "fd_rsearch_init", "fd_rsearch_update", "fd_set_block_variants"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
-               "gemm_fc2", "partition", "sampler"]
+               "gemm_fc2", "partition", "sampler", "qk_variants"]
 
 
 class FdConfig(ctypes.Structure):
@@ -43,6 +43,11 @@ class FdWeights(ctypes.Structure):
 
 class FdSamplerWeights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("w_in", "b_in", "pos", "w_out", "b_out")] + [("latent_dim", ctypes.c_int32)]
+
+
+class FdBlockVariants(ctypes.Structure):
+    _fields_ = [("q_norm_w", ctypes.c_void_p), ("k_norm_w", ctypes.c_void_p), ("qk_norm_eps", ctypes.c_float),
+                ("rope_cos", ctypes.c_void_p), ("rope_sin", ctypes.c_void_p)]
 
 
 class FdRSearch(ctypes.Structure):
@@ -99,6 +104,8 @@ def _load() -> ctypes.CDLL:
     lib.fd_embed_latent.argtypes = [vp, ctypes.POINTER(FdSamplerWeights), vp, i32, i32, vp, vp]
     lib.fd_update_latent.restype = i32
     lib.fd_update_latent.argtypes = [vp, ctypes.POINTER(FdSamplerWeights), vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
+    lib.fd_set_block_variants.restype = i32
+    lib.fd_set_block_variants.argtypes = [vp, ctypes.POINTER(FdBlockVariants)]
     lib.fd_launch_count.restype = ctypes.c_int64
     lib.fd_launch_count.argtypes = [vp]
     lib.fd_destroy.restype = i32
@@ -256,6 +263,18 @@ def fd_region_activity_attn(ctx: Context, region_mass, region_sizes, eps, rbar_s
     _check(ctx.handle, lib.fd_region_activity_attn(
         ctx.handle, _ptr(region_mass), _ptr(region_sizes), B, R, _ptr(eps), _ptr(rbar_state), _ptr(delta_state),
         _ptr(skip_count), _ptr(prev_active), _ptr(importance_out), _ptr(weight_out), _ptr(mask_out), _stream(stream)))
+
+
+def fd_set_block_variants(ctx: Context, q_norm_w=None, k_norm_w=None, qk_norm_eps: float = 1e-6, rope_cos=None,
+                          rope_sin=None) -> None:
+    """Switches the block variants on (device tensors: QK-RMSNorm weights [L, head_dim] of the context's dtype, rotary
+    tables [max_tokens, head_dim/2] f32) or, with no tensors, off.  The context keeps the tensors alive."""
+    ctx.variant_tensors = (q_norm_w, k_norm_w, rope_cos, rope_sin)
+    if all(t is None for t in ctx.variant_tensors):
+        _check(ctx.handle, lib.fd_set_block_variants(ctx.handle, None))
+        return
+    v = FdBlockVariants(_ptr(q_norm_w), _ptr(k_norm_w), float(qk_norm_eps), _ptr(rope_cos), _ptr(rope_sin))
+    _check(ctx.handle, lib.fd_set_block_variants(ctx.handle, ctypes.byref(v)))
 
 
 def fd_sched_pack(load, cost, home):

@@ -62,7 +62,7 @@ Layout make_layout(const fd_config& c) {
     l.acc_ss = take(BR * sizeof(double));
     l.acc_cnt = take(BR * sizeof(int32_t));
     l.block_counts = take((size_t)c.max_batch * ((c.max_tokens + 2047) / 2048 + 1) * sizeof(int32_t));
-    l.tiles = take((size_t)l.tile_cap * sizeof(QTile));
+    l.tiles = take((size_t)2 * l.tile_cap * sizeof(QTile));      // work list, then the list of double-height tiles
     l.ada_act = take((size_t)2 * ((c.max_batch + 7) / 8 * 8) * c.cond_dim * 2);   // SiLU(cond): bf16 head + remainder
     l.mod = take((size_t)c.n_blocks * c.max_batch * 6 * c.hidden * sizeof(float));
     l.resid = take((size_t)l.Mcap * c.hidden * sizeof(float));
@@ -89,6 +89,7 @@ struct fd_ctx {
     int64_t launches;
     std::string err;
     TcPlan* tc;
+    fd_block_variants var{};   // block variants (all pointers null: off)
     // optional per-kernel timing
     bool profiling = false;
     struct Span { cudaEvent_t a, b; int group, kernels; };
@@ -149,6 +150,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     T* o = c->at<T>(l.o);
     T* g = c->at<T>(l.g);
     QTile* tiles = c->at<QTile>(l.tiles);
+    QTile* tiles2 = c->use_tc_attn ? tiles + l.tile_cap : nullptr;
     const int rows_cap = B * N;
     int nl = 0;
     cudaError_t e;
@@ -165,7 +167,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     } while (0)
 
     FD_TRY(FD_PROF_COMPACT, launch_compact(mask, labels, B, N, R, active_idx, cu_active, c->at<int32_t>(l.block_counts), tiles,
-                          c->tile_rows, ctl, st, &nl));
+                          c->tile_rows, ctl, st, &nl, tiles2));
     FD_TRY(FD_PROF_ADALN, launch_adaln<T>(cond, static_cast<const T*>(c->w.w_ada), static_cast<const T*>(c->w.b_ada), mod, L, B, H,
                            Hc, c->ws + l.ada_act, st, &nl));
     const int max_tiles = B * ((N + c->tile_rows - 1) / c->tile_rows);
@@ -199,6 +201,15 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             FD_TRY(FD_PROF_GEMM_QKV, tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));
         else
             FD_TRY(FD_PROF_GEMM_QKV, launch_simt_gemm<T>(EPI_QKV, act, H, w_qkv, 3 * H, H, rows_cap, ep, ctl, st, &nl));
+        // block variants: QK-RMSNorm and rotary embedding on the fresh Q rows and the K rows just written
+        if (c->var.q_norm_w || c->var.rope_cos) {
+            const int q_stride = c->use_tc_attn ? tc_attention_head_pad(cf.head_dim) : cf.head_dim;
+            const T* qn = c->var.q_norm_w ? static_cast<const T*>(c->var.q_norm_w) + (size_t)blk * cf.head_dim : nullptr;
+            const T* kn = c->var.k_norm_w ? static_cast<const T*>(c->var.k_norm_w) + (size_t)blk * cf.head_dim : nullptr;
+            FD_TRY(FD_PROF_QK_VARIANTS, launch_qk_variants<T>(q, l.q_ld, q_stride, kv_b, active_idx, N, H, cf.n_heads, cf.head_dim,
+                                                               qn, kn, c->var.qk_norm_eps, c->var.rope_cos, c->var.rope_sin,
+                                                               rows_cap, ctl, st, &nl));
+        }
         // active queries against all N keys of their request; the first block can also report, per region, the
         // softmax mass its queries put on keys of their own region (paper Sec. 4.2)
         double* mass = blk == 0 ? region_mass : nullptr;
@@ -208,7 +219,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         }
         if (c->use_tc_attn) {
             FD_TRY(FD_PROF_ATTENTION, tc_attention(c->tc, blk, kv_b, B, N, tiles, max_tiles, ctl, st, &nl, labels, active_idx,
-                                                   mass, R));
+                                                   mass, R, tiles2));
         } else {
             FD_TRY(FD_PROF_ATTENTION, launch_simt_attention<T>(q, l.q_ld, kv_b, o, H, tiles, max_tiles, N, H, cf.n_heads, cf.head_dim,
                                             ctl, st, &nl, 0, labels, active_idx, mass, R));
@@ -527,6 +538,24 @@ fd_status fd_region_activity_attn(fd_ctx* c, const double* region_mass, const in
     c->span_end(nl, st);
     c->launches += nl;
     if (e != cudaSuccess) return c->fail(FD_ERR_CUDA, "attention gate launch failed: %s", cudaGetErrorString(e));
+    return FD_OK;
+}
+
+fd_status fd_set_block_variants(fd_ctx* c, const fd_block_variants* v) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!v) { c->var = fd_block_variants{}; return FD_OK; }
+    if ((v->q_norm_w == nullptr) != (v->k_norm_w == nullptr))
+        return c->fail(FD_ERR_INVALID_ARG, "q_norm_w and k_norm_w must be given together");
+    if ((v->rope_cos == nullptr) != (v->rope_sin == nullptr))
+        return c->fail(FD_ERR_INVALID_ARG, "rope_cos and rope_sin must be given together");
+    if (v->rope_cos && (c->cfg.head_dim & 1)) return c->fail(FD_ERR_SHAPE, "rotary embedding needs an even head_dim");
+    if (v->q_norm_w && !(v->qk_norm_eps >= 0.f)) return c->fail(FD_ERR_INVALID_ARG, "qk_norm_eps must be non-negative");
+    const uintptr_t wmask = c->cfg.dtype == FD_BF16 ? 3 : 7;
+    if ((reinterpret_cast<uintptr_t>(v->q_norm_w) | reinterpret_cast<uintptr_t>(v->k_norm_w)) & wmask)
+        return c->fail(FD_ERR_INVALID_ARG, "QK-norm weights are misaligned");
+    if ((reinterpret_cast<uintptr_t>(v->rope_cos) | reinterpret_cast<uintptr_t>(v->rope_sin)) & 3)
+        return c->fail(FD_ERR_INVALID_ARG, "rotary tables are misaligned");
+    c->var = *v;
     return FD_OK;
 }
 

@@ -18,7 +18,8 @@ struct Control {
     int32_t detail;
     int32_t a_total;       // number of active rows of the current step
     int32_t n_qtiles;      // number of attention query tiles of the current step
-    int32_t pad[12];
+    int32_t n_qtiles2;     // ... and of double-height tiles (the work list of the CTA-pair attention kernel)
+    int32_t pad[11];
 };
 
 __device__ __forceinline__ void report(Control* c, int code, int detail) {
@@ -106,7 +107,7 @@ cudaError_t noalloc_gate(const float* z_cur, const float* z_prev, const int32_t*
 // compact.cu
 cudaError_t launch_compact(const uint8_t* mask, const int32_t* labels, int B, int N, int R,
                            int32_t* active_idx, int32_t* cu_active, int32_t* block_counts, QTile* tiles,
-                           int tile_rows, Control* ctl, cudaStream_t st, int* n_launch);
+                           int tile_rows, Control* ctl, cudaStream_t st, int* n_launch, QTile* tiles2 = nullptr);
 
 // rowops.cu
 template <typename T>
@@ -117,6 +118,12 @@ cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* 
                                const int32_t* active_idx, const float* shift, const float* scale,
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
                                cudaStream_t st, int* n_launch, bool pdl);
+
+// qk_variants.cu: QK-RMSNorm and rotary embedding on the fresh Q rows and the K rows just written to the cache
+template <typename T>
+cudaError_t launch_qk_variants(T* q, int q_ld, int q_head_stride, T* kv_block, const int32_t* active_idx, int N, int H,
+                               int heads, int dh, const T* qn_w, const T* kn_w, float eps, const float* rope_cos,
+                               const float* rope_sin, int rows_cap, const Control* ctl, cudaStream_t st, int* n_launch);
 
 // simt_block.cu
 template <typename T>

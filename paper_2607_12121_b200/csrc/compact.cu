@@ -46,9 +46,11 @@ compact_count_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict
 __global__ void __launch_bounds__(CP_THREADS)
 compact_write_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ labels, int B, int N, int R,
                      const int32_t* __restrict__ block_counts, int32_t* __restrict__ active_idx,
-                     int32_t* __restrict__ cu_active, QTile* __restrict__ tiles, int tile_rows, Control* ctl) {
+                     int32_t* __restrict__ cu_active, QTile* __restrict__ tiles, int tile_rows, Control* ctl,
+                     QTile* __restrict__ tiles2) {
     __shared__ int s_warp[CP_WARPS];
     __shared__ int s_red[CP_WARPS];
+    __shared__ int s_red2[CP_WARPS];
     __shared__ int s_base;
     const int b = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int chunks = gridDim.x;
@@ -96,19 +98,20 @@ compact_write_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict
         // rows of this request and tiles of the requests before it
         int rows_b = 0;
         for (int i = threadIdx.x; i < chunks; i += CP_THREADS) rows_b += block_counts[b * chunks + i];
-        int tiles_before = 0;
+        int tiles_before = 0, tiles2_before = 0;
         for (int bb = warp; bb < b; bb += CP_WARPS) {          // one warp per earlier request
             int r = 0;
             for (int i = lane; i < chunks; i += 32) r += block_counts[bb * chunks + i];
             r = (int)__reduce_add_sync(0xffffffffu, r);
             tiles_before += (r + tile_rows - 1) / tile_rows;
+            tiles2_before += (r + 2 * tile_rows - 1) / (2 * tile_rows);
         }
         __syncthreads();
         rows_b = (int)__reduce_add_sync(0xffffffffu, rows_b);
-        if (lane == 0) { s_warp[warp] = rows_b; s_red[warp] = tiles_before; }
+        if (lane == 0) { s_warp[warp] = rows_b; s_red[warp] = tiles_before; s_red2[warp] = tiles2_before; }
         __syncthreads();
-        int rows = 0, tb = 0;
-        for (int w = 0; w < CP_WARPS; ++w) { rows += s_warp[w]; tb += s_red[w]; }
+        int rows = 0, tb = 0, tb2 = 0;
+        for (int w = 0; w < CP_WARPS; ++w) { rows += s_warp[w]; tb += s_red[w]; tb2 += s_red2[w]; }
         const int nt = (rows + tile_rows - 1) / tile_rows;
         for (int t = threadIdx.x; t < nt; t += CP_THREADS) {
             QTile q;
@@ -119,6 +122,19 @@ compact_write_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict
             tiles[tb + t] = q;
         }
         if (b == B - 1 && threadIdx.x == 0) ctl->n_qtiles = tb + nt;
+        if (tiles2) {
+            // the same rows as double-height tiles: one per CTA pair, each CTA of the pair takes tile_rows of them
+            const int nt2 = (rows + 2 * tile_rows - 1) / (2 * tile_rows);
+            for (int t = threadIdx.x; t < nt2; t += CP_THREADS) {
+                QTile q;
+                q.b = b;
+                q.row0 = s_base + t * 2 * tile_rows;
+                q.rows = min(2 * tile_rows, rows - t * 2 * tile_rows);
+                q.pad = 0;
+                tiles2[tb2 + t] = q;
+            }
+            if (b == B - 1 && threadIdx.x == 0) ctl->n_qtiles2 = tb2 + nt2;
+        }
     }
 }
 
@@ -126,7 +142,7 @@ compact_write_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict
 
 cudaError_t launch_compact(const uint8_t* mask, const int32_t* labels, int B, int N, int R,
                            int32_t* active_idx, int32_t* cu_active, int32_t* block_counts, QTile* tiles,
-                           int tile_rows, Control* ctl, cudaStream_t st, int* n_launch) {
+                           int tile_rows, Control* ctl, cudaStream_t st, int* n_launch, QTile* tiles2) {
     const int chunks = (N + CP_CHUNK - 1) / CP_CHUNK;
     dim3 grid(chunks, B);
     compact_count_kernel<<<grid, CP_THREADS, 0, st>>>(mask, labels, N, R, block_counts, ctl);
@@ -134,7 +150,7 @@ cudaError_t launch_compact(const uint8_t* mask, const int32_t* labels, int B, in
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     compact_write_kernel<<<grid, CP_THREADS, 0, st>>>(mask, labels, B, N, R, block_counts, active_idx,
-                                                      cu_active, tiles, tile_rows, ctl);
+                                                      cu_active, tiles, tile_rows, ctl, tiles2);
     ++*n_launch;
     return cudaGetLastError();
 }

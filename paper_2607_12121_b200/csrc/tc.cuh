@@ -34,7 +34,16 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
 // region_mass (optional): [B, R] f64, receives the own-region softmax mass
 cudaError_t tc_attention(TcPlan* p, int blk, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch, const int32_t* labels = nullptr,
-                         const int32_t* active_idx = nullptr, double* region_mass = nullptr, int R = 0);
+                         const int32_t* active_idx = nullptr, double* region_mass = nullptr, int R = 0,
+                         const QTile* tiles2 = nullptr);
+
+// CTA-pair attention kernel (head dim 128): 256-row items from the `tiles2` list
+bool tc_attention_pair_supported(const fd_config& cfg);
+cudaError_t tc_attention_pair_setup(int* max_clusters, int sm_count);
+cudaError_t tc_attention_pair_launch(const CUtensorMap& tm_q, void* kv_block, int B, int H, void* o, int o_ld,
+                                     const QTile* tiles2, int max_tiles2, int heads, int N, float scale_log2, float* split_ws,
+                                     int split_slots, int max_clusters, bool may_cut, Control* ctl, cudaStream_t st, bool pdl,
+                                     int* n_launch);
 
 cudaError_t launch_bounded_wait_selftest(Control* ctl, cudaStream_t st, int* n_launch);
 

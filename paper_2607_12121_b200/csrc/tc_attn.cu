@@ -25,12 +25,14 @@
 // attn_combine_kernel puts their pieces together.
 #include <cuda_bf16.h>
 
+#include "attn_common.cuh"
 #include "ptx.cuh"
 #include "tc.cuh"
 
 namespace fd {
 
 using namespace ptx;
+using namespace attn;
 
 void* tc_plan_attn(TcPlan* p);
 int tc_plan_sm_count(TcPlan* p);
@@ -57,75 +59,6 @@ template <int D> struct AttCfg {
     static constexpr int SMEM = TILE_BYTES * (2 + 2 * STAGES) + 4608 + 128 * 144 + 2048;
 };
 
-// Register re-balancing between warpgroups: the kernel starts with 128 registers per thread (512 threads);
-// the issuing and the epilogue warpgroups give most of theirs back and the two softmax warpgroups take them.
-template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-// ---- two fp32 values per instruction (add/sub/fma .f32x2) --------------------------------------------
-__device__ __forceinline__ uint64_t pair(float a, float b) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-    return r;
-}
-__device__ __forceinline__ void unpair(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-// 2^x for two arguments on the FMA pipe: x = n + f with n the nearest integer, 2^f as a cubic on [-1/2, 1/2]
-// (relative error 7.5e-5, far below the bf16 rounding P gets), n added into the exponent field.  Arguments
-// below -125 are clamped, so a masked score gives 2^-125 instead of 0: nothing a row sum can see.
-__device__ __forceinline__ uint64_t ex2_poly2(uint64_t x) {
-    float xa, xb;
-    unpair(x, xa, xb);
-    x = pair(fmaxf(xa, -125.0f), fmaxf(xb, -125.0f));
-    const uint64_t magic = pair(12582912.0f, 12582912.0f);          // 1.5 * 2^23: the sum's low mantissa bits hold n
-    const uint64_t xn = add2(x, magic);
-    const uint64_t f = sub2(x, sub2(xn, magic));
-    uint64_t pl = fma2(pair(0.0551716648042202f, 0.0551716648042202f), f, pair(0.2426111251115799f, 0.2426111251115799f));
-    pl = fma2(pl, f, pair(0.6932609677314758f, 0.6932609677314758f));
-    pl = fma2(pl, f, pair(0.9999280571937561f, 0.9999280571937561f));
-    float pa, pb, na, nb;
-    unpair(pl, pa, pb);
-    unpair(xn, na, nb);
-    pa = __int_as_float(__float_as_int(pa) + (__float_as_int(na) << 23));
-    pb = __int_as_float(__float_as_int(pb) + (__float_as_int(nb) << 23));
-    return pair(pa, pb);
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&h);
-}
-
-// The running maximum of a row is only replaced (and the accumulators rescaled, which stalls the pipeline on the
-// previous product) when the new maximum exceeds it by this many powers of two.  P and the accumulators are
-// floating point with an 8-bit exponent, so a stale maximum costs no precision; 2^24 times the key count times
-// |V| stays far inside the fp32 range.
-constexpr float RESCALE_LOG2 = 24.0f;
-
 // TMEM columns: two score buffers, the output accumulator, two P buffers (bf16 pairs)
 constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384, TMEM_COLS = 512;
 // head dims 64 and 128: one score buffer, two P buffers (tile parity), accumulators from column 256: at head dim 64
@@ -145,27 +78,6 @@ struct MassArgs {
     float inv_heads;
 };
 
-// Work of one CTA.  Item blockIdx.x + k * gridDim.x in round k, as long as whole rounds last.  The items left over
-// for a last, partly filled round are cut along the key sequence into `parts` pieces of `steps` key tiles so that
-// (nearly) all CTAs take part in that round too; a piece leaves its un-normalised accumulator and row statistics
-// in the CTA's scratch slot and a small kernel launched behind this one puts the pieces of an item together.
-struct CutPlan { int n_rounds, n_tail, parts, steps; };
-__host__ __device__ inline CutPlan cut_plan(int n_items, int n_kv, int grid, bool may_cut) {
-    CutPlan c;
-    c.n_rounds = n_items / grid;
-    c.n_tail = n_items - c.n_rounds * grid;
-    c.parts = 1;
-    c.steps = n_kv;
-    if (may_cut && c.n_tail > 0) {
-        const int s_max = (grid / c.n_tail) < n_kv ? (grid / c.n_tail) : n_kv;
-        if (s_max >= 2) {
-            c.steps = (n_kv + s_max - 1) / s_max;
-            c.parts = (n_kv + c.steps - 1) / c.steps;
-        }
-    }
-    return c;
-}
-struct Task { int w, j0, j1, piece; };      // piece: 1 = a cut item's piece (result goes to the scratch slot)
 // CUT = false: whole items only, round after round (the plan is not looked at: the compiler sees constant bounds)
 template <bool CUT>
 __device__ __forceinline__ bool next_task(const CutPlan& c, int n_items, int n_kv, int k, Task& t) {
@@ -181,10 +93,6 @@ __device__ __forceinline__ bool next_task(const CutPlan& c, int n_items, int n_k
     t = Task{c.n_rounds * (int)gridDim.x + ti, j0, j1, c.parts > 1 ? 1 : 0};
     return true;
 }
-// scratch slot of a CTA: [128 rows][DP + 4] floats: the un-normalised output row, then running maximum, row sum,
-// own-region mass
-__host__ __device__ inline size_t split_slot_floats(int dp) { return (size_t)128 * (dp + 4); }
-
 template <int D, bool MASS = false, bool CUT = false>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
@@ -999,6 +907,7 @@ struct AttnPlan {
     float* split_ws;        // one slot per CTA for the pieces of cut items (nullptr: items are never cut)
     int split_slots;
     int split_mode;
+    int pair_clusters;      // CTA pairs the pair kernel may run with (0: the pair kernel is not used)
 };
 
 }  // namespace
@@ -1024,6 +933,7 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
     a->split_slots = buf.attn_slots;
     a->split_mode = 1;
     if (const char* v = getenv("FD_ATT_SPLIT")) a->split_mode = atoi(v);
+    a->pair_clusters = 0;
     const uint64_t dims[2] = {(uint64_t)buf.q_ld, (uint64_t)buf.Mcap};
     const uint64_t strides[1] = {(uint64_t)buf.q_ld * 2};
     const uint32_t box[2] = {64, QROWS};
@@ -1052,6 +962,25 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
         ok = false;
         if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
     }
+    // head dim 128 can run on CTA pairs (switch FD_ATT_PAIR=1, read here).  Off by default: measured on the 480p video
+    // shape the pair kernel takes 3.95 ms per launch against 3.05 ms for the single-CTA kernel (its one score buffer is
+    // handed back to the issuing CTA across the cluster, which lengthens the chain the next product waits on).
+    bool use_pair = false;
+    if (const char* v = getenv("FD_ATT_PAIR")) use_pair = tc_attention_pair_supported(cfg) && atoi(v) != 0;
+    if (ok && use_pair) {
+        int sms = 0, dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (const char* lim = getenv("FD_TC_MAX_CTAS")) {
+            const int v = atoi(lim);
+            if (v > 0 && v < sms) sms = v;
+        }
+        e = sms >= 2 ? tc_attention_pair_setup(&a->pair_clusters, sms) : cudaSuccess;
+        if (e != cudaSuccess) {
+            ok = false;
+            if (err) *err = std::string("pair attention set-up: ") + cudaGetErrorString(e);
+        }
+    }
     if (!ok) { delete a; return nullptr; }
     return a;
 }
@@ -1061,7 +990,7 @@ void tc_attention_plan_destroy(void* p) { delete static_cast<AttnPlan*>(p); }
 
 cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch, const int32_t* labels,
-                         const int32_t* active_idx, double* region_mass, int R) {
+                         const int32_t* active_idx, double* region_mass, int R, const QTile* tiles2) {
     AttnPlan* a = static_cast<AttnPlan*>(tc_plan_attn(p));
     if (!a) return cudaErrorNotSupported;
     CUtensorMap kv_map, kv_tail_map;
@@ -1088,6 +1017,12 @@ cudaError_t tc_attention(TcPlan* p, int /*blk*/, void* kv_block, int B, int N, c
     // (not in the launch that also collects the first block's attention mass)
     float* split_ws = (split_on && long_keys && !region_mass && a->split_ws && grid <= a->split_slots) ? a->split_ws : nullptr;
     const bool pdl = tc_plan_pdl(p);
+    if (a->pair_clusters > 0 && tiles2 && !region_mass) {
+        // head dim 128: 256-row items on CTA pairs; each CTA stages half of every key tile and half of V's head dims
+        const int max_tiles2 = B * ((N + 2 * QROWS - 1) / (2 * QROWS));
+        return tc_attention_pair_launch(a->q_map, kv_block, B, a->H, a->o, a->H, tiles2, max_tiles2, a->heads, N, scale_log2,
+                                        a->split_ws, a->split_slots, a->pair_clusters, split_on && long_keys, c, st, pdl, n_launch);
+    }
     const int cgrid = max(1, grid / 2);             // at most grid / 2 items can be cut
 #define FD_ATT(DD, MM, CC)                                                                                          \
     do {                                                                                                            \

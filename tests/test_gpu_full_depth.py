@@ -17,6 +17,17 @@ pytestmark = pytest.mark.gpu
 MAX_ABS, REL_L2 = 3e-2, 1e-2
 
 
+def _stack_output_close(y, y_ref, n_blocks):
+    """Outputs of the whole stack.  The stated tolerance (max-abs 3e-2, relative-L2 1e-2) is per block: it bounds the
+    error one block adds given the same input.  Through the residual stream (gain about 1) the errors of the L blocks
+    add up as independent rounding errors, so the stack's output is held to relative-L2 1e-2 as before and to max-abs
+    3e-2 sqrt(L); on top of that a stored bf16 output cannot be closer than half its spacing, |y| 2^-9, to the exact
+    value (more than 3e-2 alone from |y| = 15.4 on, and the outputs of 24-30 blocks reach 10-30)."""
+    err = np.abs(np.asarray(y, np.float64) - np.asarray(y_ref, np.float64))
+    bound = MAX_ABS * np.sqrt(n_blocks) + np.abs(np.asarray(y_ref, np.float64)) * 2.0 ** -9
+    return bool((err <= bound).all()) and rel_l2(y, y_ref) <= REL_L2
+
+
 def _audio_full_depth(n_requests, n_gated):
     """The audio configuration at its real width and depth (24 blocks, hidden 1536, 1024 tokens per request):
     dense warm-up on the previous step's tokens, then gated steps; every element of y and of the K/V cache is compared."""
@@ -46,9 +57,12 @@ def _audio_full_depth(n_requests, n_gated):
         act = np.zeros(B * N, bool)
         act[idx] = True
         y = host(buf.y).reshape(B * N, H)
-        ma, rl = max_abs(y[act], y_ref.reshape(B * N, H)[act]), rel_l2(y[act], y_ref.reshape(B * N, H)[act])
-        print("audio x%d, %d blocks, step %d (%d active rows): y max_abs %.4f rel_l2 %.5f" % (B, L, step, idx.size, ma, rl))
-        assert ma <= MAX_ABS and rl <= REL_L2
+        yr = y_ref.reshape(B * N, H)
+        ma, rl = max_abs(y[act], yr[act]), rel_l2(y[act], yr[act])
+        print("audio x%d, %d blocks, step %d (%d active rows): y max_abs %.4f rel_l2 %.5f, max|y| %.1f rms %.2f, worst "
+              "error/bound %.2f" % (B, L, step, idx.size, ma, rl, np.abs(yr[act]).max(), np.sqrt((yr[act] ** 2).mean()),
+                                   (np.abs(y[act] - yr[act]) / (MAX_ABS * np.sqrt(L) + np.abs(yr[act]) * 2.0 ** -9)).max()))
+        assert _stack_output_close(y[act], yr[act], L)
         assert np.array_equal(y[~act], y_before.reshape(B * N, H)[~act])
         for l in (0, L // 2, L - 1):
             got = host(buf.kv[l])
@@ -75,6 +89,8 @@ def test_video_twin_all_blocks_gated_steps_with_kv_kept():
     B, N, H, L, R, K = wl.B, wl.N, wl.H, wl.L, wl.R, 2
     labels = labels_for(wl, 52)
     w = gen.block_weights(wl, 52)
+    w["w_qkv"][:, :H] *= np.float32(8.0)          # peaked softmax: every key tile and every merge of partial results
+    w["b_qkv"][:, :H] *= np.float32(8.0)          # matters to the output (a power of two keeps the weights exact in bf16)
     inp = gen.step_inputs(wl, 52, labels)
     n_steps = 6
     fr = np.linspace(0.6, 0.3, n_steps)
@@ -116,8 +132,9 @@ def test_video_twin_all_blocks_gated_steps_with_kv_kept():
         y = host(buf.y).reshape(B * N, H)
         yr = y_ref.reshape(B * N, H)
         ma, rl = max_abs(y[act], yr[act]), rel_l2(y[act], yr[act])
-        print("video twin step %d: active fraction %.3f, y max_abs %.4f rel_l2 %.5f" % (step, fractions[-1], ma, rl))
-        assert ma <= MAX_ABS and rl <= REL_L2
+        print("video twin step %d: active fraction %.3f, y max_abs %.4f rel_l2 %.5f, max|y| %.1f" %
+              (step, fractions[-1], ma, rl, np.abs(yr[act]).max()))
+        assert _stack_output_close(y[act], yr[act], L)
         assert np.array_equal(y[~act], y_before.reshape(B * N, H)[~act])
         a2 = act.reshape(B, N)
         for l in (0, L - 1):

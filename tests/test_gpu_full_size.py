@@ -114,7 +114,10 @@ def test_video_full_shape():
 # tile left out, a wrong rescale) moves y by less than the tolerance.  Scaling the query projection makes the
 # softmax peaked (a handful of keys carry most of a row's mass), so every key tile and the order-independent
 # merging of partial results matter to y; the MMDiT and video shapes run the cut-and-combine path at its real lengths.
-PEAK_GAIN = 8.0
+# Gain 4: measured on a B200, a library that leaves the last key tile out of P V then misses by max-abs 0.37-0.73
+# (12-24 times the tolerance) at all four shapes, while the correct one stays at 0.016-0.025; from gain 8 on (video)
+# the bf16 rounding of the queries itself moves near-tied softmax rows past the tolerance.
+PEAK_GAIN = 4.0
 
 
 def test_audio_full_shape_peaked_attention():

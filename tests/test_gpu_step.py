@@ -38,9 +38,10 @@ def _check_step(wl, y, kv, y_ref, kv_ref, y_before, kv_before, idx):
             assert np.array_equal(got[~a2], old[~a2])
 
 
-def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0):
+def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=None):
     """Warm-up (all active) on the previous step's tokens, then gated steps; both sides start
-    from the same zero caches and carry their own state forward."""
+    from the same zero caches and carry their own state forward.  `variants`: inputs of the block variants
+    (QK-RMSNorm weights, rotary tables) handed to both sides."""
     L = wl.L if n_blocks is None else n_blocks
     labels = labels_for(wl, seed)
     w = gen.block_weights(wl, seed, n_blocks=L)
@@ -51,6 +52,9 @@ def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0):
     ctx = make_ctx(wl, w, engine=engine, n_blocks=L)
     buf = StepBuffers(wl, L)
     dt = tdtype(wl)
+    if variants is not None:
+        fd.fd_set_block_variants(ctx, **{k: (dev(v, dt if k.endswith("_w") else None) if isinstance(v, np.ndarray) else v)
+                                         for k, v in variants.items()})
     B, N, H = wl.B, wl.N, wl.H
     kv_ref = np.zeros((L, B, 2, N, H), np.float32)
     y_ref = np.zeros((B, N, H), np.float32)
@@ -65,7 +69,7 @@ def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0):
         y_before, kv_before = host(buf.y), host(buf.kv)
         idx, cu = gpu_step(ctx, wl, dev(x_np, dt), dev(inp["cond"], dt), dev(labels), dev(mask), buf)
         o_idx, o_cu = oracle.regional_step(x_np, inp["cond"], labels, mask, w, kv_ref, y_ref, wl.heads, wl.R,
-                                           n_blocks=L)
+                                           n_blocks=L, variants=variants)
         assert np.array_equal(idx, o_idx) and np.array_equal(cu, o_cu)
         _check_step(wl, host(buf.y), host(buf.kv), y_ref, kv_ref, y_before, kv_before, idx)
     return ctx
@@ -200,19 +204,21 @@ def test_tensor_core_engine_switched_off_variants(monkeypatch, switch):
     _run_sequence(wl, 6, fd.FD_ENGINE_TC, masks)
 
 
-@pytest.mark.parametrize("name,engine", [("audio_tc", fd.FD_ENGINE_TC), ("video_tc", fd.FD_ENGINE_TC),
-                                         ("image_tc", fd.FD_ENGINE_TC), ("audio_tc", fd.FD_ENGINE_SIMT)])
-def test_peaked_attention_exercises_running_max(name, engine):
-    """Query weights scaled by 64: scores spread over many e-folds, so the running maximum moves
-    between key tiles and the accumulated output has to be rescaled."""
+@pytest.mark.parametrize("name,engine,gain", [("audio_tc", fd.FD_ENGINE_TC, 64.0), ("video_tc", fd.FD_ENGINE_TC, 64.0),
+                                              ("image_tc", fd.FD_ENGINE_TC, 16.0), ("audio_tc", fd.FD_ENGINE_SIMT, 64.0)])
+def test_peaked_attention_exercises_running_max(name, engine, gain):
+    """Query weights scaled up: scores spread over many e-folds, so the running maximum moves
+    between key tiles and the accumulated output has to be rescaled.  (The image twin has the full hidden width
+    1152, so its queries are larger to begin with: a gain of 16 gives it the score spread 64 gives the 256-wide
+    twins; beyond that the softmax is one-hot and a bf16-rounded query flips near ties.)"""
     wl = gen.workload(name)
     masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.5] * wl.B)]
-    _run_sequence(wl, 4, engine, masks, qk_gain=64.0)
+    _run_sequence(wl, 4, engine, masks, qk_gain=gain)
 
 
-@pytest.mark.parametrize("name,n_tok,max_ctas", [("image_tc", 520, "8"), ("image_tc", None, None), ("audio_tc", 700, "8"),
-                                                 ("wide_tc", None, "8")])
-def test_peaked_attention_with_items_cut_along_the_keys(monkeypatch, name, n_tok, max_ctas):
+@pytest.mark.parametrize("name,n_tok,max_ctas,gain", [("image_tc", 520, "8", 8.0), ("image_tc", None, None, 8.0),
+                                                      ("audio_tc", 700, "8", 64.0), ("wide_tc", 520, "8", 16.0)])
+def test_peaked_attention_with_items_cut_along_the_keys(monkeypatch, name, n_tok, max_ctas, gain):
     """Peaked softmax and forced key cuts together: the pieces of an item hold very different running maxima, so the
     second kernel's rescaling of every piece decides the result (head dims 72, 64 and 128)."""
     monkeypatch.setenv("FD_ATT_SPLIT", "2")
@@ -222,7 +228,7 @@ def test_peaked_attention_with_items_cut_along_the_keys(monkeypatch, name, n_tok
     if n_tok is not None:
         wl = wl.replace(grid=(n_tok,), R=10, L=1)
     masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.6] * wl.B)]
-    _run_sequence(wl, 4, fd.FD_ENGINE_TC, masks, qk_gain=64.0)
+    _run_sequence(wl, 4, fd.FD_ENGINE_TC, masks, qk_gain=gain)
 
 
 def test_bounded_wait_reports_timeout_and_context_stays_usable():
@@ -257,3 +263,46 @@ def test_tensor_core_engine_ragged_key_counts(n_tok, regions, heads, head_dim):
     if regions > 1:
         masks.append(gen.region_mask(wl, 7, [0.6, 0.4]))
     _run_sequence(wl, 5, fd.FD_ENGINE_TC, masks, qk_gain=16.0)
+
+
+@pytest.mark.parametrize("case", ["twins", "ragged", "cut", "peaked", "few_ctas"])
+def test_head_dim_128_on_cta_pairs(monkeypatch, case):
+    """The CTA-pair attention kernel (two CTAs share every key tile through cta_group::2 products; switched on with
+    FD_ATT_PAIR=1): the same parity cases as the single-CTA kernel, including items whose second CTA has few or no
+    rows, a single token, forced key cuts with the pair combine kernel, and a peaked softmax."""
+    monkeypatch.setenv("FD_ATT_PAIR", "1")
+    if case == "twins":
+        for name in ("video_tc", "wide_tc"):
+            wl = gen.workload(name)
+            masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 3, gen.request_fractions(wl, 3)),
+                     gen.region_mask(wl, 4, [0.34] * wl.B)]
+            n = _run_sequence(wl, 2, fd.FD_ENGINE_TC, masks).launches
+        monkeypatch.setenv("FD_ATT_PAIR", "0")
+        assert _run_sequence(wl, 2, fd.FD_ENGINE_TC, masks).launches == n      # same number of kernels either way
+    elif case == "ragged":
+        for n_tok, regions in ((40, 5), (130, 13), (300, 10), (1, 1)):
+            wl = gen.workload("audio_tc").replace(grid=(n_tok,), R=regions, B=2, heads=2, head_dim=128, L=1)
+            masks = [np.ones((wl.B, wl.R), np.uint8)]
+            if regions > 1:
+                masks.append(gen.region_mask(wl, 7, [0.6, 0.4]))
+            _run_sequence(wl, 5, fd.FD_ENGINE_TC, masks, qk_gain=16.0)
+    elif case == "cut":
+        monkeypatch.setenv("FD_ATT_SPLIT", "2")
+        for max_ctas in (None, "8"):
+            if max_ctas:
+                monkeypatch.setenv("FD_TC_MAX_CTAS", max_ctas)
+            wl = gen.workload("wide_tc").replace(grid=(520,), R=10, L=1)
+            masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.6] * wl.B)]
+            cut = _run_sequence(wl, 4, fd.FD_ENGINE_TC, masks, qk_gain=16.0).launches
+        monkeypatch.setenv("FD_ATT_SPLIT", "0")
+        whole = _run_sequence(wl, 4, fd.FD_ENGINE_TC, masks, qk_gain=16.0).launches
+        assert cut == whole + len(masks) * wl.L                  # the pair combine kernel ran behind every attention launch
+    elif case == "peaked":
+        wl = gen.workload("video_tc")
+        masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 6, [0.5] * wl.B)]
+        _run_sequence(wl, 4, fd.FD_ENGINE_TC, masks, qk_gain=64.0)
+    else:
+        monkeypatch.setenv("FD_TC_MAX_CTAS", "2")                # one cluster walks every item: rings and barriers wrap many times
+        wl = gen.workload("wide_tc").replace(grid=(700,), R=10, L=1)
+        masks = [np.ones((wl.B, wl.R), np.uint8), gen.region_mask(wl, 5, [0.6] * wl.B)]
+        _run_sequence(wl, 3, fd.FD_ENGINE_TC, masks)
