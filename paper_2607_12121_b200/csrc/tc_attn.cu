@@ -963,8 +963,8 @@ void* tc_attention_plan_create(const fd_config& cfg, const TcBuffers& buf, std::
         if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
     }
     // head dim 128 can run on CTA pairs (switch FD_ATT_PAIR=1, read here).  Off by default: measured on the 480p video
-    // shape the pair kernel takes 3.95 ms per launch against 3.05 ms for the single-CTA kernel (its one score buffer is
-    // handed back to the issuing CTA across the cluster, which lengthens the chain the next product waits on).
+    // shape the pair kernel takes 4.4 ms per launch against 3.05 ms for the single-CTA kernel (the reasons, with the
+    // timestamps that show them, are in the pair kernel's file header).
     bool use_pair = false;
     if (const char* v = getenv("FD_ATT_PAIR")) use_pair = tc_attention_pair_supported(cfg) && atoi(v) != 0;
     if (ok && use_pair) {

@@ -11,8 +11,16 @@
 // draws 8.6 TB/s from L2 across the chip).  No load is multicast: every CTA fetches what it stages itself.
 // Key tiles are 64 keys so that each softmax warpgroup has a score buffer of its own (2 x 64 score columns, 2 x 32
 // P columns and 2 x 128 accumulator columns of TMEM): the product for tile g + 2 then only needs the scores of
-// tile g to have left its buffer, which happened a whole tile earlier, and the hand-back of a buffer to the
-// issuing CTA (a cross-CTA barrier) is off the critical chain.
+// tile g to have left its buffer, which happened a whole tile earlier.
+// MEASURED, AND WHY THIS KERNEL IS NOT THE DEFAULT (switch FD_ATT_PAIR=1): on the 480p video shape it halves the
+// bytes drawn from L2 (11.7 GB per launch against 23.4 GB), yet takes 4.4 ms per launch against 3.05 ms for the
+// single-CTA kernel (3.95 ms with 128-key tiles and one shared score buffer).  Timestamps taken inside the kernel show
+// why: the issuing thread needs about 70 ns per cta_group::2 product instruction whatever its size (0.55 us for the
+// eight N = 64 products of a score tile, 0.35 us for the four of P V), where the products themselves are 16-33 ns of
+// tensor-core work each; a pair instruction only pays off when it carries N = 256 columns, as in the GEMMs.  An
+// attention key tile cannot be that wide: its scores, P and two accumulators must fit the 512 TMEM columns.
+// Passing the second CTA's barrier arrivals through relay threads instead of the softmax warps made it slower still
+// (6.0 ms): every extra hop across the cluster adds most of a microsecond to the chain product -> softmax -> product.
 //   warp 0        TMA producer (each CTA): Q tile double buffered across items, K / V halves in a ring
 //   warps 1, 2    of the pair's first CTA issue S = Q K^T and O += P V for both CTAs; completion is
 //                 broadcast to both CTAs' barriers with multicast commits
