@@ -186,8 +186,22 @@ typedef struct {
     float qk_norm_eps;
     const float* rope_cos;
     const float* rope_sin;
+    const void* q_norm_w_text; /* [L, head_dim]: QK-norm weights of the second stream (fd_set_text_stream), both or */
+    const void* k_norm_w_text; /* neither; NULL = the second stream shares q_norm_w / k_norm_w                    */
 } fd_block_variants;
 fd_status fd_set_block_variants(fd_ctx* ctx, const fd_block_variants* v);
+
+/*
+ * Dual-stream blocks (the joint text-image architecture of the paper's FLUX.1-dev and SD3-Medium models; no
+ * definition in the paper, this is the published structure): the tokens of a request belong to one of two streams,
+ * and a token's stream selects the weights of everything that acts per token -- the adaLN conditioning (w_ada,
+ * b_ada), the QKV projection, the QK-norm weights, the out-projection and the MLP -- while the attention stays joint
+ * over all tokens of the request.  The second stream is the always-active tokens (label R: the text tokens of a
+ * joint text-image request); `text_weights` has the layout of fd_weights and is borrowed until the next call or
+ * fd_destroy.  NULL returns to a single stream.  Each projection then runs as two launches: one finishes the first
+ * stream's rows, one walks only the row tiles that hold rows of the second stream.
+ */
+fd_status fd_set_text_stream(fd_ctx* ctx, const fd_weights* text_weights);
 
 /*
  * The Patch Gate on the paper's own signal (Sec. 4.2): the refinement importance of a patch is the block mean of

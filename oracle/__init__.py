@@ -28,6 +28,16 @@ from .gate import activity_gate, attention_gate, attention_mass, compact, initia
 from .sampler import embed as sampler_embed, update as sampler_update, token_drift  # noqa: F401
 from .partitioner import partition, partition_request, saliency, quantise, allocate, best_cut  # noqa: F401
 
+class _Stream(ctypes.Structure):          # fdo_stream of regional_block.c
+    _fields_ = [(n, ctypes.c_void_p) for n in ("mod", "w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2",
+                                               "qn_w", "kn_w")]
+
+
+class _DenseWeights(ctypes.Structure):    # fdo_dense_weights of dense_block.c
+    _fields_ = [(n, ctypes.c_void_p) for n in ("w_ada", "b_ada", "w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2",
+                                               "b_fc2", "qn_w", "kn_w")]
+
+
 _lib = None
 _f = ctypes.POINTER(ctypes.c_float)
 _i = ctypes.POINTER(ctypes.c_int32)
@@ -42,6 +52,8 @@ def _load():
         _lib.fdo_dense_block.restype = ctypes.c_int
         _lib.fdo_regional_block_v.restype = ctypes.c_int
         _lib.fdo_dense_block_v.restype = ctypes.c_int
+        _lib.fdo_regional_block_s.restype = ctypes.c_int
+        _lib.fdo_dense_block_d.restype = ctypes.c_int
     return _lib
 
 
@@ -71,44 +83,53 @@ def adaln(cond: np.ndarray, w_ada: np.ndarray, b_ada: np.ndarray) -> np.ndarray:
     return mod
 
 
-def _variant_args(variants, l: int, dh: int, N: int):
-    """ctypes arguments of the block variants of block ``l`` (QK-RMSNorm weights [L,dh], RoPE tables [N,dh/2]);
-    ``variants`` is None or a dict with any of q_norm_w, k_norm_w, qk_norm_eps, rope_cos, rope_sin."""
-    v = variants or {}
-    keep = []
-
-    def arr(a, shape):
-        if a is None:
-            return None
-        a = _c(a)
-        assert a.shape == shape, (a.shape, shape)
-        keep.append(a)
-        return _fp(a)
-
-    qn = arr(None if v.get("q_norm_w") is None else v["q_norm_w"][l], (dh,))
-    kn = arr(None if v.get("k_norm_w") is None else v["k_norm_w"][l], (dh,))
-    rc = arr(v.get("rope_cos"), (N, dh // 2))
-    rs = arr(v.get("rope_sin"), (N, dh // 2))
-    return (qn, kn, ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))), rc, rs), keep
+def _addr(a: Optional[np.ndarray], keep: list) -> Optional[int]:
+    if a is None:
+        return None
+    a = _c(a)
+    keep.append(a)
+    return a.ctypes.data
 
 
 def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w: Dict[str, np.ndarray],
                    l: int, kv_l: np.ndarray, heads: int, ln_eps: float = 1e-6,
-                   finish: Optional[np.ndarray] = None, variants=None) -> np.ndarray:
-    """One block over the compact rows ``u_in`` [A,H]; ``kv_l`` [B,2,N,H] is updated in place."""
+                   finish: Optional[np.ndarray] = None, variants=None, mod_text: Optional[np.ndarray] = None,
+                   tok_text: Optional[np.ndarray] = None) -> np.ndarray:
+    """One block over the compact rows ``u_in`` [A,H]; ``kv_l`` [B,2,N,H] is updated in place.
+    Dual stream: ``variants["text"]`` holds the second stream's weights (same keys as ``w``, optionally its own
+    q_norm_w / k_norm_w), ``mod_text`` [B,6H] its adaLN vectors and ``tok_text`` [B*N] u8 marks its tokens."""
     A, H = u_in.shape
     B, _, N, _ = kv_l.shape
     M = w["w_fc1"].shape[1]
+    dh = H // heads
     assert kv_l.dtype == np.float32 and kv_l.flags["C_CONTIGUOUS"]
     u_out = np.zeros((A, H), np.float32)
     fin = None if finish is None else np.ascontiguousarray(finish, np.int32)
-    vargs, _keep = _variant_args(variants, l, H // heads, N)
-    rc = _load().fdo_regional_block_v(
-        B, N, H, heads, H // heads, M, A, _ip(np.ascontiguousarray(active_idx, np.int32)), _fp(_c(mod)),
-        _fp(_c(w["w_qkv"][l])), _fp(_c(w["b_qkv"][l])), _fp(_c(w["w_o"][l])), _fp(_c(w["b_o"][l])),
-        _fp(_c(w["w_fc1"][l])), _fp(_c(w["b_fc1"][l])), _fp(_c(w["w_fc2"][l])), _fp(_c(w["b_fc2"][l])),
-        ctypes.c_float(ln_eps), _fp(_c(u_in)), _fp(u_out), _fp(kv_l),
-        0 if fin is None else int(fin.size), _ip(fin), *vargs)
+    v = variants or {}
+    keep: list = []
+
+    def stream(ws, md, qn, kn):
+        return _Stream(_addr(md, keep), *[_addr(ws[k][l], keep) for k in ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1",
+                                                                            "w_fc2", "b_fc2")],
+                       _addr(None if qn is None else qn[l], keep), _addr(None if kn is None else kn[l], keep))
+
+    img = stream(w, mod, v.get("q_norm_w"), v.get("k_norm_w"))
+    txt, tt = None, None
+    if v.get("text") is not None:
+        t = v["text"]
+        assert mod_text is not None and tok_text is not None
+        txt = ctypes.byref(stream(t["weights"], mod_text, t.get("q_norm_w", v.get("q_norm_w")),
+                                  t.get("k_norm_w", v.get("k_norm_w"))))
+        tt = np.ascontiguousarray(tok_text, np.uint8)
+        keep.append(tt)
+    rc_, rs_ = _addr(v.get("rope_cos"), keep), _addr(v.get("rope_sin"), keep)
+    if rc_ is not None:
+        assert keep[-2].shape == (N, dh // 2)
+    rc = _load().fdo_regional_block_s(
+        B, N, H, heads, dh, M, A, _ip(np.ascontiguousarray(active_idx, np.int32)), ctypes.byref(img), txt,
+        None if tt is None else tt.ctypes.data_as(ctypes.c_void_p), ctypes.c_float(ln_eps), _fp(_c(u_in)), _fp(u_out), _fp(kv_l),
+        0 if fin is None else int(fin.size), _ip(fin), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))),
+        ctypes.c_void_p(rc_), ctypes.c_void_p(rs_))
     assert rc == 0
     return u_out
 
@@ -126,9 +147,13 @@ def regional_step(x: np.ndarray, cond: np.ndarray, labels: np.ndarray, mask: np.
     L = w["w_qkv"].shape[0] if n_blocks is None else n_blocks
     active_idx, cu_active = compact(mask, labels, R)
     u = np.ascontiguousarray(x.reshape(B * N, H)[active_idx], np.float32)
+    text = (variants or {}).get("text")
+    tok_text = None if text is None else (np.asarray(labels) == R).reshape(-1).astype(np.uint8)   # always-active tokens
     for l in range(L):
         mod = adaln(cond, w["w_ada"][l], w["b_ada"][l])
-        u = regional_block(u, active_idx, mod, w, l, kv[l], heads, ln_eps, variants=variants)
+        mod_t = None if text is None else adaln(cond, text["weights"]["w_ada"][l], text["weights"]["b_ada"][l])
+        u = regional_block(u, active_idx, mod, w, l, kv[l], heads, ln_eps, variants=variants, mod_text=mod_t,
+                           tok_text=tok_text)
     y.reshape(B * N, H)[active_idx] = u
     return active_idx, cu_active
 
@@ -156,18 +181,34 @@ def block0_queries(x, cond, w, active_idx, ln_eps: float = 1e-6) -> np.ndarray:
 
 def dense_block(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], l: int, heads: int,
                 ln_eps: float = 1e-6, variants=None):
-    """One ungated block on whole matrices. Returns x_out [B,N,H], kv [B,2,N,H]."""
+    """One ungated block on whole matrices. Returns x_out [B,N,H], kv [B,2,N,H].  Dual stream: ``variants["text"]``
+    = {"weights": second weight set, "n_text": trailing tokens of every request that belong to it}."""
     B, N, H = x.shape
     M = w["w_fc1"].shape[1]
     Hc = cond.shape[1]
+    dh = H // heads
     x_out = np.empty((B, N, H), np.float32)
     kv = np.empty((B, 2, N, H), np.float32)
-    vargs, _keep = _variant_args(variants, l, H // heads, N)
-    rc = _load().fdo_dense_block_v(
-        B, N, H, heads, H // heads, M, Hc, _fp(_c(cond)), _fp(_c(w["w_ada"][l])), _fp(_c(w["b_ada"][l])),
-        _fp(_c(w["w_qkv"][l])), _fp(_c(w["b_qkv"][l])), _fp(_c(w["w_o"][l])), _fp(_c(w["b_o"][l])),
-        _fp(_c(w["w_fc1"][l])), _fp(_c(w["b_fc1"][l])), _fp(_c(w["w_fc2"][l])), _fp(_c(w["b_fc2"][l])),
-        ctypes.c_float(ln_eps), _fp(_c(x)), _fp(x_out), _fp(kv), *vargs)
+    v = variants or {}
+    keep: list = []
+
+    def weights(ws, qn, kn):
+        return _DenseWeights(*[_addr(ws[k][l], keep) for k in ("w_ada", "b_ada", "w_qkv", "b_qkv", "w_o", "b_o", "w_fc1",
+                                                                 "b_fc1", "w_fc2", "b_fc2")],
+                             _addr(None if qn is None else qn[l], keep), _addr(None if kn is None else kn[l], keep))
+
+    wi = weights(w, v.get("q_norm_w"), v.get("k_norm_w"))
+    wt, n_text = None, 0
+    if v.get("text") is not None:
+        t = v["text"]
+        wt = ctypes.byref(weights(t["weights"], t.get("q_norm_w", v.get("q_norm_w")), t.get("k_norm_w", v.get("k_norm_w"))))
+        n_text = int(t["n_text"])
+    rc_, rs_ = _addr(v.get("rope_cos"), keep), _addr(v.get("rope_sin"), keep)
+    if rc_ is not None:
+        assert keep[-2].shape == (N, dh // 2)
+    rc = _load().fdo_dense_block_d(
+        B, N, H, heads, dh, M, Hc, _fp(_c(cond)), ctypes.byref(wi), wt, n_text, ctypes.c_float(ln_eps), _fp(_c(x)), _fp(x_out),
+        _fp(kv), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))), ctypes.c_void_p(rc_), ctypes.c_void_p(rs_))
     assert rc == 0
     return x_out, kv
 

@@ -126,13 +126,30 @@ int fdo_dense_qk_variants(int N, int heads, int dh, float* Q, float* K, const fl
  * x_in, x_out [B,N,H]; kv_out [B,2,N,H] receives K and V of every position.
  * cond [B,Hc]; adaLN chunk order shift_msa, scale_msa, gate_msa, shift_mlp, scale_mlp, gate_mlp.
  * fdo_dense_block_v adds the block variants (NULL = off): qn_w, kn_w [dh]; rope_cos, rope_sin [N, dh/2].
+ * fdo_dense_block_d is the dual-stream block of joint text-image models: the last n_text tokens of every request
+ * form a second stream with weights of its own for everything that acts per token (conditioning, QKV projection,
+ * QK-norm, out-projection, MLP); the attention runs over all N tokens together.  Written on row ranges of whole
+ * matrices: rows [0, N - n_text) with the first weight set, rows [N - n_text, N) with the second.
  */
+typedef struct {
+    const float *w_ada, *b_ada, *w_qkv, *b_qkv, *w_o, *b_o, *w_fc1, *b_fc1, *w_fc2, *b_fc2, *qn_w, *kn_w;
+} fdo_dense_weights;
+
+int fdo_dense_block_d(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+                      const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
+                      const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
+                      const float* rope_sin);
+
 int fdo_dense_block_v(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const float* w_ada, const float* b_ada, const float* w_qkv, const float* b_qkv,
                       const float* w_o, const float* b_o, const float* w_fc1, const float* b_fc1,
                       const float* w_fc2, const float* b_fc2, float ln_eps, const float* x_in,
                       float* x_out, float* kv_out, const float* qn_w, const float* kn_w, float qk_eps,
-                      const float* rope_cos, const float* rope_sin);
+                      const float* rope_cos, const float* rope_sin) {
+    const fdo_dense_weights w = {w_ada, b_ada, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, qn_w, kn_w};
+    return fdo_dense_block_d(B, N, H, heads, dh, M, Hc, cond, &w, NULL, 0, ln_eps, x_in, x_out, kv_out, qk_eps, rope_cos,
+                             rope_sin);
+}
 
 int fdo_dense_block(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                     const float* w_ada, const float* b_ada, const float* w_qkv, const float* b_qkv,
@@ -143,17 +160,17 @@ int fdo_dense_block(int B, int N, int H, int heads, int dh, int M, int Hc, const
                              b_fc2, ln_eps, x_in, x_out, kv_out, NULL, NULL, 0.f, NULL, NULL);
 }
 
-int fdo_dense_block_v(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
-                      const float* w_ada, const float* b_ada, const float* w_qkv, const float* b_qkv,
-                      const float* w_o, const float* b_o, const float* w_fc1, const float* b_fc1,
-                      const float* w_fc2, const float* b_fc2, float ln_eps, const float* x_in,
-                      float* x_out, float* kv_out, const float* qn_w, const float* kn_w, float qk_eps,
-                      const float* rope_cos, const float* rope_sin) {
+int fdo_dense_block_d(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+                      const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
+                      const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
+                      const float* rope_sin) {
     if (heads * dh != H) return 2;
     if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
+    if (!wt) n_text = 0;
+    if (n_text < 0 || n_text > N) return 4;
     const size_t NH = (size_t)N * H;
     float* act = (float*)malloc(sizeof(float) * (size_t)Hc);
-    float* mod = (float*)malloc(sizeof(float) * (size_t)6 * H);
+    float* mod = (float*)malloc(sizeof(float) * (size_t)2 * 6 * H);
     float* xh = (float*)malloc(sizeof(float) * NH);
     float* qkv = (float*)malloc(sizeof(float) * NH * 3);
     float* Q = (float*)malloc(sizeof(float) * NH);
@@ -163,51 +180,73 @@ int fdo_dense_block_v(int B, int N, int H, int heads, int dh, int M, int Hc, con
     float* hid = (float*)malloc(sizeof(float) * (size_t)N * M);
     int rc = 0;
     if (!act || !mod || !xh || !qkv || !Q || !att || !proj || !res || !hid) { rc = 1; goto done; }
+    /* the two streams as row ranges [lo, hi) of a request's N rows; the second range is empty for a single stream */
+    const int range_lo[2] = {0, N - n_text}, range_hi[2] = {N - n_text, N};
+    const fdo_dense_weights* ws[2] = {wi, wt ? wt : wi};
 
     for (int b = 0; b < B; ++b) {
         const float* X = x_in + (size_t)b * NH;
         float* Kc = kv_out + ((size_t)b * 2 + 0) * NH;
         float* Vc = kv_out + ((size_t)b * 2 + 1) * NH;
 
-        /* conditioning: six H-vectors from SiLU(cond) */
+        /* conditioning: six H-vectors per stream from SiLU(cond) */
         for (int c = 0; c < Hc; ++c) {
             const double v = (double)cond[(size_t)b * Hc + c];
             act[c] = (float)(v / (1.0 + exp(-v)));
         }
-        matmul_nt_bias(act, w_ada, b_ada, 1, Hc, 6 * H, mod);
-        const float *shift_a = mod, *scale_a = mod + H, *gate_a = mod + 2 * H;
-        const float *shift_m = mod + 3 * H, *scale_m = mod + 4 * H, *gate_m = mod + 5 * H;
+        for (int s = 0; s < 2; ++s) matmul_nt_bias(act, ws[s]->w_ada, ws[s]->b_ada, 1, Hc, 6 * H, mod + (size_t)s * 6 * H);
 
-        /* attention branch */
-        layernorm_modulate(X, (size_t)N, H, shift_a, scale_a, ln_eps, xh);
-        matmul_nt_bias(xh, w_qkv, b_qkv, (size_t)N, H, 3 * H, qkv);
+        /* attention branch: per-stream modulation and projection, then joint attention */
+        for (int s = 0; s < 2; ++s) {
+            const size_t lo = (size_t)range_lo[s], n = (size_t)(range_hi[s] - range_lo[s]);
+            if (!n) continue;
+            const float* md = mod + (size_t)s * 6 * H;
+            layernorm_modulate(X + lo * H, n, H, md, md + H, ln_eps, xh + lo * H);
+            matmul_nt_bias(xh + lo * H, ws[s]->w_qkv, ws[s]->b_qkv, n, H, 3 * H, qkv + lo * 3 * H);
+        }
         for (int t = 0; t < N; ++t) {
             memcpy(Q + (size_t)t * H, qkv + (size_t)t * 3 * H, sizeof(float) * (size_t)H);
             memcpy(Kc + (size_t)t * H, qkv + (size_t)t * 3 * H + H, sizeof(float) * (size_t)H);
             memcpy(Vc + (size_t)t * H, qkv + (size_t)t * 3 * H + 2 * H, sizeof(float) * (size_t)H);
         }
-        if (qn_w) rms_norm_heads(Q, N, heads, dh, qn_w, qk_eps);
-        if (kn_w) rms_norm_heads(Kc, N, heads, dh, kn_w, qk_eps);
+        for (int s = 0; s < 2; ++s) {
+            const size_t lo = (size_t)range_lo[s];
+            const int n = range_hi[s] - range_lo[s];
+            if (!n) continue;
+            if (ws[s]->qn_w) rms_norm_heads(Q + lo * H, n, heads, dh, ws[s]->qn_w, qk_eps);
+            if (ws[s]->kn_w) rms_norm_heads(Kc + lo * H, n, heads, dh, ws[s]->kn_w, qk_eps);
+        }
         if (rope_cos) {
             rotate_pairs(Q, N, heads, dh, rope_cos, rope_sin);
             rotate_pairs(Kc, N, heads, dh, rope_cos, rope_sin);
         }
         full_attention(Q, Kc, Vc, N, heads, dh, att);
-        matmul_nt_bias(att, w_o, b_o, (size_t)N, H, H, proj);
-        for (size_t e = 0; e < NH; ++e)
-            res[e] = (float)((double)X[e] + (double)gate_a[e % H] * (double)proj[e]);
-
-        /* MLP branch */
-        layernorm_modulate(res, (size_t)N, H, shift_m, scale_m, ln_eps, xh);
-        matmul_nt_bias(xh, w_fc1, b_fc1, (size_t)N, H, M, hid);
-        for (size_t e = 0; e < (size_t)N * M; ++e) {
-            const double a = (double)hid[e];
-            hid[e] = (float)(0.5 * a * (1.0 + tanh(0.79788456080286535588 * (a + 0.044715 * a * a * a))));
+        for (int s = 0; s < 2; ++s) {
+            const size_t lo = (size_t)range_lo[s], n = (size_t)(range_hi[s] - range_lo[s]);
+            if (!n) continue;
+            const float* gate_a = mod + (size_t)s * 6 * H + 2 * H;
+            matmul_nt_bias(att + lo * H, ws[s]->w_o, ws[s]->b_o, n, H, H, proj + lo * H);
+            for (size_t e = lo * H; e < (lo + n) * H; ++e)
+                res[e] = (float)((double)X[e] + (double)gate_a[e % H] * (double)proj[e]);
         }
-        matmul_nt_bias(hid, w_fc2, b_fc2, (size_t)N, M, H, proj);
+
+        /* MLP branch, per stream */
         float* Y = x_out + (size_t)b * NH;
-        for (size_t e = 0; e < NH; ++e)
-            Y[e] = (float)((double)res[e] + (double)gate_m[e % H] * (double)proj[e]);
+        for (int s = 0; s < 2; ++s) {
+            const size_t lo = (size_t)range_lo[s], n = (size_t)(range_hi[s] - range_lo[s]);
+            if (!n) continue;
+            const float* md = mod + (size_t)s * 6 * H;
+            layernorm_modulate(res + lo * H, n, H, md + 3 * H, md + 4 * H, ln_eps, xh + lo * H);
+            matmul_nt_bias(xh + lo * H, ws[s]->w_fc1, ws[s]->b_fc1, n, H, M, hid + lo * M);
+            for (size_t e = lo * M; e < (lo + n) * M; ++e) {
+                const double a = (double)hid[e];
+                hid[e] = (float)(0.5 * a * (1.0 + tanh(0.79788456080286535588 * (a + 0.044715 * a * a * a))));
+            }
+            matmul_nt_bias(hid + lo * M, ws[s]->w_fc2, ws[s]->b_fc2, n, M, H, proj + lo * H);
+            const float* gate_m = md + 5 * H;
+            for (size_t e = lo * H; e < (lo + n) * H; ++e)
+                Y[e] = (float)((double)res[e] + (double)gate_m[e % H] * (double)proj[e]);
+        }
     }
 done:
     free(act); free(mod); free(xh); free(qkv); free(Q); free(att); free(proj); free(res); free(hid);

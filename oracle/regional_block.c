@@ -123,14 +123,34 @@ int fdo_adaln(int B, int H, int Hc, const float* cond, const float* w_ada, const
  * Rows outside `finish` get no u_out.
  * fdo_regional_block_v adds the block variants: qn_w, kn_w [dh] (QK-RMSNorm, NULL = off), rope_cos, rope_sin
  * [N, dh/2] (NULL = off).
+ * fdo_regional_block_s adds the dual-stream form of joint text-image blocks (the architecture of the paper's
+ * FLUX / SD3 models; this build's reading): a token belongs to one of two streams, and its stream selects the
+ * weights of every per-token operation -- the adaLN vectors, the QKV projection, the QK-norm weights, the
+ * out-projection and the MLP -- while the attention stays joint over all tokens of the request.  tok_text[B*N] marks
+ * the tokens of the second ("text") stream; txt = NULL means a single stream.
  */
+typedef struct {
+    const float *mod;                       /* [B,6H] adaLN vectors of this block for this stream */
+    const float *w_qkv, *b_qkv, *w_o, *b_o, *w_fc1, *b_fc1, *w_fc2, *b_fc2;
+    const float *qn_w, *kn_w;               /* [dh] or NULL */
+} fdo_stream;
+
+int fdo_regional_block_s(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
+                         const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
+                         float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
+                         float qk_eps, const float* rope_cos, const float* rope_sin);
+
 int fdo_regional_block_v(int B, int N, int H, int heads, int dh, int M, int A,
                          const int32_t* active_idx, const float* mod,
                          const float* w_qkv, const float* b_qkv, const float* w_o, const float* b_o,
                          const float* w_fc1, const float* b_fc1, const float* w_fc2, const float* b_fc2,
                          float ln_eps, const float* u_in, float* u_out, float* kv,
                          int n_finish, const int32_t* finish,
-                         const float* qn_w, const float* kn_w, float qk_eps, const float* rope_cos, const float* rope_sin);
+                         const float* qn_w, const float* kn_w, float qk_eps, const float* rope_cos, const float* rope_sin) {
+    const fdo_stream one = {mod, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, qn_w, kn_w};
+    return fdo_regional_block_s(B, N, H, heads, dh, M, A, active_idx, &one, NULL, NULL, ln_eps, u_in, u_out, kv, n_finish,
+                                finish, qk_eps, rope_cos, rope_sin);
+}
 
 int fdo_regional_block(int B, int N, int H, int heads, int dh, int M, int A,
                        const int32_t* active_idx, const float* mod,
@@ -142,13 +162,10 @@ int fdo_regional_block(int B, int N, int H, int heads, int dh, int M, int A,
                                 b_fc2, ln_eps, u_in, u_out, kv, n_finish, finish, NULL, NULL, 0.f, NULL, NULL);
 }
 
-int fdo_regional_block_v(int B, int N, int H, int heads, int dh, int M, int A,
-                       const int32_t* active_idx, const float* mod,
-                       const float* w_qkv, const float* b_qkv, const float* w_o, const float* b_o,
-                       const float* w_fc1, const float* b_fc1, const float* w_fc2, const float* b_fc2,
-                         float ln_eps, const float* u_in, float* u_out, float* kv,
-                         int n_finish, const int32_t* finish,
-                         const float* qn_w, const float* kn_w, float qk_eps, const float* rope_cos, const float* rope_sin) {
+int fdo_regional_block_s(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
+                         const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
+                         float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
+                         float qk_eps, const float* rope_cos, const float* rope_sin) {
     if (heads * dh != H) return 2;
     if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
     (void)B;
@@ -168,10 +185,11 @@ int fdo_regional_block_v(int B, int N, int H, int heads, int dh, int M, int A,
 #pragma omp for schedule(dynamic, 4)
             for (int a = 0; a < A; ++a) {
                 const int b = active_idx[a] / N, j = active_idx[a] % N;
-                const float* md = mod + (size_t)b * 6 * H;
+                const fdo_stream* st = (txt && tok_text[active_idx[a]]) ? txt : img;      /* the token's stream */
+                const float* md = st->mod + (size_t)b * 6 * H;
                 row_ln_modulate(u_in + (size_t)a * H, md + 0 * H, md + 1 * H, H, ln_eps, uh);
-                row_linear(uh, w_qkv, b_qkv, H, 3 * H, qkv);
-                row_qk_variants(qkv, qkv + H, heads, dh, j, qn_w, kn_w, qk_eps, rope_cos, rope_sin);
+                row_linear(uh, st->w_qkv, st->b_qkv, H, 3 * H, qkv);
+                row_qk_variants(qkv, qkv + H, heads, dh, j, st->qn_w, st->kn_w, qk_eps, rope_cos, rope_sin);
                 memcpy(q_all + (size_t)a * H, qkv, sizeof(float) * (size_t)H);
                 memcpy(kv + (((size_t)b * 2 + 0) * N + j) * H, qkv + H, sizeof(float) * (size_t)H);
                 memcpy(kv + (((size_t)b * 2 + 1) * N + j) * H, qkv + 2 * H, sizeof(float) * (size_t)H);
@@ -201,7 +219,8 @@ int fdo_regional_block_v(int B, int N, int H, int heads, int dh, int M, int A,
             for (int i = 0; i < n_rows; ++i) {
                 const int a = finish ? finish[i] : i;
                 const int b = active_idx[a] / N;
-                const float* md = mod + (size_t)b * 6 * H;
+                const fdo_stream* st = (txt && tok_text[active_idx[a]]) ? txt : img;
+                const float* md = st->mod + (size_t)b * 6 * H;
                 const float* Kb = kv + ((size_t)b * 2 + 0) * N * H;
                 const float* Vb = kv + ((size_t)b * 2 + 1) * N * H;
                 const float* q = q_all + (size_t)a * H;
@@ -226,13 +245,13 @@ int fdo_regional_block_v(int B, int N, int H, int heads, int dh, int M, int A,
                     for (int c = 0; c < dh; ++c) o[h * dh + c] = (float)(oacc[c] / denom);
                 }
                 const float* u = u_in + (size_t)a * H;
-                row_linear(o, w_o, b_o, H, H, proj);
+                row_linear(o, st->w_o, st->b_o, H, H, proj);
                 for (int c = 0; c < H; ++c)
                     r1[c] = (float)((double)u[c] + (double)md[2 * H + c] * (double)proj[c]);
                 row_ln_modulate(r1, md + 3 * H, md + 4 * H, H, ln_eps, mh);
-                row_linear(mh, w_fc1, b_fc1, H, M, g);
+                row_linear(mh, st->w_fc1, st->b_fc1, H, M, g);
                 for (int c = 0; c < M; ++c) g[c] = (float)gelu_tanh_d((double)g[c]);
-                row_linear(g, w_fc2, b_fc2, M, H, proj);
+                row_linear(g, st->w_fc2, st->b_fc2, M, H, proj);
                 float* out = u_out + (size_t)a * H;
                 for (int c = 0; c < H; ++c)
                     out[c] = (float)((double)r1[c] + (double)md[5 * H + c] * (double)proj[c]);

@@ -23,7 +23,8 @@ EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region
            "fd_regional_step", "fd_poll_status", "fd_launch_count", "fd_destroy", "fd_last_error",
            "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait",
            "fd_embed_latent", "fd_update_latent", "fd_regional_step_mass", "fd_region_activity_attn",
-           "fd_sched_pack", "fd_sched_form_batch", "fd_rsearch_init", "fd_rsearch_update", "fd_set_block_variants"]
+           "fd_sched_pack", "fd_sched_form_batch", "fd_rsearch_init", "fd_rsearch_update", "fd_set_block_variants",
+           "fd_set_text_stream"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
                "gemm_fc2", "partition", "sampler", "qk_variants"]
@@ -47,7 +48,8 @@ class FdSamplerWeights(ctypes.Structure):
 
 class FdBlockVariants(ctypes.Structure):
     _fields_ = [("q_norm_w", ctypes.c_void_p), ("k_norm_w", ctypes.c_void_p), ("qk_norm_eps", ctypes.c_float),
-                ("rope_cos", ctypes.c_void_p), ("rope_sin", ctypes.c_void_p)]
+                ("rope_cos", ctypes.c_void_p), ("rope_sin", ctypes.c_void_p), ("q_norm_w_text", ctypes.c_void_p),
+                ("k_norm_w_text", ctypes.c_void_p)]
 
 
 class FdRSearch(ctypes.Structure):
@@ -106,6 +108,8 @@ def _load() -> ctypes.CDLL:
     lib.fd_update_latent.argtypes = [vp, ctypes.POINTER(FdSamplerWeights), vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     lib.fd_set_block_variants.restype = i32
     lib.fd_set_block_variants.argtypes = [vp, ctypes.POINTER(FdBlockVariants)]
+    lib.fd_set_text_stream.restype = i32
+    lib.fd_set_text_stream.argtypes = [vp, ctypes.POINTER(FdWeights)]
     lib.fd_launch_count.restype = ctypes.c_int64
     lib.fd_launch_count.argtypes = [vp]
     lib.fd_destroy.restype = i32
@@ -266,15 +270,30 @@ def fd_region_activity_attn(ctx: Context, region_mass, region_sizes, eps, rbar_s
 
 
 def fd_set_block_variants(ctx: Context, q_norm_w=None, k_norm_w=None, qk_norm_eps: float = 1e-6, rope_cos=None,
-                          rope_sin=None) -> None:
+                          rope_sin=None, q_norm_w_text=None, k_norm_w_text=None) -> None:
     """Switches the block variants on (device tensors: QK-RMSNorm weights [L, head_dim] of the context's dtype, rotary
-    tables [max_tokens, head_dim/2] f32) or, with no tensors, off.  The context keeps the tensors alive."""
-    ctx.variant_tensors = (q_norm_w, k_norm_w, rope_cos, rope_sin)
+    tables [max_tokens, head_dim/2] f32; *_text: the second stream's norm weights) or, with no tensors, off.  The
+    context keeps the tensors alive."""
+    ctx.variant_tensors = (q_norm_w, k_norm_w, rope_cos, rope_sin, q_norm_w_text, k_norm_w_text)
     if all(t is None for t in ctx.variant_tensors):
         _check(ctx.handle, lib.fd_set_block_variants(ctx.handle, None))
         return
-    v = FdBlockVariants(_ptr(q_norm_w), _ptr(k_norm_w), float(qk_norm_eps), _ptr(rope_cos), _ptr(rope_sin))
+    v = FdBlockVariants(_ptr(q_norm_w), _ptr(k_norm_w), float(qk_norm_eps), _ptr(rope_cos), _ptr(rope_sin),
+                        _ptr(q_norm_w_text), _ptr(k_norm_w_text))
     _check(ctx.handle, lib.fd_set_block_variants(ctx.handle, ctypes.byref(v)))
+
+
+def fd_set_text_stream(ctx: Context, text_weights: Optional[Dict[str, "object"]]) -> None:
+    """Dual-stream blocks: the tokens with label R use ``text_weights`` (same keys and layout as the context's own
+    weights; device tensors the context keeps alive); None returns to a single stream."""
+    ctx.text_weights = text_weights
+    if text_weights is None:
+        _check(ctx.handle, lib.fd_set_text_stream(ctx.handle, None))
+        return
+    for k, t in text_weights.items():
+        assert t.is_cuda and t.is_contiguous() and t.dtype == ctx.dtype, k
+    w = FdWeights(**{k: text_weights[k].data_ptr() for k, _ in FdWeights._fields_})
+    _check(ctx.handle, lib.fd_set_text_stream(ctx.handle, ctypes.byref(w)))
 
 
 def fd_sched_pack(load, cost, home):

@@ -25,7 +25,7 @@ thread_local std::string g_create_error;
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-    size_t control, acc_ss, acc_cnt, block_counts, tiles, ada_act, mod, resid, act, q, o, g, part, attn_ws, total;
+    size_t control, acc_ss, acc_cnt, block_counts, tiles, text_tiles, ada_act, mod, resid, act, q, o, g, part, attn_ws, total;
     int Mcap, q_ld, tile_cap;
 };
 
@@ -63,8 +63,10 @@ Layout make_layout(const fd_config& c) {
     l.acc_cnt = take(BR * sizeof(int32_t));
     l.block_counts = take((size_t)c.max_batch * ((c.max_tokens + 2047) / 2048 + 1) * sizeof(int32_t));
     l.tiles = take((size_t)2 * l.tile_cap * sizeof(QTile));      // work list, then the list of double-height tiles
+    // dual stream: the 128-row and the 256-row tiles that hold rows of the second stream
+    l.text_tiles = take(((size_t)l.Mcap / 128 + (size_t)l.Mcap / 256 + 2) * sizeof(int32_t));
     l.ada_act = take((size_t)2 * ((c.max_batch + 7) / 8 * 8) * c.cond_dim * 2);   // SiLU(cond): bf16 head + remainder
-    l.mod = take((size_t)c.n_blocks * c.max_batch * 6 * c.hidden * sizeof(float));
+    l.mod = take((size_t)2 * c.n_blocks * c.max_batch * 6 * c.hidden * sizeof(float));   // adaLN vectors, then the second stream's
     l.resid = take((size_t)l.Mcap * c.hidden * sizeof(float));
     l.act = take((size_t)l.Mcap * c.hidden * es);
     l.q = take((size_t)l.Mcap * l.q_ld * es);
@@ -90,6 +92,8 @@ struct fd_ctx {
     std::string err;
     TcPlan* tc;
     fd_block_variants var{};   // block variants (all pointers null: off)
+    fd_weights text_w{};       // second stream's weights (dual stream; w_qkv null: single stream)
+    bool dual = false;
     // optional per-kernel timing
     bool profiling = false;
     struct Span { cudaEvent_t a, b; int group, kernels; };
@@ -170,26 +174,43 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
                           c->tile_rows, ctl, st, &nl, tiles2));
     FD_TRY(FD_PROF_ADALN, launch_adaln<T>(cond, static_cast<const T*>(c->w.w_ada), static_cast<const T*>(c->w.b_ada), mod, L, B, H,
                            Hc, c->ws + l.ada_act, st, &nl));
+    // dual stream: tokens with label R use a second weight set for everything that acts per token
+    const bool dual = c->dual;
+    const long long text_mod_off = (long long)L * B * 6 * H;         // second stream's adaLN vectors follow the first's
+    int32_t* text128 = c->at<int32_t>(l.text_tiles);
+    int32_t* text256 = text128 + l.Mcap / 128 + 1;
+    TextSel ts{nullptr, 0, 0};
+    if (dual) {
+        FD_TRY(FD_PROF_ADALN, launch_adaln<T>(cond, static_cast<const T*>(c->text_w.w_ada), static_cast<const T*>(c->text_w.b_ada),
+                                               mod + text_mod_off, L, B, H, Hc, c->ws + l.ada_act, st, &nl));
+        FD_TRY(FD_PROF_COMPACT, launch_text_tiles(active_idx, labels, R, rows_cap, text128, text256, ctl, st, &nl));
+        ts = TextSel{labels, R, text_mod_off};
+    }
+    // One launch per stream where the weights differ: the first finishes the first stream's rows (all rows when there
+    // is a single stream), the second walks the row tiles that hold rows of the second stream and finishes those.
+    auto stream_ptr = [&](const void* base0, const void* base1, size_t off, int pass) -> const T* {
+        return static_cast<const T*>(pass ? base1 : base0) + off;
+    };
+    const int n_pass = dual ? 2 : 1;
     const int max_tiles = B * ((N + c->tile_rows - 1) / c->tile_rows);
     const bool pdl = c->use_tc && c->tc && tc_plan_pdl(c->tc);
     for (int blk = 0; blk < L; ++blk) {
         const float* mod_b = mod + (size_t)blk * B * 6 * H;
-        const T* w_qkv = static_cast<const T*>(c->w.w_qkv) + (size_t)blk * 3 * H * H;
-        const T* w_o = static_cast<const T*>(c->w.w_o) + (size_t)blk * H * H;
-        const T* w_fc1 = static_cast<const T*>(c->w.w_fc1) + (size_t)blk * M * H;
-        const T* w_fc2 = static_cast<const T*>(c->w.w_fc2) + (size_t)blk * H * M;
         T* kv_b = kv + (size_t)blk * B * 2 * N * H;
 
         EpiParams ep{};
         ep.active_idx = active_idx;
         ep.N = N;
         ep.H = H;
+        ep.labels = labels;
+        ep.R = R;
+        ep.group = -1;
+        ep.text_mod_off = (int32_t)text_mod_off;
 
         // gather (first block) or read the residual stream; LayerNorm; attention-branch modulation
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(blk == 0 ? x : nullptr, resid, resid, act, active_idx, mod_b + 0 * H,
-                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl));
+                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts));
         // QKV projection; K and V rows go straight into the cache
-        ep.bias = static_cast<const T*>(c->w.b_qkv) + (size_t)blk * 3 * H;
         ep.q = q;
         ep.q_ld = l.q_ld;
         if (c->use_tc_attn && tc_attention_head_pad(cf.head_dim) != cf.head_dim) {
@@ -197,21 +218,31 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             ep.q_head_pad = tc_attention_head_pad(cf.head_dim);
         }
         ep.kv = kv_b;
-        if (c->use_tc)
-            FD_TRY(FD_PROF_GEMM_QKV, tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));
-        else
-            FD_TRY(FD_PROF_GEMM_QKV, launch_simt_gemm<T>(EPI_QKV, act, H, w_qkv, 3 * H, H, rows_cap, ep, ctl, st, &nl));
+        for (int pass = 0; pass < n_pass; ++pass) {
+            ep.group = dual ? pass : -1;
+            ep.bias = stream_ptr(c->w.b_qkv, c->text_w.b_qkv, (size_t)blk * 3 * H, pass);
+            if (c->use_tc)
+                FD_TRY(FD_PROF_GEMM_QKV, tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl, pass == 1));
+            else
+                FD_TRY(FD_PROF_GEMM_QKV, launch_simt_gemm<T>(EPI_QKV, act, H, stream_ptr(c->w.w_qkv, c->text_w.w_qkv, (size_t)blk * 3 * H * H, pass),
+                                                             3 * H, H, rows_cap, ep, ctl, st, &nl));
+        }
         // block variants: QK-RMSNorm and rotary embedding on the fresh Q rows and the K rows just written
         if (c->var.q_norm_w || c->var.rope_cos) {
             const int q_stride = c->use_tc_attn ? tc_attention_head_pad(cf.head_dim) : cf.head_dim;
-            const T* qn = c->var.q_norm_w ? static_cast<const T*>(c->var.q_norm_w) + (size_t)blk * cf.head_dim : nullptr;
-            const T* kn = c->var.k_norm_w ? static_cast<const T*>(c->var.k_norm_w) + (size_t)blk * cf.head_dim : nullptr;
+            auto norm_w = [&](const void* base) -> const T* {
+                return base ? static_cast<const T*>(base) + (size_t)blk * cf.head_dim : nullptr;
+            };
+            const bool text_norm = dual && c->var.q_norm_w_text != nullptr;
             FD_TRY(FD_PROF_QK_VARIANTS, launch_qk_variants<T>(q, l.q_ld, q_stride, kv_b, active_idx, N, H, cf.n_heads, cf.head_dim,
-                                                               qn, kn, c->var.qk_norm_eps, c->var.rope_cos, c->var.rope_sin,
-                                                               rows_cap, ctl, st, &nl));
+                                                               norm_w(c->var.q_norm_w), norm_w(c->var.k_norm_w), c->var.qk_norm_eps,
+                                                               c->var.rope_cos, c->var.rope_sin, rows_cap, ctl, st, &nl,
+                                                               text_norm ? norm_w(c->var.q_norm_w_text) : nullptr,
+                                                               text_norm ? norm_w(c->var.k_norm_w_text) : nullptr,
+                                                               text_norm ? labels : nullptr, R));
         }
-        // active queries against all N keys of their request; the first block can also report, per region, the
-        // softmax mass its queries put on keys of their own region (paper Sec. 4.2)
+        // active queries against all N keys of their request (joint over both streams); the first block can also
+        // report, per region, the softmax mass its queries put on keys of their own region (paper Sec. 4.2)
         double* mass = blk == 0 ? region_mass : nullptr;
         if (mass) {
             e = cudaMemsetAsync(mass, 0, (size_t)B * R * sizeof(double), st);
@@ -224,32 +255,44 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             FD_TRY(FD_PROF_ATTENTION, launch_simt_attention<T>(q, l.q_ld, kv_b, o, H, tiles, max_tiles, N, H, cf.n_heads, cf.head_dim,
                                             ctl, st, &nl, 0, labels, active_idx, mass, R));
         }
-        // out-projection, gated residual
-        ep.bias = static_cast<const T*>(c->w.b_o) + (size_t)blk * H;
+        // out-projection, gated residual (a row's gate vector is its stream's: the epilogue adds the offset)
         ep.resid = resid;
         ep.gate = mod_b + 2 * H;
         ep.y = nullptr;
-        if (c->use_tc)
-            FD_TRY(FD_PROF_GEMM_OUT, tc_gemm(c->tc, TC_GEMM_OUT, blk, ep, ctl, st, &nl));
-        else
-            FD_TRY(FD_PROF_GEMM_OUT, launch_simt_gemm<T>(EPI_RESID, o, H, w_o, H, H, rows_cap, ep, ctl, st, &nl));
+        for (int pass = 0; pass < n_pass; ++pass) {
+            ep.group = dual ? pass : -1;
+            ep.bias = stream_ptr(c->w.b_o, c->text_w.b_o, (size_t)blk * H, pass);
+            if (c->use_tc)
+                FD_TRY(FD_PROF_GEMM_OUT, tc_gemm(c->tc, TC_GEMM_OUT, blk, ep, ctl, st, &nl, pass == 1));
+            else
+                FD_TRY(FD_PROF_GEMM_OUT, launch_simt_gemm<T>(EPI_RESID, o, H, stream_ptr(c->w.w_o, c->text_w.w_o, (size_t)blk * H * H, pass), H, H,
+                                                             rows_cap, ep, ctl, st, &nl));
+        }
         // MLP branch
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, mod_b + 3 * H, mod_b + 4 * H, 6 * H, N,
-                                     H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl));
-        ep.bias = static_cast<const T*>(c->w.b_fc1) + (size_t)blk * M;
+                                     H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts));
         ep.out = g;
         ep.out_ld = M;
-        if (c->use_tc)
-            FD_TRY(FD_PROF_GEMM_FC1, tc_gemm(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl));
-        else
-            FD_TRY(FD_PROF_GEMM_FC1, launch_simt_gemm<T>(EPI_GELU, act, H, w_fc1, M, H, rows_cap, ep, ctl, st, &nl));
-        ep.bias = static_cast<const T*>(c->w.b_fc2) + (size_t)blk * H;
+        for (int pass = 0; pass < n_pass; ++pass) {
+            ep.group = dual ? pass : -1;
+            ep.bias = stream_ptr(c->w.b_fc1, c->text_w.b_fc1, (size_t)blk * M, pass);
+            if (c->use_tc)
+                FD_TRY(FD_PROF_GEMM_FC1, tc_gemm(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl, pass == 1));
+            else
+                FD_TRY(FD_PROF_GEMM_FC1, launch_simt_gemm<T>(EPI_GELU, act, H, stream_ptr(c->w.w_fc1, c->text_w.w_fc1, (size_t)blk * M * H, pass), M,
+                                                             H, rows_cap, ep, ctl, st, &nl));
+        }
         ep.gate = mod_b + 5 * H;
         ep.y = (blk == L - 1) ? y_ : nullptr;       // the last block scatters the rows back
-        if (c->use_tc)
-            FD_TRY(FD_PROF_GEMM_FC2, tc_gemm(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl));
-        else
-            FD_TRY(FD_PROF_GEMM_FC2, launch_simt_gemm<T>(EPI_RESID, g, M, w_fc2, H, M, rows_cap, ep, ctl, st, &nl));
+        for (int pass = 0; pass < n_pass; ++pass) {
+            ep.group = dual ? pass : -1;
+            ep.bias = stream_ptr(c->w.b_fc2, c->text_w.b_fc2, (size_t)blk * H, pass);
+            if (c->use_tc)
+                FD_TRY(FD_PROF_GEMM_FC2, tc_gemm(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl, pass == 1));
+            else
+                FD_TRY(FD_PROF_GEMM_FC2, launch_simt_gemm<T>(EPI_RESID, g, M, stream_ptr(c->w.w_fc2, c->text_w.w_fc2, (size_t)blk * H * M, pass), H,
+                                                             M, rows_cap, ep, ctl, st, &nl));
+        }
     }
 #undef FD_TRY
     c->launches += nl;
@@ -551,11 +594,38 @@ fd_status fd_set_block_variants(fd_ctx* c, const fd_block_variants* v) {
     if (v->rope_cos && (c->cfg.head_dim & 1)) return c->fail(FD_ERR_SHAPE, "rotary embedding needs an even head_dim");
     if (v->q_norm_w && !(v->qk_norm_eps >= 0.f)) return c->fail(FD_ERR_INVALID_ARG, "qk_norm_eps must be non-negative");
     const uintptr_t wmask = c->cfg.dtype == FD_BF16 ? 3 : 7;
-    if ((reinterpret_cast<uintptr_t>(v->q_norm_w) | reinterpret_cast<uintptr_t>(v->k_norm_w)) & wmask)
+    if ((reinterpret_cast<uintptr_t>(v->q_norm_w) | reinterpret_cast<uintptr_t>(v->k_norm_w) |
+         reinterpret_cast<uintptr_t>(v->q_norm_w_text) | reinterpret_cast<uintptr_t>(v->k_norm_w_text)) & wmask)
         return c->fail(FD_ERR_INVALID_ARG, "QK-norm weights are misaligned");
+    if ((v->q_norm_w_text == nullptr) != (v->k_norm_w_text == nullptr) || (v->q_norm_w_text && !v->q_norm_w))
+        return c->fail(FD_ERR_INVALID_ARG, "the second stream's QK-norm weights come in pairs and need the first stream's");
     if ((reinterpret_cast<uintptr_t>(v->rope_cos) | reinterpret_cast<uintptr_t>(v->rope_sin)) & 3)
         return c->fail(FD_ERR_INVALID_ARG, "rotary tables are misaligned");
     c->var = *v;
+    return FD_OK;
+}
+
+fd_status fd_set_text_stream(fd_ctx* c, const fd_weights* text_weights) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    int32_t* text128 = c->at<int32_t>(c->lay.text_tiles);
+    int32_t* text256 = text128 + c->lay.Mcap / 128 + 1;
+    if (!text_weights) {
+        c->dual = false;
+        c->text_w = fd_weights{};
+        if (c->tc) tc_plan_set_text(c->tc, nullptr, text128, text256, nullptr);
+        return FD_OK;
+    }
+    const void* wp[10] = {text_weights->w_qkv, text_weights->b_qkv, text_weights->w_o, text_weights->b_o, text_weights->w_fc1,
+                          text_weights->b_fc1, text_weights->w_fc2, text_weights->b_fc2, text_weights->w_ada, text_weights->b_ada};
+    for (const void* p : wp)
+        if (!p || !aligned16(p)) return c->fail(FD_ERR_INVALID_ARG, "weight pointer null or not 16-byte aligned");
+    if (c->tc) {
+        std::string err;
+        if (!tc_plan_set_text(c->tc, text_weights, text128, text256, &err))
+            return c->fail(FD_ERR_CUDA, "tensor maps of the second stream's weights: %s", err.c_str());
+    }
+    c->text_w = *text_weights;
+    c->dual = true;
     return FD_OK;
 }
 

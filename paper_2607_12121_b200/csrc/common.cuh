@@ -19,7 +19,8 @@ struct Control {
     int32_t a_total;       // number of active rows of the current step
     int32_t n_qtiles;      // number of attention query tiles of the current step
     int32_t n_qtiles2;     // ... and of double-height tiles (the work list of the CTA-pair attention kernel)
-    int32_t pad[11];
+    int32_t n_text_tiles[2];   // dual stream: row tiles (128 rows / 256 rows) that hold rows of the second stream
+    int32_t pad[9];
 };
 
 __device__ __forceinline__ void report(Control* c, int code, int detail) {
@@ -80,6 +81,18 @@ struct EpiParams {
     // EPI_GELU
     void* out;                 // [Mcap,n_out] storage type
     int32_t out_ld;
+    // dual stream: a launch finishes only the rows of one stream (tokens with label R form the second one)
+    const int32_t* labels;     // [B*N] or nullptr
+    int32_t R;
+    int32_t group;             // -1: every row; 0: rows of the first stream only; 1: rows of the second stream only
+    int32_t text_mod_off;      // offset (floats) from a request's adaLN vectors to those of the second stream
+};
+
+// Per-row choice of the second stream's adaLN vectors in the row kernels (labels == nullptr: single stream).
+struct TextSel {
+    const int32_t* labels;     // [B*N]
+    int32_t R;
+    long long mod_off;         // offset (floats) from the first stream's vectors to the second stream's
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -108,6 +121,10 @@ cudaError_t noalloc_gate(const float* z_cur, const float* z_prev, const int32_t*
 cudaError_t launch_compact(const uint8_t* mask, const int32_t* labels, int B, int N, int R,
                            int32_t* active_idx, int32_t* cu_active, int32_t* block_counts, QTile* tiles,
                            int tile_rows, Control* ctl, cudaStream_t st, int* n_launch, QTile* tiles2 = nullptr);
+// dual stream: ascending lists of the 128-row and of the 256-row tiles of the compact rows that contain at least one
+// row of the second stream (label R); counts go to ctl->n_text_tiles.  lists: [cap128 + cap256] ints.
+cudaError_t launch_text_tiles(const int32_t* active_idx, const int32_t* labels, int R, int rows_cap, int32_t* list128,
+                              int32_t* list256, Control* ctl, cudaStream_t st, int* n_launch);
 
 // rowops.cu
 template <typename T>
@@ -117,13 +134,15 @@ template <typename T>
 cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
                                const int32_t* active_idx, const float* shift, const float* scale,
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
-                               cudaStream_t st, int* n_launch, bool pdl);
+                               cudaStream_t st, int* n_launch, bool pdl, TextSel ts = TextSel{nullptr, 0, 0});
 
 // qk_variants.cu: QK-RMSNorm and rotary embedding on the fresh Q rows and the K rows just written to the cache
 template <typename T>
 cudaError_t launch_qk_variants(T* q, int q_ld, int q_head_stride, T* kv_block, const int32_t* active_idx, int N, int H,
                                int heads, int dh, const T* qn_w, const T* kn_w, float eps, const float* rope_cos,
-                               const float* rope_sin, int rows_cap, const Control* ctl, cudaStream_t st, int* n_launch);
+                               const float* rope_sin, int rows_cap, const Control* ctl, cudaStream_t st, int* n_launch,
+                               const T* qn_w_text = nullptr, const T* kn_w_text = nullptr, const int32_t* labels = nullptr,
+                               int R = 0);
 
 // simt_block.cu
 template <typename T>

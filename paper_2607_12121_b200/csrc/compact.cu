@@ -138,7 +138,56 @@ compact_write_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict
     }
 }
 
+// Dual stream: which 128-row and which 256-row tiles of the compact rows hold at least one row of the second stream
+// (label R).  One CTA: a thread per 128-row tile flags it, a ballot-based prefix keeps the lists ascending.
+__global__ void __launch_bounds__(CP_THREADS)
+text_tiles_kernel(const int32_t* __restrict__ active_idx, const int32_t* __restrict__ labels, int R,
+                  int32_t* __restrict__ list128, int32_t* __restrict__ list256, Control* ctl) {
+    __shared__ int s_cnt[CP_WARPS];
+    __shared__ int s_base[2];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int a_total = ctl->a_total;
+    const int n128 = (a_total + 127) / 128;
+    if (threadIdx.x == 0) { s_base[0] = 0; s_base[1] = 0; }
+    __syncthreads();
+    for (int gran = 0; gran < 2; ++gran) {
+        const int rows = gran ? 256 : 128;
+        const int n_tiles = gran ? (a_total + 255) / 256 : n128;
+        int32_t* list = gran ? list256 : list128;
+        for (int t0 = 0; t0 < n_tiles; t0 += CP_THREADS) {
+            const int t = t0 + threadIdx.x;
+            bool has = false;
+            if (t < n_tiles) {
+                const int r1 = min(a_total, (t + 1) * rows);
+                for (int r = t * rows; r < r1 && !has; ++r) has = labels[active_idx[r]] == R;
+            }
+            const unsigned bal = __ballot_sync(0xffffffffu, has);
+            if (lane == 0) s_cnt[warp] = __popc(bal);
+            __syncthreads();
+            int pos = s_base[gran];
+            for (int w = 0; w < warp; ++w) pos += s_cnt[w];
+            if (has) list[pos + __popc(bal & ((1u << lane) - 1u))] = t;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                int tot = 0;
+                for (int w = 0; w < CP_WARPS; ++w) tot += s_cnt[w];
+                s_base[gran] += tot;
+            }
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) { ctl->n_text_tiles[0] = s_base[0]; ctl->n_text_tiles[1] = s_base[1]; }
+}
+
 }  // namespace
+
+cudaError_t launch_text_tiles(const int32_t* active_idx, const int32_t* labels, int R, int rows_cap, int32_t* list128,
+                              int32_t* list256, Control* ctl, cudaStream_t st, int* n_launch) {
+    (void)rows_cap;
+    text_tiles_kernel<<<1, CP_THREADS, 0, st>>>(active_idx, labels, R, list128, list256, ctl);
+    ++*n_launch;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_compact(const uint8_t* mask, const int32_t* labels, int B, int N, int R,
                            int32_t* active_idx, int32_t* cu_active, int32_t* block_counts, QTile* tiles,

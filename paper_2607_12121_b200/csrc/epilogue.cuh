@@ -100,14 +100,15 @@ __device__ __forceinline__ uint4* unit_ptr(uint8_t* stage, int row, int u) {
 // What lane t knows about "its" row (row_base + t) of the warp's 32 rows, computed once per tile so that the
 // chunk loops contain no divisions and no 64-bit multiplies; other lanes fetch it with shuffles.
 struct RowInfo {
-    int gate_off;      // b * 6H: offset of the request's adaLN vectors
+    uint32_t valid;    // bit t: row t of the warp's 32 exists and belongs to the stream this launch finishes (same in all lanes)
+    int gate_off;      // b * 6H: offset of the request's adaLN vectors (of the row's stream)
     uint32_t y_lo, y_hi;   // tok * H: element offset of the row in y (EPI_RESID) or of the token in the K plane (EPI_QKV)
 };
 
 // EPI_RESID: 32 fp32 accumulator columns per row; resid += gate * (acc + bias); the last block also
 // scatters the row into y.
 __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
-                                                     int n_rows, int col0, const uint32_t* acc, const RowInfo& ri) {
+                                                     int col0, const uint32_t* acc, const RowInfo& ri) {
     using T = __nv_bfloat16;
 #pragma unroll
     for (int u = 0; u < 8; ++u) *unit_ptr(stage, lane, u) = make_uint4(acc[4 * u], acc[4 * u + 1], acc[4 * u + 2], acc[4 * u + 3]);
@@ -129,12 +130,12 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int go = __shfl_sync(0xffffffffu, ri.gate_off, 4 * i + rsub);
-            if (4 * i + rsub < n_rows) gv[i] = __ldg(reinterpret_cast<const float4*>(gp + go));
+            if ((ri.valid >> (4 * i + rsub)) & 1u) gv[i] = __ldg(reinterpret_cast<const float4*>(gp + go));
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int r = 4 * i + rsub;
-            if (r < n_rows) {
+            if ((ri.valid >> r) & 1u) {
                 const uint4 a = *unit_ptr(stage, r, u);
                 const float x = gv[i].x * (__uint_as_float(a.x) + bias[0]), y = gv[i].y * (__uint_as_float(a.y) + bias[1]);
                 const float z = gv[i].z * (__uint_as_float(a.z) + bias[2]), w = gv[i].w * (__uint_as_float(a.w) + bias[3]);
@@ -151,7 +152,7 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
     for (int i = 0; i < 8; ++i) {
         const int r = 4 * i + rsub;
         const int go = __shfl_sync(0xffffffffu, ri.gate_off, r);
-        if (r < n_rows) {
+        if ((ri.valid >> r) & 1u) {
             rv[i] = *reinterpret_cast<const float4*>(rp + i * rstride);
             gv[i] = __ldg(reinterpret_cast<const float4*>(gp + go));
         }
@@ -160,7 +161,7 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
     for (int i = 0; i < 8; ++i) {
         const int r = 4 * i + rsub;
         const uint32_t ylo = __shfl_sync(0xffffffffu, ri.y_lo, r), yhi = __shfl_sync(0xffffffffu, ri.y_hi, r);
-        if (r < n_rows) {
+        if ((ri.valid >> r) & 1u) {
             const uint4 a = *unit_ptr(stage, r, u);
             float4 v = rv[i];
             v.x = fmaf(gv[i].x, __uint_as_float(a.x) + bias[0], v.x); v.y = fmaf(gv[i].y, __uint_as_float(a.y) + bias[1], v.y);
@@ -177,7 +178,7 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
 // issues per-thread reductions at about 9 bytes per clock, which made this epilogue as long as the main loop of a
 // K = 1536 tile; the bulk form hands whole 128-byte rows to the L2.
 __device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
-                                                         int n_rows, int col0, const uint32_t* acc, const RowInfo& ri,
+                                                         int col0, const uint32_t* acc, const RowInfo& ri,
                                                          const CUtensorMap* tm_r) {
     using T = __nv_bfloat16;
     if (lane == 0) ptx::bulk_wait_read_all();                      // the previous chunk's reduction has read the tile
@@ -194,10 +195,10 @@ __device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, ui
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int go = __shfl_sync(0xffffffffu, ri.gate_off, 4 * i + rsub);
-        gv[i] = 4 * i + rsub < n_rows ? __ldg(reinterpret_cast<const float4*>(gp + go)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        gv[i] = ((ri.valid >> (4 * i + rsub)) & 1u) ? __ldg(reinterpret_cast<const float4*>(gp + go)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     // The tile is rewritten in place, row by row: the eight lanes of a row read their (swizzled) units, then write the
-    // row's 128 bytes in plain order; rows past the last active row add zeros.
+    // row's 128 bytes in plain order; rows past the last active row (or of the other stream) add zeros.
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int r = 4 * i + rsub;
@@ -216,7 +217,7 @@ __device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, ui
 // EPI_QKV / EPI_GELU: 64 fp32 accumulator columns per row, bf16 outputs (8 columns per 16-byte unit).
 template <int KIND>
 __device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
-                                                    int n_rows, int col0, const uint32_t* acc, const RowInfo& ri) {
+                                                    int col0, const uint32_t* acc, const RowInfo& ri) {
     using T = __nv_bfloat16;
     const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ep.bias) + col0);
 #pragma unroll
@@ -245,7 +246,7 @@ __device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int r = 4 * i + rsub;
-            if (r < n_rows) *reinterpret_cast<uint4*>(ob + i * ostride) = *unit_ptr(stage, r, u);
+            if ((ri.valid >> r) & 1u) *reinterpret_cast<uint4*>(ob + i * ostride) = *unit_ptr(stage, r, u);
         }
     } else {
         const int sec = col0 / ep.H;                              // the 64 columns of a chunk share their section
@@ -258,7 +259,7 @@ __device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int r = 4 * i + rsub;
-                if (r < n_rows) *reinterpret_cast<uint4*>(qb + i * qstride) = *unit_ptr(stage, r, u);
+                if ((ri.valid >> r) & 1u) *reinterpret_cast<uint4*>(qb + i * qstride) = *unit_ptr(stage, r, u);
             }
         } else {
             T* kvb = reinterpret_cast<T*>(ep.kv) + (size_t)(sec - 1) * ep.N * ep.H + c;     // K plane, or V plane N*H further
@@ -266,7 +267,7 @@ __device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t
             for (int i = 0; i < 8; ++i) {
                 const int r = 4 * i + rsub;
                 const uint32_t lo = __shfl_sync(0xffffffffu, ri.y_lo, r), hi = __shfl_sync(0xffffffffu, ri.y_hi, r);
-                if (r < n_rows) *reinterpret_cast<uint4*>(kvb + (((size_t)hi << 32) | lo)) = *unit_ptr(stage, r, u);
+                if ((ri.valid >> r) & 1u) *reinterpret_cast<uint4*>(kvb + (((size_t)hi << 32) | lo)) = *unit_ptr(stage, r, u);
             }
         }
     }
@@ -290,15 +291,22 @@ __device__ __forceinline__ void epilogue_prefetch_resid(const EpiParams& ep, int
 // fetch it while the tile's products are still running.
 template <int KIND>
 __device__ __forceinline__ RowInfo epilogue_row_info(const EpiParams& ep, int lane, int row_base, int a_total) {
-    RowInfo ri{0, 0u, 0u};
-    if (KIND != EPI_GELU && row_base + lane < a_total) {
+    RowInfo ri{0u, 0, 0u, 0u};
+    bool ok = row_base + lane < a_total;
+    if ((KIND != EPI_GELU || ep.group >= 0) && ok) {
         const int tok = ep.active_idx[row_base + lane];
         const int b = tok / ep.N;
         ri.gate_off = b * 6 * ep.H;
+        if (ep.group >= 0) {                                     // dual stream: this launch owns one stream's rows
+            const int text = ep.labels[tok] == ep.R ? 1 : 0;
+            ok = text == ep.group;
+            if (text) ri.gate_off += ep.text_mod_off;
+        }
         const size_t off = KIND == EPI_RESID ? (size_t)tok * ep.H : ((size_t)b * 2 * ep.N + (tok - b * ep.N)) * ep.H;
         ri.y_lo = (uint32_t)off;
         ri.y_hi = (uint32_t)(off >> 32);
     }
+    ri.valid = __ballot_sync(0xffffffffu, ok);
     return ri;
 }
 
@@ -307,8 +315,8 @@ template <int KIND>
 __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stage, int lane, int row_base, int a_total,
                                               uint32_t t_row, int tile_col0, int c_begin, int c_end, const RowInfo& ri,
                                               const CUtensorMap* tm_r = nullptr) {
-    const bool live = row_base < a_total;                        // warp-uniform
-    const int n_rows = a_total - row_base;
+    const bool live = ri.valid != 0u;                            // warp-uniform
+    (void)a_total;
     if constexpr (KIND == EPI_RESID) {
 #pragma unroll 1
         for (int c0 = c_begin; c0 < c_end; c0 += 32) {
@@ -316,8 +324,8 @@ __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stag
             ptx::tmem_ld32(t_row + c0, r);
             ptx::tmem_wait_ld();
             if (live) {
-                if (tm_r && !ep.y) epilogue_resid_chunk_tma(ep, stage, lane, row_base, n_rows, tile_col0 + c0, r, ri, tm_r);
-                else epilogue_resid_chunk(ep, stage, lane, row_base, n_rows, tile_col0 + c0, r, ri);
+                if (tm_r && !ep.y) epilogue_resid_chunk_tma(ep, stage, lane, row_base, tile_col0 + c0, r, ri, tm_r);
+                else epilogue_resid_chunk(ep, stage, lane, row_base, tile_col0 + c0, r, ri);
             }
         }
     } else {
@@ -327,7 +335,7 @@ __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stag
             ptx::tmem_ld32(t_row + c0, r);
             ptx::tmem_ld32(t_row + c0 + 32, r + 32);
             ptx::tmem_wait_ld();
-            if (live) epilogue_bf16_chunk<KIND>(ep, stage, lane, row_base, n_rows, tile_col0 + c0, r, ri);
+            if (live) epilogue_bf16_chunk<KIND>(ep, stage, lane, row_base, tile_col0 + c0, r, ri);
         }
     }
 }

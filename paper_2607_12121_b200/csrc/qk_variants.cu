@@ -72,7 +72,8 @@ template <typename T, int MAXP>
 __global__ void __launch_bounds__(QKV_THREADS)
 qk_variants_kernel(T* __restrict__ q, int q_ld, int q_head_stride, T* __restrict__ kv, const int32_t* __restrict__ active_idx,
                    int N, int H, int heads, int dh, const T* __restrict__ qn_w, const T* __restrict__ kn_w, float eps,
-                   const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, const Control* __restrict__ ctl) {
+                   const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, const Control* __restrict__ ctl,
+                   const T* __restrict__ qn_w_text, const T* __restrict__ kn_w_text, const int32_t* __restrict__ labels, int R) {
     const int lane = threadIdx.x & 31;
     const int warps = gridDim.x * (QKV_THREADS / 32);
     const long long units = (long long)ctl->a_total * heads;
@@ -82,8 +83,9 @@ qk_variants_kernel(T* __restrict__ q, int q_ld, int q_head_stride, T* __restrict
         const int b = tok / N, j = tok - b * N;
         const float* cs = rope_cos ? rope_cos + (size_t)j * (dh >> 1) : nullptr;
         const float* sn = rope_cos ? rope_sin + (size_t)j * (dh >> 1) : nullptr;
-        head_slice<T, MAXP>(q + (size_t)row * q_ld + (size_t)h * q_head_stride, dh, qn_w, eps, cs, sn, lane);
-        head_slice<T, MAXP>(kv + (((size_t)b * 2 + 0) * N + j) * H + (size_t)h * dh, dh, kn_w, eps, cs, sn, lane);
+        const bool text = labels && qn_w_text && labels[tok] == R;        // dual stream: the second stream's norm weights
+        head_slice<T, MAXP>(q + (size_t)row * q_ld + (size_t)h * q_head_stride, dh, text ? qn_w_text : qn_w, eps, cs, sn, lane);
+        head_slice<T, MAXP>(kv + (((size_t)b * 2 + 0) * N + j) * H + (size_t)h * dh, dh, text ? kn_w_text : kn_w, eps, cs, sn, lane);
     }
 }
 
@@ -92,24 +94,26 @@ qk_variants_kernel(T* __restrict__ q, int q_ld, int q_head_stride, T* __restrict
 template <typename T>
 cudaError_t launch_qk_variants(T* q, int q_ld, int q_head_stride, T* kv_block, const int32_t* active_idx, int N, int H,
                                int heads, int dh, const T* qn_w, const T* kn_w, float eps, const float* rope_cos,
-                               const float* rope_sin, int rows_cap, const Control* ctl, cudaStream_t st, int* n_launch) {
+                               const float* rope_sin, int rows_cap, const Control* ctl, cudaStream_t st, int* n_launch,
+                               const T* qn_w_text, const T* kn_w_text, const int32_t* labels, int R) {
     const long long max_units = (long long)rows_cap * heads;
     const int grid = (int)max(1LL, min((max_units + QKV_THREADS / 32 - 1) / (QKV_THREADS / 32), 148LL * 16));
     if (dh <= 64)
         qk_variants_kernel<T, 1><<<grid, QKV_THREADS, 0, st>>>(q, q_ld, q_head_stride, kv_block, active_idx, N, H, heads, dh, qn_w,
-                                                               kn_w, eps, rope_cos, rope_sin, ctl);
+                                                               kn_w, eps, rope_cos, rope_sin, ctl, qn_w_text, kn_w_text, labels, R);
     else
         qk_variants_kernel<T, 2><<<grid, QKV_THREADS, 0, st>>>(q, q_ld, q_head_stride, kv_block, active_idx, N, H, heads, dh, qn_w,
-                                                               kn_w, eps, rope_cos, rope_sin, ctl);
+                                                               kn_w, eps, rope_cos, rope_sin, ctl, qn_w_text, kn_w_text, labels, R);
     ++*n_launch;
     return cudaGetLastError();
 }
 
 template cudaError_t launch_qk_variants<float>(float*, int, int, float*, const int32_t*, int, int, int, int, const float*,
                                                const float*, float, const float*, const float*, int, const Control*,
-                                               cudaStream_t, int*);
+                                               cudaStream_t, int*, const float*, const float*, const int32_t*, int);
 template cudaError_t launch_qk_variants<__nv_bfloat16>(__nv_bfloat16*, int, int, __nv_bfloat16*, const int32_t*, int, int, int,
                                                        int, const __nv_bfloat16*, const __nv_bfloat16*, float, const float*,
-                                                       const float*, int, const Control*, cudaStream_t, int*);
+                                                       const float*, int, const Control*, cudaStream_t, int*,
+                                                       const __nv_bfloat16*, const __nv_bfloat16*, const int32_t*, int);
 
 }  // namespace fd

@@ -224,7 +224,7 @@ __global__ void __launch_bounds__(LN_THREADS, 8)
 ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
                    float* __restrict__ resid_out, T* __restrict__ out, const int32_t* __restrict__ active_idx,
                    const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
-                   int H, float ln_eps, const Control* __restrict__ ctl) {
+                   int H, float ln_eps, const Control* __restrict__ ctl, TextSel ts) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     ptx::pdl_wait();                              // the rows come from the kernel launched just before
     const int a_total = ctl->a_total;
@@ -251,8 +251,10 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
         const float var = fmaxf(sq / (float)H - dm * dm, 0.f);
         const float rstd = rsqrtf(var + ln_eps);
         const float mean = x0 + dm;
-        const float* sh = shift + (size_t)b * mod_stride;
-        const float* sc = scale + (size_t)b * mod_stride;
+        // dual stream: a token with label R takes the second stream's vectors
+        const long long soff = (ts.labels && ts.labels[tok] == ts.R) ? ts.mod_off : 0;
+        const float* sh = shift + (size_t)b * mod_stride + soff;
+        const float* sc = scale + (size_t)b * mod_stride + soff;
 #pragma unroll 4
         for (int i = 0; i < nv; ++i) {
             const int c = (i * 32 + lane) * 4;
@@ -288,7 +290,7 @@ __global__ void __launch_bounds__(LN_THREADS, 6)
 ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
                        float* __restrict__ resid_out, T* __restrict__ out, const int32_t* __restrict__ active_idx,
                        const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
-                       float ln_eps, const Control* __restrict__ ctl) {
+                       float ln_eps, const Control* __restrict__ ctl, TextSel ts) {
     constexpr int H = NV * 128;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     ptx::pdl_wait();                              // the rows come from the kernel launched just before
@@ -337,8 +339,9 @@ ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__
         const float rstd = rsqrtf(fmaxf(sq / (float)H - dm * dm, 0.f) + ln_eps);
         const float mean = x0 + dm;
         const int b = tok / N;
-        const float4* sc4 = reinterpret_cast<const float4*>(scale + (size_t)b * mod_stride) + lane;
-        const float4* sh4 = reinterpret_cast<const float4*>(shift + (size_t)b * mod_stride) + lane;
+        const long long soff = (ts.labels && ts.labels[tok] == ts.R) ? ts.mod_off : 0;      // dual stream
+        const float4* sc4 = reinterpret_cast<const float4*>(scale + (size_t)b * mod_stride + soff) + lane;
+        const float4* sh4 = reinterpret_cast<const float4*>(shift + (size_t)b * mod_stride + soff) + lane;
         T* dst = out + (size_t)row * H + lane * 4;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
@@ -369,7 +372,7 @@ ln_modulate_generic_kernel(const T* __restrict__ x_gather, const float* __restri
                            float* __restrict__ resid_out, T* __restrict__ out,
                            const int32_t* __restrict__ active_idx, const float* __restrict__ shift,
                            const float* __restrict__ scale, int mod_stride, int N, int H, float ln_eps,
-                           const Control* __restrict__ ctl) {
+                           const Control* __restrict__ ctl, TextSel ts) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int a_total = ctl->a_total;
     for (int row = blockIdx.x * (LN_THREADS / 32) + warp; row < a_total; row += gridDim.x * (LN_THREADS / 32)) {
@@ -384,8 +387,9 @@ ln_modulate_generic_kernel(const T* __restrict__ x_gather, const float* __restri
         float sq = 0.f;
         for (int c = lane; c < H; c += 32) { const float d = at(c) - mean; sq = fmaf(d, d, sq); }
         const float rstd = rsqrtf(warp_sum(sq) / (float)H + ln_eps);
-        const float* sh = shift + (size_t)b * mod_stride;
-        const float* sc = scale + (size_t)b * mod_stride;
+        const long long soff = (ts.labels && ts.labels[tok] == ts.R) ? ts.mod_off : 0;      // dual stream
+        const float* sh = shift + (size_t)b * mod_stride + soff;
+        const float* sc = scale + (size_t)b * mod_stride + soff;
         for (int c = lane; c < H; c += 32) {
             const float u = at(c);
             if (x_gather && resid_out) resid_out[(size_t)row * H + c] = u;
@@ -428,16 +432,16 @@ template <typename T>
 cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
                                const int32_t* active_idx, const float* shift, const float* scale,
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
-                               cudaStream_t st, int* n_launch, bool pdl) {
+                               cudaStream_t st, int* n_launch, bool pdl, TextSel ts) {
     const int rows_per_cta = LN_THREADS / 32;
     const int grid = max(1, min((rows_cap + rows_per_cta - 1) / rows_per_cta, 148 * 16));
 #define FD_LN_REG(NV)                                                                                              \
     if (H == NV * 128) {                                                                                           \
         cudaError_t e = x_gather                                                                                    \
             ? ptx::launch_kernel(ln_modulate_reg_kernel<T, NV, true>, grid, LN_THREADS, 0, st, pdl, x_gather,      \
-                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl)   \
+                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl, ts) \
             : ptx::launch_kernel(ln_modulate_reg_kernel<T, NV, false>, grid, LN_THREADS, 0, st, pdl, x_gather,     \
-                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl);  \
+                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl, ts); \
         ++*n_launch;                                                                                               \
         return e;                                                                                                  \
     }
@@ -447,12 +451,12 @@ cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* 
 #undef FD_LN_REG
     if (H % 128 == 0) {
         cudaError_t e = ptx::launch_kernel(ln_modulate_kernel<T>, grid, LN_THREADS, 0, st, pdl, x_gather, resid_in, resid_out,
-                                           out, active_idx, shift, scale, mod_stride, N, H, ln_eps, ctl);
+                                           out, active_idx, shift, scale, mod_stride, N, H, ln_eps, ctl, ts);
         ++*n_launch;
         return e;
     } else
         ln_modulate_generic_kernel<T><<<grid, LN_THREADS, 0, st>>>(x_gather, resid_in, resid_out, out, active_idx,
-                                                                  shift, scale, mod_stride, N, H, ln_eps, ctl);
+                                                                  shift, scale, mod_stride, N, H, ln_eps, ctl, ts);
     ++*n_launch;
     return cudaGetLastError();
 }
@@ -463,9 +467,9 @@ template cudaError_t launch_adaln<__nv_bfloat16>(const __nv_bfloat16*, const __n
                                                  float*, int, int, int, int, void*, cudaStream_t, int*);
 template cudaError_t launch_ln_modulate<float>(const float*, const float*, float*, float*, const int32_t*,
                                                const float*, const float*, int, int, int, int, float, const Control*,
-                                               cudaStream_t, int*, bool);
+                                               cudaStream_t, int*, bool, TextSel);
 template cudaError_t launch_ln_modulate<__nv_bfloat16>(const __nv_bfloat16*, const float*, float*, __nv_bfloat16*,
                                                        const int32_t*, const float*, const float*, int, int, int, int,
-                                                       float, const Control*, cudaStream_t, int*, bool);
+                                                       float, const Control*, cudaStream_t, int*, bool, TextSel);
 
 }  // namespace fd

@@ -58,7 +58,16 @@ simt_gemm_kernel(const T* __restrict__ a, int lda, const T* __restrict__ w, int 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int row = row0 + ty * 4 + i;
-        if (row < a_total) epilogue4<T, KIND>(ep, row, col, ep.active_idx[row], acc[i]);
+        if (row < a_total) {
+            const int tok = ep.active_idx[row];
+            // dual stream: a launch finishes only the rows of its stream, with that stream's adaLN vectors
+            const int text = ep.group >= 0 && ep.labels[tok] == ep.R ? 1 : 0;
+            if (ep.group < 0 || text == ep.group) {
+                EpiParams e2 = ep;
+                if (text && e2.gate) e2.gate += ep.text_mod_off;
+                epilogue4<T, KIND>(e2, row, col, tok, acc[i]);
+            }
+        }
     }
 }
 

@@ -29,8 +29,10 @@ constexpr int TC_ATTENTION_SLOTS = 256;    // CTAs the attention scratch has roo
 size_t tc_attention_scratch_bytes(int head_dim);
 TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffers& buf, std::string* err);
 void tc_plan_destroy(TcPlan* p);
+// text_pass: the second stream's weights, over the row tiles that hold rows of that stream (dual stream)
 cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
-                    int* n_launch);
+                    int* n_launch, bool text_pass = false);
+bool tc_plan_set_text(TcPlan* p, const fd_weights* w, const int32_t* list128, const int32_t* list256, std::string* err);
 // region_mass (optional): [B, R] f64, receives the own-region softmax mass
 cudaError_t tc_attention(TcPlan* p, int blk, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch, const int32_t* labels = nullptr,

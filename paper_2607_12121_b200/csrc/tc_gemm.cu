@@ -37,7 +37,7 @@ template <int BN> struct GemmCfg {
 template <int KIND, int BN>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int n_out,
-               int k_dim, EpiParams ep, Control* ctl) {
+               int k_dim, EpiParams ep, Control* ctl, const int32_t* __restrict__ m_list) {
     using Cfg = GemmCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int B_TILE_BYTES = Cfg::B_TILE_BYTES;
@@ -75,7 +75,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     pdl_trigger();
     pdl_wait();
     const int a_total = ctl->a_total;
-    const int m_tiles = (a_total + BM - 1) / BM;
+    // row tiles: all of them, or (dual stream, second pass) the listed ones that hold rows of the second stream
+    const int m_tiles = m_list ? ctl->n_text_tiles[0] : (a_total + BM - 1) / BM;
     const int n_tiles = n_out / BN;
     const int total_tiles = m_tiles * n_tiles;
     const int k_tiles = k_dim / BK;
@@ -85,7 +86,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m = tile / n_tiles, n = tile % n_tiles;
+                const int m = m_list ? m_list[tile / n_tiles] : tile / n_tiles, n = tile % n_tiles;
                 for (int kt = 0; kt < k_tiles; ++kt, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
@@ -129,7 +130,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         uint32_t t_it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t_it) {
-            const int m = tile / n_tiles, n = tile % n_tiles;
+            const int m = m_list ? m_list[tile / n_tiles] : tile / n_tiles, n = tile % n_tiles;
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
             if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * BM + quad * 32, a_total, n * BN + chalf * (BN / 2), BN / 2);
@@ -177,7 +178,7 @@ template <int KIND, int PAIR_BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                     const __grid_constant__ CUtensorMap tm_r, int n_out, int k_dim, int stream_a, int tma_resid, EpiParams ep,
-                    Control* ctl) {
+                    Control* ctl, const int32_t* __restrict__ m_list) {
     constexpr int PAIR_B_BYTES = PairCfg<PAIR_BN>::B_BYTES, PAIR_STAGE_BYTES = PairCfg<PAIR_BN>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -216,7 +217,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     pdl_trigger();
     pdl_wait();
     const int a_total = ctl->a_total;
-    const int m_pairs = (a_total + 2 * BM - 1) / (2 * BM);
+    // 256-row tiles: all of them, or (dual stream, second pass) the listed ones that hold rows of the second stream
+    const int m_pairs = m_list ? ctl->n_text_tiles[1] : (a_total + 2 * BM - 1) / (2 * BM);
     const int n_tiles = n_out / PAIR_BN;
     const int total_tiles = m_pairs * n_tiles;
     const int k_tiles = k_dim / BK;
@@ -227,7 +229,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             bool ok = true;
             const uint64_t evict_first = l2_evict_first();
             for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
-                const int m = tile / n_tiles, n = tile % n_tiles;
+                const int m = m_list ? m_list[tile / n_tiles] : tile / n_tiles, n = tile % n_tiles;
                 for (int kt = 0; kt < k_tiles; ++kt, ++it) {
                     const int s = it % PAIR_STAGES;
                     const uint32_t ph = (it / PAIR_STAGES) & 1;
@@ -280,7 +282,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         uint32_t t_it = 0;
         bool ok = true;
         for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
-            const int m = tile / n_tiles, n = tile % n_tiles;
+            const int m = m_list ? m_list[tile / n_tiles] : tile / n_tiles, n = tile % n_tiles;
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
             if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * 2 * BM + (int)rank * BM + quad * 32, a_total,
@@ -390,6 +392,9 @@ struct TcPlan {
     CUtensorMap resid_map;      // fp32 residual stream [Mcap, H], 32 x 32 boxes for the bulk reductions of EPI_RESID
     bool tma_resid;
     CUtensorMap* w_maps;        // [L][4]
+    CUtensorMap* w_maps_text;   // [L][4] second stream's weights (dual stream), or nullptr
+    const int32_t* text_list128;    // device lists of the row tiles that hold rows of the second stream
+    const int32_t* text_list256;
     // attention (filled by the attention part)
     void* attn;
 };
@@ -410,6 +415,8 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
     p->cfg = cfg;
     p->buf = buf;
     p->w_maps = new CUtensorMap[(size_t)cfg.n_blocks * 4];
+    p->w_maps_text = nullptr;
+    p->text_list128 = p->text_list256 = nullptr;
     p->attn = nullptr;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -508,6 +515,7 @@ void tc_plan_destroy(TcPlan* p) {
     if (!p) return;
     tc_attention_plan_destroy(p->attn);
     delete[] p->w_maps;
+    delete[] p->w_maps_text;
     delete p;
 }
 
@@ -521,10 +529,44 @@ void* tc_plan_attn(TcPlan* p) { return p->attn; }
 bool tc_plan_pdl(TcPlan* p) { return p->pdl; }
 int tc_plan_sm_count(TcPlan* p) { return p->sm_count; }
 
+// Dual stream: tensor maps of the second stream's weights (w == nullptr: back to a single stream) and the device lists
+// of row tiles its launches walk.
+bool tc_plan_set_text(TcPlan* p, const fd_weights* w, const int32_t* list128, const int32_t* list256, std::string* err) {
+    delete[] p->w_maps_text;
+    p->w_maps_text = nullptr;
+    p->text_list128 = list128;
+    p->text_list256 = list256;
+    if (!w) return true;
+    const fd_config& cfg = p->cfg;
+    const int H = cfg.hidden, M = cfg.mlp_dim;
+    const int n_out[4] = {3 * H, H, M, H};
+    const int kdim[4] = {H, H, H, M};
+    const char* w_base[4] = {static_cast<const char*>(w->w_qkv), static_cast<const char*>(w->w_o),
+                             static_cast<const char*>(w->w_fc1), static_cast<const char*>(w->w_fc2)};
+    p->w_maps_text = new CUtensorMap[(size_t)cfg.n_blocks * 4];
+    for (int g = 0; g < 4; ++g) {
+        const GemmSpec& s = p->spec[g];
+        for (int l = 0; l < cfg.n_blocks; ++l) {
+            const uint64_t wd[2] = {(uint64_t)kdim[g], (uint64_t)n_out[g]};
+            const uint64_t strides[1] = {(uint64_t)kdim[g] * 2};
+            const uint32_t wb[2] = {BK, s.pair_bn ? (uint32_t)s.pair_bn / 2 : (uint32_t)s.bn};
+            void* base = const_cast<char*>(w_base[g]) + (size_t)l * n_out[g] * kdim[g] * 2;
+            if (!encode_tmap_bf16(&p->w_maps_text[(size_t)l * 4 + g], base, 2, wd, strides, wb, 128, err)) {
+                delete[] p->w_maps_text;
+                p->w_maps_text = nullptr;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
 cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
-                    int* n_launch) {
+                    int* n_launch, bool text_pass) {
     const GemmSpec& s = p->spec[kind];
-    const CUtensorMap& wm = p->w_maps[(size_t)blk * 4 + kind];
+    if (text_pass && !p->w_maps_text) return cudaErrorInvalidValue;
+    const CUtensorMap& wm = text_pass ? p->w_maps_text[(size_t)blk * 4 + kind] : p->w_maps[(size_t)blk * 4 + kind];
+    const int32_t* m_list = text_pass ? (s.pair_bn ? p->text_list256 : p->text_list128) : nullptr;
     Control* c = const_cast<Control*>(ctl);
     const int grid = p->sm_count;
     if (s.pair_bn) {
@@ -535,7 +577,7 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
         cudaError_t e = cudaSuccess;
 #define FD_LAUNCH_PAIR(K, N) \
     e = launch_kernel(tc_gemm_pair_kernel<K, N>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, s.a, wm, p->resid_map, s.n_out, s.k, \
-                      stream_a, p->tma_resid ? 1 : 0, ep, c)
+                      stream_a, p->tma_resid ? 1 : 0, ep, c, m_list)
         if (kind == TC_GEMM_QKV) {
             if (s.pair_bn == 256) FD_LAUNCH_PAIR(EPI_QKV, 256); else FD_LAUNCH_PAIR(EPI_QKV, 192);
         } else if (kind == TC_GEMM_FC1) {
@@ -549,7 +591,7 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
     }
     cudaError_t e = cudaSuccess;
 #define FD_LAUNCH(K, N) \
-    e = launch_kernel(tc_gemm_kernel<K, N>, grid, GEMM_THREADS, GemmCfg<N>::SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c)
+    e = launch_kernel(tc_gemm_kernel<K, N>, grid, GEMM_THREADS, GemmCfg<N>::SMEM, st, p->pdl, s.a, wm, s.n_out, s.k, ep, c, m_list)
     if (kind == TC_GEMM_QKV) {
         if (s.bn == 256) FD_LAUNCH(EPI_QKV, 256); else FD_LAUNCH(EPI_QKV, 128);
     } else if (kind == TC_GEMM_FC1) {

@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 MAX_ABS, REL_L2 = 3e-2, 1e-2
 
 
-def _full_shape_block(name, seed, fractions, n_sample=160, with_mass=False, qk_gain=1.0):
+def _full_shape_block(name, seed, fractions, n_sample=160, with_mass=False, qk_gain=1.0, text_seed=None):
     wl = gen.workload(name).replace(L=1)
     B, N, H = wl.B, wl.N, wl.H
     labels = labels_for(wl, seed)
@@ -32,6 +32,13 @@ def _full_shape_block(name, seed, fractions, n_sample=160, with_mass=False, qk_g
     ctx = make_ctx(wl, w, n_blocks=1)
     buf = StepBuffers(wl, 1)
     dt = tdtype(wl)
+    variants, mod_t, tok_text = None, None, None
+    if text_seed is not None:       # dual stream: the text tokens (label R) run through a second weight set
+        wt = gen.block_weights(wl, text_seed, n_blocks=1)
+        fd.fd_set_text_stream(ctx, {k: dev(v, dt) for k, v in wt.items()})
+        variants = {"text": {"weights": wt, "n_text": wl.n_text}}
+        mod_t = oracle.adaln(inp["cond"], wt["w_ada"][0], wt["b_ada"][0])
+        tok_text = (labels == wl.R).reshape(-1).astype(np.uint8)
     buf.kv.copy_(dev(kv0, dt))
     buf.y.copy_(dev(y0, dt))
     if with_mass:       # the step that also collects the first block's own-region attention mass (Sec. 4.2)
@@ -51,7 +58,11 @@ def _full_shape_block(name, seed, fractions, n_sample=160, with_mass=False, qk_g
     kv_ref = kv0[0].copy()
     pick = np.unique(np.concatenate([np.linspace(0, o_idx.size - 1, n_sample).astype(np.int32),
                                      o_cu[1:] - 1, o_cu[:-1]]).clip(0, o_idx.size - 1)).astype(np.int32)
-    out = oracle.regional_block(u, o_idx, mod, w, 0, kv_ref, wl.heads, finish=pick)
+    if text_seed is not None:       # make sure text rows are among the finished sample
+        text_rows = np.nonzero(tok_text[o_idx])[0]
+        pick = np.unique(np.concatenate([pick, text_rows[:: max(1, text_rows.size // 24)]])).astype(np.int32)
+    out = oracle.regional_block(u, o_idx, mod, w, 0, kv_ref, wl.heads, finish=pick, variants=variants, mod_text=mod_t,
+                                tok_text=tok_text)
 
     act = np.zeros(B * N, bool)
     act[o_idx] = True
@@ -89,6 +100,11 @@ def test_image_full_shape():
 
 def test_mmdit_full_shape_with_text_tokens():
     _full_shape_block("mmdit", 23, [0.34, 0.76])
+
+
+def test_mmdit_full_shape_dual_stream():
+    """The joint text-image configuration with its real structure: 154 text tokens per request on weights of their own."""
+    _full_shape_block("mmdit", 28, [0.34, 0.76], text_seed=128)
 
 
 def test_audio_full_shape_attention_mass():

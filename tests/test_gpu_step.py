@@ -38,10 +38,11 @@ def _check_step(wl, y, kv, y_ref, kv_ref, y_before, kv_before, idx):
             assert np.array_equal(got[~a2], old[~a2])
 
 
-def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=None):
+def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=None, text_seed=None):
     """Warm-up (all active) on the previous step's tokens, then gated steps; both sides start
     from the same zero caches and carry their own state forward.  `variants`: inputs of the block variants
-    (QK-RMSNorm weights, rotary tables) handed to both sides."""
+    (QK-RMSNorm weights, rotary tables) handed to both sides.  `text_seed`: dual stream, the always-active tokens
+    (label R) get a second weight set drawn from this seed."""
     L = wl.L if n_blocks is None else n_blocks
     labels = labels_for(wl, seed)
     w = gen.block_weights(wl, seed, n_blocks=L)
@@ -52,9 +53,24 @@ def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=
     ctx = make_ctx(wl, w, engine=engine, n_blocks=L)
     buf = StepBuffers(wl, L)
     dt = tdtype(wl)
+    variants = dict(variants) if variants is not None else None
+    if text_seed is not None:
+        wt = gen.block_weights(wl, text_seed, n_blocks=L)
+        if qk_gain != 1.0:
+            wt["w_qkv"][:, :wl.H] *= np.float32(qk_gain)
+            wt["b_qkv"][:, :wl.H] *= np.float32(qk_gain)
+        fd.fd_set_text_stream(ctx, {k: dev(v[:L], dt) for k, v in wt.items()})
+        text = {"weights": wt, "n_text": wl.n_text}
+        if variants is not None and "q_norm_w" in variants:     # the second stream normalises with weights of its own
+            tv = gen.block_variants(wl, text_seed, n_blocks=L, rope=False)
+            text.update(q_norm_w=tv["q_norm_w"], k_norm_w=tv["k_norm_w"])
     if variants is not None:
-        fd.fd_set_block_variants(ctx, **{k: (dev(v, dt if k.endswith("_w") else None) if isinstance(v, np.ndarray) else v)
-                                         for k, v in variants.items()})
+        kw = {k: (dev(v, dt if k.endswith("_w") else None) if isinstance(v, np.ndarray) else v) for k, v in variants.items()}
+        if text_seed is not None and "q_norm_w" in variants:
+            kw.update(q_norm_w_text=dev(text["q_norm_w"], dt), k_norm_w_text=dev(text["k_norm_w"], dt))
+        fd.fd_set_block_variants(ctx, **kw)
+    if text_seed is not None:
+        variants = dict(variants or {}, text=text)
     B, N, H = wl.B, wl.N, wl.H
     kv_ref = np.zeros((L, B, 2, N, H), np.float32)
     y_ref = np.zeros((B, N, H), np.float32)
