@@ -190,6 +190,34 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             bool ok = true;
             int item_i = 0;
             Task tk;
+            // The V tile of a key tile is requested one tile behind its K tile: K(g+1), then V(g).  A V stage is released
+            // by the product P V two tiles back, long after the K stage of the same tile (released by S = Q K^T); issuing
+            // K(g), V(g), K(g+1) in turn held every K load back behind that wait (timestamps at head dim 128, where the
+            // rings are two stages deep: the S = Q K^T issuer waited 0.5 us of every 1.2 us tile for its K tile; -12 % on
+            // the 480p video shape, -3 % at head dim 72).  With the five stages of head dim 64 nothing is held back and the
+            // lag only costs a tile of V prefetch (+3 to +5 % there), so it is off.
+            constexpr bool V_LAG = D != 64;
+            int pv_head = 0, pv_j = 0, pv_b = -1;        // the V tile still to be requested (pv_b < 0: none)
+            uint32_t pv_g = 0;
+            auto load_v = [&](int head, int j, int b, uint32_t g) -> bool {
+                const int s = g % STAGES;
+                if (!mbar_wait(&v_empty[s], ((g / STAGES) & 1) ^ 1, abort_flag)) return false;
+                mbar_expect_tx(&v_full[s], TILE_BYTES);
+                if constexpr (D == 72) {
+                    // V of a 72-wide head as five 16-column blocks (32-byte swizzle): one product of width 80 then
+                    // reads all of them, where a 64-wide plus a 16-wide block would need two products per 16 keys
+#pragma unroll
+                    for (int a = 0; a < 5; ++a)
+                        tma_load_3d(sV + s * TILE_BYTES + a * TAIL_BYTES, &tm_kv_tail, head * D + a * 16, j * KEYS, b * 2 + 1,
+                                    &v_full[s]);
+                } else {
+#pragma unroll
+                    for (int sb = 0; sb < Cfg::SUBS; ++sb)
+                        tma_load_3d(sV + s * TILE_BYTES + sb * SUB_BYTES, &tm_kv, head * D + sb * 64, j * KEYS, b * 2 + 1,
+                                    &v_full[s]);
+                }
+                return true;
+            };
             for (int k = 0; ok && next_task<CUT>(cut, n_items, n_kv, k, tk); ++k, ++item_i) {
                 const int w = tk.w;
                 const QTile t = tiles[w % n_tiles];
@@ -214,23 +242,15 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if constexpr (D == 72)
                         tma_load_3d(sK + s * TILE_BYTES + SUB_BYTES, &tm_kv_tail, head * D + 64, j * KEYS, t.b * 2 + 0,
                                     &k_full[s]);
-                    if (!mbar_wait(&v_empty[s], ph, abort_flag)) { ok = false; break; }
-                    mbar_expect_tx(&v_full[s], TILE_BYTES);
-                    if constexpr (D == 72) {
-                        // V of a 72-wide head as five 16-column blocks (32-byte swizzle): one product of width 80 then
-                        // reads all of them, where a 64-wide plus a 16-wide block would need two products per 16 keys
-#pragma unroll
-                        for (int a = 0; a < 5; ++a)
-                            tma_load_3d(sV + s * TILE_BYTES + a * TAIL_BYTES, &tm_kv_tail, head * D + a * 16, j * KEYS,
-                                        t.b * 2 + 1, &v_full[s]);
+                    if constexpr (V_LAG) {
+                        if (pv_b >= 0 && !load_v(pv_head, pv_j, pv_b, pv_g)) { ok = false; break; }
+                        pv_head = head; pv_j = j; pv_b = t.b; pv_g = gk;
                     } else {
-#pragma unroll
-                        for (int sb = 0; sb < Cfg::SUBS; ++sb)
-                            tma_load_3d(sV + s * TILE_BYTES + sb * SUB_BYTES, &tm_kv, head * D + sb * 64, j * KEYS,
-                                        t.b * 2 + 1, &v_full[s]);
+                        if (!load_v(head, j, t.b, gk)) { ok = false; break; }
                     }
                 }
             }
+            if (ok && pv_b >= 0 && !load_v(pv_head, pv_j, pv_b, pv_g)) ok = false;
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 400 + (int)blockIdx.x);
         }
     } else if (warp == 1) {
