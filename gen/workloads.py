@@ -372,3 +372,16 @@ def block_variants(wl: Workload, seed: int, n_blocks: Optional[int] = None, qk_n
         out["rope_cos"] = np.cos(ang).astype(np.float32)
         out["rope_sin"] = np.sin(ang).astype(np.float32)
     return out
+
+
+def cross_attention(wl: Workload, seed: int, n_ctx: int, n_blocks: Optional[int] = None, std: float = 0.02) -> Dict[str, np.ndarray]:
+    """Inputs of the cross-attention variant: query / out projections ~N(0, std) per block (w_q, w_o [L,H,H]; b_q, b_o
+    [L,H]) and the context's keys and values ~N(0, 0.5) (ctx_kv [L,B,2,n_ctx,H]; they stand for a text encoder's states
+    already projected by the caller), rounded to the storage type."""
+    L = wl.L if n_blocks is None else n_blocks
+    H = wl.H
+    g = _rng(seed, 1414)
+    out = {k: _store(wl, g.standard_normal(s, dtype=np.float32) * np.float32(std))
+           for k, s in (("w_q", (L, H, H)), ("b_q", (L, H)), ("w_o", (L, H, H)), ("b_o", (L, H)))}
+    out["ctx_kv"] = _store(wl, g.standard_normal((L, wl.B, 2, n_ctx, H), dtype=np.float32) * np.float32(0.5))
+    return out

@@ -38,6 +38,10 @@ class _DenseWeights(ctypes.Structure):    # fdo_dense_weights of dense_block.c
                                                "b_fc2", "qn_w", "kn_w")]
 
 
+class _Cross(ctypes.Structure):           # fdo_cross / fdo_dense_cross
+    _fields_ = [(n, ctypes.c_void_p) for n in ("w_q", "b_q", "w_o", "b_o", "ctx_kv")] + [("T", ctypes.c_int)]
+
+
 _lib = None
 _f = ctypes.POINTER(ctypes.c_float)
 _i = ctypes.POINTER(ctypes.c_int32)
@@ -54,6 +58,8 @@ def _load():
         _lib.fdo_dense_block_v.restype = ctypes.c_int
         _lib.fdo_regional_block_s.restype = ctypes.c_int
         _lib.fdo_dense_block_d.restype = ctypes.c_int
+        _lib.fdo_regional_block_x.restype = ctypes.c_int
+        _lib.fdo_dense_block_x.restype = ctypes.c_int
     return _lib
 
 
@@ -91,6 +97,20 @@ def _addr(a: Optional[np.ndarray], keep: list) -> Optional[int]:
     return a.ctypes.data
 
 
+def _cross_arg(v, l: int, B: int, H: int, keep: list):
+    """fdo_cross of block ``l`` from variants["cross"] = {w_q [L,H,H], b_q [L,H], w_o, b_o, ctx_kv [L,B,2,T,H]}."""
+    c = v.get("cross")
+    if c is None:
+        return None
+    kvc = _c(c["ctx_kv"][l])
+    assert kvc.shape[0] == B and kvc.shape[1] == 2 and kvc.shape[3] == H
+    keep.append(kvc)
+    st = _Cross(_addr(c["w_q"][l], keep), _addr(c["b_q"][l], keep), _addr(c["w_o"][l], keep), _addr(c["b_o"][l], keep),
+                kvc.ctypes.data, int(kvc.shape[2]))
+    keep.append(st)
+    return ctypes.byref(st)
+
+
 def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w: Dict[str, np.ndarray],
                    l: int, kv_l: np.ndarray, heads: int, ln_eps: float = 1e-6,
                    finish: Optional[np.ndarray] = None, variants=None, mod_text: Optional[np.ndarray] = None,
@@ -125,11 +145,11 @@ def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w:
     rc_, rs_ = _addr(v.get("rope_cos"), keep), _addr(v.get("rope_sin"), keep)
     if rc_ is not None:
         assert keep[-2].shape == (N, dh // 2)
-    rc = _load().fdo_regional_block_s(
+    rc = _load().fdo_regional_block_x(
         B, N, H, heads, dh, M, A, _ip(np.ascontiguousarray(active_idx, np.int32)), ctypes.byref(img), txt,
         None if tt is None else tt.ctypes.data_as(ctypes.c_void_p), ctypes.c_float(ln_eps), _fp(_c(u_in)), _fp(u_out), _fp(kv_l),
         0 if fin is None else int(fin.size), _ip(fin), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))),
-        ctypes.c_void_p(rc_), ctypes.c_void_p(rs_))
+        ctypes.c_void_p(rc_), ctypes.c_void_p(rs_), _cross_arg(v, l, B, H, keep))
     assert rc == 0
     return u_out
 
@@ -206,9 +226,10 @@ def dense_block(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], l: in
     rc_, rs_ = _addr(v.get("rope_cos"), keep), _addr(v.get("rope_sin"), keep)
     if rc_ is not None:
         assert keep[-2].shape == (N, dh // 2)
-    rc = _load().fdo_dense_block_d(
+    rc = _load().fdo_dense_block_x(
         B, N, H, heads, dh, M, Hc, _fp(_c(cond)), ctypes.byref(wi), wt, n_text, ctypes.c_float(ln_eps), _fp(_c(x)), _fp(x_out),
-        _fp(kv), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))), ctypes.c_void_p(rc_), ctypes.c_void_p(rs_))
+        _fp(kv), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))), ctypes.c_void_p(rc_), ctypes.c_void_p(rs_),
+        _cross_arg(v, l, B, H, keep))
     assert rc == 0
     return x_out, kv
 

@@ -46,20 +46,25 @@ static void layernorm_modulate(const float* X, size_t rows, int H, const float* 
     }
 }
 
-/* O[i, h*dh + c] = sum_t softmax_t(Q_i . K_t / sqrt(dh)) V[t, h*dh + c], all N x N pairs */
+/* O[i, h*dh + c] = sum_t softmax_t(Q_i . K_t / sqrt(dh)) V[t, h*dh + c]: N queries against all T keys (T = N for the
+ * block's self-attention) */
+static void attention_nt(const float* Q, const float* K, const float* V, int N, int T, int heads, int dh, float* O);
 static void full_attention(const float* Q, const float* K, const float* V, int N, int heads, int dh,
                            float* O) {
+    attention_nt(Q, K, V, N, N, heads, dh, O);
+}
+static void attention_nt(const float* Q, const float* K, const float* V, int N, int T, int heads, int dh, float* O) {
     const int H = heads * dh;
     const double scale = 1.0 / sqrt((double)dh);
 #pragma omp parallel
     {
-        double* s = (double*)malloc(sizeof(double) * (size_t)N);
+        double* s = (double*)malloc(sizeof(double) * (size_t)T);
         double* acc = (double*)malloc(sizeof(double) * (size_t)dh);
 #pragma omp for schedule(dynamic, 1) collapse(2)
         for (int i = 0; i < N; ++i)
             for (int h = 0; h < heads; ++h) {
                 double mx = -INFINITY;
-                for (int t = 0; t < N; ++t) {
+                for (int t = 0; t < T; ++t) {
                     double d = 0.0;
                     for (int c = 0; c < dh; ++c)
                         d += (double)Q[(size_t)i * H + h * dh + c] * (double)K[(size_t)t * H + h * dh + c];
@@ -68,7 +73,7 @@ static void full_attention(const float* Q, const float* K, const float* V, int N
                 }
                 double z = 0.0;
                 for (int c = 0; c < dh; ++c) acc[c] = 0.0;
-                for (int t = 0; t < N; ++t) {
+                for (int t = 0; t < T; ++t) {
                     const double e = exp(s[t] - mx);
                     z += e;
                     for (int c = 0; c < dh; ++c) acc[c] += e * (double)V[(size_t)t * H + h * dh + c];
@@ -135,10 +140,29 @@ typedef struct {
     const float *w_ada, *b_ada, *w_qkv, *b_qkv, *w_o, *b_o, *w_fc1, *b_fc1, *w_fc2, *b_fc2, *qn_w, *kn_w;
 } fdo_dense_weights;
 
+/*
+ * fdo_dense_block_x adds cross-attention to a fixed context (reading of the text-conditioning path of Wan2.1 /
+ * StableAudio-type blocks): after the self-attention update, res <- res + (Attn(LN(res) W_q^T + b_q, K_ctx, V_ctx)) W_o^T
+ * + b_o, plain LayerNorm, no modulation, no gate; ctx_kv [B,2,T,H] is given.  On whole matrices: the LayerNorm is the
+ * modulated one with zero shift and scale.
+ */
+typedef struct {
+    const float *w_q, *b_q, *w_o, *b_o, *ctx_kv;
+    int T;
+} fdo_dense_cross;
+
+int fdo_dense_block_x(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+                      const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
+                      const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
+                      const float* rope_sin, const fdo_dense_cross* cross);
+
 int fdo_dense_block_d(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
                       const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
-                      const float* rope_sin);
+                      const float* rope_sin) {
+    return fdo_dense_block_x(B, N, H, heads, dh, M, Hc, cond, wi, wt, n_text, ln_eps, x_in, x_out, kv_out, qk_eps, rope_cos,
+                             rope_sin, NULL);
+}
 
 int fdo_dense_block_v(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const float* w_ada, const float* b_ada, const float* w_qkv, const float* b_qkv,
@@ -160,10 +184,10 @@ int fdo_dense_block(int B, int N, int H, int heads, int dh, int M, int Hc, const
                              b_fc2, ln_eps, x_in, x_out, kv_out, NULL, NULL, 0.f, NULL, NULL);
 }
 
-int fdo_dense_block_d(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+int fdo_dense_block_x(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
                       const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
-                      const float* rope_sin) {
+                      const float* rope_sin, const fdo_dense_cross* cross) {
     if (heads * dh != H) return 2;
     if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
     if (!wt) n_text = 0;
@@ -228,6 +252,19 @@ int fdo_dense_block_d(int B, int N, int H, int heads, int dh, int M, int Hc, con
             matmul_nt_bias(att + lo * H, ws[s]->w_o, ws[s]->b_o, n, H, H, proj + lo * H);
             for (size_t e = lo * H; e < (lo + n) * H; ++e)
                 res[e] = (float)((double)X[e] + (double)gate_a[e % H] * (double)proj[e]);
+        }
+
+        if (cross) {
+            /* cross-attention of all N rows to the request's T context tokens; plain LayerNorm = zero shift and scale */
+            float* zero = (float*)calloc((size_t)H, sizeof(float));
+            if (!zero) { rc = 1; goto done; }
+            layernorm_modulate(res, (size_t)N, H, zero, zero, ln_eps, xh);
+            free(zero);
+            matmul_nt_bias(xh, cross->w_q, cross->b_q, (size_t)N, H, H, Q);
+            attention_nt(Q, cross->ctx_kv + ((size_t)b * 2 + 0) * cross->T * H, cross->ctx_kv + ((size_t)b * 2 + 1) * cross->T * H,
+                         N, cross->T, heads, dh, att);
+            matmul_nt_bias(att, cross->w_o, cross->b_o, (size_t)N, H, H, proj);
+            for (size_t e = 0; e < NH; ++e) res[e] = (float)((double)res[e] + (double)proj[e]);
         }
 
         /* MLP branch, per stream */

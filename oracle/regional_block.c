@@ -135,10 +135,32 @@ typedef struct {
     const float *qn_w, *kn_w;               /* [dh] or NULL */
 } fdo_stream;
 
+/*
+ * Cross-attention to a fixed context (the text-conditioning path of the paper's Wan2.1 / StableAudio-type models;
+ * not defined in the paper, this build's reading): between the self-attention update and the MLP,
+ *     r1 <- r1 + W_o . Attn(LN(r1) W_q^T + b_q, K_ctx, V_ctx) + b_o
+ * with a plain LayerNorm (no affine, no modulation), softmax(q k^T / sqrt(dh)) per head over the T context tokens
+ * of the row's request, and no gate.  K_ctx and V_ctx do not change over the denoising steps and are given:
+ * ctx_kv [B,2,T,H].  cross = NULL: no cross-attention.
+ */
+typedef struct {
+    const float *w_q, *b_q, *w_o, *b_o;     /* [H,H], [H] */
+    const float *ctx_kv;                    /* [B,2,T,H] */
+    int T;
+} fdo_cross;
+
+int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
+                         const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
+                         float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
+                         float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross);
+
 int fdo_regional_block_s(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
                          const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
                          float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
-                         float qk_eps, const float* rope_cos, const float* rope_sin);
+                         float qk_eps, const float* rope_cos, const float* rope_sin) {
+    return fdo_regional_block_x(B, N, H, heads, dh, M, A, active_idx, img, txt, tok_text, ln_eps, u_in, u_out, kv, n_finish,
+                                finish, qk_eps, rope_cos, rope_sin, NULL);
+}
 
 int fdo_regional_block_v(int B, int N, int H, int heads, int dh, int M, int A,
                          const int32_t* active_idx, const float* mod,
@@ -162,10 +184,10 @@ int fdo_regional_block(int B, int N, int H, int heads, int dh, int M, int A,
                                 b_fc2, ln_eps, u_in, u_out, kv, n_finish, finish, NULL, NULL, 0.f, NULL, NULL);
 }
 
-int fdo_regional_block_s(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
+int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
                          const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
                          float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
-                         float qk_eps, const float* rope_cos, const float* rope_sin) {
+                         float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross) {
     if (heads * dh != H) return 2;
     if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
     (void)B;
@@ -204,7 +226,7 @@ int fdo_regional_block_s(int B, int N, int H, int heads, int dh, int M, int A, c
     const double sm_scale = 1.0 / sqrt((double)dh);
 #pragma omp parallel
     {
-        double* s = (double*)malloc(sizeof(double) * (size_t)N);
+        double* s = (double*)malloc(sizeof(double) * (size_t)(cross && cross->T > N ? cross->T : N));
         double* oacc = (double*)malloc(sizeof(double) * (size_t)dh);
         float* o = (float*)malloc(sizeof(float) * (size_t)H);
         float* proj = (float*)malloc(sizeof(float) * (size_t)H);
@@ -248,6 +270,38 @@ int fdo_regional_block_s(int B, int N, int H, int heads, int dh, int M, int A, c
                 row_linear(o, st->w_o, st->b_o, H, H, proj);
                 for (int c = 0; c < H; ++c)
                     r1[c] = (float)((double)u[c] + (double)md[2 * H + c] * (double)proj[c]);
+                if (cross) {
+                    /* cross-attention of this row to the T context tokens of its request */
+                    const int T = cross->T;
+                    const float* Kc = cross->ctx_kv + ((size_t)b * 2 + 0) * T * H;
+                    const float* Vc = cross->ctx_kv + ((size_t)b * 2 + 1) * T * H;
+                    double mean = 0.0, var = 0.0;
+                    for (int c = 0; c < H; ++c) mean += (double)r1[c];
+                    mean /= (double)H;
+                    for (int c = 0; c < H; ++c) { const double d = (double)r1[c] - mean; var += d * d; }
+                    const double rstd = 1.0 / sqrt(var / (double)H + (double)ln_eps);
+                    for (int c = 0; c < H; ++c) mh[c] = (float)(((double)r1[c] - mean) * rstd);
+                    row_linear(mh, cross->w_q, cross->b_q, H, H, proj);              /* proj holds the cross queries */
+                    for (int h = 0; h < heads; ++h) {
+                        double smax = -INFINITY;
+                        for (int t = 0; t < T; ++t) {
+                            double acc = 0.0;
+                            for (int c = 0; c < dh; ++c) acc += (double)proj[h * dh + c] * (double)Kc[(size_t)t * H + h * dh + c];
+                            s[t] = acc * sm_scale;
+                            if (s[t] > smax) smax = s[t];
+                        }
+                        double denom = 0.0;
+                        for (int c = 0; c < dh; ++c) oacc[c] = 0.0;
+                        for (int t = 0; t < T; ++t) {
+                            const double p = exp(s[t] - smax);
+                            denom += p;
+                            for (int c = 0; c < dh; ++c) oacc[c] += p * (double)Vc[(size_t)t * H + h * dh + c];
+                        }
+                        for (int c = 0; c < dh; ++c) o[h * dh + c] = (float)(oacc[c] / denom);
+                    }
+                    row_linear(o, cross->w_o, cross->b_o, H, H, proj);
+                    for (int c = 0; c < H; ++c) r1[c] = (float)((double)r1[c] + (double)proj[c]);
+                }
                 row_ln_modulate(r1, md + 3 * H, md + 4 * H, H, ln_eps, mh);
                 row_linear(mh, st->w_fc1, st->b_fc1, H, M, g);
                 for (int c = 0; c < M; ++c) g[c] = (float)gelu_tanh_d((double)g[c]);
