@@ -204,6 +204,32 @@ fd_status fd_set_block_variants(fd_ctx* ctx, const fd_block_variants* v);
 fd_status fd_set_text_stream(fd_ctx* ctx, const fd_weights* text_weights);
 
 /*
+ * Cross-attention to a fixed context (the text conditioning of the paper's Wan2.1 and PixArt-style blocks; no equation
+ * of the paper covers it, the reading is the published block structure of those models).  When set, every block
+ * does, between the self-attention update and the MLP branch and for the active rows only,
+ *     r <- r + W_o . Attn(LN(r) W_q^T + b_q, K_ctx, V_ctx) + b_o
+ * with LN the plain LayerNorm of the block (ln_eps; no scale, shift or adaLN modulation), Attn the per-head
+ * softmax(q k^T / sqrt(head_dim)) over the n_ctx context tokens of the row's request, and no gate.  The context's
+ * keys and values are the caller's (a text encoder's states, projected once per prompt): they do not depend on
+ * the step, so region skipping leaves them alone, and a skipped row keeps its cached block output as before.
+ * DEVICE pointers in the storage type, 16-byte aligned, owned by the caller and alive while set:
+ *   w_q, w_o [L, H, H] (out, in), b_q, b_o [L, H], ctx_kv [L, ctx_batch, 2, n_ctx, H] (keys then values; heads
+ *   side by side as in the self-attention cache).  n_ctx >= 1.  A step with B != ctx_batch fails with
+ *   FD_ERR_SHAPE.  In a dual-stream context both streams use this one set.  NULL switches it off.  Host call, no
+ *   launch; takes effect from the next step.
+ */
+typedef struct fd_cross_attention {
+    const void* w_q;
+    const void* b_q;
+    const void* w_o;
+    const void* b_o;
+    const void* ctx_kv;
+    int n_ctx;
+    int ctx_batch;
+} fd_cross_attention;
+fd_status fd_set_cross_attention(fd_ctx* ctx, const fd_cross_attention* cross);
+
+/*
  * The Patch Gate on the paper's own signal (Sec. 4.2): the refinement importance of a patch is the block mean of
  * the self-attention matrix over the patch,  R_i = (1/|A_i|^2) sum_{u,v in A_i} SA[u,v],  and the gate weights are
  * the normalised changes  Delta_i = |R_i - Rbar_i|  (Rbar_i = the importance at the patch's last executed step;
@@ -334,7 +360,8 @@ enum {
     FD_PROF_PARTITION = 9,
     FD_PROF_SAMPLER = 10, /* patch embedding, final layer, latent update */
     FD_PROF_QK_VARIANTS = 11, /* QK-RMSNorm + rotary embedding (block variants) */
-    FD_PROF_GROUPS = 12
+    FD_PROF_CROSS = 12,   /* cross-attention: LayerNorm, query projection, attention, out-projection */
+    FD_PROF_GROUPS = 13
 };
 fd_status fd_profile_enable(fd_ctx* ctx, int enable);
 fd_status fd_profile_read(fd_ctx* ctx, void* cuda_stream, float* ms_out, int32_t* kernels_out);

@@ -24,10 +24,10 @@ EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region
            "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait",
            "fd_embed_latent", "fd_update_latent", "fd_regional_step_mass", "fd_region_activity_attn",
            "fd_sched_pack", "fd_sched_form_batch", "fd_rsearch_init", "fd_rsearch_update", "fd_set_block_variants",
-           "fd_set_text_stream"]
+           "fd_set_text_stream", "fd_set_cross_attention"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
-               "gemm_fc2", "partition", "sampler", "qk_variants"]
+               "gemm_fc2", "partition", "sampler", "qk_variants", "cross_attention"]
 
 
 class FdConfig(ctypes.Structure):
@@ -50,6 +50,11 @@ class FdBlockVariants(ctypes.Structure):
     _fields_ = [("q_norm_w", ctypes.c_void_p), ("k_norm_w", ctypes.c_void_p), ("qk_norm_eps", ctypes.c_float),
                 ("rope_cos", ctypes.c_void_p), ("rope_sin", ctypes.c_void_p), ("q_norm_w_text", ctypes.c_void_p),
                 ("k_norm_w_text", ctypes.c_void_p)]
+
+
+class FdCrossAttention(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("w_q", "b_q", "w_o", "b_o", "ctx_kv")] + \
+               [("n_ctx", ctypes.c_int32), ("ctx_batch", ctypes.c_int32)]
 
 
 class FdRSearch(ctypes.Structure):
@@ -110,6 +115,8 @@ def _load() -> ctypes.CDLL:
     lib.fd_set_block_variants.argtypes = [vp, ctypes.POINTER(FdBlockVariants)]
     lib.fd_set_text_stream.restype = i32
     lib.fd_set_text_stream.argtypes = [vp, ctypes.POINTER(FdWeights)]
+    lib.fd_set_cross_attention.restype = i32
+    lib.fd_set_cross_attention.argtypes = [vp, ctypes.POINTER(FdCrossAttention)]
     lib.fd_launch_count.restype = ctypes.c_int64
     lib.fd_launch_count.argtypes = [vp]
     lib.fd_destroy.restype = i32
@@ -294,6 +301,22 @@ def fd_set_text_stream(ctx: Context, text_weights: Optional[Dict[str, "object"]]
         assert t.is_cuda and t.is_contiguous() and t.dtype == ctx.dtype, k
     w = FdWeights(**{k: text_weights[k].data_ptr() for k, _ in FdWeights._fields_})
     _check(ctx.handle, lib.fd_set_text_stream(ctx.handle, ctypes.byref(w)))
+
+
+def fd_set_cross_attention(ctx: Context, cross: Optional[Dict[str, "object"]]) -> None:
+    """Cross-attention to a fixed context in every block: ``cross`` holds device tensors of the context's dtype, w_q, w_o
+    [L, H, H], b_q, b_o [L, H] and ctx_kv [L, B, 2, n_ctx, H] (the context keeps them alive); None switches it off."""
+    ctx.cross = cross
+    if cross is None:
+        _check(ctx.handle, lib.fd_set_cross_attention(ctx.handle, None))
+        return
+    for k in ("w_q", "b_q", "w_o", "b_o", "ctx_kv"):
+        t = cross[k]
+        assert t.is_cuda and t.is_contiguous() and t.dtype == ctx.dtype, k
+    kv = cross["ctx_kv"]
+    assert kv.dim() == 5 and kv.shape[2] == 2
+    x = FdCrossAttention(*(cross[k].data_ptr() for k in ("w_q", "b_q", "w_o", "b_o", "ctx_kv")), int(kv.shape[3]), int(kv.shape[1]))
+    _check(ctx.handle, lib.fd_set_cross_attention(ctx.handle, ctypes.byref(x)))
 
 
 def fd_sched_pack(load, cost, home):

@@ -25,7 +25,7 @@ thread_local std::string g_create_error;
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-    size_t control, acc_ss, acc_cnt, block_counts, tiles, text_tiles, ada_act, mod, resid, act, q, o, g, part, attn_ws, total;
+    size_t control, acc_ss, acc_cnt, block_counts, tiles, text_tiles, consts, ada_act, mod, resid, act, q, o, g, part, attn_ws, total;
     int Mcap, q_ld, tile_cap;
 };
 
@@ -65,6 +65,7 @@ Layout make_layout(const fd_config& c) {
     l.tiles = take((size_t)2 * l.tile_cap * sizeof(QTile));      // work list, then the list of double-height tiles
     // dual stream: the 128-row and the 256-row tiles that hold rows of the second stream
     l.text_tiles = take(((size_t)l.Mcap / 128 + (size_t)l.Mcap / 256 + 2) * sizeof(int32_t));
+    l.consts = take((size_t)2 * c.hidden * sizeof(float));       // [H] zeros, then [H] ones
     l.ada_act = take((size_t)2 * ((c.max_batch + 7) / 8 * 8) * c.cond_dim * 2);   // SiLU(cond): bf16 head + remainder
     l.mod = take((size_t)2 * c.n_blocks * c.max_batch * 6 * c.hidden * sizeof(float));   // adaLN vectors, then the second stream's
     l.resid = take((size_t)l.Mcap * c.hidden * sizeof(float));
@@ -94,6 +95,7 @@ struct fd_ctx {
     fd_block_variants var{};   // block variants (all pointers null: off)
     fd_weights text_w{};       // second stream's weights (dual stream; w_qkv null: single stream)
     bool dual = false;
+    fd_cross_attention cross{};   // cross-attention to a fixed context (w_q null: off)
     // optional per-kernel timing
     bool profiling = false;
     struct Span { cudaEvent_t a, b; int group, kernels; };
@@ -193,6 +195,11 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     };
     const int n_pass = dual ? 2 : 1;
     const int max_tiles = B * ((N + c->tile_rows - 1) / c->tile_rows);
+    const fd_cross_attention& xa = c->cross;
+    if (xa.w_q && B != xa.ctx_batch)
+        return c->fail(FD_ERR_SHAPE, "B=%d differs from the cross-attention context's batch %d", B, xa.ctx_batch);
+    const float* zeros = c->at<float>(l.consts);
+    const float* ones = zeros + H;
     const bool pdl = c->use_tc && c->tc && tc_plan_pdl(c->tc);
     for (int blk = 0; blk < L; ++blk) {
         const float* mod_b = mod + (size_t)blk * B * 6 * H;
@@ -267,6 +274,34 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             else
                 FD_TRY(FD_PROF_GEMM_OUT, launch_simt_gemm<T>(EPI_RESID, o, H, stream_ptr(c->w.w_o, c->text_w.w_o, (size_t)blk * H * H, pass), H, H,
                                                              rows_cap, ep, ctl, st, &nl));
+        }
+        // cross-attention to the fixed context: plain LayerNorm, query projection, the attention kernel over the
+        // context's keys and values in place of the cache, out-projection added without a gate
+        if (xa.w_q) {
+            const T* ctx_b = static_cast<const T*>(xa.ctx_kv) + (size_t)blk * B * 2 * xa.n_ctx * H;
+            FD_TRY(FD_PROF_CROSS, launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, zeros, zeros, 0, N, H, rows_cap,
+                                                        cf.ln_eps, ctl, st, &nl, pdl, TextSel{nullptr, 0, 0}));
+            ep.group = -1;
+            ep.bias = static_cast<const T*>(xa.b_q) + (size_t)blk * H;
+            if (c->use_tc)
+                FD_TRY(FD_PROF_CROSS, tc_gemm(c->tc, TC_GEMM_XQ, blk, ep, ctl, st, &nl));
+            else
+                FD_TRY(FD_PROF_CROSS, launch_simt_gemm<T>(EPI_QKV, act, H, static_cast<const T*>(xa.w_q) + (size_t)blk * H * H, H, H,
+                                                          rows_cap, ep, ctl, st, &nl));
+            if (c->use_tc_attn)
+                FD_TRY(FD_PROF_CROSS, tc_attention(c->tc, blk, const_cast<T*>(ctx_b), B, xa.n_ctx, tiles, max_tiles, ctl, st, &nl));
+            else
+                FD_TRY(FD_PROF_CROSS, launch_simt_attention<T>(q, l.q_ld, ctx_b, o, H, tiles, max_tiles, xa.n_ctx, H, cf.n_heads,
+                                                               cf.head_dim, ctl, st, &nl, 0, nullptr, nullptr, nullptr, 0));
+            ep.gate = ones;
+            ep.ungated = 1;
+            ep.bias = static_cast<const T*>(xa.b_o) + (size_t)blk * H;
+            if (c->use_tc)
+                FD_TRY(FD_PROF_CROSS, tc_gemm(c->tc, TC_GEMM_XO, blk, ep, ctl, st, &nl));
+            else
+                FD_TRY(FD_PROF_CROSS, launch_simt_gemm<T>(EPI_RESID, o, H, static_cast<const T*>(xa.w_o) + (size_t)blk * H * H, H, H,
+                                                          rows_cap, ep, ctl, st, &nl));
+            ep.ungated = 0;
         }
         // MLP branch
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, mod_b + 3 * H, mod_b + 4 * H, 6 * H, N,
@@ -354,6 +389,11 @@ fd_status fd_create(const fd_config* cfg, const fd_weights* weights, void* works
     // control block and gate accumulators start at zero; the compact buffers start finite
     e = cudaMemset(workspace, 0, lay.ada_act);
     if (e == cudaSuccess) e = cudaMemset(c->ws + lay.resid, 0, lay.part - lay.resid);
+    if (e == cudaSuccess) {
+        const std::vector<float> one(cfg->hidden, 1.0f);
+        e = cudaMemcpy(c->ws + lay.consts + (size_t)cfg->hidden * sizeof(float), one.data(), one.size() * sizeof(float),
+                       cudaMemcpyHostToDevice);
+    }
     if (e == cudaSuccess && use_tc) {
         TcBuffers tb{};
         tb.act = c->ws + lay.act; tb.q = c->ws + lay.q; tb.o = c->ws + lay.o; tb.g = c->ws + lay.g;
@@ -626,6 +666,27 @@ fd_status fd_set_text_stream(fd_ctx* c, const fd_weights* text_weights) {
     }
     c->text_w = *text_weights;
     c->dual = true;
+    return FD_OK;
+}
+
+fd_status fd_set_cross_attention(fd_ctx* c, const fd_cross_attention* x) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!x) {
+        c->cross = fd_cross_attention{};
+        if (c->tc) tc_plan_set_cross(c->tc, nullptr, nullptr, nullptr);
+        return FD_OK;
+    }
+    const void* wp[5] = {x->w_q, x->b_q, x->w_o, x->b_o, x->ctx_kv};
+    for (const void* p : wp)
+        if (!p || !aligned16(p)) return c->fail(FD_ERR_INVALID_ARG, "cross-attention pointer null or not 16-byte aligned");
+    if (x->n_ctx < 1 || x->ctx_batch < 1 || x->ctx_batch > c->cfg.max_batch)
+        return c->fail(FD_ERR_SHAPE, "n_ctx must be positive and ctx_batch in [1, max_batch]");
+    if (c->tc) {
+        std::string err;
+        if (!tc_plan_set_cross(c->tc, x->w_q, x->w_o, &err))
+            return c->fail(FD_ERR_CUDA, "tensor maps of the cross-attention weights: %s", err.c_str());
+    }
+    c->cross = *x;
     return FD_OK;
 }
 

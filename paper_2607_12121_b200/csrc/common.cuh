@@ -86,6 +86,7 @@ struct EpiParams {
     int32_t R;
     int32_t group;             // -1: every row; 0: rows of the first stream only; 1: rows of the second stream only
     int32_t text_mod_off;      // offset (floats) from a request's adaLN vectors to those of the second stream
+    int32_t ungated;           // EPI_RESID: `gate` is one [H] vector for every row (cross-attention passes ones)
 };
 
 // Per-row choice of the second stream's adaLN vectors in the row kernels (labels == nullptr: single stream).

@@ -53,7 +53,7 @@ __device__ __forceinline__ void epilogue4(const EpiParams& ep, int row, int col,
         }
     } else if constexpr (KIND == EPI_RESID) {
         const int b = tok / ep.N;
-        const float4 g = *reinterpret_cast<const float4*>(ep.gate + (size_t)b * 6 * ep.H + col);
+        const float4 g = *reinterpret_cast<const float4*>(ep.gate + (ep.ungated ? (size_t)0 : (size_t)b * 6 * ep.H) + col);
         float* rp = ep.resid + (size_t)row * ep.H + col;
         float4 r = *reinterpret_cast<const float4*>(rp);
         r.x = fmaf(g.x, v[0], r.x); r.y = fmaf(g.y, v[1], r.y);
@@ -296,11 +296,11 @@ __device__ __forceinline__ RowInfo epilogue_row_info(const EpiParams& ep, int la
     if ((KIND != EPI_GELU || ep.group >= 0) && ok) {
         const int tok = ep.active_idx[row_base + lane];
         const int b = tok / ep.N;
-        ri.gate_off = b * 6 * ep.H;
+        ri.gate_off = ep.ungated ? 0 : b * 6 * ep.H;
         if (ep.group >= 0) {                                     // dual stream: this launch owns one stream's rows
             const int text = ep.labels[tok] == ep.R ? 1 : 0;
             ok = text == ep.group;
-            if (text) ri.gate_off += ep.text_mod_off;
+            if (text && !ep.ungated) ri.gate_off += ep.text_mod_off;
         }
         const size_t off = KIND == EPI_RESID ? (size_t)tok * ep.H : ((size_t)b * 2 * ep.N + (tok - b * ep.N)) * ep.H;
         ri.y_lo = (uint32_t)off;

@@ -64,7 +64,7 @@ simt_gemm_kernel(const T* __restrict__ a, int lda, const T* __restrict__ w, int 
             const int text = ep.group >= 0 && ep.labels[tok] == ep.R ? 1 : 0;
             if (ep.group < 0 || text == ep.group) {
                 EpiParams e2 = ep;
-                if (text && e2.gate) e2.gate += ep.text_mod_off;
+                if (text && e2.gate && !ep.ungated) e2.gate += ep.text_mod_off;
                 epilogue4<T, KIND>(e2, row, col, tok, acc[i]);
             }
         }

@@ -18,7 +18,8 @@ struct TcBuffers {  // compact activation buffers inside the workspace (bf16)
     int attn_slots;
 };
 
-enum TcGemmKind { TC_GEMM_QKV = 0, TC_GEMM_OUT = 1, TC_GEMM_FC1 = 2, TC_GEMM_FC2 = 3 };
+// the last two are the cross-attention's projections (query: activations -> Q buffer; out: attention output -> residual)
+enum TcGemmKind { TC_GEMM_QKV = 0, TC_GEMM_OUT = 1, TC_GEMM_FC1 = 2, TC_GEMM_FC2 = 3, TC_GEMM_XQ = 4, TC_GEMM_XO = 5 };
 
 bool tc_supported(const fd_config& cfg, std::string* why);
 bool tc_attention_supported(const fd_config& cfg);
@@ -33,6 +34,8 @@ void tc_plan_destroy(TcPlan* p);
 cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
                     int* n_launch, bool text_pass = false);
 bool tc_plan_set_text(TcPlan* p, const fd_weights* w, const int32_t* list128, const int32_t* list256, std::string* err);
+// cross-attention: tensor maps of its two [L, H, H] projection weights (both nullptr: off)
+bool tc_plan_set_cross(TcPlan* p, const void* w_q, const void* w_o, std::string* err);
 // region_mass (optional): [B, R] f64, receives the own-region softmax mass
 cudaError_t tc_attention(TcPlan* p, int blk, void* kv_block, int B, int N, const QTile* tiles, int max_tiles,
                          const Control* ctl, cudaStream_t st, int* n_launch, const int32_t* labels = nullptr,

@@ -388,11 +388,12 @@ struct TcPlan {
     int sm_count;
     bool pdl;                   // launch the tensor-core kernels with programmatic stream serialization
     int pair_ctas;              // grid of the CTA-pair kernel: 2 x co-resident clusters
-    GemmSpec spec[4];
+    GemmSpec spec[6];           // indexed by TcGemmKind
     CUtensorMap resid_map;      // fp32 residual stream [Mcap, H], 32 x 32 boxes for the bulk reductions of EPI_RESID
     bool tma_resid;
     CUtensorMap* w_maps;        // [L][4]
     CUtensorMap* w_maps_text;   // [L][4] second stream's weights (dual stream), or nullptr
+    CUtensorMap* w_maps_cross;  // [L][2] cross-attention's query and out projections, or nullptr
     const int32_t* text_list128;    // device lists of the row tiles that hold rows of the second stream
     const int32_t* text_list256;
     // attention (filled by the attention part)
@@ -416,6 +417,7 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
     p->buf = buf;
     p->w_maps = new CUtensorMap[(size_t)cfg.n_blocks * 4];
     p->w_maps_text = nullptr;
+    p->w_maps_cross = nullptr;
     p->text_list128 = p->text_list256 = nullptr;
     p->attn = nullptr;
     int dev = 0;
@@ -431,13 +433,13 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
     bool use_pair = true;       // switch: FD_TC_PAIR=0 keeps every GEMM on the single-CTA kernel
     if (const char* v = getenv("FD_TC_PAIR")) use_pair = atoi(v) != 0;
     const int H = cfg.hidden, M = cfg.mlp_dim;
-    const int n_out[4] = {3 * H, H, M, H};
-    const int kdim[4] = {H, H, H, M};
-    void* a_base[4] = {buf.act, buf.o, buf.act, buf.g};
+    const int n_out[6] = {3 * H, H, M, H, H, H};
+    const int kdim[6] = {H, H, H, M, H, H};
+    void* a_base[6] = {buf.act, buf.o, buf.act, buf.g, buf.act, buf.o};
     const char* w_base[4] = {static_cast<const char*>(w.w_qkv), static_cast<const char*>(w.w_o),
                              static_cast<const char*>(w.w_fc1), static_cast<const char*>(w.w_fc2)};
     bool ok = true;
-    for (int g = 0; g < 4 && ok; ++g) {
+    for (int g = 0; g < 6 && ok; ++g) {
         GemmSpec& s = p->spec[g];
         s.n_out = n_out[g];
         s.k = kdim[g];
@@ -447,7 +449,7 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         const uint64_t strides[1] = {(uint64_t)kdim[g] * 2};
         const uint32_t box[2] = {BK, BM};
         ok = encode_tmap_bf16(&s.a, a_base[g], 2, dims, strides, box, 128, err);
-        for (int l = 0; l < cfg.n_blocks && ok; ++l) {
+        for (int l = 0; l < cfg.n_blocks && ok && g < 4; ++l) {
             const uint64_t wd[2] = {(uint64_t)kdim[g], (uint64_t)n_out[g]};
             const uint32_t wb[2] = {BK, s.pair_bn ? (uint32_t)s.pair_bn / 2 : (uint32_t)s.bn};
             void* base = const_cast<char*>(w_base[g]) + (size_t)l * n_out[g] * kdim[g] * 2;
@@ -516,6 +518,7 @@ void tc_plan_destroy(TcPlan* p) {
     tc_attention_plan_destroy(p->attn);
     delete[] p->w_maps;
     delete[] p->w_maps_text;
+    delete[] p->w_maps_cross;
     delete p;
 }
 
@@ -561,11 +564,42 @@ bool tc_plan_set_text(TcPlan* p, const fd_weights* w, const int32_t* list128, co
     return true;
 }
 
-cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
+bool tc_plan_set_cross(TcPlan* p, const void* w_q, const void* w_o, std::string* err) {
+    delete[] p->w_maps_cross;
+    p->w_maps_cross = nullptr;
+    if (!w_q || !w_o) return true;
+    const fd_config& cfg = p->cfg;
+    const int H = cfg.hidden;
+    const char* w_base[2] = {static_cast<const char*>(w_q), static_cast<const char*>(w_o)};
+    p->w_maps_cross = new CUtensorMap[(size_t)cfg.n_blocks * 2];
+    for (int g = 0; g < 2; ++g) {
+        const GemmSpec& s = p->spec[TC_GEMM_XQ + g];
+        for (int l = 0; l < cfg.n_blocks; ++l) {
+            const uint64_t wd[2] = {(uint64_t)H, (uint64_t)H};
+            const uint64_t strides[1] = {(uint64_t)H * 2};
+            const uint32_t wb[2] = {BK, s.pair_bn ? (uint32_t)s.pair_bn / 2 : (uint32_t)s.bn};
+            void* base = const_cast<char*>(w_base[g]) + (size_t)l * H * H * 2;
+            if (!encode_tmap_bf16(&p->w_maps_cross[(size_t)l * 2 + g], base, 2, wd, strides, wb, 128, err)) {
+                delete[] p->w_maps_cross;
+                p->w_maps_cross = nullptr;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind_in, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
                     int* n_launch, bool text_pass) {
-    const GemmSpec& s = p->spec[kind];
-    if (text_pass && !p->w_maps_text) return cudaErrorInvalidValue;
-    const CUtensorMap& wm = text_pass ? p->w_maps_text[(size_t)blk * 4 + kind] : p->w_maps[(size_t)blk * 4 + kind];
+    const GemmSpec& s = p->spec[kind_in];
+    const bool cross = kind_in >= TC_GEMM_XQ;
+    if (text_pass && (!p->w_maps_text || cross)) return cudaErrorInvalidValue;
+    if (cross && !p->w_maps_cross) return cudaErrorInvalidValue;
+    const CUtensorMap& wm = cross       ? p->w_maps_cross[(size_t)blk * 2 + (kind_in - TC_GEMM_XQ)]
+                            : text_pass ? p->w_maps_text[(size_t)blk * 4 + kind_in]
+                                        : p->w_maps[(size_t)blk * 4 + kind_in];
+    // the cross-attention's projections run the kernels of the projections they resemble
+    const TcGemmKind kind = kind_in == TC_GEMM_XQ ? TC_GEMM_QKV : kind_in == TC_GEMM_XO ? TC_GEMM_OUT : kind_in;
     const int32_t* m_list = text_pass ? (s.pair_bn ? p->text_list256 : p->text_list128) : nullptr;
     Control* c = const_cast<Control*>(ctl);
     const int grid = p->sm_count;

@@ -38,11 +38,11 @@ def _check_step(wl, y, kv, y_ref, kv_ref, y_before, kv_before, idx):
             assert np.array_equal(got[~a2], old[~a2])
 
 
-def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=None, text_seed=None):
+def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=None, text_seed=None, n_ctx=None):
     """Warm-up (all active) on the previous step's tokens, then gated steps; both sides start
     from the same zero caches and carry their own state forward.  `variants`: inputs of the block variants
     (QK-RMSNorm weights, rotary tables) handed to both sides.  `text_seed`: dual stream, the always-active tokens
-    (label R) get a second weight set drawn from this seed."""
+    (label R) get a second weight set drawn from this seed.  `n_ctx`: cross-attention to a context of that many tokens."""
     L = wl.L if n_blocks is None else n_blocks
     labels = labels_for(wl, seed)
     w = gen.block_weights(wl, seed, n_blocks=L)
@@ -71,6 +71,12 @@ def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=
         fd.fd_set_block_variants(ctx, **kw)
     if text_seed is not None:
         variants = dict(variants or {}, text=text)
+    if n_ctx is not None:
+        cross = gen.cross_attention(wl, seed, n_ctx, n_blocks=L)
+        cross["w_q"] *= np.float32(qk_gain)
+        cross["b_q"] *= np.float32(qk_gain)
+        fd.fd_set_cross_attention(ctx, {k: dev(v, dt) for k, v in cross.items()})
+        variants = dict(variants or {}, cross=cross)
     B, N, H = wl.B, wl.N, wl.H
     kv_ref = np.zeros((L, B, 2, N, H), np.float32)
     y_ref = np.zeros((B, N, H), np.float32)
