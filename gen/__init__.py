@@ -9,5 +9,5 @@ identical arrays without sharing any code of the method itself.
 from .workloads import (  # noqa: F401
     Workload, WORKLOADS, workload, round_bf16, block_weights, step_inputs,
     uniform_labels, latent_pair, saliency_map, region_mask, mask_schedule,
-    region_sigma, request_fractions, sampler_weights, latent_sequence, block_variants, cross_attention,
+    region_sigma, request_fractions, sampler_weights, latent_sequence, block_variants, cross_attention, fp8_operands,
 )

@@ -385,3 +385,27 @@ def cross_attention(wl: Workload, seed: int, n_ctx: int, n_blocks: Optional[int]
            for k, s in (("w_q", (L, H, H)), ("b_q", (L, H)), ("w_o", (L, H, H)), ("b_o", (L, H)))}
     out["ctx_kv"] = _store(wl, g.standard_normal((L, wl.B, 2, n_ctx, H), dtype=np.float32) * np.float32(0.5))
     return out
+
+
+def fp8_operands(wl: Workload, w: Dict[str, np.ndarray], seed: int, n_blocks: Optional[int] = None) -> Dict[str, np.ndarray]:
+    """Inputs of the FP8-operand variant from a weight set: the QKV, fc1 and fc2 matrices quantised per output row to
+    E4M3 (scale s = max|row| / 448, fp32; codes by the library's float8 cast of row / s), and per-block activation
+    scales drawn per tensor (the normalised inputs of QKV and fc1 ~U[0.02, 0.04], the GELU output ~U[0.01, 0.02]; an
+    activation beyond 448 scales saturates on both sides alike).  Returns, per matrix, the codes c_* (uint8), their
+    values w_* (float32) and the scales s_*, and a_scale [L, 3]."""
+    import torch
+    L = wl.L if n_blocks is None else n_blocks
+    out: Dict[str, np.ndarray] = {}
+    for name in ("qkv", "fc1", "fc2"):
+        W = torch.from_numpy(np.ascontiguousarray(w["w_" + name][:L], dtype=np.float32))
+        s = (W.abs().amax(dim=-1) / 448.0).clamp_min(1e-12)
+        q = (W / s[..., None]).to(torch.float8_e4m3fn)
+        out["c_" + name] = q.view(torch.uint8).numpy().copy()
+        out["w_" + name] = q.to(torch.float32).numpy().copy()
+        out["s_" + name] = s.numpy().astype(np.float32)
+    g = _rng(seed, 1515)
+    a = np.empty((L, 3), np.float32)
+    a[:, 0:2] = g.uniform(0.02, 0.04, (L, 2))
+    a[:, 2] = g.uniform(0.01, 0.02, L)
+    out["a_scale"] = a
+    return out

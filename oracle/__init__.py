@@ -42,6 +42,11 @@ class _Cross(ctypes.Structure):           # fdo_cross / fdo_dense_cross
     _fields_ = [(n, ctypes.c_void_p) for n in ("w_q", "b_q", "w_o", "b_o", "ctx_kv")] + [("T", ctypes.c_int)]
 
 
+class _Fp8(ctypes.Structure):             # fdo_fp8 / fdo_dense_fp8
+    _fields_ = [(n, ctypes.c_void_p) for n in ("w_qkv", "s_qkv", "w_fc1", "s_fc1", "w_fc2", "s_fc2")] + \
+               [(n, ctypes.c_float) for n in ("a_qkv", "a_fc1", "a_fc2")]
+
+
 _lib = None
 _f = ctypes.POINTER(ctypes.c_float)
 _i = ctypes.POINTER(ctypes.c_int32)
@@ -60,6 +65,11 @@ def _load():
         _lib.fdo_dense_block_d.restype = ctypes.c_int
         _lib.fdo_regional_block_x.restype = ctypes.c_int
         _lib.fdo_dense_block_x.restype = ctypes.c_int
+        _lib.fdo_regional_block_q.restype = ctypes.c_int
+        _lib.fdo_dense_block_q.restype = ctypes.c_int
+        _lib.fdo_regional_e4m3.restype = None
+        _lib.fdo_dense_e4m3.restype = None
+        _lib.fdo_regional_linear_fp8.restype = None
     return _lib
 
 
@@ -111,6 +121,36 @@ def _cross_arg(v, l: int, B: int, H: int, keep: list):
     return ctypes.byref(st)
 
 
+def _fp8_arg(v, l: int, keep: list):
+    """fdo_fp8 of block ``l`` from variants["fp8"] = {w_qkv [L,3H,H], s_qkv [L,3H], w_fc1, s_fc1, w_fc2, s_fc2: the E4M3
+    values of the quantised weights and their per-row scales; a_scale [L,3]: activation scales of QKV, fc1, fc2}."""
+    f = v.get("fp8")
+    if f is None:
+        return None
+    a = np.asarray(f["a_scale"], np.float32)[l]
+    st = _Fp8(*(_addr(f[k][l], keep) for k in ("w_qkv", "s_qkv", "w_fc1", "s_fc1", "w_fc2", "s_fc2")),
+              float(a[0]), float(a[1]), float(a[2]))
+    keep.append(st)
+    return ctypes.byref(st)
+
+
+def e4m3(x: np.ndarray, program: str = "regional") -> np.ndarray:
+    """Nearest E4M3 value of every element (ties to even, saturating at 448), by either C program's quantiser."""
+    x = _c(x)
+    y = np.empty_like(x)
+    getattr(_load(), "fdo_regional_e4m3" if program == "regional" else "fdo_dense_e4m3")(int(x.size), _fp(x), _fp(y))
+    return y
+
+
+def linear_fp8(x: np.ndarray, a_scale: float, w8: np.ndarray, w_scale: np.ndarray, bias: np.ndarray) -> np.ndarray:
+    """One row through the FP8 projection of the regional program: x [K], w8 [O,K] E4M3 values, w_scale, bias [O]."""
+    x, w8, w_scale, bias = _c(x), _c(w8), _c(w_scale), _c(bias)
+    y = np.empty(w8.shape[0], np.float32)
+    _load().fdo_regional_linear_fp8(_fp(x), ctypes.c_float(a_scale), _fp(w8), _fp(w_scale), _fp(bias), int(w8.shape[1]),
+                                    int(w8.shape[0]), _fp(y))
+    return y
+
+
 def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w: Dict[str, np.ndarray],
                    l: int, kv_l: np.ndarray, heads: int, ln_eps: float = 1e-6,
                    finish: Optional[np.ndarray] = None, variants=None, mod_text: Optional[np.ndarray] = None,
@@ -145,11 +185,11 @@ def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w:
     rc_, rs_ = _addr(v.get("rope_cos"), keep), _addr(v.get("rope_sin"), keep)
     if rc_ is not None:
         assert keep[-2].shape == (N, dh // 2)
-    rc = _load().fdo_regional_block_x(
+    rc = _load().fdo_regional_block_q(
         B, N, H, heads, dh, M, A, _ip(np.ascontiguousarray(active_idx, np.int32)), ctypes.byref(img), txt,
         None if tt is None else tt.ctypes.data_as(ctypes.c_void_p), ctypes.c_float(ln_eps), _fp(_c(u_in)), _fp(u_out), _fp(kv_l),
         0 if fin is None else int(fin.size), _ip(fin), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))),
-        ctypes.c_void_p(rc_), ctypes.c_void_p(rs_), _cross_arg(v, l, B, H, keep))
+        ctypes.c_void_p(rc_), ctypes.c_void_p(rs_), _cross_arg(v, l, B, H, keep), _fp8_arg(v, l, keep))
     assert rc == 0
     return u_out
 
@@ -226,10 +266,10 @@ def dense_block(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], l: in
     rc_, rs_ = _addr(v.get("rope_cos"), keep), _addr(v.get("rope_sin"), keep)
     if rc_ is not None:
         assert keep[-2].shape == (N, dh // 2)
-    rc = _load().fdo_dense_block_x(
+    rc = _load().fdo_dense_block_q(
         B, N, H, heads, dh, M, Hc, _fp(_c(cond)), ctypes.byref(wi), wt, n_text, ctypes.c_float(ln_eps), _fp(_c(x)), _fp(x_out),
         _fp(kv), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))), ctypes.c_void_p(rc_), ctypes.c_void_p(rs_),
-        _cross_arg(v, l, B, H, keep))
+        _cross_arg(v, l, B, H, keep), _fp8_arg(v, l, keep))
     assert rc == 0
     return x_out, kv
 

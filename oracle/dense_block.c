@@ -28,6 +28,57 @@ static void matmul_nt_bias(const float* X, const float* W, const float* bias, si
         }
 }
 
+/*
+ * FP8 operands (not in the paper; this build's reading).  A projection with both operands in the 8-bit floating-point
+ * format E4M3 (sign, 4 exponent bits biased by 7, 3 mantissa bits, gradual underflow below 2^-6, largest magnitude
+ * 448, no infinity): the weight matrix arrives quantised, W[o,:] = s_w[o] * W8[o,:]; the activation matrix is divided
+ * by its scale a (multiplied by the fp32 reciprocal) and rounded to the nearest E4M3 value, ties to the even mantissa,
+ * magnitudes past 448 clamped; Y[r,o] = (sum_k X8[r,k] W8[o,k]) * (a * s_w[o]) + bias[o] with an exact sum.
+ * The rounding is done on the bit pattern of the fp32 value.
+ */
+static float to_e4m3_value(float t) {
+    uint32_t u;
+    memcpy(&u, &t, 4);
+    const uint32_t sign = u & 0x80000000u;
+    uint32_t mag = u & 0x7fffffffu;
+    if (mag > 0x7f800000u) return t;                      /* NaN stays NaN */
+    if (mag >= 0x43e00000u) {
+        mag = 0x43e00000u;                                /* 448 */
+    } else if (mag < 0x3c800000u) {                       /* below 2^-6: multiples of 2^-9 */
+        float a;
+        memcpy(&a, &mag, 4);
+        volatile float r = a + 16384.0f;                  /* fp32 spacing at 2^14 is 2^-9: the add rounds to the grid, ties to even */
+        r = r - 16384.0f;
+        a = r;
+        memcpy(&mag, &a, 4);
+    } else {                                              /* keep three mantissa bits, round the other twenty */
+        mag += 0x7ffffu + ((mag >> 20) & 1u);
+        mag &= 0xfff00000u;
+    }
+    u = sign | mag;
+    memcpy(&t, &u, 4);
+    return t;
+}
+
+static int matmul_nt_bias_fp8(const float* X, float a_scale, const float* W8, const float* w_scale, const float* bias,
+                              size_t rows, int K, int O, float* Y) {
+    float* X8 = (float*)malloc(sizeof(float) * rows * (size_t)K);
+    if (!X8) return 1;
+    const float inv = 1.0f / a_scale;
+    for (size_t e = 0; e < rows * (size_t)K; ++e) X8[e] = to_e4m3_value(X[e] * inv);
+#pragma omp parallel for schedule(static)
+    for (size_t r = 0; r < rows; ++r)
+        for (int o = 0; o < O; ++o) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k) acc += (double)X8[r * K + k] * (double)W8[(size_t)o * K + k];
+            Y[r * O + o] = (float)(acc * ((double)a_scale * (double)w_scale[o]) + (double)bias[o]);
+        }
+    free(X8);
+    return 0;
+}
+
+void fdo_dense_e4m3(int n, const float* x, float* y) { for (int i = 0; i < n; ++i) y[i] = to_e4m3_value(x[i]); }
+
 /* rows of one request: LayerNorm without affine, then * (1 + scale) + shift */
 static void layernorm_modulate(const float* X, size_t rows, int H, const float* shift,
                                const float* scale, float eps, float* Y) {
@@ -151,10 +202,24 @@ typedef struct {
     int T;
 } fdo_dense_cross;
 
+/* fdo_dense_block_q: the QKV, fc1 and fc2 projections with FP8 operands (single stream only; q8 = NULL: off) */
+typedef struct {
+    const float *w_qkv, *s_qkv, *w_fc1, *s_fc1, *w_fc2, *s_fc2;   /* E4M3 weight values and per-row scales */
+    float a_qkv, a_fc1, a_fc2;                                    /* activation scales */
+} fdo_dense_fp8;
+
+int fdo_dense_block_q(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+                      const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
+                      const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
+                      const float* rope_sin, const fdo_dense_cross* cross, const fdo_dense_fp8* q8);
+
 int fdo_dense_block_x(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
                       const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
-                      const float* rope_sin, const fdo_dense_cross* cross);
+                      const float* rope_sin, const fdo_dense_cross* cross) {
+    return fdo_dense_block_q(B, N, H, heads, dh, M, Hc, cond, wi, wt, n_text, ln_eps, x_in, x_out, kv_out, qk_eps, rope_cos,
+                             rope_sin, cross, NULL);
+}
 
 int fdo_dense_block_d(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
@@ -184,11 +249,12 @@ int fdo_dense_block(int B, int N, int H, int heads, int dh, int M, int Hc, const
                              b_fc2, ln_eps, x_in, x_out, kv_out, NULL, NULL, 0.f, NULL, NULL);
 }
 
-int fdo_dense_block_x(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
+int fdo_dense_block_q(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
                       const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
-                      const float* rope_sin, const fdo_dense_cross* cross) {
+                      const float* rope_sin, const fdo_dense_cross* cross, const fdo_dense_fp8* q8) {
     if (heads * dh != H) return 2;
+    if (q8 && wt) return 5;
     if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
     if (!wt) n_text = 0;
     if (n_text < 0 || n_text > N) return 4;
@@ -226,7 +292,11 @@ int fdo_dense_block_x(int B, int N, int H, int heads, int dh, int M, int Hc, con
             if (!n) continue;
             const float* md = mod + (size_t)s * 6 * H;
             layernorm_modulate(X + lo * H, n, H, md, md + H, ln_eps, xh + lo * H);
-            matmul_nt_bias(xh + lo * H, ws[s]->w_qkv, ws[s]->b_qkv, n, H, 3 * H, qkv + lo * 3 * H);
+            if (q8) {
+                if (matmul_nt_bias_fp8(xh + lo * H, q8->a_qkv, q8->w_qkv, q8->s_qkv, ws[s]->b_qkv, n, H, 3 * H, qkv + lo * 3 * H)) { rc = 1; goto done; }
+            } else {
+                matmul_nt_bias(xh + lo * H, ws[s]->w_qkv, ws[s]->b_qkv, n, H, 3 * H, qkv + lo * 3 * H);
+            }
         }
         for (int t = 0; t < N; ++t) {
             memcpy(Q + (size_t)t * H, qkv + (size_t)t * 3 * H, sizeof(float) * (size_t)H);
@@ -274,12 +344,20 @@ int fdo_dense_block_x(int B, int N, int H, int heads, int dh, int M, int Hc, con
             if (!n) continue;
             const float* md = mod + (size_t)s * 6 * H;
             layernorm_modulate(res + lo * H, n, H, md + 3 * H, md + 4 * H, ln_eps, xh + lo * H);
-            matmul_nt_bias(xh + lo * H, ws[s]->w_fc1, ws[s]->b_fc1, n, H, M, hid + lo * M);
+            if (q8) {
+                if (matmul_nt_bias_fp8(xh + lo * H, q8->a_fc1, q8->w_fc1, q8->s_fc1, ws[s]->b_fc1, n, H, M, hid + lo * M)) { rc = 1; goto done; }
+            } else {
+                matmul_nt_bias(xh + lo * H, ws[s]->w_fc1, ws[s]->b_fc1, n, H, M, hid + lo * M);
+            }
             for (size_t e = lo * M; e < (lo + n) * M; ++e) {
                 const double a = (double)hid[e];
                 hid[e] = (float)(0.5 * a * (1.0 + tanh(0.79788456080286535588 * (a + 0.044715 * a * a * a))));
             }
-            matmul_nt_bias(hid + lo * M, ws[s]->w_fc2, ws[s]->b_fc2, n, M, H, proj + lo * H);
+            if (q8) {
+                if (matmul_nt_bias_fp8(hid + lo * M, q8->a_fc2, q8->w_fc2, q8->s_fc2, ws[s]->b_fc2, n, M, H, proj + lo * H)) { rc = 1; goto done; }
+            } else {
+                matmul_nt_bias(hid + lo * M, ws[s]->w_fc2, ws[s]->b_fc2, n, M, H, proj + lo * H);
+            }
             const float* gate_m = md + 5 * H;
             for (size_t e = lo * H; e < (lo + n) * H; ++e)
                 Y[e] = (float)((double)res[e] + (double)gate_m[e % H] * (double)proj[e]);

@@ -37,6 +37,53 @@ static void row_linear(const float* x, const float* w, const float* bias, int K,
     }
 }
 
+/*
+ * FP8 operands (not in the paper: this build's reading of 8-bit floating-point inference as commonly deployed for
+ * the paper's models).  The QKV, fc1 and fc2 projections take both operands in the OCP E4M3 format (1 sign, 4
+ * exponent bits with bias 7, 3 mantissa bits; subnormals 2^-9 apart below 2^-6; largest finite value 448; no
+ * infinities): the weights were quantised beforehand, row o of W standing for s_w[o] * w8[o,:], and the activation row
+ * is quantised on the way in with one scale per tensor, x8[k] = E4M3(x[k] * (1 / a)), round to nearest even, values
+ * beyond +-448 saturating.  The products of the 8-bit values are summed exactly (fp64 here) and scaled back:
+ * y[o] = (sum_k x8[k] w8[o,k]) * (a * s_w[o]) + bias[o].  The out-projection and everything else stay as they are.
+ */
+static float e4m3_nearest(float t) {
+    if (t != t) return t;
+    const float a = fabsf(t);
+    if (a >= 448.0f) return copysignf(448.0f, t);
+    float step;
+    if (a < 0.015625f) {
+        step = 0.001953125f;                          /* below 2^-6: the subnormal grid */
+    } else {
+        int e;
+        frexpf(a, &e);                                /* a in [2^(e-1), 2^e): eight steps per binade */
+        step = ldexpf(1.0f, e - 4);
+    }
+    return copysignf(rintf(a / step) * step, t);     /* a / step is exact; rintf rounds ties to even */
+}
+
+/* the 8-bit form of row_linear; xq [K] is scratch for the quantised row */
+static void row_linear_fp8(const float* x, float a_scale, const float* w8, const float* w_scale, const float* bias,
+                           int K, int O, float* xq, float* y) {
+    const float inv = 1.0f / a_scale;
+    for (int k = 0; k < K; ++k) xq[k] = e4m3_nearest(x[k] * inv);
+    for (int o = 0; o < O; ++o) {
+        const float* wr = w8 + (size_t)o * K;
+        double acc = 0.0;
+        for (int k = 0; k < K; ++k) acc += (double)xq[k] * (double)wr[k];
+        y[o] = (float)(acc * ((double)a_scale * (double)w_scale[o]) + (double)bias[o]);
+    }
+}
+
+/* quantiser and projection on their own, for the pins */
+void fdo_regional_e4m3(int n, const float* x, float* y) { for (int i = 0; i < n; ++i) y[i] = e4m3_nearest(x[i]); }
+void fdo_regional_linear_fp8(const float* x, float a_scale, const float* w8, const float* w_scale, const float* bias,
+                             int K, int O, float* y) {
+    float* xq = (float*)malloc(sizeof(float) * (size_t)K);
+    if (!xq) return;
+    row_linear_fp8(x, a_scale, w8, w_scale, bias, K, O, xq, y);
+    free(xq);
+}
+
 /* LayerNorm (biased variance, no affine) followed by (1+scale), shift */
 static void row_ln_modulate(const float* u, const float* shift, const float* scale, int H,
                             float ln_eps, float* out) {
@@ -149,10 +196,27 @@ typedef struct {
     int T;
 } fdo_cross;
 
+/* FP8 operands of the QKV, fc1 and fc2 projections (single stream only); fp8 = NULL: off */
+typedef struct {
+    const float *w_qkv, *s_qkv;             /* [3H,H] E4M3 values of the quantised weights, [3H] scales per output row */
+    const float *w_fc1, *s_fc1;             /* [M,H], [M] */
+    const float *w_fc2, *s_fc2;             /* [H,M], [H] */
+    float a_qkv, a_fc1, a_fc2;              /* activation scales: the inputs of QKV, fc1 and fc2 */
+} fdo_fp8;
+
+int fdo_regional_block_q(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
+                         const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
+                         float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
+                         float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross,
+                         const fdo_fp8* fp8);
+
 int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
                          const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
                          float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
-                         float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross);
+                         float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross) {
+    return fdo_regional_block_q(B, N, H, heads, dh, M, A, active_idx, img, txt, tok_text, ln_eps, u_in, u_out, kv, n_finish,
+                                finish, qk_eps, rope_cos, rope_sin, cross, NULL);
+}
 
 int fdo_regional_block_s(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
                          const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
@@ -184,12 +248,14 @@ int fdo_regional_block(int B, int N, int H, int heads, int dh, int M, int A,
                                 b_fc2, ln_eps, u_in, u_out, kv, n_finish, finish, NULL, NULL, 0.f, NULL, NULL);
 }
 
-int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
+int fdo_regional_block_q(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
                          const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
                          float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
-                         float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross) {
+                         float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross,
+                         const fdo_fp8* fp8) {
     if (heads * dh != H) return 2;
     if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
+    if (fp8 && txt) return 5;
     (void)B;
     float* q_all = (float*)malloc(sizeof(float) * (size_t)(A > 0 ? A : 1) * H);
     if (!q_all) return 1;
@@ -200,7 +266,8 @@ int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, c
     {
         float* uh = (float*)malloc(sizeof(float) * (size_t)H);
         float* qkv = (float*)malloc(sizeof(float) * (size_t)3 * H);
-        if (!uh || !qkv) {
+        float* xq = (float*)malloc(sizeof(float) * (size_t)H);
+        if (!uh || !qkv || !xq) {
 #pragma omp atomic write
             err = 1;
         } else {
@@ -210,14 +277,15 @@ int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, c
                 const fdo_stream* st = (txt && tok_text[active_idx[a]]) ? txt : img;      /* the token's stream */
                 const float* md = st->mod + (size_t)b * 6 * H;
                 row_ln_modulate(u_in + (size_t)a * H, md + 0 * H, md + 1 * H, H, ln_eps, uh);
-                row_linear(uh, st->w_qkv, st->b_qkv, H, 3 * H, qkv);
+                if (fp8) row_linear_fp8(uh, fp8->a_qkv, fp8->w_qkv, fp8->s_qkv, st->b_qkv, H, 3 * H, xq, qkv);
+                else row_linear(uh, st->w_qkv, st->b_qkv, H, 3 * H, qkv);
                 row_qk_variants(qkv, qkv + H, heads, dh, j, st->qn_w, st->kn_w, qk_eps, rope_cos, rope_sin);
                 memcpy(q_all + (size_t)a * H, qkv, sizeof(float) * (size_t)H);
                 memcpy(kv + (((size_t)b * 2 + 0) * N + j) * H, qkv + H, sizeof(float) * (size_t)H);
                 memcpy(kv + (((size_t)b * 2 + 1) * N + j) * H, qkv + 2 * H, sizeof(float) * (size_t)H);
             }
         }
-        free(uh); free(qkv);
+        free(uh); free(qkv); free(xq);
     }
     if (err) { free(q_all); return err; }
 
@@ -233,7 +301,8 @@ int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, c
         float* r1 = (float*)malloc(sizeof(float) * (size_t)H);
         float* mh = (float*)malloc(sizeof(float) * (size_t)H);
         float* g = (float*)malloc(sizeof(float) * (size_t)M);
-        if (!s || !oacc || !o || !proj || !r1 || !mh || !g) {
+        float* xq = (float*)malloc(sizeof(float) * (size_t)(M > H ? M : H));
+        if (!s || !oacc || !o || !proj || !r1 || !mh || !g || !xq) {
 #pragma omp atomic write
             err = 1;
         } else {
@@ -303,15 +372,17 @@ int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, c
                     for (int c = 0; c < H; ++c) r1[c] = (float)((double)r1[c] + (double)proj[c]);
                 }
                 row_ln_modulate(r1, md + 3 * H, md + 4 * H, H, ln_eps, mh);
-                row_linear(mh, st->w_fc1, st->b_fc1, H, M, g);
+                if (fp8) row_linear_fp8(mh, fp8->a_fc1, fp8->w_fc1, fp8->s_fc1, st->b_fc1, H, M, xq, g);
+                else row_linear(mh, st->w_fc1, st->b_fc1, H, M, g);
                 for (int c = 0; c < M; ++c) g[c] = (float)gelu_tanh_d((double)g[c]);
-                row_linear(g, st->w_fc2, st->b_fc2, M, H, proj);
+                if (fp8) row_linear_fp8(g, fp8->a_fc2, fp8->w_fc2, fp8->s_fc2, st->b_fc2, M, H, xq, proj);
+                else row_linear(g, st->w_fc2, st->b_fc2, M, H, proj);
                 float* out = u_out + (size_t)a * H;
                 for (int c = 0; c < H; ++c)
                     out[c] = (float)((double)r1[c] + (double)md[5 * H + c] * (double)proj[c]);
             }
         }
-        free(s); free(oacc); free(o); free(proj); free(r1); free(mh); free(g);
+        free(s); free(oacc); free(o); free(proj); free(r1); free(mh); free(g); free(xq);
     }
     free(q_all);
     return err;
