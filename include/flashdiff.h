@@ -230,6 +230,32 @@ typedef struct fd_cross_attention {
 fd_status fd_set_cross_attention(fd_ctx* ctx, const fd_cross_attention* cross);
 
 /*
+ * FP8 operands for the QKV, fc1 and fc2 projections (8-bit inference of the paper's models; the paper does not
+ * cover it, the convention is this library's).  Both operands of those three products are OCP E4M3 values (4
+ * exponent bits, bias 7, 3 mantissa bits, largest magnitude 448, no infinities):
+ *   weights     quantised by the caller, row o of W standing for s[o] * w8[o, :]
+ *               (w8_* DEVICE, E4M3 bytes, [L, 3H, H], [L, M, H], [L, H, M]; s_* DEVICE f32 [L, 3H], [L, M], [L, H]);
+ *   activations quantised by the library where they are produced (the two modulated LayerNorm outputs, the GELU
+ *               output) as E4M3(value * (1 / a)), round to nearest even, saturating, with one scale a per tensor and
+ *               block: a_scale, a HOST array [L, 3] (inputs of QKV, fc1, fc2), copied by this call;
+ *   result      (exact products, fp32 accumulation) * (a * s[o]) + bias, then as without FP8.
+ * The attention, the out-projection, the cross-attention and all vector work stay in bf16 / fp32.  Tensor-core
+ * engine with bf16 storage only, hidden and mlp_dim multiples of 192 or 256 (else FD_ERR_UNSUPPORTED); not
+ * together with a second stream (fd_set_text_stream).  Pointers 16-byte aligned, owned by the caller and alive
+ * while set.  NULL switches it off.  Host call, no launch; takes effect from the next step.
+ */
+typedef struct fd_fp8_operands {
+    const void* w8_qkv;
+    const float* s_qkv;
+    const void* w8_fc1;
+    const float* s_fc1;
+    const void* w8_fc2;
+    const float* s_fc2;
+    const float* a_scale;
+} fd_fp8_operands;
+fd_status fd_set_fp8_operands(fd_ctx* ctx, const fd_fp8_operands* fp8);
+
+/*
  * The Patch Gate on the paper's own signal (Sec. 4.2): the refinement importance of a patch is the block mean of
  * the self-attention matrix over the patch,  R_i = (1/|A_i|^2) sum_{u,v in A_i} SA[u,v],  and the gate weights are
  * the normalised changes  Delta_i = |R_i - Rbar_i|  (Rbar_i = the importance at the patch's last executed step;
@@ -363,6 +389,17 @@ enum {
     FD_PROF_CROSS = 12,   /* cross-attention: LayerNorm, query projection, attention, out-projection */
     FD_PROF_GROUPS = 13
 };
+/*
+ * Inspection of the step's intermediate buffers (they live in the caller's workspace): returns the DEVICE address and
+ * the size in bytes of one of them, as the last fd_regional_step left it (valid rows: the step's active rows, compact
+ * order).  For tests and debugging; nothing is launched and nothing is copied.
+ *   FD_BUF_ACT     [rows, H]   the last modulated-LayerNorm output: storage type, or E4M3 bytes with FP8 operands
+ *   FD_BUF_HIDDEN  [rows, M]   the last block's MLP hidden activations: storage type, or E4M3 bytes with FP8 operands
+ *   FD_BUF_RESID   [rows, H]   f32 residual stream after the last block (tensor-core engine)
+ */
+enum { FD_BUF_ACT = 0, FD_BUF_HIDDEN = 1, FD_BUF_RESID = 2 };
+fd_status fd_debug_buffer(fd_ctx* ctx, int which, void** device_ptr_out, size_t* bytes_out);
+
 fd_status fd_profile_enable(fd_ctx* ctx, int enable);
 fd_status fd_profile_read(fd_ctx* ctx, void* cuda_stream, float* ms_out, int32_t* kernels_out);
 

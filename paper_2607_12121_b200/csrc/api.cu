@@ -96,6 +96,8 @@ struct fd_ctx {
     fd_weights text_w{};       // second stream's weights (dual stream; w_qkv null: single stream)
     bool dual = false;
     fd_cross_attention cross{};   // cross-attention to a fixed context (w_q null: off)
+    fd_fp8_operands fp8{};        // FP8 operands of QKV, fc1, fc2 (w8_qkv null: off)
+    std::vector<float> fp8_a;     // [L, 3] activation scales (host copy)
     // optional per-kernel timing
     bool profiling = false;
     struct Span { cudaEvent_t a, b; int group, kernels; };
@@ -200,6 +202,8 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         return c->fail(FD_ERR_SHAPE, "B=%d differs from the cross-attention context's batch %d", B, xa.ctx_batch);
     const float* zeros = c->at<float>(l.consts);
     const float* ones = zeros + H;
+    const bool f8 = c->fp8.w8_qkv != nullptr;
+    if (f8 && dual) return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands and a second stream cannot be combined");
     const bool pdl = c->use_tc && c->tc && tc_plan_pdl(c->tc);
     for (int blk = 0; blk < L; ++blk) {
         const float* mod_b = mod + (size_t)blk * B * 6 * H;
@@ -214,9 +218,13 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         ep.group = -1;
         ep.text_mod_off = (int32_t)text_mod_off;
 
+        // FP8 operands: this block's activation scales (inputs of QKV, fc1, fc2)
+        const float a_qkv = f8 ? c->fp8_a[(size_t)blk * 3 + 0] : 0.f, a_fc1 = f8 ? c->fp8_a[(size_t)blk * 3 + 1] : 0.f;
+        const float a_fc2 = f8 ? c->fp8_a[(size_t)blk * 3 + 2] : 0.f;
         // gather (first block) or read the residual stream; LayerNorm; attention-branch modulation
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(blk == 0 ? x : nullptr, resid, resid, act, active_idx, mod_b + 0 * H,
-                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts));
+                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts,
+                                     f8 ? 1.0f / a_qkv : 0.f));
         // QKV projection; K and V rows go straight into the cache
         ep.q = q;
         ep.q_ld = l.q_ld;
@@ -228,7 +236,11 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         for (int pass = 0; pass < n_pass; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_qkv, c->text_w.b_qkv, (size_t)blk * 3 * H, pass);
-            if (c->use_tc)
+            if (f8) {
+                ep.col_scale = c->fp8.s_qkv + (size_t)blk * 3 * H;
+                ep.act_scale = a_qkv;
+                FD_TRY(FD_PROF_GEMM_QKV, tc_gemm_fp8(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));
+            } else if (c->use_tc)
                 FD_TRY(FD_PROF_GEMM_QKV, tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl, pass == 1));
             else
                 FD_TRY(FD_PROF_GEMM_QKV, launch_simt_gemm<T>(EPI_QKV, act, H, stream_ptr(c->w.w_qkv, c->text_w.w_qkv, (size_t)blk * 3 * H * H, pass),
@@ -305,13 +317,18 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         }
         // MLP branch
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, mod_b + 3 * H, mod_b + 4 * H, 6 * H, N,
-                                     H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts));
+                                     H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts, f8 ? 1.0f / a_fc1 : 0.f));
         ep.out = g;
         ep.out_ld = M;
         for (int pass = 0; pass < n_pass; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_fc1, c->text_w.b_fc1, (size_t)blk * M, pass);
-            if (c->use_tc)
+            if (f8) {
+                ep.col_scale = c->fp8.s_fc1 + (size_t)blk * M;
+                ep.act_scale = a_fc1;
+                ep.out_inv_scale = 1.0f / a_fc2;            // the hidden activations leave as E4M3 bytes, row stride M
+                FD_TRY(FD_PROF_GEMM_FC1, tc_gemm_fp8(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl));
+            } else if (c->use_tc)
                 FD_TRY(FD_PROF_GEMM_FC1, tc_gemm(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl, pass == 1));
             else
                 FD_TRY(FD_PROF_GEMM_FC1, launch_simt_gemm<T>(EPI_GELU, act, H, stream_ptr(c->w.w_fc1, c->text_w.w_fc1, (size_t)blk * M * H, pass), M,
@@ -322,7 +339,11 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         for (int pass = 0; pass < n_pass; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_fc2, c->text_w.b_fc2, (size_t)blk * H, pass);
-            if (c->use_tc)
+            if (f8) {
+                ep.col_scale = c->fp8.s_fc2 + (size_t)blk * H;
+                ep.act_scale = a_fc2;
+                FD_TRY(FD_PROF_GEMM_FC2, tc_gemm_fp8(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl));
+            } else if (c->use_tc)
                 FD_TRY(FD_PROF_GEMM_FC2, tc_gemm(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl, pass == 1));
             else
                 FD_TRY(FD_PROF_GEMM_FC2, launch_simt_gemm<T>(EPI_RESID, g, M, stream_ptr(c->w.w_fc2, c->text_w.w_fc2, (size_t)blk * H * M, pass), H,
@@ -690,6 +711,33 @@ fd_status fd_set_cross_attention(fd_ctx* c, const fd_cross_attention* x) {
     return FD_OK;
 }
 
+fd_status fd_set_fp8_operands(fd_ctx* c, const fd_fp8_operands* f) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!f) {
+        c->fp8 = fd_fp8_operands{};
+        c->fp8_a.clear();
+        if (c->tc) tc_plan_set_fp8(c->tc, nullptr, nullptr, nullptr, nullptr);
+        return FD_OK;
+    }
+    if (!c->use_tc || !c->tc) return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands need the tensor-core engine (bf16 storage)");
+    if (c->dual) return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands and a second stream cannot be combined");
+    const void* wp[6] = {f->w8_qkv, f->s_qkv, f->w8_fc1, f->s_fc1, f->w8_fc2, f->s_fc2};
+    for (const void* p : wp)
+        if (!p || !aligned16(p)) return c->fail(FD_ERR_INVALID_ARG, "FP8 operand pointer null or not 16-byte aligned");
+    if (!f->a_scale) return c->fail(FD_ERR_INVALID_ARG, "a_scale is null");
+    const size_t n = (size_t)c->cfg.n_blocks * 3;
+    for (size_t i = 0; i < n; ++i)
+        if (!(f->a_scale[i] > 0.f) || !(1.0f / f->a_scale[i] < 3.0e38f))
+            return c->fail(FD_ERR_INVALID_ARG, "activation scales must be positive and finite");
+    std::string err;
+    if (!tc_plan_set_fp8(c->tc, f->w8_qkv, f->w8_fc1, f->w8_fc2, &err))
+        return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands: %s", err.c_str());
+    c->fp8 = *f;
+    c->fp8_a.assign(f->a_scale, f->a_scale + n);
+    c->fp8.a_scale = nullptr;                 // the host array was copied
+    return FD_OK;
+}
+
 fd_status fd_poll_status(fd_ctx* c, void* cuda_stream) {
     if (!c) return FD_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -701,6 +749,20 @@ fd_status fd_poll_status(fd_ctx* c, void* cuda_stream) {
         cudaMemsetAsync(c->ctl(), 0, 2 * sizeof(int32_t), st);
         return c->fail(static_cast<fd_status>(h.status), "device-side check failed: code %d, detail %d", h.status,
                        h.detail);
+    }
+    return FD_OK;
+}
+
+fd_status fd_debug_buffer(fd_ctx* c, int which, void** device_ptr_out, size_t* bytes_out) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    if (!device_ptr_out || !bytes_out) return c->fail(FD_ERR_INVALID_ARG, "null output pointer");
+    const Layout& l = c->lay;
+    const size_t es = c->cfg.dtype == FD_BF16 ? 2 : 4;
+    switch (which) {
+        case FD_BUF_ACT: *device_ptr_out = c->ws + l.act; *bytes_out = (size_t)l.Mcap * c->cfg.hidden * es; break;
+        case FD_BUF_HIDDEN: *device_ptr_out = c->ws + l.g; *bytes_out = (size_t)l.Mcap * c->cfg.mlp_dim * es; break;
+        case FD_BUF_RESID: *device_ptr_out = c->ws + l.resid; *bytes_out = (size_t)l.Mcap * c->cfg.hidden * sizeof(float); break;
+        default: return c->fail(FD_ERR_INVALID_ARG, "unknown buffer %d", which);
     }
     return FD_OK;
 }

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -40,6 +41,13 @@ template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v
 template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// four values to E4M3 bytes (round to nearest even, saturating at 448), first value in the low byte
+__device__ __forceinline__ uint32_t pack4_e4m3(float a, float b, float c, float d) {
+    const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
+    const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(c, d), __NV_SATFINITE, __NV_E4M3);
+    return lo | (hi << 16);
+}
 
 __device__ __forceinline__ float gelu_tanh(float a) {
     const float c = 0.7978845608028654f;
@@ -87,6 +95,11 @@ struct EpiParams {
     int32_t group;             // -1: every row; 0: rows of the first stream only; 1: rows of the second stream only
     int32_t text_mod_off;      // offset (floats) from a request's adaLN vectors to those of the second stream
     int32_t ungated;           // EPI_RESID: `gate` is one [H] vector for every row (cross-attention passes ones)
+    // FP8 operands (the kernels built for them): the accumulator is scaled by col_scale[col] * act_scale before the
+    // bias; EPI_GELU then writes `out` as E4M3 bytes of value * out_inv_scale (row stride out_ld bytes)
+    const float* col_scale;    // [n_out] f32
+    float act_scale;
+    float out_inv_scale;
 };
 
 // Per-row choice of the second stream's adaLN vectors in the row kernels (labels == nullptr: single stream).
@@ -135,7 +148,8 @@ template <typename T>
 cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
                                const int32_t* active_idx, const float* shift, const float* scale,
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
-                               cudaStream_t st, int* n_launch, bool pdl, TextSel ts = TextSel{nullptr, 0, 0});
+                               cudaStream_t st, int* n_launch, bool pdl, TextSel ts = TextSel{nullptr, 0, 0},
+                               float fp8_inv_scale = 0.f);   // > 0 (bf16 engine): `out` receives E4M3 bytes of value * this
 
 // qk_variants.cu: QK-RMSNorm and rotary embedding on the fresh Q rows and the K rows just written to the cache
 template <typename T>

@@ -107,6 +107,8 @@ struct RowInfo {
 
 // EPI_RESID: 32 fp32 accumulator columns per row; resid += gate * (acc + bias); the last block also
 // scatters the row into y.
+// F8: the accumulator holds products of 8-bit operands and is scaled by col_scale[col] * act_scale before the bias.
+template <bool F8>
 __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
                                                      int col0, const uint32_t* acc, const RowInfo& ri) {
     using T = __nv_bfloat16;
@@ -117,6 +119,21 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
     const int col = col0 + u * 4;
     float bias[4];
     load4<T>(reinterpret_cast<const T*>(ep.bias) + col, bias);
+    float4 cs = make_float4(1.f, 1.f, 1.f, 1.f);
+    if constexpr (F8) {
+        cs = __ldg(reinterpret_cast<const float4*>(ep.col_scale + col));
+        cs.x *= ep.act_scale; cs.y *= ep.act_scale; cs.z *= ep.act_scale; cs.w *= ep.act_scale;
+    }
+    // acc (+ scaling) + bias of one staged unit
+    auto lin = [&](const uint4& a, float& x, float& y, float& z, float& w) {
+        if constexpr (F8) {
+            x = fmaf(__uint_as_float(a.x), cs.x, bias[0]); y = fmaf(__uint_as_float(a.y), cs.y, bias[1]);
+            z = fmaf(__uint_as_float(a.z), cs.z, bias[2]); w = fmaf(__uint_as_float(a.w), cs.w, bias[3]);
+        } else {
+            x = __uint_as_float(a.x) + bias[0]; y = __uint_as_float(a.y) + bias[1];
+            z = __uint_as_float(a.z) + bias[2]; w = __uint_as_float(a.w) + bias[3];
+        }
+    };
     float* rp = ep.resid + (size_t)(row_base + rsub) * ep.H + col;      // rows rsub, rsub + 4, ...
     const size_t rstride = (size_t)4 * ep.H;
     const float* gp = ep.gate + col;
@@ -137,8 +154,9 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
             const int r = 4 * i + rsub;
             if ((ri.valid >> r) & 1u) {
                 const uint4 a = *unit_ptr(stage, r, u);
-                const float x = gv[i].x * (__uint_as_float(a.x) + bias[0]), y = gv[i].y * (__uint_as_float(a.y) + bias[1]);
-                const float z = gv[i].z * (__uint_as_float(a.z) + bias[2]), w = gv[i].w * (__uint_as_float(a.w) + bias[3]);
+                float x, y, z, w;
+                lin(a, x, y, z, w);
+                x *= gv[i].x; y *= gv[i].y; z *= gv[i].z; w *= gv[i].w;
                 asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(rp + i * rstride), "f"(x), "f"(y), "f"(z), "f"(w)
                              : "memory");
             }
@@ -164,8 +182,10 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
         if ((ri.valid >> r) & 1u) {
             const uint4 a = *unit_ptr(stage, r, u);
             float4 v = rv[i];
-            v.x = fmaf(gv[i].x, __uint_as_float(a.x) + bias[0], v.x); v.y = fmaf(gv[i].y, __uint_as_float(a.y) + bias[1], v.y);
-            v.z = fmaf(gv[i].z, __uint_as_float(a.z) + bias[2], v.z); v.w = fmaf(gv[i].w, __uint_as_float(a.w) + bias[3], v.w);
+            float x, y, z, w;
+            lin(a, x, y, z, w);
+            v.x = fmaf(gv[i].x, x, v.x); v.y = fmaf(gv[i].y, y, v.y);
+            v.z = fmaf(gv[i].z, z, v.z); v.w = fmaf(gv[i].w, w, v.w);
             *reinterpret_cast<float4*>(rp + i * rstride) = v;
             store4<T>(yb + (((size_t)yhi << 32) | ylo) + col, v.x, v.y, v.z, v.w);
         }
@@ -177,6 +197,7 @@ __device__ __forceinline__ void epilogue_resid_chunk(const EpiParams& ep, uint8_
 // plain fp32 rows and one bulk tensor reduction adds the tile onto the residual stream.  The SM's load/store path
 // issues per-thread reductions at about 9 bytes per clock, which made this epilogue as long as the main loop of a
 // K = 1536 tile; the bulk form hands whole 128-byte rows to the L2.
+template <bool F8>
 __device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
                                                          int col0, const uint32_t* acc, const RowInfo& ri,
                                                          const CUtensorMap* tm_r) {
@@ -191,6 +212,11 @@ __device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, ui
     float bias[4];
     load4<T>(reinterpret_cast<const T*>(ep.bias) + col, bias);
     const float* gp = ep.gate + col;
+    float4 cs = make_float4(1.f, 1.f, 1.f, 1.f);
+    if constexpr (F8) {
+        cs = __ldg(reinterpret_cast<const float4*>(ep.col_scale + col));
+        cs.x *= ep.act_scale; cs.y *= ep.act_scale; cs.z *= ep.act_scale; cs.w *= ep.act_scale;
+    }
     float4 gv[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -205,8 +231,13 @@ __device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, ui
         const uint4 a = *unit_ptr(stage, r, u);
         __syncwarp();
         float4 v;
-        v.x = gv[i].x * (__uint_as_float(a.x) + bias[0]); v.y = gv[i].y * (__uint_as_float(a.y) + bias[1]);
-        v.z = gv[i].z * (__uint_as_float(a.z) + bias[2]); v.w = gv[i].w * (__uint_as_float(a.w) + bias[3]);
+        if constexpr (F8) {
+            v.x = gv[i].x * fmaf(__uint_as_float(a.x), cs.x, bias[0]); v.y = gv[i].y * fmaf(__uint_as_float(a.y), cs.y, bias[1]);
+            v.z = gv[i].z * fmaf(__uint_as_float(a.z), cs.z, bias[2]); v.w = gv[i].w * fmaf(__uint_as_float(a.w), cs.w, bias[3]);
+        } else {
+            v.x = gv[i].x * (__uint_as_float(a.x) + bias[0]); v.y = gv[i].y * (__uint_as_float(a.y) + bias[1]);
+            v.z = gv[i].z * (__uint_as_float(a.z) + bias[2]); v.w = gv[i].w * (__uint_as_float(a.w) + bias[3]);
+        }
         *reinterpret_cast<float4*>(stage + r * 128 + u * 16) = v;
     }
     ptx::fence_proxy_async_smem();
@@ -215,29 +246,64 @@ __device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, ui
 }
 
 // EPI_QKV / EPI_GELU: 64 fp32 accumulator columns per row, bf16 outputs (8 columns per 16-byte unit).
-template <int KIND>
+// F8: the accumulator holds products of 8-bit operands and is scaled by col_scale[col] * act_scale before the bias;
+// EPI_GELU then writes its 64 values per row as 64 E4M3 bytes of value * out_inv_scale (the fc2 operand).
+template <int KIND, bool F8>
 __device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
                                                     int col0, const uint32_t* acc, const RowInfo& ri) {
     using T = __nv_bfloat16;
     const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ep.bias) + col0);
+    const float4* sp = reinterpret_cast<const float4*>(ep.col_scale + col0);
+    uint32_t q8[4];                                            // F8 GELU: four values per word, a 16-byte unit per two u
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
         const uint4 b = __ldg(bp + u);
         const uint32_t w[4] = {b.x, b.y, b.z, b.w};
         float v[8];
+        if constexpr (F8) {
+            const float4 s0 = __ldg(sp + 2 * u), s1 = __ldg(sp + 2 * u + 1);
+            const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            v[2 * k] = __uint_as_float(acc[8 * u + 2 * k]) + __uint_as_float(w[k] << 16);
-            v[2 * k + 1] = __uint_as_float(acc[8 * u + 2 * k + 1]) + __uint_as_float(w[k] & 0xffff0000u);
+            for (int k = 0; k < 4; ++k) {
+                v[2 * k] = fmaf(__uint_as_float(acc[8 * u + 2 * k]), sc[2 * k] * ep.act_scale, __uint_as_float(w[k] << 16));
+                v[2 * k + 1] = fmaf(__uint_as_float(acc[8 * u + 2 * k + 1]), sc[2 * k + 1] * ep.act_scale,
+                                    __uint_as_float(w[k] & 0xffff0000u));
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                v[2 * k] = __uint_as_float(acc[8 * u + 2 * k]) + __uint_as_float(w[k] << 16);
+                v[2 * k + 1] = __uint_as_float(acc[8 * u + 2 * k + 1]) + __uint_as_float(w[k] & 0xffff0000u);
+            }
         }
         if constexpr (KIND == EPI_GELU) {
 #pragma unroll
             for (int k = 0; k < 8; ++k) v[k] = gelu_tanh_fast(v[k]);
         }
-        *unit_ptr(stage, lane, u) = make_uint4(pack2_bf16(v[0], v[1]), pack2_bf16(v[2], v[3]), pack2_bf16(v[4], v[5]),
-                                               pack2_bf16(v[6], v[7]));
+        if constexpr (KIND == EPI_GELU && F8) {
+            const float qs = ep.out_inv_scale;
+            q8[2 * (u & 1)] = pack4_e4m3(v[0] * qs, v[1] * qs, v[2] * qs, v[3] * qs);
+            q8[2 * (u & 1) + 1] = pack4_e4m3(v[4] * qs, v[5] * qs, v[6] * qs, v[7] * qs);
+            if (u & 1) *unit_ptr(stage, lane, u >> 1) = make_uint4(q8[0], q8[1], q8[2], q8[3]);
+        } else {
+            *unit_ptr(stage, lane, u) = make_uint4(pack2_bf16(v[0], v[1]), pack2_bf16(v[2], v[3]), pack2_bf16(v[4], v[5]),
+                                                   pack2_bf16(v[6], v[7]));
+        }
     }
     __syncwarp();
+    if constexpr (KIND == EPI_GELU && F8) {
+        // lane t: unit t % 4 (16 columns) of rows 8 i + t / 4: every store instruction covers eight 64-byte row segments
+        const int u4 = lane & 3, rs8 = lane >> 2;
+        uint8_t* ob = reinterpret_cast<uint8_t*>(ep.out) + (size_t)(row_base + rs8) * ep.out_ld + col0 + u4 * 16;
+        const size_t ostride = (size_t)8 * ep.out_ld;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = 8 * i + rs8;
+            if ((ri.valid >> r) & 1u) *reinterpret_cast<uint4*>(ob + i * ostride) = *unit_ptr(stage, r, u4);
+        }
+        __syncwarp();
+        return;
+    }
     const int u = lane & 7, rsub = lane >> 3;
     const int col = col0 + u * 8;
     if constexpr (KIND == EPI_GELU) {
@@ -311,7 +377,7 @@ __device__ __forceinline__ RowInfo epilogue_row_info(const EpiParams& ep, int la
 }
 
 // one warp's share of a tile: rows [row_base, row_base + 32), columns [c_begin, c_end) of the accumulator at t_row
-template <int KIND>
+template <int KIND, bool F8 = false>
 __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stage, int lane, int row_base, int a_total,
                                               uint32_t t_row, int tile_col0, int c_begin, int c_end, const RowInfo& ri,
                                               const CUtensorMap* tm_r = nullptr) {
@@ -324,8 +390,8 @@ __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stag
             ptx::tmem_ld32(t_row + c0, r);
             ptx::tmem_wait_ld();
             if (live) {
-                if (tm_r && !ep.y) epilogue_resid_chunk_tma(ep, stage, lane, row_base, tile_col0 + c0, r, ri, tm_r);
-                else epilogue_resid_chunk(ep, stage, lane, row_base, tile_col0 + c0, r, ri);
+                if (tm_r && !ep.y) epilogue_resid_chunk_tma<F8>(ep, stage, lane, row_base, tile_col0 + c0, r, ri, tm_r);
+                else epilogue_resid_chunk<F8>(ep, stage, lane, row_base, tile_col0 + c0, r, ri);
             }
         }
     } else {
@@ -335,7 +401,7 @@ __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stag
             ptx::tmem_ld32(t_row + c0, r);
             ptx::tmem_ld32(t_row + c0 + 32, r + 32);
             ptx::tmem_wait_ld();
-            if (live) epilogue_bf16_chunk<KIND>(ep, stage, lane, row_base, tile_col0 + c0, r, ri);
+            if (live) epilogue_bf16_chunk<KIND, F8>(ep, stage, lane, row_base, tile_col0 + c0, r, ri);
         }
     }
 }

@@ -224,7 +224,7 @@ __global__ void __launch_bounds__(LN_THREADS, 8)
 ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
                    float* __restrict__ resid_out, T* __restrict__ out, const int32_t* __restrict__ active_idx,
                    const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
-                   int H, float ln_eps, const Control* __restrict__ ctl, TextSel ts) {
+                   int H, float ln_eps, const Control* __restrict__ ctl, TextSel ts, float fp8_inv) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     ptx::pdl_wait();                              // the rows come from the kernel launched just before
     const int a_total = ctl->a_total;
@@ -268,6 +268,11 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
             const float o3 = (v[3] - mean) * rstd * (1.f + s4.w) + h4.w;
             T* dst = out + r0 + c;
             if constexpr (sizeof(T) == 2) {
+                if (fp8_inv > 0.f) {          // FP8 operands: the projection reads this row as E4M3
+                    *reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(out) + r0 + c) =
+                        pack4_e4m3(o0 * fp8_inv, o1 * fp8_inv, o2 * fp8_inv, o3 * fp8_inv);
+                    continue;
+                }
                 const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
                 uint2 u;
                 u.x = *reinterpret_cast<const uint32_t*>(&p0);
@@ -290,7 +295,7 @@ __global__ void __launch_bounds__(LN_THREADS, 6)
 ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__ resid_in,
                        float* __restrict__ resid_out, T* __restrict__ out, const int32_t* __restrict__ active_idx,
                        const float* __restrict__ shift, const float* __restrict__ scale, int mod_stride, int N,
-                       float ln_eps, const Control* __restrict__ ctl, TextSel ts) {
+                       float ln_eps, const Control* __restrict__ ctl, TextSel ts, float fp8_inv) {
     constexpr int H = NV * 128;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     ptx::pdl_wait();                              // the rows come from the kernel launched just before
@@ -352,6 +357,11 @@ ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__
             const float o2 = (v[i][2] - mean) * rstd * (1.f + s4.z) + h4.z;
             const float o3 = (v[i][3] - mean) * rstd * (1.f + s4.w) + h4.w;
             if constexpr (sizeof(T) == 2) {
+                if (fp8_inv > 0.f) {          // FP8 operands: the projection reads this row as E4M3
+                    *reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(out) + (size_t)row * H + lane * 4 + i * 128) =
+                        pack4_e4m3(o0 * fp8_inv, o1 * fp8_inv, o2 * fp8_inv, o3 * fp8_inv);
+                    continue;
+                }
                 const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
                 uint2 u;
                 u.x = *reinterpret_cast<const uint32_t*>(&p0);
@@ -432,16 +442,17 @@ template <typename T>
 cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
                                const int32_t* active_idx, const float* shift, const float* scale,
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
-                               cudaStream_t st, int* n_launch, bool pdl, TextSel ts) {
+                               cudaStream_t st, int* n_launch, bool pdl, TextSel ts, float fp8_inv) {
+    if (fp8_inv > 0.f && (sizeof(T) != 2 || H % 128 != 0)) return cudaErrorInvalidValue;
     const int rows_per_cta = LN_THREADS / 32;
     const int grid = max(1, min((rows_cap + rows_per_cta - 1) / rows_per_cta, 148 * 16));
 #define FD_LN_REG(NV)                                                                                              \
     if (H == NV * 128) {                                                                                           \
         cudaError_t e = x_gather                                                                                    \
             ? ptx::launch_kernel(ln_modulate_reg_kernel<T, NV, true>, grid, LN_THREADS, 0, st, pdl, x_gather,      \
-                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl, ts) \
+                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl, ts, fp8_inv) \
             : ptx::launch_kernel(ln_modulate_reg_kernel<T, NV, false>, grid, LN_THREADS, 0, st, pdl, x_gather,     \
-                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl, ts); \
+                                 resid_in, resid_out, out, active_idx, shift, scale, mod_stride, N, ln_eps, ctl, ts, fp8_inv); \
         ++*n_launch;                                                                                               \
         return e;                                                                                                  \
     }
@@ -451,7 +462,7 @@ cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* 
 #undef FD_LN_REG
     if (H % 128 == 0) {
         cudaError_t e = ptx::launch_kernel(ln_modulate_kernel<T>, grid, LN_THREADS, 0, st, pdl, x_gather, resid_in, resid_out,
-                                           out, active_idx, shift, scale, mod_stride, N, H, ln_eps, ctl, ts);
+                                           out, active_idx, shift, scale, mod_stride, N, H, ln_eps, ctl, ts, fp8_inv);
         ++*n_launch;
         return e;
     } else
@@ -467,9 +478,9 @@ template cudaError_t launch_adaln<__nv_bfloat16>(const __nv_bfloat16*, const __n
                                                  float*, int, int, int, int, void*, cudaStream_t, int*);
 template cudaError_t launch_ln_modulate<float>(const float*, const float*, float*, float*, const int32_t*,
                                                const float*, const float*, int, int, int, int, float, const Control*,
-                                               cudaStream_t, int*, bool, TextSel);
+                                               cudaStream_t, int*, bool, TextSel, float);
 template cudaError_t launch_ln_modulate<__nv_bfloat16>(const __nv_bfloat16*, const float*, float*, __nv_bfloat16*,
                                                        const int32_t*, const float*, const float*, int, int, int, int,
-                                                       float, const Control*, cudaStream_t, int*, bool, TextSel);
+                                                       float, const Control*, cudaStream_t, int*, bool, TextSel, float);
 
 }  // namespace fd

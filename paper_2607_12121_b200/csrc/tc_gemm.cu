@@ -174,7 +174,9 @@ template <int PAIR_BN> struct PairCfg {
     static constexpr int TMEM_COLS = 512;                            // two accumulators of PAIR_BN columns
 };
 
-template <int KIND, int PAIR_BN>
+// F8: both operands are E4M3 bytes; a stage holds the same bytes and thus twice the depth of K (128 values), the
+// products are kind::f8f6f4 and the epilogue scales the accumulator (see EpiParams).
+template <int KIND, int PAIR_BN, bool F8 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                     const __grid_constant__ CUtensorMap tm_r, int n_out, int k_dim, int stream_a, int tma_resid, EpiParams ep,
@@ -221,7 +223,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     const int m_pairs = m_list ? ctl->n_text_tiles[1] : (a_total + 2 * BM - 1) / (2 * BM);
     const int n_tiles = n_out / PAIR_BN;
     const int total_tiles = m_pairs * n_tiles;
-    const int k_tiles = k_dim / BK;
+    constexpr int BKE = F8 ? 2 * BK : BK;               // values of K per stage (128 bytes per row either way)
+    const int k_tiles = k_dim / BKE;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -237,17 +240,17 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                     const uint32_t bar = map_to_cta(smem_u32(&full[s]), 0);     // the first CTA's barrier counts both halves
                     if (rank == 0) mbar_expect_tx(&full[s], 2 * PAIR_STAGE_BYTES);
                     if (stream_a)
-                        tma_load_2d_pair_hint(sA + s * A_TILE_BYTES, &tm_a, kt * BK, m * 2 * BM + (int)rank * BM, bar, evict_first);
+                        tma_load_2d_pair_hint(sA + s * A_TILE_BYTES, &tm_a, kt * BKE, m * 2 * BM + (int)rank * BM, bar, evict_first);
                     else
-                        tma_load_2d_pair(sA + s * A_TILE_BYTES, &tm_a, kt * BK, m * 2 * BM + (int)rank * BM, bar);
-                    tma_load_2d_pair(sB + s * PAIR_B_BYTES, &tm_b, kt * BK, n * PAIR_BN + (int)rank * (PAIR_BN / 2), bar);
+                        tma_load_2d_pair(sA + s * A_TILE_BYTES, &tm_a, kt * BKE, m * 2 * BM + (int)rank * BM, bar);
+                    tma_load_2d_pair(sB + s * PAIR_B_BYTES, &tm_b, kt * BKE, n * PAIR_BN + (int)rank * (PAIR_BN / 2), bar);
                 }
             }
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 700 + (int)blockIdx.x);
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = idesc_bf16(2 * BM, PAIR_BN, 0, 0);
+            constexpr uint32_t idesc = F8 ? idesc_e4m3(2 * BM, PAIR_BN) : idesc_bf16(2 * BM, PAIR_BN, 0, 0);
             uint32_t it = 0, t_it = 0;
             bool ok = true;
             for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
@@ -263,8 +266,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                     const uint64_t da = smem_desc(smem_u32(sA + s * A_TILE_BYTES), 16, 1024, SWZ_128B);
                     const uint64_t db = smem_desc(smem_u32(sB + s * PAIR_B_BYTES), 16, 1024, SWZ_128B);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        mma_bf16_ss_pair(d, da + 2 * k, db + 2 * k, idesc, (kt | k) != 0);
+                    for (int k = 0; k < BK / 16; ++k) {       // 32 bytes of K per product, either operand type
+                        if constexpr (F8) mma_f8_ss_pair(d, da + 2 * k, db + 2 * k, idesc, (kt | k) != 0);
+                        else mma_bf16_ss_pair(d, da + 2 * k, db + 2 * k, idesc, (kt | k) != 0);
+                    }
                     mma_commit_pair(&empty[s], 0x3);          // frees the stage in both CTAs
                 }
                 if (ok) mma_commit_pair(&tfull[acc], 0x3);    // both CTAs' epilogues may read their rows
@@ -292,7 +297,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             if (!mbar_wait(&tfull[acc], aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * PAIR_BN;
-            epilogue_warp<KIND>(ep, epi_stage + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane,
+            epilogue_warp<KIND, F8>(ep, epi_stage + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane,
                                 m * 2 * BM + (int)rank * BM + quad * 32, a_total, t_row, n * PAIR_BN, c_lo, c_hi, ri,
                                 (KIND == EPI_RESID && tma_resid) ? &tm_r : nullptr);
             tc_fence_before();
@@ -394,6 +399,8 @@ struct TcPlan {
     CUtensorMap* w_maps;        // [L][4]
     CUtensorMap* w_maps_text;   // [L][4] second stream's weights (dual stream), or nullptr
     CUtensorMap* w_maps_cross;  // [L][2] cross-attention's query and out projections, or nullptr
+    CUtensorMap* w_maps_f8;     // [L][3] E4M3 weights of QKV, fc1, fc2 (FP8 operands), or nullptr
+    CUtensorMap a_maps_f8[2];   // the activation buffer and the MLP hidden buffer read as E4M3 bytes
     const int32_t* text_list128;    // device lists of the row tiles that hold rows of the second stream
     const int32_t* text_list256;
     // attention (filled by the attention part)
@@ -418,6 +425,7 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
     p->w_maps = new CUtensorMap[(size_t)cfg.n_blocks * 4];
     p->w_maps_text = nullptr;
     p->w_maps_cross = nullptr;
+    p->w_maps_f8 = nullptr;
     p->text_list128 = p->text_list256 = nullptr;
     p->attn = nullptr;
     int dev = 0;
@@ -478,6 +486,12 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         FD_SET_PAIR(EPI_QKV, 256) FD_SET_PAIR(EPI_RESID, 256) FD_SET_PAIR(EPI_GELU, 256)
         FD_SET_PAIR(EPI_QKV, 192) FD_SET_PAIR(EPI_RESID, 192) FD_SET_PAIR(EPI_GELU, 192)
 #undef FD_SET_PAIR
+#define FD_SET_PAIR8(K, N)                                                                                 \
+    if (e == cudaSuccess)                                                                                  \
+        e = cudaFuncSetAttribute(tc_gemm_pair_kernel<K, N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<N>::SMEM);
+        FD_SET_PAIR8(EPI_QKV, 256) FD_SET_PAIR8(EPI_RESID, 256) FD_SET_PAIR8(EPI_GELU, 256)
+        FD_SET_PAIR8(EPI_QKV, 192) FD_SET_PAIR8(EPI_RESID, 192) FD_SET_PAIR8(EPI_GELU, 192)
+#undef FD_SET_PAIR8
         if (e != cudaSuccess) {
             ok = false;
             if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
@@ -519,6 +533,7 @@ void tc_plan_destroy(TcPlan* p) {
     delete[] p->w_maps;
     delete[] p->w_maps_text;
     delete[] p->w_maps_cross;
+    delete[] p->w_maps_f8;
     delete p;
 }
 
@@ -587,6 +602,74 @@ bool tc_plan_set_cross(TcPlan* p, const void* w_q, const void* w_o, std::string*
         }
     }
     return true;
+}
+
+// FP8 operands: tensor maps of the E4M3 weights (all nullptr: off) and of the two activation buffers read as bytes.
+// Needs the CTA-pair kernel for the three projections.
+bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const void* w8_fc2, std::string* err) {
+    delete[] p->w_maps_f8;
+    p->w_maps_f8 = nullptr;
+    if (!w8_qkv || !w8_fc1 || !w8_fc2) return true;
+    const fd_config& cfg = p->cfg;
+    const TcGemmKind kinds[3] = {TC_GEMM_QKV, TC_GEMM_FC1, TC_GEMM_FC2};
+    const char* w_base[3] = {static_cast<const char*>(w8_qkv), static_cast<const char*>(w8_fc1), static_cast<const char*>(w8_fc2)};
+    for (int g = 0; g < 3; ++g)
+        if (!p->spec[kinds[g]].pair_bn || p->spec[kinds[g]].k % 128) {
+            if (err) *err = "FP8 operands need the CTA-pair kernel (output widths multiples of 192 or 256) and K a multiple of 128";
+            return false;
+        }
+    p->w_maps_f8 = new CUtensorMap[(size_t)cfg.n_blocks * 3];
+    bool ok = true;
+    void* a_base[2] = {p->buf.act, p->buf.g};
+    const int a_k[2] = {cfg.hidden, cfg.mlp_dim};
+    for (int i = 0; i < 2 && ok; ++i) {
+        const uint64_t dims[2] = {(uint64_t)a_k[i], (uint64_t)p->buf.Mcap};
+        const uint64_t strides[1] = {(uint64_t)a_k[i]};
+        const uint32_t box[2] = {128, BM};
+        ok = encode_tmap(&p->a_maps_f8[i], CU_TENSOR_MAP_DATA_TYPE_UINT8, a_base[i], 2, dims, strides, box, 128, err);
+    }
+    for (int g = 0; g < 3 && ok; ++g) {
+        const GemmSpec& s = p->spec[kinds[g]];
+        for (int l = 0; l < cfg.n_blocks && ok; ++l) {
+            const uint64_t wd[2] = {(uint64_t)s.k, (uint64_t)s.n_out};
+            const uint64_t strides[1] = {(uint64_t)s.k};
+            const uint32_t wb[2] = {128, (uint32_t)s.pair_bn / 2};
+            void* base = const_cast<char*>(w_base[g]) + (size_t)l * s.n_out * s.k;
+            ok = encode_tmap(&p->w_maps_f8[(size_t)l * 3 + g], CU_TENSOR_MAP_DATA_TYPE_UINT8, base, 2, wd, strides, wb, 128, err);
+        }
+    }
+    if (!ok) {
+        delete[] p->w_maps_f8;
+        p->w_maps_f8 = nullptr;
+    }
+    return ok;
+}
+
+cudaError_t tc_gemm_fp8(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
+                        int* n_launch) {
+    if (!p->w_maps_f8 || (kind != TC_GEMM_QKV && kind != TC_GEMM_FC1 && kind != TC_GEMM_FC2)) return cudaErrorInvalidValue;
+    const GemmSpec& s = p->spec[kind];
+    const int g = kind == TC_GEMM_QKV ? 0 : kind == TC_GEMM_FC1 ? 1 : 2;
+    const CUtensorMap& wm = p->w_maps_f8[(size_t)blk * 3 + g];
+    const CUtensorMap& am = p->a_maps_f8[kind == TC_GEMM_FC2 ? 1 : 0];
+    Control* c = const_cast<Control*>(ctl);
+    const int pgrid = max(2, min(p->sm_count & ~1, p->pair_ctas));
+    const int stream_a = kind == TC_GEMM_FC2 ? 1 : 0;
+    const int32_t* no_list = nullptr;
+    cudaError_t e = cudaSuccess;
+#define FD_LAUNCH_PAIR8(K, N) \
+    e = launch_kernel(tc_gemm_pair_kernel<K, N, true>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, am, wm, p->resid_map, s.n_out, \
+                      s.k, stream_a, p->tma_resid ? 1 : 0, ep, c, no_list)
+    if (kind == TC_GEMM_QKV) {
+        if (s.pair_bn == 256) FD_LAUNCH_PAIR8(EPI_QKV, 256); else FD_LAUNCH_PAIR8(EPI_QKV, 192);
+    } else if (kind == TC_GEMM_FC1) {
+        if (s.pair_bn == 256) FD_LAUNCH_PAIR8(EPI_GELU, 256); else FD_LAUNCH_PAIR8(EPI_GELU, 192);
+    } else {
+        if (s.pair_bn == 256) FD_LAUNCH_PAIR8(EPI_RESID, 256); else FD_LAUNCH_PAIR8(EPI_RESID, 192);
+    }
+#undef FD_LAUNCH_PAIR8
+    ++*n_launch;
+    return e;
 }
 
 cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind_in, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
