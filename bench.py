@@ -413,6 +413,42 @@ class Engine:
             out["kernels"] = self.kernel_table(steps, A_b, peaks)
         return out, A_b, step_flops
 
+    def fp8_measure(self, steps, peaks, ms_bf16, fraction=None):
+        """The same gated step with FP8 operands for the QKV, fc1 and fc2 projections: the bf16 weights quantised per
+        output row to E4M3 on the device (library cast), fixed activation scales.  Step time, the three projections'
+        rates against twice the measured bf16 peaks (the nominal fp8 : bf16 ratio), then back to bf16."""
+        torch, fd, wl = self.torch, self.fd, self.wl
+        self.set_fraction(fraction)                       # the active set ms_bf16 was measured on
+        ops = {}
+        for name in ("qkv", "fc1", "fc2"):
+            W = self.weights["w_" + name].float()
+            sc = (W.abs().amax(dim=-1) / 448.0).clamp_min(1e-12)
+            ops["w8_" + name] = (W / sc[..., None]).to(torch.float8_e4m3fn).view(torch.uint8).contiguous()
+            ops["s_" + name] = sc.contiguous()
+            del W
+        a = np.empty((wl.L, 3), np.float32)
+        a[:, 0:2], a[:, 2] = 1.0 / 32, 1.0 / 64
+        ops["a_scale"] = a
+        try:
+            fd.fd_set_fp8_operands(self.ctx, ops)
+        except fd.FlashDiffError as e:
+            return {"unavailable": str(e)}
+        for _ in range(3):
+            self.gated_step()
+        A_b, A = self.active()
+        ms = self.timed(self.gated_step, steps)
+        table = self.kernel_table(max(2, steps // 2), A_b, peaks)
+        fd.fd_set_fp8_operands(self.ctx, None)
+        self.dense_step(self.x_prev)                      # the cached state as the bf16 step left it
+        out = {"step_ms": round(ms, 4), "active_tokens": A, "speedup_vs_bf16": round(ms_bf16 / ms, 3), "dtype": "e4m3 x e4m3 -> f32 (QKV, fc1, fc2)",
+               "peak": "2 x the measured bf16 peaks (nominal ratio)", "kernels": {}}
+        for k in ("gemm_qkv", "gemm_fc1", "gemm_fc2"):
+            if k in table:
+                t = table[k]
+                out["kernels"][k] = {"avg_call_us": t["avg_call_us"], "tflops": t["tflops"],
+                                     "frac_burst": round(t["frac_burst"] / 2, 3), "frac_sustained": round(t["frac_sustained"] / 2, 3)}
+        return out
+
     def close(self):
         st = self.fd.fd_destroy(self.ctx)
         self.__dict__.clear()                 # drops the weights, caches and inputs
@@ -430,6 +466,7 @@ def side_workload(name, seed, dev, rep, steps, warmup, peaks):
         sweep[tag] = {k: r[k] for k in ("active_fraction", "step_ms", "tflops", "speedup_vs_dense", "t_over_f_dense")}
     if sweep:
         res["sweep"] = sweep
+    res["fp8_operands"] = eng.fp8_measure(steps, peaks, res["step_ms"])
     eng.close()
     del eng
     torch.cuda.empty_cache()
@@ -636,6 +673,9 @@ def run_ours(args):
             r, _, _ = eng.measure(max(5, args.steps // 4), 3, peaks, fraction=f, kernels=False, dense_ms=ms_dense)
             sweep[tag] = {k: r[k] for k in ("active_fraction", "step_ms", "tflops", "speedup_vs_dense", "t_over_f_dense")}
     weight_gb = sum(t.numel() * t.element_size() for t in eng.weights.values()) / 1e9
+    fp8 = None
+    if world == 1 and not args.no_extras:
+        fp8 = eng.fp8_measure(max(5, args.steps // 2), peaks, ms_reg, args.fraction)
     st_destroy = eng.close()
     del eng, x, cond, y, z_cur, z_prev, eps
     torch.cuda.empty_cache()
@@ -664,7 +704,7 @@ def run_ours(args):
         "step_tflops": round(value / world, 1), "step_frac_burst": round(value / world / burst, 4),
         "step_frac_sustained": round(value / world / sust, 4),
         "kernels": breakdown, "sweep": sweep, "workloads": others,
-        "activity_probe": probe,
+        "activity_probe": probe, "fp8_operands": fp8,
     }
 
     line = {
