@@ -7,8 +7,9 @@
 //   S = Q K^T   M = 256 (both CTAs' query rows), N = 64 keys;  each CTA stages 32 of the tile's keys
 //   O += P V    M = 256, N = 128 head dims;            each CTA stages all 64 keys of 64 of the head dims
 // so a CTA brings in half of every K / V tile: the pair pulls each key and value from L2 once, where two
-// independent CTAs pull it twice -- and at this head dim the single-CTA kernel is paced by that traffic (it
-// draws 8.6 TB/s from L2 across the chip).  No load is multicast: every CTA fetches what it stages itself.
+// independent CTAs pull it twice (the single-CTA kernel draws 8.6-10 TB/s from L2 across the chip at this head dim,
+// which turned out to be a third of what that path sustains: not what paces it).  No load is multicast: every CTA
+// fetches what it stages itself.
 // Key tiles are 64 keys so that each softmax warpgroup has a score buffer of its own (2 x 64 score columns, 2 x 32
 // P columns and 2 x 128 accumulator columns of TMEM): the product for tile g + 2 then only needs the scores of
 // tile g to have left its buffer, which happened a whole tile earlier.
