@@ -44,12 +44,20 @@ def _codes_close(got, want, max_fraction):
     assert near.all()
 
 
-@pytest.mark.parametrize("name", ["image_tc", "wide_tc", "audio_tc"])
+def _stage_workload(name):
+    if name == "audio_width":                   # the audio configuration's width (hidden 1536, MLP 6144), 384 tokens
+        return gen.workload("audio").replace(name=name, L=1, B=1, grid=(384,), R=24)
+    if name == "video_width":                   # the video configuration's width (12 heads of 128, MLP 8960), 384 tokens
+        return gen.workload("audio").replace(name=name, L=1, B=1, grid=(384,), R=24, heads=12, head_dim=128, M=8960)
+    return gen.workload(name).replace(L=1)
+
+
+@pytest.mark.parametrize("name", ["image_tc", "wide_tc", "audio_tc", "audio_width", "video_width"])
 def test_fp8_projections_stage_by_stage(name):
     """One block, every row active, attention gate zero (the residual entering the MLP branch is then the block's input
     exactly): each 8-bit projection is checked against exact arithmetic on the library's own quantised operands, read
     from the step's intermediate buffers, so that no rounding decision taken upstream blurs the comparison."""
-    wl = gen.workload(name).replace(L=1)
+    wl = _stage_workload(name)
     seed = 11
     H, M = wl.H, wl.M
     labels = labels_for(wl, seed)

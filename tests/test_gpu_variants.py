@@ -19,15 +19,17 @@ def _masks(wl):
             gen.region_mask(wl, 4, [0.34] * wl.B)]
 
 
-@pytest.mark.parametrize("name,engine", [("tiny", fd.FD_ENGINE_SIMT), ("audio_small", fd.FD_ENGINE_SIMT),
-                                         ("image_small", fd.FD_ENGINE_SIMT), ("audio_tc", fd.FD_ENGINE_TC),
-                                         ("image_tc", fd.FD_ENGINE_TC), ("wide_tc", fd.FD_ENGINE_TC),
-                                         ("mmdit_tc", fd.FD_ENGINE_TC), ("video_tc", fd.FD_ENGINE_TC)])
-@pytest.mark.parametrize("which", ["both", "norm", "rope"])
+_CONFIGS = [("tiny", fd.FD_ENGINE_SIMT), ("audio_small", fd.FD_ENGINE_SIMT), ("image_small", fd.FD_ENGINE_SIMT),
+            ("audio_tc", fd.FD_ENGINE_TC), ("image_tc", fd.FD_ENGINE_TC), ("wide_tc", fd.FD_ENGINE_TC),
+            ("mmdit_tc", fd.FD_ENGINE_TC), ("video_tc", fd.FD_ENGINE_TC)]
+# both variants together everywhere; each one alone on three configurations
+_CASES = [(n, e, "both") for n, e in _CONFIGS] + [(n, e, w) for n, e in _CONFIGS if n in ("audio_small", "audio_tc", "image_tc")
+                                                   for w in ("norm", "rope")]
+
+
+@pytest.mark.parametrize("name,engine,which", _CASES)
 def test_variants_match_the_oracle(name, engine, which):
     wl = gen.workload(name)
-    if which != "both" and name not in ("audio_small", "audio_tc", "image_tc"):
-        pytest.skip("single variants are covered on three configurations")
     var = gen.block_variants(wl, 9, qk_norm=which != "rope", rope=which != "norm")
     masks = _masks(wl) if name != "tiny" else list(gen.mask_schedule(wl, 0, 3))
     # larger query / key weights: the variants then change the attention visibly (weights stay exact in bf16)
