@@ -396,8 +396,12 @@ enum {
  *   FD_BUF_ACT     [rows, H]   the last modulated-LayerNorm output: storage type, or E4M3 bytes with FP8 operands
  *   FD_BUF_HIDDEN  [rows, M]   the last block's MLP hidden activations: storage type, or E4M3 bytes with FP8 operands
  *   FD_BUF_RESID   [rows, H]   f32 residual stream after the last block (tensor-core engine)
+ *   FD_BUF_Q       [rows, q_ld] the last block's query rows, storage type; q_ld = bytes / (rows capacity * element size):
+ *                              n_heads * head_dim, except that the tensor-core attention stores a 72-wide head in 80
+ *                              columns (the last 8 zero)
+ *   FD_BUF_ATTN    [rows, H]   the last block's self-attention output (or the cross-attention's, when that is set)
  */
-enum { FD_BUF_ACT = 0, FD_BUF_HIDDEN = 1, FD_BUF_RESID = 2 };
+enum { FD_BUF_ACT = 0, FD_BUF_HIDDEN = 1, FD_BUF_RESID = 2, FD_BUF_Q = 3, FD_BUF_ATTN = 4 };
 fd_status fd_debug_buffer(fd_ctx* ctx, int which, void** device_ptr_out, size_t* bytes_out);
 
 fd_status fd_profile_enable(fd_ctx* ctx, int enable);

@@ -327,7 +327,7 @@ def fd_set_cross_attention(ctx: Context, cross: Optional[Dict[str, "object"]]) -
     _check(ctx.handle, lib.fd_set_cross_attention(ctx.handle, ctypes.byref(x)))
 
 
-FD_BUF_ACT, FD_BUF_HIDDEN, FD_BUF_RESID = 0, 1, 2
+FD_BUF_ACT, FD_BUF_HIDDEN, FD_BUF_RESID, FD_BUF_Q, FD_BUF_ATTN = 0, 1, 2, 3, 4
 
 
 def fd_debug_buffer(ctx: Context, which: int):

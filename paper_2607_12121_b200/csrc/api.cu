@@ -762,6 +762,8 @@ fd_status fd_debug_buffer(fd_ctx* c, int which, void** device_ptr_out, size_t* b
         case FD_BUF_ACT: *device_ptr_out = c->ws + l.act; *bytes_out = (size_t)l.Mcap * c->cfg.hidden * es; break;
         case FD_BUF_HIDDEN: *device_ptr_out = c->ws + l.g; *bytes_out = (size_t)l.Mcap * c->cfg.mlp_dim * es; break;
         case FD_BUF_RESID: *device_ptr_out = c->ws + l.resid; *bytes_out = (size_t)l.Mcap * c->cfg.hidden * sizeof(float); break;
+        case FD_BUF_Q: *device_ptr_out = c->ws + l.q; *bytes_out = (size_t)l.Mcap * l.q_ld * es; break;
+        case FD_BUF_ATTN: *device_ptr_out = c->ws + l.o; *bytes_out = (size_t)l.Mcap * c->cfg.hidden * es; break;
         default: return c->fail(FD_ERR_INVALID_ARG, "unknown buffer %d", which);
     }
     return FD_OK;

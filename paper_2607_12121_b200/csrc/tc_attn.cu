@@ -415,81 +415,96 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int i = 0; i < 128; ++i) if (i >= rem) sr[i] = 0xff800000u;          // -inf
                     }
-                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                    for (int i = 0; i < 128; i += 8) {           // three-input maxima: half the instructions
-                        mx0 = max3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
-                        mx1 = max3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
-                        mx2 = max3(mx2, __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
-                        mx3 = max3(mx3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
-                    }
-                    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
                     // the P buffer is free, and O_par complete, once the product of this warpgroup's previous tile is done
                     if (g >= 2 && !mbar_wait(&pv_done[par * 2], ((g >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
-                    if (first) {
-                        m = mx;
-                    } else {
-                        const bool need = (mx - m) * scale_log2 > RESCALE_LOG2;
-                        if (__any_sync(0xffffffffu, need)) {
-                            tc_fence_after();
-                            const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
-                            if (need) { l *= f; own *= f; m = mx; }
+                    // The tile's own maximum is only computed when it is needed: for the warpgroup's first tile of an
+                    // item, and when a tile's row sum shows that some score outgrew the reference maximum m by more
+                    // than the rescaling threshold (p <= 2^24 for all 128 keys keeps the sum at or below 2^31; an
+                    // overflow gives inf or NaN, which fails the same comparison).  Then the tile is done again with
+                    // its true maximum: P is simply overwritten, nothing has consumed it yet.  (The mass variant keeps
+                    // the maximum per tile: its label bookkeeping could not be redone.)
+                    bool with_max = first || MASS;
 #pragma unroll 1
-                            for (int c = 0; c < D / 8; ++c) {    // rare, and 128 scores are live: small pieces
-                                uint32_t orr[8];
-                                tmem_ld8(o_addr + c * 8, orr);
-                                tmem_wait_ld();
+                    for (;;) {
+                        if (with_max) {
+                            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
-                                tmem_st8(o_addr + c * 8, orr);
+                            for (int i = 0; i < 128; i += 8) {   // three-input maxima: half the instructions
+                                mx0 = max3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+                                mx1 = max3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+                                mx2 = max3(mx2, __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
+                                mx3 = max3(mx3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
                             }
-                            tmem_wait_st();
-                        }
-                    }
-                    const float mb = m * scale_log2;
-                    const uint64_t nmb2 = pair(-mb, -mb);
-                    uint64_t sua = pair(0.f, 0.f), sub_ = pair(0.f, 0.f);
+                            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                            if (first) {
+                                m = mx;
+                            } else {
+                                const bool need = (mx - m) * scale_log2 > RESCALE_LOG2;
+                                if (__any_sync(0xffffffffu, need)) {
+                                    tc_fence_after();
+                                    const float f = need ? ex2((m - mx) * scale_log2) : 1.0f;
+                                    if (need) { l *= f; own *= f; m = mx; }
+#pragma unroll 1
+                                    for (int c = 0; c < D / 8; ++c) {    // rare, and 128 scores are live: small pieces
+                                        uint32_t orr[8];
+                                        tmem_ld8(o_addr + c * 8, orr);
+                                        tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        int kl = -2;                             // MASS: label of key `lane` of this chunk
-                        if constexpr (MASS) {
-                            const int k0 = j * KEYS + c * 32 + lane;
-                            if (k0 < N) kl = __ldg(key_lab + k0);
-                        }
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int i = 0; i < 16; i += 4) {
-                            float p[8];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const uint64_t x = fma2(pair(__uint_as_float(sr[c * 32 + 2 * i + 2 * e]),
-                                                             __uint_as_float(sr[c * 32 + 2 * i + 2 * e + 1])), sc2, nmb2);
-                                // all on the special-function unit: one warp per scheduler and stream of tiles is bound
-                                // by instruction issue, and the cubic costs six times the instructions (measured: no share
-                                // 4 % faster at 1024 keys than a quarter, within 1 % at 8192)
-                                float xa, xb;
-                                unpair(x, xa, xb);
-                                p[2 * e] = ex2(xa);
-                                p[2 * e + 1] = ex2(xb);
-                            }
-                            sua = add2(sua, add2(pair(p[0], p[1]), pair(p[2], p[3])));
-                            sub_ = add2(sub_, add2(pair(p[4], p[5]), pair(p[6], p[7])));
-                            if constexpr (MASS) {
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    const int klk = __shfl_sync(0xffffffffu, kl, 2 * i + e);
-                                    own += klk == my_lab ? p[e] : 0.f;
+                                        for (int i = 0; i < 8; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
+                                        tmem_st8(o_addr + c * 8, orr);
+                                    }
+                                    tmem_wait_st();
                                 }
                             }
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) pk[i + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
                         }
-                        tmem_st16(p_addr + c * 16, pk);
-                    }
-                    {
+                        const float mb = m * scale_log2;
+                        const uint64_t nmb2 = pair(-mb, -mb);
+                        uint64_t sua = pair(0.f, 0.f), sub_ = pair(0.f, 0.f);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            int kl = -2;                             // MASS: label of key `lane` of this chunk
+                            if constexpr (MASS) {
+                                const int k0 = j * KEYS + c * 32 + lane;
+                                if (k0 < N) kl = __ldg(key_lab + k0);
+                            }
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int i = 0; i < 16; i += 4) {
+                                float p[8];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const uint64_t x = fma2(pair(__uint_as_float(sr[c * 32 + 2 * i + 2 * e]),
+                                                                 __uint_as_float(sr[c * 32 + 2 * i + 2 * e + 1])), sc2, nmb2);
+                                    // all on the special-function unit: a cubic on the FMA pipe costs six times the
+                                    // instructions (measured: no share 4 % faster at 1024 keys than a quarter, within
+                                    // 1 % at 8192)
+                                    float xa, xb;
+                                    unpair(x, xa, xb);
+                                    p[2 * e] = ex2(xa);
+                                    p[2 * e + 1] = ex2(xb);
+                                }
+                                sua = add2(sua, add2(pair(p[0], p[1]), pair(p[2], p[3])));
+                                sub_ = add2(sub_, add2(pair(p[4], p[5]), pair(p[6], p[7])));
+                                if constexpr (MASS) {
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) {
+                                        const int klk = __shfl_sync(0xffffffffu, kl, 2 * i + e);
+                                        own += klk == my_lab ? p[e] : 0.f;
+                                    }
+                                }
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) pk[i + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
+                            }
+                            tmem_st16(p_addr + c * 16, pk);
+                        }
                         float s0, s1;
                         unpair(add2(sua, sub_), s0, s1);
-                        l += s0 + s1;
+                        const float tile_sum = s0 + s1;
+                        if (with_max || !__any_sync(0xffffffffu, !(tile_sum <= 2147483648.0f))) {
+                            l += tile_sum;
+                            break;
+                        }
+                        with_max = true;
                     }
                     tmem_wait_st();
                     tc_fence_before();
