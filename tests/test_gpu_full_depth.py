@@ -85,14 +85,26 @@ def test_video_twin_all_blocks_gated_steps_with_kv_kept():
     """The video configuration's scaled-down twin, all 30 blocks: warm-up, then 6 steps whose masks come from the
     gate (state carried from step to step, target fraction falling from 0.6 to 0.3, forced reactivation after 2
     skipped steps), the K/V cache and the cached outputs kept across steps on both sides."""
+    _video_twin(None, 6, 2)
+
+
+def test_video_twin_fifty_step_schedule():
+    """The whole 50-step schedule of the video configuration (target fraction falling linearly from 0.6 to 0.3, forced
+    reactivation after 5 skipped steps as in the paper's default) on the twin with 4 of its blocks: regions stay
+    frozen for up to 5 steps, their K/V rows that long stale, and come back forced, dozens of times over."""
+    _video_twin(4, 50, 5)
+
+
+def _video_twin(n_blocks, n_steps, K):
     wl = gen.workload("video_twin")
-    B, N, H, L, R, K = wl.B, wl.N, wl.H, wl.L, wl.R, 2
+    if n_blocks is not None:
+        wl = wl.replace(L=n_blocks)
+    B, N, H, L, R = wl.B, wl.N, wl.H, wl.L, wl.R
     labels = labels_for(wl, 52)
     w = gen.block_weights(wl, 52)
     w["w_qkv"][:, :H] *= np.float32(8.0)          # peaked softmax: every key tile and every merge of partial results
     w["b_qkv"][:, :H] *= np.float32(8.0)          # matters to the output (a power of two keeps the weights exact in bf16)
     inp = gen.step_inputs(wl, 52, labels)
-    n_steps = 6
     fr = np.linspace(0.6, 0.3, n_steps)
     lat = gen.latent_sequence(wl, 52, labels, [[f] * B for f in fr])
     ctx = make_ctx(wl, w, max_skip_k=K)
@@ -132,8 +144,9 @@ def test_video_twin_all_blocks_gated_steps_with_kv_kept():
         y = host(buf.y).reshape(B * N, H)
         yr = y_ref.reshape(B * N, H)
         ma, rl = max_abs(y[act], yr[act]), rel_l2(y[act], yr[act])
-        print("video twin step %d: active fraction %.3f, y max_abs %.4f rel_l2 %.5f, max|y| %.1f" %
-              (step, fractions[-1], ma, rl, np.abs(yr[act]).max()))
+        if n_steps <= 10 or step % 10 == 9:
+            print("video twin (%d blocks) step %d: active fraction %.3f, y max_abs %.4f rel_l2 %.5f, max|y| %.1f" %
+                  (L, step, fractions[-1], ma, rl, np.abs(yr[act]).max()))
         assert _stack_output_close(y[act], yr[act], L)
         assert np.array_equal(y[~act], y_before.reshape(B * N, H)[~act])
         a2 = act.reshape(B, N)
