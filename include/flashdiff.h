@@ -240,9 +240,13 @@ fd_status fd_set_cross_attention(fd_ctx* ctx, const fd_cross_attention* cross);
  *               block: a_scale, a HOST array [L, 3] (inputs of QKV, fc1, fc2), copied by this call;
  *   result      (exact products, fp32 accumulation) * (a * s[o]) + bias, then as without FP8.
  * The attention, the out-projection, the cross-attention and all vector work stay in bf16 / fp32.  Tensor-core
- * engine with bf16 storage only, hidden and mlp_dim multiples of 192 or 256 (else FD_ERR_UNSUPPORTED); not
- * together with a second stream (fd_set_text_stream).  Pointers 16-byte aligned, owned by the caller and alive
- * while set.  NULL switches it off.  Host call, no launch; takes effect from the next step.
+ * engine with bf16 storage only, hidden and mlp_dim multiples of 192 or 256 (else FD_ERR_UNSUPPORTED).  Pointers
+ * 16-byte aligned, owned by the caller and alive while set.  NULL switches it off.  Host call, no launch; takes effect
+ * from the next step.
+ * With a second stream (fd_set_text_stream) that stream's three projections need 8-bit operands of their own, given
+ * by fd_set_fp8_text_stream in the same form (its own quantised weights, row scales and activation scales; a row is
+ * quantised with the scale of the stream it belongs to); a step that finds FP8 operands and a second stream but not
+ * the second stream's operands fails with FD_ERR_UNSUPPORTED.
  */
 typedef struct fd_fp8_operands {
     const void* w8_qkv;
@@ -254,6 +258,7 @@ typedef struct fd_fp8_operands {
     const float* a_scale;
 } fd_fp8_operands;
 fd_status fd_set_fp8_operands(fd_ctx* ctx, const fd_fp8_operands* fp8);
+fd_status fd_set_fp8_text_stream(fd_ctx* ctx, const fd_fp8_operands* fp8_text);
 
 /*
  * The Patch Gate on the paper's own signal (Sec. 4.2): the refinement importance of a patch is the block mean of

@@ -123,7 +123,8 @@ def _cross_arg(v, l: int, B: int, H: int, keep: list):
 
 def _fp8_arg(v, l: int, keep: list):
     """fdo_fp8 of block ``l`` from variants["fp8"] = {w_qkv [L,3H,H], s_qkv [L,3H], w_fc1, s_fc1, w_fc2, s_fc2: the E4M3
-    values of the quantised weights and their per-row scales; a_scale [L,3]: activation scales of QKV, fc1, fc2}."""
+    values of the quantised weights and their per-row scales; a_scale [L,3]: activation scales of QKV, fc1, fc2}
+    (the second stream's: variants["text"]["fp8"], handed over as the dict itself)."""
     f = v.get("fp8")
     if f is None:
         return None
@@ -189,7 +190,8 @@ def regional_block(u_in: np.ndarray, active_idx: np.ndarray, mod: np.ndarray, w:
         B, N, H, heads, dh, M, A, _ip(np.ascontiguousarray(active_idx, np.int32)), ctypes.byref(img), txt,
         None if tt is None else tt.ctypes.data_as(ctypes.c_void_p), ctypes.c_float(ln_eps), _fp(_c(u_in)), _fp(u_out), _fp(kv_l),
         0 if fin is None else int(fin.size), _ip(fin), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))),
-        ctypes.c_void_p(rc_), ctypes.c_void_p(rs_), _cross_arg(v, l, B, H, keep), _fp8_arg(v, l, keep))
+        ctypes.c_void_p(rc_), ctypes.c_void_p(rs_), _cross_arg(v, l, B, H, keep), _fp8_arg(v, l, keep),
+        _fp8_arg(v.get("text") or {}, l, keep))
     assert rc == 0
     return u_out
 
@@ -269,7 +271,7 @@ def dense_block(x: np.ndarray, cond: np.ndarray, w: Dict[str, np.ndarray], l: in
     rc = _load().fdo_dense_block_q(
         B, N, H, heads, dh, M, Hc, _fp(_c(cond)), ctypes.byref(wi), wt, n_text, ctypes.c_float(ln_eps), _fp(_c(x)), _fp(x_out),
         _fp(kv), ctypes.c_float(float(v.get("qk_norm_eps", 1e-6))), ctypes.c_void_p(rc_), ctypes.c_void_p(rs_),
-        _cross_arg(v, l, B, H, keep), _fp8_arg(v, l, keep))
+        _cross_arg(v, l, B, H, keep), _fp8_arg(v, l, keep), _fp8_arg(v.get("text") or {}, l, keep))
     assert rc == 0
     return x_out, kv
 

@@ -202,7 +202,8 @@ typedef struct {
     int T;
 } fdo_dense_cross;
 
-/* fdo_dense_block_q: the QKV, fc1 and fc2 projections with FP8 operands (single stream only; q8 = NULL: off) */
+/* fdo_dense_block_q: the QKV, fc1 and fc2 projections with FP8 operands (q8 = NULL: off; q8t: the second stream's
+ * operands, given exactly when there is a second stream) */
 typedef struct {
     const float *w_qkv, *s_qkv, *w_fc1, *s_fc1, *w_fc2, *s_fc2;   /* E4M3 weight values and per-row scales */
     float a_qkv, a_fc1, a_fc2;                                    /* activation scales */
@@ -211,14 +212,14 @@ typedef struct {
 int fdo_dense_block_q(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
                       const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
-                      const float* rope_sin, const fdo_dense_cross* cross, const fdo_dense_fp8* q8);
+                      const float* rope_sin, const fdo_dense_cross* cross, const fdo_dense_fp8* q8, const fdo_dense_fp8* q8t);
 
 int fdo_dense_block_x(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
                       const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
                       const float* rope_sin, const fdo_dense_cross* cross) {
     return fdo_dense_block_q(B, N, H, heads, dh, M, Hc, cond, wi, wt, n_text, ln_eps, x_in, x_out, kv_out, qk_eps, rope_cos,
-                             rope_sin, cross, NULL);
+                             rope_sin, cross, NULL, NULL);
 }
 
 int fdo_dense_block_d(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
@@ -252,9 +253,10 @@ int fdo_dense_block(int B, int N, int H, int heads, int dh, int M, int Hc, const
 int fdo_dense_block_q(int B, int N, int H, int heads, int dh, int M, int Hc, const float* cond,
                       const fdo_dense_weights* wi, const fdo_dense_weights* wt, int n_text, float ln_eps,
                       const float* x_in, float* x_out, float* kv_out, float qk_eps, const float* rope_cos,
-                      const float* rope_sin, const fdo_dense_cross* cross, const fdo_dense_fp8* q8) {
+                      const float* rope_sin, const fdo_dense_cross* cross, const fdo_dense_fp8* q8, const fdo_dense_fp8* q8t) {
     if (heads * dh != H) return 2;
-    if (q8 && wt) return 5;
+    if ((q8 != NULL && wt != NULL) != (q8t != NULL)) return 5;
+    const fdo_dense_fp8* q8s[2] = {q8, q8t};
     if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
     if (!wt) n_text = 0;
     if (n_text < 0 || n_text > N) return 4;
@@ -293,7 +295,7 @@ int fdo_dense_block_q(int B, int N, int H, int heads, int dh, int M, int Hc, con
             const float* md = mod + (size_t)s * 6 * H;
             layernorm_modulate(X + lo * H, n, H, md, md + H, ln_eps, xh + lo * H);
             if (q8) {
-                if (matmul_nt_bias_fp8(xh + lo * H, q8->a_qkv, q8->w_qkv, q8->s_qkv, ws[s]->b_qkv, n, H, 3 * H, qkv + lo * 3 * H)) { rc = 1; goto done; }
+                if (matmul_nt_bias_fp8(xh + lo * H, q8s[s]->a_qkv, q8s[s]->w_qkv, q8s[s]->s_qkv, ws[s]->b_qkv, n, H, 3 * H, qkv + lo * 3 * H)) { rc = 1; goto done; }
             } else {
                 matmul_nt_bias(xh + lo * H, ws[s]->w_qkv, ws[s]->b_qkv, n, H, 3 * H, qkv + lo * 3 * H);
             }
@@ -345,7 +347,7 @@ int fdo_dense_block_q(int B, int N, int H, int heads, int dh, int M, int Hc, con
             const float* md = mod + (size_t)s * 6 * H;
             layernorm_modulate(res + lo * H, n, H, md + 3 * H, md + 4 * H, ln_eps, xh + lo * H);
             if (q8) {
-                if (matmul_nt_bias_fp8(xh + lo * H, q8->a_fc1, q8->w_fc1, q8->s_fc1, ws[s]->b_fc1, n, H, M, hid + lo * M)) { rc = 1; goto done; }
+                if (matmul_nt_bias_fp8(xh + lo * H, q8s[s]->a_fc1, q8s[s]->w_fc1, q8s[s]->s_fc1, ws[s]->b_fc1, n, H, M, hid + lo * M)) { rc = 1; goto done; }
             } else {
                 matmul_nt_bias(xh + lo * H, ws[s]->w_fc1, ws[s]->b_fc1, n, H, M, hid + lo * M);
             }
@@ -354,7 +356,7 @@ int fdo_dense_block_q(int B, int N, int H, int heads, int dh, int M, int Hc, con
                 hid[e] = (float)(0.5 * a * (1.0 + tanh(0.79788456080286535588 * (a + 0.044715 * a * a * a))));
             }
             if (q8) {
-                if (matmul_nt_bias_fp8(hid + lo * M, q8->a_fc2, q8->w_fc2, q8->s_fc2, ws[s]->b_fc2, n, M, H, proj + lo * H)) { rc = 1; goto done; }
+                if (matmul_nt_bias_fp8(hid + lo * M, q8s[s]->a_fc2, q8s[s]->w_fc2, q8s[s]->s_fc2, ws[s]->b_fc2, n, M, H, proj + lo * H)) { rc = 1; goto done; }
             } else {
                 matmul_nt_bias(hid + lo * M, ws[s]->w_fc2, ws[s]->b_fc2, n, M, H, proj + lo * H);
             }

@@ -196,7 +196,8 @@ typedef struct {
     int T;
 } fdo_cross;
 
-/* FP8 operands of the QKV, fc1 and fc2 projections (single stream only); fp8 = NULL: off */
+/* FP8 operands of the QKV, fc1 and fc2 projections; fp8 = NULL: off.  With two streams each has its own quantised
+ * weights and activation scales: fp8_txt for the second one (both or neither). */
 typedef struct {
     const float *w_qkv, *s_qkv;             /* [3H,H] E4M3 values of the quantised weights, [3H] scales per output row */
     const float *w_fc1, *s_fc1;             /* [M,H], [M] */
@@ -208,14 +209,14 @@ int fdo_regional_block_q(int B, int N, int H, int heads, int dh, int M, int A, c
                          const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
                          float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
                          float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross,
-                         const fdo_fp8* fp8);
+                         const fdo_fp8* fp8, const fdo_fp8* fp8_txt);
 
 int fdo_regional_block_x(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
                          const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
                          float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
                          float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross) {
     return fdo_regional_block_q(B, N, H, heads, dh, M, A, active_idx, img, txt, tok_text, ln_eps, u_in, u_out, kv, n_finish,
-                                finish, qk_eps, rope_cos, rope_sin, cross, NULL);
+                                finish, qk_eps, rope_cos, rope_sin, cross, NULL, NULL);
 }
 
 int fdo_regional_block_s(int B, int N, int H, int heads, int dh, int M, int A, const int32_t* active_idx,
@@ -252,10 +253,10 @@ int fdo_regional_block_q(int B, int N, int H, int heads, int dh, int M, int A, c
                          const fdo_stream* img, const fdo_stream* txt, const uint8_t* tok_text,
                          float ln_eps, const float* u_in, float* u_out, float* kv, int n_finish, const int32_t* finish,
                          float qk_eps, const float* rope_cos, const float* rope_sin, const fdo_cross* cross,
-                         const fdo_fp8* fp8) {
+                         const fdo_fp8* fp8, const fdo_fp8* fp8_txt) {
     if (heads * dh != H) return 2;
     if ((rope_cos == NULL) != (rope_sin == NULL) || (rope_cos && (dh & 1))) return 3;
-    if (fp8 && txt) return 5;
+    if ((fp8 != NULL && txt != NULL) != (fp8_txt != NULL)) return 5;
     (void)B;
     float* q_all = (float*)malloc(sizeof(float) * (size_t)(A > 0 ? A : 1) * H);
     if (!q_all) return 1;
@@ -277,7 +278,8 @@ int fdo_regional_block_q(int B, int N, int H, int heads, int dh, int M, int A, c
                 const fdo_stream* st = (txt && tok_text[active_idx[a]]) ? txt : img;      /* the token's stream */
                 const float* md = st->mod + (size_t)b * 6 * H;
                 row_ln_modulate(u_in + (size_t)a * H, md + 0 * H, md + 1 * H, H, ln_eps, uh);
-                if (fp8) row_linear_fp8(uh, fp8->a_qkv, fp8->w_qkv, fp8->s_qkv, st->b_qkv, H, 3 * H, xq, qkv);
+                const fdo_fp8* f8 = (st == txt) ? fp8_txt : fp8;               /* the stream's 8-bit operands */
+                if (f8) row_linear_fp8(uh, f8->a_qkv, f8->w_qkv, f8->s_qkv, st->b_qkv, H, 3 * H, xq, qkv);
                 else row_linear(uh, st->w_qkv, st->b_qkv, H, 3 * H, qkv);
                 row_qk_variants(qkv, qkv + H, heads, dh, j, st->qn_w, st->kn_w, qk_eps, rope_cos, rope_sin);
                 memcpy(q_all + (size_t)a * H, qkv, sizeof(float) * (size_t)H);
@@ -372,10 +374,11 @@ int fdo_regional_block_q(int B, int N, int H, int heads, int dh, int M, int A, c
                     for (int c = 0; c < H; ++c) r1[c] = (float)((double)r1[c] + (double)proj[c]);
                 }
                 row_ln_modulate(r1, md + 3 * H, md + 4 * H, H, ln_eps, mh);
-                if (fp8) row_linear_fp8(mh, fp8->a_fc1, fp8->w_fc1, fp8->s_fc1, st->b_fc1, H, M, xq, g);
+                const fdo_fp8* f8 = (st == txt) ? fp8_txt : fp8;
+                if (f8) row_linear_fp8(mh, f8->a_fc1, f8->w_fc1, f8->s_fc1, st->b_fc1, H, M, xq, g);
                 else row_linear(mh, st->w_fc1, st->b_fc1, H, M, g);
                 for (int c = 0; c < M; ++c) g[c] = (float)gelu_tanh_d((double)g[c]);
-                if (fp8) row_linear_fp8(g, fp8->a_fc2, fp8->w_fc2, fp8->s_fc2, st->b_fc2, M, H, xq, proj);
+                if (f8) row_linear_fp8(g, f8->a_fc2, f8->w_fc2, f8->s_fc2, st->b_fc2, M, H, xq, proj);
                 else row_linear(g, st->w_fc2, st->b_fc2, M, H, proj);
                 float* out = u_out + (size_t)a * H;
                 for (int c = 0; c < H; ++c)

@@ -24,7 +24,7 @@ EXPORTS = ["fd_workspace_bytes", "fd_create", "fd_partition_regions", "fd_region
            "fd_profile_enable", "fd_profile_read", "fd_region_activity_noalloc", "fd_selftest_bounded_wait",
            "fd_embed_latent", "fd_update_latent", "fd_regional_step_mass", "fd_region_activity_attn",
            "fd_sched_pack", "fd_sched_form_batch", "fd_rsearch_init", "fd_rsearch_update", "fd_set_block_variants",
-           "fd_set_text_stream", "fd_set_cross_attention", "fd_set_fp8_operands", "fd_debug_buffer"]
+           "fd_set_text_stream", "fd_set_cross_attention", "fd_set_fp8_operands", "fd_debug_buffer", "fd_set_fp8_text_stream"]
 FD_NOALLOC_MAX_REGION_SLOTS = 16384
 PROF_GROUPS = ["activity", "compact", "adaln", "ln_modulate", "gemm_qkv", "attention", "gemm_out", "gemm_fc1",
                "gemm_fc2", "partition", "sampler", "qk_variants", "cross_attention"]
@@ -123,6 +123,8 @@ def _load() -> ctypes.CDLL:
     lib.fd_debug_buffer.argtypes = [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_size_t)]
     lib.fd_set_fp8_operands.restype = i32
     lib.fd_set_fp8_operands.argtypes = [vp, ctypes.POINTER(FdFp8Operands)]
+    lib.fd_set_fp8_text_stream.restype = i32
+    lib.fd_set_fp8_text_stream.argtypes = [vp, ctypes.POINTER(FdFp8Operands)]
     lib.fd_set_cross_attention.restype = i32
     lib.fd_set_cross_attention.argtypes = [vp, ctypes.POINTER(FdCrossAttention)]
     lib.fd_launch_count.restype = ctypes.c_int64
@@ -337,13 +339,17 @@ def fd_debug_buffer(ctx: Context, which: int):
     return int(p.value), int(n.value)
 
 
-def fd_set_fp8_operands(ctx: Context, fp8: Optional[Dict[str, "object"]]) -> None:
+def fd_set_fp8_operands(ctx: Context, fp8: Optional[Dict[str, "object"]], text_stream: bool = False) -> None:
     """FP8 operands for QKV, fc1 and fc2: ``fp8`` holds device tensors w8_qkv, w8_fc1, w8_fc2 (uint8 E4M3 codes, [L, out,
     in]), s_qkv, s_fc1, s_fc2 (float32 [L, out]; the context keeps all six alive) and a_scale, a host float32 array
-    [L, 3] of activation scales; None switches it off."""
-    ctx.fp8 = fp8
+    [L, 3] of activation scales; None switches it off.  ``text_stream``: the second stream's set."""
+    call = lib.fd_set_fp8_text_stream if text_stream else lib.fd_set_fp8_operands
+    if text_stream:
+        ctx.fp8_text = fp8
+    else:
+        ctx.fp8 = fp8
     if fp8 is None:
-        _check(ctx.handle, lib.fd_set_fp8_operands(ctx.handle, None))
+        _check(ctx.handle, call(ctx.handle, None))
         return
     import numpy as np
     for k in ("w8_qkv", "w8_fc1", "w8_fc2"):
@@ -352,7 +358,7 @@ def fd_set_fp8_operands(ctx: Context, fp8: Optional[Dict[str, "object"]]) -> Non
         assert fp8[k].is_cuda and fp8[k].is_contiguous() and str(fp8[k].dtype) == "torch.float32", k
     a = np.ascontiguousarray(fp8["a_scale"], dtype=np.float32)
     f = FdFp8Operands(*(fp8[k].data_ptr() for k in ("w8_qkv", "s_qkv", "w8_fc1", "s_fc1", "w8_fc2", "s_fc2")), a.ctypes.data)
-    _check(ctx.handle, lib.fd_set_fp8_operands(ctx.handle, ctypes.byref(f)))
+    _check(ctx.handle, call(ctx.handle, ctypes.byref(f)))
 
 
 def fd_sched_pack(load, cost, home):

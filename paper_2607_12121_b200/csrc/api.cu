@@ -98,6 +98,8 @@ struct fd_ctx {
     fd_cross_attention cross{};   // cross-attention to a fixed context (w_q null: off)
     fd_fp8_operands fp8{};        // FP8 operands of QKV, fc1, fc2 (w8_qkv null: off)
     std::vector<float> fp8_a;     // [L, 3] activation scales (host copy)
+    fd_fp8_operands fp8_text{};   // the second stream's FP8 operands (dual stream with FP8 operands)
+    std::vector<float> fp8_text_a;
     // optional per-kernel timing
     bool profiling = false;
     struct Span { cudaEvent_t a, b; int group, kernels; };
@@ -188,7 +190,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         FD_TRY(FD_PROF_ADALN, launch_adaln<T>(cond, static_cast<const T*>(c->text_w.w_ada), static_cast<const T*>(c->text_w.b_ada),
                                                mod + text_mod_off, L, B, H, Hc, c->ws + l.ada_act, st, &nl));
         FD_TRY(FD_PROF_COMPACT, launch_text_tiles(active_idx, labels, R, rows_cap, text128, text256, ctl, st, &nl));
-        ts = TextSel{labels, R, text_mod_off};
+        ts = TextSel{labels, R, text_mod_off, 0.f};
     }
     // One launch per stream where the weights differ: the first finishes the first stream's rows (all rows when there
     // is a single stream), the second walks the row tiles that hold rows of the second stream and finishes those.
@@ -203,7 +205,10 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     const float* zeros = c->at<float>(l.consts);
     const float* ones = zeros + H;
     const bool f8 = c->fp8.w8_qkv != nullptr;
-    if (f8 && dual) return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands and a second stream cannot be combined");
+    if (f8 && dual && !c->fp8_text.w8_qkv)
+        return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands with a second stream need that stream's operands too (fd_set_fp8_text_stream)");
+    const fd_fp8_operands* f8ops[2] = {&c->fp8, &c->fp8_text};
+    const std::vector<float>* f8a[2] = {&c->fp8_a, &c->fp8_text_a};
     const bool pdl = c->use_tc && c->tc && tc_plan_pdl(c->tc);
     for (int blk = 0; blk < L; ++blk) {
         const float* mod_b = mod + (size_t)blk * B * 6 * H;
@@ -219,12 +224,16 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         ep.text_mod_off = (int32_t)text_mod_off;
 
         // FP8 operands: this block's activation scales (inputs of QKV, fc1, fc2)
-        const float a_qkv = f8 ? c->fp8_a[(size_t)blk * 3 + 0] : 0.f, a_fc1 = f8 ? c->fp8_a[(size_t)blk * 3 + 1] : 0.f;
-        const float a_fc2 = f8 ? c->fp8_a[(size_t)blk * 3 + 2] : 0.f;
+        // [stream][QKV, fc1, fc2]
+        float a8[2][3] = {{0.f, 0.f, 0.f}, {0.f, 0.f, 0.f}};
+        for (int sx = 0; f8 && sx < n_pass; ++sx)
+            for (int g8 = 0; g8 < 3; ++g8) a8[sx][g8] = (*f8a[sx])[(size_t)blk * 3 + g8];
+        TextSel ts1 = ts, ts2 = ts;                          // per-row scale of the second stream's rows
+        if (f8 && dual) { ts1.fp8_inv_text = 1.0f / a8[1][0]; ts2.fp8_inv_text = 1.0f / a8[1][1]; }
         // gather (first block) or read the residual stream; LayerNorm; attention-branch modulation
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(blk == 0 ? x : nullptr, resid, resid, act, active_idx, mod_b + 0 * H,
-                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts,
-                                     f8 ? 1.0f / a_qkv : 0.f));
+                                     mod_b + 1 * H, 6 * H, N, H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts1,
+                                     f8 ? 1.0f / a8[0][0] : 0.f));
         // QKV projection; K and V rows go straight into the cache
         ep.q = q;
         ep.q_ld = l.q_ld;
@@ -237,9 +246,9 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_qkv, c->text_w.b_qkv, (size_t)blk * 3 * H, pass);
             if (f8) {
-                ep.col_scale = c->fp8.s_qkv + (size_t)blk * 3 * H;
-                ep.act_scale = a_qkv;
-                FD_TRY(FD_PROF_GEMM_QKV, tc_gemm_fp8(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl));
+                ep.col_scale = f8ops[pass]->s_qkv + (size_t)blk * 3 * H;
+                ep.act_scale = a8[pass][0];
+                FD_TRY(FD_PROF_GEMM_QKV, tc_gemm_fp8(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl, pass == 1));
             } else if (c->use_tc)
                 FD_TRY(FD_PROF_GEMM_QKV, tc_gemm(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl, pass == 1));
             else
@@ -317,17 +326,17 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         }
         // MLP branch
         FD_TRY(FD_PROF_LN, launch_ln_modulate<T>(nullptr, resid, nullptr, act, active_idx, mod_b + 3 * H, mod_b + 4 * H, 6 * H, N,
-                                     H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts, f8 ? 1.0f / a_fc1 : 0.f));
+                                     H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts2, f8 ? 1.0f / a8[0][1] : 0.f));
         ep.out = g;
         ep.out_ld = M;
         for (int pass = 0; pass < n_pass; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_fc1, c->text_w.b_fc1, (size_t)blk * M, pass);
             if (f8) {
-                ep.col_scale = c->fp8.s_fc1 + (size_t)blk * M;
-                ep.act_scale = a_fc1;
-                ep.out_inv_scale = 1.0f / a_fc2;            // the hidden activations leave as E4M3 bytes, row stride M
-                FD_TRY(FD_PROF_GEMM_FC1, tc_gemm_fp8(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl));
+                ep.col_scale = f8ops[pass]->s_fc1 + (size_t)blk * M;
+                ep.act_scale = a8[pass][1];
+                ep.out_inv_scale = 1.0f / a8[pass][2];      // the hidden activations leave as E4M3 bytes, row stride M
+                FD_TRY(FD_PROF_GEMM_FC1, tc_gemm_fp8(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl, pass == 1));
             } else if (c->use_tc)
                 FD_TRY(FD_PROF_GEMM_FC1, tc_gemm(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl, pass == 1));
             else
@@ -340,9 +349,9 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_fc2, c->text_w.b_fc2, (size_t)blk * H, pass);
             if (f8) {
-                ep.col_scale = c->fp8.s_fc2 + (size_t)blk * H;
-                ep.act_scale = a_fc2;
-                FD_TRY(FD_PROF_GEMM_FC2, tc_gemm_fp8(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl));
+                ep.col_scale = f8ops[pass]->s_fc2 + (size_t)blk * H;
+                ep.act_scale = a8[pass][2];
+                FD_TRY(FD_PROF_GEMM_FC2, tc_gemm_fp8(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl, pass == 1));
             } else if (c->use_tc)
                 FD_TRY(FD_PROF_GEMM_FC2, tc_gemm(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl, pass == 1));
             else
@@ -711,16 +720,18 @@ fd_status fd_set_cross_attention(fd_ctx* c, const fd_cross_attention* x) {
     return FD_OK;
 }
 
-fd_status fd_set_fp8_operands(fd_ctx* c, const fd_fp8_operands* f) {
-    if (!c) return FD_ERR_INVALID_ARG;
+namespace {
+// shared by the two FP8 entry points: checks, tensor maps, host copy of the activation scales
+fd_status set_fp8(fd_ctx* c, const fd_fp8_operands* f, bool text) {
+    fd_fp8_operands& dst = text ? c->fp8_text : c->fp8;
+    std::vector<float>& dst_a = text ? c->fp8_text_a : c->fp8_a;
     if (!f) {
-        c->fp8 = fd_fp8_operands{};
-        c->fp8_a.clear();
-        if (c->tc) tc_plan_set_fp8(c->tc, nullptr, nullptr, nullptr, nullptr);
+        dst = fd_fp8_operands{};
+        dst_a.clear();
+        if (c->tc) tc_plan_set_fp8(c->tc, nullptr, nullptr, nullptr, nullptr, text);
         return FD_OK;
     }
     if (!c->use_tc || !c->tc) return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands need the tensor-core engine (bf16 storage)");
-    if (c->dual) return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands and a second stream cannot be combined");
     const void* wp[6] = {f->w8_qkv, f->s_qkv, f->w8_fc1, f->s_fc1, f->w8_fc2, f->s_fc2};
     for (const void* p : wp)
         if (!p || !aligned16(p)) return c->fail(FD_ERR_INVALID_ARG, "FP8 operand pointer null or not 16-byte aligned");
@@ -730,12 +741,23 @@ fd_status fd_set_fp8_operands(fd_ctx* c, const fd_fp8_operands* f) {
         if (!(f->a_scale[i] > 0.f) || !(1.0f / f->a_scale[i] < 3.0e38f))
             return c->fail(FD_ERR_INVALID_ARG, "activation scales must be positive and finite");
     std::string err;
-    if (!tc_plan_set_fp8(c->tc, f->w8_qkv, f->w8_fc1, f->w8_fc2, &err))
+    if (!tc_plan_set_fp8(c->tc, f->w8_qkv, f->w8_fc1, f->w8_fc2, &err, text))
         return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands: %s", err.c_str());
-    c->fp8 = *f;
-    c->fp8_a.assign(f->a_scale, f->a_scale + n);
-    c->fp8.a_scale = nullptr;                 // the host array was copied
+    dst = *f;
+    dst_a.assign(f->a_scale, f->a_scale + n);
+    dst.a_scale = nullptr;                    // the host array was copied
     return FD_OK;
+}
+}  // namespace
+
+fd_status fd_set_fp8_operands(fd_ctx* c, const fd_fp8_operands* f) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    return set_fp8(c, f, false);
+}
+
+fd_status fd_set_fp8_text_stream(fd_ctx* c, const fd_fp8_operands* f) {
+    if (!c) return FD_ERR_INVALID_ARG;
+    return set_fp8(c, f, true);
 }
 
 fd_status fd_poll_status(fd_ctx* c, void* cuda_stream) {

@@ -107,6 +107,7 @@ struct TextSel {
     const int32_t* labels;     // [B*N]
     int32_t R;
     long long mod_off;         // offset (floats) from the first stream's vectors to the second stream's
+    float fp8_inv_text;        // FP8 operands: the second stream's 1 / activation scale (its rows are quantised with it)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -148,7 +149,7 @@ template <typename T>
 cudaError_t launch_ln_modulate(const T* x_gather, const float* resid_in, float* resid_out, T* out,
                                const int32_t* active_idx, const float* shift, const float* scale,
                                int mod_stride, int N, int H, int rows_cap, float ln_eps, const Control* ctl,
-                               cudaStream_t st, int* n_launch, bool pdl, TextSel ts = TextSel{nullptr, 0, 0},
+                               cudaStream_t st, int* n_launch, bool pdl, TextSel ts = TextSel{nullptr, 0, 0, 0.f},
                                float fp8_inv_scale = 0.f);   // > 0 (bf16 engine): `out` receives E4M3 bytes of value * this
 
 // qk_variants.cu: QK-RMSNorm and rotary embedding on the fresh Q rows and the K rows just written to the cache

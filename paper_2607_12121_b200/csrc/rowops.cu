@@ -252,7 +252,9 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
         const float rstd = rsqrtf(var + ln_eps);
         const float mean = x0 + dm;
         // dual stream: a token with label R takes the second stream's vectors
-        const long long soff = (ts.labels && ts.labels[tok] == ts.R) ? ts.mod_off : 0;
+        const bool text_row = ts.labels && ts.labels[tok] == ts.R;
+        const long long soff = text_row ? ts.mod_off : 0;
+        const float q_inv = text_row ? ts.fp8_inv_text : fp8_inv;      // FP8 operands: the row's stream's scale
         const float* sh = shift + (size_t)b * mod_stride + soff;
         const float* sc = scale + (size_t)b * mod_stride + soff;
 #pragma unroll 4
@@ -270,7 +272,7 @@ ln_modulate_kernel(const T* __restrict__ x_gather, const float* __restrict__ res
             if constexpr (sizeof(T) == 2) {
                 if (fp8_inv > 0.f) {          // FP8 operands: the projection reads this row as E4M3
                     *reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(out) + r0 + c) =
-                        pack4_e4m3(o0 * fp8_inv, o1 * fp8_inv, o2 * fp8_inv, o3 * fp8_inv);
+                        pack4_e4m3(o0 * q_inv, o1 * q_inv, o2 * q_inv, o3 * q_inv);
                     continue;
                 }
                 const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
@@ -344,7 +346,9 @@ ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__
         const float rstd = rsqrtf(fmaxf(sq / (float)H - dm * dm, 0.f) + ln_eps);
         const float mean = x0 + dm;
         const int b = tok / N;
-        const long long soff = (ts.labels && ts.labels[tok] == ts.R) ? ts.mod_off : 0;      // dual stream
+        const bool text_row = ts.labels && ts.labels[tok] == ts.R;                          // dual stream
+        const long long soff = text_row ? ts.mod_off : 0;
+        const float q_inv = text_row ? ts.fp8_inv_text : fp8_inv;      // FP8 operands: the row's stream's scale
         const float4* sc4 = reinterpret_cast<const float4*>(scale + (size_t)b * mod_stride + soff) + lane;
         const float4* sh4 = reinterpret_cast<const float4*>(shift + (size_t)b * mod_stride + soff) + lane;
         T* dst = out + (size_t)row * H + lane * 4;
@@ -359,7 +363,7 @@ ln_modulate_reg_kernel(const T* __restrict__ x_gather, const float* __restrict__
             if constexpr (sizeof(T) == 2) {
                 if (fp8_inv > 0.f) {          // FP8 operands: the projection reads this row as E4M3
                     *reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(out) + (size_t)row * H + lane * 4 + i * 128) =
-                        pack4_e4m3(o0 * fp8_inv, o1 * fp8_inv, o2 * fp8_inv, o3 * fp8_inv);
+                        pack4_e4m3(o0 * q_inv, o1 * q_inv, o2 * q_inv, o3 * q_inv);
                     continue;
                 }
                 const __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);

@@ -35,9 +35,11 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, co
                     int* n_launch, bool text_pass = false);
 bool tc_plan_set_text(TcPlan* p, const fd_weights* w, const int32_t* list128, const int32_t* list256, std::string* err);
 // FP8 operands: QKV, fc1 and fc2 with E4M3 weights [L, n_out, K] bytes (all nullptr: off); tc_gemm_fp8 runs one of them
-bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const void* w8_fc2, std::string* err);
+// (text: the second stream's set; text_pass: the launch over the row tiles that hold rows of the second stream)
+bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const void* w8_fc2, std::string* err,
+                     bool text = false);
 cudaError_t tc_gemm_fp8(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
-                        int* n_launch);
+                        int* n_launch, bool text_pass = false);
 // cross-attention: tensor maps of its two [L, H, H] projection weights (both nullptr: off)
 bool tc_plan_set_cross(TcPlan* p, const void* w_q, const void* w_o, std::string* err);
 // region_mass (optional): [B, R] f64, receives the own-region softmax mass

@@ -400,6 +400,7 @@ struct TcPlan {
     CUtensorMap* w_maps_text;   // [L][4] second stream's weights (dual stream), or nullptr
     CUtensorMap* w_maps_cross;  // [L][2] cross-attention's query and out projections, or nullptr
     CUtensorMap* w_maps_f8;     // [L][3] E4M3 weights of QKV, fc1, fc2 (FP8 operands), or nullptr
+    CUtensorMap* w_maps_f8_text;    // [L][3] the second stream's, or nullptr
     CUtensorMap a_maps_f8[2];   // the activation buffer and the MLP hidden buffer read as E4M3 bytes
     const int32_t* text_list128;    // device lists of the row tiles that hold rows of the second stream
     const int32_t* text_list256;
@@ -426,6 +427,7 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
     p->w_maps_text = nullptr;
     p->w_maps_cross = nullptr;
     p->w_maps_f8 = nullptr;
+    p->w_maps_f8_text = nullptr;
     p->text_list128 = p->text_list256 = nullptr;
     p->attn = nullptr;
     int dev = 0;
@@ -534,6 +536,7 @@ void tc_plan_destroy(TcPlan* p) {
     delete[] p->w_maps_text;
     delete[] p->w_maps_cross;
     delete[] p->w_maps_f8;
+    delete[] p->w_maps_f8_text;
     delete p;
 }
 
@@ -606,9 +609,10 @@ bool tc_plan_set_cross(TcPlan* p, const void* w_q, const void* w_o, std::string*
 
 // FP8 operands: tensor maps of the E4M3 weights (all nullptr: off) and of the two activation buffers read as bytes.
 // Needs the CTA-pair kernel for the three projections.
-bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const void* w8_fc2, std::string* err) {
-    delete[] p->w_maps_f8;
-    p->w_maps_f8 = nullptr;
+bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const void* w8_fc2, std::string* err, bool text) {
+    CUtensorMap*& maps = text ? p->w_maps_f8_text : p->w_maps_f8;
+    delete[] maps;
+    maps = nullptr;
     if (!w8_qkv || !w8_fc1 || !w8_fc2) return true;
     const fd_config& cfg = p->cfg;
     const TcGemmKind kinds[3] = {TC_GEMM_QKV, TC_GEMM_FC1, TC_GEMM_FC2};
@@ -618,7 +622,7 @@ bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const vo
             if (err) *err = "FP8 operands need the CTA-pair kernel (output widths multiples of 192 or 256) and K a multiple of 128";
             return false;
         }
-    p->w_maps_f8 = new CUtensorMap[(size_t)cfg.n_blocks * 3];
+    maps = new CUtensorMap[(size_t)cfg.n_blocks * 3];
     bool ok = true;
     void* a_base[2] = {p->buf.act, p->buf.g};
     const int a_k[2] = {cfg.hidden, cfg.mlp_dim};
@@ -635,27 +639,28 @@ bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const vo
             const uint64_t strides[1] = {(uint64_t)s.k};
             const uint32_t wb[2] = {128, (uint32_t)s.pair_bn / 2};
             void* base = const_cast<char*>(w_base[g]) + (size_t)l * s.n_out * s.k;
-            ok = encode_tmap(&p->w_maps_f8[(size_t)l * 3 + g], CU_TENSOR_MAP_DATA_TYPE_UINT8, base, 2, wd, strides, wb, 128, err);
+            ok = encode_tmap(&maps[(size_t)l * 3 + g], CU_TENSOR_MAP_DATA_TYPE_UINT8, base, 2, wd, strides, wb, 128, err);
         }
     }
     if (!ok) {
-        delete[] p->w_maps_f8;
-        p->w_maps_f8 = nullptr;
+        delete[] maps;
+        maps = nullptr;
     }
     return ok;
 }
 
 cudaError_t tc_gemm_fp8(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
-                        int* n_launch) {
-    if (!p->w_maps_f8 || (kind != TC_GEMM_QKV && kind != TC_GEMM_FC1 && kind != TC_GEMM_FC2)) return cudaErrorInvalidValue;
+                        int* n_launch, bool text_pass) {
+    const CUtensorMap* maps = text_pass ? p->w_maps_f8_text : p->w_maps_f8;
+    if (!maps || (kind != TC_GEMM_QKV && kind != TC_GEMM_FC1 && kind != TC_GEMM_FC2)) return cudaErrorInvalidValue;
     const GemmSpec& s = p->spec[kind];
     const int g = kind == TC_GEMM_QKV ? 0 : kind == TC_GEMM_FC1 ? 1 : 2;
-    const CUtensorMap& wm = p->w_maps_f8[(size_t)blk * 3 + g];
+    const CUtensorMap& wm = maps[(size_t)blk * 3 + g];
     const CUtensorMap& am = p->a_maps_f8[kind == TC_GEMM_FC2 ? 1 : 0];
     Control* c = const_cast<Control*>(ctl);
     const int pgrid = max(2, min(p->sm_count & ~1, p->pair_ctas));
     const int stream_a = kind == TC_GEMM_FC2 ? 1 : 0;
-    const int32_t* no_list = nullptr;
+    const int32_t* no_list = text_pass ? p->text_list256 : nullptr;   // second stream: the row tiles that hold its rows
     cudaError_t e = cudaSuccess;
 #define FD_LAUNCH_PAIR8(K, N) \
     e = launch_kernel(tc_gemm_pair_kernel<K, N, true>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, am, wm, p->resid_map, s.n_out, \

@@ -114,6 +114,14 @@ def test_fp8_operands_with_variants_and_cross_attention():
     _run_sequence(wl, 3, fd.FD_ENGINE_TC, _masks(wl), fp8=True, variants=gen.block_variants(wl, 9), n_ctx=77, qk_gain=4.0)
 
 
+@pytest.mark.parametrize("n_text,B", [(154, 2), (300, 2), (5, 4)])
+def test_fp8_operands_with_two_streams(n_text, B):
+    """Each stream with its own 8-bit weights and activation scales; text segments shorter and longer than a row tile,
+    several requests per tile."""
+    wl = gen.workload("mmdit_tc").replace(n_text=n_text, B=B)
+    _run_sequence(wl, 6, fd.FD_ENGINE_TC, _masks(wl), fp8=True, text_seed=91)
+
+
 def test_fp8_operands_few_ctas(monkeypatch):
     monkeypatch.setenv("FD_TC_MAX_CTAS", "6")                  # every CTA pair walks many tiles: rings and accumulators wrap
     wl = gen.workload("audio_tc")
@@ -141,11 +149,19 @@ def test_fp8_argument_checks_and_switch_off(monkeypatch):
     with pytest.raises(fd.FlashDiffError):                      # a non-positive activation scale
         fd.fd_set_fp8_operands(ctx, dict(args, a_scale=np.zeros_like(f8["a_scale"])))
     fd.fd_set_text_stream(ctx, {k: dev(v, torch.bfloat16) for k, v in gen.block_weights(wl, 80).items()})
-    with pytest.raises(fd.FlashDiffError) as ei:                # not together with a second stream
-        fd.fd_set_fp8_operands(ctx, args)
-    assert ei.value.status == fd.FD_ERR_UNSUPPORTED
-    fd.fd_set_text_stream(ctx, None)
     fd.fd_set_fp8_operands(ctx, args)
+    labels = gen.uniform_labels(wl)
+    inp = gen.step_inputs(wl, 2, labels)
+    buf = StepBuffers(wl, 1)
+    with pytest.raises(fd.FlashDiffError) as ei:                # a second stream without 8-bit operands of its own
+        gpu_step(ctx, wl, dev(inp["x_cur"], torch.bfloat16), dev(inp["cond"], torch.bfloat16), dev(labels),
+                 dev(np.ones((wl.B, wl.R), np.uint8)), buf)
+    assert ei.value.status == fd.FD_ERR_UNSUPPORTED
+    fd.fd_set_fp8_operands(ctx, args, text_stream=True)
+    gpu_step(ctx, wl, dev(inp["x_cur"], torch.bfloat16), dev(inp["cond"], torch.bfloat16), dev(labels),
+             dev(np.ones((wl.B, wl.R), np.uint8)), buf)
+    fd.fd_set_fp8_operands(ctx, None, text_stream=True)
+    fd.fd_set_text_stream(ctx, None)
     fd.fd_set_fp8_operands(ctx, None)
     assert fd.fd_destroy(ctx) == fd.FD_OK
     _run_sequence(wl, 2, fd.FD_ENGINE_TC, _masks(wl))           # without it the block is what it was

@@ -88,6 +88,12 @@ def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=
         fd.fd_set_fp8_operands(ctx, dict({"w8_" + k: dev(f8["c_" + k]) for k in ("qkv", "fc1", "fc2")},
                                          **{"s_" + k: dev(f8["s_" + k]) for k in ("qkv", "fc1", "fc2")}, a_scale=f8["a_scale"]))
         variants = dict(variants or {}, fp8=f8)
+        if text_seed is not None:                                # the second stream quantises with operands of its own
+            f8t = gen.fp8_operands(wl, wt, text_seed, n_blocks=L)
+            fd.fd_set_fp8_operands(ctx, dict({"w8_" + k: dev(f8t["c_" + k]) for k in ("qkv", "fc1", "fc2")},
+                                             **{"s_" + k: dev(f8t["s_" + k]) for k in ("qkv", "fc1", "fc2")},
+                                             a_scale=f8t["a_scale"]), text_stream=True)
+            variants["text"] = dict(variants["text"], fp8=f8t)
     B, N, H = wl.B, wl.N, wl.H
     kv_ref = np.zeros((L, B, 2, N, H), np.float32)
     y_ref = np.zeros((B, N, H), np.float32)
@@ -109,6 +115,8 @@ def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=
             # first and 1.6e-2 after the second, that is up to ~0.6 of the rounding noise the format itself adds.  So
             # the bounds widen by 0.6 of what FP8 changes in the oracle (same state, same inputs, operands unquantised).
             plain = {k: v for k, v in (variants or {}).items() if k != "fp8"}
+            if "text" in plain:
+                plain["text"] = {k: v for k, v in plain["text"].items() if k != "fp8"}
             kv_p, y_p = kv_ref.copy(), y_ref.copy()
             oracle.regional_step(x_np, inp["cond"], labels, mask, w, kv_p, y_p, wl.heads, wl.R, n_blocks=L, variants=plain or None)
         o_idx, o_cu = oracle.regional_step(x_np, inp["cond"], labels, mask, w, kv_ref, y_ref, wl.heads, wl.R,

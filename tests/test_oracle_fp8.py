@@ -150,3 +150,48 @@ def test_dense_block_with_fp8_operands_against_torch_fp64():
     assert np.quantile(err, 0.999) <= 2e-5 and err.max() <= 5e-3
     np.testing.assert_allclose(kv[:, 0], k.numpy(), rtol=0, atol=5e-3)
     assert np.quantile(np.abs(kv[:, 0] - k.numpy()), 0.999) <= 2e-5
+
+
+# ---- FP8 operands with two streams: each stream has its own quantised weights and activation scales ----
+WL2 = gen.workload("tiny").replace(name="q2", H=64, heads=2, head_dim=32, M=128, Hc=48, grid=(40,), n_text=8, B=2, R=5, D=8,
+                                   L=2, labels="segments")
+
+
+def _setup2(seed):
+    w = gen.block_weights(WL2, seed)
+    wt = gen.block_weights(WL2, seed + 100)
+    labels = gen.uniform_labels(WL2)
+    inp = gen.step_inputs(WL2, seed, labels)
+    return w, wt, labels, inp
+
+
+def test_same_fp8_operands_in_both_streams_is_the_single_stream_bit_for_bit():
+    w, _, labels, inp = _setup2(8)
+    f8 = gen.fp8_operands(WL2, w, 8)
+    one = {"fp8": f8}
+    two = {"fp8": f8, "text": {"weights": w, "n_text": WL2.n_text, "fp8": f8}}
+    y1, kv1 = oracle.dense_step(inp["x_cur"], inp["cond"], w, WL2.heads, variants=one)
+    y2, kv2 = oracle.dense_step(inp["x_cur"], inp["cond"], w, WL2.heads, variants=two)
+    assert np.array_equal(y1.view(np.uint32), y2.view(np.uint32)) and np.array_equal(kv1.view(np.uint32), kv2.view(np.uint32))
+
+
+def test_all_active_equals_dense_bit_for_bit_with_fp8_operands_in_two_streams():
+    w, wt, labels, inp = _setup2(9)
+    var = {"fp8": gen.fp8_operands(WL2, w, 9), "text": {"weights": wt, "n_text": WL2.n_text, "fp8": gen.fp8_operands(WL2, wt, 10)}}
+    B, N, H = inp["x_cur"].shape
+    y_d, kv_d = oracle.dense_step(inp["x_cur"], inp["cond"], w, WL2.heads, variants=var)
+    kv = np.full((WL2.L, B, 2, N, H), np.nan, np.float32)
+    y = np.full((B, N, H), np.nan, np.float32)
+    oracle.regional_step(inp["x_cur"], inp["cond"], labels, np.ones((B, WL2.R), np.uint8), w, kv, y, WL2.heads, WL2.R, variants=var)
+    assert np.array_equal(y.view(np.uint32), y_d.view(np.uint32)) and np.array_equal(kv.view(np.uint32), kv_d.view(np.uint32))
+    # the text rows really go through their own 8-bit operands: swapping the text stream's set changes them
+    var2 = dict(var, text=dict(var["text"], fp8=gen.fp8_operands(WL2, wt, 11)))
+    y_o, _ = oracle.dense_step(inp["x_cur"], inp["cond"], w, WL2.heads, variants=var2)
+    assert np.abs(y_o - y_d)[:, WL2.n_grid:].max() > 1e-5
+
+
+def test_one_streams_fp8_operands_without_the_others_are_refused():
+    w, wt, labels, inp = _setup2(12)
+    with pytest.raises(Exception):
+        oracle.dense_step(inp["x_cur"], inp["cond"], w, WL2.heads,
+                          variants={"fp8": gen.fp8_operands(WL2, w, 12), "text": {"weights": wt, "n_text": WL2.n_text}})
