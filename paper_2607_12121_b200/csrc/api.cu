@@ -162,6 +162,14 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     QTile* tiles = c->at<QTile>(l.tiles);
     QTile* tiles2 = c->use_tc_attn ? tiles + l.tile_cap : nullptr;
     const int rows_cap = B * N;
+    // what the switches set on the context ask of this step, checked before anything is launched
+    const bool dual = c->dual;
+    const fd_cross_attention& xa = c->cross;
+    if (xa.w_q && B != xa.ctx_batch)
+        return c->fail(FD_ERR_SHAPE, "B=%d differs from the cross-attention context's batch %d", B, xa.ctx_batch);
+    const bool f8 = c->fp8.w8_qkv != nullptr;
+    if (f8 && dual && !c->fp8_text.w8_qkv)
+        return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands with a second stream need that stream's operands too (fd_set_fp8_text_stream)");
     int nl = 0;
     cudaError_t e;
 #define FD_TRY(group, call)                                                                              \
@@ -181,7 +189,6 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     FD_TRY(FD_PROF_ADALN, launch_adaln<T>(cond, static_cast<const T*>(c->w.w_ada), static_cast<const T*>(c->w.b_ada), mod, L, B, H,
                            Hc, c->ws + l.ada_act, st, &nl));
     // dual stream: tokens with label R use a second weight set for everything that acts per token
-    const bool dual = c->dual;
     const long long text_mod_off = (long long)L * B * 6 * H;         // second stream's adaLN vectors follow the first's
     int32_t* text128 = c->at<int32_t>(l.text_tiles);
     int32_t* text256 = text128 + l.Mcap / 128 + 1;
@@ -199,14 +206,8 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
     };
     const int n_pass = dual ? 2 : 1;
     const int max_tiles = B * ((N + c->tile_rows - 1) / c->tile_rows);
-    const fd_cross_attention& xa = c->cross;
-    if (xa.w_q && B != xa.ctx_batch)
-        return c->fail(FD_ERR_SHAPE, "B=%d differs from the cross-attention context's batch %d", B, xa.ctx_batch);
     const float* zeros = c->at<float>(l.consts);
     const float* ones = zeros + H;
-    const bool f8 = c->fp8.w8_qkv != nullptr;
-    if (f8 && dual && !c->fp8_text.w8_qkv)
-        return c->fail(FD_ERR_UNSUPPORTED, "FP8 operands with a second stream need that stream's operands too (fd_set_fp8_text_stream)");
     const fd_fp8_operands* f8ops[2] = {&c->fp8, &c->fp8_text};
     const std::vector<float>* f8a[2] = {&c->fp8_a, &c->fp8_text_a};
     const bool pdl = c->use_tc && c->tc && tc_plan_pdl(c->tc);
