@@ -449,6 +449,56 @@ class Engine:
                                      "frac_burst": round(t["frac_burst"] / 2, 3), "frac_sustained": round(t["frac_sustained"] / 2, 3)}
         return out
 
+    def variants_measure(self, steps, ms_plain, fraction=None):
+        """The same gated step with the block variants of the paper's models switched on, one at a time: QK-RMSNorm +
+        rotary embedding, cross-attention to a 512-token context, and (workloads with text tokens) a second weight set
+        for the always-active tokens.  Step time and the cost against the plain step on the same active set."""
+        torch, fd, wl, dev = self.torch, self.fd, self.wl, self.dev
+        L, H, B, N = wl.L, wl.H, wl.B, wl.N
+        g = torch.Generator(device=dev)
+        g.manual_seed(self.seed + 17)
+        self.set_fraction(fraction)
+
+        def draw(shape, std, mean=0.0, dt=None):
+            t = torch.empty(shape, dtype=torch.float32, device=dev)
+            t.normal_(mean, std, generator=g)
+            return t.to(self.dt if dt is None else dt).contiguous()
+
+        def timed_step():
+            for _ in range(3):
+                self.gated_step()
+            return self.timed(self.gated_step, steps)
+
+        out = {}
+        try:
+            half = wl.head_dim // 2
+            ang = torch.arange(N, device=dev, dtype=torch.float32)[:, None] * \
+                (10000.0 ** (-torch.arange(half, device=dev, dtype=torch.float32) / half))[None, :]
+            fd.fd_set_block_variants(self.ctx, q_norm_w=draw((L, wl.head_dim), 0.1, 1.0), k_norm_w=draw((L, wl.head_dim), 0.1, 1.0),
+                                     rope_cos=torch.cos(ang).contiguous(), rope_sin=torch.sin(ang).contiguous())
+            ms = timed_step()
+            fd.fd_set_block_variants(self.ctx)
+            out["qk_norm_rope"] = {"step_ms": round(ms, 4), "extra": round(ms / ms_plain - 1.0, 4)}
+            T = 512
+            fd.fd_set_cross_attention(self.ctx, {"w_q": draw((L, H, H), 0.02), "b_q": draw((L, H), 0.02), "w_o": draw((L, H, H), 0.02),
+                                                 "b_o": draw((L, H), 0.02), "ctx_kv": draw((L, B, 2, T, H), 0.5)})
+            ms = timed_step()
+            fd.fd_set_cross_attention(self.ctx, None)
+            extra_flops = L * (4.0 * H * H + 4.0 * T * H)            # per active row: two projections + the attention
+            out["cross_attention"] = {"context_tokens": T, "step_ms": round(ms, 4), "extra": round(ms / ms_plain - 1.0, 4),
+                                      "extra_flops_per_active_row": extra_flops}
+            if wl.n_text > 0:
+                fd.fd_set_text_stream(self.ctx, device_weights(wl, self.seed + 29, dev))
+                ms = timed_step()
+                fd.fd_set_text_stream(self.ctx, None)
+                out["dual_stream"] = {"text_tokens_per_request": wl.n_text, "step_ms": round(ms, 4),
+                                      "extra": round(ms / ms_plain - 1.0, 4)}
+        except fd.FlashDiffError as e:
+            out["unavailable"] = str(e)
+        self.dense_step(self.x_prev)                      # the cached state as the plain step left it
+        torch.cuda.empty_cache()
+        return out
+
     def close(self):
         st = self.fd.fd_destroy(self.ctx)
         self.__dict__.clear()                 # drops the weights, caches and inputs
@@ -467,6 +517,7 @@ def side_workload(name, seed, dev, rep, steps, warmup, peaks):
     if sweep:
         res["sweep"] = sweep
     res["fp8_operands"] = eng.fp8_measure(steps, peaks, res["step_ms"])
+    res["variants"] = eng.variants_measure(max(5, steps // 2), res["step_ms"])
     eng.close()
     del eng
     torch.cuda.empty_cache()
@@ -673,9 +724,10 @@ def run_ours(args):
             r, _, _ = eng.measure(max(5, args.steps // 4), 3, peaks, fraction=f, kernels=False, dense_ms=ms_dense)
             sweep[tag] = {k: r[k] for k in ("active_fraction", "step_ms", "tflops", "speedup_vs_dense", "t_over_f_dense")}
     weight_gb = sum(t.numel() * t.element_size() for t in eng.weights.values()) / 1e9
-    fp8 = None
+    fp8 = variants = None
     if world == 1 and not args.no_extras:
         fp8 = eng.fp8_measure(max(5, args.steps // 2), peaks, ms_reg, args.fraction)
+        variants = eng.variants_measure(max(5, args.steps // 2), ms_reg, args.fraction)
     st_destroy = eng.close()
     del eng, x, cond, y, z_cur, z_prev, eps
     torch.cuda.empty_cache()
@@ -704,7 +756,7 @@ def run_ours(args):
         "step_tflops": round(value / world, 1), "step_frac_burst": round(value / world / burst, 4),
         "step_frac_sustained": round(value / world / sust, 4),
         "kernels": breakdown, "sweep": sweep, "workloads": others,
-        "activity_probe": probe, "fp8_operands": fp8,
+        "activity_probe": probe, "fp8_operands": fp8, "variants": variants,
     }
 
     line = {

@@ -18,7 +18,8 @@
  * restricted forms of a kernel and are not part of the interface: FD_PDL=0 (fully serialised
  * launches), FD_TC_PAIR=0 (single-CTA GEMM tiles), FD_TMA_RESID=0 (per-thread residual
  * reductions), FD_ATT_SPLIT=0|2 (never / always cut attention items along the keys),
- * FD_TC_MAX_CTAS=n (cap on persistent CTAs).
+ * FD_TC_MAX_CTAS=n (cap on persistent CTAs), FD_ATT_PAIR=1 (CTA-pair attention kernel at head dim 128), and, read at
+ * every step, FD_TC_GROUPED=0 (dual stream: one launch per stream and projection instead of one grouped launch).
  */
 #ifndef FLASHDIFF_H_
 #define FLASHDIFF_H_
@@ -198,8 +199,9 @@ fd_status fd_set_block_variants(fd_ctx* ctx, const fd_block_variants* v);
  * b_ada), the QKV projection, the QK-norm weights, the out-projection and the MLP -- while the attention stays joint
  * over all tokens of the request.  The second stream is the always-active tokens (label R: the text tokens of a
  * joint text-image request); `text_weights` has the layout of fd_weights and is borrowed until the next call or
- * fd_destroy.  NULL returns to a single stream.  Each projection then runs as two launches: one finishes the first
- * stream's rows, one walks only the row tiles that hold rows of the second stream.
+ * fd_destroy.  NULL returns to a single stream.  Each projection then walks every row tile with the first stream's
+ * weights and, in the same launch, the row tiles that hold rows of the second stream with the second stream's
+ * weights; a tile's epilogue finishes only the rows of its own stream.
  */
 fd_status fd_set_text_stream(fd_ctx* ctx, const fd_weights* text_weights);
 

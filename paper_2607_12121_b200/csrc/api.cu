@@ -243,7 +243,18 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             ep.q_head_pad = tc_attention_head_pad(cf.head_dim);
         }
         ep.kv = kv_b;
-        for (int pass = 0; pass < n_pass; ++pass) {
+        // (dual stream: one grouped launch where the CTA-pair kernel runs the projection, else one launch per stream)
+        const bool grp_qkv = dual && c->use_tc && tc_plan_grouped(c->tc, TC_GEMM_QKV);
+        if (grp_qkv) {
+            ep.bias = stream_ptr(c->w.b_qkv, c->text_w.b_qkv, (size_t)blk * 3 * H, 0);
+            ep.bias2 = stream_ptr(c->w.b_qkv, c->text_w.b_qkv, (size_t)blk * 3 * H, 1);
+            if (f8) {
+                ep.col_scale = f8ops[0]->s_qkv + (size_t)blk * 3 * H; ep.act_scale = a8[0][0];
+                ep.col_scale2 = f8ops[1]->s_qkv + (size_t)blk * 3 * H; ep.act_scale2 = a8[1][0];
+            }
+            FD_TRY(FD_PROF_GEMM_QKV, tc_gemm_both(c->tc, TC_GEMM_QKV, blk, ep, ctl, st, &nl, f8));
+        }
+        for (int pass = 0; pass < n_pass && !grp_qkv; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_qkv, c->text_w.b_qkv, (size_t)blk * 3 * H, pass);
             if (f8) {
@@ -288,7 +299,13 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         ep.resid = resid;
         ep.gate = mod_b + 2 * H;
         ep.y = nullptr;
-        for (int pass = 0; pass < n_pass; ++pass) {
+        const bool grp_out = dual && c->use_tc && tc_plan_grouped(c->tc, TC_GEMM_OUT);
+        if (grp_out) {
+            ep.bias = stream_ptr(c->w.b_o, c->text_w.b_o, (size_t)blk * H, 0);
+            ep.bias2 = stream_ptr(c->w.b_o, c->text_w.b_o, (size_t)blk * H, 1);
+            FD_TRY(FD_PROF_GEMM_OUT, tc_gemm_both(c->tc, TC_GEMM_OUT, blk, ep, ctl, st, &nl, false));
+        }
+        for (int pass = 0; pass < n_pass && !grp_out; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_o, c->text_w.b_o, (size_t)blk * H, pass);
             if (c->use_tc)
@@ -330,7 +347,17 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
                                      H, rows_cap, cf.ln_eps, ctl, st, &nl, pdl, ts2, f8 ? 1.0f / a8[0][1] : 0.f));
         ep.out = g;
         ep.out_ld = M;
-        for (int pass = 0; pass < n_pass; ++pass) {
+        const bool grp_fc1 = dual && c->use_tc && tc_plan_grouped(c->tc, TC_GEMM_FC1);
+        if (grp_fc1) {
+            ep.bias = stream_ptr(c->w.b_fc1, c->text_w.b_fc1, (size_t)blk * M, 0);
+            ep.bias2 = stream_ptr(c->w.b_fc1, c->text_w.b_fc1, (size_t)blk * M, 1);
+            if (f8) {
+                ep.col_scale = f8ops[0]->s_fc1 + (size_t)blk * M; ep.act_scale = a8[0][1]; ep.out_inv_scale = 1.0f / a8[0][2];
+                ep.col_scale2 = f8ops[1]->s_fc1 + (size_t)blk * M; ep.act_scale2 = a8[1][1]; ep.out_inv_scale2 = 1.0f / a8[1][2];
+            }
+            FD_TRY(FD_PROF_GEMM_FC1, tc_gemm_both(c->tc, TC_GEMM_FC1, blk, ep, ctl, st, &nl, f8));
+        }
+        for (int pass = 0; pass < n_pass && !grp_fc1; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_fc1, c->text_w.b_fc1, (size_t)blk * M, pass);
             if (f8) {
@@ -346,7 +373,17 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         }
         ep.gate = mod_b + 5 * H;
         ep.y = (blk == L - 1) ? y_ : nullptr;       // the last block scatters the rows back
-        for (int pass = 0; pass < n_pass; ++pass) {
+        const bool grp_fc2 = dual && c->use_tc && tc_plan_grouped(c->tc, TC_GEMM_FC2);
+        if (grp_fc2) {
+            ep.bias = stream_ptr(c->w.b_fc2, c->text_w.b_fc2, (size_t)blk * H, 0);
+            ep.bias2 = stream_ptr(c->w.b_fc2, c->text_w.b_fc2, (size_t)blk * H, 1);
+            if (f8) {
+                ep.col_scale = f8ops[0]->s_fc2 + (size_t)blk * H; ep.act_scale = a8[0][2];
+                ep.col_scale2 = f8ops[1]->s_fc2 + (size_t)blk * H; ep.act_scale2 = a8[1][2];
+            }
+            FD_TRY(FD_PROF_GEMM_FC2, tc_gemm_both(c->tc, TC_GEMM_FC2, blk, ep, ctl, st, &nl, f8));
+        }
+        for (int pass = 0; pass < n_pass && !grp_fc2; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_fc2, c->text_w.b_fc2, (size_t)blk * H, pass);
             if (f8) {

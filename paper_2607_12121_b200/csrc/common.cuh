@@ -100,6 +100,11 @@ struct EpiParams {
     const float* col_scale;    // [n_out] f32
     float act_scale;
     float out_inv_scale;
+    // dual stream in one launch (the grouped form of the CTA-pair kernel): what the second stream's tiles use instead
+    const void* bias2;
+    const float* col_scale2;
+    float act_scale2;
+    float out_inv_scale2;
 };
 
 // Per-row choice of the second stream's adaLN vectors in the row kernels (labels == nullptr: single stream).

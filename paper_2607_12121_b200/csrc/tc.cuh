@@ -40,6 +40,10 @@ bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const vo
                      bool text = false);
 cudaError_t tc_gemm_fp8(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
                         int* n_launch, bool text_pass = false);
+// dual stream in one launch (the grouped form of the CTA-pair kernel): true where it can run this projection
+bool tc_plan_grouped(TcPlan* p, TcGemmKind kind);
+cudaError_t tc_gemm_both(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
+                         int* n_launch, bool fp8);
 // cross-attention: tensor maps of its two [L, H, H] projection weights (both nullptr: off)
 bool tc_plan_set_cross(TcPlan* p, const void* w_q, const void* w_o, std::string* err);
 // region_mass (optional): [B, R] f64, receives the own-region softmax mass

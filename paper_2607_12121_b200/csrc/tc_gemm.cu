@@ -176,11 +176,14 @@ template <int PAIR_BN> struct PairCfg {
 
 // F8: both operands are E4M3 bytes; a stage holds the same bytes and thus twice the depth of K (128 values), the
 // products are kind::f8f6f4 and the epilogue scales the accumulator (see EpiParams).
-template <int KIND, int PAIR_BN, bool F8 = false>
+// GROUPED (dual stream in one launch): the tile sequence is every row tile with the first stream's weights (tm_b),
+// followed by the listed row tiles -- those that hold rows of the second stream -- with the second stream's weights
+// (tm_b2); a tile's epilogue finishes only the rows of its own stream.
+template <int KIND, int PAIR_BN, bool F8 = false, bool GROUPED = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                     const __grid_constant__ CUtensorMap tm_r, int n_out, int k_dim, int stream_a, int tma_resid, EpiParams ep,
-                    Control* ctl, const int32_t* __restrict__ m_list) {
+                    Control* ctl, const int32_t* __restrict__ m_list, const __grid_constant__ CUtensorMap tm_b2) {
     constexpr int PAIR_B_BYTES = PairCfg<PAIR_BN>::B_BYTES, PAIR_STAGE_BYTES = PairCfg<PAIR_BN>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -205,6 +208,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         fence_barrier_init();
         prefetch_tmap(&tm_a);
         prefetch_tmap(&tm_b);
+        if (GROUPED) prefetch_tmap(&tm_b2);
     }
     if (warp == 1) {
         tmem_alloc_pair(tmem_slot, PairCfg<PAIR_BN>::TMEM_COLS);
@@ -220,9 +224,20 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     pdl_wait();
     const int a_total = ctl->a_total;
     // 256-row tiles: all of them, or (dual stream, second pass) the listed ones that hold rows of the second stream
-    const int m_pairs = m_list ? ctl->n_text_tiles[1] : (a_total + 2 * BM - 1) / (2 * BM);
+    const int m_all = (a_total + 2 * BM - 1) / (2 * BM);
+    const int m_pairs = GROUPED ? m_all : (m_list ? ctl->n_text_tiles[1] : m_all);
     const int n_tiles = n_out / PAIR_BN;
-    const int total_tiles = m_pairs * n_tiles;
+    const int tiles0 = m_pairs * n_tiles;                                  // GROUPED: the first stream's tiles come first
+    const int total_tiles = tiles0 + (GROUPED ? ctl->n_text_tiles[1] * n_tiles : 0);
+    // row tile, column tile and stream of the tile at position `tile` of the sequence
+    auto locate = [&](int tile, int& m, int& n, int& grp) {
+        if (GROUPED && tile >= tiles0) {
+            const int t2 = tile - tiles0;
+            m = m_list[t2 / n_tiles]; n = t2 % n_tiles; grp = 1;
+        } else {
+            m = (!GROUPED && m_list) ? m_list[tile / n_tiles] : tile / n_tiles; n = tile % n_tiles; grp = 0;
+        }
+    };
     constexpr int BKE = F8 ? 2 * BK : BK;               // values of K per stage (128 bytes per row either way)
     const int k_tiles = k_dim / BKE;
 
@@ -232,7 +247,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             bool ok = true;
             const uint64_t evict_first = l2_evict_first();
             for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
-                const int m = m_list ? m_list[tile / n_tiles] : tile / n_tiles, n = tile % n_tiles;
+                int m, n, grp;
+                locate(tile, m, n, grp);
+                const CUtensorMap* wmap = (GROUPED && grp) ? &tm_b2 : &tm_b;
                 for (int kt = 0; kt < k_tiles; ++kt, ++it) {
                     const int s = it % PAIR_STAGES;
                     const uint32_t ph = (it / PAIR_STAGES) & 1;
@@ -243,7 +260,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                         tma_load_2d_pair_hint(sA + s * A_TILE_BYTES, &tm_a, kt * BKE, m * 2 * BM + (int)rank * BM, bar, evict_first);
                     else
                         tma_load_2d_pair(sA + s * A_TILE_BYTES, &tm_a, kt * BKE, m * 2 * BM + (int)rank * BM, bar);
-                    tma_load_2d_pair(sB + s * PAIR_B_BYTES, &tm_b, kt * BKE, n * PAIR_BN + (int)rank * (PAIR_BN / 2), bar);
+                    tma_load_2d_pair(sB + s * PAIR_B_BYTES, wmap, kt * BKE, n * PAIR_BN + (int)rank * (PAIR_BN / 2), bar);
                 }
             }
             if (!ok) report(ctl, FD_ERR_TIMEOUT, 700 + (int)blockIdx.x);
@@ -286,8 +303,19 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         const int c_lo = chalf == 0 ? 0 : C_SPLIT, c_hi = chalf == 0 ? C_SPLIT : PAIR_BN;
         uint32_t t_it = 0;
         bool ok = true;
+        const void* bias0 = ep.bias;
+        const float* col_scale0 = ep.col_scale;
+        const float act_scale0 = ep.act_scale, out_inv_scale0 = ep.out_inv_scale;
         for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
-            const int m = m_list ? m_list[tile / n_tiles] : tile / n_tiles, n = tile % n_tiles;
+            int m, n, grp;
+            locate(tile, m, n, grp);
+            if constexpr (GROUPED) {                        // this tile's stream: its rows, bias and scales
+                ep.group = grp;
+                ep.bias = grp ? ep.bias2 : bias0;
+                ep.col_scale = grp ? ep.col_scale2 : col_scale0;
+                ep.act_scale = grp ? ep.act_scale2 : act_scale0;
+                ep.out_inv_scale = grp ? ep.out_inv_scale2 : out_inv_scale0;
+            }
             const uint32_t acc = t_it & 1, aph = (t_it >> 1) & 1;
             if (KIND == EPI_RESID && ep.y)
                 epilogue_prefetch_resid(ep, lane, m * 2 * BM + (int)rank * BM + quad * 32, a_total,
@@ -494,6 +522,14 @@ TcPlan* tc_plan_create(const fd_config& cfg, const fd_weights& w, const TcBuffer
         FD_SET_PAIR8(EPI_QKV, 256) FD_SET_PAIR8(EPI_RESID, 256) FD_SET_PAIR8(EPI_GELU, 256)
         FD_SET_PAIR8(EPI_QKV, 192) FD_SET_PAIR8(EPI_RESID, 192) FD_SET_PAIR8(EPI_GELU, 192)
 #undef FD_SET_PAIR8
+#define FD_SET_PAIRG(K, N, F)                                                                              \
+    if (e == cudaSuccess)                                                                                  \
+        e = cudaFuncSetAttribute(tc_gemm_pair_kernel<K, N, F, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<N>::SMEM);
+        FD_SET_PAIRG(EPI_QKV, 256, false) FD_SET_PAIRG(EPI_RESID, 256, false) FD_SET_PAIRG(EPI_GELU, 256, false)
+        FD_SET_PAIRG(EPI_QKV, 192, false) FD_SET_PAIRG(EPI_RESID, 192, false) FD_SET_PAIRG(EPI_GELU, 192, false)
+        FD_SET_PAIRG(EPI_QKV, 256, true) FD_SET_PAIRG(EPI_RESID, 256, true) FD_SET_PAIRG(EPI_GELU, 256, true)
+        FD_SET_PAIRG(EPI_QKV, 192, true) FD_SET_PAIRG(EPI_RESID, 192, true) FD_SET_PAIRG(EPI_GELU, 192, true)
+#undef FD_SET_PAIRG
         if (e != cudaSuccess) {
             ok = false;
             if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
@@ -649,6 +685,48 @@ bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const vo
     return ok;
 }
 
+// Dual stream in one launch: every row tile with the first stream's weights, then the row tiles that hold rows of the
+// second stream with the second stream's weights (ep.bias2 and, with FP8 operands, ep.col_scale2 / act_scale2 /
+// out_inv_scale2 are that stream's).  Available where the CTA-pair kernel runs the projection (switch FD_TC_GROUPED=0
+// keeps the two launches).
+bool tc_plan_grouped(TcPlan* p, TcGemmKind kind) {
+    const char* v = getenv("FD_TC_GROUPED");
+    const bool on = !v || atoi(v) != 0;
+    return on && kind <= TC_GEMM_FC2 && p->spec[kind].pair_bn != 0 && p->w_maps_text != nullptr;
+}
+
+cudaError_t tc_gemm_both(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
+                         int* n_launch, bool fp8) {
+    if (!tc_plan_grouped(p, kind)) return cudaErrorInvalidValue;
+    const GemmSpec& s = p->spec[kind];
+    const int g = kind == TC_GEMM_QKV ? 0 : kind == TC_GEMM_FC1 ? 1 : 2;
+    if (fp8 && (!p->w_maps_f8 || !p->w_maps_f8_text || kind == TC_GEMM_OUT)) return cudaErrorInvalidValue;
+    const CUtensorMap& wm = fp8 ? p->w_maps_f8[(size_t)blk * 3 + g] : p->w_maps[(size_t)blk * 4 + kind];
+    const CUtensorMap& wm2 = fp8 ? p->w_maps_f8_text[(size_t)blk * 3 + g] : p->w_maps_text[(size_t)blk * 4 + kind];
+    const CUtensorMap& am = fp8 ? p->a_maps_f8[kind == TC_GEMM_FC2 ? 1 : 0] : s.a;
+    Control* c = const_cast<Control*>(ctl);
+    const int pgrid = max(2, min(p->sm_count & ~1, p->pair_ctas));
+    const int stream_a = kind == TC_GEMM_FC2 ? 1 : 0;
+    cudaError_t e = cudaSuccess;
+#define FD_LAUNCH_BOTH(K, N, F)                                                                                          \
+    e = launch_kernel(tc_gemm_pair_kernel<K, N, F, true>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, am, wm, p->resid_map, \
+                      s.n_out, s.k, stream_a, p->tma_resid ? 1 : 0, ep, c, p->text_list256, wm2)
+#define FD_LAUNCH_BOTH_N(K, F) do { if (s.pair_bn == 256) FD_LAUNCH_BOTH(K, 256, F); else FD_LAUNCH_BOTH(K, 192, F); } while (0)
+    if (fp8) {
+        if (kind == TC_GEMM_QKV) FD_LAUNCH_BOTH_N(EPI_QKV, true);
+        else if (kind == TC_GEMM_FC1) FD_LAUNCH_BOTH_N(EPI_GELU, true);
+        else FD_LAUNCH_BOTH_N(EPI_RESID, true);
+    } else {
+        if (kind == TC_GEMM_QKV) FD_LAUNCH_BOTH_N(EPI_QKV, false);
+        else if (kind == TC_GEMM_FC1) FD_LAUNCH_BOTH_N(EPI_GELU, false);
+        else FD_LAUNCH_BOTH_N(EPI_RESID, false);
+    }
+#undef FD_LAUNCH_BOTH_N
+#undef FD_LAUNCH_BOTH
+    ++*n_launch;
+    return e;
+}
+
 cudaError_t tc_gemm_fp8(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
                         int* n_launch, bool text_pass) {
     const CUtensorMap* maps = text_pass ? p->w_maps_f8_text : p->w_maps_f8;
@@ -664,7 +742,7 @@ cudaError_t tc_gemm_fp8(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep
     cudaError_t e = cudaSuccess;
 #define FD_LAUNCH_PAIR8(K, N) \
     e = launch_kernel(tc_gemm_pair_kernel<K, N, true>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, am, wm, p->resid_map, s.n_out, \
-                      s.k, stream_a, p->tma_resid ? 1 : 0, ep, c, no_list)
+                      s.k, stream_a, p->tma_resid ? 1 : 0, ep, c, no_list, wm)
     if (kind == TC_GEMM_QKV) {
         if (s.pair_bn == 256) FD_LAUNCH_PAIR8(EPI_QKV, 256); else FD_LAUNCH_PAIR8(EPI_QKV, 192);
     } else if (kind == TC_GEMM_FC1) {
@@ -699,7 +777,7 @@ cudaError_t tc_gemm(TcPlan* p, TcGemmKind kind_in, int blk, const EpiParams& ep,
         cudaError_t e = cudaSuccess;
 #define FD_LAUNCH_PAIR(K, N) \
     e = launch_kernel(tc_gemm_pair_kernel<K, N>, pgrid, GEMM_THREADS, PairCfg<N>::SMEM, st, p->pdl, s.a, wm, p->resid_map, s.n_out, s.k, \
-                      stream_a, p->tma_resid ? 1 : 0, ep, c, m_list)
+                      stream_a, p->tma_resid ? 1 : 0, ep, c, m_list, wm)
         if (kind == TC_GEMM_QKV) {
             if (s.pair_bn == 256) FD_LAUNCH_PAIR(EPI_QKV, 256); else FD_LAUNCH_PAIR(EPI_QKV, 192);
         } else if (kind == TC_GEMM_FC1) {

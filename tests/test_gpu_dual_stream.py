@@ -37,6 +37,12 @@ def test_dual_stream_row_tile_lists(n_text, B):
     _run_sequence(wl, 3, fd.FD_ENGINE_TC, masks, text_seed=78)
 
 
+def test_dual_stream_as_two_launches_per_projection(monkeypatch):
+    monkeypatch.setenv("FD_TC_GROUPED", "0")                   # not the grouped launch: one launch per stream
+    wl = gen.workload("mmdit_tc")
+    _run_sequence(wl, 5, fd.FD_ENGINE_TC, _masks(wl), variants=gen.block_variants(wl, 9), text_seed=81)
+
+
 def test_dual_stream_with_single_cta_gemm_tiles(monkeypatch):
     monkeypatch.setenv("FD_TC_PAIR", "0")                      # the 128-row tile list
     wl = gen.workload("mmdit_tc").replace(L=1)
