@@ -6,7 +6,9 @@ gate (activity score + mask) -> compaction -> all transformer blocks on the acti
 Headline workload: the 480p video configuration (30 blocks, hidden 1536, 12 heads x 128, 32760 tokens,
 256 regions), the largest one that fits a single GPU.  With one GPU the audio, image and joint text-image
 configurations are measured as well (step, dense step, per-kernel rates) and the active fraction is swept;
-all of it lands inside the line's `roofline` object.
+all of it lands inside the line's `roofline` object, together with the same step with FP8 operands for three of the
+four projections (`fp8_operands`) and with the block variants of the paper's models switched on one at a time
+(`variants`: QK-RMSNorm + rotary embedding, cross-attention, a second weight set for the text tokens).
 
   python bench.py --gpus 1 --steps 20 --warmup 5
   python bench.py --gpus 4                 # starts 4 replicas (one process per GPU) by itself
