@@ -472,6 +472,8 @@ class Engine:
             return self.timed(self.gated_step, steps)
 
         out = {}
+        ms_plain = timed_step()                           # measured again here: the clock drifts over a long run
+        out["plain_step_ms"] = round(ms_plain, 4)
         try:
             half = wl.head_dim // 2
             ang = torch.arange(N, device=dev, dtype=torch.float32)[:, None] * \

@@ -279,7 +279,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
                                                                c->var.rope_cos, c->var.rope_sin, rows_cap, ctl, st, &nl,
                                                                text_norm ? norm_w(c->var.q_norm_w_text) : nullptr,
                                                                text_norm ? norm_w(c->var.k_norm_w_text) : nullptr,
-                                                               text_norm ? labels : nullptr, R));
+                                                               text_norm ? labels : nullptr, R, pdl));
         }
         // active queries against all N keys of their request (joint over both streams); the first block can also
         // report, per region, the softmax mass its queries put on keys of their own region (paper Sec. 4.2)

@@ -163,7 +163,7 @@ cudaError_t launch_qk_variants(T* q, int q_ld, int q_head_stride, T* kv_block, c
                                int heads, int dh, const T* qn_w, const T* kn_w, float eps, const float* rope_cos,
                                const float* rope_sin, int rows_cap, const Control* ctl, cudaStream_t st, int* n_launch,
                                const T* qn_w_text = nullptr, const T* kn_w_text = nullptr, const int32_t* labels = nullptr,
-                               int R = 0);
+                               int R = 0, bool pdl = false);
 
 // simt_block.cu
 template <typename T>

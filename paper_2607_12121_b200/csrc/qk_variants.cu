@@ -6,6 +6,7 @@
 // K row the projection has just written into the cache, in place, so the cache holds keys in their final form
 // and rows of skipped tokens are never touched.  Memory bound: reads and writes 2 * A * H elements.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace fd {
 
@@ -76,6 +77,7 @@ qk_variants_kernel(T* __restrict__ q, int q_ld, int q_head_stride, T* __restrict
                    const T* __restrict__ qn_w_text, const T* __restrict__ kn_w_text, const int32_t* __restrict__ labels, int R) {
     const int lane = threadIdx.x & 31;
     const int warps = gridDim.x * (QKV_THREADS / 32);
+    ptx::pdl_wait();                              // the rows come from the projection launched just before
     const long long units = (long long)ctl->a_total * heads;
     for (long long u = (long long)blockIdx.x * (QKV_THREADS / 32) + (threadIdx.x >> 5); u < units; u += warps) {
         const int row = (int)(u / heads), h = (int)(u - (long long)row * heads);
@@ -87,6 +89,7 @@ qk_variants_kernel(T* __restrict__ q, int q_ld, int q_head_stride, T* __restrict
         head_slice<T, MAXP>(q + (size_t)row * q_ld + (size_t)h * q_head_stride, dh, text ? qn_w_text : qn_w, eps, cs, sn, lane);
         head_slice<T, MAXP>(kv + (((size_t)b * 2 + 0) * N + j) * H + (size_t)h * dh, dh, text ? kn_w_text : kn_w, eps, cs, sn, lane);
     }
+    ptx::pdl_trigger();
 }
 
 }  // namespace
@@ -95,25 +98,28 @@ template <typename T>
 cudaError_t launch_qk_variants(T* q, int q_ld, int q_head_stride, T* kv_block, const int32_t* active_idx, int N, int H,
                                int heads, int dh, const T* qn_w, const T* kn_w, float eps, const float* rope_cos,
                                const float* rope_sin, int rows_cap, const Control* ctl, cudaStream_t st, int* n_launch,
-                               const T* qn_w_text, const T* kn_w_text, const int32_t* labels, int R) {
+                               const T* qn_w_text, const T* kn_w_text, const int32_t* labels, int R, bool pdl) {
     const long long max_units = (long long)rows_cap * heads;
     const int grid = (int)max(1LL, min((max_units + QKV_THREADS / 32 - 1) / (QKV_THREADS / 32), 148LL * 16));
+    // launched like its neighbours (programmatic stream serialization when the engine uses it): a plainly serialized
+    // launch between the projection and the attention would also break their overlap
+    cudaError_t e;
     if (dh <= 64)
-        qk_variants_kernel<T, 1><<<grid, QKV_THREADS, 0, st>>>(q, q_ld, q_head_stride, kv_block, active_idx, N, H, heads, dh, qn_w,
-                                                               kn_w, eps, rope_cos, rope_sin, ctl, qn_w_text, kn_w_text, labels, R);
+        e = ptx::launch_kernel(qk_variants_kernel<T, 1>, grid, QKV_THREADS, 0, st, pdl, q, q_ld, q_head_stride, kv_block, active_idx, N,
+                               H, heads, dh, qn_w, kn_w, eps, rope_cos, rope_sin, ctl, qn_w_text, kn_w_text, labels, R);
     else
-        qk_variants_kernel<T, 2><<<grid, QKV_THREADS, 0, st>>>(q, q_ld, q_head_stride, kv_block, active_idx, N, H, heads, dh, qn_w,
-                                                               kn_w, eps, rope_cos, rope_sin, ctl, qn_w_text, kn_w_text, labels, R);
+        e = ptx::launch_kernel(qk_variants_kernel<T, 2>, grid, QKV_THREADS, 0, st, pdl, q, q_ld, q_head_stride, kv_block, active_idx, N,
+                               H, heads, dh, qn_w, kn_w, eps, rope_cos, rope_sin, ctl, qn_w_text, kn_w_text, labels, R);
     ++*n_launch;
-    return cudaGetLastError();
+    return e;
 }
 
 template cudaError_t launch_qk_variants<float>(float*, int, int, float*, const int32_t*, int, int, int, int, const float*,
                                                const float*, float, const float*, const float*, int, const Control*,
-                                               cudaStream_t, int*, const float*, const float*, const int32_t*, int);
+                                               cudaStream_t, int*, const float*, const float*, const int32_t*, int, bool);
 template cudaError_t launch_qk_variants<__nv_bfloat16>(__nv_bfloat16*, int, int, __nv_bfloat16*, const int32_t*, int, int, int,
                                                        int, const __nv_bfloat16*, const __nv_bfloat16*, float, const float*,
                                                        const float*, int, const Control*, cudaStream_t, int*,
-                                                       const __nv_bfloat16*, const __nv_bfloat16*, const int32_t*, int);
+                                                       const __nv_bfloat16*, const __nv_bfloat16*, const int32_t*, int, bool);
 
 }  // namespace fd
