@@ -19,7 +19,8 @@
  * launches), FD_TC_PAIR=0 (single-CTA GEMM tiles), FD_TMA_RESID=0 (per-thread residual
  * reductions), FD_ATT_SPLIT=0|2 (never / always cut attention items along the keys),
  * FD_TC_MAX_CTAS=n (cap on persistent CTAs), FD_ATT_PAIR=1 (CTA-pair attention kernel at head dim 128), and, read at
- * every step, FD_TC_GROUPED=0 (dual stream: one launch per stream and projection instead of one grouped launch).
+ * every step, FD_TC_GROUPED=0 (dual stream: one launch per stream and projection instead of one grouped launch) and
+ * FD_QK_FUSED=0 (QK-RMSNorm / rotary embedding in a kernel of their own instead of the QKV projection's epilogue).
  */
 #ifndef FLASHDIFF_H_
 #define FLASHDIFF_H_

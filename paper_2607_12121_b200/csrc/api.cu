@@ -243,6 +243,23 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
             ep.q_head_pad = tc_attention_head_pad(cf.head_dim);
         }
         ep.kv = kv_b;
+        // block variants inside the projection's epilogue where the tile shapes allow it, else in a kernel behind it
+        const bool have_var = c->var.q_norm_w || c->var.rope_cos;
+        const bool qk_fused = have_var && c->use_tc && tc_plan_qk_fusable(c->tc);
+        auto norm_w = [&](const void* base) -> const T* {
+            return base ? static_cast<const T*>(base) + (size_t)blk * cf.head_dim : nullptr;
+        };
+        const bool text_norm = dual && c->var.q_norm_w_text != nullptr;
+        if (qk_fused) {
+            ep.qk_head_dim = cf.head_dim;
+            ep.qk_eps = c->var.qk_norm_eps;
+            ep.qn_w = norm_w(c->var.q_norm_w);
+            ep.kn_w = norm_w(c->var.k_norm_w);
+            ep.qn_w2 = text_norm ? norm_w(c->var.q_norm_w_text) : ep.qn_w;
+            ep.kn_w2 = text_norm ? norm_w(c->var.k_norm_w_text) : ep.kn_w;
+            ep.rope_cos = c->var.rope_cos;
+            ep.rope_sin = c->var.rope_sin;
+        }
         // (dual stream: one grouped launch where the CTA-pair kernel runs the projection, else one launch per stream)
         const bool grp_qkv = dual && c->use_tc && tc_plan_grouped(c->tc, TC_GEMM_QKV);
         if (grp_qkv) {
@@ -257,6 +274,7 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
         for (int pass = 0; pass < n_pass && !grp_qkv; ++pass) {
             ep.group = dual ? pass : -1;
             ep.bias = stream_ptr(c->w.b_qkv, c->text_w.b_qkv, (size_t)blk * 3 * H, pass);
+            if (qk_fused && pass == 1) { ep.qn_w = ep.qn_w2; ep.kn_w = ep.kn_w2; }
             if (f8) {
                 ep.col_scale = f8ops[pass]->s_qkv + (size_t)blk * 3 * H;
                 ep.act_scale = a8[pass][0];
@@ -267,13 +285,10 @@ fd_status run_step(fd_ctx* c, const void* x_, const void* cond_, const int32_t* 
                 FD_TRY(FD_PROF_GEMM_QKV, launch_simt_gemm<T>(EPI_QKV, act, H, stream_ptr(c->w.w_qkv, c->text_w.w_qkv, (size_t)blk * 3 * H * H, pass),
                                                              3 * H, H, rows_cap, ep, ctl, st, &nl));
         }
+        ep.qk_head_dim = 0;                          // (the cross-attention's query projection shares this epilogue)
         // block variants: QK-RMSNorm and rotary embedding on the fresh Q rows and the K rows just written
-        if (c->var.q_norm_w || c->var.rope_cos) {
+        if (have_var && !qk_fused) {
             const int q_stride = c->use_tc_attn ? tc_attention_head_pad(cf.head_dim) : cf.head_dim;
-            auto norm_w = [&](const void* base) -> const T* {
-                return base ? static_cast<const T*>(base) + (size_t)blk * cf.head_dim : nullptr;
-            };
-            const bool text_norm = dual && c->var.q_norm_w_text != nullptr;
             FD_TRY(FD_PROF_QK_VARIANTS, launch_qk_variants<T>(q, l.q_ld, q_stride, kv_b, active_idx, N, H, cf.n_heads, cf.head_dim,
                                                                norm_w(c->var.q_norm_w), norm_w(c->var.k_norm_w), c->var.qk_norm_eps,
                                                                c->var.rope_cos, c->var.rope_sin, rows_cap, ctl, st, &nl,

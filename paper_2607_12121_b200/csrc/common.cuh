@@ -100,7 +100,18 @@ struct EpiParams {
     const float* col_scale;    // [n_out] f32
     float act_scale;
     float out_inv_scale;
+    // EPI_QKV with the block variants fused (qk_head_dim != 0: 64 or 128, heads aligned with the epilogue's column
+    // chunks): per head slice of a query / key row, RMS normalisation with the channel weights qn_w / kn_w [head_dim]
+    // (nullptr: none) and rotation of the channel pairs by the row's angles rope_cos/sin [N, head_dim / 2] (nullptr: none)
+    int32_t qk_head_dim;
+    float qk_eps;
+    const void* qn_w;
+    const void* kn_w;
+    const float* rope_cos;
+    const float* rope_sin;
     // dual stream in one launch (the grouped form of the CTA-pair kernel): what the second stream's tiles use instead
+    const void* qn_w2;
+    const void* kn_w2;
     const void* bias2;
     const float* col_scale2;
     float act_scale2;

@@ -103,6 +103,7 @@ struct RowInfo {
     uint32_t valid;    // bit t: row t of the warp's 32 exists and belongs to the stream this launch finishes (same in all lanes)
     int gate_off;      // b * 6H: offset of the request's adaLN vectors (of the row's stream)
     uint32_t y_lo, y_hi;   // tok * H: element offset of the row in y (EPI_RESID) or of the token in the K plane (EPI_QKV)
+    int pos;           // EPI_QKV: the token's index inside its request (row of the rotary tables)
 };
 
 // EPI_RESID: 32 fp32 accumulator columns per row; resid += gate * (acc + bias); the last block also
@@ -248,9 +249,20 @@ __device__ __forceinline__ void epilogue_resid_chunk_tma(const EpiParams& ep, ui
 // EPI_QKV / EPI_GELU: 64 fp32 accumulator columns per row, bf16 outputs (8 columns per 16-byte unit).
 // F8: the accumulator holds products of 8-bit operands and is scaled by col_scale[col] * act_scale before the bias;
 // EPI_GELU then writes its 64 values per row as 64 E4M3 bytes of value * out_inv_scale (the fc2 operand).
+// QkVar: block variants fused into EPI_QKV for this chunk (all lanes alike): the lane's row is scaled by `rs` (its
+// head's 1 / rms) and the channel weights gamma[64] (this chunk's part of the head; nullptr: no normalisation), then
+// its channel pairs are rotated by the row's angles cs / sn [32] (this chunk's part; nullptr: no rotation).
+struct QkVar {
+    float rs;
+    const __nv_bfloat16* gamma;
+    const float* cs;
+    const float* sn;
+};
+
 template <int KIND, bool F8>
 __device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t* stage, int lane, int row_base,
-                                                    int col0, const uint32_t* acc, const RowInfo& ri) {
+                                                    int col0, const uint32_t* acc, const RowInfo& ri,
+                                                    const QkVar* var = nullptr) {
     using T = __nv_bfloat16;
     const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ep.bias) + col0);
     const float4* sp = reinterpret_cast<const float4*>(ep.col_scale + col0);
@@ -279,6 +291,30 @@ __device__ __forceinline__ void epilogue_bf16_chunk(const EpiParams& ep, uint8_t
         if constexpr (KIND == EPI_GELU) {
 #pragma unroll
             for (int k = 0; k < 8; ++k) v[k] = gelu_tanh_fast(v[k]);
+        }
+        if constexpr (KIND == EPI_QKV) {
+            if (var) {
+                if (var->gamma) {
+                    const uint4 g = __ldg(reinterpret_cast<const uint4*>(var->gamma) + u);
+                    const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        v[2 * k] *= var->rs * __uint_as_float(gw[k] << 16);
+                        v[2 * k + 1] *= var->rs * __uint_as_float(gw[k] & 0xffff0000u);
+                    }
+                }
+                if (var->cs) {
+                    const float4 c4 = __ldg(reinterpret_cast<const float4*>(var->cs) + u);
+                    const float4 s4 = __ldg(reinterpret_cast<const float4*>(var->sn) + u);
+                    const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float a = v[2 * k], b = v[2 * k + 1];
+                        v[2 * k] = a * cc[k] - b * ss[k];
+                        v[2 * k + 1] = a * ss[k] + b * cc[k];
+                    }
+                }
+            }
         }
         if constexpr (KIND == EPI_GELU && F8) {
             const float qs = ep.out_inv_scale;
@@ -357,7 +393,7 @@ __device__ __forceinline__ void epilogue_prefetch_resid(const EpiParams& ep, int
 // fetch it while the tile's products are still running.
 template <int KIND>
 __device__ __forceinline__ RowInfo epilogue_row_info(const EpiParams& ep, int lane, int row_base, int a_total) {
-    RowInfo ri{0u, 0, 0u, 0u};
+    RowInfo ri{0u, 0, 0u, 0u, 0};
     bool ok = row_base + lane < a_total;
     if ((KIND != EPI_GELU || ep.group >= 0) && ok) {
         const int tok = ep.active_idx[row_base + lane];
@@ -371,6 +407,7 @@ __device__ __forceinline__ RowInfo epilogue_row_info(const EpiParams& ep, int la
         const size_t off = KIND == EPI_RESID ? (size_t)tok * ep.H : ((size_t)b * 2 * ep.N + (tok - b * ep.N)) * ep.H;
         ri.y_lo = (uint32_t)off;
         ri.y_hi = (uint32_t)(off >> 32);
+        ri.pos = tok - b * ep.N;
     }
     ri.valid = __ballot_sync(0xffffffffu, ok);
     return ri;
@@ -395,6 +432,66 @@ __device__ __forceinline__ void epilogue_warp(const EpiParams& ep, uint8_t* stag
             }
         }
     } else {
+        if constexpr (KIND == EPI_QKV) {
+            if (ep.qk_head_dim) {
+                // Block variants fused: one head (of Q, K or V) at a time.  The head's sum of squares needs all of its
+                // columns, which are one or two chunks of the accumulator: a first pass over them only sums, the
+                // second one normalises, rotates and stores (the accumulator is read twice; it sits in TMEM).
+                using T = __nv_bfloat16;
+                const int dh = ep.qk_head_dim;
+#pragma unroll 1
+                for (int h0 = c_begin; h0 < c_end; h0 += dh) {
+                    const int col_h = tile_col0 + h0;
+                    const int sec = col_h / ep.H;                        // 0: queries, 1: keys, 2: values
+                    const T* gamma = sec == 0 ? static_cast<const T*>(ep.qn_w) : sec == 1 ? static_cast<const T*>(ep.kn_w) : nullptr;
+                    const bool rot = sec < 2 && ep.rope_cos != nullptr;
+                    QkVar var{1.f, nullptr, nullptr, nullptr};
+                    if (gamma) {
+                        float ssq = 0.f;
+#pragma unroll 1
+                        for (int c0 = h0; c0 < h0 + dh; c0 += 64) {
+                            uint32_t r[64];
+                            ptx::tmem_ld32(t_row + c0, r);
+                            ptx::tmem_ld32(t_row + c0 + 32, r + 32);
+                            ptx::tmem_wait_ld();
+                            const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ep.bias) + tile_col0 + c0);
+                            const float4* sp = reinterpret_cast<const float4*>(ep.col_scale + tile_col0 + c0);
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const uint4 b = __ldg(bp + u);
+                                const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+                                float sc[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
+                                if constexpr (F8) {
+                                    const float4 s0 = __ldg(sp + 2 * u), s1 = __ldg(sp + 2 * u + 1);
+                                    sc[0] = s0.x * ep.act_scale; sc[1] = s0.y * ep.act_scale; sc[2] = s0.z * ep.act_scale; sc[3] = s0.w * ep.act_scale;
+                                    sc[4] = s1.x * ep.act_scale; sc[5] = s1.y * ep.act_scale; sc[6] = s1.z * ep.act_scale; sc[7] = s1.w * ep.act_scale;
+                                }
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    const float a = fmaf(__uint_as_float(r[8 * u + 2 * k]), sc[2 * k], __uint_as_float(w[k] << 16));
+                                    const float bb = fmaf(__uint_as_float(r[8 * u + 2 * k + 1]), sc[2 * k + 1], __uint_as_float(w[k] & 0xffff0000u));
+                                    ssq = fmaf(a, a, ssq);
+                                    ssq = fmaf(bb, bb, ssq);
+                                }
+                            }
+                        }
+                        var.rs = rsqrtf(ssq / (float)dh + ep.qk_eps);
+                    }
+#pragma unroll 1
+                    for (int c0 = h0; c0 < h0 + dh; c0 += 64) {
+                        uint32_t r[64];
+                        ptx::tmem_ld32(t_row + c0, r);
+                        ptx::tmem_ld32(t_row + c0 + 32, r + 32);
+                        ptx::tmem_wait_ld();
+                        var.gamma = gamma ? gamma + (c0 - h0) : nullptr;
+                        var.cs = rot ? ep.rope_cos + (size_t)ri.pos * (dh >> 1) + ((c0 - h0) >> 1) : nullptr;
+                        var.sn = rot ? ep.rope_sin + (size_t)ri.pos * (dh >> 1) + ((c0 - h0) >> 1) : nullptr;
+                        if (live) epilogue_bf16_chunk<KIND, F8>(ep, stage, lane, row_base, tile_col0 + c0, r, ri, (gamma || rot) ? &var : nullptr);
+                    }
+                }
+                return;
+            }
+        }
 #pragma unroll 1
         for (int c0 = c_begin; c0 < c_end; c0 += 64) {
             uint32_t r[64];

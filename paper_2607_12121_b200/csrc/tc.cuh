@@ -42,6 +42,7 @@ cudaError_t tc_gemm_fp8(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep
                         int* n_launch, bool text_pass = false);
 // dual stream in one launch (the grouped form of the CTA-pair kernel): true where it can run this projection
 bool tc_plan_grouped(TcPlan* p, TcGemmKind kind);
+bool tc_plan_qk_fusable(TcPlan* p);          // the QKV epilogue applies QK-RMSNorm / rotary embedding itself
 cudaError_t tc_gemm_both(TcPlan* p, TcGemmKind kind, int blk, const EpiParams& ep, const Control* ctl, cudaStream_t st,
                          int* n_launch, bool fp8);
 // cross-attention: tensor maps of its two [L, H, H] projection weights (both nullptr: off)

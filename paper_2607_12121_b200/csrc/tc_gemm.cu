@@ -304,6 +304,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         uint32_t t_it = 0;
         bool ok = true;
         const void* bias0 = ep.bias;
+        const void* qn0 = ep.qn_w;
+        const void* kn0 = ep.kn_w;
         const float* col_scale0 = ep.col_scale;
         const float act_scale0 = ep.act_scale, out_inv_scale0 = ep.out_inv_scale;
         for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++t_it) {
@@ -312,6 +314,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             if constexpr (GROUPED) {                        // this tile's stream: its rows, bias and scales
                 ep.group = grp;
                 ep.bias = grp ? ep.bias2 : bias0;
+                ep.qn_w = grp ? ep.qn_w2 : qn0;
+                ep.kn_w = grp ? ep.kn_w2 : kn0;
                 ep.col_scale = grp ? ep.col_scale2 : col_scale0;
                 ep.act_scale = grp ? ep.act_scale2 : act_scale0;
                 ep.out_inv_scale = grp ? ep.out_inv_scale2 : out_inv_scale0;
@@ -689,6 +693,16 @@ bool tc_plan_set_fp8(TcPlan* p, const void* w8_qkv, const void* w8_fc1, const vo
 // second stream with the second stream's weights (ep.bias2 and, with FP8 operands, ep.col_scale2 / act_scale2 /
 // out_inv_scale2 are that stream's).  Available where the CTA-pair kernel runs the projection (switch FD_TC_GROUPED=0
 // keeps the two launches).
+// The QKV epilogue can apply QK-RMSNorm and the rotary embedding itself when every head is a whole number of its
+// 64-column chunks inside one warp's column range: head dim 64 at either tile width, head dim 128 at 256-wide tiles
+// (switch FD_QK_FUSED=0 keeps the separate kernel).
+bool tc_plan_qk_fusable(TcPlan* p) {
+    const char* v = getenv("FD_QK_FUSED");
+    if (v && atoi(v) == 0) return false;
+    const int bn = p->spec[TC_GEMM_QKV].pair_bn, dh = p->cfg.head_dim;
+    return bn != 0 && (dh == 64 || (dh == 128 && bn == 256));
+}
+
 bool tc_plan_grouped(TcPlan* p, TcGemmKind kind) {
     const char* v = getenv("FD_TC_GROUPED");
     const bool on = !v || atoi(v) != 0;

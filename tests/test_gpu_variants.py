@@ -36,6 +36,15 @@ def test_variants_match_the_oracle(name, engine, which):
     _run_sequence(wl, 2, engine, masks, qk_gain=4.0, variants=var)
 
 
+@pytest.mark.parametrize("name", ["audio_tc", "wide_tc", "mmdit_tc"])
+def test_variants_in_their_own_kernel_behind_the_projection(monkeypatch, name):
+    """Head dims 64 and 128 normally get the variants inside the QKV epilogue; the separate kernel (what head dim 72 and
+    the CUDA-core engine use) on the same shapes."""
+    monkeypatch.setenv("FD_QK_FUSED", "0")
+    wl = gen.workload(name)
+    _run_sequence(wl, 7, fd.FD_ENGINE_TC, _masks(wl), qk_gain=4.0, variants=gen.block_variants(wl, 9))
+
+
 def test_variants_can_be_switched_off_again_and_bad_arguments_are_refused():
     wl = gen.workload("audio_tc")
     w = gen.block_weights(wl, 2)
