@@ -129,6 +129,11 @@ def _run_sequence(wl, seed, engine, masks, n_blocks=None, qk_gain=1.0, variants=
             widen = (0.6 * max_abs(ya, yp), 0.6 * rel_l2(yp, ya))
             sel = act.reshape(B, N)[:, None].repeat(2, 1)                    # [B, 2, N]: the fresh K and V rows
             widen_kv = (0.6 * max_abs(kv_ref[:, sel], kv_p[:, sel]), 0.6 * rel_l2(kv_p[:, sel], kv_ref[:, sel]))
+        if variants and "q_norm_w" in variants and wl.dtype == "bf16":
+            # Normalised keys are of order one with tails of 4-5: storing such a value in bf16 costs up to |k| 2^-9,
+            # and where the variants run in a kernel of their own behind the projection the key is rounded twice
+            # (before and after the normalisation), so the absolute bound carries 2 |k| 2^-9 of the largest stored key.
+            widen_kv = (widen_kv[0] + float(np.abs(kv_ref).max()) * 2.0 ** -8, widen_kv[1])
         _check_step(wl, host(buf.y), host(buf.kv), y_ref, kv_ref, y_before, kv_before, idx, widen, widen_kv)
     return ctx
 
