@@ -451,7 +451,7 @@ class Engine:
                                      "frac_burst": round(t["frac_burst"] / 2, 3), "frac_sustained": round(t["frac_sustained"] / 2, 3)}
         return out
 
-    def variants_measure(self, steps, ms_plain, fraction=None):
+    def variants_measure(self, steps, fraction=None):
         """The same gated step with the block variants of the paper's models switched on, one at a time: QK-RMSNorm +
         rotary embedding, cross-attention to a 512-token context, and (workloads with text tokens) a second weight set
         for the always-active tokens.  Step time and the cost against the plain step on the same active set."""
@@ -467,36 +467,43 @@ class Engine:
             return t.to(self.dt if dt is None else dt).contiguous()
 
         def timed_step():
-            for _ in range(3):
+            for _ in range(2):
                 self.gated_step()
             return self.timed(self.gated_step, steps)
 
+        def compare(switch_on, switch_off):
+            """Plain and variant step alternately, three times each; medians (under the power cap the clock drifts over
+            seconds, which would bias whichever form ran second)."""
+            tp, tv = [], []
+            for _ in range(3):
+                switch_off()
+                tp.append(timed_step())
+                switch_on()
+                tv.append(timed_step())
+            switch_off()
+            p_ms, v_ms = float(np.median(tp)), float(np.median(tv))
+            return {"plain_step_ms": round(p_ms, 4), "step_ms": round(v_ms, 4), "extra": round(v_ms / p_ms - 1.0, 4)}
+
         out = {}
-        ms_plain = timed_step()                           # measured again here: the clock drifts over a long run
-        out["plain_step_ms"] = round(ms_plain, 4)
         try:
             half = wl.head_dim // 2
             ang = torch.arange(N, device=dev, dtype=torch.float32)[:, None] * \
                 (10000.0 ** (-torch.arange(half, device=dev, dtype=torch.float32) / half))[None, :]
-            fd.fd_set_block_variants(self.ctx, q_norm_w=draw((L, wl.head_dim), 0.1, 1.0), k_norm_w=draw((L, wl.head_dim), 0.1, 1.0),
-                                     rope_cos=torch.cos(ang).contiguous(), rope_sin=torch.sin(ang).contiguous())
-            ms = timed_step()
-            fd.fd_set_block_variants(self.ctx)
-            out["qk_norm_rope"] = {"step_ms": round(ms, 4), "extra": round(ms / ms_plain - 1.0, 4)}
+            qk = dict(q_norm_w=draw((L, wl.head_dim), 0.1, 1.0), k_norm_w=draw((L, wl.head_dim), 0.1, 1.0),
+                      rope_cos=torch.cos(ang).contiguous(), rope_sin=torch.sin(ang).contiguous())
+            out["qk_norm_rope"] = compare(lambda: fd.fd_set_block_variants(self.ctx, **qk), lambda: fd.fd_set_block_variants(self.ctx))
             T = 512
-            fd.fd_set_cross_attention(self.ctx, {"w_q": draw((L, H, H), 0.02), "b_q": draw((L, H), 0.02), "w_o": draw((L, H, H), 0.02),
-                                                 "b_o": draw((L, H), 0.02), "ctx_kv": draw((L, B, 2, T, H), 0.5)})
-            ms = timed_step()
-            fd.fd_set_cross_attention(self.ctx, None)
-            extra_flops = L * (4.0 * H * H + 4.0 * T * H)            # per active row: two projections + the attention
-            out["cross_attention"] = {"context_tokens": T, "step_ms": round(ms, 4), "extra": round(ms / ms_plain - 1.0, 4),
-                                      "extra_flops_per_active_row": extra_flops}
+            cross = {"w_q": draw((L, H, H), 0.02), "b_q": draw((L, H), 0.02), "w_o": draw((L, H, H), 0.02),
+                     "b_o": draw((L, H), 0.02), "ctx_kv": draw((L, B, 2, T, H), 0.5)}
+            out["cross_attention"] = dict(compare(lambda: fd.fd_set_cross_attention(self.ctx, cross),
+                                                  lambda: fd.fd_set_cross_attention(self.ctx, None)),
+                                          context_tokens=T, extra_flops_per_active_row=L * (4.0 * H * H + 4.0 * T * H))
+            del cross
             if wl.n_text > 0:
-                fd.fd_set_text_stream(self.ctx, device_weights(wl, self.seed + 29, dev))
-                ms = timed_step()
-                fd.fd_set_text_stream(self.ctx, None)
-                out["dual_stream"] = {"text_tokens_per_request": wl.n_text, "step_ms": round(ms, 4),
-                                      "extra": round(ms / ms_plain - 1.0, 4)}
+                wt = device_weights(wl, self.seed + 29, dev)
+                out["dual_stream"] = dict(compare(lambda: fd.fd_set_text_stream(self.ctx, wt), lambda: fd.fd_set_text_stream(self.ctx, None)),
+                                          text_tokens_per_request=wl.n_text)
+                del wt
         except fd.FlashDiffError as e:
             out["unavailable"] = str(e)
         self.dense_step(self.x_prev)                      # the cached state as the plain step left it
@@ -521,7 +528,7 @@ def side_workload(name, seed, dev, rep, steps, warmup, peaks):
     if sweep:
         res["sweep"] = sweep
     res["fp8_operands"] = eng.fp8_measure(steps, peaks, res["step_ms"])
-    res["variants"] = eng.variants_measure(max(5, steps // 2), res["step_ms"])
+    res["variants"] = eng.variants_measure(max(4, steps // 4))
     eng.close()
     del eng
     torch.cuda.empty_cache()
@@ -731,7 +738,7 @@ def run_ours(args):
     fp8 = variants = None
     if world == 1 and not args.no_extras:
         fp8 = eng.fp8_measure(max(5, args.steps // 2), peaks, ms_reg, args.fraction)
-        variants = eng.variants_measure(max(5, args.steps // 2), ms_reg, args.fraction)
+        variants = eng.variants_measure(max(4, args.steps // 4), args.fraction)
     st_destroy = eng.close()
     del eng, x, cond, y, z_cur, z_prev, eps
     torch.cuda.empty_cache()
