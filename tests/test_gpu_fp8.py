@@ -170,3 +170,27 @@ def test_fp8_argument_checks_and_switch_off(monkeypatch):
     with pytest.raises(fd.FlashDiffError) as ei:
         fd.fd_set_fp8_operands(ctx, args)
     assert ei.value.status == fd.FD_ERR_UNSUPPORTED
+
+
+def test_empty_mask_with_fp8_operands_and_variants_touches_nothing():
+    """No active row at all (device-side row count zero): every kernel of the step, the 8-bit projections and the
+    fused variants included, finds nothing to do and leaves y and the cache as they were."""
+    wl = gen.workload("audio_tc")
+    labels = gen.uniform_labels(wl)
+    w = gen.block_weights(wl, 8)
+    inp = gen.step_inputs(wl, 8, labels)
+    ctx = make_ctx(wl, w, engine=fd.FD_ENGINE_TC)
+    f8 = gen.fp8_operands(wl, w, 8)
+    fd.fd_set_fp8_operands(ctx, dict({"w8_" + k: dev(f8["c_" + k]) for k in ("qkv", "fc1", "fc2")},
+                                     **{"s_" + k: dev(f8["s_" + k]) for k in ("qkv", "fc1", "fc2")}, a_scale=f8["a_scale"]))
+    var = gen.block_variants(wl, 9)
+    fd.fd_set_block_variants(ctx, **{k: (dev(v, torch.bfloat16 if k.endswith("_w") else None) if isinstance(v, np.ndarray) else v)
+                                     for k, v in var.items()})
+    buf = StepBuffers(wl, wl.L)
+    buf.y.fill_(1.5)
+    buf.kv.fill_(-2.0)
+    idx, cu = gpu_step(ctx, wl, dev(inp["x_cur"], torch.bfloat16), dev(inp["cond"], torch.bfloat16), dev(labels),
+                       dev(np.zeros((wl.B, wl.R), np.uint8)), buf)
+    assert idx.size == 0 and not cu.any()
+    assert (host(buf.y) == 1.5).all() and (host(buf.kv) == -2.0).all()
+    assert fd.fd_destroy(ctx) == fd.FD_OK
