@@ -37,6 +37,12 @@ def test_dual_stream_row_tile_lists(n_text, B):
     _run_sequence(wl, 3, fd.FD_ENGINE_TC, masks, text_seed=78)
 
 
+def test_dual_stream_grouped_launch_with_few_ctas(monkeypatch):
+    monkeypatch.setenv("FD_TC_MAX_CTAS", "4")                  # two CTA pairs walk every tile of both groups in turn
+    wl = gen.workload("mmdit_tc").replace(n_text=300, B=3)
+    _run_sequence(wl, 8, fd.FD_ENGINE_TC, _masks(wl), variants=gen.block_variants(wl, 9), text_seed=83)
+
+
 def test_dual_stream_as_two_launches_per_projection(monkeypatch):
     monkeypatch.setenv("FD_TC_GROUPED", "0")                   # not the grouped launch: one launch per stream
     wl = gen.workload("mmdit_tc")
