@@ -4,11 +4,13 @@
 // One work item = one query tile (up to 128 compact rows of one request) x one head.  Persistent,
 // warp-specialised CTAs of four warpgroups walk the device-built work list:
 //   warp 0       TMA producer: Q tile (double buffered across items), K and V tiles (128 keys) in rings
-//   warp 1       issues S = Q K^T (tcgen05.mma, both operands in shared memory) into one of two TMEM
-//                score buffers as soon as the softmax has handed that buffer back
+//   warp 1       issues S = Q K^T (tcgen05.mma, both operands in shared memory) into the TMEM score buffer
+//                as soon as the softmax has handed it back (one buffer; the older mass layouts below use two)
 //   warp 2       issues O += P V with P read from TMEM and V as an N-major shared-memory operand
-//   warps 4..11  softmax: tcgen05.ld of the scores, running maximum with lazy rescaling of O (only
-//                when it grew by more than 2^24), exp2, P written to TMEM as packed bf16
+//   warps 4..11  softmax: tcgen05.ld of the scores, a reference maximum per row with lazy rescaling of O (a
+//                tile's own maximum is computed only for a warpgroup's first tile of an item and when a
+//                tile's row sum shows a score more than 2^24 above the reference), exp2, P written to TMEM
+//                as packed bf16
 //   warps 12..15 item epilogue (merge, normalise, store) while the softmax warps go on
 // Warpgroup p takes the key tiles of parity p with its own P buffer,
 // accumulator O_p and running maximum / row sum: one thread per row copies the tile's 128 scores to
